@@ -1,0 +1,148 @@
+"""CPU oracle for HiLS attention -- TEST INFRASTRUCTURE, not product code.
+
+Thin ctypes wrapper around ``hils_oracle.c`` (plain C, fp64).  Only the tests,
+the smoke check and the benchmark's CPU-baseline leg may import this package;
+the CUDA library and its Python binding never do, and this package imports
+nothing from them.
+
+Parity status: the paper prints no numeric example, so every function here is
+pinned by identities (see tests/test_oracle_pins.py); absolute agreement with
+the authors' own implementation is unpinned.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "hils_oracle.c")
+_SO = os.path.join(_HERE, "libhils_oracle.so")
+_lib = None
+
+
+class _Params(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int), ("Hq", ctypes.c_int), ("Hkv", ctypes.c_int), ("Hl", ctypes.c_int),
+                ("Lq", ctypes.c_int), ("T", ctypes.c_int), ("C", ctypes.c_int),
+                ("d", ctypes.c_int), ("S", ctypes.c_int), ("K", ctypes.c_int), ("W", ctypes.c_int),
+                ("scale", ctypes.c_double), ("group_mode", ctypes.c_int)]
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (OpenMP) if the shared object is missing or stale."""
+    if (not force and os.path.exists(_SO) and os.path.getmtime(_SO) >= os.path.getmtime(_SRC)):
+        return _SO
+    tmp = _SO + ".tmp%d" % os.getpid()
+    cmd = ["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-std=c11", "-o", tmp, _SRC, "-lm"]
+    subprocess.run(cmd, check=True)
+    os.replace(tmp, _SO)
+    return _SO
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        _lib = ctypes.CDLL(_SO)
+        _lib.hils_oracle_rows.restype = ctypes.c_int
+        _lib.hils_oracle_num_threads.restype = ctypes.c_int
+    return _lib
+
+
+def num_threads() -> int:
+    return int(_load().hils_oracle_num_threads())
+
+
+def _f32(a) -> np.ndarray:
+    """fp32 C-contiguous numpy view/copy of a numpy array or a CPU torch tensor (bf16 widens exactly)."""
+    if hasattr(a, "detach"):
+        a = a.detach().to("cpu").float().contiguous().numpy()
+    return np.ascontiguousarray(a, dtype=np.float32)
+
+
+def _ptr(a: Optional[np.ndarray], ct):
+    return None if a is None else a.ctypes.data_as(ctypes.POINTER(ct))
+
+
+def hils_rows(q, k, v, landmarks, bias, *, S: int, K: int, W: int = 1, scale: float = 0.0,
+              row_b, row_qi, row_pos, sel_idx=None, attend: bool = True, group_mode: int = 0,
+              want_alpha: bool = False):
+    """Run the oracle on a list of query rows.
+
+    q [B,Hq,Lq,d]; k,v [B,Hkv,T,d]; landmarks [B,Hl,C,d]; bias [B,Hl,C] or None.
+    Row r is q[row_b[r], :, row_qi[r], :] at sequence position row_pos[r].
+    If ``sel_idx`` ([n,Hkv,K] int32, ascending, -1 padded) is given it is used as the
+    selection instead of computing one.
+    Returns dict(sel_idx, margin, out, lse[, alpha]) as numpy arrays indexed by row.
+    """
+    lib = _load()
+    q = _f32(q); k = _f32(k); v = _f32(v); landmarks = _f32(landmarks)
+    bias_a = None if bias is None else _f32(bias)
+    B, Hq, Lq, d = q.shape
+    _, Hkv, T, _ = k.shape
+    _, Hl, C, _ = landmarks.shape
+    row_b = np.ascontiguousarray(row_b, dtype=np.int32)
+    row_qi = np.ascontiguousarray(row_qi, dtype=np.int32)
+    row_pos = np.ascontiguousarray(row_pos, dtype=np.int64)
+    n = row_b.shape[0]
+    p = _Params(B, Hq, Hkv, Hl, Lq, T, C, d, S, K, W, float(scale), group_mode)
+    sel_mode = 0
+    if sel_idx is None:
+        sel = np.full((n, Hkv, K), -1, dtype=np.int32)
+    else:
+        sel = np.ascontiguousarray(sel_idx, dtype=np.int32).reshape(n, Hkv, K).copy()
+        sel_mode = 1
+    margin = np.full((n, Hkv), np.inf, dtype=np.float64)
+    out = np.zeros((n, Hq, d), dtype=np.float64) if attend else None
+    lse = np.zeros((n, Hq), dtype=np.float64) if attend else None
+    alpha = np.zeros((n, Hq, K + 1), dtype=np.float64) if (attend and want_alpha) else None
+    rc = lib.hils_oracle_rows(
+        ctypes.byref(p), _ptr(q, ctypes.c_float), _ptr(k, ctypes.c_float), _ptr(v, ctypes.c_float),
+        _ptr(landmarks, ctypes.c_float), _ptr(bias_a, ctypes.c_float),
+        ctypes.c_int64(n), _ptr(row_b, ctypes.c_int32), _ptr(row_qi, ctypes.c_int32),
+        _ptr(row_pos, ctypes.c_int64), ctypes.c_int(sel_mode), ctypes.c_int(1 if attend else 0),
+        _ptr(sel, ctypes.c_int32), _ptr(margin, ctypes.c_double),
+        _ptr(out, ctypes.c_double), _ptr(lse, ctypes.c_double), _ptr(alpha, ctypes.c_double))
+    if rc != 0:
+        raise ValueError("hils_oracle_rows rejected its arguments (rc=%d)" % rc)
+    res = {"sel_idx": sel, "margin": margin, "out": out, "lse": lse}
+    if alpha is not None:
+        res["alpha"] = alpha
+    return res
+
+
+def hils_prefill(q, k, v, landmarks, bias=None, *, S: int, K: int, W: int = 1, scale: float = 0.0,
+                 rows=None, sel_idx=None, group_mode: int = 0, want_alpha: bool = False):
+    """Prefill oracle: every position (or the positions in ``rows``) of every sequence.
+
+    Returns arrays shaped [B, n_rows, ...]: sel_idx [B,n,Hkv,K], margin [B,n,Hkv],
+    out [B,n,Hq,d], lse [B,n,Hq].
+    """
+    B, L = q.shape[0], q.shape[2]
+    rows = np.arange(L, dtype=np.int64) if rows is None else np.asarray(rows, dtype=np.int64)
+    n = rows.shape[0]
+    row_b = np.repeat(np.arange(B, dtype=np.int32), n)
+    row_pos = np.tile(rows, B)
+    if sel_idx is not None:
+        sel_idx = np.asarray(sel_idx).reshape(B * n, -1, K)
+    res = hils_rows(q, k, v, landmarks, bias, S=S, K=K, W=W, scale=scale, row_b=row_b,
+                    row_qi=row_pos.astype(np.int32), row_pos=row_pos, sel_idx=sel_idx,
+                    group_mode=group_mode, want_alpha=want_alpha)
+    return {key: val.reshape((B, n) + val.shape[1:]) for key, val in res.items() if val is not None}
+
+
+def hils_decode(q, k_cache, v_cache, landmarks, bias, seq_lens, *, S: int, K: int, W: int = 1,
+                scale: float = 0.0, sel_idx=None, group_mode: int = 0, want_alpha: bool = False):
+    """Decode oracle: one query per sequence at position seq_lens[b]-1 (its own k,v are in the cache).
+
+    q [B,Hq,d].  Returns sel_idx [B,Hkv,K], margin [B,Hkv], out [B,Hq,d], lse [B,Hq].
+    """
+    qn = _f32(q)
+    B, Hq, d = qn.shape
+    seq = np.asarray(seq_lens.cpu() if hasattr(seq_lens, "cpu") else seq_lens, dtype=np.int64)
+    return hils_rows(qn.reshape(B, Hq, 1, d), k_cache, v_cache, landmarks, bias, S=S, K=K, W=W,
+                     scale=scale, row_b=np.arange(B, dtype=np.int32), row_qi=np.zeros(B, dtype=np.int32),
+                     row_pos=seq - 1, sel_idx=sel_idx, group_mode=group_mode, want_alpha=want_alpha)

@@ -1,0 +1,257 @@
+/*
+ * HiLS attention -- CPU oracle.  TEST INFRASTRUCTURE, NOT PRODUCT CODE.
+ *
+ * A plain, slow, double-precision restatement of the forward HiLS attention
+ * operator, written from the paper's equations.  It shares no code with the
+ * CUDA library and must never be linked, imported or called by it; only the
+ * tests, the smoke check and the benchmark's CPU-baseline leg use it.
+ *
+ * What it computes, for a query at position i of sequence b (0-based positions
+ * and chunk ids), for every KV group g and every query head h of that group:
+ *
+ *   Sec. 2.1      chunk of token j: c(j) = floor(j / S);
+ *                 aligned left edge of the local window
+ *                 l(i) = floor((i - W + 1) / S) * S  (floor toward -inf, clamped at 0);
+ *                 candidate chunks C_i = {0, ..., l(i)/S - 1}.
+ *   Eq. (surrogate top-k), App. C Eq. (HiLS GQA)
+ *                 per-head surrogate score  s^h_c = scale * q^h . k'_c + b'_c,
+ *                 group score u_c = max_h s^h_c, selected set I = the min(K, |C_i|)
+ *                 candidates with the largest u_c (full stable sort; equal scores
+ *                 go to the lower chunk id).
+ *   Eq. (chunk mass)  local branch: logits scale * q^h . k_j for j in [l(i), i],
+ *                 their log-sum-exp lambda_loc = log Z_swa and softmax output o_loc.
+ *   Eq. (HiLS weights), App. C
+ *                 every selected chunk gets its own softmax over its S tokens
+ *                 (output o_c); chunks and the local branch are mixed with
+ *                 alpha = softmax({s^h_c : c in I} U {lambda_loc}), using the
+ *                 PER-HEAD surrogate score of each selected chunk:
+ *                   out = alpha_loc * o_loc + sum_c alpha_c * o_c
+ *                   lse = log( sum_c exp(s^h_c) + Z_swa ).
+ *
+ * No blocking, fusion or reordering beyond the steps above.  Inputs are fp32
+ * arrays (bf16 data is widened exactly by the caller); all arithmetic is fp64
+ * with libm exp/log.
+ *
+ * Pinned by tests/test_oracle_pins.py (closed forms, invariants, library
+ * attention on reductions, an independent dense-weight brute force).  The paper
+ * prints no worked numeric example, so absolute values against the authors'
+ * own implementation are unpinned; the semantics are pinned by those identities.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+typedef struct {
+    int B, Hq, Hkv, Hl;   /* Hl in {Hkv, Hq}: number of landmark heads                */
+    int Lq;               /* query rows stored per (b, head) in q                       */
+    int T;                /* key/value tokens stored per (b, kv head)                   */
+    int C;                /* landmark rows stored per (b, landmark head)                */
+    int d, S, K, W;
+    double scale;         /* <= 0 means 1/sqrt(d)                                       */
+    int group_mode;       /* 0: u_c = max_h s^h_c (App. C); 1: max_h of softmax_c(s^h)  */
+} hils_oracle_params;
+
+static long floordiv(long a, long b) {
+    long q = a / b;
+    if ((a % b != 0) && ((a < 0) != (b < 0))) q -= 1;
+    return q;
+}
+
+static double dotf(const float *a, const float *b, int n) {
+    double acc = 0.0;
+    for (int t = 0; t < n; ++t) acc += (double)a[t] * (double)b[t];
+    return acc;
+}
+
+typedef struct { double u; int c; } cand_t;
+
+/* order: larger score first; equal scores -> lower chunk id first */
+static int cand_cmp(const void *pa, const void *pb) {
+    const cand_t *a = (const cand_t *)pa, *b = (const cand_t *)pb;
+    if (a->u > b->u) return -1;
+    if (a->u < b->u) return 1;
+    return (a->c > b->c) - (a->c < b->c);
+}
+
+static int int_cmp(const void *pa, const void *pb) {
+    int a = *(const int *)pa, b = *(const int *)pb;
+    return (a > b) - (a < b);
+}
+
+/* softmax attention of one query over rows [lo, hi) of K/V; returns m + log Z, writes o[d] */
+static double attend_span(const float *q, const float *k, const float *v, long lo, long hi,
+                          int d, double scale, double *o, double *logits) {
+    long n = hi - lo;
+    double m = -INFINITY;
+    for (long j = 0; j < n; ++j) {
+        logits[j] = scale * dotf(q, k + (lo + j) * d, d);
+        if (logits[j] > m) m = logits[j];
+    }
+    double Z = 0.0;
+    for (int t = 0; t < d; ++t) o[t] = 0.0;
+    for (long j = 0; j < n; ++j) {
+        double p = exp(logits[j] - m);
+        Z += p;
+        const float *vr = v + (lo + j) * d;
+        for (int t = 0; t < d; ++t) o[t] += p * (double)vr[t];
+    }
+    for (int t = 0; t < d; ++t) o[t] /= Z;
+    return m + log(Z);
+}
+
+/*
+ * Rows: row r is the query of sequence row_b[r], stored at q[row_b, :, row_qi[r], :],
+ * sitting at sequence position row_pos[r].
+ *
+ * sel_mode 0: compute the selection (Eq. surrogate top-k) and write it to sel_idx/margin.
+ * sel_mode 1: take sel_idx as given (ascending ids, -1 padded) and only attend.
+ * do_attend 0: selection only (out/lse untouched).
+ *
+ * Outputs (any may be NULL): sel_idx [n_rows, Hkv, K] int32 ascending, -1 padded;
+ * margin [n_rows, Hkv] = (K-th best group score) - ((K+1)-th best), +inf if none is cut;
+ * out [n_rows, Hq, d]; lse [n_rows, Hq]; alpha [n_rows, Hq, K+1] (selected slots, then local).
+ * Returns 0, or -1 on bad arguments.
+ */
+int hils_oracle_rows(const hils_oracle_params *p,
+                     const float *q, const float *k, const float *v,
+                     const float *landmarks, const float *bias,
+                     int64_t n_rows, const int32_t *row_b, const int32_t *row_qi,
+                     const int64_t *row_pos,
+                     int sel_mode, int do_attend,
+                     int32_t *sel_idx, double *margin,
+                     double *out, double *lse, double *alpha)
+{
+    if (!p || p->Hq % p->Hkv != 0 || (p->Hl != p->Hkv && p->Hl != p->Hq) || p->S <= 0 ||
+        p->K < 0 || p->W < 1 || !sel_idx)
+        return -1;
+    const int G = p->Hq / p->Hkv, d = p->d, S = p->S, K = p->K;
+    const double scale = p->scale > 0 ? p->scale : 1.0 / sqrt((double)d);
+    const int64_t work = n_rows * p->Hkv;
+    int status = 0;
+
+#pragma omp parallel for schedule(dynamic, 4)
+    for (int64_t w = 0; w < work; ++w) {
+        const int64_t r = w / p->Hkv;
+        const int g = (int)(w % p->Hkv);
+        const int b = row_b[r];
+        const long i = (long)row_pos[r];
+        long lo = floordiv(i - p->W + 1, S) * S;             /* l(i), Sec. 2.1 */
+        if (lo < 0) lo = 0;
+        const int ncand = (int)(lo / S);                     /* |C_i| */
+        if (i >= p->T || ncand > p->C) { status = -1; continue; }
+
+        double *shat = (double *)malloc(sizeof(double) * (size_t)(G * (ncand > 0 ? ncand : 1)));
+        cand_t *cand = (cand_t *)malloc(sizeof(cand_t) * (size_t)(ncand > 0 ? ncand : 1));
+        double *logits = (double *)malloc(sizeof(double) * (size_t)((i - lo + 1) > S ? (i - lo + 1) : S));
+        double *o_part = (double *)malloc(sizeof(double) * (size_t)d);
+        double *lam = (double *)malloc(sizeof(double) * (size_t)(K + 1));
+        double *o_all = (double *)malloc(sizeof(double) * (size_t)(K + 1) * (size_t)d);
+
+        /* per-head surrogate scores s^h_c for every candidate chunk */
+        for (int rr = 0; rr < G; ++rr) {
+            const int h = g * G + rr;
+            const int hl = (p->Hl == p->Hq) ? h : g;
+            const float *qv = q + (((size_t)b * p->Hq + h) * p->Lq + row_qi[r]) * d;
+            for (int c = 0; c < ncand; ++c) {
+                const float *lm = landmarks + (((size_t)b * p->Hl + hl) * p->C + c) * d;
+                double s = scale * dotf(qv, lm, d);
+                if (bias) s += (double)bias[((size_t)b * p->Hl + hl) * p->C + c];
+                shat[rr * ncand + c] = s;
+            }
+        }
+
+        int32_t *sel = sel_idx + ((size_t)r * p->Hkv + g) * K;
+        int n = 0;
+        if (sel_mode == 0) {
+            /* group score: max over the heads of the group (App. C) */
+            for (int c = 0; c < ncand; ++c) { cand[c].c = c; cand[c].u = -INFINITY; }
+            if (p->group_mode == 0) {
+                for (int rr = 0; rr < G; ++rr)
+                    for (int c = 0; c < ncand; ++c)
+                        if (shat[rr * ncand + c] > cand[c].u) cand[c].u = shat[rr * ncand + c];
+            } else {
+                /* variant of Sec. 4.1: normalise each head's scores over the candidates first */
+                for (int rr = 0; rr < G; ++rr) {
+                    double m = -INFINITY, Z = 0.0;
+                    for (int c = 0; c < ncand; ++c) if (shat[rr * ncand + c] > m) m = shat[rr * ncand + c];
+                    for (int c = 0; c < ncand; ++c) Z += exp(shat[rr * ncand + c] - m);
+                    for (int c = 0; c < ncand; ++c) {
+                        double wgt = exp(shat[rr * ncand + c] - m) / Z;
+                        if (wgt > cand[c].u) cand[c].u = wgt;
+                    }
+                }
+            }
+            qsort(cand, (size_t)ncand, sizeof(cand_t), cand_cmp);
+            n = ncand < K ? ncand : K;
+            if (margin)
+                margin[(size_t)r * p->Hkv + g] = (ncand > K && K > 0) ? cand[K - 1].u - cand[K].u : INFINITY;
+            for (int t = 0; t < n; ++t) sel[t] = cand[t].c;
+            qsort(sel, (size_t)n, sizeof(int32_t), int_cmp);
+            for (int t = n; t < K; ++t) sel[t] = -1;
+        } else {
+            for (int t = 0; t < K; ++t) if (sel[t] >= 0) n = t + 1;
+        }
+
+        if (do_attend) {
+            const float *kg = k + ((size_t)b * p->Hkv + g) * (size_t)p->T * d;
+            const float *vg = v + ((size_t)b * p->Hkv + g) * (size_t)p->T * d;
+            for (int rr = 0; rr < G; ++rr) {
+                const int h = g * G + rr;
+                const float *qv = q + (((size_t)b * p->Hq + h) * p->Lq + row_qi[r]) * d;
+                int nslot = 0;
+                /* each selected chunk: its own softmax; mass comes from the surrogate score */
+                for (int t = 0; t < n; ++t) {
+                    const int c = sel[t];
+                    if (c < 0) continue;
+                    if (c >= ncand) { status = -1; continue; }
+                    attend_span(qv, kg, vg, (long)c * S, (long)(c + 1) * S, d, scale,
+                                o_all + (size_t)nslot * d, logits);
+                    lam[nslot] = shat[rr * ncand + c];
+                    ++nslot;
+                }
+                /* local branch: tokens l(i)..i, mass is its own Z_swa */
+                const double lam_loc = attend_span(qv, kg, vg, lo, i + 1, d, scale, o_part, logits);
+                double Mx = lam_loc;
+                for (int t = 0; t < nslot; ++t) if (lam[t] > Mx) Mx = lam[t];
+                double D = exp(lam_loc - Mx);
+                for (int t = 0; t < nslot; ++t) D += exp(lam[t] - Mx);
+                const double a_loc = exp(lam_loc - Mx) / D;
+                if (out) {
+                    double *orow = out + ((size_t)r * p->Hq + h) * d;
+                    for (int x = 0; x < d; ++x) orow[x] = a_loc * o_part[x];
+                    for (int t = 0; t < nslot; ++t) {
+                        const double a = exp(lam[t] - Mx) / D;
+                        for (int x = 0; x < d; ++x) orow[x] += a * o_all[(size_t)t * d + x];
+                    }
+                }
+                if (lse) lse[(size_t)r * p->Hq + h] = Mx + log(D);
+                if (alpha) {
+                    double *ar = alpha + ((size_t)r * p->Hq + h) * (K + 1);
+                    for (int t = 0; t < K; ++t) ar[t] = 0.0;
+                    int slot = 0;
+                    for (int t = 0; t < n; ++t) {
+                        if (sel[t] < 0) continue;
+                        ar[t] = exp(lam[slot] - Mx) / D;
+                        ++slot;
+                    }
+                    ar[K] = a_loc;
+                }
+            }
+        }
+        free(shat); free(cand); free(logits); free(o_part); free(lam); free(o_all);
+    }
+    return status;
+}
+
+int hils_oracle_num_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}

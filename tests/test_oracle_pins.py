@@ -1,0 +1,380 @@
+"""Pins for the CPU oracle: closed forms, invariants, library attention on
+reductions, and an independent brute force.  Each test names the passage of the
+paper that fixes the expected behaviour.  None of these needs a GPU.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from brute_force import brute_force_prefill
+
+
+def rand_inputs(seed, B=1, Hq=2, Hkv=1, L=96, d=8, S=16, Hl=None, amp=1.0, with_bias=False):
+    rng = np.random.default_rng(seed)
+    Hl = Hkv if Hl is None else Hl
+    C = L // S
+    q = (amp * rng.standard_normal((B, Hq, L, d))).astype(np.float32)
+    k = (amp * rng.standard_normal((B, Hkv, L, d))).astype(np.float32)
+    v = rng.standard_normal((B, Hkv, L, d)).astype(np.float32)
+    lm = (amp * rng.standard_normal((B, Hl, C, d))).astype(np.float32)
+    bias = rng.uniform(0, math.log(S), (B, Hl, C)).astype(np.float32) if with_bias else None
+    return q, k, v, lm, bias
+
+
+def causal_sdpa(q, k, v, scale):
+    """Library causal softmax attention in fp64: q [H,L,d], k,v [H,L,d] -> out, lse."""
+    qt, kt, vt = (torch.from_numpy(np.asarray(x, np.float64)) for x in (q, k, v))
+    out = torch.nn.functional.scaled_dot_product_attention(qt, kt, vt, is_causal=True, scale=scale)
+    logits = (qt @ kt.transpose(-1, -2)) * scale
+    L = q.shape[-2]
+    mask = torch.ones(L, L, dtype=torch.bool).tril()
+    lse = torch.logsumexp(logits.masked_fill(~mask, -math.inf), dim=-1)
+    return out.numpy(), lse.numpy()
+
+
+def sdpa_span(qrow, k, v, scale):
+    """Library softmax attention of one query [d] over k,v [n,d]."""
+    qt = torch.from_numpy(np.asarray(qrow, np.float64))[None, None, :]
+    kt = torch.from_numpy(np.asarray(k, np.float64))[None]
+    vt = torch.from_numpy(np.asarray(v, np.float64))[None]
+    o = torch.nn.functional.scaled_dot_product_attention(qt, kt, vt, scale=scale)
+    return o[0, 0].numpy()
+
+
+# ---------------------------------------------------------------- P1
+def test_first_chunk_is_plain_causal_attention():
+    """Rows with no candidate chunk (i < S, W = 1) see only the local branch:
+    Eq. (chunk mass) / App. C middle case -> causal softmax attention and its logsumexp."""
+    S, d = 16, 8
+    q, k, v, lm, _ = rand_inputs(1, Hq=2, Hkv=1, L=64, d=d, S=S)
+    res = oracle.hils_prefill(q, k, v, lm, None, S=S, K=3)
+    scale = 1 / math.sqrt(d)
+    ref_o, ref_lse = causal_sdpa(q[0], np.repeat(k[0], 2, 0), np.repeat(v[0], 2, 0), scale)
+    got_o = res["out"][0].transpose(1, 0, 2)      # [Hq, L, d]
+    got_lse = res["lse"][0].T
+    np.testing.assert_allclose(got_o[:, :S], ref_o[:, :S], atol=1e-12)
+    np.testing.assert_allclose(got_lse[:, :S], ref_lse[:, :S], atol=1e-12)
+    assert (res["sel_idx"][0, :S] == -1).all()
+    assert np.isinf(res["margin"][0, :S]).all()
+
+
+# ---------------------------------------------------------------- P2
+@pytest.mark.parametrize("G", [1, 2, 4])
+def test_chunk_size_one_equals_full_attention(G):
+    """S = 1, landmarks = keys, no bias, K >= L: the surrogate mass exp(s_ic) equals the
+    exact chunk mass, so Eq. (HiLS weights) is an equality with full causal attention."""
+    L, d = 40, 8
+    q, k, v, _, _ = rand_inputs(2, Hq=G, Hkv=1, L=L, d=d, S=1)
+    res = oracle.hils_prefill(q, k, v, k.copy(), None, S=1, K=L)
+    scale = 1 / math.sqrt(d)
+    ref_o, ref_lse = causal_sdpa(q[0], np.repeat(k[0], G, 0), np.repeat(v[0], G, 0), scale)
+    np.testing.assert_allclose(res["out"][0].transpose(1, 0, 2), ref_o, atol=1e-12)
+    np.testing.assert_allclose(res["lse"][0].T, ref_lse, atol=1e-12)
+
+
+def test_chunk_size_one_topk_is_topk_tokens():
+    """S = 1, G = 1, K < candidates: softmax over the K past tokens with the largest logit
+    plus the token itself (Eq. surrogate top-k with exact masses)."""
+    L, d, K = 48, 8, 5
+    q, k, v, _, _ = rand_inputs(3, Hq=1, Hkv=1, L=L, d=d, S=1)
+    res = oracle.hils_prefill(q, k, v, k.copy(), None, S=1, K=K)
+    scale = 1 / math.sqrt(d)
+    for i in [0, 3, 7, 20, 47]:
+        s = scale * (k[0, 0, :i].astype(np.float64) @ q[0, 0, i].astype(np.float64))
+        top = sorted(sorted(range(i), key=lambda c: (-s[c], c))[:K])
+        assert list(res["sel_idx"][0, i, 0][: len(top)]) == top
+        toks = top + [i]
+        ref = sdpa_span(q[0, 0, i], k[0, 0, toks], v[0, 0, toks], scale)
+        np.testing.assert_allclose(res["out"][0, i, 0], ref, atol=1e-12)
+
+
+# ---------------------------------------------------------------- P3
+def test_identical_keys_with_log_s_bias_equals_full_attention():
+    """Keys identical inside each chunk, landmark = that key, bias = log S (the uniform
+    limit of the entropy bias, Prop. 3.1): s_hat = log Z exactly, so with every chunk
+    selected the output is full causal attention; with K < candidates and G = 1 it is
+    naive block-sparse attention (Eq. naive BSA weights) with top-K by exact mass."""
+    S, C, d = 8, 6, 8
+    L = S * C
+    rng = np.random.default_rng(4)
+    kap = rng.standard_normal((1, 1, C, d)).astype(np.float32)
+    k = np.repeat(kap, S, axis=2)
+    q = rng.standard_normal((1, 1, L, d)).astype(np.float32)
+    v = rng.standard_normal((1, 1, L, d)).astype(np.float32)
+    bias = np.full((1, 1, C), math.log(S), np.float32)
+    scale = 1 / math.sqrt(d)
+    res = oracle.hils_prefill(q, k, v, kap, bias, S=S, K=C)
+    ref_o, ref_lse = causal_sdpa(q[0], k[0], v[0], scale)
+    # log(S) is rounded to fp32 in the bias array -> agreement to fp32 epsilon of the weights
+    np.testing.assert_allclose(res["out"][0, :, 0], ref_o[0], atol=5e-7)
+    np.testing.assert_allclose(res["lse"][0, :, 0], ref_lse[0], atol=5e-7)
+    # K < candidates: naive BSA = flat softmax over the top-K chunks by exact mass + local tokens
+    K = 2
+    res = oracle.hils_prefill(q, k, v, kap, bias, S=S, K=K)
+    for i in [L - 1, L - 5, 3 * S + 2]:
+        ci = i // S
+        logit = scale * (k[0, 0].astype(np.float64) @ q[0, 0, i].astype(np.float64))
+        mass = [np.exp(logit[c * S:(c + 1) * S]).sum() for c in range(ci)]
+        top = sorted(sorted(range(ci), key=lambda c: (-mass[c], c))[:K])
+        assert list(res["sel_idx"][0, i, 0]) == top
+        toks = [j for c in top for j in range(c * S, (c + 1) * S)] + list(range(ci * S, i + 1))
+        ref = sdpa_span(q[0, 0, i], k[0, 0, toks], v[0, 0, toks], scale)
+        np.testing.assert_allclose(res["out"][0, i, 0], ref, atol=5e-7)
+
+
+# ---------------------------------------------------------------- P4
+def test_top1_is_sigmoid_mix_of_two_attentions():
+    """K = 1: out = sig * Attn(q, K_c, V_c) + (1 - sig) * CausalAttn_local with
+    sig = sigmoid(s_hat_c - log Z_swa)  (Eq. surrogate top-k, Eq. HiLS weights)."""
+    S, d = 16, 8
+    q, k, v, lm, bias = rand_inputs(5, Hq=1, Hkv=1, L=80, d=d, S=S, with_bias=True)
+    res = oracle.hils_prefill(q, k, v, lm, bias, S=S, K=1)
+    scale = 1 / math.sqrt(d)
+    for i in [16, 31, 50, 79]:
+        ci = i // S
+        sh = scale * (lm[0, 0, :ci].astype(np.float64) @ q[0, 0, i].astype(np.float64)) + bias[0, 0, :ci]
+        c = int(np.argmax(sh))
+        assert res["sel_idx"][0, i, 0, 0] == c
+        o_c = sdpa_span(q[0, 0, i], k[0, 0, c * S:(c + 1) * S], v[0, 0, c * S:(c + 1) * S], scale)
+        o_l = sdpa_span(q[0, 0, i], k[0, 0, ci * S:i + 1], v[0, 0, ci * S:i + 1], scale)
+        loc = scale * (k[0, 0, ci * S:i + 1].astype(np.float64) @ q[0, 0, i].astype(np.float64))
+        log_z = np.log(np.exp(loc).sum())
+        sig = 1 / (1 + math.exp(-(sh[c] - log_z)))
+        np.testing.assert_allclose(res["out"][0, i, 0], sig * o_c + (1 - sig) * o_l, atol=1e-12)
+        np.testing.assert_allclose(res["lse"][0, i, 0], np.log(np.exp(sh[c]) + np.exp(log_z)), atol=1e-12)
+
+
+# ---------------------------------------------------------------- P5
+def test_weights_sum_to_one():
+    """Inter-chunk weights are a softmax (Eq. surrogate top-k: Z_hat is their sum) and the
+    intra-chunk weights are normalised, so constant V is reproduced and shifts pass through."""
+    S, d, K = 16, 8, 3
+    q, k, v, lm, bias = rand_inputs(6, Hq=4, Hkv=2, L=112, d=d, S=S, with_bias=True)
+    res = oracle.hils_prefill(q, k, v, lm, bias, S=S, K=K, want_alpha=True)
+    np.testing.assert_allclose(res["alpha"].sum(-1), 1.0, atol=1e-13)
+    v0 = np.broadcast_to(np.arange(d, dtype=np.float32), v.shape).copy()
+    res0 = oracle.hils_prefill(q, k, v0, lm, bias, S=S, K=K)
+    np.testing.assert_allclose(res0["out"], np.broadcast_to(np.arange(d), res0["out"].shape), atol=1e-12)
+    shift = np.linspace(-1, 1, d).astype(np.float32)
+    res1 = oracle.hils_prefill(q, k, v + shift, lm, bias, S=S, K=K)
+    np.testing.assert_allclose(res1["out"], res["out"] + (v + shift - v)[0, 0, 0].astype(np.float64), atol=1e-6)
+
+
+# ---------------------------------------------------------------- P6
+def test_invariance_to_order_of_selected_chunks_and_permutations():
+    """Eq. (HiLS weights) treats chunks independently and uses no positions beyond causality:
+    (a) the order in which selected chunks are listed does not matter; (b) permuting tokens
+    inside a past chunk, or (c) permuting whole past chunks (with landmarks and bias), leaves
+    later queries unchanged (selection maps through the permutation)."""
+    S, d, K = 8, 8, 3
+    L = 10 * S
+    q, k, v, lm, bias = rand_inputs(7, Hq=2, Hkv=1, L=L, d=d, S=S, with_bias=True)
+    base = oracle.hils_prefill(q, k, v, lm, bias, S=S, K=K)
+    rows = np.arange(6 * S, L)
+
+    # (a) feed the selection back in descending order
+    sel_rev = base["sel_idx"][:, rows][..., ::-1].copy()
+    rev = oracle.hils_prefill(q, k, v, lm, bias, S=S, K=K, rows=rows, sel_idx=sel_rev)
+    np.testing.assert_allclose(rev["out"], base["out"][:, rows], atol=1e-13)
+    np.testing.assert_allclose(rev["lse"], base["lse"][:, rows], atol=1e-13)
+
+    # (b) permute tokens inside chunk 2 (K and V rows jointly)
+    rng = np.random.default_rng(0)
+    perm = rng.permutation(S)
+    k2, v2 = k.copy(), v.copy()
+    k2[:, :, 2 * S:3 * S] = k[:, :, 2 * S:3 * S][:, :, perm]
+    v2[:, :, 2 * S:3 * S] = v[:, :, 2 * S:3 * S][:, :, perm]
+    r2 = oracle.hils_prefill(q, k2, v2, lm, bias, S=S, K=K, rows=rows)
+    np.testing.assert_allclose(r2["out"], base["out"][:, rows], atol=1e-13)
+    assert (r2["sel_idx"] == base["sel_idx"][:, rows]).all()
+
+    # (c) permute the first 6 chunks as wholes
+    cp = rng.permutation(6)
+    inv = np.argsort(cp)                      # old chunk c now sits at position inv[c]
+    k3, v3, lm3, b3 = k.copy(), v.copy(), lm.copy(), bias.copy()
+    for new, old in enumerate(cp):
+        k3[:, :, new * S:(new + 1) * S] = k[:, :, old * S:(old + 1) * S]
+        v3[:, :, new * S:(new + 1) * S] = v[:, :, old * S:(old + 1) * S]
+        lm3[:, :, new] = lm[:, :, old]
+        b3[:, :, new] = bias[:, :, old]
+    r3 = oracle.hils_prefill(q, k3, v3, lm3, b3, S=S, K=K, rows=rows)
+    np.testing.assert_allclose(r3["out"], base["out"][:, rows], atol=1e-13)
+    np.testing.assert_allclose(r3["lse"], base["lse"][:, rows], atol=1e-13)
+    sel_old = base["sel_idx"][:, rows]
+    mapped = np.where((sel_old >= 0) & (sel_old < 6), inv[np.clip(sel_old, 0, 5)], sel_old)
+    assert (np.sort(mapped, -1) == np.sort(r3["sel_idx"], -1)).all()
+
+
+# ---------------------------------------------------------------- P7
+def test_chunk_mass_comes_from_landmark_not_from_keys():
+    """Hierarchy (Eq. HiLS weights): adding one vector to every key of a past chunk shifts all
+    its logits equally; the intra-chunk softmax is unchanged and the inter-chunk mass comes
+    from the landmark only, so outputs do not move.  A flat softmax would move."""
+    S, d, K = 8, 8, 2
+    L = 8 * S
+    q, k, v, lm, bias = rand_inputs(8, Hq=2, Hkv=1, L=L, d=d, S=S, with_bias=True)
+    rows = np.arange(4 * S, L)
+    base = oracle.hils_prefill(q, k, v, lm, bias, S=S, K=K, rows=rows)
+    k2 = k.copy()
+    k2[:, :, 1 * S:2 * S] += np.linspace(0.5, 2.0, d).astype(np.float32)
+    moved = oracle.hils_prefill(q, k2, v, lm, bias, S=S, K=K, rows=rows)
+    assert (base["sel_idx"] == 1).any()       # the shifted chunk is used by some row
+    np.testing.assert_allclose(moved["out"], base["out"], atol=1e-6)
+    np.testing.assert_allclose(moved["lse"], base["lse"], atol=1e-12)
+
+
+# ---------------------------------------------------------------- P8
+def test_large_bias_reduces_to_attention_over_the_selected_chunk():
+    """K = 1 and a +60 bias on one chunk: that chunk takes all inter-chunk mass and the output
+    is ordinary softmax attention restricted to it (error <= e^-40)."""
+    S, d = 16, 8
+    q, k, v, lm, _ = rand_inputs(9, Hq=1, Hkv=1, L=96, d=d, S=S)
+    bias = np.zeros((1, 1, 6), np.float32)
+    bias[0, 0, 2] = 60.0
+    rows = np.arange(3 * S, 96)
+    res = oracle.hils_prefill(q, k, v, lm, bias, S=S, K=1, rows=rows)
+    assert (res["sel_idx"] == 2).all()
+    scale = 1 / math.sqrt(d)
+    for n, i in enumerate(rows):
+        ref = sdpa_span(q[0, 0, i], k[0, 0, 2 * S:3 * S], v[0, 0, 2 * S:3 * S], scale)
+        np.testing.assert_allclose(res["out"][0, n, 0], ref, atol=1e-12)
+
+
+# ---------------------------------------------------------------- P9
+def test_ties_go_to_the_lower_chunk_id():
+    """Equal group scores: the lower chunk id wins (rank over C_i with a stable order)."""
+    S, d, K = 8, 8, 3
+    L = 8 * S
+    q, k, v, lm, _ = rand_inputs(10, Hq=2, Hkv=1, L=L, d=d, S=S)
+    q0 = np.zeros_like(q)                     # all scores equal the (equal) bias
+    bias = np.full((1, 1, L // S), 0.25, np.float32)
+    res = oracle.hils_prefill(q0, k, v, lm, bias, S=S, K=K)
+    for i in [3 * S, 5 * S + 1, L - 1]:
+        assert list(res["sel_idx"][0, i, 0]) == [0, 1, 2]
+    assert (res["margin"][0, 4 * S:, 0] == 0).all()
+    lm2 = lm.copy()
+    lm2[0, 0, 5] = lm2[0, 0, 1]               # duplicate landmark: chunk 1 must beat chunk 5
+    res = oracle.hils_prefill(q, k, v, lm2, None, S=S, K=1)
+    for i in range(6 * S, L):
+        assert res["sel_idx"][0, i, 0, 0] != 5
+
+
+# ---------------------------------------------------------------- P10
+def test_gqa_group_max_and_per_head_weights():
+    """App. C: the group score is the max over the heads of the KV group, selection is shared,
+    the fusion weight stays per head.  Identical heads behave like G = 1; a chunk that only
+    one head likes is selected for all heads and gets a small weight in the others."""
+    S, d, K = 8, 8, 2
+    L = 8 * S
+    q, k, v, lm, _ = rand_inputs(11, Hq=1, Hkv=1, L=L, d=d, S=S)
+    q4 = np.repeat(q, 4, axis=1)
+    r1 = oracle.hils_prefill(q, k, v, lm, None, S=S, K=K)
+    r4 = oracle.hils_prefill(q4, k, v, lm, None, S=S, K=K)
+    assert (r1["sel_idx"] == r4["sel_idx"]).all()
+    for h in range(4):
+        np.testing.assert_allclose(r4["out"][:, :, h], r1["out"][:, :, 0], atol=1e-14)
+    # head 0 strongly aligned with landmark 3, head 1 anti-aligned
+    q2 = np.concatenate([q, q], axis=1) * 0.01
+    q2[0, 0, :, :] += 20 * lm[0, 0, 3] / np.linalg.norm(lm[0, 0, 3])
+    q2[0, 1, :, :] -= 20 * lm[0, 0, 3] / np.linalg.norm(lm[0, 0, 3])
+    rows = np.arange(5 * S, L)
+    r = oracle.hils_prefill(q2, k, v, lm, None, S=S, K=K, rows=rows, want_alpha=True)
+    assert (r["sel_idx"] == 3).any(-1).all()
+    slot = np.argmax(r["sel_idx"][0, :, 0] == 3, axis=-1)
+    a0 = r["alpha"][0, np.arange(len(rows)), 0, slot]
+    a1 = r["alpha"][0, np.arange(len(rows)), 1, slot]
+    assert (a0 > 0.5).all() and (a1 < 1e-3).all()
+
+
+# ---------------------------------------------------------------- P11
+@pytest.mark.parametrize("S,K,G,W,d,Hl_q,with_bias", [
+    (1, 2, 1, 1, 4, False, False),
+    (4, 1, 2, 1, 8, False, True),
+    (4, 3, 4, 4, 4, False, True),
+    (16, 2, 2, 1, 8, True, True),
+    (16, 99, 1, 35, 8, False, False),
+    (4, 3, 2, 11, 8, True, True),
+    (16, 3, 4, 16, 4, False, False),
+])
+def test_brute_force_dense_weight_matrix(S, K, G, W, d, Hl_q, with_bias):
+    """Everything at once against an independent numpy program that builds the dense weight
+    matrix from the three cases of App. C Eq. (HiLS GQA) and multiplies by V."""
+    Hkv = 2
+    Hq = Hkv * G
+    L = 96 if S > 1 else 40
+    q, k, v, lm, bias = rand_inputs(100 + S + K, Hq=Hq, Hkv=Hkv, L=L, d=d, S=S,
+                                    Hl=Hq if Hl_q else Hkv, with_bias=with_bias)
+    res = oracle.hils_prefill(q, k, v, lm, bias, S=S, K=K, W=W)
+    bo, blse, bsel, wts = brute_force_prefill(q[0], k[0], v[0], lm[0], None if bias is None else bias[0],
+                                              S, K, W)
+    np.testing.assert_allclose(res["out"][0].transpose(1, 0, 2), bo, atol=1e-12)
+    np.testing.assert_allclose(res["lse"][0].T, blse, atol=1e-12)
+    np.testing.assert_allclose(wts.sum(-1), 1.0, atol=1e-12)       # dense rows sum to 1
+    for g in range(Hkv):
+        for i in range(L):
+            got = [c for c in res["sel_idx"][0, i, g] if c >= 0]
+            assert got == bsel[g][i], (g, i)
+
+
+def test_support_is_k_chunks_plus_local():
+    """Sec. 7.1: a query's cost is its fixed retrieval budget K x S tokens plus the local
+    window (2048 tokens for S=64, K=32 in the paper's setting): the dense weight row has
+    exactly min(K, candidates) * S + local non-zeros."""
+    with open(__import__("os").path.join(__import__("os").path.dirname(__file__), "golden",
+                                         "retrieval_budget.txt")) as f:
+        vals = dict(line.split("=") for line in f.read().split() if "=" in line)
+    assert int(vals["S"]) * int(vals["K"]) == int(vals["tokens"])
+    S, K = 4, 3
+    q, k, v, lm, _ = rand_inputs(12, Hq=1, Hkv=1, L=64, d=4, S=S)
+    _, _, _, wts = brute_force_prefill(q[0], k[0], v[0], lm[0], None, S, K)
+    res = oracle.hils_prefill(q, k, v, lm, None, S=S, K=K)
+    for i in range(64):
+        nsel = int((res["sel_idx"][0, i, 0] >= 0).sum())
+        assert nsel == min(K, i // S)
+        assert int((wts[0, i] > 0).sum()) == nsel * S + (i % S) + 1
+
+
+# ---------------------------------------------------------------- P12
+def test_decode_equals_last_row_of_prefill_with_partial_chunk():
+    """Decode is the same operator for one query at position seq_len-1; the query's own,
+    possibly partial, chunk is local and only complete chunks are candidates."""
+    S, d, K = 16, 8, 2
+    q, k, v, lm, bias = rand_inputs(13, B=3, Hq=4, Hkv=2, L=112, d=d, S=S, with_bias=True)
+    seq = np.array([112, 71, 16], dtype=np.int32)
+    full = oracle.hils_prefill(q, k, v, lm, bias, S=S, K=K)
+    qd = np.stack([q[b, :, seq[b] - 1] for b in range(3)])
+    dec = oracle.hils_decode(qd, k, v, lm, bias, seq, S=S, K=K)
+    for b in range(3):
+        i = seq[b] - 1
+        np.testing.assert_allclose(dec["out"][b], full["out"][b, i], atol=1e-14)
+        np.testing.assert_allclose(dec["lse"][b], full["lse"][b, i], atol=1e-14)
+        assert (dec["sel_idx"][b] == full["sel_idx"][b, i]).all()
+    # the tail of the cache beyond seq_len is never read: poison it
+    k2, v2, lm2 = k.copy(), v.copy(), lm.copy()
+    k2[1, :, 71:] = np.nan; v2[1, :, 71:] = np.nan; lm2[1, :, 70 // S:] = np.nan
+    dec2 = oracle.hils_decode(qd, k2, v2, lm2, bias, seq, S=S, K=K)
+    np.testing.assert_allclose(dec2["out"][1], dec["out"][1], atol=0)
+
+
+def test_window_candidates_follow_aligned_left_edge():
+    """Sec. 2.1: l(i) = floor((i-W+1)/S)*S, candidates are chunks 0..l(i)/S-1."""
+    S, K, W = 8, 50, 19
+    q, k, v, lm, _ = rand_inputs(14, Hq=1, Hkv=1, L=80, d=4, S=S)
+    res = oracle.hils_prefill(q, k, v, lm, None, S=S, K=K, W=W)
+    for i in range(80):
+        lo = max(0, math.floor((i - W + 1) / S) * S)
+        assert int((res["sel_idx"][0, i, 0] >= 0).sum()) == lo // S
+
+
+def test_normalised_group_mode_is_available_and_differs_only_in_selection():
+    """Sec. 4.1 words the GQA rule on normalised chunk weights; App. C on raw scores (the one
+    used).  With G = 1 both give the same ranking."""
+    S, K = 8, 2
+    q, k, v, lm, _ = rand_inputs(15, Hq=1, Hkv=1, L=64, d=8, S=S)
+    a = oracle.hils_prefill(q, k, v, lm, None, S=S, K=K, group_mode=0)
+    b = oracle.hils_prefill(q, k, v, lm, None, S=S, K=K, group_mode=1)
+    assert (a["sel_idx"] == b["sel_idx"]).all()
+    np.testing.assert_allclose(a["out"], b["out"], atol=0)
