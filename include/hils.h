@@ -1,0 +1,137 @@
+/*
+ * hils.h -- C ABI of the B200 (sm_100a) HiLS attention library.
+ *
+ * HiLS (Hierarchical Landmark Sparse) attention, forward pass.  For a query at
+ * position i (0-based) with chunk size S and local window W:
+ *
+ *   Sec. 2.1   l(i) = max(0, floor((i - W + 1) / S)) * S is the chunk-aligned left edge of the
+ *              local window; candidate chunks are C_i = {0 .. l(i)/S - 1}.
+ *   Eq. (surrogate top-k), App. C Eq. (HiLS GQA)
+ *              per-head surrogate score  s^h_c = scale * q^h . k'_c + b'_c  against the landmark
+ *              (chunk summary key) k'_c and bias b'_c of every candidate chunk; group score
+ *              u_c = max over the query heads of one KV group; the min(K, |C_i|) chunks with the
+ *              largest u_c are selected for the whole group (equal scores: lower chunk id wins).
+ *   Eq. (chunk mass)   local branch: causal softmax over tokens l(i)..i, with mass Z_swa.
+ *   Eq. (HiLS weights) each selected chunk is attended with its own softmax over its S tokens;
+ *              the per-chunk outputs and the local output are mixed with
+ *              softmax({s^h_c : c selected} U {log Z_swa}) -- per head.
+ *              lse = log( sum_c exp(s^h_c) + Z_swa ).
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer owned by the caller unless the entry point says HOST.
+ *   - The library never allocates, frees or synchronises (except where stated); all work is
+ *     enqueued on `stream`.  Outputs are fully overwritten.
+ *   - Tensors are contiguous, last dimension fastest, base pointers 16-byte aligned:
+ *       q, out      [B, Hq, L, d]          (decode: [B, Hq, d])
+ *       k, v        [B, Hkv, T, d]         T = L for prefill, T_max for decode
+ *       landmarks   [B, Hl, C, d]          C = params.C rows per landmark head; row c is only read
+ *                                          when chunk c is complete and precedes the local window
+ *       bias        [B, Hl, C] fp32 or NULL (NULL means 0)
+ *       lse         [B, Hq, L] fp32        (decode: [B, Hq])
+ *       sel_idx     [B, Hkv, L, K] int32   (decode: [B, Hkv, K]) ascending chunk ids, -1 padded
+ *       seq_lens    [B] int32              decode: tokens in the cache INCLUDING the new one; the
+ *                                          query sits at position seq_lens[b]-1, 1 <= seq_lens <= T_max
+ *   - Argument errors are found on the host and returned before anything is launched.
+ *     Device-side anomalies (a wait that ran out, an out-of-range chunk id) set a status word in
+ *     the workspace (read it with hils_poll_status); kernels never trap.
+ *   - Status codes are negative on error; no exception crosses this boundary.
+ */
+#ifndef HILS_H_
+#define HILS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    HILS_OK = 0,
+    HILS_ERR_INVALID_ARG = -1,   /* null pointer, non-positive size, Hq % Hkv != 0, ...           */
+    HILS_ERR_UNSUPPORTED = -2,   /* a shape or option this build has no kernel for                */
+    HILS_ERR_ALIGNMENT = -3,     /* a base pointer is not 16-byte aligned                         */
+    HILS_ERR_WORKSPACE = -4,     /* workspace missing or smaller than hils_workspace_bytes()      */
+    HILS_ERR_CUDA = -5,          /* a CUDA runtime call failed (launch, copy, attribute)          */
+    HILS_ERR_DEVICE_TIMEOUT = -6,/* a bounded device-side wait ran out                            */
+    HILS_ERR_DEVICE_INDEX = -7   /* a kernel met a chunk id outside its valid range               */
+} hils_status;
+
+typedef enum { HILS_F32 = 0, HILS_BF16 = 1 } hils_dtype;
+
+/* Which implementation to run.  AUTO picks the fastest kernel set that supports the shape;
+ * GENERIC forces the shape-agnostic CUDA-core kernels (any d multiple of 32 up to 256,
+ * any chunk size up to 128, any window). */
+typedef enum { HILS_IMPL_AUTO = 0, HILS_IMPL_GENERIC = 1, HILS_IMPL_FAST = 2 } hils_impl;
+
+typedef struct hils_params {
+    int32_t B, Hq, Hkv;
+    int32_t Hl;          /* landmark heads: Hkv (one landmark per chunk per KV head) or Hq          */
+    int32_t L;           /* prefill: number of query tokens == number of kv tokens; decode: ignored */
+    int32_t T_max;       /* kv tokens allocated per (b, kv head); prefill: 0 means L                */
+    int32_t C;           /* landmark rows allocated per (b, landmark head); 0 means T / chunk_size  */
+    int32_t d;           /* head dimension                                                          */
+    int32_t chunk_size;  /* S                                                                       */
+    int32_t top_k;       /* K                                                                       */
+    int32_t window;      /* W of Sec. 2.1; 1 = the query's own chunk is the local region            */
+    float   scale;       /* logit scale; 0 means 1/sqrt(d)                                          */
+    int32_t dtype;       /* hils_dtype of q, k, v, landmarks, out                                   */
+    int32_t impl;        /* hils_impl                                                               */
+} hils_params;
+
+/* Bytes of device scratch hils_prefill (is_decode = 0) or hils_decode (is_decode = 1) needs for
+ * these parameters.  Returns 0 if the parameters are invalid.  The first 256 bytes hold the
+ * device status word; the caller must zero them once after allocation. */
+size_t hils_workspace_bytes(const hils_params* params, int is_decode);
+
+/* Prefill: Eq. (surrogate top-k) + Eq. (HiLS weights) (GQA form: App. C) for all L positions of
+ * every sequence.  `lse` and `sel_idx` may not be NULL.  Asynchronous on `stream`
+ * (a cudaStream_t passed as void*). */
+int hils_prefill(const hils_params* params, const void* q, const void* k, const void* v,
+                 const void* landmarks, const float* bias,
+                 void* out, float* lse, int32_t* sel_idx,
+                 void* workspace, size_t workspace_bytes, void* stream);
+
+/* Decode: the same operator for one query per sequence at position seq_lens[b]-1 over a contiguous
+ * KV cache that already holds the new token's k and v (the query attends to itself through the
+ * local branch, Sec. 2.1: j <= i).  The query's own, possibly partial, chunk is local; only
+ * complete earlier chunks are candidates. */
+int hils_decode(const hils_params* params, const void* q, const void* k_cache, const void* v_cache,
+                const void* landmarks, const float* bias, const int32_t* seq_lens,
+                void* out, float* lse, int32_t* sel_idx,
+                void* workspace, size_t workspace_bytes, void* stream);
+
+/* Bytes of device memory the *_host entry points need for staging (inputs + outputs + workspace). */
+size_t hils_host_arena_bytes(const hils_params* params, int is_decode);
+
+/* Same operators with HOST input and output buffers (pinned memory recommended).  Inputs are copied
+ * to `device_arena` (a DEVICE buffer of at least hils_host_arena_bytes()), the device entry point
+ * runs, and out / lse / sel_idx are copied back, all enqueued on `stream`.  The call returns
+ * without synchronising: results are valid once the stream has been synchronised.  The arena's
+ * first 256 bytes are the status word (zero them once). */
+int hils_prefill_host(const hils_params* params, const void* q_host, const void* k_host,
+                      const void* v_host, const void* landmarks_host, const float* bias_host,
+                      void* out_host, float* lse_host, int32_t* sel_idx_host,
+                      void* device_arena, size_t arena_bytes, void* stream);
+int hils_decode_host(const hils_params* params, const void* q_host, const void* k_cache_host,
+                     const void* v_cache_host, const void* landmarks_host, const float* bias_host,
+                     const int32_t* seq_lens_host,
+                     void* out_host, float* lse_host, int32_t* sel_idx_host,
+                     void* device_arena, size_t arena_bytes, void* stream);
+
+/* Reads the device status word at the start of `workspace` (synchronises `stream`).
+ * Returns HILS_OK, HILS_ERR_DEVICE_TIMEOUT, HILS_ERR_DEVICE_INDEX or HILS_ERR_CUDA. */
+int hils_poll_status(const void* workspace, void* stream);
+
+/* Number of kernels the last hils_prefill / hils_decode call of this thread enqueued. */
+int hils_last_launch_count(void);
+
+const char* hils_status_string(int status);
+
+/* Library version, "major.minor". */
+const char* hils_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HILS_H_ */

@@ -28,7 +28,7 @@ class _Params(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int), ("Hq", ctypes.c_int), ("Hkv", ctypes.c_int), ("Hl", ctypes.c_int),
                 ("Lq", ctypes.c_int), ("T", ctypes.c_int), ("C", ctypes.c_int),
                 ("d", ctypes.c_int), ("S", ctypes.c_int), ("K", ctypes.c_int), ("W", ctypes.c_int),
-                ("scale", ctypes.c_double), ("group_mode", ctypes.c_int)]
+                ("scale", ctypes.c_double), ("group_mode", ctypes.c_int), ("in_bf16", ctypes.c_int)]
 
 
 def build(force: bool = False) -> str:
@@ -56,11 +56,21 @@ def num_threads() -> int:
     return int(_load().hils_oracle_num_threads())
 
 
+def _is_bf16(a) -> bool:
+    return hasattr(a, "detach") and str(a.dtype) == "torch.bfloat16"
+
+
 def _f32(a) -> np.ndarray:
     """fp32 C-contiguous numpy view/copy of a numpy array or a CPU torch tensor (bf16 widens exactly)."""
     if hasattr(a, "detach"):
         a = a.detach().to("cpu").float().contiguous().numpy()
     return np.ascontiguousarray(a, dtype=np.float32)
+
+
+def _raw_bf16(a) -> np.ndarray:
+    """The 16-bit patterns of a CPU bf16 torch tensor as a uint16 numpy array (no copy if contiguous)."""
+    import torch
+    return a.detach().to("cpu").contiguous().view(torch.int16).numpy().view(np.uint16)
 
 
 def _ptr(a: Optional[np.ndarray], ct):
@@ -79,7 +89,9 @@ def hils_rows(q, k, v, landmarks, bias, *, S: int, K: int, W: int = 1, scale: fl
     Returns dict(sel_idx, margin, out, lse[, alpha]) as numpy arrays indexed by row.
     """
     lib = _load()
-    q = _f32(q); k = _f32(k); v = _f32(v); landmarks = _f32(landmarks)
+    in_bf16 = int(all(_is_bf16(t) for t in (q, k, v, landmarks)))
+    conv = _raw_bf16 if in_bf16 else _f32
+    q = conv(q); k = conv(k); v = conv(v); landmarks = conv(landmarks)
     bias_a = None if bias is None else _f32(bias)
     B, Hq, Lq, d = q.shape
     _, Hkv, T, _ = k.shape
@@ -88,7 +100,7 @@ def hils_rows(q, k, v, landmarks, bias, *, S: int, K: int, W: int = 1, scale: fl
     row_qi = np.ascontiguousarray(row_qi, dtype=np.int32)
     row_pos = np.ascontiguousarray(row_pos, dtype=np.int64)
     n = row_b.shape[0]
-    p = _Params(B, Hq, Hkv, Hl, Lq, T, C, d, S, K, W, float(scale), group_mode)
+    p = _Params(B, Hq, Hkv, Hl, Lq, T, C, d, S, K, W, float(scale), group_mode, in_bf16)
     sel_mode = 0
     if sel_idx is None:
         sel = np.full((n, Hkv, K), -1, dtype=np.int32)
@@ -100,8 +112,8 @@ def hils_rows(q, k, v, landmarks, bias, *, S: int, K: int, W: int = 1, scale: fl
     lse = np.zeros((n, Hq), dtype=np.float64) if attend else None
     alpha = np.zeros((n, Hq, K + 1), dtype=np.float64) if (attend and want_alpha) else None
     rc = lib.hils_oracle_rows(
-        ctypes.byref(p), _ptr(q, ctypes.c_float), _ptr(k, ctypes.c_float), _ptr(v, ctypes.c_float),
-        _ptr(landmarks, ctypes.c_float), _ptr(bias_a, ctypes.c_float),
+        ctypes.byref(p), ctypes.c_void_p(q.ctypes.data), ctypes.c_void_p(k.ctypes.data),
+        ctypes.c_void_p(v.ctypes.data), ctypes.c_void_p(landmarks.ctypes.data), _ptr(bias_a, ctypes.c_float),
         ctypes.c_int64(n), _ptr(row_b, ctypes.c_int32), _ptr(row_qi, ctypes.c_int32),
         _ptr(row_pos, ctypes.c_int64), ctypes.c_int(sel_mode), ctypes.c_int(1 if attend else 0),
         _ptr(sel, ctypes.c_int32), _ptr(margin, ctypes.c_double),
@@ -140,7 +152,7 @@ def hils_decode(q, k_cache, v_cache, landmarks, bias, seq_lens, *, S: int, K: in
 
     q [B,Hq,d].  Returns sel_idx [B,Hkv,K], margin [B,Hkv], out [B,Hq,d], lse [B,Hq].
     """
-    qn = _f32(q)
+    qn = q if _is_bf16(q) else _f32(q)
     B, Hq, d = qn.shape
     seq = np.asarray(seq_lens.cpu() if hasattr(seq_lens, "cpu") else seq_lens, dtype=np.int64)
     return hils_rows(qn.reshape(B, Hq, 1, d), k_cache, v_cache, landmarks, bias, S=S, K=K, W=W,

@@ -29,8 +29,8 @@
  *                   lse = log( sum_c exp(s^h_c) + Z_swa ).
  *
  * No blocking, fusion or reordering beyond the steps above.  Inputs are fp32
- * arrays (bf16 data is widened exactly by the caller); all arithmetic is fp64
- * with libm exp/log.
+ * or raw bf16 arrays, widened exactly to fp64 element by element; all
+ * arithmetic is fp64 with libm exp/log.
  *
  * Pinned by tests/test_oracle_pins.py (closed forms, invariants, library
  * attention on reductions, an independent dense-weight brute force).  The paper
@@ -54,6 +54,7 @@ typedef struct {
     int d, S, K, W;
     double scale;         /* <= 0 means 1/sqrt(d)                                       */
     int group_mode;       /* 0: u_c = max_h s^h_c (App. C); 1: max_h of softmax_c(s^h)  */
+    int in_bf16;          /* 0: q,k,v,landmarks are float32; 1: raw bfloat16 (uint16)   */
 } hils_oracle_params;
 
 static long floordiv(long a, long b) {
@@ -62,9 +63,18 @@ static long floordiv(long a, long b) {
     return q;
 }
 
-static double dotf(const float *a, const float *b, int n) {
+/* element i of a float32 or raw-bfloat16 array, widened exactly to double */
+static double ld(const void *base, size_t i, int bf16) {
+    if (!bf16) return (double)((const float *)base)[i];
+    uint32_t bits = (uint32_t)((const uint16_t *)base)[i] << 16;
+    float f;
+    memcpy(&f, &bits, sizeof f);
+    return (double)f;
+}
+
+static double dotx(const void *a, size_t ia, const void *b, size_t ib, int n, int bf16) {
     double acc = 0.0;
-    for (int t = 0; t < n; ++t) acc += (double)a[t] * (double)b[t];
+    for (int t = 0; t < n; ++t) acc += ld(a, ia + t, bf16) * ld(b, ib + t, bf16);
     return acc;
 }
 
@@ -84,12 +94,12 @@ static int int_cmp(const void *pa, const void *pb) {
 }
 
 /* softmax attention of one query over rows [lo, hi) of K/V; returns m + log Z, writes o[d] */
-static double attend_span(const float *q, const float *k, const float *v, long lo, long hi,
-                          int d, double scale, double *o, double *logits) {
+static double attend_span(const void *q, size_t iq, const void *k, const void *v, size_t ikv,
+                          long lo, long hi, int d, double scale, int bf16, double *o, double *logits) {
     long n = hi - lo;
     double m = -INFINITY;
     for (long j = 0; j < n; ++j) {
-        logits[j] = scale * dotf(q, k + (lo + j) * d, d);
+        logits[j] = scale * dotx(q, iq, k, ikv + (size_t)(lo + j) * d, d, bf16);
         if (logits[j] > m) m = logits[j];
     }
     double Z = 0.0;
@@ -97,8 +107,7 @@ static double attend_span(const float *q, const float *k, const float *v, long l
     for (long j = 0; j < n; ++j) {
         double p = exp(logits[j] - m);
         Z += p;
-        const float *vr = v + (lo + j) * d;
-        for (int t = 0; t < d; ++t) o[t] += p * (double)vr[t];
+        for (int t = 0; t < d; ++t) o[t] += p * ld(v, ikv + (size_t)(lo + j) * d + t, bf16);
     }
     for (int t = 0; t < d; ++t) o[t] /= Z;
     return m + log(Z);
@@ -118,8 +127,8 @@ static double attend_span(const float *q, const float *k, const float *v, long l
  * Returns 0, or -1 on bad arguments.
  */
 int hils_oracle_rows(const hils_oracle_params *p,
-                     const float *q, const float *k, const float *v,
-                     const float *landmarks, const float *bias,
+                     const void *q, const void *k, const void *v,
+                     const void *landmarks, const float *bias,
                      int64_t n_rows, const int32_t *row_b, const int32_t *row_qi,
                      const int64_t *row_pos,
                      int sel_mode, int do_attend,
@@ -129,7 +138,7 @@ int hils_oracle_rows(const hils_oracle_params *p,
     if (!p || p->Hq % p->Hkv != 0 || (p->Hl != p->Hkv && p->Hl != p->Hq) || p->S <= 0 ||
         p->K < 0 || p->W < 1 || !sel_idx)
         return -1;
-    const int G = p->Hq / p->Hkv, d = p->d, S = p->S, K = p->K;
+    const int G = p->Hq / p->Hkv, d = p->d, S = p->S, K = p->K, bf = p->in_bf16;
     const double scale = p->scale > 0 ? p->scale : 1.0 / sqrt((double)d);
     const int64_t work = n_rows * p->Hkv;
     int status = 0;
@@ -156,10 +165,10 @@ int hils_oracle_rows(const hils_oracle_params *p,
         for (int rr = 0; rr < G; ++rr) {
             const int h = g * G + rr;
             const int hl = (p->Hl == p->Hq) ? h : g;
-            const float *qv = q + (((size_t)b * p->Hq + h) * p->Lq + row_qi[r]) * d;
+            const size_t iq = (((size_t)b * p->Hq + h) * p->Lq + row_qi[r]) * d;
             for (int c = 0; c < ncand; ++c) {
-                const float *lm = landmarks + (((size_t)b * p->Hl + hl) * p->C + c) * d;
-                double s = scale * dotf(qv, lm, d);
+                const size_t ilm = (((size_t)b * p->Hl + hl) * p->C + c) * d;
+                double s = scale * dotx(q, iq, landmarks, ilm, d, bf);
                 if (bias) s += (double)bias[((size_t)b * p->Hl + hl) * p->C + c];
                 shat[rr * ncand + c] = s;
             }
@@ -198,24 +207,23 @@ int hils_oracle_rows(const hils_oracle_params *p,
         }
 
         if (do_attend) {
-            const float *kg = k + ((size_t)b * p->Hkv + g) * (size_t)p->T * d;
-            const float *vg = v + ((size_t)b * p->Hkv + g) * (size_t)p->T * d;
+            const size_t ikv = ((size_t)b * p->Hkv + g) * (size_t)p->T * d;
             for (int rr = 0; rr < G; ++rr) {
                 const int h = g * G + rr;
-                const float *qv = q + (((size_t)b * p->Hq + h) * p->Lq + row_qi[r]) * d;
+                const size_t iq = (((size_t)b * p->Hq + h) * p->Lq + row_qi[r]) * d;
                 int nslot = 0;
                 /* each selected chunk: its own softmax; mass comes from the surrogate score */
                 for (int t = 0; t < n; ++t) {
                     const int c = sel[t];
                     if (c < 0) continue;
                     if (c >= ncand) { status = -1; continue; }
-                    attend_span(qv, kg, vg, (long)c * S, (long)(c + 1) * S, d, scale,
+                    attend_span(q, iq, k, v, ikv, (long)c * S, (long)(c + 1) * S, d, scale, bf,
                                 o_all + (size_t)nslot * d, logits);
                     lam[nslot] = shat[rr * ncand + c];
                     ++nslot;
                 }
                 /* local branch: tokens l(i)..i, mass is its own Z_swa */
-                const double lam_loc = attend_span(qv, kg, vg, lo, i + 1, d, scale, o_part, logits);
+                const double lam_loc = attend_span(q, iq, k, v, ikv, lo, i + 1, d, scale, bf, o_part, logits);
                 double Mx = lam_loc;
                 for (int t = 0; t < nslot; ++t) if (lam[t] > Mx) Mx = lam[t];
                 double D = exp(lam_loc - Mx);

@@ -1,0 +1,261 @@
+"""ctypes binding of libhils.so -- argument marshalling only.
+
+Every step of the operator runs in the CUDA kernels of the library; this module checks tensor
+types, builds the parameter struct, provides the workspace from torch's allocator and passes raw
+device pointers and the current CUDA stream through the C ABI declared in include/hils.h.
+There is no CPU or PyTorch fallback: if the shared library is missing, every call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Dict, Optional, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libhils.so")
+
+HILS_F32, HILS_BF16 = 0, 1
+IMPL_AUTO, IMPL_GENERIC, IMPL_FAST = 0, 1, 2
+_IMPL = {"auto": IMPL_AUTO, "generic": IMPL_GENERIC, "fast": IMPL_FAST}
+
+EXPORTS = [
+    "hils_workspace_bytes", "hils_prefill", "hils_decode", "hils_host_arena_bytes",
+    "hils_prefill_host", "hils_decode_host", "hils_poll_status", "hils_last_launch_count",
+    "hils_status_string", "hils_version",
+]
+
+
+class HilsParams(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("Hq", ctypes.c_int32), ("Hkv", ctypes.c_int32), ("Hl", ctypes.c_int32),
+                ("L", ctypes.c_int32), ("T_max", ctypes.c_int32), ("C", ctypes.c_int32), ("d", ctypes.c_int32),
+                ("chunk_size", ctypes.c_int32), ("top_k", ctypes.c_int32), ("window", ctypes.c_int32),
+                ("scale", ctypes.c_float), ("dtype", ctypes.c_int32), ("impl", ctypes.c_int32)]
+
+
+class HilsError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s failed: %s (%d)" % (where, status_string(status), status))
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Loads libhils.so from the package directory; raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(
+            "HiLS CUDA library not built: %s is missing. Run `python -m paper_2607_02980_b200.build` "
+            "(there is no CPU fallback)." % LIB_PATH)
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32p, f32p = ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p
+    pp = ctypes.POINTER(HilsParams)
+    lib.hils_workspace_bytes.restype = ctypes.c_size_t
+    lib.hils_workspace_bytes.argtypes = [pp, ctypes.c_int]
+    lib.hils_host_arena_bytes.restype = ctypes.c_size_t
+    lib.hils_host_arena_bytes.argtypes = [pp, ctypes.c_int]
+    lib.hils_prefill.restype = ctypes.c_int
+    lib.hils_prefill.argtypes = [pp, vp, vp, vp, vp, f32p, vp, f32p, i32p, vp, ctypes.c_size_t, vp]
+    lib.hils_decode.restype = ctypes.c_int
+    lib.hils_decode.argtypes = [pp, vp, vp, vp, vp, f32p, i32p, vp, f32p, i32p, vp, ctypes.c_size_t, vp]
+    lib.hils_prefill_host.restype = ctypes.c_int
+    lib.hils_prefill_host.argtypes = [pp, vp, vp, vp, vp, f32p, vp, f32p, i32p, vp, ctypes.c_size_t, vp]
+    lib.hils_decode_host.restype = ctypes.c_int
+    lib.hils_decode_host.argtypes = [pp, vp, vp, vp, vp, f32p, i32p, vp, f32p, i32p, vp, ctypes.c_size_t, vp]
+    lib.hils_poll_status.restype = ctypes.c_int
+    lib.hils_poll_status.argtypes = [vp, vp]
+    lib.hils_last_launch_count.restype = ctypes.c_int
+    lib.hils_status_string.restype = ctypes.c_char_p
+    lib.hils_status_string.argtypes = [ctypes.c_int]
+    lib.hils_version.restype = ctypes.c_char_p
+    _lib = lib
+    return lib
+
+
+def status_string(status: int) -> str:
+    return load_library().hils_status_string(int(status)).decode()
+
+
+def version() -> str:
+    return load_library().hils_version().decode()
+
+
+def last_launch_count() -> int:
+    return int(load_library().hils_last_launch_count())
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return HILS_F32
+    if t.dtype == torch.bfloat16:
+        return HILS_BF16
+    raise TypeError("HiLS supports float32 and bfloat16 tensors, got %s" % t.dtype)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _check(t: torch.Tensor, name: str, shape: Tuple[int, ...], dtype, cuda: bool):
+    if tuple(t.shape) != tuple(shape):
+        raise ValueError("%s has shape %s, expected %s" % (name, tuple(t.shape), tuple(shape)))
+    if t.dtype != dtype:
+        raise TypeError("%s has dtype %s, expected %s" % (name, t.dtype, dtype))
+    if not t.is_contiguous():
+        raise ValueError("%s must be contiguous" % name)
+    if cuda != t.is_cuda:
+        raise ValueError("%s must live on %s" % (name, "a CUDA device" if cuda else "the host"))
+
+
+def make_params(*, B, Hq, Hkv, Hl, L, T_max, C, d, chunk_size, top_k, window=1, scale=0.0, dtype, impl="auto"):
+    return HilsParams(B, Hq, Hkv, Hl, L, T_max, C, d, chunk_size, top_k, window, float(scale), dtype, _IMPL[impl])
+
+
+def workspace_bytes(params: HilsParams, is_decode: bool) -> int:
+    return int(load_library().hils_workspace_bytes(ctypes.byref(params), 1 if is_decode else 0))
+
+
+def host_arena_bytes(params: HilsParams, is_decode: bool) -> int:
+    return int(load_library().hils_host_arena_bytes(ctypes.byref(params), 1 if is_decode else 0))
+
+
+def alloc_workspace(params: HilsParams, is_decode: bool, device) -> torch.Tensor:
+    n = workspace_bytes(params, is_decode)
+    if n == 0:
+        raise HilsError(-2, "hils_workspace_bytes")
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    ws[:256].zero_()
+    return ws
+
+
+def _stream_ptr(stream) -> ctypes.c_void_p:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def hils_prefill(q, k, v, landmarks, chunk_size: int, top_k: int, out=None, lse=None, sel_idx=None, stream=None, *,
+                 bias=None, window: int = 1, scale: float = 0.0, impl: str = "auto", workspace=None):
+    """HiLS prefill on CUDA tensors: q [B,Hq,L,d], k,v [B,Hkv,L,d], landmarks [B,Hl,C,d].
+
+    Returns (out [B,Hq,L,d], lse [B,Hq,L] fp32, sel_idx [B,Hkv,L,K] int32).  Asynchronous on the
+    given (default: current) CUDA stream.
+    """
+    lib = load_library()
+    B, Hq, L, d = q.shape
+    Hkv, T = k.shape[1], k.shape[2]
+    Hl, C = landmarks.shape[1], landmarks.shape[2]
+    dt = q.dtype
+    _check(q, "q", (B, Hq, L, d), dt, True)
+    _check(k, "k", (B, Hkv, T, d), dt, True)
+    _check(v, "v", (B, Hkv, T, d), dt, True)
+    _check(landmarks, "landmarks", (B, Hl, C, d), dt, True)
+    if bias is not None:
+        _check(bias, "bias", (B, Hl, C), torch.float32, True)
+    out = torch.empty_like(q) if out is None else out
+    lse = torch.empty((B, Hq, L), dtype=torch.float32, device=q.device) if lse is None else lse
+    sel_idx = torch.empty((B, Hkv, L, top_k), dtype=torch.int32, device=q.device) if sel_idx is None else sel_idx
+    _check(out, "out", (B, Hq, L, d), dt, True)
+    _check(lse, "lse", (B, Hq, L), torch.float32, True)
+    _check(sel_idx, "sel_idx", (B, Hkv, L, top_k), torch.int32, True)
+    p = make_params(B=B, Hq=Hq, Hkv=Hkv, Hl=Hl, L=L, T_max=T, C=C, d=d, chunk_size=chunk_size, top_k=top_k,
+                    window=window, scale=scale, dtype=_dtype_code(q), impl=impl)
+    ws = alloc_workspace(p, False, q.device) if workspace is None else workspace
+    rc = lib.hils_prefill(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(landmarks), _ptr(bias), _ptr(out),
+                          _ptr(lse), _ptr(sel_idx), _ptr(ws), ws.numel(), _stream_ptr(stream))
+    if rc != 0:
+        raise HilsError(rc, "hils_prefill")
+    return out, lse, sel_idx
+
+
+def hils_decode(q, k_cache, v_cache, landmarks, seq_lens, chunk_size: int, top_k: int, out=None, lse=None,
+                sel_idx=None, stream=None, *, bias=None, window: int = 1, scale: float = 0.0, impl: str = "auto",
+                workspace=None):
+    """HiLS single-token decode: q [B,Hq,d], caches [B,Hkv,T_max,d], seq_lens [B] int32 (CUDA).
+
+    Returns (out [B,Hq,d], lse [B,Hq], sel_idx [B,Hkv,K])."""
+    lib = load_library()
+    B, Hq, d = q.shape
+    Hkv, T = k_cache.shape[1], k_cache.shape[2]
+    Hl, C = landmarks.shape[1], landmarks.shape[2]
+    dt = q.dtype
+    _check(q, "q", (B, Hq, d), dt, True)
+    _check(k_cache, "k_cache", (B, Hkv, T, d), dt, True)
+    _check(v_cache, "v_cache", (B, Hkv, T, d), dt, True)
+    _check(landmarks, "landmarks", (B, Hl, C, d), dt, True)
+    _check(seq_lens, "seq_lens", (B,), torch.int32, True)
+    if bias is not None:
+        _check(bias, "bias", (B, Hl, C), torch.float32, True)
+    out = torch.empty_like(q) if out is None else out
+    lse = torch.empty((B, Hq), dtype=torch.float32, device=q.device) if lse is None else lse
+    sel_idx = torch.empty((B, Hkv, top_k), dtype=torch.int32, device=q.device) if sel_idx is None else sel_idx
+    _check(out, "out", (B, Hq, d), dt, True)
+    _check(lse, "lse", (B, Hq), torch.float32, True)
+    _check(sel_idx, "sel_idx", (B, Hkv, top_k), torch.int32, True)
+    p = make_params(B=B, Hq=Hq, Hkv=Hkv, Hl=Hl, L=0, T_max=T, C=C, d=d, chunk_size=chunk_size, top_k=top_k,
+                    window=window, scale=scale, dtype=_dtype_code(q), impl=impl)
+    ws = alloc_workspace(p, True, q.device) if workspace is None else workspace
+    rc = lib.hils_decode(ctypes.byref(p), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(landmarks), _ptr(bias),
+                         _ptr(seq_lens), _ptr(out), _ptr(lse), _ptr(sel_idx), _ptr(ws), ws.numel(),
+                         _stream_ptr(stream))
+    if rc != 0:
+        raise HilsError(rc, "hils_decode")
+    return out, lse, sel_idx
+
+
+class HostRunner:
+    """End-to-end calls with HOST tensors through hils_prefill_host / hils_decode_host.
+
+    Owns the device arena (allocated once from torch) and pinned output buffers; each `run`
+    enqueues host->device copies, the kernels and device->host copies on the current stream.
+    """
+
+    def __init__(self, params: HilsParams, is_decode: bool, device="cuda"):
+        self.params, self.is_decode = params, is_decode
+        n = host_arena_bytes(params, is_decode)
+        if n == 0:
+            raise HilsError(-2, "hils_host_arena_bytes")
+        self.arena = torch.empty(n + 256, dtype=torch.uint8, device=device)
+        off = (-self.arena.data_ptr()) % 256
+        self.arena = self.arena[off:off + n]
+        self.arena[:256].zero_()
+        p = params
+        R = 1 if is_decode else p.L
+        dt = torch.float32 if p.dtype == HILS_F32 else torch.bfloat16
+        oshape = (p.B, p.Hq, p.d) if is_decode else (p.B, p.Hq, R, p.d)
+        lshape = (p.B, p.Hq) if is_decode else (p.B, p.Hq, R)
+        sshape = (p.B, p.Hkv, p.top_k) if is_decode else (p.B, p.Hkv, R, p.top_k)
+        self.out = torch.empty(oshape, dtype=dt).pin_memory()
+        self.lse = torch.empty(lshape, dtype=torch.float32).pin_memory()
+        self.sel = torch.empty(sshape, dtype=torch.int32).pin_memory()
+
+    def bytes_per_step(self, tensors: Dict[str, torch.Tensor]) -> Tuple[int, int]:
+        h2d = sum(t.numel() * t.element_size() for t in tensors.values() if t is not None)
+        d2h = sum(t.numel() * t.element_size() for t in (self.out, self.lse, self.sel))
+        return h2d, d2h
+
+    def run(self, q, k, v, landmarks, bias=None, seq_lens=None, stream=None):
+        lib = load_library()
+        for name, t in (("q", q), ("k", k), ("v", v), ("landmarks", landmarks)):
+            if t.is_cuda or not t.is_contiguous():
+                raise ValueError("%s must be a contiguous host tensor" % name)
+        sp = _stream_ptr(stream)
+        if self.is_decode:
+            rc = lib.hils_decode_host(ctypes.byref(self.params), _ptr(q), _ptr(k), _ptr(v), _ptr(landmarks),
+                                      _ptr(bias), _ptr(seq_lens), _ptr(self.out), _ptr(self.lse), _ptr(self.sel),
+                                      _ptr(self.arena), self.arena.numel(), sp)
+        else:
+            rc = lib.hils_prefill_host(ctypes.byref(self.params), _ptr(q), _ptr(k), _ptr(v), _ptr(landmarks),
+                                       _ptr(bias), _ptr(self.out), _ptr(self.lse), _ptr(self.sel),
+                                       _ptr(self.arena), self.arena.numel(), sp)
+        if rc != 0:
+            raise HilsError(rc, "hils_decode_host" if self.is_decode else "hils_prefill_host")
+        return self.out, self.lse, self.sel
+
+
+def poll_status(workspace: torch.Tensor, stream=None) -> int:
+    return int(load_library().hils_poll_status(_ptr(workspace), _stream_ptr(stream)))

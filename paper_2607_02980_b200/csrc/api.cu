@@ -1,0 +1,246 @@
+// C ABI of the HiLS library: argument validation, kernel-set dispatch, host-buffer variants.
+#include <string.h>
+
+#include "internal.h"
+
+namespace hils {
+namespace {
+
+thread_local int g_last_launches = 0;
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline size_t elem_bytes(int dtype) { return dtype == HILS_F32 ? 4 : 2; }
+
+// Fills `s` from the public parameters; returns a status.
+int make_shape(const hils_params* p, int is_decode, Shape* s) {
+    if (!p) return HILS_ERR_INVALID_ARG;
+    if (p->B < 1 || p->Hq < 1 || p->Hkv < 1 || p->d < 1 || p->chunk_size < 1 || p->top_k < 1 || p->window < 1)
+        return HILS_ERR_INVALID_ARG;
+    if (p->Hq % p->Hkv != 0) return HILS_ERR_INVALID_ARG;
+    if (p->Hl != p->Hkv && p->Hl != p->Hq) return HILS_ERR_INVALID_ARG;
+    if (p->dtype != HILS_F32 && p->dtype != HILS_BF16) return HILS_ERR_INVALID_ARG;
+    if (p->impl < HILS_IMPL_AUTO || p->impl > HILS_IMPL_FAST) return HILS_ERR_INVALID_ARG;
+    if (!(p->scale >= 0.f)) return HILS_ERR_INVALID_ARG;
+    s->B = p->B; s->Hq = p->Hq; s->Hkv = p->Hkv; s->Hl = p->Hl; s->G = p->Hq / p->Hkv;
+    s->d = p->d; s->S = p->chunk_size; s->K = p->top_k; s->W = p->window;
+    s->scale = p->scale > 0.f ? p->scale : 1.0f / sqrtf(static_cast<float>(p->d));
+    s->is_decode = is_decode;
+    if (is_decode) {
+        if (p->T_max < 1) return HILS_ERR_INVALID_ARG;
+        s->R = 1;
+        s->T = p->T_max;
+    } else {
+        if (p->L < 1) return HILS_ERR_INVALID_ARG;
+        s->R = p->L;
+        s->T = p->T_max > 0 ? p->T_max : p->L;
+        if (s->T < p->L) return HILS_ERR_INVALID_ARG;
+    }
+    s->C = p->C > 0 ? p->C : s->T / s->S;
+    // every candidate chunk of the last position must have a landmark row
+    const int last = is_decode ? s->T - 1 : p->L - 1;
+    const int max_cand = local_lo(last, s->W, s->S) / s->S;
+    if (s->C < max_cand) return HILS_ERR_INVALID_ARG;
+    return HILS_OK;
+}
+
+enum class Path { Generic, DecodeFast, PrefillFast };
+
+int pick_path(const Shape& s, const hils_params* p, Path* path) {
+    const bool fast_ok = s.is_decode ? decode_fast_supports(s, p->dtype) : prefill_fast_supports(s, p->dtype);
+    if (p->impl == HILS_IMPL_FAST) {
+        if (!fast_ok) return HILS_ERR_UNSUPPORTED;
+        *path = s.is_decode ? Path::DecodeFast : Path::PrefillFast;
+        return HILS_OK;
+    }
+    if (p->impl == HILS_IMPL_AUTO && fast_ok) {
+        *path = s.is_decode ? Path::DecodeFast : Path::PrefillFast;
+        return HILS_OK;
+    }
+    if (!generic_supports(s)) return HILS_ERR_UNSUPPORTED;
+    *path = Path::Generic;
+    return HILS_OK;
+}
+
+size_t scratch_bytes(const Shape& s, Path path) {
+    switch (path) {
+        case Path::DecodeFast: return decode_fast_scratch_bytes(s);
+        case Path::PrefillFast: return prefill_fast_scratch_bytes(s);
+        default: return 0;
+    }
+}
+
+int run(const hils_params* p, int is_decode, const void* q, const void* k, const void* v, const void* lm,
+        const float* bias, const int32_t* seq_lens, void* out, float* lse, int32_t* sel, void* ws,
+        size_t ws_bytes, void* stream_v) {
+    g_last_launches = 0;
+    Shape s;
+    int rc = make_shape(p, is_decode, &s);
+    if (rc != HILS_OK) return rc;
+    if (!q || !k || !v || !lm || !out || !lse || !sel || (is_decode && !seq_lens)) return HILS_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(lm) || !aligned16(out) ||
+        (reinterpret_cast<uintptr_t>(lse) & 3u) || (reinterpret_cast<uintptr_t>(sel) & 3u) ||
+        (bias && (reinterpret_cast<uintptr_t>(bias) & 3u)))
+        return HILS_ERR_ALIGNMENT;
+    Path path;
+    rc = pick_path(s, p, &path);
+    if (rc != HILS_OK) return rc;
+    const size_t need = kStatusBytes + scratch_bytes(s, path);
+    if (!ws || ws_bytes < need) return HILS_ERR_WORKSPACE;
+    if (!aligned16(ws)) return HILS_ERR_ALIGNMENT;
+    Tensors t{q, k, v, lm, bias, seq_lens, out, lse, sel, static_cast<int*>(ws),
+              static_cast<char*>(ws) + kStatusBytes, ws_bytes - kStatusBytes};
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    int n;
+    switch (path) {
+        case Path::DecodeFast: n = launch_decode_fast(s, t, stream); break;
+        case Path::PrefillFast: n = launch_prefill_fast(s, t, stream); break;
+        default: n = launch_generic(s, p->dtype, t, stream); break;
+    }
+    if (n < 0) return n;
+    g_last_launches = n;
+    return HILS_OK;
+}
+
+struct ArenaLayout {
+    size_t q, k, v, lm, bias, seq, out, lse, sel, ws, total;
+    size_t q_b, kv_b, lm_b, bias_b, seq_b, out_b, lse_b, sel_b, ws_b;
+};
+
+int arena_layout(const hils_params* p, int is_decode, ArenaLayout* a) {
+    Shape s;
+    int rc = make_shape(p, is_decode, &s);
+    if (rc != HILS_OK) return rc;
+    const size_t eb = elem_bytes(p->dtype);
+    const size_t rows = static_cast<size_t>(s.B) * s.Hq * s.R;
+    a->q_b = rows * s.d * eb;
+    a->kv_b = static_cast<size_t>(s.B) * s.Hkv * s.T * s.d * eb;
+    a->lm_b = static_cast<size_t>(s.B) * s.Hl * s.C * s.d * eb;
+    a->bias_b = static_cast<size_t>(s.B) * s.Hl * s.C * 4;
+    a->seq_b = static_cast<size_t>(s.B) * 4;
+    a->out_b = a->q_b;
+    a->lse_b = rows * 4;
+    a->sel_b = static_cast<size_t>(s.B) * s.Hkv * s.R * s.K * 4;
+    a->ws_b = hils_workspace_bytes(p, is_decode);
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    a->ws = take(a->ws_b);        // first, so that the arena's head is the status word
+    a->q = take(a->q_b); a->k = take(a->kv_b); a->v = take(a->kv_b); a->lm = take(a->lm_b);
+    a->bias = take(a->bias_b); a->seq = take(a->seq_b); a->out = take(a->out_b);
+    a->lse = take(a->lse_b); a->sel = take(a->sel_b);
+    a->total = off;
+    return HILS_OK;
+}
+
+int run_host(const hils_params* p, int is_decode, const void* q, const void* k, const void* v, const void* lm,
+             const float* bias, const int32_t* seq_lens, void* out, float* lse, int32_t* sel, void* arena,
+             size_t arena_bytes, void* stream_v) {
+    ArenaLayout a;
+    int rc = arena_layout(p, is_decode, &a);
+    if (rc != HILS_OK) return rc;
+    if (!q || !k || !v || !lm || !out || !lse || !sel || (is_decode && !seq_lens)) return HILS_ERR_INVALID_ARG;
+    if (!arena || arena_bytes < a.total) return HILS_ERR_WORKSPACE;
+    if (reinterpret_cast<uintptr_t>(arena) & 255u) return HILS_ERR_ALIGNMENT;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    char* base = static_cast<char*>(arena);
+    bool ok = true;
+    ok &= cudaMemcpyAsync(base + a.q, q, a.q_b, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    ok &= cudaMemcpyAsync(base + a.k, k, a.kv_b, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    ok &= cudaMemcpyAsync(base + a.v, v, a.kv_b, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    ok &= cudaMemcpyAsync(base + a.lm, lm, a.lm_b, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    if (bias) ok &= cudaMemcpyAsync(base + a.bias, bias, a.bias_b, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    if (is_decode)
+        ok &= cudaMemcpyAsync(base + a.seq, seq_lens, a.seq_b, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    if (!ok) return HILS_ERR_CUDA;
+    rc = run(p, is_decode, base + a.q, base + a.k, base + a.v, base + a.lm,
+             bias ? reinterpret_cast<const float*>(base + a.bias) : nullptr,
+             is_decode ? reinterpret_cast<const int32_t*>(base + a.seq) : nullptr, base + a.out,
+             reinterpret_cast<float*>(base + a.lse), reinterpret_cast<int32_t*>(base + a.sel), base + a.ws,
+             a.ws_b, stream_v);
+    if (rc != HILS_OK) return rc;
+    ok &= cudaMemcpyAsync(out, base + a.out, a.out_b, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    ok &= cudaMemcpyAsync(lse, base + a.lse, a.lse_b, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    ok &= cudaMemcpyAsync(sel, base + a.sel, a.sel_b, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    return ok ? HILS_OK : HILS_ERR_CUDA;
+}
+
+}  // namespace
+}  // namespace hils
+
+using namespace hils;
+
+extern "C" {
+
+size_t hils_workspace_bytes(const hils_params* params, int is_decode) {
+    Shape s;
+    if (make_shape(params, is_decode, &s) != HILS_OK) return 0;
+    Path path;
+    if (pick_path(s, params, &path) != HILS_OK) return 0;
+    return kStatusBytes + align_up(scratch_bytes(s, path), 256);
+}
+
+int hils_prefill(const hils_params* params, const void* q, const void* k, const void* v, const void* landmarks,
+                 const float* bias, void* out, float* lse, int32_t* sel_idx, void* workspace,
+                 size_t workspace_bytes, void* stream) {
+    return run(params, 0, q, k, v, landmarks, bias, nullptr, out, lse, sel_idx, workspace, workspace_bytes, stream);
+}
+
+int hils_decode(const hils_params* params, const void* q, const void* k_cache, const void* v_cache,
+                const void* landmarks, const float* bias, const int32_t* seq_lens, void* out, float* lse,
+                int32_t* sel_idx, void* workspace, size_t workspace_bytes, void* stream) {
+    return run(params, 1, q, k_cache, v_cache, landmarks, bias, seq_lens, out, lse, sel_idx, workspace,
+               workspace_bytes, stream);
+}
+
+size_t hils_host_arena_bytes(const hils_params* params, int is_decode) {
+    ArenaLayout a;
+    if (arena_layout(params, is_decode, &a) != HILS_OK || a.ws_b == 0) return 0;
+    return a.total;
+}
+
+int hils_prefill_host(const hils_params* params, const void* q_host, const void* k_host, const void* v_host,
+                      const void* landmarks_host, const float* bias_host, void* out_host, float* lse_host,
+                      int32_t* sel_idx_host, void* device_arena, size_t arena_bytes, void* stream) {
+    return run_host(params, 0, q_host, k_host, v_host, landmarks_host, bias_host, nullptr, out_host, lse_host,
+                    sel_idx_host, device_arena, arena_bytes, stream);
+}
+
+int hils_decode_host(const hils_params* params, const void* q_host, const void* k_cache_host,
+                     const void* v_cache_host, const void* landmarks_host, const float* bias_host,
+                     const int32_t* seq_lens_host, void* out_host, float* lse_host, int32_t* sel_idx_host,
+                     void* device_arena, size_t arena_bytes, void* stream) {
+    return run_host(params, 1, q_host, k_cache_host, v_cache_host, landmarks_host, bias_host, seq_lens_host,
+                    out_host, lse_host, sel_idx_host, device_arena, arena_bytes, stream);
+}
+
+int hils_poll_status(const void* workspace, void* stream) {
+    if (!workspace) return HILS_ERR_INVALID_ARG;
+    int word = 0;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(&word, workspace, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) return HILS_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return HILS_ERR_CUDA;
+    if (word == 0) return HILS_OK;
+    if (word == kDevTimeout) return HILS_ERR_DEVICE_TIMEOUT;
+    if (word == kDevBadIndex) return HILS_ERR_DEVICE_INDEX;
+    return HILS_ERR_CUDA;
+}
+
+int hils_last_launch_count(void) { return g_last_launches; }
+
+const char* hils_status_string(int status) {
+    switch (status) {
+        case HILS_OK: return "ok";
+        case HILS_ERR_INVALID_ARG: return "invalid argument";
+        case HILS_ERR_UNSUPPORTED: return "unsupported shape or option";
+        case HILS_ERR_ALIGNMENT: return "pointer not sufficiently aligned";
+        case HILS_ERR_WORKSPACE: return "workspace missing or too small";
+        case HILS_ERR_CUDA: return "CUDA runtime error";
+        case HILS_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+        case HILS_ERR_DEVICE_INDEX: return "device-side index out of range";
+        default: return "unknown status";
+    }
+}
+
+const char* hils_version(void) { return "0.1"; }
+
+}  // extern "C"

@@ -1,0 +1,39 @@
+// Host-side launch functions shared between the translation units of the library.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "common.cuh"
+
+namespace hils {
+
+struct Tensors {
+    const void* q;
+    const void* k;
+    const void* v;
+    const void* landmarks;
+    const float* bias;
+    const int32_t* seq_lens;   // decode only
+    void* out;
+    float* lse;
+    int32_t* sel_idx;
+    int* status;               // device status word
+    void* scratch;             // workspace past the status block
+    size_t scratch_bytes;
+};
+
+// Each launcher returns the number of kernels it enqueued, or a negative hils_status.
+int launch_generic(const Shape& s, int dtype, const Tensors& t, cudaStream_t stream);
+bool generic_supports(const Shape& s);
+
+int launch_decode_fast(const Shape& s, const Tensors& t, cudaStream_t stream);
+bool decode_fast_supports(const Shape& s, int dtype);
+size_t decode_fast_scratch_bytes(const Shape& s);
+
+int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream);
+bool prefill_fast_supports(const Shape& s, int dtype);
+size_t prefill_fast_scratch_bytes(const Shape& s);
+
+}  // namespace hils

@@ -1,0 +1,179 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle, element by element on
+seeded inputs.  Small cases span several tiles and ragged tails; the full-size configurations are
+checked on sampled rows / sequences in the launch configuration the benchmark times."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2607_02980_b200 as hils
+from paper_2607_02980_b200 import workloads as wl
+from parity import check_decode, check_prefill
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def to_dev(d):
+    return {k: v.to(DEV) for k, v in d.items()}
+
+
+def run_prefill(cfg, inp, impl, bias=None, W=1):
+    g = to_dev(inp)
+    out, lse, sel = hils.hils_prefill(g["q"], g["k"], g["v"], g["landmarks"], cfg.S, cfg.K,
+                                      bias=None if bias is None else bias.to(DEV), window=W, impl=impl)
+    torch.cuda.synchronize()
+    return out, lse, sel
+
+
+def run_decode(cfg, inp, impl, bias=None, W=1):
+    g = to_dev(inp)
+    ws_out = hils.hils_decode(g["q"], g["k"], g["v"], g["landmarks"], g["seq_lens"], cfg.S, cfg.K,
+                              bias=None if bias is None else bias.to(DEV), window=W, impl=impl)
+    torch.cuda.synchronize()
+    return ws_out
+
+
+def fast_or_skip(cfg, mode_decode, W=1, Hl=None):
+    p = hils.make_params(B=cfg.B, Hq=cfg.Hq, Hkv=cfg.Hkv, Hl=cfg.Hkv if Hl is None else Hl,
+                         L=0 if mode_decode else cfg.L, T_max=cfg.L, C=cfg.C, d=cfg.d, chunk_size=cfg.S,
+                         top_k=cfg.K, window=W, dtype=0 if cfg.dtype == "f32" else 1, impl="fast")
+    if hils.workspace_bytes(p, mode_decode) == 0:
+        pytest.skip("no fast kernel set for this shape")
+
+
+PREFILL_SMALL = {
+    "cfg0_tiny_f32": wl.CONFIGS[0],
+    "gqa_bf16_2k": wl.CONFIGS[1].scaled(L=2048),
+    "gqa_bf16_ragged_b2": wl.CONFIGS[1].scaled(B=2, Hq=8, Hkv=2, L=1000, K=8, seed=21),
+    "bf16_k_ge_chunks": wl.CONFIGS[1].scaled(Hq=8, Hkv=2, L=640, K=64, seed=22),
+    "bf16_d64_g2_s32": wl.CONFIGS[1].scaled(Hq=4, Hkv=2, L=777, d=64, S=32, K=5, seed=23),
+    "f32_g4_k33": wl.CONFIGS[0].scaled(Hq=4, Hkv=1, L=2500, d=128, K=33, seed=24, n_needles=2),
+}
+
+
+@pytest.mark.parametrize("impl", ["generic", "fast"])
+@pytest.mark.parametrize("name", list(PREFILL_SMALL))
+def test_prefill_small(name, impl):
+    cfg = PREFILL_SMALL[name]
+    if impl == "fast":
+        fast_or_skip(cfg, False)
+    inp = wl.make_prefill_inputs(cfg, "cpu")
+    out, lse, sel = run_prefill(cfg, inp, impl)
+    stats = check_prefill(cfg, inp, out, lse, sel)
+    print(name, impl, stats)
+
+
+@pytest.mark.parametrize("impl", ["generic", "fast"])
+def test_prefill_window_bias_and_per_head_landmarks(impl):
+    """General local window W, entropy-like bias, and one landmark per query head (App. C)."""
+    cfg = wl.CONFIGS[0].scaled(Hq=4, Hkv=2, L=600, d=32, S=16, K=5, seed=31)
+    if impl == "fast":
+        fast_or_skip(cfg, False, W=100, Hl=cfg.Hq)
+    inp = wl.make_prefill_inputs(cfg, "cpu")
+    g = torch.Generator().manual_seed(5)
+    inp["landmarks"] = torch.randn((1, cfg.Hq, cfg.C, cfg.d), generator=g) * 0.5
+    bias = torch.rand((1, cfg.Hq, cfg.C), generator=g) * float(np.log(cfg.S))
+    out, lse, sel = run_prefill(cfg, inp, impl, bias=bias, W=100)
+    check_prefill(cfg, inp, out, lse, sel, bias=bias, W=100)
+
+
+@pytest.mark.parametrize("impl", ["generic", "fast"])
+def test_prefill_bias_only(impl):
+    cfg = wl.CONFIGS[1].scaled(L=1536, K=6, seed=32)
+    if impl == "fast":
+        fast_or_skip(cfg, False)
+    inp = wl.make_prefill_inputs(cfg, "cpu")
+    bias = wl.make_bias(cfg, "cpu")
+    out, lse, sel = run_prefill(cfg, inp, impl, bias=bias)
+    check_prefill(cfg, inp, out, lse, sel, bias=bias)
+
+
+def test_prefill_ties_go_to_lower_chunk_and_runs_are_deterministic():
+    cfg = wl.CONFIGS[1].scaled(Hq=8, Hkv=2, L=1024, K=3, seed=33, n_needles=0)
+    inp = wl.make_prefill_inputs(cfg, "cpu")
+    inp["q"].zero_()                                   # every score equals 0: ties everywhere
+    for impl in ("generic", "auto"):
+        out, lse, sel = run_prefill(cfg, inp, impl)
+        s = sel.cpu().numpy()
+        for i in (64 * 3, 64 * 7 + 5, 1023):
+            assert (s[0, :, i] == np.array([0, 1, 2])).all()
+        out2, lse2, sel2 = run_prefill(cfg, inp, impl)
+        assert torch.equal(sel, sel2)
+    inp = wl.make_prefill_inputs(cfg.scaled(n_needles=2), "cpu")
+    a = run_prefill(cfg, inp, "auto")
+    b = run_prefill(cfg, inp, "auto")
+    assert torch.equal(a[2], b[2])
+    assert (a[0].float() - b[0].float()).abs().max() <= 1e-2
+
+
+DECODE_SMALL = {
+    "bf16_ragged": (wl.CONFIGS[3].scaled(B=6, L=4096, K=8, seed=41), [4096, 4095, 1, 63, 2049, 640]),
+    "bf16_k_ge_chunks": (wl.CONFIGS[3].scaled(B=3, L=2048, K=64, seed=42), [2048, 1000, 65]),
+    "bf16_cfg4_like": (wl.CONFIGS[4].scaled(B=2, L=32768, K=64, seed=43), [32768, 32700]),
+    "f32_g1_d64": (wl.CONFIGS[0].scaled(mode="decode", B=4, L=1024, K=4, seed=44), [1024, 1, 64, 500]),
+}
+
+
+@pytest.mark.parametrize("impl", ["generic", "fast"])
+@pytest.mark.parametrize("name", list(DECODE_SMALL))
+def test_decode_small(name, impl):
+    cfg, seq = DECODE_SMALL[name]
+    if impl == "fast":
+        fast_or_skip(cfg, True)
+    inp = wl.make_decode_inputs(cfg, "cpu", seq_lens=torch.tensor(seq, dtype=torch.int32))
+    out, lse, sel = run_decode(cfg, inp, impl)
+    stats = check_decode(cfg, inp, out, lse, sel)
+    print(name, impl, stats)
+
+
+@pytest.mark.parametrize("impl", ["generic", "fast"])
+def test_decode_with_bias(impl):
+    cfg = wl.CONFIGS[3].scaled(B=3, L=8192, K=16, seed=45)
+    if impl == "fast":
+        fast_or_skip(cfg, True)
+    inp = wl.make_decode_inputs(cfg, "cpu", seq_lens=torch.tensor([8192, 8000, 4097], dtype=torch.int32))
+    bias = wl.make_bias(cfg, "cpu")
+    out, lse, sel = run_decode(cfg, inp, impl, bias=bias)
+    check_decode(cfg, inp, out, lse, sel, bias=bias)
+
+
+def test_decode_invalid_seq_len_sets_status_without_fault():
+    cfg = wl.CONFIGS[3].scaled(B=2, L=1024, K=4, seed=46)
+    inp = wl.make_decode_inputs(cfg, "cpu", seq_lens=torch.tensor([1024, 512], dtype=torch.int32))
+    g = to_dev(inp)
+    g["seq_lens"] = torch.tensor([1024, 0], dtype=torch.int32, device=DEV)
+    p = hils.make_params(B=2, Hq=cfg.Hq, Hkv=cfg.Hkv, Hl=cfg.Hkv, L=0, T_max=cfg.L, C=cfg.C, d=cfg.d,
+                         chunk_size=cfg.S, top_k=cfg.K, dtype=1, impl="auto")
+    ws = hils.alloc_workspace(p, True, DEV)
+    out, lse, sel = hils.hils_decode(g["q"], g["k"], g["v"], g["landmarks"], g["seq_lens"], cfg.S, cfg.K, workspace=ws)
+    assert hils.poll_status(ws) == -7
+    assert (sel[1] == -1).all()
+    ws[:256].zero_()
+    g["seq_lens"][1] = 512
+    hils.hils_decode(g["q"], g["k"], g["v"], g["landmarks"], g["seq_lens"], cfg.S, cfg.K, workspace=ws)
+    assert hils.poll_status(ws) == 0
+
+
+def test_host_entry_points_match_device_entry_points():
+    cfg = wl.CONFIGS[1].scaled(L=1024, K=4, seed=47)
+    inp = wl.make_prefill_inputs(cfg, "cpu")
+    out, lse, sel = run_prefill(cfg, inp, "auto")
+    p = hils.make_params(B=cfg.B, Hq=cfg.Hq, Hkv=cfg.Hkv, Hl=cfg.Hkv, L=cfg.L, T_max=cfg.L, C=cfg.C, d=cfg.d,
+                         chunk_size=cfg.S, top_k=cfg.K, dtype=1, impl="auto")
+    runner = hils.HostRunner(p, False, DEV)
+    pinned = {k: v.pin_memory() for k, v in inp.items()}
+    ho, hl, hs = runner.run(pinned["q"], pinned["k"], pinned["v"], pinned["landmarks"])
+    torch.cuda.synchronize()
+    assert torch.equal(hs, sel.cpu())
+    assert (ho.float() - out.cpu().float()).abs().max() <= 1e-2
+    dcfg = wl.CONFIGS[3].scaled(B=2, L=2048, K=4, seed=48)
+    dinp = wl.make_decode_inputs(dcfg, "cpu", seq_lens=torch.tensor([2048, 777], dtype=torch.int32))
+    o, l, s = run_decode(dcfg, dinp, "auto")
+    dp = hils.make_params(B=2, Hq=dcfg.Hq, Hkv=dcfg.Hkv, Hl=dcfg.Hkv, L=0, T_max=dcfg.L, C=dcfg.C, d=dcfg.d,
+                          chunk_size=dcfg.S, top_k=dcfg.K, dtype=1, impl="auto")
+    r2 = hils.HostRunner(dp, True, DEV)
+    pd = {k: v.pin_memory() for k, v in dinp.items()}
+    ho, hl, hs = r2.run(pd["q"], pd["k"], pd["v"], pd["landmarks"], seq_lens=pd["seq_lens"])
+    torch.cuda.synchronize()
+    assert torch.equal(hs, s.cpu())
+    assert (ho.float() - o.cpu().float()).abs().max() <= 1e-2
