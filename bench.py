@@ -1,0 +1,454 @@
+#!/usr/bin/env python
+"""HiLS attention benchmark: one JSON line per run.
+
+A "step" is one pass of the whole hot path (landmark scoring, group max, top-K selection, local
+attention, per-chunk attention, fusion) over one batch of seeded synthetic input, through the C ABI.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg1|cfg0|cfg2|cfg3|cfg4]
+                  [--impl ours|reference] [--extra]
+
+Prefill workloads report effective TFLOP/s on the gathered FLOP (what the method must do, not what
+dense attention would); decode workloads report GB/s on the algorithmic bytes (landmarks scanned +
+selected K/V chunks).  With N > 1 every rank runs an independent replica of the workload (the path
+shards over batch / KV groups with no exchange), and `value` is the sum over ranks divided by the
+slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2607_02980_b200 import workloads as wl
+
+# dram bytes per launch of the dominant kernel from ncu captures (see profiles/); None = not captured
+NCU_TRAFFIC_BYTES = {}
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["_source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["_source"] = "fallback"
+    return p
+
+
+# ----------------------------------------------------------------------------- algorithmic work
+def prefill_flops(cfg):
+    """(gathered FLOP, scoring FLOP) of one prefill call with W = 1."""
+    i = np.arange(cfg.L, dtype=np.float64)
+    ci = np.floor(i / cfg.S)
+    gathered = 4.0 * cfg.d * (np.minimum(cfg.K, ci) * cfg.S + (i % cfg.S) + 1)
+    scoring = 2.0 * cfg.d * ci
+    return float(gathered.sum()) * cfg.Hq * cfg.B, float(scoring.sum()) * cfg.Hq * cfg.B
+
+
+def prefill_flops_rows(cfg, rows):
+    i = np.asarray(rows, dtype=np.float64)
+    ci = np.floor(i / cfg.S)
+    return float((4.0 * cfg.d * (np.minimum(cfg.K, ci) * cfg.S + (i % cfg.S) + 1)).sum()) * cfg.Hq * cfg.B
+
+
+def decode_bytes(cfg, seq_lens):
+    """(landmark bytes scanned, gathered K/V bytes) of one decode call, bf16/fp32 element size."""
+    eb = 4 if cfg.dtype == "f32" else 2
+    seq = np.asarray(seq_lens, dtype=np.int64)
+    ncand = (seq - 1) // cfg.S
+    local = (seq - 1) % cfg.S + 1
+    lm = float(ncand.sum()) * cfg.Hkv * cfg.d * eb
+    kv = float((np.minimum(cfg.K, ncand) * cfg.S + local).sum()) * cfg.Hkv * cfg.d * eb * 2
+    return lm, kv
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu, self.rows, self.proc, self.thread = gpu_index, [], None, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.QUERY, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        def pump():
+            for line in self.proc.stdout:
+                self.rows.append([x.strip() for x in line.split(",")])
+        self.thread = threading.Thread(target=pump, daemon=True)
+        self.thread.start()
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for r in self.rows:
+            if len(r) < 9:
+                continue
+            try:
+                sm.append(float(r[1])); mx.append(float(r[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------- workloads
+def pick_cfg(name):
+    idx = {"cfg0": 0, "cfg1": 1, "cfg2": 2, "cfg3": 3, "cfg4": 4}[name]
+    return wl.CONFIGS[idx]
+
+
+def params_for(hils, cfg, decode, impl="auto"):
+    return hils.make_params(B=cfg.B, Hq=cfg.Hq, Hkv=cfg.Hkv, Hl=cfg.Hkv, L=0 if decode else cfg.L, T_max=cfg.L,
+                            C=cfg.C, d=cfg.d, chunk_size=cfg.S, top_k=cfg.K, window=1,
+                            dtype=0 if cfg.dtype == "f32" else 1, impl=impl)
+
+
+class Workload:
+    """Device-resident inputs/outputs of one configuration and the call that runs one step."""
+
+    def __init__(self, hils, cfg, device, n_query_sets=8):
+        self.hils, self.cfg, self.dev = hils, cfg, device
+        self.decode = cfg.mode == "decode"
+        self.p = params_for(hils, cfg, self.decode)
+        self.ws = hils.alloc_workspace(self.p, self.decode, device)
+        if self.decode:
+            self.inp = wl.make_decode_inputs(cfg, device)
+            # distinct query sets (different selected chunks) so that gathered chunks are not L2 hits
+            self.queries = [self.inp["q"]] + [
+                wl.make_decode_queries(cfg, self.inp["landmarks"], self.inp["seq_lens"], s)
+                for s in range(1, n_query_sets)]
+            self.out = torch.empty_like(self.inp["q"])
+            self.lse = torch.empty((cfg.B, cfg.Hq), dtype=torch.float32, device=device)
+            self.sel = torch.empty((cfg.B, cfg.Hkv, cfg.K), dtype=torch.int32, device=device)
+            lm_b, kv_b = decode_bytes(cfg, self.inp["seq_lens"].cpu().numpy())
+            self.work, self.work_aux = lm_b + kv_b, kv_b
+            self.unit, self.metric = "GB/s", "hils_decode_algorithmic_GBps"
+        else:
+            self.inp = wl.make_prefill_inputs(cfg, device)
+            self.out = torch.empty_like(self.inp["q"])
+            self.lse = torch.empty((cfg.B, cfg.Hq, cfg.L), dtype=torch.float32, device=device)
+            self.sel = torch.empty((cfg.B, cfg.Hkv, cfg.L, cfg.K), dtype=torch.int32, device=device)
+            self.work, self.work_aux = prefill_flops(cfg)
+            self.unit, self.metric = "TFLOP/s", "hils_prefill_effective_TFLOPs"
+        self.flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=device) if self.decode else None
+        self.step_no = 0
+
+    def step(self):
+        i = self.inp
+        if self.decode:
+            q = self.queries[self.step_no % len(self.queries)]
+            self.step_no += 1
+            self.hils.hils_decode(q, i["k"], i["v"], i["landmarks"], i["seq_lens"], self.cfg.S, self.cfg.K,
+                                  out=self.out, lse=self.lse, sel_idx=self.sel, workspace=self.ws)
+        else:
+            self.hils.hils_prefill(i["q"], i["k"], i["v"], i["landmarks"], self.cfg.S, self.cfg.K,
+                                   out=self.out, lse=self.lse, sel_idx=self.sel, workspace=self.ws)
+
+    def between_steps(self):
+        if self.flush is not None:
+            self.flush.fill_(1)                  # 256 MB write: evicts the 126 MB L2
+
+    def rate(self, seconds_per_step, n_replicas=1):
+        scale = 1e12 if self.unit == "TFLOP/s" else 1e9
+        return self.work * n_replicas / seconds_per_step / scale
+
+
+def time_steps(w, steps, warmup, barrier):
+    """K steps timed with CUDA events on the launching stream; flushes sit outside the event pairs."""
+    for _ in range(warmup):
+        w.between_steps()
+        w.step()
+    torch.cuda.synchronize()
+    barrier()
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    traces = []
+    for s in range(steps):
+        w.between_steps()
+        starts[s].record()
+        w.step()
+        ends[s].record()
+        tr = w.hils.trace_read()
+        if tr:
+            traces.append(tr)
+    torch.cuda.synchronize()
+    barrier()
+    ms = [starts[s].elapsed_time(ends[s]) for s in range(steps)]
+    return ms, traces
+
+
+def summarise_traces(traces):
+    agg = {}
+    for tr in traces:
+        for name, ms in tr:
+            agg.setdefault(name, []).append(ms)
+    return {k: float(np.mean(v)) for k, v in agg.items()}
+
+
+def roofline_for(w, kernel_ms, peaks):
+    """Roofline entry of the dominant kernel of one step."""
+    if not kernel_ms:
+        return None
+    name = max(kernel_ms, key=kernel_ms.get)
+    sec = kernel_ms[name] * 1e-3
+    src = "of measured" if peaks["_source"] == "measured" else "of fallback"
+    if w.decode:
+        lm_b, kv_b = decode_bytes(w.cfg, w.inp["seq_lens"].cpu().numpy())
+        algo = kv_b if "attend" in name else (lm_b if ("score" in name or "select" in name) else lm_b + kv_b)
+        ach = algo / sec / 1e9
+        return {"kernel": name, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": ach / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get((w.cfg.name, name)),
+                "algorithmic_bytes": algo, "kernel_ms": kernel_ms[name], "peak_source": src}
+    gathered, scoring = prefill_flops(w.cfg)
+    algo = scoring if ("score" in name or "select" in name) else gathered
+    if w.cfg.dtype == "f32":
+        # fp32 path on plain FMA units: 148 SMs x 128 lanes x 2 FLOP x max SM clock
+        peak = 148 * 128 * 2 * peaks.get("sm_max_mhz", 1965.0) * 1e6 / 1e12
+        bound = "alu"
+    else:
+        peak = peaks["bf16_tflops"]
+        bound = "tensor"
+    ach = algo / sec / 1e12
+    return {"kernel": name, "bound": bound, "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak,
+            "traffic": NCU_TRAFFIC_BYTES.get((w.cfg.name, name)), "algorithmic_flops": algo,
+            "kernel_ms": kernel_ms[name], "peak_source": src}
+
+
+# ----------------------------------------------------------------------------- CPU oracle legs
+def oracle_sample(cfg, inp_cpu, budget_rows):
+    """Times the oracle, as it stands, on a bounded sample of the workload.  Returns (value, sample, secs)."""
+    import oracle
+    if cfg.mode == "prefill":
+        rows = wl.sample_rows(cfg, budget_rows).numpy()
+        t0 = time.perf_counter()
+        oracle.hils_prefill(inp_cpu["q"], inp_cpu["k"], inp_cpu["v"], inp_cpu["landmarks"], None, S=cfg.S, K=cfg.K,
+                            rows=rows)
+        dt = time.perf_counter() - t0
+        val = prefill_flops_rows(cfg, rows) / dt / 1e12
+        return val, "%d seeded query positions x all %d heads of %s" % (len(rows), cfg.Hq, cfg.name), dt
+    nb = min(cfg.B, budget_rows)
+    sub = {k: v[:nb] for k, v in inp_cpu.items()}
+    t0 = time.perf_counter()
+    oracle.hils_decode(sub["q"], sub["k"], sub["v"], sub["landmarks"], None, sub["seq_lens"], S=cfg.S, K=cfg.K)
+    dt = time.perf_counter() - t0
+    lm_b, kv_b = decode_bytes(cfg, sub["seq_lens"].numpy())
+    return (lm_b + kv_b) / dt / 1e9, "first %d of %d sequences of %s" % (nb, cfg.B, cfg.name), dt
+
+
+def reference_cfg_inputs(cfg):
+    """Host inputs for the oracle legs.  Large decode caches are cut to the first sequences."""
+    if cfg.mode == "decode":
+        small = cfg.scaled(B=min(cfg.B, 2))
+        return small, wl.make_decode_inputs(small, "cpu")
+    return cfg, wl.make_prefill_inputs(cfg, "cpu")
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    cfg = pick_cfg(args.workload)
+    small, inp = reference_cfg_inputs(cfg)
+    budget = 512 if cfg.mode == "prefill" else 2
+    vals, secs, sample = [], [], ""
+    for s in range(args.warmup + args.steps):
+        v, sample, dt = oracle_sample(small, inp, budget)
+        if s >= args.warmup:
+            vals.append(v); secs.append(dt)
+    value = float(np.mean(vals))
+    unit = "TFLOP/s" if cfg.mode == "prefill" else "GB/s"
+    line = {"impl": "reference", "metric": "hils_prefill_effective_TFLOPs" if cfg.mode == "prefill"
+            else "hils_decode_algorithmic_GBps", "value": value, "unit": unit, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": float(np.mean(secs)) * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg.name, "note": "each step = the CPU oracle on a bounded sample"},
+            "cpu_baseline": {"value": value, "unit": unit, "cores": oracle.num_threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------- main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="cfg1", choices=["cfg0", "cfg1", "cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--extra", action="store_true", help="also time the other single-GPU configurations")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import paper_2607_02980_b200 as hils
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x):
+        if dist is None:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    peaks = load_peaks()
+    cfg = pick_cfg(args.workload)
+    hils.load_library()
+    hils.trace_enable(True)
+    w = Workload(hils, cfg, dev)
+    sampler = ClockSampler(local)
+    sampler.start()
+    ms, traces = time_steps(w, args.steps, args.warmup, barrier)
+    clocks = sampler.stop()
+    launches = hils.last_launch_count() * args.steps
+    ms_step = max_over_ranks(float(np.sum(ms)) / args.steps)
+    value = w.rate(ms_step * 1e-3, world)
+    kernel_ms = summarise_traces(traces)
+
+    line = {"metric": w.metric, "value": value, "unit": w.unit, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
+            "config": {"workload": cfg.name, "B": cfg.B, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "L_or_T": cfg.L, "d": cfg.d,
+                       "chunk_size": cfg.S, "top_k": cfg.K, "window": 1, "parallelism": "replicas x%d" % world,
+                       "l2_policy": ("256 MB flush write + rotating query sets between steps" if w.decode else
+                                     "inputs+outputs %.0f MB > 126 MB L2" % (
+                                         sum(t.numel() * t.element_size() for t in list(w.inp.values()) + [w.out]) / 1e6)),
+                       "median_ms": float(np.median(ms)), "min_ms": float(np.min(ms))},
+            "clocks": clocks, "gpu_launches": launches, "kernel_ms": kernel_ms}
+    if w.decode:
+        line["decode_gathered_kv_GBps"] = None
+        for name, kms in kernel_ms.items():
+            if "attend" in name:
+                line["decode_gathered_kv_GBps"] = w.work_aux / (kms * 1e-3) / 1e9
+    else:
+        line["scoring_flops"] = w.work_aux
+        line["frac_of_nominal_2250_TFLOPs"] = value / world / 2250.0
+    roof = roofline_for(w, kernel_ms, peaks)
+    if roof:
+        line["roofline"] = roof
+
+    # ---- end to end: host buffers through the *_host entry points, copies inside the timed region
+    if not args.no_e2e:
+        hils.trace_enable(False)
+        runner = hils.HostRunner(w.p, w.decode, dev)
+        host = {k: v.cpu().pin_memory() for k, v in w.inp.items()}
+        h2d, d2h = runner.bytes_per_step({k: host[k] for k in host})
+        def e2e_step():
+            runner.run(host["q"], host["k"], host["v"], host["landmarks"], seq_lens=host.get("seq_lens"))
+        for _ in range(2):
+            e2e_step()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n_e2e = max(3, min(args.steps, 10))
+        e0.record()
+        for _ in range(n_e2e):
+            e2e_step()
+        e1.record()
+        barrier()
+        e2e_ms = max_over_ranks(e0.elapsed_time(e1) / n_e2e)
+        line["e2e"] = {"value": w.rate(e2e_ms * 1e-3, world), "unit": w.unit, "ms_per_step": e2e_ms,
+                       "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+        launches += hils.last_launch_count() * (n_e2e + 2)
+        del runner, host
+        hils.trace_enable(True)
+
+    # ---- other configurations (reported beside, never instead of, the primary workload)
+    if args.extra and world == 1:
+        extras = {}
+        del w
+        torch.cuda.empty_cache()
+        for name in ("cfg2", "cfg3", "cfg4", "cfg0"):
+            if name == args.workload:
+                continue
+            try:
+                ew = Workload(hils, pick_cfg(name), dev)
+                ems, etr = time_steps(ew, max(3, args.steps), 3, barrier)
+                ek = summarise_traces(etr)
+                ent = {"metric": ew.metric, "value": ew.rate(float(np.mean(ems)) * 1e-3), "unit": ew.unit,
+                       "ms_per_step": float(np.mean(ems)), "median_ms": float(np.median(ems)), "kernel_ms": ek,
+                       "roofline": roofline_for(ew, ek, peaks)}
+                if ew.decode:
+                    ent["frac_of_measured_hbm"] = ent["value"] / peaks["hbm_gbs"]
+                    ent["frac_of_nominal_8000_GBps"] = ent["value"] / 8000.0
+                else:
+                    ent["frac_of_measured_bf16_burst"] = ent["value"] / peaks["bf16_tflops"]
+                    ent["frac_of_nominal_2250_TFLOPs"] = ent["value"] / 2250.0
+                extras[name] = ent
+                launches += hils.last_launch_count() * (max(3, args.steps) + 3)
+                del ew
+                torch.cuda.empty_cache()
+            except Exception as exc:  # keep the primary line even if an extra fails
+                extras[name] = {"error": repr(exc)}
+        line["extra"] = extras
+
+    # ---- the oracle timed beside it on this machine's host cores (rank 0, N = 1 only)
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        small, inp_cpu = reference_cfg_inputs(cfg)
+        val, sample, secs = oracle_sample(small, inp_cpu, 2048 if cfg.mode == "prefill" else 2)
+        line["cpu_baseline"] = {"value": val, "unit": "TFLOP/s" if cfg.mode == "prefill" else "GB/s",
+                                "cores": oracle.num_threads(), "kind": "oracle", "sample": sample, "seconds": secs}
+    line["gpu_launches"] = launches
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -126,6 +126,14 @@ int hils_poll_status(const void* workspace, void* stream);
 /* Number of kernels the last hils_prefill / hils_decode call of this thread enqueued. */
 int hils_last_launch_count(void);
 
+/* Per-kernel timing for profiling (no counterpart in the paper; Sec. 7.1 reports end-to-end latency
+ * only).  hils_trace_enable(1) creates CUDA events once for the calling thread; while on, each
+ * hils_prefill / hils_decode records an event after every kernel it enqueues.  hils_trace_read
+ * waits for the last call's final event and returns the number of kernels n (<= max_kernels),
+ * writing their device times to ms[0..n) and their names, ';'-terminated, to `names`. */
+int hils_trace_enable(int on);
+int hils_trace_read(char* names, size_t names_bytes, float* ms, int max_kernels);
+
 const char* hils_status_string(int status);
 
 /* Library version, "major.minor". */

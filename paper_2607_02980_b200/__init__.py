@@ -5,8 +5,8 @@ The shared library is loaded on first use and there is no fallback when it is mi
 """
 from .binding import (HilsError, HilsParams, HostRunner, alloc_workspace, hils_decode, hils_prefill,
                       host_arena_bytes, last_launch_count, load_library, make_params, poll_status,
-                      status_string, version, workspace_bytes)
+                      status_string, trace_enable, trace_read, version, workspace_bytes)
 
 __all__ = ["HilsError", "HilsParams", "HostRunner", "alloc_workspace", "hils_decode", "hils_prefill",
            "host_arena_bytes", "last_launch_count", "load_library", "make_params", "poll_status",
-           "status_string", "version", "workspace_bytes"]
+           "status_string", "trace_enable", "trace_read", "version", "workspace_bytes"]

@@ -23,7 +23,7 @@ _IMPL = {"auto": IMPL_AUTO, "generic": IMPL_GENERIC, "fast": IMPL_FAST}
 EXPORTS = [
     "hils_workspace_bytes", "hils_prefill", "hils_decode", "hils_host_arena_bytes",
     "hils_prefill_host", "hils_decode_host", "hils_poll_status", "hils_last_launch_count",
-    "hils_status_string", "hils_version",
+    "hils_status_string", "hils_version", "hils_trace_enable", "hils_trace_read",
 ]
 
 
@@ -73,6 +73,10 @@ def load_library() -> ctypes.CDLL:
     lib.hils_status_string.restype = ctypes.c_char_p
     lib.hils_status_string.argtypes = [ctypes.c_int]
     lib.hils_version.restype = ctypes.c_char_p
+    lib.hils_trace_enable.restype = ctypes.c_int
+    lib.hils_trace_enable.argtypes = [ctypes.c_int]
+    lib.hils_trace_read.restype = ctypes.c_int
+    lib.hils_trace_read.argtypes = [ctypes.c_char_p, ctypes.c_size_t, ctypes.POINTER(ctypes.c_float), ctypes.c_int]
     _lib = lib
     return lib
 
@@ -255,6 +259,23 @@ class HostRunner:
         if rc != 0:
             raise HilsError(rc, "hils_decode_host" if self.is_decode else "hils_prefill_host")
         return self.out, self.lse, self.sel
+
+
+def trace_enable(on: bool) -> None:
+    rc = load_library().hils_trace_enable(1 if on else 0)
+    if rc != 0:
+        raise HilsError(rc, "hils_trace_enable")
+
+
+def trace_read():
+    """[(kernel name, device milliseconds)] of the last traced call (waits for it to finish)."""
+    names = ctypes.create_string_buffer(1024)
+    ms = (ctypes.c_float * 16)()
+    n = load_library().hils_trace_read(names, 1024, ms, 16)
+    if n < 0:
+        raise HilsError(n, "hils_trace_read")
+    parts = [x for x in names.value.decode().split(";") if x]
+    return [(parts[i] if i < len(parts) else "?", float(ms[i])) for i in range(n)]
 
 
 def poll_status(workspace: torch.Tensor, stream=None) -> int:

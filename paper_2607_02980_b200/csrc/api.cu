@@ -8,6 +8,34 @@ namespace {
 
 thread_local int g_last_launches = 0;
 
+constexpr int kMaxTrace = 16;
+struct Trace {
+    bool enabled = false;
+    bool have_events = false;
+    cudaEvent_t ev[kMaxTrace + 1];
+    const char* names[kMaxTrace];
+    int n = 0;
+};
+thread_local Trace g_trace;
+
+}  // namespace
+
+void trace_begin(cudaStream_t stream) {
+    Trace& t = g_trace;
+    t.n = 0;
+    if (t.enabled && t.have_events) cudaEventRecord(t.ev[0], stream);
+}
+
+void trace_mark(const char* name, cudaStream_t stream) {
+    Trace& t = g_trace;
+    if (!t.enabled || !t.have_events || t.n >= kMaxTrace) return;
+    t.names[t.n] = name;
+    ++t.n;
+    cudaEventRecord(t.ev[t.n], stream);
+}
+
+namespace {
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline size_t elem_bytes(int dtype) { return dtype == HILS_F32 ? 4 : 2; }
@@ -91,6 +119,7 @@ int run(const hils_params* p, int is_decode, const void* q, const void* k, const
     Tensors t{q, k, v, lm, bias, seq_lens, out, lse, sel, static_cast<int*>(ws),
               static_cast<char*>(ws) + kStatusBytes, ws_bytes - kStatusBytes};
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
+    trace_begin(stream);
     int n;
     switch (path) {
         case Path::DecodeFast: n = launch_decode_fast(s, t, stream); break;
@@ -226,6 +255,41 @@ int hils_poll_status(const void* workspace, void* stream) {
 }
 
 int hils_last_launch_count(void) { return g_last_launches; }
+
+int hils_trace_enable(int on) {
+    Trace& t = g_trace;
+    if (on && !t.have_events) {
+        for (int i = 0; i <= kMaxTrace; ++i)
+            if (cudaEventCreate(&t.ev[i]) != cudaSuccess) return HILS_ERR_CUDA;
+        t.have_events = true;
+    }
+    t.enabled = on != 0;
+    t.n = 0;
+    return HILS_OK;
+}
+
+int hils_trace_read(char* names, size_t names_bytes, float* ms, int max_kernels) {
+    Trace& t = g_trace;
+    if (!t.enabled || !t.have_events) return 0;
+    if (!ms || max_kernels < 0) return HILS_ERR_INVALID_ARG;
+    if (t.n > 0 && cudaEventSynchronize(t.ev[t.n]) != cudaSuccess) return HILS_ERR_CUDA;
+    size_t off = 0;
+    if (names && names_bytes) names[0] = 0;
+    int n = t.n < max_kernels ? t.n : max_kernels;
+    for (int i = 0; i < n; ++i) {
+        if (cudaEventElapsedTime(&ms[i], t.ev[i], t.ev[i + 1]) != cudaSuccess) return HILS_ERR_CUDA;
+        if (names) {
+            const size_t len = strlen(t.names[i]);
+            if (off + len + 2 <= names_bytes) {
+                memcpy(names + off, t.names[i], len);
+                off += len;
+                names[off++] = ';';
+                names[off] = 0;
+            }
+        }
+    }
+    return n;
+}
 
 const char* hils_status_string(int status) {
     switch (status) {

@@ -271,11 +271,13 @@ int launch_typed(const GArgs& a, cudaStream_t stream) {
     else if (nr == 2) generic_select_kernel<T, 2><<<sel_blocks, kWarpsPerBlock * 32, sel_smem, stream>>>(a);
     else generic_select_kernel<T, 4><<<sel_blocks, kWarpsPerBlock * 32, sel_smem, stream>>>(a);
     if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
+    trace_mark("generic_select", stream);
     const int ne = s.d / 32;
     if (ne <= 2) generic_attend_kernel<T, 2><<<att_blocks, kWarpsPerBlock * 32, att_smem, stream>>>(a);
     else if (ne <= 4) generic_attend_kernel<T, 4><<<att_blocks, kWarpsPerBlock * 32, att_smem, stream>>>(a);
     else generic_attend_kernel<T, 8><<<att_blocks, kWarpsPerBlock * 32, att_smem, stream>>>(a);
     if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
+    trace_mark("generic_attend", stream);
     return 2;
 }
 

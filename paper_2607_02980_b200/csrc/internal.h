@@ -24,6 +24,12 @@ struct Tensors {
     size_t scratch_bytes;
 };
 
+// Optional per-kernel timing: when tracing is on (hils_trace_enable), every launcher calls
+// trace_mark(name) after each kernel it enqueues; an event is recorded on the stream so that the
+// time between consecutive marks is that kernel's device time.  Off by default (no events).
+void trace_begin(cudaStream_t stream);
+void trace_mark(const char* name, cudaStream_t stream);
+
 // Each launcher returns the number of kernels it enqueued, or a negative hils_status.
 int launch_generic(const Shape& s, int dtype, const Tensors& t, cudaStream_t stream);
 bool generic_supports(const Shape& s);
