@@ -111,6 +111,9 @@ DECODE_SMALL = {
     "bf16_k_ge_chunks": (wl.CONFIGS[3].scaled(B=3, L=2048, K=64, seed=42), [2048, 1000, 65]),
     "bf16_cfg4_like": (wl.CONFIGS[4].scaled(B=2, L=32768, K=64, seed=43), [32768, 32700]),
     "f32_g1_d64": (wl.CONFIGS[0].scaled(mode="decode", B=4, L=1024, K=4, seed=44), [1024, 1, 64, 500]),
+    # many (sequence, KV head) pairs: every persistent CTA walks several pairs and wraps its TMA ring
+    "bf16_many_pairs": (wl.CONFIGS[3].scaled(B=64, L=2048, K=16, seed=49),
+                        [2048 - 37 * (i % 11) - (1 if i % 3 == 0 else 0) for i in range(64)]),
 }
 
 
