@@ -101,6 +101,35 @@ int hils_decode(const hils_params* params, const void* q, const void* k_cache, c
                 void* out, float* lse, int32_t* sel_idx,
                 void* workspace, size_t workspace_bytes, void* stream);
 
+/* hils_decode for callers that cannot allocate device memory.  (The paper has no counterpart to this
+ * entry point; it exists for integration only.)
+ *
+ * Some hosts of this library have no way to hand it a workspace: an inference server that gave all
+ * free HBM to its own KV-cache pool at start-up, so that a later cudaMalloc fails; a plugin that is
+ * only passed the tensors of one layer and has no allocator handle; a latency-critical loop that
+ * may not call cudaMalloc because it synchronises the device.  For them this call computes exactly
+ * what hils_decode computes (same kernels, same results) but keeps its scratch in a fixed 8 MiB array
+ * that is part of the library image itself; every GPU that loads libhils.so holds that array until
+ * the process exits.  The caller still passes every input and output.
+ *
+ *  - Nothing is allocated or freed, by CUDA or otherwise, on any call.
+ *  - Limit: 256 + hils_workspace_bytes(params, 1) must fit in 8 MiB, otherwise HILS_ERR_WORKSPACE is
+ *    returned before anything is launched (both benchmark decode shapes fit: B=64 x 64K tokens with
+ *    K=32 needs about 5.3 MiB, B=4 x 1M tokens with K=64 about 2.5 MiB).  Shapes outside the
+ *    bandwidth-tuned decode kernels (bf16, d=128, chunk 64, window 1, one landmark per KV head,
+ *    at most 8 query heads per KV head) return HILS_ERR_UNSUPPORTED.
+ *  - The first call on each device looks up the array's device address (with that device current);
+ *    make that first call outside any stream capture.
+ *  - The array is shared by every call in the process and keeps the previous call's contents.  The
+ *    call clears what has to start at zero (the status word; the completion counters are reset by the
+ *    kernels themselves).  Two calls whose kernels overlap on the GPU (different streams, or several
+ *    host threads) race on it: serialise them.
+ *  - device_status (DEVICE pointer, may be NULL) receives the device status word of this call:
+ *    0 = ok, 1 = a bounded wait ran out, 2 = an invalid sequence length was met. */
+int hils_decode_noalloc(const hils_params* params, const void* q, const void* k_cache, const void* v_cache,
+                        const void* landmarks, const float* bias, const int32_t* seq_lens,
+                        void* out, float* lse, int32_t* sel_idx, int32_t* device_status, void* stream);
+
 /* Bytes of device memory the *_host entry points need for staging (inputs + outputs + workspace). */
 size_t hils_host_arena_bytes(const hils_params* params, int is_decode);
 

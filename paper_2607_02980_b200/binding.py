@@ -23,7 +23,7 @@ _IMPL = {"auto": IMPL_AUTO, "generic": IMPL_GENERIC, "fast": IMPL_FAST}
 EXPORTS = [
     "hils_workspace_bytes", "hils_prefill", "hils_decode", "hils_host_arena_bytes",
     "hils_prefill_host", "hils_decode_host", "hils_poll_status", "hils_last_launch_count",
-    "hils_status_string", "hils_version", "hils_trace_enable", "hils_trace_read",
+    "hils_status_string", "hils_version", "hils_trace_enable", "hils_trace_read", "hils_decode_noalloc",
 ]
 
 
@@ -67,6 +67,8 @@ def load_library() -> ctypes.CDLL:
     lib.hils_prefill_host.argtypes = [pp, vp, vp, vp, vp, f32p, vp, f32p, i32p, vp, ctypes.c_size_t, vp]
     lib.hils_decode_host.restype = ctypes.c_int
     lib.hils_decode_host.argtypes = [pp, vp, vp, vp, vp, f32p, i32p, vp, f32p, i32p, vp, ctypes.c_size_t, vp]
+    lib.hils_decode_noalloc.restype = ctypes.c_int
+    lib.hils_decode_noalloc.argtypes = [pp, vp, vp, vp, vp, f32p, i32p, vp, f32p, i32p, i32p, vp]
     lib.hils_poll_status.restype = ctypes.c_int
     lib.hils_poll_status.argtypes = [vp, vp]
     lib.hils_last_launch_count.restype = ctypes.c_int
@@ -208,6 +210,43 @@ def hils_decode(q, k_cache, v_cache, landmarks, seq_lens, chunk_size: int, top_k
                          _stream_ptr(stream))
     if rc != 0:
         raise HilsError(rc, "hils_decode")
+    return out, lse, sel_idx
+
+
+def hils_decode_noalloc(q, k_cache, v_cache, landmarks, seq_lens, chunk_size: int, top_k: int, out, lse, sel_idx,
+                        stream=None, *, bias=None, scale: float = 0.0, device_status=None):
+    """hils_decode without a workspace: the library's own fixed device array holds the scratch.
+
+    For embedders that cannot allocate device memory (all HBM already given to a KV-cache pool, no
+    allocator handle, or a loop that must not call cudaMalloc).  Every output tensor has to be
+    passed in; this wrapper allocates nothing either.  Calls share one scratch array, so calls whose
+    kernels could overlap on the GPU must be serialised by the caller.  `device_status` is an optional
+    int32 CUDA tensor of one element that receives the device status word (0 = ok).
+    """
+    lib = load_library()
+    B, Hq, d = q.shape
+    Hkv, T = k_cache.shape[1], k_cache.shape[2]
+    Hl, C = landmarks.shape[1], landmarks.shape[2]
+    dt = q.dtype
+    _check(q, "q", (B, Hq, d), dt, True)
+    _check(k_cache, "k_cache", (B, Hkv, T, d), dt, True)
+    _check(v_cache, "v_cache", (B, Hkv, T, d), dt, True)
+    _check(landmarks, "landmarks", (B, Hl, C, d), dt, True)
+    _check(seq_lens, "seq_lens", (B,), torch.int32, True)
+    if bias is not None:
+        _check(bias, "bias", (B, Hl, C), torch.float32, True)
+    _check(out, "out", (B, Hq, d), dt, True)
+    _check(lse, "lse", (B, Hq), torch.float32, True)
+    _check(sel_idx, "sel_idx", (B, Hkv, top_k), torch.int32, True)
+    if device_status is not None:
+        _check(device_status, "device_status", (1,), torch.int32, True)
+    p = make_params(B=B, Hq=Hq, Hkv=Hkv, Hl=Hl, L=0, T_max=T, C=C, d=d, chunk_size=chunk_size, top_k=top_k,
+                    window=1, scale=scale, dtype=_dtype_code(q), impl="auto")
+    rc = lib.hils_decode_noalloc(ctypes.byref(p), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(landmarks),
+                                 _ptr(bias), _ptr(seq_lens), _ptr(out), _ptr(lse), _ptr(sel_idx),
+                                 _ptr(device_status), _stream_ptr(stream))
+    if rc != 0:
+        raise HilsError(rc, "hils_decode_noalloc")
     return out, lse, sel_idx
 
 

@@ -221,6 +221,29 @@ int hils_decode(const hils_params* params, const void* q, const void* k_cache, c
                workspace_bytes, stream);
 }
 
+int hils_decode_noalloc(const hils_params* params, const void* q, const void* k_cache, const void* v_cache,
+                        const void* landmarks, const float* bias, const int32_t* seq_lens, void* out, float* lse,
+                        int32_t* sel_idx, int32_t* device_status, void* stream) {
+    g_last_launches = 0;
+    Shape s;
+    int rc = make_shape(params, 1, &s);
+    if (rc != HILS_OK) return rc;
+    if (!q || !k_cache || !v_cache || !landmarks || !seq_lens || !out || !lse || !sel_idx) return HILS_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k_cache) || !aligned16(v_cache) || !aligned16(landmarks) || !aligned16(out) ||
+        (reinterpret_cast<uintptr_t>(lse) & 3u) || (reinterpret_cast<uintptr_t>(sel_idx) & 3u) ||
+        (bias && (reinterpret_cast<uintptr_t>(bias) & 3u)) ||
+        (device_status && (reinterpret_cast<uintptr_t>(device_status) & 3u)))
+        return HILS_ERR_ALIGNMENT;
+    if (!decode_fast_supports(s, params->dtype)) return HILS_ERR_UNSUPPORTED;
+    Tensors t{q, k_cache, v_cache, landmarks, bias, seq_lens, out, lse, sel_idx, nullptr, nullptr, 0};
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    trace_begin(st);
+    const int n = launch_decode_noalloc(s, t, device_status, st);
+    if (n < 0) return n;
+    g_last_launches = n;
+    return HILS_OK;
+}
+
 size_t hils_host_arena_bytes(const hils_params* params, int is_decode) {
     ArenaLayout a;
     if (arena_layout(params, is_decode, &a) != HILS_OK || a.ws_b == 0) return 0;

@@ -765,4 +765,43 @@ int launch_decode_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
     return 3;
 }
 
+// ------------------------------------------------------------------------- allocation-free variant
+// Scratch for callers that cannot obtain device memory themselves.  The array belongs to the loaded
+// library image: every GPU that loads libhils.so carries these 8 MiB until the process exits.
+constexpr size_t kNoAllocBytes = 8u << 20;
+constexpr int kMaxDevices = 64;
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
+
+size_t decode_noalloc_capacity() { return kNoAllocBytes; }
+
+int launch_decode_noalloc(const Shape& s, const Tensors& t_in, int32_t* device_status, cudaStream_t stream) {
+    const size_t need = kStatusBytes + decode_fast_scratch_bytes(s);
+    if (need > kNoAllocBytes) return HILS_ERR_WORKSPACE;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return HILS_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return HILS_ERR_UNSUPPORTED;
+    // In host code `g_noalloc_scratch` is only a handle for the symbol, not an address a kernel can
+    // use: the device address is looked up once per device, with that device current.
+    static void* dev_ptr[kMaxDevices] = {};
+    if (!dev_ptr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return HILS_ERR_CUDA;
+        dev_ptr[dev] = p;
+    }
+    unsigned char* base = static_cast<unsigned char*>(dev_ptr[dev]);
+    // The array keeps whatever the previous call left: the status word has to start at zero
+    // (the per-pair completion counters are re-zeroed by decode_select on every call).
+    if (cudaMemsetAsync(base, 0, kStatusBytes, stream) != cudaSuccess) return HILS_ERR_CUDA;
+    Tensors t = t_in;
+    t.status = reinterpret_cast<int*>(base);
+    t.scratch = base + kStatusBytes;
+    t.scratch_bytes = kNoAllocBytes - kStatusBytes;
+    const int n = launch_decode_fast(s, t, stream);
+    if (n < 0) return n;
+    if (device_status &&
+        cudaMemcpyAsync(device_status, base, sizeof(int32_t), cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
+        return HILS_ERR_CUDA;
+    return n;
+}
+
 }  // namespace hils

@@ -38,6 +38,10 @@ int launch_decode_fast(const Shape& s, const Tensors& t, cudaStream_t stream);
 bool decode_fast_supports(const Shape& s, int dtype);
 size_t decode_fast_scratch_bytes(const Shape& s);
 
+// Decode fast path run on the library's own static device scratch (see hils_decode_noalloc).
+int launch_decode_noalloc(const Shape& s, const Tensors& t, int32_t* device_status, cudaStream_t stream);
+size_t decode_noalloc_capacity();
+
 int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream);
 bool prefill_fast_supports(const Shape& s, int dtype);
 size_t prefill_fast_scratch_bytes(const Shape& s);
