@@ -328,7 +328,24 @@ def main():
     ap.add_argument("--extra", action="store_true", help="also time the other single-GPU configurations")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--profile-run", action="store_true",
+                    help="only run warmup+steps calls of the workload (for ncu captures); no timing extras")
+    ap.add_argument("--batch", type=int, default=0, help="profile runs: override the batch size (smaller footprint)")
     args = ap.parse_args()
+    if args.profile_run:
+        import paper_2607_02980_b200 as hils
+        torch.cuda.set_device(0)
+        cfg = pick_cfg(args.workload)
+        if args.batch > 0:
+            cfg = cfg.scaled(B=args.batch)
+        w = Workload(hils, cfg, torch.device("cuda", 0), n_query_sets=2)
+        for _ in range(args.warmup + args.steps):
+            w.between_steps()
+            w.step()
+        torch.cuda.synchronize()
+        print(json.dumps({"profile_run": cfg.name, "B": cfg.B, "calls": args.warmup + args.steps,
+                          "kernels_per_call": hils.last_launch_count()}))
+        return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
     if args.impl == "reference":

@@ -633,6 +633,13 @@ prefill_fuse_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_cons
     }
 }
 
+// HILS_FORCE_MMA_SELECT=1 keeps the warp-MMA selection kernel even where the tcgen05 one applies
+// (used to cross-check the two).
+const bool g_force_mma_select = [] {
+    const char* e = getenv("HILS_FORCE_MMA_SELECT");
+    return e != nullptr && e[0] == '1';
+}();
+
 struct Plan {
     int qb, max_tiles;
     size_t off_cnt, off_cursor, off_ntiles, zero_bytes, off_off, off_toff, off_entries, off_tiles, off_obuf, off_lam,
@@ -724,8 +731,13 @@ int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
 
     int launches = 0;
     const int tiles_per_seq = (s.R + kS - 1) / kS;
-    prefill_select_kernel<<<static_cast<unsigned>(pairs) * tiles_per_seq, 160, sel_smem, stream>>>(map_lm, a);
-    if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
+    if (prefill_select_tc_supports(s) && !g_force_mma_select) {
+        const int rc = launch_prefill_select_tc(s, t.q, t.landmarks, t.bias, t.sel_idx, t.status, stream);
+        if (rc < 0) return rc;
+    } else {
+        prefill_select_kernel<<<static_cast<unsigned>(pairs) * tiles_per_seq, 160, sel_smem, stream>>>(map_lm, a);
+        if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
+    }
     trace_mark("prefill_select", stream);
     ++launches;
 

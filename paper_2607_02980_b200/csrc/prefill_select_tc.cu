@@ -1,0 +1,268 @@
+// Landmark scoring + exact top-K for prefill on the 5th-generation tensor cores (tcgen05 + TMEM).
+//
+// One CTA per (sequence, KV head, 128-token tile).  The tile's queries (4 heads x 128 tokens x 128 d)
+// stay in shared memory; landmark tiles of 64 chunks stream through a TMA ring.  One thread issues
+// tcgen05.mma (M = 128 tokens, N = 64 chunks, K = 128) once per head into tensor memory, double
+// buffered; the four epilogue warps own one token per thread (token = TMEM lane), read the four
+// heads' scores, take the group max (App. C) and keep the token's exact running top-K
+// (Eq. surrogate top-k; equal scores go to the lower chunk id) in a private shared-memory list.
+#include "internal.h"
+#include "tma.cuh"
+
+namespace hils {
+namespace {
+
+constexpr int kD = 128;
+constexpr int kS = 64;
+constexpr int kG = 4;
+constexpr int kTileTok = 128;
+constexpr int kLmStages = 2;
+constexpr int kLmStageBytes = kS * kD * 2;          // 64 landmark rows = two 8 KB K-blocks
+constexpr int kQBytes = kG * kTileTok * kD * 2;     // 128 KB
+constexpr int kQueueCap = 32;
+constexpr int kMaxK = 32;
+constexpr int kThreads = 192;                       // 4 epilogue warps, 1 TMA warp, 1 MMA warp
+constexpr uint32_t kTmemCols = 512;                 // 2 buffers x 4 heads x 64 columns
+
+struct TcArgs {
+    Shape s;
+    const float* bias;
+    int32_t* sel;
+    int* status;
+};
+
+struct TcSmem {
+    uint64_t q_full;
+    uint64_t full[kLmStages];
+    uint64_t empty[kLmStages];
+    uint64_t tmem_full[2];
+    uint64_t tmem_empty[2];
+    uint32_t tmem_base;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_lm,
+                         const TcArgs a) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* qs = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* lms = qs + kQBytes;
+    unsigned long long* lists = reinterpret_cast<unsigned long long*>(lms + kLmStages * kLmStageBytes);
+    unsigned long long* queue = lists + kMaxK * kTileTok;
+    TcSmem& sm = *reinterpret_cast<TcSmem*>(queue + kQueueCap * kTileTok);
+
+    const Shape& s = a.s;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int pairs = s.B * s.Hkv;
+    const int tiles_per_seq = (s.R + kTileTok - 1) / kTileTok;
+    const int ti = tiles_per_seq - 1 - static_cast<int>(blockIdx.x) / pairs;     // heavy tiles first
+    const int pair = static_cast<int>(blockIdx.x) % pairs;
+    const int b = pair / s.Hkv, gk = pair % s.Hkv;
+    // W = 1: tokens of the first 64 rows see chunks 0..2ti-1, the second 64 rows also chunk 2ti
+    const bool second_half = ti * kTileTok + kS < s.R;
+    const int ncand_max = second_half ? 2 * ti + 1 : 2 * ti;
+    const int nsteps = (ncand_max + kS - 1) / kS;
+    const int K = s.K;
+
+    if (tid == 0) {
+        mbar_init(&sm.q_full, 1);
+        for (int i = 0; i < kLmStages; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&sm.tmem_full[i], 1); mbar_init(&sm.tmem_empty[i], 4); }
+        mbar_fence_init();
+        tma_prefetch_desc(&map_q);
+        tma_prefetch_desc(&map_lm);
+    }
+    if (warp == 5) tmem_alloc(&sm.tmem_base, kTmemCols);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = sm.tmem_base;
+
+    if (warp == 4) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0 && nsteps > 0) {
+            mbar_expect_tx(&sm.q_full, kQBytes);
+            for (int h = 0; h < kG; ++h) {
+                const int row = (b * s.Hq + gk * kG + h) * s.R + ti * kTileTok;
+                tma_load_2d(qs + h * 32768, &map_q, &sm.q_full, 0, row);
+                tma_load_2d(qs + h * 32768 + 16384, &map_q, &sm.q_full, 64, row);
+            }
+            int issued = 0;
+            for (int it = 0; it < nsteps; ++it) {
+                const int st = it % kLmStages;
+                if (it >= kLmStages && !mbar_wait(&sm.empty[st], ((it / kLmStages) - 1) & 1)) {
+                    set_status(a.status, kDevTimeout);
+                    break;
+                }
+                uint8_t* dst = lms + st * kLmStageBytes;
+                const int row = pair * s.C + it * kS;
+                mbar_expect_tx(&sm.full[st], kLmStageBytes);
+                tma_load_2d(dst, &map_lm, &sm.full[st], 0, row);
+                tma_load_2d(dst + 8192, &map_lm, &sm.full[st], 64, row);
+                ++issued;
+            }
+            // own copies in flight: every issued stage and the query tile must have landed before exit
+            mbar_wait(&sm.q_full, 0);
+            for (int it = max(0, issued - kLmStages); it < issued; ++it)
+                mbar_wait(&sm.full[it % kLmStages], (it / kLmStages) & 1);
+        }
+    } else if (warp == 5) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0 && nsteps > 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(kTileTok, kS);
+            bool ok = mbar_wait(&sm.q_full, 0);
+            for (int it = 0; it < nsteps && ok; ++it) {
+                const int st = it % kLmStages, buf = it & 1;
+                ok = mbar_wait(&sm.full[st], (it / kLmStages) & 1);
+                if (ok && it >= 2) ok = mbar_wait(&sm.tmem_empty[buf], ((it >> 1) - 1) & 1);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t lm_addr = smem_u32(lms + st * kLmStageBytes);
+#pragma unroll
+                for (int h = 0; h < kG; ++h) {
+                    const uint32_t d_tmem = tmem_base + buf * 256 + h * kS;
+                    const uint32_t q_addr = smem_u32(qs + h * 32768);
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint64_t da = umma_desc_k128(q_addr + (ks >> 2) * 16384 + (ks & 3) * 32);
+                        const uint64_t db = umma_desc_k128(lm_addr + (ks >> 2) * 8192 + (ks & 3) * 32);
+                        umma_bf16(d_tmem, da, db, idesc, ks > 0 ? 1u : 0u);
+                    }
+                }
+                umma_commit(&sm.empty[st]);            // landmark stage reusable once these MMAs are done
+                umma_commit(&sm.tmem_full[buf]);       // scores of this step readable
+            }
+            if (!ok) set_status(a.status, kDevTimeout);
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue: one token per thread
+        const int row = warp * 32 + lane;
+        const int tok = ti * kTileTok + row;
+        const int my_ncand = row < kS ? 2 * ti : 2 * ti + 1;
+        const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
+        unsigned long long* mylist = lists + tid;          // entry e at mylist[e * 128]
+        unsigned long long* myq = queue + tid;
+        const float* bias = a.bias ? a.bias + static_cast<long long>(pair) * s.C : nullptr;
+        unsigned long long tau = 0ull;
+        int cnt = 0, pmin = 0, qn = 0;
+        bool ok = true;
+
+        auto drain = [&]() {
+            int mx = qn;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(kFullMask, mx, o));
+            for (int i = 0; i < mx; ++i) {
+                if (i < qn) {
+                    const unsigned long long key = myq[i * kTileTok];
+                    if (key > tau) {
+                        bool rescan = true;
+                        if (cnt < K) {
+                            mylist[cnt * kTileTok] = key;
+                            ++cnt;
+                            rescan = cnt == K;
+                        } else {
+                            mylist[pmin * kTileTok] = key;
+                        }
+                        if (rescan) {
+                            unsigned long long mn = ~0ull;
+                            int pm = 0;
+                            for (int e = 0; e < K; ++e) {
+                                const unsigned long long x = mylist[e * kTileTok];
+                                if (x < mn) { mn = x; pm = e; }
+                            }
+                            tau = mn;
+                            pmin = pm;
+                        }
+                    }
+                }
+            }
+            qn = 0;
+        };
+
+        for (int it = 0; it < nsteps && ok; ++it) {
+            const int buf = it & 1;
+            ok = mbar_wait(&sm.tmem_full[buf], (it >> 1) & 1);
+            if (!ok) break;
+            tc_fence_after_sync();
+#pragma unroll 1
+            for (int cb = 0; cb < 4; ++cb) {
+                float um[16], r[16];
+                const uint32_t col = buf * 256 + cb * 16;
+                tmem_ld16(t_lane + col, um);
+#pragma unroll
+                for (int h = 1; h < kG; ++h) {
+                    tmem_ld16(t_lane + col + h * kS, r);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) um[j] = fmaxf(um[j], r[j]);
+                }
+                const int c0 = it * kS + cb * 16;
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const int c = c0 + j;
+                    if (c < my_ncand) {
+                        float u = um[j] * s.scale;
+                        if (bias) u += bias[c];
+                        const unsigned long long key = select_key(u, c);
+                        if (key > tau) {
+                            myq[qn * kTileTok] = key;
+                            ++qn;
+                        }
+                    }
+                }
+                if (__any_sync(kFullMask, qn > kQueueCap - 16)) drain();
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.tmem_empty[buf]);
+        }
+        if (!ok && lane == 0) set_status(a.status, kDevTimeout);
+        drain();
+
+        // ascending chunk ids, -1 padded
+        if (tok < s.R) {
+            int32_t* sel = a.sel + (static_cast<long long>(pair) * s.R + tok) * K;
+            for (int e = 0; e < cnt; ++e) {
+                const int id = key_chunk(mylist[e * kTileTok]);
+                int rank = 0;
+                for (int j = 0; j < cnt; ++j) rank += key_chunk(mylist[j * kTileTok]) < id ? 1 : 0;
+                sel[rank] = id;
+            }
+            for (int e = cnt; e < K; ++e) sel[e] = -1;
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    if (warp == 5) tmem_dealloc(tmem_base, kTmemCols);
+}
+
+}  // namespace
+
+bool prefill_select_tc_supports(const Shape& s) {
+    return s.K <= kMaxK && static_cast<long long>(s.B) * s.Hq * s.R < (1ll << 31);
+}
+
+int launch_prefill_select_tc(const Shape& s, const void* q, const void* landmarks, const float* bias, int32_t* sel,
+                             int* status, cudaStream_t stream) {
+    const int pairs = s.B * s.Hkv;
+    CUtensorMap map_q, map_lm;
+    if (!make_bf16_2d_map(&map_q, q, static_cast<uint64_t>(s.B) * s.Hq * s.R, kD, 64, kTileTok) ||
+        !make_bf16_2d_map(&map_lm, landmarks, static_cast<uint64_t>(pairs) * s.C, kD, 64, kS))
+        return HILS_ERR_CUDA;
+    const size_t smem = kQBytes + kLmStages * kLmStageBytes + sizeof(unsigned long long) * (kMaxK + kQueueCap) * kTileTok +
+                        sizeof(TcSmem) + 1024;
+    static bool attr_done = false;
+    if (!attr_done) {
+        if (cudaFuncSetAttribute(prefill_select_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(smem)) != cudaSuccess)
+            return HILS_ERR_CUDA;
+        attr_done = true;
+    }
+    TcArgs a{s, bias, sel, status};
+    const int tiles = (s.R + kTileTok - 1) / kTileTok;
+    prefill_select_tc_kernel<<<static_cast<unsigned>(pairs) * tiles, kThreads, smem, stream>>>(map_q, map_lm, a);
+    if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
+    return 1;
+}
+
+}  // namespace hils
