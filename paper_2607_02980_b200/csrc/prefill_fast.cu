@@ -39,17 +39,19 @@ struct PArgs {
     int32_t* sel;
     int* status;
     // scratch (per token block)
-    int* cnt;               // [pairs*C] selectors of each (pair, chunk) in the block
+    int* cnt;               // [pairs*nc] rows of each (pair, chunk) in the block: selectors + own tokens
     int* cursor;            // [pairs*C]
     int* n_tiles;           // [1] (+ padding)
     int* off;               // [pairs*C] exclusive prefix of cnt
     int* toff;              // [pairs*C] exclusive prefix of tiles per (pair, chunk)
-    int* entries;           // [pairs*QB*K] (token_local << 8) | slot, grouped by (pair, chunk)
+    int* entries;           // [pairs*QB*(K+1)] (token_local << 8) | slot, grouped by (pair, chunk);
+                            // slot K marks the token's own chunk (local branch)
     int4* tiles;            // [max_tiles] {pair, chunk, first entry, rows}
-    __nv_bfloat16* obuf;    // [pairs*QB*K][G][128] normalised per-chunk outputs
-    float* lam;             // [pairs*QB][G][K] per-head surrogate scores of the selected chunks
+    __nv_bfloat16* obuf;    // [pairs*QB*(K+1)][G][128] normalised per-chunk outputs (slot K: local)
+    float* lam;             // [pairs*QB][G][K+1] per-head surrogate scores; slot K: log Z_swa
     int i0, i1;             // token block [i0, i1)
     int qb;                 // tokens per block the obuf / lam strides are sized for
+    int nc;                 // chunk slots per pair in cnt/off/...: max(C, ceil(L / S))
     int max_tiles;
 };
 
@@ -239,17 +241,23 @@ prefill_select_kernel(const __grid_constant__ CUtensorMap map_lm, const PArgs a)
 }
 
 // ------------------------------------------------------------------------------------------ invert
+// Chunk attended by slot `slot` of token i0+il: a selected chunk, or (slot K) the token's own chunk.
+__device__ __forceinline__ int slot_chunk(const PArgs& a, int pair, int il, int slot) {
+    if (slot == a.s.K) return (a.i0 + il) / kS;
+    return a.sel[(static_cast<long long>(pair) * a.s.R + a.i0 + il) * a.s.K + slot];
+}
+
 __global__ void invert_count_kernel(const PArgs a) {
     const Shape& s = a.s;
-    const int K = s.K, nblk = a.i1 - a.i0;
-    const long long total = static_cast<long long>(s.B) * s.Hkv * nblk * K;
+    const int K1 = s.K + 1, nblk = a.i1 - a.i0;
+    const long long total = static_cast<long long>(s.B) * s.Hkv * nblk * K1;
     for (long long x = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; x < total;
          x += static_cast<long long>(gridDim.x) * blockDim.x) {
-        const int slot = static_cast<int>(x % K);
-        const int il = static_cast<int>((x / K) % nblk);
-        const int pair = static_cast<int>(x / (static_cast<long long>(K) * nblk));
-        const int c = a.sel[(static_cast<long long>(pair) * s.R + a.i0 + il) * K + slot];
-        if (c >= 0) atomicAdd(&a.cnt[pair * s.C + c], 1);
+        const int slot = static_cast<int>(x % K1);
+        const int il = static_cast<int>((x / K1) % nblk);
+        const int pair = static_cast<int>(x / (static_cast<long long>(K1) * nblk));
+        const int c = slot_chunk(a, pair, il, slot);
+        if (c >= 0) atomicAdd(&a.cnt[pair * a.nc + c], 1);
     }
 }
 
@@ -258,7 +266,7 @@ __global__ void __launch_bounds__(1024) invert_scan_kernel(const PArgs a) {
     __shared__ int wsum_e[32], wsum_t[32];
     __shared__ int carry_e, carry_t;
     const Shape& s = a.s;
-    const int n = s.B * s.Hkv * s.C;
+    const int n = s.B * s.Hkv * a.nc;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (tid == 0) { carry_e = 0; carry_t = 0; }
     __syncthreads();
@@ -280,7 +288,7 @@ __global__ void __launch_bounds__(1024) invert_scan_kernel(const PArgs a) {
         if (x < n) {
             a.off[x] = oe;
             a.toff[x] = ot;
-            const int pair = x / s.C, c = x % s.C;
+            const int pair = x / a.nc, c = x % a.nc;
             for (int k = 0; k < ct; ++k)
                 if (ot + k < a.max_tiles)
                     a.tiles[ot + k] = make_int4(pair, c, oe + k * kTileTok, min(kTileTok, ce - k * kTileTok));
@@ -294,16 +302,16 @@ __global__ void __launch_bounds__(1024) invert_scan_kernel(const PArgs a) {
 
 __global__ void invert_fill_kernel(const PArgs a) {
     const Shape& s = a.s;
-    const int K = s.K, nblk = a.i1 - a.i0;
-    const long long total = static_cast<long long>(s.B) * s.Hkv * nblk * K;
+    const int K1 = s.K + 1, nblk = a.i1 - a.i0;
+    const long long total = static_cast<long long>(s.B) * s.Hkv * nblk * K1;
     for (long long x = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; x < total;
          x += static_cast<long long>(gridDim.x) * blockDim.x) {
-        const int slot = static_cast<int>(x % K);
-        const int il = static_cast<int>((x / K) % nblk);
-        const int pair = static_cast<int>(x / (static_cast<long long>(K) * nblk));
-        const int c = a.sel[(static_cast<long long>(pair) * s.R + a.i0 + il) * K + slot];
+        const int slot = static_cast<int>(x % K1);
+        const int il = static_cast<int>((x / K1) % nblk);
+        const int pair = static_cast<int>(x / (static_cast<long long>(K1) * nblk));
+        const int c = slot_chunk(a, pair, il, slot);
         if (c >= 0) {
-            const int idx = pair * s.C + c;
+            const int idx = pair * a.nc + c;
             const int pos = a.off[idx] + atomicAdd(&a.cursor[idx], 1);
             a.entries[pos] = (il << 8) | slot;
         }
@@ -409,16 +417,26 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
             }
             if (tid < 16) {
                 // landmark of this chunk as row 0 of a 9th key tile (rows 1..7 stay zero)
-                const uint4 v = *reinterpret_cast<const uint4*>(a.lm + (static_cast<long long>(pair) * s.C + c) * kD + tid * 8);
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                if (c < s.C) v = *reinterpret_cast<const uint4*>(a.lm + (static_cast<long long>(pair) * s.C + c) * kD + tid * 8);
                 *reinterpret_cast<uint4*>(lmt + (tid >> 3) * 1024 + swz128(0, tid & 7)) = v;
             }
             const bool ok = mbar_wait(&sm.bar, phase);
             phase ^= 1u;
-            __syncthreads();
             if (!ok) {
                 if (tid == 0) set_status(a.status, kDevTimeout);
                 return;
             }
+            const int nv = min(kS, s.R - c * kS);
+            if (nv < kS) {
+                // last, partial chunk of the sequence: rows past its end may hold anything; zero the
+                // V rows so that they meet their zero probabilities safely
+                for (int x = tid; x < (kS - nv) * 16; x += 128) {
+                    const int row = nv + (x >> 4), piece = x & 15;
+                    *reinterpret_cast<uint4*>(kv + 16384 + (piece >> 3) * 8192 + swz128(row, piece & 7)) = make_uint4(0u, 0u, 0u, 0u);
+                }
+            }
+            __syncthreads();
             cur_pair = pair;
             cur_c = c;
         }
@@ -445,9 +463,17 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
                 mma_bf16_16816(sl, aq[2 * kp + 1], r2, r3);
             }
         }
+        // rows of the chunk's own tokens (slot K) are the local branch: causal inside the chunk
+        const bool locA = (eA & 255) == K, locB = (eB & 255) == K;
+        const int limA = locA ? a.i0 + ilA - c * kS : kS - 1, limB = locB ? a.i0 + ilB - c * kS : kS - 1;
         float mA = -INFINITY, mB = -INFINITY;
 #pragma unroll
         for (int nt = 0; nt < 8; ++nt) {
+            const int key = nt * 8 + 2 * t;
+            if (key > limA) sc[nt][0] = -INFINITY;
+            if (key + 1 > limA) sc[nt][1] = -INFINITY;
+            if (key > limB) sc[nt][2] = -INFINITY;
+            if (key + 1 > limB) sc[nt][3] = -INFINITY;
             mA = fmaxf(mA, fmaxf(sc[nt][0], sc[nt][1]));
             mB = fmaxf(mB, fmaxf(sc[nt][2], sc[nt][3]));
         }
@@ -475,11 +501,14 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
             *reinterpret_cast<uint32_t*>(stg + (g + 8) * kStgPitch + (i * 8 + 2 * t) * 2) = pack_bf16(o[i][2] * iB, o[i][3] * iB);
         }
         if (t == 0) {
-            const float bb = a.bias ? a.bias[static_cast<long long>(pair) * s.C + c] : 0.f;
+            const float bb = (a.bias && c < s.C) ? a.bias[static_cast<long long>(pair) * s.C + c] : 0.f;
+            // mass of the row's chunk: the surrogate score, or log Z_swa for the local branch
             if (g < rows)
-                a.lam[((static_cast<long long>(pair) * a.qb + ilA) * kG + warp) * K + (eA & 255)] = sl[0] * s.scale + bb;
+                a.lam[((static_cast<long long>(pair) * a.qb + ilA) * kG + warp) * (K + 1) + (eA & 255)] =
+                    locA ? mA * s.scale + __logf(zA) : sl[0] * s.scale + bb;
             if (g + 8 < rows)
-                a.lam[((static_cast<long long>(pair) * a.qb + ilB) * kG + warp) * K + (eB & 255)] = sl[2] * s.scale + bb;
+                a.lam[((static_cast<long long>(pair) * a.qb + ilB) * kG + warp) * (K + 1) + (eB & 255)] =
+                    locB ? mB * s.scale + __logf(zB) : sl[2] * s.scale + bb;
         }
         __syncwarp();
         // coalesced 256-byte rows: 16 lanes x 16 B per row, two rows per instruction
@@ -489,7 +518,7 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
             if (row < rows) {
                 const int e = a.entries[first + row];
                 const uint4 v = *reinterpret_cast<const uint4*>(stg + row * kStgPitch + piece * 16);
-                __nv_bfloat16* dst = a.obuf + (((static_cast<long long>(pair) * a.qb + (e >> 8)) * K + (e & 255)) * kG + warp) * kD;
+                __nv_bfloat16* dst = a.obuf + (((static_cast<long long>(pair) * a.qb + (e >> 8)) * (K + 1) + (e & 255)) * kG + warp) * kD;
                 *reinterpret_cast<uint4*>(dst + piece * 8) = v;
             }
         }
@@ -498,139 +527,91 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
 }
 
 // ------------------------------------------------------------------------------------------ fuse
-constexpr int kFusePitch = 132;                // floats per staged local-output row
+// One warp per (sequence, KV head, token): softmax over {surrogate scores of the selected chunks} U
+// {log Z_swa} per head (Eq. HiLS weights, inter-chunk factor) and the weighted sum of the rows that
+// prefill_attend wrote.  Pure streaming: a slot's 4 heads are 1 KB contiguous (two 16-byte loads per
+// lane); lane l covers head l/16 (and head 2 + l/16), elements 8*(l%16)..+7.
+constexpr int kFuseWarps = 8;
 
-struct FuseSmem {
-    uint64_t bar;
-    alignas(16) float stage[kG][16 * kFusePitch];     // read back with 16-byte loads
-};
-
-__global__ void __launch_bounds__(128, 2)
-prefill_fuse_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
-                    const PArgs a) {
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* kv = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    FuseSmem& sm = *reinterpret_cast<FuseSmem*>(kv + 32768);
+__global__ void __launch_bounds__(kFuseWarps * 32) prefill_fuse_kernel(const PArgs a) {
+    __shared__ float wsm[kFuseWarps][kG][68];
     const Shape& s = a.s;
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int g = lane >> 2, t = lane & 3;
-    const int K = s.K;
-    const int pairs = s.B * s.Hkv;
-    const int pair = static_cast<int>(blockIdx.x) % pairs;
-    const int ci = a.i0 / kS + static_cast<int>(blockIdx.x) / pairs;
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+    const int K = s.K, K1 = K + 1, nblk = a.i1 - a.i0;
+    const long long total = static_cast<long long>(s.B) * s.Hkv * nblk;
+    const long long w = static_cast<long long>(blockIdx.x) * kFuseWarps + wib;
+    if (w >= total) return;
+    const int il = static_cast<int>(w % nblk);
+    const int pair = static_cast<int>(w / nblk);
     const int b = pair / s.Hkv, gk = pair % s.Hkv;
-    const float sl2 = s.scale * kLog2e;
-    const int nsel = min(K, ci);                 // W = 1: every token of chunk ci has ci candidates
-
-    if (tid == 0) {
-        mbar_init(&sm.bar, 1);
-        mbar_fence_init();
-        const int row = pair * s.T + ci * kS;
-        mbar_expect_tx(&sm.bar, 32768);
-        tma_load_2d(kv, &map_k, &sm.bar, 0, row);
-        tma_load_2d(kv + 8192, &map_k, &sm.bar, 64, row);
-        tma_load_2d(kv + 16384, &map_v, &sm.bar, 0, row);
-        tma_load_2d(kv + 24576, &map_v, &sm.bar, 64, row);
+    const int tok = a.i0 + il;
+    const int nsel = min(K, tok / kS);               // W = 1: a token of chunk ci has ci candidates
+    const float* lrow = a.lam + (static_cast<long long>(pair) * a.qb + il) * kG * K1;
+    float (*wv)[68] = wsm[wib];
+    float lse_h = 0.f;
+#pragma unroll
+    for (int h = 0; h < kG; ++h) {
+        const float l0 = lane < nsel ? lrow[h * K1 + lane] : -INFINITY;
+        const float l1 = lane + 32 < nsel ? lrow[h * K1 + lane + 32] : -INFINITY;
+        const float ll = lrow[h * K1 + K];
+        const float Mx = warp_max(fmaxf(fmaxf(l0, l1), ll));
+        const float e0 = __expf(l0 - Mx), e1 = __expf(l1 - Mx), el = __expf(ll - Mx);
+        const float D = warp_sum(e0 + e1) + el;
+        const float inv = 1.f / D;
+        if (lane < nsel) wv[h][lane] = e0 * inv;
+        if (lane + 32 < nsel) wv[h][lane + 32] = e1 * inv;
+        if (lane == 0) wv[h][64] = el * inv;
+        if (lane == h) lse_h = Mx + __logf(D);
     }
-    __syncthreads();
-    const bool ok = mbar_wait(&sm.bar, 0);
-    if (!ok) {
-        if (tid == 0) set_status(a.status, kDevTimeout);
-        return;
-    }
-    const int nv = min(kS, s.R - ci * kS);
-    if (nv < kS) {
-        // rows past the end of the sequence may hold anything: zero them before they meet P = 0
-        for (int x = tid; x < (kS - nv) * 16; x += 128) {
-            const int row = nv + (x >> 4), piece = x & 15;
-            *reinterpret_cast<uint4*>(kv + 16384 + (piece >> 3) * 8192 + swz128(row, piece & 7)) = make_uint4(0u, 0u, 0u, 0u);
+    __syncwarp();
+    const int hA = lane >> 4, hB = 2 + (lane >> 4), piece = lane & 15;
+    const __nv_bfloat16* ob = a.obuf + (static_cast<long long>(pair) * a.qb + il) * K1 * kG * kD;
+    float accA[8], accB[8];
+#pragma unroll
+    for (int x = 0; x < 8; ++x) { accA[x] = 0.f; accB[x] = 0.f; }
+    auto fma8 = [](float (&acc)[8], const uint4& raw, float wgt) {
+        const uint32_t wd[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+            acc[2 * x] = fmaf(wgt, __uint_as_float(wd[x] << 16), acc[2 * x]);
+            acc[2 * x + 1] = fmaf(wgt, __uint_as_float(wd[x] & 0xffff0000u), acc[2 * x + 1]);
         }
-        __syncthreads();
+    };
+    // local slot first, then the selected slots four at a time (8 loads in flight per lane)
+    {
+        const __nv_bfloat16* row = ob + static_cast<long long>(K) * kG * kD;
+        const uint4 ra = __ldg(reinterpret_cast<const uint4*>(row + lane * 8));
+        const uint4 rb = __ldg(reinterpret_cast<const uint4*>(row + 256 + lane * 8));
+        fma8(accA, ra, wv[hA][64]);
+        fma8(accB, rb, wv[hB][64]);
     }
-    const uint32_t ks_addr = smem_u32(kv), vs_addr = ks_addr + 16384;
-    const int h = gk * kG + warp;
-    const __nv_bfloat16* qh = a.q + (static_cast<long long>(b) * s.Hq + h) * s.R * kD;
-    float* stg = sm.stage[warp];
-
-    for (int mt = 0; mt < 4; ++mt) {
-        const int rowA = mt * 16 + g, rowB = rowA + 8;           // position inside the chunk
-        const int tokA = ci * kS + rowA, tokB = ci * kS + rowB;
-        if (ci * kS + mt * 16 >= s.R) break;
-        uint32_t aq[8][4];
-        load_q_frags(qh + static_cast<long long>(min(tokA, s.R - 1)) * kD,
-                     qh + static_cast<long long>(min(tokB, s.R - 1)) * kD, t, aq);
-        float sc[8][4];
-        qk16(aq, ks_addr, lane, 2 * mt + 2, sc);
-        float mA = -INFINITY, mB = -INFINITY;
+    for (int sl0 = 0; sl0 < nsel; sl0 += 4) {
+        uint4 ra[4], rb[4];
 #pragma unroll
-        for (int nt = 0; nt < 8; ++nt) {
+        for (int u = 0; u < 4; ++u) {
+            const int sl = min(sl0 + u, nsel - 1);
+            const __nv_bfloat16* row = ob + static_cast<long long>(sl) * kG * kD;
+            ra[u] = __ldg(reinterpret_cast<const uint4*>(row + lane * 8));
+            rb[u] = __ldg(reinterpret_cast<const uint4*>(row + 256 + lane * 8));
+        }
 #pragma unroll
-            for (int v = 0; v < 4; ++v) {
-                const int key = nt * 8 + 2 * t + (v & 1);
-                const int row = v < 2 ? rowA : rowB;
-                if (key > row) sc[nt][v] = -INFINITY;              // causal: j <= i
+        for (int u = 0; u < 4; ++u) {
+            if (sl0 + u < nsel) {
+                fma8(accA, ra[u], wv[hA][sl0 + u]);
+                fma8(accB, rb[u], wv[hB][sl0 + u]);
             }
-            mA = fmaxf(mA, fmaxf(sc[nt][0], sc[nt][1]));
-            mB = fmaxf(mB, fmaxf(sc[nt][2], sc[nt][3]));
         }
-        mA = fmaxf(mA, __shfl_xor_sync(kFullMask, mA, 1)); mA = fmaxf(mA, __shfl_xor_sync(kFullMask, mA, 2));
-        mB = fmaxf(mB, __shfl_xor_sync(kFullMask, mB, 1)); mB = fmaxf(mB, __shfl_xor_sync(kFullMask, mB, 2));
-        float zA = 0.f, zB = 0.f;
-#pragma unroll
-        for (int nt = 0; nt < 8; ++nt) {
-            sc[nt][0] = exp2f((sc[nt][0] - mA) * sl2); sc[nt][1] = exp2f((sc[nt][1] - mA) * sl2);
-            sc[nt][2] = exp2f((sc[nt][2] - mB) * sl2); sc[nt][3] = exp2f((sc[nt][3] - mB) * sl2);
-            zA += sc[nt][0] + sc[nt][1];
-            zB += sc[nt][2] + sc[nt][3];
-        }
-        zA += __shfl_xor_sync(kFullMask, zA, 1); zA += __shfl_xor_sync(kFullMask, zA, 2);
-        zB += __shfl_xor_sync(kFullMask, zB, 1); zB += __shfl_xor_sync(kFullMask, zB, 2);
-        float o[16][4];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
-        pv16(sc, vs_addr, lane, mt + 1, o);
-        const float iA = 1.f / zA, iB = 1.f / zB;
-        const float lamA = mA * s.scale + __logf(zA), lamB = mB * s.scale + __logf(zB);   // log Z_swa
-        __syncwarp();
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            *reinterpret_cast<float2*>(stg + g * kFusePitch + i * 8 + 2 * t) = make_float2(o[i][0] * iA, o[i][1] * iA);
-            *reinterpret_cast<float2*>(stg + (g + 8) * kFusePitch + i * 8 + 2 * t) = make_float2(o[i][2] * iB, o[i][3] * iB);
-        }
-        __syncwarp();
-        // mix: one row at a time, lanes across the head dimension (4 elements each)
-        for (int r = 0; r < 16; ++r) {
-            const int tok = ci * kS + mt * 16 + r;
-            const float lam_loc = __shfl_sync(kFullMask, r < 8 ? lamA : lamB, (r & 7) * 4);
-            if (tok >= s.R) continue;
-            const int il = tok - a.i0;
-            const float* lrow = a.lam + ((static_cast<long long>(pair) * a.qb + il) * kG + warp) * K;
-            const float l0 = lane < nsel ? lrow[lane] : -INFINITY;
-            const float l1 = lane + 32 < nsel ? lrow[lane + 32] : -INFINITY;
-            const float Mx = warp_max(fmaxf(fmaxf(l0, l1), lam_loc));
-            const float e0 = __expf(l0 - Mx), e1 = __expf(l1 - Mx), el = __expf(lam_loc - Mx);
-            const float D = warp_sum(e0 + e1) + el;
-            const float inv = 1.f / D;
-            const float4 ol = *reinterpret_cast<const float4*>(stg + r * kFusePitch + lane * 4);
-            float acc0 = ol.x * el, acc1 = ol.y * el, acc2 = ol.z * el, acc3 = ol.w * el;
-            const __nv_bfloat16* ob = a.obuf + ((static_cast<long long>(pair) * a.qb + il) * K * kG + warp) * kD + lane * 4;
-            for (int sl = 0; sl < nsel; ++sl) {
-                const float w = __shfl_sync(kFullMask, sl < 32 ? e0 : e1, sl & 31);
-                const uint2 raw = __ldg(reinterpret_cast<const uint2*>(ob + static_cast<long long>(sl) * kG * kD));
-                acc0 = fmaf(w, __uint_as_float(raw.x << 16), acc0);
-                acc1 = fmaf(w, __uint_as_float(raw.x & 0xffff0000u), acc1);
-                acc2 = fmaf(w, __uint_as_float(raw.y << 16), acc2);
-                acc3 = fmaf(w, __uint_as_float(raw.y & 0xffff0000u), acc3);
-            }
-            const long long orow = (static_cast<long long>(b) * s.Hq + h) * s.R + tok;
-            uint2 packed;
-            packed.x = pack_bf16(acc0 * inv, acc1 * inv);
-            packed.y = pack_bf16(acc2 * inv, acc3 * inv);
-            *reinterpret_cast<uint2*>(a.out + orow * kD + lane * 4) = packed;
-            if (lane == 0) a.lse[orow] = Mx + __logf(D);
-        }
-        __syncwarp();
     }
+    const long long rowA = (static_cast<long long>(b) * s.Hq + gk * kG + hA) * s.R + tok;
+    const long long rowB = (static_cast<long long>(b) * s.Hq + gk * kG + hB) * s.R + tok;
+    uint4 pa, pb;
+    pa.x = pack_bf16(accA[0], accA[1]); pa.y = pack_bf16(accA[2], accA[3]);
+    pa.z = pack_bf16(accA[4], accA[5]); pa.w = pack_bf16(accA[6], accA[7]);
+    pb.x = pack_bf16(accB[0], accB[1]); pb.y = pack_bf16(accB[2], accB[3]);
+    pb.z = pack_bf16(accB[4], accB[5]); pb.w = pack_bf16(accB[6], accB[7]);
+    *reinterpret_cast<uint4*>(a.out + rowA * kD + piece * 8) = pa;
+    *reinterpret_cast<uint4*>(a.out + rowB * kD + piece * 8) = pb;
+    if (lane < kG) a.lse[(static_cast<long long>(b) * s.Hq + gk * kG + lane) * s.R + tok] = lse_h;
 }
 
 // HILS_FORCE_MMA_SELECT=1 keeps the warp-MMA selection kernel even where the tcgen05 one applies
@@ -641,7 +622,7 @@ const bool g_force_mma_select = [] {
 }();
 
 struct Plan {
-    int qb, max_tiles;
+    int qb, nc, max_tiles;
     size_t off_cnt, off_cursor, off_ntiles, zero_bytes, off_off, off_toff, off_entries, off_tiles, off_obuf, off_lam,
         total;
 };
@@ -651,19 +632,21 @@ Plan make_plan(const Shape& s) {
     const size_t pairs = static_cast<size_t>(s.B) * s.Hkv;
     const size_t blk = static_cast<size_t>(s.R < kQB ? (s.R + kS - 1) / kS * kS : kQB);
     p.qb = static_cast<int>(blk);
-    p.max_tiles = static_cast<int>(pairs * blk * s.K / kTileTok + pairs * s.C);
+    const size_t nc = static_cast<size_t>(s.C > (s.R + kS - 1) / kS ? s.C : (s.R + kS - 1) / kS);
+    p.nc = static_cast<int>(nc);
+    p.max_tiles = static_cast<int>(pairs * blk * (s.K + 1) / kTileTok + pairs * nc);
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = (off + bytes + 255) / 256 * 256; return o; };
-    p.off_cnt = take(sizeof(int) * pairs * s.C);
-    p.off_cursor = take(sizeof(int) * pairs * s.C);
+    p.off_cnt = take(sizeof(int) * pairs * nc);
+    p.off_cursor = take(sizeof(int) * pairs * nc);
     p.off_ntiles = take(256);
     p.zero_bytes = off;                         // cnt, cursor, n_tiles are cleared together per block
-    p.off_off = take(sizeof(int) * pairs * s.C);
-    p.off_toff = take(sizeof(int) * pairs * s.C);
-    p.off_entries = take(sizeof(int) * pairs * blk * s.K);
+    p.off_off = take(sizeof(int) * pairs * nc);
+    p.off_toff = take(sizeof(int) * pairs * nc);
+    p.off_entries = take(sizeof(int) * pairs * blk * (s.K + 1));
     p.off_tiles = take(sizeof(int4) * static_cast<size_t>(p.max_tiles));
-    p.off_obuf = take(sizeof(__nv_bfloat16) * pairs * blk * s.K * kG * kD);
-    p.off_lam = take(sizeof(float) * pairs * blk * kG * s.K);
+    p.off_obuf = take(sizeof(__nv_bfloat16) * pairs * blk * (s.K + 1) * kG * kD);
+    p.off_lam = take(sizeof(float) * pairs * blk * kG * (s.K + 1));
     p.total = off;
     return p;
 }
@@ -704,6 +687,7 @@ int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
     a.lam = reinterpret_cast<float*>(sc + p.off_lam);
     a.max_tiles = p.max_tiles;
     a.qb = p.qb;
+    a.nc = p.nc;
     a.i0 = 0;
     a.i1 = 0;
 
@@ -715,16 +699,13 @@ int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
 
     const size_t sel_smem = kSelStages * kSelStageBytes + 64 + sizeof(unsigned long long) * 64 * (s.K + 1) + 1024;
     const size_t att_smem = 32768 + 2048 + sizeof(AttSmem) + 1024;
-    const size_t fuse_smem = 32768 + sizeof(FuseSmem) + 1024;
     static bool attr_done = false;
     if (!attr_done) {
         const size_t sel_max = kSelStages * kSelStageBytes + 64 + sizeof(unsigned long long) * 64 * 65 + 1024;
         if (cudaFuncSetAttribute(prefill_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(sel_max)) != cudaSuccess ||
             cudaFuncSetAttribute(prefill_attend_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(att_smem)) != cudaSuccess ||
-            cudaFuncSetAttribute(prefill_fuse_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(fuse_smem)) != cudaSuccess)
+                                 static_cast<int>(att_smem)) != cudaSuccess)
             return HILS_ERR_CUDA;
         attr_done = true;
     }
@@ -746,7 +727,7 @@ int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
         a.i1 = s.R < i0 + kQB ? s.R : i0 + kQB;
         const int nblk = a.i1 - a.i0;
         if (cudaMemsetAsync(sc + p.off_cnt, 0, p.zero_bytes, stream) != cudaSuccess) return HILS_ERR_CUDA;
-        const long long elems = static_cast<long long>(pairs) * nblk * s.K;
+        const long long elems = static_cast<long long>(pairs) * nblk * (s.K + 1);
         const long long want = (elems + 255) / 256;
         const unsigned eb = static_cast<unsigned>(want < 148 * 16 ? want : 148 * 16);
         invert_count_kernel<<<eb, 256, 0, stream>>>(a);
@@ -757,8 +738,8 @@ int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
         prefill_attend_kernel<<<148 * 2, 128, att_smem, stream>>>(map_k, map_v, a);
         if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
         trace_mark("prefill_attend", stream);
-        const int chunks_blk = (nblk + kS - 1) / kS;
-        prefill_fuse_kernel<<<static_cast<unsigned>(pairs) * chunks_blk, 128, fuse_smem, stream>>>(map_k, map_v, a);
+        const long long fuse_warps = static_cast<long long>(pairs) * nblk;
+        prefill_fuse_kernel<<<static_cast<unsigned>((fuse_warps + kFuseWarps - 1) / kFuseWarps), kFuseWarps * 32, 0, stream>>>(a);
         if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
         trace_mark("prefill_fuse", stream);
         launches += 5;
