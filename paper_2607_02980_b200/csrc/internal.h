@@ -47,6 +47,12 @@ bool prefill_select_tc_supports(const Shape& s);
 int launch_prefill_select_tc(const Shape& s, const void* q, const void* landmarks, const float* bias, int32_t* sel,
                              int* status, cudaStream_t stream);
 
+// tcgen05 chunk-major attention over the tile table built by the invert kernels (32-token tiles).
+int attend_tc_tile_tokens();
+int launch_prefill_attend_tc(const Shape& s, const void* q, const void* k, const void* v, const void* landmarks,
+                             const float* bias, const int* entries, const void* tiles, const int* n_tiles, void* obuf,
+                             float* lam, int* status, int i0, int qb, cudaStream_t stream);
+
 int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream);
 bool prefill_fast_supports(const Shape& s, int dtype);
 size_t prefill_fast_scratch_bytes(const Shape& s);

@@ -1,0 +1,495 @@
+// Chunk-major gathered attention for prefill on tcgen05 tensor cores (bf16, d = 128, S = 64, G = 4).
+//
+// A tile is 32 (token, slot) entries of one chunk x 4 heads = 128 query rows (one TMEM lane each).
+// Per tile:  S = Q K_c^T (M=128, N=80: 64 keys + the chunk's landmark as key 64, K=128) -> tensor memory;
+//            each epilogue thread owns one row: mask (local rows are causal), the chunk's own softmax
+//            (Eq. HiLS weights, intra-chunk factor), P as bf16 back to shared memory;
+//            O = P V_c (M=128, N=128, K=64, V pre-transposed once per chunk) -> tensor memory;
+//            normalised bf16 rows and the row's chunk mass (surrogate score, or log Z_swa for the
+//            local branch) go to the buffers that prefill_fuse mixes.
+// Warp roles: 0-7 epilogue (warps 0-3 take even tiles, 4-7 odd tiles; a warp reads the TMEM lane quarter
+// warp % 4), 8-11 producers (cp.async gather of Q rows, TMA of K/V, V transpose), 12 MMA issue.
+// S/P/O are double buffered, three gathered Q tiles are in flight, K/V is double buffered per chunk.
+#include "internal.h"
+#include "tma.cuh"
+
+namespace hils {
+namespace {
+
+constexpr int kD = 128;
+constexpr int kS = 64;
+constexpr int kG = 4;
+constexpr int kTok = 32;                        // entries per tile
+constexpr int kRows = kTok * kG;                // 128
+constexpr int kNS = 80;                         // score columns: 64 keys + landmark (+15 zero rows)
+constexpr int kKBytes = kNS * 128 * 2;          // two 64-dim K-blocks of 80 rows
+constexpr int kVtBytes = kD * 128;              // 128 d-rows x 64 keys
+constexpr int kVrawBytes = kS * kD * 2;
+constexpr int kQBytes = kRows * kD * 2;         // 32 KB
+constexpr int kPBytes = kRows * 128;            // 16 KB
+constexpr int kBatch = 128;                     // tile records cached per batch
+constexpr int kQSlots = 3;                      // gathered Q tiles in flight
+constexpr int kMetaSlots = 8;                   // ring of tile descriptors (producers are < 8 tiles ahead of the epilogue)
+constexpr int kProdThreads = 128;
+constexpr int kEpiThreads = 256;
+constexpr int kThreads = kEpiThreads + kProdThreads + 32;
+constexpr int kProdWarp0 = kEpiThreads / 32;
+constexpr int kMmaWarp = kProdWarp0 + kProdThreads / 32;
+constexpr float kLog2e = 1.4426950408889634f;
+
+struct AtcSmem {
+    uint64_t kraw_full;       // TMA of K rows + raw V landed
+    uint64_t kv_ready[2];     // K tile (with landmark row) and transposed V usable by the MMA
+    uint64_t kv_empty[2];     // every MMA that reads this K/V buffer has completed
+    uint64_t q_full[kQSlots]; // gathered Q rows landed and fenced (one arrival per producer warp)
+    uint64_t q_empty[kQSlots];// the S MMA that reads this Q tile has completed
+    uint64_t s_full[2];       // S = Q K^T in tensor memory
+    uint64_t s_empty[2];      // epilogue has read S
+    uint64_t p_full[2];       // P written to shared memory and fenced
+    uint64_t o_full[2];       // O = P V in tensor memory
+    uint64_t o_empty[2];      // epilogue has read O
+    uint32_t tmem_base;
+    int abort_flag;
+    int tile_ent[kMetaSlots][kTok];   // entries of the tiles in flight
+    int tile_meta[kMetaSlots][4];     // pair, chunk, tokens, unused
+    const __nv_bfloat16* rowptr[2][kRows];
+    long long orow[2][kRows];         // obuf element offset of each row of the tile in S/P/O slot i (-1: padding)
+    int4 recs[kBatch];
+};
+
+struct AtcArgs {
+    Shape s;
+    const __nv_bfloat16* q;
+    const __nv_bfloat16* lm;
+    const float* bias;
+    const int* entries;
+    const int4* tiles;
+    const int* n_tiles;
+    __nv_bfloat16* obuf;
+    float* lam;
+    int* status;
+    int i0, qb;
+};
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ void producer_barrier() { asm volatile("bar.sync 2, %0;" ::"n"(kProdThreads) : "memory"); }
+
+__global__ void __launch_bounds__(kThreads, 1)
+prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                         const AtcArgs a) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* kbuf = base;                                   // [2][kKBytes]
+    uint8_t* vt = kbuf + 2 * kKBytes;                       // [2][kVtBytes]
+    uint8_t* vraw = vt + 2 * kVtBytes;                      // [kVrawBytes]
+    uint8_t* qbuf = vraw + kVrawBytes;                      // [kQSlots][kQBytes]
+    uint8_t* pbuf = qbuf + kQSlots * kQBytes;               // [2][kPBytes]
+    AtcSmem& sm = *reinterpret_cast<AtcSmem*>(pbuf + 2 * kPBytes);
+
+    const Shape& s = a.s;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int K1 = s.K + 1;
+    const int n_tiles = *a.n_tiles;
+    const long long lo = static_cast<long long>(blockIdx.x) * n_tiles / gridDim.x;
+    const long long hi = static_cast<long long>(blockIdx.x + 1) * n_tiles / gridDim.x;
+
+    if (tid == 0) {
+        mbar_init(&sm.kraw_full, 1);
+        for (int i = 0; i < kQSlots; ++i) { mbar_init(&sm.q_full[i], 4); mbar_init(&sm.q_empty[i], 1); }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&sm.kv_ready[i], 1);
+            mbar_init(&sm.kv_empty[i], 1);
+            mbar_init(&sm.s_full[i], 1);
+            mbar_init(&sm.s_empty[i], 4);
+            mbar_init(&sm.p_full[i], 4);
+            mbar_init(&sm.o_full[i], 1);
+            mbar_init(&sm.o_empty[i], 4);
+        }
+        mbar_fence_init();
+        sm.abort_flag = 0;
+        tma_prefetch_desc(&map_k);
+        tma_prefetch_desc(&map_v);
+    }
+    // rows 64..79 of both K-blocks of both K buffers: landmark row + zero rows (TMA never writes them)
+    for (int x = tid; x < 2 * 2 * 16 * 8; x += kThreads) {
+        const int bufi = x >> 8, kb = (x >> 7) & 1, row = 64 + ((x >> 3) & 15), pc = x & 7;
+        *reinterpret_cast<uint4*>(kbuf + bufi * kKBytes + kb * (kNS * 128) + swz128(row, pc)) = make_uint4(0u, 0u, 0u, 0u);
+    }
+    if (warp == kMmaWarp) tmem_alloc(&sm.tmem_base, 512);
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = sm.tmem_base;
+
+    // running counters (identical in every role): tiles and chunk loads processed so far by this CTA
+    uint32_t tcount = 0, ccount = 0;
+
+    for (long long b0 = lo; b0 < hi; b0 += kBatch) {
+        const int nb = static_cast<int>(min(static_cast<long long>(kBatch), hi - b0));
+        for (int x = tid; x < nb; x += kThreads) sm.recs[x] = a.tiles[b0 + x];
+        __syncthreads();
+        if (sm.abort_flag) break;
+
+        if (warp >= kProdWarp0 && warp < kMmaWarp) {
+            // ================================================================ producers (128 threads)
+            const int ptid = tid - kEpiThreads, pw = warp - kProdWarp0;
+            uint32_t tc = tcount, cc = ccount;
+            int cur_pair = -1, cur_c = -1;
+            bool next_issued = false;          // (producer thread 0) K/V of the upcoming chunk already requested
+            bool dead = false;
+            // entry of this thread's row for the upcoming tile, fetched one tile ahead
+            int e_next = a.entries[sm.recs[0].z + min(ptid >> 2, sm.recs[0].w - 1)];
+            int e_next2 = nb > 1 ? a.entries[sm.recs[1].z + min(ptid >> 2, sm.recs[1].w - 1)] : 0;
+            for (int ti = 0; ti < nb; ++ti) {
+                const int4 rec = sm.recs[ti];
+                const int pair = rec.x, c = rec.y, ntok = rec.w;
+                const int e = e_next;
+                e_next = e_next2;
+                if (ti + 2 < nb) e_next2 = a.entries[sm.recs[ti + 2].z + min(ptid >> 2, sm.recs[ti + 2].w - 1)];
+                if (pair != cur_pair || c != cur_c) {
+                    // ---- new chunk: make its K/V usable
+                    const uint32_t cbuf = cc & 1u;
+                    if (ptid == 0 && !next_issued) {
+                        if (cc >= 2 && !mbar_wait(&sm.kv_empty[cbuf], ((cc >> 1) - 1) & 1)) dead = true;
+                        if (!dead) {
+                            const int row = pair * s.T + c * kS;
+                            mbar_expect_tx(&sm.kraw_full, 2 * 8192 + kVrawBytes);
+                            tma_load_2d(kbuf + cbuf * kKBytes, &map_k, &sm.kraw_full, 0, row);
+                            tma_load_2d(kbuf + cbuf * kKBytes + kNS * 128, &map_k, &sm.kraw_full, 64, row);
+                            tma_load_2d(vraw, &map_v, &sm.kraw_full, 0, row);
+                            tma_load_2d(vraw + 8192, &map_v, &sm.kraw_full, 64, row);
+                        }
+                    }
+                    next_issued = false;
+                    if (!dead && !mbar_wait(&sm.kraw_full, cc & 1)) dead = true;
+                    if (dead) break;
+                    // landmark row (key 64) of both K-blocks
+                    if (ptid < 16) {
+                        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                        if (c < s.C) v = *reinterpret_cast<const uint4*>(a.lm + (static_cast<long long>(pair) * s.C + c) * kD + ptid * 8);
+                        *reinterpret_cast<uint4*>(kbuf + cbuf * kKBytes + (ptid >> 3) * (kNS * 128) + swz128(64, ptid & 7)) = v;
+                    }
+                    // V^T: 8x8 blocks through ldmatrix.trans (8 of the 32 blocks per warp); keys past the
+                    // end of the sequence become 0
+                    const int nv = min(kS, s.R - c * kS);
+                    uint8_t* vtb = vt + cbuf * kVtBytes;
+                    const uint32_t vraw_addr = smem_u32(vraw);
+#pragma unroll 2
+                    for (int bi = 0; bi < 8; ++bi) {
+                        const int blk = pw * 8 + bi;
+                        // block = 16 keys x 16 dims: four 8x8 matrices (keys lo/hi x dims lo/hi)
+                        const int k0 = (blk & 3) * 16, d0 = (blk >> 2) * 16;
+                        const int mat = lane >> 3;
+                        const int row = k0 + (mat & 1) * 8 + (lane & 7);
+                        const int dim = d0 + (mat >> 1) * 8;
+                        uint32_t r0, r1, r2, r3;
+                        ldmatrix_x4_trans(vraw_addr + (dim >> 6) * 8192 + swz128(row, (dim & 63) >> 3), r0, r1, r2, r3);
+                        // thread (g,t): r0 = V[k0+2t..+1][d0+g], r1 = V[k0+8+2t..][d0+g], r2/r3: dims d0+8+g
+                        const int g = lane >> 2, t = lane & 3;
+                        const uint32_t vals[4] = {r0, r1, r2, r3};
+#pragma unroll
+                        for (int m = 0; m < 4; ++m) {
+                            const int dd = d0 + (m >> 1) * 8 + g;
+                            const int key = k0 + (m & 1) * 8 + 2 * t;
+                            uint32_t v = vals[m];
+                            if (key >= nv) v = 0u;
+                            else if (key + 1 >= nv) v &= 0x0000ffffu;
+                            *reinterpret_cast<uint32_t*>(vtb + swz128(dd, key >> 3) + (key & 7) * 2) = v;
+                        }
+                    }
+                    fence_proxy_async_smem();
+                    producer_barrier();
+                    if (ptid == 0) mbar_arrive(&sm.kv_ready[cbuf]);
+                    cur_pair = pair;
+                    cur_c = c;
+                    ++cc;
+                }
+                // ---- look ahead (producer thread 0): request the next chunk's K/V as soon as its buffer is free
+                if (ptid == 0 && !next_issued) {
+                    int tj = ti + 1;
+                    while (tj < nb && sm.recs[tj].x == pair && sm.recs[tj].y == c) ++tj;
+                    const uint32_t nbuf = cc & 1u;
+                    if (tj < nb && (cc < 2 || mbar_try_wait(&sm.kv_empty[nbuf], ((cc >> 1) - 1) & 1))) {
+                        const int row = sm.recs[tj].x * s.T + sm.recs[tj].y * kS;
+                        mbar_expect_tx(&sm.kraw_full, 2 * 8192 + kVrawBytes);
+                        tma_load_2d(kbuf + nbuf * kKBytes, &map_k, &sm.kraw_full, 0, row);
+                        tma_load_2d(kbuf + nbuf * kKBytes + kNS * 128, &map_k, &sm.kraw_full, 64, row);
+                        tma_load_2d(vraw, &map_v, &sm.kraw_full, 0, row);
+                        tma_load_2d(vraw + 8192, &map_v, &sm.kraw_full, 64, row);
+                        next_issued = true;
+                    }
+                }
+                // ---- gather the tile's 128 query rows (token-major, head-minor) into the swizzled Q tile
+                const uint32_t qs = tc % kQSlots, ms = tc % kMetaSlots, rb = tc & 1u;
+                if (tc >= kQSlots && !mbar_wait(&sm.q_empty[qs], ((tc / kQSlots) - 1) & 1)) { dead = true; break; }
+                {
+                    // thread ptid owns row ptid for the address table
+                    const int tk = ptid >> 2, hd = ptid & 3;
+                    const int bb = pair / s.Hkv, gk = pair % s.Hkv;
+                    sm.rowptr[rb][ptid] = a.q + ((static_cast<long long>(bb) * s.Hq + gk * kG + hd) * s.R + a.i0 + (e >> 8)) * kD;
+                    if (hd == 0) sm.tile_ent[ms][tk] = e;
+                    if (ptid == 0) { sm.tile_meta[ms][0] = pair; sm.tile_meta[ms][1] = c; sm.tile_meta[ms][2] = ntok; }
+                    producer_barrier();
+                    const uint32_t qaddr = smem_u32(qbuf + qs * kQBytes);
+                    const int p16 = lane & 15;
+                    const uint32_t koff = (p16 >> 3) * 16384;
+                    // all 16 source addresses first, then the 16 copies back to back
+                    const __nv_bfloat16* src[16];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) src[j] = sm.rowptr[rb][pw * 32 + 2 * j + (lane >> 4)] + p16 * 8;
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const int row = pw * 32 + 2 * j + (lane >> 4);       // a half-warp copies one 256-byte row
+                        cp_async16(qaddr + koff + swz128(row, p16 & 7), src[j]);
+                    }
+                    cp_async_commit();
+                }
+                // the previous tile's rows have landed by now: publish them
+                if (tc > tcount) {
+                    cp_async_wait<1>();
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sm.q_full[(tc - 1) % kQSlots]);
+                }
+                ++tc;
+            }
+            cp_async_wait<0>();
+            if (tc > tcount && !dead) {
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.q_full[(tc - 1) % kQSlots]);
+            }
+            if (dead && lane == 0) { set_status(a.status, kDevTimeout); atomicExch(&sm.abort_flag, 1); }
+            if (ptid == 0 && next_issued) mbar_wait(&sm.kraw_full, cc & 1);       // own copy in flight: let it land
+        } else if (warp == kMmaWarp) {
+            // ================================================================ MMA issuer
+            if (lane == 0) {
+                constexpr uint32_t idesc_s = umma_idesc_bf16(kRows, kNS);
+                constexpr uint32_t idesc_o = umma_idesc_bf16(kRows, kD);
+                uint32_t cc = ccount;
+                int cur_pair = -1, cur_c = -1;
+                uint32_t cbuf_of[2] = {0u, 0u};        // K/V buffer used by the tile in S/P/O slot i
+                bool ok = true;
+                // Two in-order queues (S MMAs, O MMAs) served by polling: an O MMA whose probabilities are
+                // ready is never held up by a Q tile that has not arrived yet, and vice versa.
+                int ns = 0, no = 0;                    // next tile (batch index) to issue S / O for
+                uint32_t idle = 0;
+                while (no < nb && ok) {
+                    bool progressed = false;
+                    if (ns < nb && ns < no + 2) {
+                        const uint32_t tcv = tcount + ns, sl = tcv & 1u, qs = tcv % kQSlots;
+                        const int4 rec = sm.recs[ns];
+                        const bool newc = rec.x != cur_pair || rec.y != cur_c;
+                        bool ready = mbar_try_wait(&sm.q_full[qs], (tcv / kQSlots) & 1);
+                        if (ready && newc) ready = mbar_try_wait(&sm.kv_ready[cc & 1u], (cc >> 1) & 1);
+                        if (ready && tcv >= 2) ready = mbar_try_wait(&sm.s_empty[sl], ((tcv >> 1) - 1) & 1);
+                        if (ready) {
+                            if (newc) { cur_pair = rec.x; cur_c = rec.y; ++cc; }
+                            const uint32_t cb = (cc - 1) & 1u;
+                            cbuf_of[sl] = cb;
+                            tc_fence_after_sync();
+                            const uint32_t qa = smem_u32(qbuf + qs * kQBytes), ka = smem_u32(kbuf + cb * kKBytes);
+#pragma unroll
+                            for (int ks = 0; ks < 8; ++ks)
+                                umma_bf16(tmem_base + sl * 128, umma_desc_k128(qa + (ks >> 2) * 16384 + (ks & 3) * 32),
+                                          umma_desc_k128(ka + (ks >> 2) * (kNS * 128) + (ks & 3) * 32), idesc_s, ks > 0 ? 1u : 0u);
+                            umma_commit(&sm.s_full[sl]);
+                            umma_commit(&sm.q_empty[qs]);
+                            ++ns;
+                            progressed = true;
+                        }
+                    }
+                    if (no < ns) {
+                        const uint32_t tcv = tcount + no, sl = tcv & 1u, cb = cbuf_of[sl];
+                        bool ready = mbar_try_wait(&sm.p_full[sl], (tcv >> 1) & 1);
+                        if (ready && tcv >= 2) ready = mbar_try_wait(&sm.o_empty[sl], ((tcv >> 1) - 1) & 1);
+                        if (ready) {
+                            tc_fence_after_sync();
+                            const uint32_t pa = smem_u32(pbuf + sl * kPBytes), va = smem_u32(vt + cb * kVtBytes);
+#pragma unroll
+                            for (int ks = 0; ks < 4; ++ks)
+                                umma_bf16(tmem_base + 256 + sl * 128, umma_desc_k128(pa + ks * 32), umma_desc_k128(va + ks * 32),
+                                          idesc_o, ks > 0 ? 1u : 0u);
+                            umma_commit(&sm.o_full[sl]);
+                            // last tile of its chunk in this batch: the K/V buffer is free once these MMAs are done
+                            const bool last = no + 1 >= nb || sm.recs[no + 1].x != sm.recs[no].x || sm.recs[no + 1].y != sm.recs[no].y;
+                            if (last) umma_commit(&sm.kv_empty[cb]);
+                            ++no;
+                            progressed = true;
+                        }
+                    }
+                    if (progressed) {
+                        idle = 0;
+                    } else {
+                        if (++idle > kSpinLimit) ok = false;          // bounded: give up instead of hanging
+                        if (idle > 64) __nanosleep(idle > 4096 ? 256 : 32);
+                    }
+                }
+                if (!ok) { set_status(a.status, kDevTimeout); atomicExch(&sm.abort_flag, 1); }
+            }
+        } else {
+            // ================================================================ epilogue: one row per thread
+            const int grp = warp >> 2;                       // tiles of parity grp, S/P/O slot grp
+            const int row = (warp & 3) * 32 + lane;
+            const int tk = row >> 2, hd = row & 3;
+            const uint32_t t_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+            const float sl2 = s.scale * kLog2e;
+            const uint32_t sl = static_cast<uint32_t>(grp);
+            uint8_t* pslot = pbuf + sl * kPBytes;
+            bool ok = true;
+            for (int ti = 0; ti < nb && ok; ++ti) {
+                const uint32_t tcv = tcount + ti;
+                if ((tcv & 1u) != sl) continue;
+                // ---------------- scores -> probabilities
+                ok = mbar_wait(&sm.s_full[sl], (tcv >> 1) & 1);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t ms = tcv % kMetaSlots;
+                const int pair = sm.tile_meta[ms][0], c = sm.tile_meta[ms][1], ntok = sm.tile_meta[ms][2];
+                const int e = sm.tile_ent[ms][tk];
+                const int il = e >> 8, slot = e & 255;
+                const bool local = slot == s.K;
+                const int lim = local ? a.i0 + il - c * kS : kS - 1;        // last visible key of the chunk
+                float zi;
+                {
+                    float v[64];
+                    tmem_ld64(t_lane + sl * 128, v);
+                    const float lmk = tmem_ld1(t_lane + sl * 128 + 64);
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sm.s_empty[sl]);
+                    float m = -INFINITY;
+                    if (__any_sync(kFullMask, local)) {
+#pragma unroll
+                        for (int j = 0; j < 64; ++j) {
+                            if (j > lim) v[j] = -INFINITY;
+                            m = fmaxf(m, v[j]);
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 64; ++j) m = fmaxf(m, v[j]);
+                    }
+                    float z = 0.f;
+                    const float ms2 = m * sl2;
+#pragma unroll
+                    for (int pc = 0; pc < 8; ++pc) {
+                        uint32_t pk[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const float p0 = ex2_approx(fmaf(v[pc * 8 + 2 * j], sl2, -ms2));
+                            const float p1 = ex2_approx(fmaf(v[pc * 8 + 2 * j + 1], sl2, -ms2));
+                            z += p0 + p1;
+                            pk[j] = pack_bf16(p0, p1);
+                        }
+                        *reinterpret_cast<uint4*>(pslot + swz128(row, pc)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    }
+                    zi = 1.f / z;
+                    const bool real = tk < ntok;
+                    sm.orow[sl][row] = real ? (((static_cast<long long>(pair) * a.qb + il) * K1 + slot) * kG + hd) * kD : -1;
+                    if (real) {
+                        const float bb = (a.bias && c < s.C) ? a.bias[static_cast<long long>(pair) * s.C + c] : 0.f;
+                        a.lam[((static_cast<long long>(pair) * a.qb + il) * kG + hd) * K1 + slot] =
+                            local ? m * s.scale + __logf(z) : lmk * s.scale + bb;
+                    }
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.p_full[sl]);
+                // ---------------- O = P V -> normalised bf16 rows
+                ok = mbar_wait(&sm.o_full[sl], (tcv >> 1) & 1);
+                if (!ok) break;
+                tc_fence_after_sync();
+                // P has been consumed: its slot stages the output, 64 columns (128 bytes per row) at a time,
+                // so that every store instruction writes four full 128-byte segments
+                long long offs[8];
+#pragma unroll
+                for (int it = 0; it < 8; ++it) offs[it] = sm.orow[sl][(warp & 3) * 32 + it * 4 + (lane >> 3)];
+#pragma unroll 1
+                for (int hb = 0; hb < 2; ++hb) {
+                    {
+                        float v[64];
+                        tmem_ld64(t_lane + 256 + sl * 128 + hb * 64, v);
+#pragma unroll
+                        for (int pc = 0; pc < 8; ++pc) {
+                            uint32_t pk[4];
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) pk[j] = pack_bf16(v[pc * 8 + 2 * j] * zi, v[pc * 8 + 2 * j + 1] * zi);
+                            *reinterpret_cast<uint4*>(pslot + swz128(row, pc)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        }
+                    }
+                    __syncwarp();
+#pragma unroll
+                    for (int it = 0; it < 8; ++it) {
+                        const int r = (warp & 3) * 32 + it * 4 + (lane >> 3), pc = lane & 7;
+                        const long long off = offs[it];
+                        if (off >= 0)      // streaming store: written once, read once by prefill_fuse
+                            __stcs(reinterpret_cast<uint4*>(a.obuf + off + hb * 64 + pc * 8),
+                                   *reinterpret_cast<const uint4*>(pslot + swz128(r, pc)));
+                    }
+                    __syncwarp();
+                }
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.o_empty[sl]);
+            }
+            if (!ok && lane == 0) { set_status(a.status, kDevTimeout); atomicExch(&sm.abort_flag, 1); }
+        }
+        // every role advances the shared counters identically
+        {
+            uint32_t chunks = 0;
+            int cp = -1, cq = -1;
+            for (int ti = 0; ti < nb; ++ti)
+                if (sm.recs[ti].x != cp || sm.recs[ti].y != cq) { ++chunks; cp = sm.recs[ti].x; cq = sm.recs[ti].y; }
+            tcount += static_cast<uint32_t>(nb);
+            ccount += chunks;
+        }
+        __syncthreads();
+        if (sm.abort_flag) break;
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    if (warp == kMmaWarp) tmem_dealloc(tmem_base, 512);
+}
+
+}  // namespace
+
+int attend_tc_tile_tokens() { return kTok; }
+
+int launch_prefill_attend_tc(const Shape& s, const void* q, const void* k, const void* v, const void* landmarks,
+                             const float* bias, const int* entries, const void* tiles, const int* n_tiles, void* obuf,
+                             float* lam, int* status, int i0, int qb, cudaStream_t stream) {
+    const int pairs = s.B * s.Hkv;
+    CUtensorMap map_k, map_v;
+    const uint64_t kv_rows = static_cast<uint64_t>(pairs) * s.T;
+    if (!make_bf16_2d_map(&map_k, k, kv_rows, kD, 64, kS) || !make_bf16_2d_map(&map_v, v, kv_rows, kD, 64, kS))
+        return HILS_ERR_CUDA;
+    const size_t smem = 2 * kKBytes + 2 * kVtBytes + kVrawBytes + kQSlots * kQBytes + 2 * kPBytes + sizeof(AtcSmem) + 1024;
+    static bool attr_done = false;
+    if (!attr_done) {
+        if (cudaFuncSetAttribute(prefill_attend_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(smem)) != cudaSuccess)
+            return HILS_ERR_CUDA;
+        attr_done = true;
+    }
+    AtcArgs a{s, static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(landmarks), bias, entries,
+              static_cast<const int4*>(tiles), n_tiles, static_cast<__nv_bfloat16*>(obuf), lam, status, i0, qb};
+    prefill_attend_tc_kernel<<<148, kThreads, smem, stream>>>(map_k, map_v, a);
+    if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
+    return 1;
+}
+
+}  // namespace hils

@@ -23,7 +23,9 @@ namespace {
 constexpr int kD = 128;
 constexpr int kS = 64;
 constexpr int kG = 4;
-constexpr int kQB = 8192;                    // tokens per pass of the invert/attend/fuse phases
+constexpr int kQB = 4096;                    // tokens per pass of the invert/attend/fuse phases: the block's
+                                             // queries (QB x 32 heads x 256 B = 32 MB) stay L2-resident while
+                                             // they are gathered once per selected chunk
 constexpr int kTileTok = 16;                 // tokens per attend tile (x 4 heads = 64 MMA rows)
 constexpr int kSelStages = 3;
 constexpr int kSelStageBytes = kS * kD * 2;  // 64 landmark rows
@@ -52,6 +54,7 @@ struct PArgs {
     int i0, i1;             // token block [i0, i1)
     int qb;                 // tokens per block the obuf / lam strides are sized for
     int nc;                 // chunk slots per pair in cnt/off/...: max(C, ceil(L / S))
+    int tile_tok;           // entries per attend tile: 32 (tcgen05 kernel) or 16 (warp-MMA kernel)
     int max_tiles;
 };
 
@@ -273,7 +276,7 @@ __global__ void __launch_bounds__(1024) invert_scan_kernel(const PArgs a) {
     for (int base = 0; base < n; base += 1024) {
         const int x = base + tid;
         const int ce = x < n ? a.cnt[x] : 0;
-        const int ct = (ce + kTileTok - 1) / kTileTok;
+        const int ct = (ce + a.tile_tok - 1) / a.tile_tok;
         int ie = ce, it = ct;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -291,7 +294,7 @@ __global__ void __launch_bounds__(1024) invert_scan_kernel(const PArgs a) {
             const int pair = x / a.nc, c = x % a.nc;
             for (int k = 0; k < ct; ++k)
                 if (ot + k < a.max_tiles)
-                    a.tiles[ot + k] = make_int4(pair, c, oe + k * kTileTok, min(kTileTok, ce - k * kTileTok));
+                    a.tiles[ot + k] = make_int4(pair, c, oe + k * a.tile_tok, min(a.tile_tok, ce - k * a.tile_tok));
         }
         __syncthreads();
         if (tid == 1023) { carry_e = oe + ce; carry_t = ot + ct; }
@@ -580,8 +583,8 @@ __global__ void __launch_bounds__(kFuseWarps * 32) prefill_fuse_kernel(const PAr
     // local slot first, then the selected slots four at a time (8 loads in flight per lane)
     {
         const __nv_bfloat16* row = ob + static_cast<long long>(K) * kG * kD;
-        const uint4 ra = __ldg(reinterpret_cast<const uint4*>(row + lane * 8));
-        const uint4 rb = __ldg(reinterpret_cast<const uint4*>(row + 256 + lane * 8));
+        const uint4 ra = __ldcs(reinterpret_cast<const uint4*>(row + lane * 8));
+        const uint4 rb = __ldcs(reinterpret_cast<const uint4*>(row + 256 + lane * 8));
         fma8(accA, ra, wv[hA][64]);
         fma8(accB, rb, wv[hB][64]);
     }
@@ -591,8 +594,8 @@ __global__ void __launch_bounds__(kFuseWarps * 32) prefill_fuse_kernel(const PAr
         for (int u = 0; u < 4; ++u) {
             const int sl = min(sl0 + u, nsel - 1);
             const __nv_bfloat16* row = ob + static_cast<long long>(sl) * kG * kD;
-            ra[u] = __ldg(reinterpret_cast<const uint4*>(row + lane * 8));
-            rb[u] = __ldg(reinterpret_cast<const uint4*>(row + 256 + lane * 8));
+            ra[u] = __ldcs(reinterpret_cast<const uint4*>(row + lane * 8));
+            rb[u] = __ldcs(reinterpret_cast<const uint4*>(row + 256 + lane * 8));
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
@@ -614,10 +617,14 @@ __global__ void __launch_bounds__(kFuseWarps * 32) prefill_fuse_kernel(const PAr
     if (lane < kG) a.lse[(static_cast<long long>(b) * s.Hq + gk * kG + lane) * s.R + tok] = lse_h;
 }
 
-// HILS_FORCE_MMA_SELECT=1 keeps the warp-MMA selection kernel even where the tcgen05 one applies
-// (used to cross-check the two).
+// HILS_FORCE_MMA_SELECT=1 / HILS_FORCE_MMA_ATTEND=1 keep the warp-MMA kernels even where the tcgen05
+// ones apply (used to cross-check the two implementations).
 const bool g_force_mma_select = [] {
     const char* e = getenv("HILS_FORCE_MMA_SELECT");
+    return e != nullptr && e[0] == '1';
+}();
+const bool g_force_mma_attend = [] {
+    const char* e = getenv("HILS_FORCE_MMA_ATTEND");
     return e != nullptr && e[0] == '1';
 }();
 
@@ -688,6 +695,7 @@ int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
     a.max_tiles = p.max_tiles;
     a.qb = p.qb;
     a.nc = p.nc;
+    a.tile_tok = g_force_mma_attend ? kTileTok : attend_tc_tile_tokens();
     a.i0 = 0;
     a.i1 = 0;
 
@@ -735,8 +743,14 @@ int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
         invert_fill_kernel<<<eb, 256, 0, stream>>>(a);
         if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
         trace_mark("prefill_invert", stream);
-        prefill_attend_kernel<<<148 * 2, 128, att_smem, stream>>>(map_k, map_v, a);
-        if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
+        if (g_force_mma_attend) {
+            prefill_attend_kernel<<<148 * 2, 128, att_smem, stream>>>(map_k, map_v, a);
+            if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
+        } else {
+            const int rc = launch_prefill_attend_tc(s, t.q, t.k, t.v, t.landmarks, t.bias, a.entries, a.tiles, a.n_tiles,
+                                                    a.obuf, a.lam, t.status, a.i0, a.qb, stream);
+            if (rc < 0) return rc;
+        }
         trace_mark("prefill_attend", stream);
         const long long fuse_warps = static_cast<long long>(pairs) * nblk;
         prefill_fuse_kernel<<<static_cast<unsigned>((fuse_warps + kFuseWarps - 1) / kFuseWarps), kFuseWarps * 32, 0, stream>>>(a);
