@@ -100,9 +100,10 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
     const Shape& s = a.s;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int K1 = s.K + 1;
-    const int n_tiles = *a.n_tiles;
-    const long long lo = static_cast<long long>(blockIdx.x) * n_tiles / gridDim.x;
-    const long long hi = static_cast<long long>(blockIdx.x + 1) * n_tiles / gridDim.x;
+    // a.n_tiles points at {first tile of this query block, first tile of the next one}
+    const int t_begin = a.n_tiles[0], n_tiles = a.n_tiles[1] - t_begin;
+    const long long lo = t_begin + static_cast<long long>(blockIdx.x) * n_tiles / gridDim.x;
+    const long long hi = t_begin + static_cast<long long>(blockIdx.x + 1) * n_tiles / gridDim.x;
 
     if (tid == 0) {
         mbar_init(&sm.kraw_full, 1);

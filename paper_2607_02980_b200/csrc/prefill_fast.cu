@@ -23,7 +23,7 @@ namespace {
 constexpr int kD = 128;
 constexpr int kS = 64;
 constexpr int kG = 4;
-constexpr int kQB = 4096;                    // tokens per pass of the invert/attend/fuse phases: the block's
+constexpr int kQBDefault = 4096;             // tokens per pass of the invert/attend/fuse phases: the block's
                                              // queries (QB x 32 heads x 256 B = 32 MB) stay L2-resident while
                                              // they are gathered once per selected chunk
 constexpr int kTileTok = 16;                 // tokens per attend tile (x 4 heads = 64 MMA rows)
@@ -41,9 +41,9 @@ struct PArgs {
     int32_t* sel;
     int* status;
     // scratch (per token block)
-    int* cnt;               // [pairs*nc] rows of each (pair, chunk) in the block: selectors + own tokens
+    int* cnt;               // [n_blocks*pairs*nc] rows of each (block, pair, chunk): selectors + own tokens
     int* cursor;            // [pairs*C]
-    int* n_tiles;           // [1] (+ padding)
+    int* blk_toff;          // [n_blocks + 1] first tile of every query block (tiles are grouped by block)
     int* off;               // [pairs*C] exclusive prefix of cnt
     int* toff;              // [pairs*C] exclusive prefix of tiles per (pair, chunk)
     int* entries;           // [pairs*QB*(K+1)] (token_local << 8) | slot, grouped by (pair, chunk);
@@ -51,7 +51,9 @@ struct PArgs {
     int4* tiles;            // [max_tiles] {pair, chunk, first entry, rows}
     __nv_bfloat16* obuf;    // [pairs*QB*(K+1)][G][128] normalised per-chunk outputs (slot K: local)
     float* lam;             // [pairs*QB][G][K+1] per-head surrogate scores; slot K: log Z_swa
-    int i0, i1;             // token block [i0, i1)
+    int i0, i1;             // token block [i0, i1) of the attend / fuse launch
+    int blk;                // its index
+    int n_blocks;           // query blocks of qb tokens
     int qb;                 // tokens per block the obuf / lam strides are sized for
     int nc;                 // chunk slots per pair in cnt/off/...: max(C, ceil(L / S))
     int tile_tok;           // entries per attend tile: 32 (tcgen05 kernel) or 16 (warp-MMA kernel)
@@ -245,22 +247,22 @@ prefill_select_kernel(const __grid_constant__ CUtensorMap map_lm, const PArgs a)
 
 // ------------------------------------------------------------------------------------------ invert
 // Chunk attended by slot `slot` of token i0+il: a selected chunk, or (slot K) the token's own chunk.
-__device__ __forceinline__ int slot_chunk(const PArgs& a, int pair, int il, int slot) {
-    if (slot == a.s.K) return (a.i0 + il) / kS;
-    return a.sel[(static_cast<long long>(pair) * a.s.R + a.i0 + il) * a.s.K + slot];
+__device__ __forceinline__ int slot_chunk(const PArgs& a, int pair, int tok, int slot) {
+    if (slot == a.s.K) return tok / kS;
+    return a.sel[(static_cast<long long>(pair) * a.s.R + tok) * a.s.K + slot];
 }
 
 __global__ void invert_count_kernel(const PArgs a) {
     const Shape& s = a.s;
-    const int K1 = s.K + 1, nblk = a.i1 - a.i0;
-    const long long total = static_cast<long long>(s.B) * s.Hkv * nblk * K1;
+    const int K1 = s.K + 1, pairs = s.B * s.Hkv;
+    const long long total = static_cast<long long>(pairs) * s.R * K1;
     for (long long x = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; x < total;
          x += static_cast<long long>(gridDim.x) * blockDim.x) {
         const int slot = static_cast<int>(x % K1);
-        const int il = static_cast<int>((x / K1) % nblk);
-        const int pair = static_cast<int>(x / (static_cast<long long>(K1) * nblk));
-        const int c = slot_chunk(a, pair, il, slot);
-        if (c >= 0) atomicAdd(&a.cnt[pair * a.nc + c], 1);
+        const int tok = static_cast<int>((x / K1) % s.R);
+        const int pair = static_cast<int>(x / (static_cast<long long>(K1) * s.R));
+        const int c = slot_chunk(a, pair, tok, slot);
+        if (c >= 0) atomicAdd(&a.cnt[(static_cast<long long>(tok / a.qb) * pairs + pair) * a.nc + c], 1);
     }
 }
 
@@ -269,7 +271,8 @@ __global__ void __launch_bounds__(1024) invert_scan_kernel(const PArgs a) {
     __shared__ int wsum_e[32], wsum_t[32];
     __shared__ int carry_e, carry_t;
     const Shape& s = a.s;
-    const int n = s.B * s.Hkv * a.nc;
+    const int per_blk = s.B * s.Hkv * a.nc;
+    const int n = per_blk * a.n_blocks;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (tid == 0) { carry_e = 0; carry_t = 0; }
     __syncthreads();
@@ -291,7 +294,8 @@ __global__ void __launch_bounds__(1024) invert_scan_kernel(const PArgs a) {
         if (x < n) {
             a.off[x] = oe;
             a.toff[x] = ot;
-            const int pair = x / a.nc, c = x % a.nc;
+            const int pair = (x % per_blk) / a.nc, c = x % a.nc;
+            if (x % per_blk == 0) a.blk_toff[x / per_blk] = ot;
             for (int k = 0; k < ct; ++k)
                 if (ot + k < a.max_tiles)
                     a.tiles[ot + k] = make_int4(pair, c, oe + k * a.tile_tok, min(a.tile_tok, ce - k * a.tile_tok));
@@ -300,23 +304,23 @@ __global__ void __launch_bounds__(1024) invert_scan_kernel(const PArgs a) {
         if (tid == 1023) { carry_e = oe + ce; carry_t = ot + ct; }
         __syncthreads();
     }
-    if (tid == 0) *a.n_tiles = min(carry_t, a.max_tiles);
+    if (tid == 0) a.blk_toff[a.n_blocks] = min(carry_t, a.max_tiles);
 }
 
 __global__ void invert_fill_kernel(const PArgs a) {
     const Shape& s = a.s;
-    const int K1 = s.K + 1, nblk = a.i1 - a.i0;
-    const long long total = static_cast<long long>(s.B) * s.Hkv * nblk * K1;
+    const int K1 = s.K + 1, pairs = s.B * s.Hkv;
+    const long long total = static_cast<long long>(pairs) * s.R * K1;
     for (long long x = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; x < total;
          x += static_cast<long long>(gridDim.x) * blockDim.x) {
         const int slot = static_cast<int>(x % K1);
-        const int il = static_cast<int>((x / K1) % nblk);
-        const int pair = static_cast<int>(x / (static_cast<long long>(K1) * nblk));
-        const int c = slot_chunk(a, pair, il, slot);
+        const int tok = static_cast<int>((x / K1) % s.R);
+        const int pair = static_cast<int>(x / (static_cast<long long>(K1) * s.R));
+        const int c = slot_chunk(a, pair, tok, slot);
         if (c >= 0) {
-            const int idx = pair * a.nc + c;
+            const long long idx = (static_cast<long long>(tok / a.qb) * pairs + pair) * a.nc + c;
             const int pos = a.off[idx] + atomicAdd(&a.cursor[idx], 1);
-            a.entries[pos] = (il << 8) | slot;
+            a.entries[pos] = ((tok % a.qb) << 8) | slot;
         }
     }
 }
@@ -395,9 +399,9 @@ prefill_attend_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_co
     const int g = lane >> 2, t = lane & 3;
     const int K = s.K;
     const float sl2 = s.scale * kLog2e;
-    const int n_tiles = *a.n_tiles;
-    const long long lo = static_cast<long long>(blockIdx.x) * n_tiles / gridDim.x;
-    const long long hi = static_cast<long long>(blockIdx.x + 1) * n_tiles / gridDim.x;
+    const int t_begin = a.blk_toff[a.blk], n_tiles = a.blk_toff[a.blk + 1] - t_begin;
+    const long long lo = t_begin + static_cast<long long>(blockIdx.x) * n_tiles / gridDim.x;
+    const long long hi = t_begin + static_cast<long long>(blockIdx.x + 1) * n_tiles / gridDim.x;
 
     if (tid == 0) { mbar_init(&sm.bar, 1); mbar_fence_init(); }
     for (int x = tid; x < 2048 / 16; x += 128) reinterpret_cast<uint4*>(lmt)[x] = make_uint4(0u, 0u, 0u, 0u);
@@ -623,13 +627,19 @@ const bool g_force_mma_select = [] {
     const char* e = getenv("HILS_FORCE_MMA_SELECT");
     return e != nullptr && e[0] == '1';
 }();
+// HILS_PREFILL_QB overrides the query-block length (multiple of 64, for tuning runs).
+const int kQB = [] {
+    const char* e = getenv("HILS_PREFILL_QB");
+    const int v = e ? atoi(e) : 0;
+    return (v >= 64 && v % 64 == 0 && v <= (1 << 20)) ? v : kQBDefault;
+}();
 const bool g_force_mma_attend = [] {
     const char* e = getenv("HILS_FORCE_MMA_ATTEND");
     return e != nullptr && e[0] == '1';
 }();
 
 struct Plan {
-    int qb, nc, max_tiles;
+    int qb, nc, n_blocks, max_tiles;
     size_t off_cnt, off_cursor, off_ntiles, zero_bytes, off_off, off_toff, off_entries, off_tiles, off_obuf, off_lam,
         total;
 };
@@ -641,16 +651,18 @@ Plan make_plan(const Shape& s) {
     p.qb = static_cast<int>(blk);
     const size_t nc = static_cast<size_t>(s.C > (s.R + kS - 1) / kS ? s.C : (s.R + kS - 1) / kS);
     p.nc = static_cast<int>(nc);
-    p.max_tiles = static_cast<int>(pairs * blk * (s.K + 1) / kTileTok + pairs * nc);
+    const size_t nblocks = (static_cast<size_t>(s.R) + blk - 1) / blk;
+    p.n_blocks = static_cast<int>(nblocks);
+    p.max_tiles = static_cast<int>(pairs * s.R * (s.K + 1) / kTileTok + nblocks * pairs * nc);
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = (off + bytes + 255) / 256 * 256; return o; };
-    p.off_cnt = take(sizeof(int) * pairs * nc);
-    p.off_cursor = take(sizeof(int) * pairs * nc);
-    p.off_ntiles = take(256);
-    p.zero_bytes = off;                         // cnt, cursor, n_tiles are cleared together per block
-    p.off_off = take(sizeof(int) * pairs * nc);
-    p.off_toff = take(sizeof(int) * pairs * nc);
-    p.off_entries = take(sizeof(int) * pairs * blk * (s.K + 1));
+    p.off_cnt = take(sizeof(int) * nblocks * pairs * nc);
+    p.off_cursor = take(sizeof(int) * nblocks * pairs * nc);
+    p.off_ntiles = take(sizeof(int) * (nblocks + 1));
+    p.zero_bytes = off;                         // cnt, cursor, blk_toff are cleared together once per call
+    p.off_off = take(sizeof(int) * nblocks * pairs * nc);
+    p.off_toff = take(sizeof(int) * nblocks * pairs * nc);
+    p.off_entries = take(sizeof(int) * pairs * s.R * (s.K + 1));
     p.off_tiles = take(sizeof(int4) * static_cast<size_t>(p.max_tiles));
     p.off_obuf = take(sizeof(__nv_bfloat16) * pairs * blk * (s.K + 1) * kG * kD);
     p.off_lam = take(sizeof(float) * pairs * blk * kG * (s.K + 1));
@@ -664,7 +676,8 @@ bool prefill_fast_supports(const Shape& s, int dtype) {
     return dtype == HILS_BF16 && !s.is_decode && s.d == kD && s.S == kS && s.W == 1 && s.Hl == s.Hkv && s.G == kG &&
            s.K >= 1 && s.K <= 64 && static_cast<long long>(s.B) * s.Hkv * s.T < (1ll << 31) &&
            static_cast<long long>(s.B) * s.Hkv * s.C < (1ll << 24) &&
-           static_cast<long long>(s.B) * s.Hkv * ((s.R + kS - 1) / kS) < (1ll << 31);
+           static_cast<long long>(s.B) * s.Hkv * ((s.R + kS - 1) / kS) < (1ll << 31) &&
+           static_cast<long long>(s.B) * s.Hkv * s.R * (s.K + 1) < (1ll << 31);
 }
 
 size_t prefill_fast_scratch_bytes(const Shape& s) { return make_plan(s).total; }
@@ -685,7 +698,9 @@ int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
     a.status = t.status;
     a.cnt = reinterpret_cast<int*>(sc + p.off_cnt);
     a.cursor = reinterpret_cast<int*>(sc + p.off_cursor);
-    a.n_tiles = reinterpret_cast<int*>(sc + p.off_ntiles);
+    a.blk_toff = reinterpret_cast<int*>(sc + p.off_ntiles);
+    a.n_blocks = p.n_blocks;
+    a.blk = 0;
     a.off = reinterpret_cast<int*>(sc + p.off_off);
     a.toff = reinterpret_cast<int*>(sc + p.off_toff);
     a.entries = reinterpret_cast<int*>(sc + p.off_entries);
@@ -730,12 +745,11 @@ int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
     trace_mark("prefill_select", stream);
     ++launches;
 
-    for (int i0 = 0; i0 < s.R; i0 += kQB) {
-        a.i0 = i0;
-        a.i1 = s.R < i0 + kQB ? s.R : i0 + kQB;
-        const int nblk = a.i1 - a.i0;
-        if (cudaMemsetAsync(sc + p.off_cnt, 0, p.zero_bytes, stream) != cudaSuccess) return HILS_ERR_CUDA;
-        const long long elems = static_cast<long long>(pairs) * nblk * (s.K + 1);
+    // inverse index for every query block at once: per-(block, pair, chunk) lists of (token, slot) entries
+    // and the table of attend tiles, grouped by block
+    if (cudaMemsetAsync(sc + p.off_cnt, 0, p.zero_bytes, stream) != cudaSuccess) return HILS_ERR_CUDA;
+    {
+        const long long elems = static_cast<long long>(pairs) * s.R * (s.K + 1);
         const long long want = (elems + 255) / 256;
         const unsigned eb = static_cast<unsigned>(want < 148 * 16 ? want : 148 * 16);
         invert_count_kernel<<<eb, 256, 0, stream>>>(a);
@@ -743,12 +757,19 @@ int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
         invert_fill_kernel<<<eb, 256, 0, stream>>>(a);
         if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
         trace_mark("prefill_invert", stream);
+        launches += 3;
+    }
+    for (int i0 = 0, blk = 0; i0 < s.R; i0 += a.qb, ++blk) {
+        a.i0 = i0;
+        a.i1 = s.R < i0 + a.qb ? s.R : i0 + a.qb;
+        a.blk = blk;
+        const int nblk = a.i1 - a.i0;
         if (g_force_mma_attend) {
             prefill_attend_kernel<<<148 * 2, 128, att_smem, stream>>>(map_k, map_v, a);
             if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
         } else {
-            const int rc = launch_prefill_attend_tc(s, t.q, t.k, t.v, t.landmarks, t.bias, a.entries, a.tiles, a.n_tiles,
-                                                    a.obuf, a.lam, t.status, a.i0, a.qb, stream);
+            const int rc = launch_prefill_attend_tc(s, t.q, t.k, t.v, t.landmarks, t.bias, a.entries, a.tiles,
+                                                    a.blk_toff + blk, a.obuf, a.lam, t.status, a.i0, a.qb, stream);
             if (rc < 0) return rc;
         }
         trace_mark("prefill_attend", stream);
@@ -756,7 +777,7 @@ int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
         prefill_fuse_kernel<<<static_cast<unsigned>((fuse_warps + kFuseWarps - 1) / kFuseWarps), kFuseWarps * 32, 0, stream>>>(a);
         if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
         trace_mark("prefill_fuse", stream);
-        launches += 5;
+        launches += 2;
     }
     return launches;
 }
