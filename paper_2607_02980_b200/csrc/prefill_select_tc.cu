@@ -198,17 +198,15 @@ prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
                     const int c = c0 + j;
-                    if (c < my_ncand) {
-                        float u = um[j] * s.scale;
-                        if (bias) u += bias[c];
-                        const unsigned long long key = select_key(u, c);
-                        if (key > tau) {
-                            myq[qn * kTileTok] = key;
-                            ++qn;
-                        }
-                    }
+                    float u = um[j] * s.scale;
+                    if (bias) u += bias[min(c, s.C - 1)];
+                    const unsigned long long key = select_key(u, c);
+                    const bool pass = c < my_ncand && key > tau;
+                    // branch-free append: the slot is written always and kept only when the key passes
+                    myq[qn * kTileTok] = key;
+                    qn += pass ? 1 : 0;
                 }
-                if (__any_sync(kFullMask, qn > kQueueCap - 16)) drain();
+                if (__any_sync(kFullMask, qn > kQueueCap - 17)) drain();
             }
             tc_fence_before_sync();
             __syncwarp();
