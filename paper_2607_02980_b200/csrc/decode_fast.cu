@@ -49,13 +49,314 @@ struct DArgs {
     float* Rh;         // [pairs, G]    max_c s^h_c over the selected chunks
     float* Eh;         // [pairs, G]    sum of wgt
     int* pair_n;       // [pairs]       number of selected chunks, -1 = invalid sequence length
-    int* done;         // [pairs]       slots finished (zeroed by decode_select)
+    int* done;         // [pairs]       slots finished (zeroed by the selection)
     float* part;       // [pairs, max_parts, G, 128] weighted partial sums
     float* loc_o;      // [pairs, G, 128] local-branch output
     float* loc_lam;    // [pairs, G]      log Z_swa
     int max_parts;
     int n_ctas;
 };
+
+// ------------------------------------------------------------------------------------------ select
+__device__ inline int block_excl_scan(int v, int* warp_tot, int& total) {
+    // exclusive prefix of v over the block in thread order; warp_tot: shared int[32]
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    int inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int n = __shfl_up_sync(kFullMask, inc, o);
+        if (lane >= o) inc += n;
+    }
+    __syncthreads();
+    if (lane == 31) warp_tot[warp] = inc;
+    __syncthreads();
+    int base = 0, tot = 0;
+    for (int w = 0; w < nw; ++w) {
+        const int x = warp_tot[w];
+        if (w < warp) base += x;
+        tot += x;
+    }
+    total = tot;
+    return base + inc - v;
+}
+
+struct SelShared {
+    int hist[kSelBins];
+    unsigned long long cand[kSelCap];
+    int sel_s[128];
+    float lam_s[8][128];
+    alignas(16) __nv_bfloat16 lm_s[64][kD + 8];    // selected landmark rows, 64 at a time (padded rows)
+    alignas(16) __nv_bfloat16 q_s[8][kD + 8];
+    int warp_tot[32];
+    int sh_i[8];
+    int is_last;
+};
+
+// Exact top-K of the group scores of one (sequence, KV head) pair (ties: lower chunk id), ascending ids,
+// then the per-head surrogate scores of the selected chunks and the fusion weights.  Called by every
+// thread of the CTA that finished the pair's scoring last; u was written by other CTAs (L2 reads).
+__device__ void select_pair(const DArgs& a, int pair, int ncand, SelShared& sh) {
+    const Shape& s = a.s;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, NT = blockDim.x;
+    const int b = pair / s.Hkv, g = pair % s.Hkv;
+    const int K = s.K, G = s.G;
+    int32_t* sel = a.sel + static_cast<long long>(pair) * K;
+    const int n = min(K, ncand);
+    const float* u = a.u + static_cast<long long>(pair) * a.Cpad;
+    int* hist = sh.hist;
+    int* sel_s = sh.sel_s;
+    int* sh_i = sh.sh_i;
+
+    if (ncand <= K) {
+        for (int t = tid; t < K; t += NT) sel_s[t] = t < ncand ? t : -1;
+        __syncthreads();
+    } else if (ncand <= 8 * NT) {
+        // --- short candidate lists: every thread keeps 8 consecutive ordered keys in registers and the
+        //     K-th best is found with a 4 x 8-bit radix select (shared-memory histograms only)
+        unsigned key[8];
+        const int cb = tid * 8;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) key[i] = cb + i < ncand ? ordered_key(__ldcg(u + cb + i)) : 0u;
+        unsigned prefix = 0u;
+        int remaining = K, n_eq = 0;
+#pragma unroll 1
+        for (int shift = 24; shift >= 0; shift -= 8) {
+            if (tid < 256) hist[tid] = 0;
+            __syncthreads();
+            const unsigned himask = shift == 24 ? 0u : (0xffffffffu << (shift + 8));
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                if (cb + i < ncand && (key[i] & himask) == (prefix & himask)) atomicAdd(&hist[(key[i] >> shift) & 255u], 1);
+            __syncthreads();
+            if (warp == 0) {
+                // lane l owns digits 255-8l .. 248-8l (top-down)
+                int loc[8], tsum = 0;
+#pragma unroll
+                for (int x = 0; x < 8; ++x) { loc[x] = hist[255 - 8 * lane - x]; tsum += loc[x]; }
+                int inc = tsum;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int nn = __shfl_up_sync(kFullMask, inc, o);
+                    if (lane >= o) inc += nn;
+                }
+                int cum = inc - tsum;
+                if (cum < remaining && inc >= remaining) {
+#pragma unroll
+                    for (int x = 0; x < 8; ++x) {
+                        if (cum + loc[x] >= remaining) { sh_i[4] = 255 - 8 * lane - x; sh_i[5] = cum; sh_i[6] = loc[x]; break; }
+                        cum += loc[x];
+                    }
+                }
+            }
+            __syncthreads();
+            prefix |= static_cast<unsigned>(sh_i[4]) << shift;
+            remaining -= sh_i[5];
+            n_eq = sh_i[6];
+        }
+        // prefix = key of the K-th best; `remaining` of the n_eq chunks with that key are taken, lowest ids first
+        int eq_before = 0, tot;
+        if (n_eq != remaining) {                        // ties across the cut (block-uniform branch)
+            int eq = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) eq += (cb + i < ncand && key[i] == prefix) ? 1 : 0;
+            eq_before = block_excl_scan(eq, sh.warp_tot, tot);
+        }
+        int cnt = 0, e = eq_before;
+        unsigned take = 0u;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            if (cb + i >= ncand) continue;
+            bool tk = key[i] > prefix;
+            if (key[i] == prefix) { tk = n_eq == remaining || e < remaining; ++e; }
+            if (tk) { take |= 1u << i; ++cnt; }
+        }
+        int pos = block_excl_scan(cnt, sh.warp_tot, tot);
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            if (take & (1u << i)) sel_s[pos++] = cb + i;
+        __syncthreads();
+    } else {
+        // --- 1. value range
+        float mn = INFINITY, mx = -INFINITY;
+        for (int c = tid; c < ncand; c += NT) { const float v = __ldcg(u + c) + 0.f; mn = fminf(mn, v); mx = fmaxf(mx, v); }
+        mn = -warp_max(-mn); mx = warp_max(mx);
+        if (lane == 0) { sh.lam_s[0][warp] = mn; sh.lam_s[1][warp] = mx; }
+        for (int i = tid; i < kSelBins; i += NT) hist[i] = 0;
+        if (tid == 0) sh_i[3] = 0;
+        __syncthreads();
+        float lo = sh.lam_s[0][0], hi = sh.lam_s[1][0];
+        for (int w = 1; w < NT / 32; ++w) { lo = fminf(lo, sh.lam_s[0][w]); hi = fmaxf(hi, sh.lam_s[1][w]); }
+        const float inv = (hi > lo) ? static_cast<float>(kSelBins - 1) / (hi - lo) : 0.f;
+        __syncthreads();
+        // --- 2. histogram over a monotone linear binning
+        for (int c = tid; c < ncand; c += NT) {
+            const int bin = max(0, min(kSelBins - 1, static_cast<int>((__ldcg(u + c) + 0.f - lo) * inv)));
+            atomicAdd(&hist[bin], 1);
+        }
+        __syncthreads();
+        // --- 3. boundary bin: the highest bin b* with count(bin >= b*) >= K.  Thread i owns the
+        //        kSelBins / NT bins below (kSelBins - 1 - i * per); a block scan gives the count above.
+        {
+            const int per = kSelBins / NT;
+            const int top = kSelBins - 1 - tid * per;
+            int tsum = 0;
+            for (int x = 0; x < per; ++x) tsum += hist[top - x];
+            int tot;
+            int cum = block_excl_scan(tsum, sh.warp_tot, tot);
+            if (cum < K && cum + tsum >= K) {
+                for (int x = 0; x < per; ++x) {
+                    const int hb = hist[top - x];
+                    if (cum + hb >= K) { sh_i[0] = top - x; sh_i[1] = cum + hb; sh_i[2] = cum; break; }
+                    cum += hb;
+                }
+            }
+        }
+        __syncthreads();
+        const int bstar = sh_i[0], m_cand = sh_i[1];
+        if (m_cand <= kSelCap) {
+            // --- 4a. gather the candidates and rank them exactly (score desc, id asc)
+            unsigned long long* cand = sh.cand;
+            for (int c = tid; c < ncand; c += NT) {
+                const float v = __ldcg(u + c);
+                const int bin = max(0, min(kSelBins - 1, static_cast<int>((v + 0.f - lo) * inv)));
+                if (bin >= bstar) cand[atomicAdd(&sh_i[3], 1)] = select_key(v, c);
+            }
+            __syncthreads();
+            unsigned long long mine[kSelCap / kSelThreads];
+            bool keep[kSelCap / kSelThreads];
+#pragma unroll
+            for (int r = 0; r < kSelCap / kSelThreads; ++r) {
+                const int i = tid + r * NT;
+                mine[r] = i < m_cand ? cand[i] : 0ull;
+                int rank = 0;
+                if (i < m_cand)
+                    for (int j = 0; j < m_cand; ++j) rank += cand[j] > mine[r] ? 1 : 0;
+                keep[r] = i < m_cand && rank < K;                  // ranks are unique
+            }
+            __syncthreads();
+#pragma unroll
+            for (int r = 0; r < kSelCap / kSelThreads; ++r) {
+                const int i = tid + r * NT;
+                if (i < m_cand && !keep[r]) cand[i] = 0ull;
+            }
+            __syncthreads();
+            // ascending ids: position = number of selected ids below mine
+#pragma unroll
+            for (int r = 0; r < kSelCap / kSelThreads; ++r) {
+                if (!keep[r]) continue;
+                const int id = key_chunk(mine[r]);
+                int pos = 0;
+                for (int j = 0; j < m_cand; ++j) {
+                    const unsigned long long o = cand[j];
+                    pos += (o != 0ull && key_chunk(o) < id) ? 1 : 0;
+                }
+                sel_s[pos] = id;
+            }
+            __syncthreads();
+        } else {
+            // --- 4b. many equal / clustered scores: exact 4 x 8-bit radix select on the ordered key,
+            //         then an ordered scan (each thread owns a contiguous range of chunk ids)
+            unsigned prefix = 0u;
+            int remaining = K;
+            for (int shift = 24; shift >= 0; shift -= 8) {
+                for (int i = tid; i < 256; i += NT) hist[i] = 0;
+                __syncthreads();
+                const unsigned himask = shift == 24 ? 0u : (0xffffffffu << (shift + 8));
+                for (int c = tid; c < ncand; c += NT) {
+                    const unsigned key = ordered_key(__ldcg(u + c));
+                    if ((key & himask) == (prefix & himask)) atomicAdd(&hist[(key >> shift) & 255u], 1);
+                }
+                __syncthreads();
+                if (tid == 0) {
+                    int cum = 0, dsel = 0;
+                    for (int dgt = 255; dgt >= 0; --dgt) {
+                        if (cum + hist[dgt] >= remaining) { dsel = dgt; break; }
+                        cum += hist[dgt];
+                    }
+                    sh_i[4] = dsel; sh_i[5] = cum;
+                }
+                __syncthreads();
+                prefix |= static_cast<unsigned>(sh_i[4]) << shift;
+                remaining -= sh_i[5];
+                __syncthreads();
+            }
+            // prefix = key of the K-th best; `remaining` of the chunks with that key are taken, lowest ids first
+            const int per = (ncand + NT - 1) / NT;
+            const int cb = min(ncand, tid * per), ce = min(ncand, cb + per);
+            int eq = 0;
+            for (int c = cb; c < ce; ++c) eq += ordered_key(__ldcg(u + c)) == prefix ? 1 : 0;
+            int tot;
+            int eq_before = block_excl_scan(eq, sh.warp_tot, tot);
+            int cnt = 0;
+            int e = eq_before;
+            for (int c = cb; c < ce; ++c) {
+                const unsigned key = ordered_key(__ldcg(u + c));
+                if (key > prefix) ++cnt;
+                else if (key == prefix) { if (e < remaining) ++cnt; ++e; }
+            }
+            int pos = block_excl_scan(cnt, sh.warp_tot, tot);
+            e = eq_before;
+            for (int c = cb; c < ce; ++c) {
+                const unsigned key = ordered_key(__ldcg(u + c));
+                bool take = key > prefix;
+                if (key == prefix) { take = e < remaining; ++e; }
+                if (take) sel_s[pos++] = c;
+            }
+            __syncthreads();
+        }
+    }
+    for (int t = tid; t < K; t += NT) sel[t] = t < n ? sel_s[t] : -1;
+
+    // --- 5. per-head surrogate scores of the selected chunks and the fusion weights: the selected
+    //        landmark rows and the G queries are staged in shared memory with one round of 16-byte
+    //        loads, then every thread computes one (chunk, head) dot product
+    const __nv_bfloat16* lm = a.lm + static_cast<long long>(pair) * s.C * kD;
+    const __nv_bfloat16* qg = a.q + (static_cast<long long>(b) * s.Hq + g * G) * kD;
+    for (int x = tid; x < G * 16; x += NT)
+        *reinterpret_cast<uint4*>(&sh.q_s[x >> 4][(x & 15) * 8]) = *reinterpret_cast<const uint4*>(qg + (x >> 4) * kD + (x & 15) * 8);
+    for (int t0 = 0; t0 < n; t0 += 64) {
+        const int nt = min(64, n - t0);
+        __syncthreads();
+        for (int x = tid; x < nt * 16; x += NT) {
+            const int t = x >> 4, pc = x & 15;
+            *reinterpret_cast<uint4*>(&sh.lm_s[t][pc * 8]) =
+                *reinterpret_cast<const uint4*>(lm + static_cast<long long>(sel_s[t0 + t]) * kD + pc * 8);
+        }
+        __syncthreads();
+        for (int x = tid; x < nt * G; x += NT) {
+            const int t = x / G, h = x % G;
+            const __nv_bfloat16* lr = sh.lm_s[t];
+            const __nv_bfloat16* qr = sh.q_s[h];
+            float acc = 0.f;
+#pragma unroll 8
+            for (int e = 0; e < kD; e += 2) {
+                const float2 lv = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(lr + e));
+                const float2 qv = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(qr + e));
+                acc = fmaf(lv.x, qv.x, acc);
+                acc = fmaf(lv.y, qv.y, acc);
+            }
+            const float bb = a.bias ? a.bias[static_cast<long long>(pair) * s.C + sel_s[t0 + t]] : 0.f;
+            sh.lam_s[h][t0 + t] = acc * s.scale + bb;
+        }
+    }
+    __syncthreads();
+    if (warp < G) {
+        const int h = warp;
+        float mx = -INFINITY;
+        for (int t = lane; t < n; t += 32) mx = fmaxf(mx, sh.lam_s[h][t]);
+        mx = warp_max(mx);
+        float sum = 0.f;
+        float* w = a.wgt + (static_cast<long long>(pair) * G + h) * K;
+        for (int t = lane; t < K; t += 32) {
+            const float e = t < n ? __expf(sh.lam_s[h][t] - mx) : 0.f;
+            w[t] = e;
+            sum += e;
+        }
+        sum = warp_sum(sum);
+        if (lane == 0) { a.Rh[pair * G + h] = mx; a.Eh[pair * G + h] = sum; }
+    }
+    if (tid == 0) { a.pair_n[pair] = n; a.done[pair] = 0; }
+}
 
 // ------------------------------------------------------------------------------------------ score
 __global__ void __launch_bounds__(kScoreThreads) decode_score_kernel(const DArgs a) {
@@ -124,225 +425,24 @@ __global__ void __launch_bounds__(kScoreThreads) decode_score_kernel(const DArgs
     pdl_launch_dependents();
 }
 
-// ------------------------------------------------------------------------------------------ select
-__device__ inline int block_excl_scan(int v, int* warp_tot, int& total) {
-    // exclusive prefix of v over the block in thread order; warp_tot: shared int[32]
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
-    int inc = v;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int n = __shfl_up_sync(kFullMask, inc, o);
-        if (lane >= o) inc += n;
-    }
-    __syncthreads();
-    if (lane == 31) warp_tot[warp] = inc;
-    __syncthreads();
-    int base = 0, tot = 0;
-    for (int w = 0; w < nw; ++w) {
-        const int x = warp_tot[w];
-        if (w < warp) base += x;
-        tot += x;
-    }
-    total = tot;
-    return base + inc - v;
-}
-
+// One CTA per (sequence, KV head) pair.
 __global__ void __launch_bounds__(kSelThreads) decode_select_kernel(const DArgs a) {
-    __shared__ int hist[kSelBins];
-    __shared__ unsigned long long cand[kSelCap];
-    __shared__ int sel_s[128];
-    __shared__ float lam_s[8][128];
-    __shared__ float red_f[32];
-    __shared__ int warp_tot[32];
-    __shared__ int sh_i[8];
-    __shared__ float sh_f[4];
-
+    __shared__ SelShared sh;
     const Shape& s = a.s;
-    const int pair = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int pair = blockIdx.x, tid = threadIdx.x;
     const int b = pair / s.Hkv, g = pair % s.Hkv;
-    const int K = s.K, G = s.G;
-    int32_t* sel = a.sel + static_cast<long long>(pair) * K;
     const int seq = a.seq_lens[b];
-    if (tid == 0) a.done[pair] = 0;
     if (seq < 1 || seq > s.T) {
         // invalid length: flag it, emit empty outputs
-        if (tid == 0) { set_status(a.status, kDevBadIndex); a.pair_n[pair] = -1; }
-        for (int t = tid; t < K; t += kSelThreads) sel[t] = -1;
-        for (int x = tid; x < G * kD; x += kSelThreads)
-            a.out[(static_cast<long long>(b) * s.Hq + g * G) * kD + x] = __float2bfloat16_rn(0.f);
-        if (tid < G) a.lse[static_cast<long long>(b) * s.Hq + g * G + tid] = 0.f;
+        if (tid == 0) { set_status(a.status, kDevBadIndex); a.pair_n[pair] = -1; a.done[pair] = 0; }
+        for (int t = tid; t < s.K; t += kSelThreads) a.sel[static_cast<long long>(pair) * s.K + t] = -1;
+        for (int x = tid; x < s.G * kD; x += kSelThreads)
+            a.out[(static_cast<long long>(b) * s.Hq + g * s.G) * kD + x] = __float2bfloat16_rn(0.f);
+        if (tid < s.G) a.lse[static_cast<long long>(b) * s.Hq + g * s.G + tid] = 0.f;
         return;
     }
-    const int ncand = (seq - 1) / kS;
-    const int n = min(K, ncand);
-    pdl_wait();                                   // group scores of decode_score are visible
-    const float* u = a.u + static_cast<long long>(pair) * a.Cpad;
-
-    if (ncand <= K) {
-        for (int t = tid; t < K; t += kSelThreads) sel_s[t] = t < ncand ? t : -1;
-        __syncthreads();
-    } else {
-        // --- 1. value range
-        float mn = INFINITY, mx = -INFINITY;
-        for (int c = tid; c < ncand; c += kSelThreads) { const float v = u[c] + 0.f; mn = fminf(mn, v); mx = fmaxf(mx, v); }
-        mn = -warp_max(-mn); mx = warp_max(mx);
-        if (lane == 0) { red_f[warp] = mn; red_f[16 + warp] = mx; }
-        for (int i = tid; i < kSelBins; i += kSelThreads) hist[i] = 0;
-        __syncthreads();
-        if (tid == 0) {
-            float lo = red_f[0], hi = red_f[16];
-            for (int w = 1; w < kSelThreads / 32; ++w) { lo = fminf(lo, red_f[w]); hi = fmaxf(hi, red_f[16 + w]); }
-            sh_f[0] = lo;
-            sh_f[1] = (hi > lo) ? static_cast<float>(kSelBins - 1) / (hi - lo) : 0.f;
-        }
-        __syncthreads();
-        const float lo = sh_f[0], inv = sh_f[1];
-        // --- 2. histogram over a monotone linear binning
-        for (int c = tid; c < ncand; c += kSelThreads) {
-            const int bin = min(kSelBins - 1, static_cast<int>((u[c] + 0.f - lo) * inv));
-            atomicAdd(&hist[bin], 1);
-        }
-        __syncthreads();
-        // --- 3. boundary bin: the highest bin b* with count(bin >= b*) >= K   (warp 0 scans from the top)
-        if (warp == 0) {
-            int carry = 0, found = -1, above = 0;
-            for (int base = kSelBins - 32; base >= 0 && found < 0; base -= 32) {
-                const int hb = hist[base + 31 - lane];               // lane 0 = highest bin of the block
-                int inc = hb;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const int nn = __shfl_up_sync(kFullMask, inc, o);
-                    if (lane >= o) inc += nn;
-                }
-                const unsigned hit = __ballot_sync(kFullMask, carry + inc >= K);
-                if (hit) {
-                    const int l = __ffs(hit) - 1;
-                    found = base + 31 - l;
-                    above = carry + __shfl_sync(kFullMask, inc - hb, l);   // count in bins above b*
-                    carry += __shfl_sync(kFullMask, inc, l);               // count in bins >= b*
-                } else {
-                    carry += __shfl_sync(kFullMask, inc, 31);
-                }
-            }
-            if (lane == 0) { sh_i[0] = found; sh_i[1] = carry; sh_i[2] = above; sh_i[3] = 0; }
-        }
-        __syncthreads();
-        const int bstar = sh_i[0], m_cand = sh_i[1];
-        if (m_cand <= kSelCap) {
-            // --- 4a. gather the candidates and rank them exactly (score desc, id asc)
-            for (int c = tid; c < ncand; c += kSelThreads) {
-                const float v = u[c];
-                const int bin = min(kSelBins - 1, static_cast<int>((v + 0.f - lo) * inv));
-                if (bin >= bstar) cand[atomicAdd(&sh_i[3], 1)] = select_key(v, c);
-            }
-            __syncthreads();
-            for (int i = tid; i < m_cand; i += kSelThreads) {
-                const unsigned long long mine = cand[i];
-                int rank = 0;
-                for (int j = 0; j < m_cand; ++j) rank += cand[j] > mine ? 1 : 0;
-                if (rank >= K) cand[i] = 0ull;                       // not selected (ranks are unique)
-            }
-            __syncthreads();
-            // ascending ids: position = number of selected ids below mine
-            for (int i = tid; i < m_cand; i += kSelThreads) {
-                const unsigned long long mine = cand[i];
-                if (mine == 0ull) continue;
-                const int id = key_chunk(mine);
-                int pos = 0;
-                for (int j = 0; j < m_cand; ++j) pos += (cand[j] != 0ull && key_chunk(cand[j]) < id) ? 1 : 0;
-                sel_s[pos] = id;
-            }
-            __syncthreads();
-        } else {
-            // --- 4b. many equal / clustered scores: exact 4 x 8-bit radix select on the ordered key,
-            //         then an ordered scan (each thread owns a contiguous range of chunk ids)
-            unsigned prefix = 0u;
-            int remaining = K;
-            for (int shift = 24; shift >= 0; shift -= 8) {
-                for (int i = tid; i < 256; i += kSelThreads) hist[i] = 0;
-                __syncthreads();
-                const unsigned himask = shift == 24 ? 0u : (0xffffffffu << (shift + 8));
-                for (int c = tid; c < ncand; c += kSelThreads) {
-                    const unsigned key = ordered_key(u[c]);
-                    if ((key & himask) == (prefix & himask)) atomicAdd(&hist[(key >> shift) & 255u], 1);
-                }
-                __syncthreads();
-                if (tid == 0) {
-                    int cum = 0, dsel = 0;
-                    for (int dgt = 255; dgt >= 0; --dgt) {
-                        if (cum + hist[dgt] >= remaining) { dsel = dgt; break; }
-                        cum += hist[dgt];
-                    }
-                    sh_i[4] = dsel; sh_i[5] = cum;
-                }
-                __syncthreads();
-                prefix |= static_cast<unsigned>(sh_i[4]) << shift;
-                remaining -= sh_i[5];
-                __syncthreads();
-            }
-            // prefix = key of the K-th best; `remaining` of the chunks with that key are taken, lowest ids first
-            const int per = (ncand + kSelThreads - 1) / kSelThreads;
-            const int cb = min(ncand, tid * per), ce = min(ncand, cb + per);
-            int eq = 0;
-            for (int c = cb; c < ce; ++c) eq += ordered_key(u[c]) == prefix ? 1 : 0;
-            int tot;
-            int eq_before = block_excl_scan(eq, warp_tot, tot);
-            int cnt = 0;
-            int e = eq_before;
-            for (int c = cb; c < ce; ++c) {
-                const unsigned key = ordered_key(u[c]);
-                if (key > prefix) ++cnt;
-                else if (key == prefix) { if (e < remaining) ++cnt; ++e; }
-            }
-            int pos = block_excl_scan(cnt, warp_tot, tot);
-            e = eq_before;
-            for (int c = cb; c < ce; ++c) {
-                const unsigned key = ordered_key(u[c]);
-                bool take = key > prefix;
-                if (key == prefix) { take = e < remaining; ++e; }
-                if (take) sel_s[pos++] = c;
-            }
-            __syncthreads();
-        }
-    }
-    for (int t = tid; t < K; t += kSelThreads) sel[t] = t < n ? sel_s[t] : -1;
-
-    // --- 5. per-head surrogate scores of the selected chunks and the fusion weights
-    const __nv_bfloat16* lm = a.lm + static_cast<long long>(pair) * s.C * kD;
-    const __nv_bfloat16* qg = a.q + (static_cast<long long>(b) * s.Hq + g * G) * kD;
-    for (int t = warp; t < n; t += kSelThreads / 32) {
-        const int c = sel_s[t];
-        const uint2 raw = *reinterpret_cast<const uint2*>(lm + static_cast<long long>(c) * kD + lane * 4);
-        const float l0 = __uint_as_float(raw.x << 16), l1 = __uint_as_float(raw.x & 0xffff0000u);
-        const float l2 = __uint_as_float(raw.y << 16), l3 = __uint_as_float(raw.y & 0xffff0000u);
-        const float bb = a.bias ? a.bias[static_cast<long long>(pair) * s.C + c] : 0.f;
-        for (int h = 0; h < G; ++h) {
-            const uint2 qr = *reinterpret_cast<const uint2*>(qg + h * kD + lane * 4);
-            float acc = l0 * __uint_as_float(qr.x << 16);
-            acc = fmaf(l1, __uint_as_float(qr.x & 0xffff0000u), acc);
-            acc = fmaf(l2, __uint_as_float(qr.y << 16), acc);
-            acc = fmaf(l3, __uint_as_float(qr.y & 0xffff0000u), acc);
-            acc = warp_sum(acc);
-            if (lane == 0) lam_s[h][t] = acc * s.scale + bb;
-        }
-    }
-    __syncthreads();
-    if (warp < G) {
-        const int h = warp;
-        float mx = -INFINITY;
-        for (int t = lane; t < n; t += 32) mx = fmaxf(mx, lam_s[h][t]);
-        mx = warp_max(mx);
-        float sum = 0.f;
-        float* w = a.wgt + (static_cast<long long>(pair) * G + h) * K;
-        for (int t = lane; t < K; t += 32) {
-            const float e = t < n ? __expf(lam_s[h][t] - mx) : 0.f;
-            w[t] = e;
-            sum += e;
-        }
-        sum = warp_sum(sum);
-        if (lane == 0) { a.Rh[pair * G + h] = mx; a.Eh[pair * G + h] = sum; }
-    }
-    if (tid == 0) a.pair_n[pair] = n;
+    pdl_wait();                                        // group scores of decode_score are visible
+    select_pair(a, pair, (seq - 1) / kS, sh);
     pdl_launch_dependents();
 }
 
@@ -748,12 +848,12 @@ int launch_decode_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(pairs);
-    cfg.blockDim = dim3(kSelThreads);
-    cfg.dynamicSmemBytes = 0;
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    cfg.gridDim = dim3(pairs);
+    cfg.blockDim = dim3(kSelThreads);
+    cfg.dynamicSmemBytes = 0;
     if (cudaLaunchKernelEx(&cfg, decode_select_kernel, a) != cudaSuccess) return HILS_ERR_CUDA;
     trace_mark("decode_select", stream);
 

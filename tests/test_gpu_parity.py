@@ -48,6 +48,9 @@ PREFILL_SMALL = {
     "bf16_k_ge_chunks": wl.CONFIGS[1].scaled(Hq=8, Hkv=2, L=640, K=64, seed=22),
     "bf16_d64_g2_s32": wl.CONFIGS[1].scaled(Hq=4, Hkv=2, L=777, d=64, S=32, K=5, seed=23),
     "f32_g4_k33": wl.CONFIGS[0].scaled(Hq=4, Hkv=1, L=2500, d=128, K=33, seed=24, n_needles=2),
+    # longer than one 4096-token query block of the fast path, ragged end, K between 32 and 64
+    "bf16_multiblock_k40": wl.CONFIGS[1].scaled(Hq=4, Hkv=1, L=8300, K=40, seed=26),
+    "bf16_multiblock_b2": wl.CONFIGS[1].scaled(B=2, Hq=8, Hkv=2, L=4200, K=12, seed=27),
 }
 
 
