@@ -5,7 +5,7 @@ A "step" is one pass of the whole hot path (landmark scoring, group max, top-K s
 attention, per-chunk attention, fusion) over one batch of seeded synthetic input, through the C ABI.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg1|cfg0|cfg2|cfg3|cfg4]
-                  [--impl ours|reference] [--extra]
+                  [--impl ours|reference] [--no-extra] [--no-e2e] [--no-cpu-baseline]
 
 Prefill workloads report effective TFLOP/s on the gathered FLOP (what the method must do, not what
 dense attention would); decode workloads report GB/s on the algorithmic bytes (landmarks scanned +
@@ -33,8 +33,15 @@ import torch
 
 from paper_2607_02980_b200 import workloads as wl
 
-# dram bytes per launch of the dominant kernel from ncu captures (see profiles/); None = not captured
-NCU_TRAFFIC_BYTES = {}
+# dram__bytes_read.sum + dram__bytes_write.sum PER LAUNCH of each workload's dominant kernel, from the ncu
+# captures summarised under profiles/.  The decode captures ran a reduced batch (8 of 64 sequences for cfg3, 1 of 4
+# for cfg4); traffic is proportional to the number of (sequence, KV head) pairs and is scaled to the full launch.
+NCU_TRAFFIC_BYTES = {
+    ("cfg1", "prefill_attend"): int((181.6 + 536.8 + 192.8 + 535.5) / 2 * 1e6),   # one 4096-token query block
+    ("cfg3", "decode_attend"): int(70.5e6 * 8),
+    ("cfg4", "decode_attend"): int(17.1e6 * 4),
+    ("cfg4", "decode_score"): int(33.57e6 * 4),
+}
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -163,7 +170,10 @@ class Workload:
             self.sel = torch.empty((cfg.B, cfg.Hkv, cfg.L, cfg.K), dtype=torch.int32, device=device)
             self.work, self.work_aux = prefill_flops(cfg)
             self.unit, self.metric = "TFLOP/s", "hils_prefill_effective_TFLOPs"
-        self.flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=device) if self.decode else None
+        # L2 flush between decode steps: write 256 MB, then read another 256 MB so that the timed kernels
+        # start from an L2 full of clean lines (dirty lines would be written back under them)
+        self.flush = torch.empty(64 * 1024 * 1024, dtype=torch.int32, device=device) if self.decode else None
+        self.flush2 = torch.zeros(64 * 1024 * 1024, dtype=torch.int32, device=device) if self.decode else None
         self.step_no = 0
 
     def step(self):
@@ -180,6 +190,7 @@ class Workload:
     def between_steps(self):
         if self.flush is not None:
             self.flush.fill_(1)                  # 256 MB write: evicts the 126 MB L2
+            self.sink = self.flush2.max()        # 256 MB read: the write-backs drain before the timed step
 
     def rate(self, seconds_per_step, n_replicas=1):
         scale = 1e12 if self.unit == "TFLOP/s" else 1e9
@@ -222,12 +233,21 @@ def summarise_traces(traces):
     return {k: float(np.mean(v)) for k, v in agg.items()}
 
 
+def launches_per_step(traces):
+    """How many launches of each traced kernel one step makes."""
+    n = {}
+    for name, _ in traces[0]:
+        n[name] = n.get(name, 0) + 1
+    return n
+
+
 def kernel_times(w, steps, barrier):
     """Per-kernel CUDA-event times: the same steps run again with the library's trace events on
     (kept out of the headline timing because an event between two kernels breaks their overlap)."""
     w.hils.trace_enable(True)
     _, traces = time_steps(w, steps, 1, barrier)
     w.hils.trace_enable(False)
+    w.launches = launches_per_step(traces) if traces else {}
     return summarise_traces(traces)
 
 
@@ -236,17 +256,20 @@ def roofline_for(w, kernel_ms, peaks):
     if not kernel_ms:
         return None
     name = max(kernel_ms, key=kernel_ms.get)
-    sec = kernel_ms[name] * 1e-3
+    nl = max(1, getattr(w, "launches", {}).get(name, 1))     # launches of that kernel per step
+    sec = kernel_ms[name] * 1e-3 / nl                        # average duration of one launch
     src = "of measured" if peaks["_source"] == "measured" else "of fallback"
+    common = {"kernel": name, "launches_per_step": nl, "kernel_ms_per_launch": sec * 1e3,
+              "traffic": NCU_TRAFFIC_BYTES.get((w.cfg.name.split("_")[0], name)), "peak_source": src}
     if w.decode:
         lm_b, kv_b = decode_bytes(w.cfg, w.inp["seq_lens"].cpu().numpy())
         algo = kv_b if "attend" in name else (lm_b if ("score" in name or "select" in name) else lm_b + kv_b)
+        algo /= nl
         ach = algo / sec / 1e9
-        return {"kernel": name, "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": ach / peaks["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get((w.cfg.name, name)),
-                "algorithmic_bytes": algo, "kernel_ms": kernel_ms[name], "peak_source": src}
+        return dict(common, bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s",
+                    frac=ach / peaks["hbm_gbs"], algorithmic_bytes=algo)
     gathered, scoring = prefill_flops(w.cfg)
-    algo = scoring if ("score" in name or "select" in name) else gathered
+    algo = (scoring if ("score" in name or "select" in name) else gathered) / nl
     if w.cfg.dtype == "f32":
         # fp32 path on plain FMA units: 148 SMs x 128 lanes x 2 FLOP x max SM clock
         peak = 148 * 128 * 2 * peaks.get("sm_max_mhz", 1965.0) * 1e6 / 1e12
@@ -255,9 +278,8 @@ def roofline_for(w, kernel_ms, peaks):
         peak = peaks["bf16_tflops"]
         bound = "tensor"
     ach = algo / sec / 1e12
-    return {"kernel": name, "bound": bound, "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak,
-            "traffic": NCU_TRAFFIC_BYTES.get((w.cfg.name, name)), "algorithmic_flops": algo,
-            "kernel_ms": kernel_ms[name], "peak_source": src}
+    return dict(common, bound=bound, achieved=ach, peak=peak, unit="TFLOP/s", frac=ach / peak,
+                algorithmic_flops=algo)
 
 
 # ----------------------------------------------------------------------------- CPU oracle legs
@@ -279,6 +301,16 @@ def oracle_sample(cfg, inp_cpu, budget_rows):
     dt = time.perf_counter() - t0
     lm_b, kv_b = decode_bytes(cfg, sub["seq_lens"].numpy())
     return (lm_b + kv_b) / dt / 1e9, "first %d of %d sequences of %s" % (nb, cfg.B, cfg.name), dt
+
+
+def oracle_sample_timed(cfg, inp_cpu, target_seconds=15.0):
+    """Pilot run, then a sample sized for about `target_seconds` of CPU work (bounded by the workload)."""
+    if cfg.mode != "prefill":
+        return oracle_sample(cfg, inp_cpu, cfg.B)
+    pilot_rows = 256
+    _, _, dt = oracle_sample(cfg, inp_cpu, pilot_rows)
+    rows = int(min(cfg.L, max(pilot_rows, pilot_rows * target_seconds / max(dt, 1e-3))))
+    return oracle_sample(cfg, inp_cpu, rows)
 
 
 def reference_cfg_inputs(cfg):
@@ -317,6 +349,18 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def aggregate_over_ranks(ms_per_step_local, work_per_replica, unit_scale, dist=None, device="cpu"):
+    """Whole-job rate of N independent replicas: every rank did `work_per_replica`; the job takes as
+    long as its slowest rank (MAX over ranks of the per-step time).  Returns (value, ms_per_step)."""
+    world, ms = 1, float(ms_per_step_local)
+    if dist is not None:
+        world = dist.get_world_size()
+        t = torch.tensor([ms], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    return work_per_replica * world / (ms * 1e-3) / unit_scale, ms
+
+
 # ----------------------------------------------------------------------------- main
 def main():
     ap = argparse.ArgumentParser()
@@ -325,7 +369,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="cfg1", choices=["cfg0", "cfg1", "cfg2", "cfg3", "cfg4"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--extra", action="store_true", help="also time the other single-GPU configurations")
+    ap.add_argument("--no-extra", action="store_true", help="skip the other single-GPU configurations")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--profile-run", action="store_true",
@@ -383,10 +427,10 @@ def main():
     sampler = ClockSampler(local)
     sampler.start()
     ms, traces = time_steps(w, args.steps, args.warmup, barrier)
-    clocks = sampler.stop()
     launches = hils.last_launch_count() * args.steps
-    ms_step = max_over_ranks(float(np.sum(ms)) / args.steps)
-    value = w.rate(ms_step * 1e-3, world)
+    timed_launches = launches
+    value, ms_step = aggregate_over_ranks(float(np.sum(ms)) / args.steps, w.work,
+                                          1e12 if w.unit == "TFLOP/s" else 1e9, dist, dev)
     kernel_ms = kernel_times(w, max(3, min(args.steps, 10)), barrier)
     launches += hils.last_launch_count() * (max(3, min(args.steps, 10)) + 1)
 
@@ -395,11 +439,11 @@ def main():
             "vs_baseline": None, "dtype": "bf16" if cfg.dtype == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": cfg.name, "B": cfg.B, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "L_or_T": cfg.L, "d": cfg.d,
                        "chunk_size": cfg.S, "top_k": cfg.K, "window": 1, "parallelism": "replicas x%d" % world,
-                       "l2_policy": ("256 MB flush write + rotating query sets between steps" if w.decode else
+                       "l2_policy": ("256 MB write + 256 MB read flush and rotating query sets between steps" if w.decode else
                                      "inputs+outputs %.0f MB > 126 MB L2" % (
                                          sum(t.numel() * t.element_size() for t in list(w.inp.values()) + [w.out]) / 1e6)),
                        "median_ms": float(np.median(ms)), "min_ms": float(np.min(ms))},
-            "clocks": clocks, "gpu_launches": launches, "kernel_ms": kernel_ms}
+            "gpu_launches": launches, "kernel_ms": kernel_ms}
     if w.decode:
         line["decode_gathered_kv_GBps"] = None
         for name, kms in kernel_ms.items():
@@ -435,8 +479,11 @@ def main():
         launches += hils.last_launch_count() * (n_e2e + 2)
         del runner, host
 
+    clocks = sampler.stop()          # sampled over the timed steps, the per-kernel pass and the e2e steps
+    line["clocks"] = clocks
+
     # ---- other configurations (reported beside, never instead of, the primary workload)
-    if args.extra and world == 1:
+    if not args.no_extra and world == 1:
         extras = {}
         del w
         torch.cuda.empty_cache()
@@ -468,10 +515,11 @@ def main():
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
         small, inp_cpu = reference_cfg_inputs(cfg)
-        val, sample, secs = oracle_sample(small, inp_cpu, 2048 if cfg.mode == "prefill" else 2)
+        val, sample, secs = oracle_sample_timed(small, inp_cpu)
         line["cpu_baseline"] = {"value": val, "unit": "TFLOP/s" if cfg.mode == "prefill" else "GB/s",
                                 "cores": oracle.num_threads(), "kind": "oracle", "sample": sample, "seconds": secs}
-    line["gpu_launches"] = launches
+    line["gpu_launches"] = timed_launches            # kernels of this library inside the timed region
+    line["gpu_launches_whole_run"] = launches        # incl. warm-up, traced, end-to-end and extra-workload passes
     if rank == 0:
         print(json.dumps(line))
     if dist is not None:

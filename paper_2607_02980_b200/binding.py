@@ -308,9 +308,9 @@ def trace_enable(on: bool) -> None:
 
 def trace_read():
     """[(kernel name, device milliseconds)] of the last traced call (waits for it to finish)."""
-    names = ctypes.create_string_buffer(8192)
-    ms = (ctypes.c_float * 128)()
-    n = load_library().hils_trace_read(names, 8192, ms, 128)
+    names = ctypes.create_string_buffer(32768)
+    ms = (ctypes.c_float * 1024)()
+    n = load_library().hils_trace_read(names, 32768, ms, 1024)
     if n < 0:
         raise HilsError(n, "hils_trace_read")
     parts = [x for x in names.value.decode().split(";") if x]

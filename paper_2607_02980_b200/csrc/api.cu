@@ -8,7 +8,7 @@ namespace {
 
 thread_local int g_last_launches = 0;
 
-constexpr int kMaxTrace = 128;
+constexpr int kMaxTrace = 1024;
 struct Trace {
     bool enabled = false;
     bool have_events = false;

@@ -49,7 +49,7 @@ int launch_prefill_select_tc(const Shape& s, const void* q, const void* landmark
 
 // tcgen05 chunk-major attention over the tile table built by the invert kernels (32-token tiles).
 int attend_tc_tile_tokens();
-int launch_prefill_attend_tc(const Shape& s, const void* q, const void* k, const void* v, const void* landmarks,
+int launch_prefill_attend_tc(const Shape& s, const void* q, const void* maps_kv, const void* landmarks,
                              const float* bias, const int* entries, const void* tiles, const int* n_tiles, void* obuf,
                              float* lam, int* status, int i0, int qb, cudaStream_t stream);
 

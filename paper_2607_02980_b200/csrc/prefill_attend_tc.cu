@@ -470,14 +470,12 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
 
 int attend_tc_tile_tokens() { return kTok; }
 
-int launch_prefill_attend_tc(const Shape& s, const void* q, const void* k, const void* v, const void* landmarks,
+int launch_prefill_attend_tc(const Shape& s, const void* q, const void* maps_kv, const void* landmarks,
                              const float* bias, const int* entries, const void* tiles, const int* n_tiles, void* obuf,
                              float* lam, int* status, int i0, int qb, cudaStream_t stream) {
-    const int pairs = s.B * s.Hkv;
-    CUtensorMap map_k, map_v;
-    const uint64_t kv_rows = static_cast<uint64_t>(pairs) * s.T;
-    if (!make_bf16_2d_map(&map_k, k, kv_rows, kD, 64, kS) || !make_bf16_2d_map(&map_v, v, kv_rows, kD, 64, kS))
-        return HILS_ERR_CUDA;
+    // maps_kv: the K and V tensor maps ([pairs*T, 128] bf16, box 64 x 64, 128B swizzle), encoded once per call
+    const CUtensorMap& map_k = static_cast<const CUtensorMap*>(maps_kv)[0];
+    const CUtensorMap& map_v = static_cast<const CUtensorMap*>(maps_kv)[1];
     const size_t smem = 2 * kKBytes + 2 * kVtBytes + kVrawBytes + kQSlots * kQBytes + 2 * kPBytes + sizeof(AtcSmem) + 1024;
     static bool attr_done = false;
     if (!attr_done) {

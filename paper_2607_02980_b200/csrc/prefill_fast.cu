@@ -768,7 +768,8 @@ int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
             prefill_attend_kernel<<<148 * 2, 128, att_smem, stream>>>(map_k, map_v, a);
             if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
         } else {
-            const int rc = launch_prefill_attend_tc(s, t.q, t.k, t.v, t.landmarks, t.bias, a.entries, a.tiles,
+            const CUtensorMap maps_kv[2] = {map_k, map_v};
+            const int rc = launch_prefill_attend_tc(s, t.q, maps_kv, t.landmarks, t.bias, a.entries, a.tiles,
                                                     a.blk_toff + blk, a.obuf, a.lam, t.status, a.i0, a.qb, stream);
             if (rc < 0) return rc;
         }
