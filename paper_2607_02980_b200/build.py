@@ -16,7 +16,7 @@ LIB = os.path.join(HERE, "libhils.so")
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-Xcompiler", "-fPIC", "-Xptxas", "-v",
-]
+] + os.environ.get("HILS_NVCC_EXTRA", "").split()      # e.g. -DNAME for tuning builds
 
 
 def _nvcc() -> str:

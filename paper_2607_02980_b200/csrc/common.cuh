@@ -92,6 +92,25 @@ __device__ inline float warp_sum(float v) {
     return v;
 }
 
+// Access policy of the prefill partial-output buffer (written once by the attend kernel, read once by the
+// fuse kernel).  Default: streaming (evict-first) both ways, so that the buffer does not push the gathered
+// queries out of L2.  -DHILS_OBUF_CACHED keeps it under the normal policy (for query blocks small enough that the
+// whole buffer stays L2-resident between the two kernels).
+__device__ inline void obuf_store(uint4* p, const uint4& v) {
+#ifdef HILS_OBUF_CACHED
+    *p = v;
+#else
+    __stcs(p, v);
+#endif
+}
+__device__ inline uint4 obuf_load(const uint4* p) {
+#ifdef HILS_OBUF_CACHED
+    return *p;
+#else
+    return __ldcs(p);
+#endif
+}
+
 __device__ inline void set_status(int* status, int code) {
     if (status) atomicCAS(status, 0, code);
 }

@@ -55,6 +55,8 @@ struct AtcSmem {
     const __nv_bfloat16* rowptr[2][kRows];
     long long orow[2][kRows];         // obuf element offset of each row of the tile in S/P/O slot i (-1: padding)
     int4 recs[kBatch];
+    int nchunks;                      // distinct (pair, chunk) runs in the current batch
+    uint8_t cfirst[kBatch + 4];       // first tile (batch index) of each run; cfirst[nchunks] = tiles in the batch
 };
 
 struct AtcArgs {
@@ -142,12 +144,26 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
         for (int x = tid; x < nb; x += kThreads) sm.recs[x] = a.tiles[b0 + x];
         __syncthreads();
         if (sm.abort_flag) break;
+        if (warp == 0) {
+            // table of chunk runs: where each run of tiles of one (pair, chunk) starts
+            int basec = 0;
+            for (int w = 0; w < kBatch / 32; ++w) {
+                const int x = w * 32 + lane;
+                const bool nw = x < nb && (x == 0 || sm.recs[x].x != sm.recs[x - 1].x || sm.recs[x].y != sm.recs[x - 1].y);
+                const unsigned m = __ballot_sync(kFullMask, nw);
+                if (nw) sm.cfirst[basec + __popc(m & ((1u << lane) - 1u))] = static_cast<uint8_t>(x);
+                basec += __popc(m);
+            }
+            if (lane == 0) { sm.cfirst[basec] = static_cast<uint8_t>(nb); sm.nchunks = basec; }
+        }
+        __syncthreads();
 
         if (warp >= kProdWarp0 && warp < kMmaWarp) {
             // ================================================================ producers (128 threads)
             const int ptid = tid - kEpiThreads, pw = warp - kProdWarp0;
             uint32_t tc = tcount, cc = ccount;
             int cur_pair = -1, cur_c = -1;
+            int ck = -1;                       // ordinal of the current chunk run within the batch
             bool next_issued = false;          // (producer thread 0) K/V of the upcoming chunk already requested
             bool dead = false;
             // entry of this thread's row for the upcoming tile, fetched one tile ahead
@@ -216,11 +232,20 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                     cur_pair = pair;
                     cur_c = c;
                     ++cc;
+                    ++ck;
+                    // warm L2 with the K/V rows of the run after the next one (the next one is requested below)
+                    if (ptid == 0 && ck + 2 < sm.nchunks) {
+                        const int4 r2 = sm.recs[sm.cfirst[ck + 2]];
+                        const int row2 = r2.x * s.T + r2.y * kS;
+                        tma_prefetch_l2_2d(&map_k, 0, row2);
+                        tma_prefetch_l2_2d(&map_k, 64, row2);
+                        tma_prefetch_l2_2d(&map_v, 0, row2);
+                        tma_prefetch_l2_2d(&map_v, 64, row2);
+                    }
                 }
                 // ---- look ahead (producer thread 0): request the next chunk's K/V as soon as its buffer is free
                 if (ptid == 0 && !next_issued) {
-                    int tj = ti + 1;
-                    while (tj < nb && sm.recs[tj].x == pair && sm.recs[tj].y == c) ++tj;
+                    const int tj = sm.cfirst[ck + 1];          // first tile of the next run (nb if none)
                     const uint32_t nbuf = cc & 1u;
                     if (tj < nb && (cc < 2 || mbar_try_wait(&sm.kv_empty[nbuf], ((cc >> 1) - 1) & 1))) {
                         const int row = sm.recs[tj].x * s.T + sm.recs[tj].y * kS;
@@ -436,8 +461,8 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                         const int r = (warp & 3) * 32 + it * 4 + (lane >> 3), pc = lane & 7;
                         const long long off = offs[it];
                         if (off >= 0)      // streaming store: written once, read once by prefill_fuse
-                            __stcs(reinterpret_cast<uint4*>(a.obuf + off + hb * 64 + pc * 8),
-                                   *reinterpret_cast<const uint4*>(pslot + swz128(r, pc)));
+                            obuf_store(reinterpret_cast<uint4*>(a.obuf + off + hb * 64 + pc * 8),
+                                       *reinterpret_cast<const uint4*>(pslot + swz128(r, pc)));
                     }
                     __syncwarp();
                 }
@@ -448,14 +473,8 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
             if (!ok && lane == 0) { set_status(a.status, kDevTimeout); atomicExch(&sm.abort_flag, 1); }
         }
         // every role advances the shared counters identically
-        {
-            uint32_t chunks = 0;
-            int cp = -1, cq = -1;
-            for (int ti = 0; ti < nb; ++ti)
-                if (sm.recs[ti].x != cp || sm.recs[ti].y != cq) { ++chunks; cp = sm.recs[ti].x; cq = sm.recs[ti].y; }
-            tcount += static_cast<uint32_t>(nb);
-            ccount += chunks;
-        }
+        tcount += static_cast<uint32_t>(nb);
+        ccount += static_cast<uint32_t>(sm.nchunks);
         __syncthreads();
         if (sm.abort_flag) break;
     }

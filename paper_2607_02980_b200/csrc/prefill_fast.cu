@@ -587,8 +587,8 @@ __global__ void __launch_bounds__(kFuseWarps * 32) prefill_fuse_kernel(const PAr
     // local slot first, then the selected slots four at a time (8 loads in flight per lane)
     {
         const __nv_bfloat16* row = ob + static_cast<long long>(K) * kG * kD;
-        const uint4 ra = __ldcs(reinterpret_cast<const uint4*>(row + lane * 8));
-        const uint4 rb = __ldcs(reinterpret_cast<const uint4*>(row + 256 + lane * 8));
+        const uint4 ra = obuf_load(reinterpret_cast<const uint4*>(row + lane * 8));
+        const uint4 rb = obuf_load(reinterpret_cast<const uint4*>(row + 256 + lane * 8));
         fma8(accA, ra, wv[hA][64]);
         fma8(accB, rb, wv[hB][64]);
     }
@@ -598,8 +598,8 @@ __global__ void __launch_bounds__(kFuseWarps * 32) prefill_fuse_kernel(const PAr
         for (int u = 0; u < 4; ++u) {
             const int sl = min(sl0 + u, nsel - 1);
             const __nv_bfloat16* row = ob + static_cast<long long>(sl) * kG * kD;
-            ra[u] = __ldcs(reinterpret_cast<const uint4*>(row + lane * 8));
-            rb[u] = __ldcs(reinterpret_cast<const uint4*>(row + 256 + lane * 8));
+            ra[u] = obuf_load(reinterpret_cast<const uint4*>(row + lane * 8));
+            rb[u] = obuf_load(reinterpret_cast<const uint4*>(row + 256 + lane * 8));
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
