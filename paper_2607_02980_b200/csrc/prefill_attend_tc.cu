@@ -4,11 +4,11 @@
 // Per tile:  S = Q K_c^T (M=128, N=80: 64 keys + the chunk's landmark as key 64, K=128) -> tensor memory;
 //            each epilogue thread owns one row: mask (local rows are causal), the chunk's own softmax
 //            (Eq. HiLS weights, intra-chunk factor), P as bf16 back to shared memory;
-//            O = P V_c (M=128, N=128, K=64, V pre-transposed once per chunk) -> tensor memory;
+//            O = P V_c (M=128, N=128, K=64, V read as an MN-major operand exactly as TMA wrote it) -> tensor memory;
 //            normalised bf16 rows and the row's chunk mass (surrogate score, or log Z_swa for the
 //            local branch) go to the buffers that prefill_fuse mixes.
 // Warp roles: 0-7 epilogue (warps 0-3 take even tiles, 4-7 odd tiles; a warp reads the TMEM lane quarter
-// warp % 4), 8-11 producers (cp.async gather of Q rows, TMA of K/V, V transpose), 12 MMA issue.
+// warp % 4), 8-11 producers (cp.async gather of Q rows, TMA of K/V), 12 MMA issue.
 // S/P/O are double buffered, three gathered Q tiles are in flight, K/V is double buffered per chunk.
 #include "internal.h"
 #include "tma.cuh"
@@ -23,8 +23,7 @@ constexpr int kTok = 32;                        // entries per tile
 constexpr int kRows = kTok * kG;                // 128
 constexpr int kNS = 80;                         // score columns: 64 keys + landmark (+15 zero rows)
 constexpr int kKBytes = kNS * 128 * 2;          // two 64-dim K-blocks of 80 rows
-constexpr int kVtBytes = kD * 128;              // 128 d-rows x 64 keys
-constexpr int kVrawBytes = kS * kD * 2;
+constexpr int kVBytes = kS * kD * 2;            // two boxes of 64 keys x 64 dims
 constexpr int kQBytes = kRows * kD * 2;         // 32 KB
 constexpr int kPBytes = kRows * 128;            // 16 KB
 constexpr int kBatch = 128;                     // tile records cached per batch
@@ -38,8 +37,8 @@ constexpr int kMmaWarp = kProdWarp0 + kProdThreads / 32;
 constexpr float kLog2e = 1.4426950408889634f;
 
 struct AtcSmem {
-    uint64_t kraw_full;       // TMA of K rows + raw V landed
-    uint64_t kv_ready[2];     // K tile (with landmark row) and transposed V usable by the MMA
+    uint64_t kraw_full;       // TMA of the K and V rows landed
+    uint64_t kv_ready[2];     // K tile (with landmark row) and V usable by the MMA
     uint64_t kv_empty[2];     // every MMA that reads this K/V buffer has completed
     uint64_t q_full[kQSlots]; // gathered Q rows landed and fenced (one arrival per producer warp)
     uint64_t q_empty[kQSlots];// the S MMA that reads this Q tile has completed
@@ -93,9 +92,8 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* kbuf = base;                                   // [2][kKBytes]
-    uint8_t* vt = kbuf + 2 * kKBytes;                       // [2][kVtBytes]
-    uint8_t* vraw = vt + 2 * kVtBytes;                      // [kVrawBytes]
-    uint8_t* qbuf = vraw + kVrawBytes;                      // [kQSlots][kQBytes]
+    uint8_t* vbuf = kbuf + 2 * kKBytes;                     // [2][kVBytes]
+    uint8_t* qbuf = vbuf + 2 * kVBytes;                     // [kQSlots][kQBytes]
     uint8_t* pbuf = qbuf + kQSlots * kQBytes;               // [2][kPBytes]
     AtcSmem& sm = *reinterpret_cast<AtcSmem*>(pbuf + 2 * kPBytes);
 
@@ -182,11 +180,11 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                         if (cc >= 2 && !mbar_wait(&sm.kv_empty[cbuf], ((cc >> 1) - 1) & 1)) dead = true;
                         if (!dead) {
                             const int row = pair * s.T + c * kS;
-                            mbar_expect_tx(&sm.kraw_full, 2 * 8192 + kVrawBytes);
+                            mbar_expect_tx(&sm.kraw_full, 2 * 8192 + kVBytes);
                             tma_load_2d(kbuf + cbuf * kKBytes, &map_k, &sm.kraw_full, 0, row);
                             tma_load_2d(kbuf + cbuf * kKBytes + kNS * 128, &map_k, &sm.kraw_full, 64, row);
-                            tma_load_2d(vraw, &map_v, &sm.kraw_full, 0, row);
-                            tma_load_2d(vraw + 8192, &map_v, &sm.kraw_full, 64, row);
+                            tma_load_2d(vbuf + cbuf * kVBytes, &map_v, &sm.kraw_full, 0, row);
+                            tma_load_2d(vbuf + cbuf * kVBytes + 8192, &map_v, &sm.kraw_full, 64, row);
                         }
                     }
                     next_issued = false;
@@ -198,34 +196,8 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                         if (c < s.C) v = *reinterpret_cast<const uint4*>(a.lm + (static_cast<long long>(pair) * s.C + c) * kD + ptid * 8);
                         *reinterpret_cast<uint4*>(kbuf + cbuf * kKBytes + (ptid >> 3) * (kNS * 128) + swz128(64, ptid & 7)) = v;
                     }
-                    // V^T: 8x8 blocks through ldmatrix.trans (8 of the 32 blocks per warp); keys past the
-                    // end of the sequence become 0
-                    const int nv = min(kS, s.R - c * kS);
-                    uint8_t* vtb = vt + cbuf * kVtBytes;
-                    const uint32_t vraw_addr = smem_u32(vraw);
-#pragma unroll 2
-                    for (int bi = 0; bi < 8; ++bi) {
-                        const int blk = pw * 8 + bi;
-                        // block = 16 keys x 16 dims: four 8x8 matrices (keys lo/hi x dims lo/hi)
-                        const int k0 = (blk & 3) * 16, d0 = (blk >> 2) * 16;
-                        const int mat = lane >> 3;
-                        const int row = k0 + (mat & 1) * 8 + (lane & 7);
-                        const int dim = d0 + (mat >> 1) * 8;
-                        uint32_t r0, r1, r2, r3;
-                        ldmatrix_x4_trans(vraw_addr + (dim >> 6) * 8192 + swz128(row, (dim & 63) >> 3), r0, r1, r2, r3);
-                        // thread (g,t): r0 = V[k0+2t..+1][d0+g], r1 = V[k0+8+2t..][d0+g], r2/r3: dims d0+8+g
-                        const int g = lane >> 2, t = lane & 3;
-                        const uint32_t vals[4] = {r0, r1, r2, r3};
-#pragma unroll
-                        for (int m = 0; m < 4; ++m) {
-                            const int dd = d0 + (m >> 1) * 8 + g;
-                            const int key = k0 + (m & 1) * 8 + 2 * t;
-                            uint32_t v = vals[m];
-                            if (key >= nv) v = 0u;
-                            else if (key + 1 >= nv) v &= 0x0000ffffu;
-                            *reinterpret_cast<uint32_t*>(vtb + swz128(dd, key >> 3) + (key & 7) * 2) = v;
-                        }
-                    }
+                    // V stays as TMA wrote it (keys x dims): the second MMA reads it as an MN-major operand.  Keys past
+                    // the end of the sequence hold other rows' data (or TMA zero fill) and meet probabilities of 0.
                     fence_proxy_async_smem();
                     producer_barrier();
                     if (ptid == 0) mbar_arrive(&sm.kv_ready[cbuf]);
@@ -249,11 +221,11 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                     const uint32_t nbuf = cc & 1u;
                     if (tj < nb && (cc < 2 || mbar_try_wait(&sm.kv_empty[nbuf], ((cc >> 1) - 1) & 1))) {
                         const int row = sm.recs[tj].x * s.T + sm.recs[tj].y * kS;
-                        mbar_expect_tx(&sm.kraw_full, 2 * 8192 + kVrawBytes);
+                        mbar_expect_tx(&sm.kraw_full, 2 * 8192 + kVBytes);
                         tma_load_2d(kbuf + nbuf * kKBytes, &map_k, &sm.kraw_full, 0, row);
                         tma_load_2d(kbuf + nbuf * kKBytes + kNS * 128, &map_k, &sm.kraw_full, 64, row);
-                        tma_load_2d(vraw, &map_v, &sm.kraw_full, 0, row);
-                        tma_load_2d(vraw + 8192, &map_v, &sm.kraw_full, 64, row);
+                        tma_load_2d(vbuf + nbuf * kVBytes, &map_v, &sm.kraw_full, 0, row);
+                        tma_load_2d(vbuf + nbuf * kVBytes + 8192, &map_v, &sm.kraw_full, 64, row);
                         next_issued = true;
                     }
                 }
@@ -303,7 +275,7 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
             // ================================================================ MMA issuer
             if (lane == 0) {
                 constexpr uint32_t idesc_s = umma_idesc_bf16(kRows, kNS);
-                constexpr uint32_t idesc_o = umma_idesc_bf16(kRows, kD);
+                constexpr uint32_t idesc_o = umma_idesc_bf16(kRows, kD) | kUmmaBMnMajor;
                 uint32_t cc = ccount;
                 int cur_pair = -1, cur_c = -1;
                 uint32_t cbuf_of[2] = {0u, 0u};        // K/V buffer used by the tile in S/P/O slot i
@@ -343,11 +315,11 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                         if (ready && tcv >= 2) ready = mbar_try_wait(&sm.o_empty[sl], ((tcv >> 1) - 1) & 1);
                         if (ready) {
                             tc_fence_after_sync();
-                            const uint32_t pa = smem_u32(pbuf + sl * kPBytes), va = smem_u32(vt + cb * kVtBytes);
+                            const uint32_t pa = smem_u32(pbuf + sl * kPBytes), va = smem_u32(vbuf + cb * kVBytes);
 #pragma unroll
-                            for (int ks = 0; ks < 4; ++ks)
-                                umma_bf16(tmem_base + 256 + sl * 128, umma_desc_k128(pa + ks * 32), umma_desc_k128(va + ks * 32),
-                                          idesc_o, ks > 0 ? 1u : 0u);
+                            for (int ks = 0; ks < 4; ++ks)      // 16 keys per step = two 8-row groups of V
+                                umma_bf16(tmem_base + 256 + sl * 128, umma_desc_k128(pa + ks * 32),
+                                          umma_desc_mn128(va + ks * 2048, 8192u, 1024u), idesc_o, ks > 0 ? 1u : 0u);
                             umma_commit(&sm.o_full[sl]);
                             // last tile of its chunk in this batch: the K/V buffer is free once these MMAs are done
                             const bool last = no + 1 >= nb || sm.recs[no + 1].x != sm.recs[no].x || sm.recs[no + 1].y != sm.recs[no].y;
@@ -495,7 +467,7 @@ int launch_prefill_attend_tc(const Shape& s, const void* q, const void* maps_kv,
     // maps_kv: the K and V tensor maps ([pairs*T, 128] bf16, box 64 x 64, 128B swizzle), encoded once per call
     const CUtensorMap& map_k = static_cast<const CUtensorMap*>(maps_kv)[0];
     const CUtensorMap& map_v = static_cast<const CUtensorMap*>(maps_kv)[1];
-    const size_t smem = 2 * kKBytes + 2 * kVtBytes + kVrawBytes + kQSlots * kQBytes + 2 * kPBytes + sizeof(AtcSmem) + 1024;
+    const size_t smem = 2 * kKBytes + 2 * kVBytes + kQSlots * kQBytes + 2 * kPBytes + sizeof(AtcSmem) + 1024;
     static bool attr_done = false;
     if (!attr_done) {
         if (cudaFuncSetAttribute(prefill_attend_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,

@@ -137,6 +137,20 @@ __device__ __forceinline__ uint64_t umma_desc_k128(uint32_t smem_addr) {
     return d;
 }
 
+// The same storage read as an MN-major operand: element (n, k) sits in row k, column n of 128-byte swizzled rows,
+// so n is the contiguous index.  lbo = bytes between 64-element blocks along n (one TMA box each),
+// sbo = bytes between 8-row groups along k.  Needs the "MN-major" bit of the instruction descriptor.
+__device__ __forceinline__ uint64_t umma_desc_mn128(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((smem_addr & 0x3ffffu) >> 4);
+    d |= static_cast<uint64_t>(lbo_bytes >> 4) << 16;
+    d |= static_cast<uint64_t>(sbo_bytes >> 4) << 32;
+    d |= static_cast<uint64_t>(1) << 46;
+    d |= static_cast<uint64_t>(2) << 61;
+    return d;
+}
+constexpr uint32_t kUmmaBMnMajor = 1u << 16;      // instruction-descriptor bit: B operand is MN-major
+
 // One warp allocates `ncols` (power of two >= 32) tensor-memory columns; the base address is written
 // to shared memory.  The same warp must free them before the CTA exits.
 __device__ __forceinline__ void tmem_alloc(uint32_t* smem_dst, uint32_t ncols) {
