@@ -5,7 +5,10 @@
 // tcgen05.mma (M = 128 tokens, N = 64 chunks, K = 128) once per head into tensor memory, double
 // buffered; the four epilogue warps own one token per thread (token = TMEM lane), read the four
 // heads' scores, take the group max (App. C) and keep the token's exact running top-K
-// (Eq. surrogate top-k; equal scores go to the lower chunk id) in a private shared-memory list.
+// (Eq. surrogate top-k; equal scores go to the lower chunk id): candidates that beat the current
+// K-th score are appended to a private buffer; when a buffer of the warp fills up, every thread sorts
+// its buffer with a register bitonic network and merges it into its sorted top list, which raises the
+// threshold.  The number of such merges grows with log(candidates / K), not with the candidates.
 #include "internal.h"
 #include "tma.cuh"
 
@@ -19,7 +22,6 @@ constexpr int kTileTok = 128;
 constexpr int kLmStages = 2;
 constexpr int kLmStageBytes = kS * kD * 2;          // 64 landmark rows = two 8 KB K-blocks
 constexpr int kQBytes = kG * kTileTok * kD * 2;     // 128 KB
-constexpr int kQueueCap = 32;
 constexpr int kMaxK = 32;
 constexpr int kThreads = 192;                       // 4 epilogue warps, 1 TMA warp, 1 MMA warp
 constexpr uint32_t kTmemCols = 512;                 // 2 buffers x 4 heads x 64 columns
@@ -40,6 +42,81 @@ struct TcSmem {
     uint32_t tmem_base;
 };
 
+// Sorts N keys in registers, largest first (bitonic network, fully unrolled: static register indices).
+template <int N>
+__device__ __forceinline__ void bitonic_sort_desc(unsigned long long (&a)[N]) {
+    constexpr int kLog = N == 32 ? 5 : 4;
+#pragma unroll
+    for (int ks = 1; ks <= kLog; ++ks) {
+#pragma unroll
+        for (int js = kLog - 1; js >= 0; --js) {
+            if (js >= ks) continue;
+            const int k = 1 << ks, j = 1 << js;
+#pragma unroll
+            for (int i = 0; i < N; ++i) {
+                const int l = i ^ j;
+                if (l > i) {
+                    const bool desc = (i & k) == 0;
+                    const unsigned long long x = a[i], y = a[l];
+                    const bool sw = desc ? (x < y) : (x > y);
+                    a[i] = sw ? y : x;
+                    a[l] = sw ? x : y;
+                }
+            }
+        }
+    }
+}
+// Sorts a bitonic sequence of N keys, largest first.
+template <int N>
+__device__ __forceinline__ void bitonic_merge_desc(unsigned long long (&a)[N]) {
+    constexpr int kLog = N == 32 ? 5 : 4;
+#pragma unroll
+    for (int js = kLog - 1; js >= 0; --js) {
+        const int j = 1 << js;
+#pragma unroll
+        for (int i = 0; i < N; ++i) {
+            const int l = i ^ j;
+            if (l > i) {
+                const unsigned long long x = a[i], y = a[l];
+                const bool sw = x < y;
+                a[i] = sw ? y : x;
+                a[l] = sw ? x : y;
+            }
+        }
+    }
+}
+
+// Merges a thread's append buffer (qn raw (score bits, chunk id) pairs at myq[e * 128]) into its sorted top list
+// (mytop[e * 128], largest first, 0 = empty): exact keys, register bitonic sort of the buffer, the N largest of
+// both lists, sorted again.  Returns the score of the K-th best key (-inf while fewer than K are known).
+// One copy of this code per N (not inlined: it is a few thousand instructions).
+template <int N>
+__device__ __noinline__ float merge_buffer(unsigned long long* mytop, const unsigned long long* myq, int qn, int K) {
+    unsigned long long kb[N];
+#pragma unroll
+    for (int e = 0; e < N; ++e) {
+        const unsigned long long raw = myq[e * kTileTok];
+        const unsigned long long key =
+            select_key(__uint_as_float(static_cast<uint32_t>(raw >> 32)), static_cast<int>(raw & 0xffffffffull));
+        kb[e] = e < qn ? key : 0ull;
+    }
+    bitonic_sort_desc<N>(kb);
+#pragma unroll
+    for (int e = 0; e < N / 2; ++e) {
+        const unsigned long long x = kb[e], y = kb[N - 1 - e];
+        const unsigned long long t0 = mytop[e * kTileTok], t1 = mytop[(N - 1 - e) * kTileTok];
+        kb[e] = t0 > y ? t0 : y;
+        kb[N - 1 - e] = t1 > x ? t1 : x;
+    }
+    bitonic_merge_desc<N>(kb);
+#pragma unroll
+    for (int e = 0; e < N; ++e) mytop[e * kTileTok] = kb[e];
+    const unsigned long long tau = mytop[(K - 1) * kTileTok];
+    return tau ? key_to_float(static_cast<uint32_t>(tau >> 32)) : -INFINITY;
+}
+
+// N = length of the per-token top list and of the append buffer: 16 for K <= 16, else 32.
+template <int N>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_lm,
                          const TcArgs a) {
@@ -48,7 +125,7 @@ prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     uint8_t* lms = qs + kQBytes;
     unsigned long long* lists = reinterpret_cast<unsigned long long*>(lms + kLmStages * kLmStageBytes);
     unsigned long long* queue = lists + kMaxK * kTileTok;
-    TcSmem& sm = *reinterpret_cast<TcSmem*>(queue + kQueueCap * kTileTok);
+    TcSmem& sm = *reinterpret_cast<TcSmem*>(queue + kMaxK * kTileTok);
 
     const Shape& s = a.s;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -139,42 +216,17 @@ prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         const int tok = ti * kTileTok + row;
         const int my_ncand = row < kS ? 2 * ti : 2 * ti + 1;
         const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
-        unsigned long long* mylist = lists + tid;          // entry e at mylist[e * 128]
-        unsigned long long* myq = queue + tid;
+        unsigned long long* mytop = lists + tid;           // sorted top list: entry e at mytop[e * 128], 0 = empty
+        unsigned long long* myq = queue + tid;             // append buffer of raw (score bits, chunk id) pairs
         const float* bias = a.bias ? a.bias + static_cast<long long>(pair) * s.C : nullptr;
-        unsigned long long tau = 0ull;
-        int cnt = 0, pmin = 0, qn = 0;
+        float tau_f = -INFINITY;           // score of the K-th best key so far: the filter of the scan
+        int qn = 0;
         bool ok = true;
-
-        auto drain = [&]() {
-            int mx = qn;
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(kFullMask, mx, o));
-            for (int i = 0; i < mx; ++i) {
-                if (i < qn) {
-                    const unsigned long long key = myq[i * kTileTok];
-                    if (key > tau) {
-                        bool rescan = true;
-                        if (cnt < K) {
-                            mylist[cnt * kTileTok] = key;
-                            ++cnt;
-                            rescan = cnt == K;
-                        } else {
-                            mylist[pmin * kTileTok] = key;
-                        }
-                        if (rescan) {
-                            unsigned long long mn = ~0ull;
-                            int pm = 0;
-                            for (int e = 0; e < K; ++e) {
-                                const unsigned long long x = mylist[e * kTileTok];
-                                if (x < mn) { mn = x; pm = e; }
-                            }
-                            tau = mn;
-                            pmin = pm;
-                        }
-                    }
-                }
-            }
+        for (int e = 0; e < N; ++e) mytop[e * kTileTok] = 0ull;
+
+        auto compact = [&]() {
+            tau_f = merge_buffer<N>(mytop, myq, qn, K);
             qn = 0;
         };
 
@@ -183,45 +235,43 @@ prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             ok = mbar_wait(&sm.tmem_full[buf], (it >> 1) & 1);
             if (!ok) break;
             tc_fence_after_sync();
+            const bool tail = (it + 1) * kS > my_ncand;     // only the last step holds chunks this token may not see
 #pragma unroll 1
             for (int cb = 0; cb < 4; ++cb) {
-                float um[16], r[16];
-                const uint32_t col = buf * 256 + cb * 16;
-                tmem_ld16(t_lane + col, um);
-#pragma unroll
-                for (int h = 1; h < kG; ++h) {
-                    tmem_ld16(t_lane + col + h * kS, r);
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) um[j] = fmaxf(um[j], r[j]);
-                }
+                float r[4][16];
+                const uint32_t col = t_lane + buf * 256 + cb * 16;
+                tmem_ld16x4(col, col + kS, col + 2 * kS, col + 3 * kS, r);
                 const int c0 = it * kS + cb * 16;
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
                     const int c = c0 + j;
-                    float u = um[j] * s.scale;
+                    float u = fmaxf(fmaxf(r[0][j], r[1][j]), fmaxf(r[2][j], r[3][j])) * s.scale;
                     if (bias) u += bias[min(c, s.C - 1)];
-                    const unsigned long long key = select_key(u, c);
-                    const bool pass = c < my_ncand && key > tau;
-                    // branch-free append: the slot is written always and kept only when the key passes
-                    myq[qn * kTileTok] = key;
+                    // first filter on the score alone (ties pass and are settled on the full key when draining);
+                    // branch-free append: the slot is written always and kept only when the candidate passes
+                    const bool pass = u >= tau_f && (!tail || c < my_ncand);
+                    myq[qn * kTileTok] = (static_cast<unsigned long long>(__float_as_uint(u)) << 32) | static_cast<uint32_t>(c);
                     qn += pass ? 1 : 0;
+                    // at most 8 appends between checks: a buffer never overflows
+                    if ((j & 7) == 7 && __any_sync(kFullMask, qn > N - 8)) compact();
                 }
-                if (__any_sync(kFullMask, qn > kQueueCap - 17)) drain();
             }
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm.tmem_empty[buf]);
         }
         if (!ok && lane == 0) set_status(a.status, kDevTimeout);
-        drain();
+        compact();
 
-        // ascending chunk ids, -1 padded
+        // the first K entries of the top list (0 = none), emitted as ascending chunk ids, -1 padded
         if (tok < s.R) {
             int32_t* sel = a.sel + (static_cast<long long>(pair) * s.R + tok) * K;
+            int cnt = 0;
+            for (int e = 0; e < K; ++e) cnt += mytop[e * kTileTok] != 0ull ? 1 : 0;
             for (int e = 0; e < cnt; ++e) {
-                const int id = key_chunk(mylist[e * kTileTok]);
+                const int id = key_chunk(mytop[e * kTileTok]);
                 int rank = 0;
-                for (int j = 0; j < cnt; ++j) rank += key_chunk(mylist[j * kTileTok]) < id ? 1 : 0;
+                for (int j = 0; j < cnt; ++j) rank += key_chunk(mytop[j * kTileTok]) < id ? 1 : 0;
                 sel[rank] = id;
             }
             for (int e = cnt; e < K; ++e) sel[e] = -1;
@@ -247,18 +297,22 @@ int launch_prefill_select_tc(const Shape& s, const void* q, const void* landmark
     if (!make_bf16_2d_map(&map_q, q, static_cast<uint64_t>(s.B) * s.Hq * s.R, kD, 64, kTileTok) ||
         !make_bf16_2d_map(&map_lm, landmarks, static_cast<uint64_t>(pairs) * s.C, kD, 64, kS))
         return HILS_ERR_CUDA;
-    const size_t smem = kQBytes + kLmStages * kLmStageBytes + sizeof(unsigned long long) * (kMaxK + kQueueCap) * kTileTok +
+    const size_t smem = kQBytes + kLmStages * kLmStageBytes + sizeof(unsigned long long) * 2 * kMaxK * kTileTok +
                         sizeof(TcSmem) + 1024;
     static bool attr_done = false;
     if (!attr_done) {
-        if (cudaFuncSetAttribute(prefill_select_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(prefill_select_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(smem)) != cudaSuccess ||
+            cudaFuncSetAttribute(prefill_select_tc_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(smem)) != cudaSuccess)
             return HILS_ERR_CUDA;
         attr_done = true;
     }
     TcArgs a{s, bias, sel, status};
     const int tiles = (s.R + kTileTok - 1) / kTileTok;
-    prefill_select_tc_kernel<<<static_cast<unsigned>(pairs) * tiles, kThreads, smem, stream>>>(map_q, map_lm, a);
+    const unsigned grid = static_cast<unsigned>(pairs) * tiles;
+    if (s.K <= 16) prefill_select_tc_kernel<16><<<grid, kThreads, smem, stream>>>(map_q, map_lm, a);
+    else prefill_select_tc_kernel<32><<<grid, kThreads, smem, stream>>>(map_q, map_lm, a);
     if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
     return 1;
 }
