@@ -49,9 +49,11 @@ int launch_prefill_select_tc(const Shape& s, const void* q, const void* landmark
 
 // tcgen05 chunk-major attention over the tile table built by the invert kernels (32-token tiles).
 int attend_tc_tile_tokens();
-int launch_prefill_attend_tc(const Shape& s, const void* q, const void* maps_kv, const void* landmarks,
-                             const float* bias, const int* entries, const void* tiles, const int* n_tiles, void* obuf,
-                             float* lam, int* status, int i0, int qb, cudaStream_t stream);
+// maps: CUtensorMap[3] = K, V ([pairs*T, 128] bf16, boxes of 64 x 64) and the partial-output buffer
+// ([entries of a block * 4 heads, 128] bf16, boxes of 64 x 32), all with the 128-byte swizzle.
+int launch_prefill_attend_tc(const Shape& s, const void* q, const void* maps, const void* landmarks,
+                             const float* bias, const int* entries, const void* tiles, const int* n_tiles, float* lam,
+                             int* status, int i0, cudaStream_t stream);
 
 int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream);
 bool prefill_fast_supports(const Shape& s, int dtype);

@@ -6,7 +6,8 @@
 //            (Eq. HiLS weights, intra-chunk factor), P as bf16 back to shared memory;
 //            O = P V_c (M=128, N=128, K=64, V read as an MN-major operand exactly as TMA wrote it) -> tensor memory;
 //            normalised bf16 rows and the row's chunk mass (surrogate score, or log Z_swa for the
-//            local branch) go to the buffers that prefill_fuse mixes.
+//            local branch) go to the buffers that prefill_fuse mixes, in entry order: a tile's 128 rows
+//            are contiguous there, so every epilogue warp hands its 32 rows to one TMA store per half.
 // Warp roles: 0-7 epilogue (warps 0-3 take even tiles, 4-7 odd tiles; a warp reads the TMEM lane quarter
 // warp % 4), 8-11 producers (cp.async gather of Q rows, TMA of K/V), 12 MMA issue.
 // S/P/O are double buffered, three gathered Q tiles are in flight, K/V is double buffered per chunk.
@@ -50,9 +51,8 @@ struct AtcSmem {
     uint32_t tmem_base;
     int abort_flag;
     int tile_ent[kMetaSlots][kTok];   // entries of the tiles in flight
-    int tile_meta[kMetaSlots][4];     // pair, chunk, tokens, unused
+    int tile_meta[kMetaSlots][4];     // pair, chunk, tokens, first entry relative to the query block
     const __nv_bfloat16* rowptr[2][kRows];
-    long long orow[2][kRows];         // obuf element offset of each row of the tile in S/P/O slot i (-1: padding)
     int4 recs[kBatch];
     int nchunks;                      // distinct (pair, chunk) runs in the current batch
     uint8_t cfirst[kBatch + 4];       // first tile (batch index) of each run; cfirst[nchunks] = tiles in the batch
@@ -66,10 +66,9 @@ struct AtcArgs {
     const int* entries;
     const int4* tiles;
     const int* n_tiles;
-    __nv_bfloat16* obuf;
     float* lam;
     int* status;
-    int i0, qb;
+    int i0;
 };
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
@@ -88,7 +87,7 @@ __device__ __forceinline__ void producer_barrier() { asm volatile("bar.sync 2, %
 
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
-                         const AtcArgs a) {
+                         const __grid_constant__ CUtensorMap map_o, const AtcArgs a) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* kbuf = base;                                   // [2][kKBytes]
@@ -99,7 +98,6 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
 
     const Shape& s = a.s;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int K1 = s.K + 1;
     // a.n_tiles points at {first tile of this query block, first tile of the next one}
     const int t_begin = a.n_tiles[0], n_tiles = a.n_tiles[1] - t_begin;
     const long long lo = t_begin + static_cast<long long>(blockIdx.x) * n_tiles / gridDim.x;
@@ -121,6 +119,7 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
         sm.abort_flag = 0;
         tma_prefetch_desc(&map_k);
         tma_prefetch_desc(&map_v);
+        tma_prefetch_desc(&map_o);
     }
     // rows 64..79 of both K-blocks of both K buffers: landmark row + zero rows (TMA never writes them)
     for (int x = tid; x < 2 * 2 * 16 * 8; x += kThreads) {
@@ -238,7 +237,7 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                     const int bb = pair / s.Hkv, gk = pair % s.Hkv;
                     sm.rowptr[rb][ptid] = a.q + ((static_cast<long long>(bb) * s.Hq + gk * kG + hd) * s.R + a.i0 + (e >> 8)) * kD;
                     if (hd == 0) sm.tile_ent[ms][tk] = e;
-                    if (ptid == 0) { sm.tile_meta[ms][0] = pair; sm.tile_meta[ms][1] = c; sm.tile_meta[ms][2] = ntok; }
+                    if (ptid == 0) { sm.tile_meta[ms][0] = pair; sm.tile_meta[ms][1] = c; sm.tile_meta[ms][2] = ntok; sm.tile_meta[ms][3] = rec.z - t_begin * kTok; }
                     producer_barrier();
                     const uint32_t qaddr = smem_u32(qbuf + qs * kQBytes);
                     const int p16 = lane & 15;
@@ -346,6 +345,7 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
             const float sl2 = s.scale * kLog2e;
             const uint32_t sl = static_cast<uint32_t>(grp);
             uint8_t* pslot = pbuf + sl * kPBytes;
+            const uint64_t pol = l2_policy_evict_first();
             bool ok = true;
             for (int ti = 0; ti < nb && ok; ++ti) {
                 const uint32_t tcv = tcount + ti;
@@ -355,7 +355,8 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                 if (!ok) break;
                 tc_fence_after_sync();
                 const uint32_t ms = tcv % kMetaSlots;
-                const int pair = sm.tile_meta[ms][0], c = sm.tile_meta[ms][1], ntok = sm.tile_meta[ms][2];
+                const int pair = sm.tile_meta[ms][0], c = sm.tile_meta[ms][1];
+                const int orow0 = sm.tile_meta[ms][3] * kG;          // first row of the tile in the output buffers
                 const int e = sm.tile_ent[ms][tk];
                 const int il = e >> 8, slot = e & 255;
                 const bool local = slot == s.K;
@@ -381,6 +382,9 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                     }
                     float z = 0.f;
                     const float ms2 = m * sl2;
+                    // this warp's rows of the slot staged the previous tile's output: its store must have read them
+                    if (lane == 0) bulk_wait_read<0>();
+                    __syncwarp();
 #pragma unroll
                     for (int pc = 0; pc < 8; ++pc) {
                         uint32_t pk[4];
@@ -394,13 +398,9 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                         *reinterpret_cast<uint4*>(pslot + swz128(row, pc)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                     }
                     zi = 1.f / z;
-                    const bool real = tk < ntok;
-                    sm.orow[sl][row] = real ? (((static_cast<long long>(pair) * a.qb + il) * K1 + slot) * kG + hd) * kD : -1;
-                    if (real) {
-                        const float bb = (a.bias && c < s.C) ? a.bias[static_cast<long long>(pair) * s.C + c] : 0.f;
-                        a.lam[((static_cast<long long>(pair) * a.qb + il) * kG + hd) * K1 + slot] =
-                            local ? m * s.scale + __logf(z) : lmk * s.scale + bb;
-                    }
+                    // chunk mass of the row (rows of a ragged tile's padding land in the list's padding)
+                    const float bb = (a.bias && c < s.C) ? a.bias[static_cast<long long>(pair) * s.C + c] : 0.f;
+                    a.lam[orow0 + row] = local ? m * s.scale + __logf(z) : lmk * s.scale + bb;
                 }
                 fence_proxy_async_smem();
                 __syncwarp();
@@ -409,34 +409,31 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                 ok = mbar_wait(&sm.o_full[sl], (tcv >> 1) & 1);
                 if (!ok) break;
                 tc_fence_after_sync();
-                // P has been consumed: its slot stages the output, 64 columns (128 bytes per row) at a time,
-                // so that every store instruction writes four full 128-byte segments
-                long long offs[8];
-#pragma unroll
-                for (int it = 0; it < 8; ++it) offs[it] = sm.orow[sl][(warp & 3) * 32 + it * 4 + (lane >> 3)];
+                // P has been consumed: the warp's 32 rows of its slot (4 KB, swizzled as the output map expects) stage
+                // the output, 64 columns at a time; one TMA store per half writes 32 full rows
+                uint8_t* wstg = pslot + (warp & 3) * 4096;
 #pragma unroll 1
                 for (int hb = 0; hb < 2; ++hb) {
+                    uint32_t pk[32];
                     {
                         float v[64];
                         tmem_ld64(t_lane + 256 + sl * 128 + hb * 64, v);
 #pragma unroll
-                        for (int pc = 0; pc < 8; ++pc) {
-                            uint32_t pk[4];
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) pk[j] = pack_bf16(v[pc * 8 + 2 * j] * zi, v[pc * 8 + 2 * j + 1] * zi);
-                            *reinterpret_cast<uint4*>(pslot + swz128(row, pc)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                        }
+                        for (int j = 0; j < 32; ++j) pk[j] = pack_bf16(v[2 * j] * zi, v[2 * j + 1] * zi);
                     }
-                    __syncwarp();
-#pragma unroll
-                    for (int it = 0; it < 8; ++it) {
-                        const int r = (warp & 3) * 32 + it * 4 + (lane >> 3), pc = lane & 7;
-                        const long long off = offs[it];
-                        if (off >= 0)      // streaming store: written once, read once by prefill_fuse
-                            obuf_store(reinterpret_cast<uint4*>(a.obuf + off + hb * 64 + pc * 8),
-                                       *reinterpret_cast<const uint4*>(pslot + swz128(r, pc)));
+                    if (hb == 1) {
+                        if (lane == 0) bulk_wait_read<0>();
+                        __syncwarp();
                     }
+#pragma unroll
+                    for (int pc = 0; pc < 8; ++pc)
+                        *reinterpret_cast<uint4*>(pslot + swz128(row, pc)) = make_uint4(pk[4 * pc], pk[4 * pc + 1], pk[4 * pc + 2], pk[4 * pc + 3]);
+                    fence_proxy_async_smem();
                     __syncwarp();
+                    if (lane == 0) {
+                        tma_store_2d(&map_o, wstg, hb * 64, orow0 + (warp & 3) * 32, pol);
+                        bulk_commit();
+                    }
                 }
                 tc_fence_before_sync();
                 __syncwarp();
@@ -461,12 +458,10 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
 
 int attend_tc_tile_tokens() { return kTok; }
 
-int launch_prefill_attend_tc(const Shape& s, const void* q, const void* maps_kv, const void* landmarks,
-                             const float* bias, const int* entries, const void* tiles, const int* n_tiles, void* obuf,
-                             float* lam, int* status, int i0, int qb, cudaStream_t stream) {
-    // maps_kv: the K and V tensor maps ([pairs*T, 128] bf16, box 64 x 64, 128B swizzle), encoded once per call
-    const CUtensorMap& map_k = static_cast<const CUtensorMap*>(maps_kv)[0];
-    const CUtensorMap& map_v = static_cast<const CUtensorMap*>(maps_kv)[1];
+int launch_prefill_attend_tc(const Shape& s, const void* q, const void* maps, const void* landmarks,
+                             const float* bias, const int* entries, const void* tiles, const int* n_tiles, float* lam,
+                             int* status, int i0, cudaStream_t stream) {
+    const CUtensorMap* m = static_cast<const CUtensorMap*>(maps);
     const size_t smem = 2 * kKBytes + 2 * kVBytes + kQSlots * kQBytes + 2 * kPBytes + sizeof(AtcSmem) + 1024;
     static bool attr_done = false;
     if (!attr_done) {
@@ -476,8 +471,8 @@ int launch_prefill_attend_tc(const Shape& s, const void* q, const void* maps_kv,
         attr_done = true;
     }
     AtcArgs a{s, static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(landmarks), bias, entries,
-              static_cast<const int4*>(tiles), n_tiles, static_cast<__nv_bfloat16*>(obuf), lam, status, i0, qb};
-    prefill_attend_tc_kernel<<<148, kThreads, smem, stream>>>(map_k, map_v, a);
+              static_cast<const int4*>(tiles), n_tiles, lam, status, i0};
+    prefill_attend_tc_kernel<<<148, kThreads, smem, stream>>>(m[0], m[1], m[2], a);
     if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
     return 1;
 }

@@ -117,6 +117,13 @@ template <int N> __device__ __forceinline__ void bulk_wait_read() {
     asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
 }
 
+// 2-D tiled TMA store of one box (shared memory laid out as the map's swizzle prescribes) with an L2 policy,
+// tracked by the issuing thread's bulk groups.  Same fencing rules as bulk_store.
+__device__ __forceinline__ void tma_store_2d(const void* map, const void* smem_src, int x, int y, uint64_t policy) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3}], [%1], %4;"
+                 ::"l"(map), "r"(smem_u32(smem_src)), "r"(x), "r"(y), "l"(policy) : "memory");
+}
+
 // Brings one box of a tiled tensor into L2 without touching shared memory.
 __device__ __forceinline__ void tma_prefetch_l2_2d(const void* map, int x, int y) {
     asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(map), "r"(x), "r"(y) : "memory");
