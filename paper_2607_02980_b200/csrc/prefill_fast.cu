@@ -43,6 +43,7 @@ struct PArgs {
     int* cnt;               // [n_blocks*pairs*nc] rows of each (block, pair, chunk): selectors + own tokens
     int* cursor;            // [pairs*C]
     int* blk_toff;          // [n_blocks + 1] first tile of every query block (tiles are grouped by block)
+    int* seg_tiles;         // [ceil(lists / 1024)] tiles of each segment of 1024 lists
     int* off;               // [n_blocks*pairs*nc] first entry of each list; every list starts on a tile boundary
     int* entries;           // [max_tiles * tile_tok] (token_local << 8) | slot, grouped by (block, pair, chunk);
                             // slot K marks the token's own chunk (local branch); list tails up to the next tile
@@ -266,45 +267,63 @@ __global__ void invert_count_kernel(const PArgs a) {
     }
 }
 
-// single CTA: exclusive prefix sum of the tiles per list, ceil(cnt / tile_tok); a list's first entry is its
-// first tile x tile_tok, so the tiles of a query block cover one contiguous, tile-aligned range of entries
+// Exclusive prefix sum of the tiles per list, ceil(cnt / tile_tok), in two launches of one CTA per 1024 lists:
+// segment sums first, then every CTA adds up the sums of the segments before its own and scans its segment.
+// A list's first entry is its first tile x tile_tok, so the tiles of a query block cover one contiguous,
+// tile-aligned range of entries.
+__global__ void __launch_bounds__(1024) invert_segsum_kernel(const PArgs a) {
+    __shared__ int wsum[32];
+    const int n = a.s.B * a.s.Hkv * a.nc * a.n_blocks;
+    const int x = blockIdx.x * 1024 + threadIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int ct = x < n ? (a.cnt[x] + a.tile_tok - 1) / a.tile_tok : 0;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) ct += __shfl_xor_sync(kFullMask, ct, o);
+    if (lane == 0) wsum[warp] = ct;
+    __syncthreads();
+    if (warp == 0) {
+        int v = wsum[lane];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFullMask, v, o);
+        if (lane == 0) a.seg_tiles[blockIdx.x] = v;
+    }
+}
+
 __global__ void __launch_bounds__(1024) invert_scan_kernel(const PArgs a) {
     __shared__ int wsum_t[32];
-    __shared__ int carry_t;
+    __shared__ int wpre[32];
     const Shape& s = a.s;
     const int per_blk = s.B * s.Hkv * a.nc;
     const int n = per_blk * a.n_blocks;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (tid == 0) carry_t = 0;
-    __syncthreads();
-    for (int base = 0; base < n; base += 1024) {
-        const int x = base + tid;
-        const int ce = x < n ? a.cnt[x] : 0;
-        const int ct = (ce + a.tile_tok - 1) / a.tile_tok;
-        int it = ct;
+    // tiles of all earlier segments
+    int pre = 0;
+    for (int sg = tid; sg < static_cast<int>(blockIdx.x); sg += 1024) pre += a.seg_tiles[sg];
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int nt = __shfl_up_sync(kFullMask, it, o);
-            if (lane >= o) it += nt;
-        }
-        if (lane == 31) wsum_t[warp] = it;
-        __syncthreads();
-        int bt = carry_t;
-        for (int w = 0; w < warp; ++w) bt += wsum_t[w];
-        const int ot = bt + it - ct, oe = ot * a.tile_tok;
-        if (x < n) {
-            a.off[x] = oe;
-            const int pair = (x % per_blk) / a.nc, c = x % a.nc;
-            if (x % per_blk == 0) a.blk_toff[x / per_blk] = ot;
-            for (int k = 0; k < ct; ++k)
-                if (ot + k < a.max_tiles)
-                    a.tiles[ot + k] = make_int4(pair, c, oe + k * a.tile_tok, min(a.tile_tok, ce - k * a.tile_tok));
-        }
-        __syncthreads();
-        if (tid == 1023) carry_t = ot + ct;
-        __syncthreads();
+    for (int o = 16; o > 0; o >>= 1) pre += __shfl_xor_sync(kFullMask, pre, o);
+    if (lane == 0) wpre[warp] = pre;
+    const int x = blockIdx.x * 1024 + tid;
+    const int ce = x < n ? a.cnt[x] : 0;
+    const int ct = (ce + a.tile_tok - 1) / a.tile_tok;
+    int it = ct;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int nt = __shfl_up_sync(kFullMask, it, o);
+        if (lane >= o) it += nt;
     }
-    if (tid == 0) a.blk_toff[a.n_blocks] = min(carry_t, a.max_tiles);
+    if (lane == 31) wsum_t[warp] = it;
+    __syncthreads();
+    int bt = 0;
+    for (int w = 0; w < 32; ++w) bt += wpre[w] + (w < warp ? wsum_t[w] : 0);
+    const int ot = bt + it - ct, oe = ot * a.tile_tok;
+    if (x < n) {
+        a.off[x] = oe;
+        const int pair = (x % per_blk) / a.nc, c = x % a.nc;
+        if (x % per_blk == 0) a.blk_toff[x / per_blk] = ot;
+        for (int k = 0; k < ct; ++k)
+            if (ot + k < a.max_tiles)
+                a.tiles[ot + k] = make_int4(pair, c, oe + k * a.tile_tok, min(a.tile_tok, ce - k * a.tile_tok));
+        if (x == n - 1) a.blk_toff[a.n_blocks] = min(ot + ct, a.max_tiles);
+    }
 }
 
 __global__ void invert_fill_kernel(const PArgs a) {
@@ -440,7 +459,7 @@ const int kQB = [] {
 }();
 struct Plan {
     int qb, nc, n_blocks, max_tiles, max_blk_tiles;
-    size_t off_cnt, off_cursor, off_ntiles, zero_bytes, off_off, off_entries, off_epos, off_tiles, off_obuf, off_lam,
+    size_t off_cnt, off_cursor, off_ntiles, zero_bytes, off_seg, off_off, off_entries, off_epos, off_tiles, off_obuf, off_lam,
         total;
 };
 
@@ -471,6 +490,7 @@ Plan make_plan(const Shape& s) {
     p.off_cursor = take(sizeof(int) * nblocks * pairs * nc);
     p.off_ntiles = take(sizeof(int) * (nblocks + 1));
     p.zero_bytes = off;                         // cnt, cursor, blk_toff are cleared together once per call
+    p.off_seg = take(sizeof(int) * ((nblocks * pairs * nc + 1023) / 1024));
     p.off_off = take(sizeof(int) * nblocks * pairs * nc);
     p.off_entries = take(sizeof(int) * all_tiles * tt);
     p.off_epos = take(sizeof(int) * pairs * s.R * (s.K + 1));
@@ -512,6 +532,7 @@ int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
     a.blk_toff = reinterpret_cast<int*>(sc + p.off_ntiles);
     a.n_blocks = p.n_blocks;
     a.blk = 0;
+    a.seg_tiles = reinterpret_cast<int*>(sc + p.off_seg);
     a.off = reinterpret_cast<int*>(sc + p.off_off);
     a.entries = reinterpret_cast<int*>(sc + p.off_entries);
     a.epos = reinterpret_cast<int*>(sc + p.off_epos);
@@ -563,11 +584,13 @@ int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
         const long long want = (elems + 255) / 256;
         const unsigned eb = static_cast<unsigned>(want < 148 * 16 ? want : 148 * 16);
         invert_count_kernel<<<eb, 256, 0, stream>>>(a);
-        invert_scan_kernel<<<1, 1024, 0, stream>>>(a);
+        const unsigned nseg = static_cast<unsigned>((static_cast<long long>(p.n_blocks) * pairs * p.nc + 1023) / 1024);
+        invert_segsum_kernel<<<nseg, 1024, 0, stream>>>(a);
+        invert_scan_kernel<<<nseg, 1024, 0, stream>>>(a);
         invert_fill_kernel<<<eb, 256, 0, stream>>>(a);
         if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
         trace_mark("prefill_invert", stream);
-        launches += 3;
+        launches += 4;
     }
     for (int i0 = 0, blk = 0; i0 < s.R; i0 += a.qb, ++blk) {
         a.i0 = i0;
