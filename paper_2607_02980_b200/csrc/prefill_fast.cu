@@ -4,16 +4,16 @@
 // path is organised CHUNK-MAJOR: K/V of a chunk are staged once and reused by every query row that
 // selected it; what moves per (token, chunk) pair is the query rows in and one bf16 output row out.
 //
-//   prefill_select  per (sequence, KV head, 64-token tile): streams landmark tiles through a TMA ring,
-//                   scores them with warp MMA for the 4 heads (Eq. surrogate top-k), takes the group
+//   prefill_select  warp-MMA scoring + top-K, the fallback for K > 32 (the tcgen05 kernel lives in
+//                   prefill_select_tc.cu): per (sequence, KV head, 64-token tile) it streams landmark tiles
+//                   through a TMA ring, scores them for the 4 heads (Eq. surrogate top-k), takes the group
 //                   max (App. C) and keeps an exact running top-K per token (ties: lower chunk id).
-//   invert_*        turns sel_idx of a token block into per-chunk lists of (token, slot) entries and a
-//                   table of 16-token tiles.
-//   prefill_attend  persistent CTAs over the tile table: Q rows gathered as MMA A fragments, the
-//                   chunk's own softmax (Eq. HiLS weights, intra-chunk factor), P V, one normalised
-//                   bf16 output row and the per-head surrogate score per (token, slot).
-//   prefill_fuse    per 64-token chunk: causal local attention (Eq. chunk mass) and the softmax over
-//                   {surrogate scores} U {log Z_swa} that mixes the rows written by prefill_attend.
+//   invert_*        turn sel_idx into per-(query block, pair, chunk) lists of (token, slot) entries, every list
+//                   starting on a tile boundary, the table of attend tiles, and the (token, slot) -> entry map.
+//   (prefill_attend_tc.cu: the tcgen05 attend kernel over that tile table; one normalised bf16 output row
+//                   and the per-head chunk mass per entry, in entry order.)
+//   prefill_fuse    per (token, KV head): the softmax over {surrogate scores} U {log Z_swa}
+//                   (Eq. HiLS weights) that mixes the rows written by the attend kernel.
 #include "internal.h"
 #include "tma.cuh"
 
@@ -352,7 +352,7 @@ __global__ void invert_fill_kernel(const PArgs a) {
 // prefill_attend wrote.  The rows are found through the entry index of every (token, slot); an entry's
 // 4 heads are 1 KB contiguous (two 16-byte loads per lane); lane l covers head l/16 (and head 2 + l/16),
 // elements 8*(l%16)..+7.
-constexpr int kFuseWarps = 8;
+constexpr int kFuseWarps = 4;
 
 __global__ void __launch_bounds__(kFuseWarps * 32) prefill_fuse_kernel(const PArgs a) {
     __shared__ float wsm[kFuseWarps][kG][68];
