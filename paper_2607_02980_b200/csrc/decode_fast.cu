@@ -3,7 +3,8 @@
 //   decode_score   streams the landmarks of every (sequence, KV head) once with 128-bit loads and
 //                  scores them against the G query heads with warp MMA (landmark rows are the A
 //                  operand straight from global memory); writes the group score u_c = max_h s^h_c.
-//   decode_select  one CTA per (sequence, KV head): exact top-K of u (ties to the lower chunk id),
+//   decode_select  one CTA per (sequence, KV head): exact top-K of u (ties to the lower chunk id) as a tree
+//                  of warp-level selections (linear-bin histogram + exact ranks in the boundary bin),
 //                  ascending ids, then the per-head surrogate scores of the selected chunks and the
 //                  fusion weights exp(s^h_c - max_c s^h_c).
 //   decode_attend  persistent CTAs over a flat list of (pair, slot) items; K/V chunks arrive through
@@ -20,9 +21,6 @@ constexpr int kD = 128;
 constexpr int kS = 64;
 constexpr int kScoreThreads = 256;
 constexpr int kScoreChunksPerCta = 256;      // 8 warps x 2 iterations x 16 chunks
-constexpr int kSelThreads = 512;
-constexpr int kSelBins = 2048;
-constexpr int kSelCap = 1024;                // candidates ranked exactly in shared memory
 constexpr int kStages = 5;
 constexpr int kStageBytes = 2 * kS * kD * 2; // K tile + V tile
 constexpr int kMaxItems = 2048;
@@ -58,258 +56,263 @@ struct DArgs {
 };
 
 // ------------------------------------------------------------------------------------------ select
-__device__ inline int block_excl_scan(int v, int* warp_tot, int& total) {
-    // exclusive prefix of v over the block in thread order; warp_tot: shared int[32]
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
-    int inc = v;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int n = __shfl_up_sync(kFullMask, inc, o);
-        if (lane >= o) inc += n;
+// Exact top-K as a tree of warp-level selections.  A warp stages up to kSelCap candidates (ordered score
+// key + chunk id) in its own shared-memory buffer, bins the scores linearly between the buffer's minimum
+// and maximum (128 warp-private counters), finds the bin that holds the K-th best, takes everything above
+// it and ranks the few candidates inside it exactly (score, then lower chunk id).  Level 1 runs one such
+// selection per warp over its slice of the pair's candidates; the survivor lists are then merged, kSelCap / K
+// lists per warp and round, until one list is left.  A member of the global top-K is in the top-K of every
+// subset that holds it, so the result is exact.  All loops are rolled on purpose: the code runs once per
+// CTA, so its size (instruction fetch), not its instruction count, sets the pace.
+constexpr int kSelMaxK = 128;
+constexpr int kSelCap = 1024 + kSelMaxK;     // staged candidates per warp: a slice round + carried survivors
+constexpr int kSelBins = 128;
+constexpr int kSelEdge = 64;                 // candidates of the boundary bin that are ranked pairwise
+
+struct SelWarp {                             // one per warp, in dynamic shared memory
+    unsigned key[kSelCap];                   // ordered score keys (>= 1)
+    int id[kSelCap];                         // chunk ids
+    unsigned long long list[kSelMaxK];       // survivors (key << 32 | id), unordered
+    unsigned long long edge[kSelEdge];       // boundary-bin candidates (key << 32 | ~id)
+    int hist[kSelBins];
+    int cnt;                                 // entries of list
+};
+
+// Selects the best min(K, n) of the n staged candidates of w into w.list / w.cnt.
+__device__ __noinline__ void warp_select(SelWarp& w, int n, int K, int lane) {
+    int nout = 0;
+    if (n <= K) {
+        for (int i = lane; i < n; i += 32) w.list[i] = (static_cast<unsigned long long>(w.key[i]) << 32) | static_cast<unsigned>(w.id[i]);
+        nout = n;
+    } else {
+        unsigned kmax = 0u, kmin = 0xffffffffu;
+#pragma unroll 4
+        for (int i = lane; i < n; i += 32) { kmax = max(kmax, w.key[i]); kmin = min(kmin, w.key[i]); }
+        kmax = __reduce_max_sync(kFullMask, kmax);
+        kmin = __reduce_min_sync(kFullMask, kmin);
+        // monotone linear binning of the scores between the extremes
+        const float lo = key_to_float(kmin), hi = key_to_float(kmax);
+        const float inv = hi > lo ? static_cast<float>(kSelBins - 1) / (hi - lo) : 0.f;
+        for (int x = lane; x < kSelBins; x += 32) w.hist[x] = 0;
+        __syncwarp();
+#pragma unroll 4
+        for (int i = lane; i < n; i += 32)
+            atomicAdd(&w.hist[max(0, min(kSelBins - 1, static_cast<int>((key_to_float(w.key[i]) - lo) * inv)))], 1);
+        __syncwarp();
+        // boundary bin b*: the highest bin with count(bin >= b*) >= K; lane l owns bins 127-4l .. 124-4l
+        int tsum = 0;
+        for (int x = 0; x < 4; ++x) tsum += w.hist[kSelBins - 1 - 4 * lane - x];
+        int inc = tsum;
+        for (int o = 1; o < 32; o <<= 1) {
+            const int nn = __shfl_up_sync(kFullMask, inc, o);
+            if (lane >= o) inc += nn;
+        }
+        int cum = inc - tsum, bstar = -1, above = 0;
+        if (cum < K && inc >= K) {
+            for (int x = 0; x < 4 && bstar < 0; ++x) {
+                const int h = w.hist[kSelBins - 1 - 4 * lane - x];
+                if (cum + h >= K) { bstar = kSelBins - 1 - 4 * lane - x; above = cum; }
+                cum += h;
+            }
+        }
+        const int src = __ffs(__ballot_sync(kFullMask, bstar >= 0)) - 1;      // exactly one lane found it
+        bstar = __shfl_sync(kFullMask, bstar, src);
+        above = __shfl_sync(kFullMask, above, src);
+        const int quota = K - above;          // >= 1 candidates of the boundary bin survive
+        const int m = w.hist[bstar];          // its population (>= quota)
+        const bool rank_edge = m != quota && m <= kSelEdge;
+        // everything above the boundary bin survives; the boundary bin goes to the edge list (or survives whole)
+        int nedge = 0;
+#pragma unroll 2
+        for (int i0 = 0; i0 < n; i0 += 32) {
+            const int i = i0 + lane;
+            int bin = -1;
+            unsigned k = 0u;
+            int c = 0;
+            if (i < n) {
+                k = w.key[i];
+                c = w.id[i];
+                bin = max(0, min(kSelBins - 1, static_cast<int>((key_to_float(k) - lo) * inv)));
+            }
+            const bool tk = bin > bstar || (bin == bstar && m == quota);
+            const unsigned bt = __ballot_sync(kFullMask, tk);
+            if (tk) w.list[nout + __popc(bt & ((1u << lane) - 1u))] = (static_cast<unsigned long long>(k) << 32) | static_cast<unsigned>(c);
+            nout += __popc(bt);
+            const bool ed = bin == bstar && rank_edge;
+            const unsigned be = __ballot_sync(kFullMask, ed);
+            if (ed) w.edge[nedge + __popc(be & ((1u << lane) - 1u))] = (static_cast<unsigned long long>(k) << 32) | (0xffffffffu - static_cast<unsigned>(c));
+            nedge += __popc(be);
+        }
+        __syncwarp();
+        if (rank_edge) {
+            // pairwise ranks inside the boundary bin (full keys: score, then lower id)
+            for (int e0 = 0; e0 < m; e0 += 32) {
+                const int e = e0 + lane;
+                const unsigned long long mine = e < m ? w.edge[e] : 0ull;
+                int rank = 0;
+                for (int j = 0; j < m; ++j) rank += w.edge[j] > mine ? 1 : 0;
+                const bool tk = e < m && rank < quota;
+                const unsigned bt = __ballot_sync(kFullMask, tk);
+                if (tk) w.list[nout + __popc(bt & ((1u << lane) - 1u))] = (mine & 0xffffffff00000000ull) | (0xffffffffu - static_cast<unsigned>(mine & 0xffffffffull));
+                nout += __popc(bt);
+            }
+        } else if (m != quota) {
+            // crowded boundary bin (clustered or equal scores): bisection on its members' keys, one bit at a time,
+            // then the lowest chunk ids among the keys on the cut
+            unsigned prefix = 0u;
+            for (int bit = 31; bit >= 0; --bit) {
+                const unsigned cand = prefix | (1u << bit);
+                int cnt = 0;
+                for (int i = lane; i < n; i += 32) {
+                    const unsigned k = w.key[i];
+                    const int bin = max(0, min(kSelBins - 1, static_cast<int>((key_to_float(k) - lo) * inv)));
+                    cnt += (bin == bstar && k >= cand) ? 1 : 0;
+                }
+                if (__reduce_add_sync(kFullMask, cnt) >= quota) prefix = cand;
+            }
+            int n_gt = 0;
+            for (int i = lane; i < n; i += 32) {
+                const unsigned k = w.key[i];
+                const int bin = max(0, min(kSelBins - 1, static_cast<int>((key_to_float(k) - lo) * inv)));
+                n_gt += (bin == bstar && k > prefix) ? 1 : 0;
+            }
+            n_gt = __reduce_add_sync(kFullMask, n_gt);
+            int q2 = quota - n_gt;            // members with key == prefix still to take, lowest ids first
+            int last_id = -1;
+            for (int i0 = 0; i0 < n; i0 += 32) {
+                const int i = i0 + lane;
+                unsigned k = 0u;
+                int bin = -1;
+                if (i < n) {
+                    k = w.key[i];
+                    bin = max(0, min(kSelBins - 1, static_cast<int>((key_to_float(k) - lo) * inv)));
+                }
+                const bool tk = bin == bstar && k > prefix;
+                const unsigned bt = __ballot_sync(kFullMask, tk);
+                if (tk) w.list[nout + __popc(bt & ((1u << lane) - 1u))] = (static_cast<unsigned long long>(k) << 32) | static_cast<unsigned>(w.id[i]);
+                nout += __popc(bt);
+            }
+            for (; q2 > 0; --q2) {
+                int best = 0x7fffffff;
+                for (int i = lane; i < n; i += 32) {
+                    const unsigned k = w.key[i];
+                    const int bin = max(0, min(kSelBins - 1, static_cast<int>((key_to_float(k) - lo) * inv)));
+                    if (bin == bstar && k == prefix && w.id[i] > last_id) best = min(best, w.id[i]);
+                }
+                best = static_cast<int>(__reduce_min_sync(kFullMask, static_cast<unsigned>(best)));
+                if (lane == 0) w.list[nout] = (static_cast<unsigned long long>(prefix) << 32) | static_cast<unsigned>(best);
+                ++nout;
+                last_id = best;
+            }
+        }
     }
-    __syncthreads();
-    if (lane == 31) warp_tot[warp] = inc;
-    __syncthreads();
-    int base = 0, tot = 0;
-    for (int w = 0; w < nw; ++w) {
-        const int x = warp_tot[w];
-        if (w < warp) base += x;
-        tot += x;
-    }
-    total = tot;
-    return base + inc - v;
+    __syncwarp();
+    if (lane == 0) w.cnt = nout;
 }
 
 struct SelShared {
-    int hist[kSelBins];
-    unsigned long long cand[kSelCap];
-    int sel_s[128];
-    float lam_s[8][128];
-    alignas(16) __nv_bfloat16 lm_s[64][kD + 8];    // selected landmark rows, 64 at a time (padded rows)
+    int sel_s[kSelMaxK];
+    float lam_s[8][kSelMaxK];
     alignas(16) __nv_bfloat16 q_s[8][kD + 8];
-    int warp_tot[32];
-    int sh_i[8];
-    int is_last;
 };
+constexpr size_t kSelLmBytes = 64 * (kD + 8) * 2;          // staged landmark rows alias the selection buffers
 
 // Exact top-K of the group scores of one (sequence, KV head) pair (ties: lower chunk id), ascending ids,
 // then the per-head surrogate scores of the selected chunks and the fusion weights.  Called by every
-// thread of the CTA that finished the pair's scoring last; u was written by other CTAs (L2 reads).
-__device__ void select_pair(const DArgs& a, int pair, int ncand, SelShared& sh) {
+// thread of the pair's CTA (nw warps); dyn: nw SelWarp buffers.
+__device__ void select_pair(const DArgs& a, int pair, int ncand, SelShared& sh, uint8_t* dyn, int nw) {
     const Shape& s = a.s;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, NT = blockDim.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int NT = nw * 32;
     const int b = pair / s.Hkv, g = pair % s.Hkv;
     const int K = s.K, G = s.G;
     int32_t* sel = a.sel + static_cast<long long>(pair) * K;
     const int n = min(K, ncand);
     const float* u = a.u + static_cast<long long>(pair) * a.Cpad;
-    int* hist = sh.hist;
     int* sel_s = sh.sel_s;
-    int* sh_i = sh.sh_i;
+    SelWarp* sw = reinterpret_cast<SelWarp*>(dyn);
 
     if (ncand <= K) {
         for (int t = tid; t < K; t += NT) sel_s[t] = t < ncand ? t : -1;
         __syncthreads();
-    } else if (ncand <= 8 * NT) {
-        // --- short candidate lists: every thread keeps 8 consecutive ordered keys in registers and the
-        //     K-th best is found with a 4 x 8-bit radix select (shared-memory histograms only)
-        unsigned key[8];
-        const int cb = tid * 8;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) key[i] = cb + i < ncand ? ordered_key(__ldcg(u + cb + i)) : 0u;
-        unsigned prefix = 0u;
-        int remaining = K, n_eq = 0;
-#pragma unroll 1
-        for (int shift = 24; shift >= 0; shift -= 8) {
-            if (tid < 256) hist[tid] = 0;
-            __syncthreads();
-            const unsigned himask = shift == 24 ? 0u : (0xffffffffu << (shift + 8));
-#pragma unroll
-            for (int i = 0; i < 8; ++i)
-                if (cb + i < ncand && (key[i] & himask) == (prefix & himask)) atomicAdd(&hist[(key[i] >> shift) & 255u], 1);
-            __syncthreads();
-            if (warp == 0) {
-                // lane l owns digits 255-8l .. 248-8l (top-down)
-                int loc[8], tsum = 0;
-#pragma unroll
-                for (int x = 0; x < 8; ++x) { loc[x] = hist[255 - 8 * lane - x]; tsum += loc[x]; }
-                int inc = tsum;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const int nn = __shfl_up_sync(kFullMask, inc, o);
-                    if (lane >= o) inc += nn;
-                }
-                int cum = inc - tsum;
-                if (cum < remaining && inc >= remaining) {
-#pragma unroll
-                    for (int x = 0; x < 8; ++x) {
-                        if (cum + loc[x] >= remaining) { sh_i[4] = 255 - 8 * lane - x; sh_i[5] = cum; sh_i[6] = loc[x]; break; }
-                        cum += loc[x];
-                    }
-                }
-            }
-            __syncthreads();
-            prefix |= static_cast<unsigned>(sh_i[4]) << shift;
-            remaining -= sh_i[5];
-            n_eq = sh_i[6];
-        }
-        // prefix = key of the K-th best; `remaining` of the n_eq chunks with that key are taken, lowest ids first
-        int eq_before = 0, tot;
-        if (n_eq != remaining) {                        // ties across the cut (block-uniform branch)
-            int eq = 0;
-#pragma unroll
-            for (int i = 0; i < 8; ++i) eq += (cb + i < ncand && key[i] == prefix) ? 1 : 0;
-            eq_before = block_excl_scan(eq, sh.warp_tot, tot);
-        }
-        int cnt = 0, e = eq_before;
-        unsigned take = 0u;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            if (cb + i >= ncand) continue;
-            bool tk = key[i] > prefix;
-            if (key[i] == prefix) { tk = n_eq == remaining || e < remaining; ++e; }
-            if (tk) { take |= 1u << i; ++cnt; }
-        }
-        int pos = block_excl_scan(cnt, sh.warp_tot, tot);
-#pragma unroll
-        for (int i = 0; i < 8; ++i)
-            if (take & (1u << i)) sel_s[pos++] = cb + i;
-        __syncthreads();
     } else {
-        // --- 1. value range
-        float mn = INFINITY, mx = -INFINITY;
-        for (int c = tid; c < ncand; c += NT) { const float v = __ldcg(u + c) + 0.f; mn = fminf(mn, v); mx = fmaxf(mx, v); }
-        mn = -warp_max(-mn); mx = warp_max(mx);
-        if (lane == 0) { sh.lam_s[0][warp] = mn; sh.lam_s[1][warp] = mx; }
-        for (int i = tid; i < kSelBins; i += NT) hist[i] = 0;
-        if (tid == 0) sh_i[3] = 0;
-        __syncthreads();
-        float lo = sh.lam_s[0][0], hi = sh.lam_s[1][0];
-        for (int w = 1; w < NT / 32; ++w) { lo = fminf(lo, sh.lam_s[0][w]); hi = fmaxf(hi, sh.lam_s[1][w]); }
-        const float inv = (hi > lo) ? static_cast<float>(kSelBins - 1) / (hi - lo) : 0.f;
-        __syncthreads();
-        // --- 2. histogram over a monotone linear binning
-        for (int c = tid; c < ncand; c += NT) {
-            const int bin = max(0, min(kSelBins - 1, static_cast<int>((__ldcg(u + c) + 0.f - lo) * inv)));
-            atomicAdd(&hist[bin], 1);
-        }
-        __syncthreads();
-        // --- 3. boundary bin: the highest bin b* with count(bin >= b*) >= K.  Thread i owns the
-        //        kSelBins / NT bins below (kSelBins - 1 - i * per); a block scan gives the count above.
+        // --- level 1: warp w owns the candidates [w * per, (w + 1) * per) and walks them in rounds of
+        //     kSelCap - K, carrying its survivors from round to round
         {
-            const int per = kSelBins / NT;
-            const int top = kSelBins - 1 - tid * per;
-            int tsum = 0;
-            for (int x = 0; x < per; ++x) tsum += hist[top - x];
-            int tot;
-            int cum = block_excl_scan(tsum, sh.warp_tot, tot);
-            if (cum < K && cum + tsum >= K) {
-                for (int x = 0; x < per; ++x) {
-                    const int hb = hist[top - x];
-                    if (cum + hb >= K) { sh_i[0] = top - x; sh_i[1] = cum + hb; sh_i[2] = cum; break; }
-                    cum += hb;
+            SelWarp& w = sw[warp];
+            const int per = ((ncand + nw - 1) / nw + 31) & ~31;
+            const int cb = min(ncand, warp * per), ce = min(ncand, cb + per);
+            int nl = 0;
+            for (int r0 = cb; r0 < ce || r0 == cb; r0 += kSelCap - kSelMaxK) {
+                const int nr = max(0, min(ce - r0, kSelCap - kSelMaxK));
+                for (int i = lane; i < nl; i += 32) {
+                    const unsigned long long v = w.list[i];
+                    w.key[nr + i] = static_cast<unsigned>(v >> 32);
+                    w.id[nr + i] = static_cast<int>(v & 0xffffffffull);
                 }
+                // sixteen loads in flight per lane (the scores come from L2)
+                for (int i0 = 0; i0 < nr; i0 += 512) {
+                    float v[16];
+#pragma unroll
+                    for (int x = 0; x < 16; ++x) {
+                        const int i = i0 + x * 32 + lane;
+                        v[x] = i < nr ? __ldcg(u + r0 + i) : 0.f;
+                    }
+#pragma unroll
+                    for (int x = 0; x < 16; ++x) {
+                        const int i = i0 + x * 32 + lane;
+                        if (i < nr) { w.key[i] = max(1u, ordered_key(v[x])); w.id[i] = r0 + i; }
+                    }
+                }
+                __syncwarp();
+                warp_select(w, nr + nl, K, lane);
+                __syncwarp();
+                nl = w.cnt;
             }
         }
         __syncthreads();
-        const int bstar = sh_i[0], m_cand = sh_i[1];
-        if (m_cand <= kSelCap) {
-            // --- 4a. gather the candidates and rank them exactly (score desc, id asc)
-            unsigned long long* cand = sh.cand;
-            for (int c = tid; c < ncand; c += NT) {
-                const float v = __ldcg(u + c);
-                const int bin = max(0, min(kSelBins - 1, static_cast<int>((v + 0.f - lo) * inv)));
-                if (bin >= bstar) cand[atomicAdd(&sh_i[3], 1)] = select_key(v, c);
-            }
-            __syncthreads();
-            unsigned long long mine[kSelCap / kSelThreads];
-            bool keep[kSelCap / kSelThreads];
-#pragma unroll
-            for (int r = 0; r < kSelCap / kSelThreads; ++r) {
-                const int i = tid + r * NT;
-                mine[r] = i < m_cand ? cand[i] : 0ull;
-                int rank = 0;
-                if (i < m_cand)
-                    for (int j = 0; j < m_cand; ++j) rank += cand[j] > mine[r] ? 1 : 0;
-                keep[r] = i < m_cand && rank < K;                  // ranks are unique
-            }
-            __syncthreads();
-#pragma unroll
-            for (int r = 0; r < kSelCap / kSelThreads; ++r) {
-                const int i = tid + r * NT;
-                if (i < m_cand && !keep[r]) cand[i] = 0ull;
-            }
-            __syncthreads();
-            // ascending ids: position = number of selected ids below mine
-#pragma unroll
-            for (int r = 0; r < kSelCap / kSelThreads; ++r) {
-                if (!keep[r]) continue;
-                const int id = key_chunk(mine[r]);
-                int pos = 0;
-                for (int j = 0; j < m_cand; ++j) {
-                    const unsigned long long o = cand[j];
-                    pos += (o != 0ull && key_chunk(o) < id) ? 1 : 0;
-                }
-                sel_s[pos] = id;
-            }
-            __syncthreads();
-        } else {
-            // --- 4b. many equal / clustered scores: exact 4 x 8-bit radix select on the ordered key,
-            //         then an ordered scan (each thread owns a contiguous range of chunk ids)
-            unsigned prefix = 0u;
-            int remaining = K;
-            for (int shift = 24; shift >= 0; shift -= 8) {
-                for (int i = tid; i < 256; i += NT) hist[i] = 0;
-                __syncthreads();
-                const unsigned himask = shift == 24 ? 0u : (0xffffffffu << (shift + 8));
-                for (int c = tid; c < ncand; c += NT) {
-                    const unsigned key = ordered_key(__ldcg(u + c));
-                    if ((key & himask) == (prefix & himask)) atomicAdd(&hist[(key >> shift) & 255u], 1);
-                }
-                __syncthreads();
-                if (tid == 0) {
-                    int cum = 0, dsel = 0;
-                    for (int dgt = 255; dgt >= 0; --dgt) {
-                        if (cum + hist[dgt] >= remaining) { dsel = dgt; break; }
-                        cum += hist[dgt];
+        // --- merge rounds: warp g gathers the lists [g * fan, (g + 1) * fan) into its staging buffer (fan x K <= kSelCap).
+        //     A round reads lists that the previous round finished; it writes only the staging arrays and, after a
+        //     barrier, its own list.
+        int lists = nw;
+        const int fan = min(4, kSelCap / K);               // few lists per warp: short rounds on many warps
+        while (lists > 1) {
+            const int groups = (lists + fan - 1) / fan;
+            int tot = 0;
+            if (warp < groups) {
+                SelWarp& w = sw[warp];
+                for (int li = warp * fan; li < min(lists, (warp + 1) * fan); ++li) {
+                    const SelWarp& src = sw[li];
+                    const int cn = src.cnt;
+                    for (int i = lane; i < cn; i += 32) {
+                        const unsigned long long v = src.list[i];
+                        w.key[tot + i] = static_cast<unsigned>(v >> 32);
+                        w.id[tot + i] = static_cast<int>(v & 0xffffffffull);
                     }
-                    sh_i[4] = dsel; sh_i[5] = cum;
+                    tot += cn;
                 }
-                __syncthreads();
-                prefix |= static_cast<unsigned>(sh_i[4]) << shift;
-                remaining -= sh_i[5];
-                __syncthreads();
             }
-            // prefix = key of the K-th best; `remaining` of the chunks with that key are taken, lowest ids first
-            const int per = (ncand + NT - 1) / NT;
-            const int cb = min(ncand, tid * per), ce = min(ncand, cb + per);
-            int eq = 0;
-            for (int c = cb; c < ce; ++c) eq += ordered_key(__ldcg(u + c)) == prefix ? 1 : 0;
-            int tot;
-            int eq_before = block_excl_scan(eq, sh.warp_tot, tot);
-            int cnt = 0;
-            int e = eq_before;
-            for (int c = cb; c < ce; ++c) {
-                const unsigned key = ordered_key(__ldcg(u + c));
-                if (key > prefix) ++cnt;
-                else if (key == prefix) { if (e < remaining) ++cnt; ++e; }
-            }
-            int pos = block_excl_scan(cnt, sh.warp_tot, tot);
-            e = eq_before;
-            for (int c = cb; c < ce; ++c) {
-                const unsigned key = ordered_key(__ldcg(u + c));
-                bool take = key > prefix;
-                if (key == prefix) { take = e < remaining; ++e; }
-                if (take) sel_s[pos++] = c;
-            }
+            __syncthreads();                               // every list of this round has been read
+            if (warp < groups) warp_select(sw[warp], tot, K, lane);
             __syncthreads();
+            lists = groups;
         }
+        // --- ascending chunk ids: position = number of selected ids below mine
+        const unsigned long long* fin = sw[0].list;
+        for (int t = tid; t < n; t += NT) {
+            const int idt = static_cast<int>(fin[t] & 0xffffffffull);
+            int pos = 0;
+            for (int j = 0; j < n; ++j) pos += static_cast<int>(fin[j] & 0xffffffffull) < idt ? 1 : 0;
+            sel_s[pos] = idt;
+        }
+        __syncthreads();
     }
     for (int t = tid; t < K; t += NT) sel[t] = t < n ? sel_s[t] : -1;
 
-    // --- 5. per-head surrogate scores of the selected chunks and the fusion weights: the selected
-    //        landmark rows and the G queries are staged in shared memory with one round of 16-byte
-    //        loads, then every thread computes one (chunk, head) dot product
+    // --- per-head surrogate scores of the selected chunks and the fusion weights: the selected
+    //     landmark rows and the G queries are staged in shared memory with one round of 16-byte
+    //     loads, then every thread computes (chunk, head) dot products
+    __nv_bfloat16 (*lm_s)[kD + 8] = reinterpret_cast<__nv_bfloat16 (*)[kD + 8]>(dyn);
     const __nv_bfloat16* lm = a.lm + static_cast<long long>(pair) * s.C * kD;
     const __nv_bfloat16* qg = a.q + (static_cast<long long>(b) * s.Hq + g * G) * kD;
     for (int x = tid; x < G * 16; x += NT)
@@ -317,15 +320,23 @@ __device__ void select_pair(const DArgs& a, int pair, int ncand, SelShared& sh) 
     for (int t0 = 0; t0 < n; t0 += 64) {
         const int nt = min(64, n - t0);
         __syncthreads();
-        for (int x = tid; x < nt * 16; x += NT) {
-            const int t = x >> 4, pc = x & 15;
-            *reinterpret_cast<uint4*>(&sh.lm_s[t][pc * 8]) =
-                *reinterpret_cast<const uint4*>(lm + static_cast<long long>(sel_s[t0 + t]) * kD + pc * 8);
+        for (int x0 = 0; x0 < nt * 16; x0 += 4 * NT) {       // four 16-byte loads in flight per thread
+            uint4 v[4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                const int x = x0 + r * NT + tid;
+                if (x < nt * 16) v[r] = *reinterpret_cast<const uint4*>(lm + static_cast<long long>(sel_s[t0 + (x >> 4)]) * kD + (x & 15) * 8);
+            }
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                const int x = x0 + r * NT + tid;
+                if (x < nt * 16) *reinterpret_cast<uint4*>(&lm_s[x >> 4][(x & 15) * 8]) = v[r];
+            }
         }
         __syncthreads();
         for (int x = tid; x < nt * G; x += NT) {
             const int t = x / G, h = x % G;
-            const __nv_bfloat16* lr = sh.lm_s[t];
+            const __nv_bfloat16* lr = lm_s[t];
             const __nv_bfloat16* qr = sh.q_s[h];
             float acc = 0.f;
 #pragma unroll 8
@@ -340,8 +351,7 @@ __device__ void select_pair(const DArgs& a, int pair, int ncand, SelShared& sh) 
         }
     }
     __syncthreads();
-    if (warp < G) {
-        const int h = warp;
+    for (int h = warp; h < G; h += nw) {
         float mx = -INFINITY;
         for (int t = lane; t < n; t += 32) mx = fmaxf(mx, sh.lam_s[h][t]);
         mx = warp_max(mx);
@@ -425,24 +435,26 @@ __global__ void __launch_bounds__(kScoreThreads) decode_score_kernel(const DArgs
     pdl_launch_dependents();
 }
 
-// One CTA per (sequence, KV head) pair.
-__global__ void __launch_bounds__(kSelThreads) decode_select_kernel(const DArgs a) {
+// One CTA per (sequence, KV head) pair: 4 warps for candidate lists of up to 4096 chunks, else 16.
+// Dynamic shared memory: one SelWarp per warp.
+__global__ void __launch_bounds__(512) decode_select_kernel(const DArgs a) {
     __shared__ SelShared sh;
+    extern __shared__ __align__(16) uint8_t sel_dyn[];
     const Shape& s = a.s;
-    const int pair = blockIdx.x, tid = threadIdx.x;
+    const int pair = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
     const int b = pair / s.Hkv, g = pair % s.Hkv;
     const int seq = a.seq_lens[b];
     if (seq < 1 || seq > s.T) {
         // invalid length: flag it, emit empty outputs
         if (tid == 0) { set_status(a.status, kDevBadIndex); a.pair_n[pair] = -1; a.done[pair] = 0; }
-        for (int t = tid; t < s.K; t += kSelThreads) a.sel[static_cast<long long>(pair) * s.K + t] = -1;
-        for (int x = tid; x < s.G * kD; x += kSelThreads)
+        for (int t = tid; t < s.K; t += nt) a.sel[static_cast<long long>(pair) * s.K + t] = -1;
+        for (int x = tid; x < s.G * kD; x += nt)
             a.out[(static_cast<long long>(b) * s.Hq + g * s.G) * kD + x] = __float2bfloat16_rn(0.f);
         if (tid < s.G) a.lse[static_cast<long long>(b) * s.Hq + g * s.G + tid] = 0.f;
         return;
     }
     pdl_wait();                                        // group scores of decode_score are visible
-    select_pair(a, pair, (seq - 1) / kS, sh);
+    select_pair(a, pair, (seq - 1) / kS, sh, sel_dyn, nt >> 5);
     pdl_launch_dependents();
 }
 
@@ -834,7 +846,9 @@ int launch_decode_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
     static bool attr_done = false;
     if (!attr_done) {
         if (cudaFuncSetAttribute(decode_attend_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(attend_smem)) != cudaSuccess)
+                                 static_cast<int>(attend_smem)) != cudaSuccess ||
+            cudaFuncSetAttribute(decode_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(sizeof(SelWarp) * 16)) != cudaSuccess)
             return HILS_ERR_CUDA;
         attr_done = true;
     }
@@ -852,9 +866,14 @@ int launch_decode_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     cfg.gridDim = dim3(pairs);
-    cfg.blockDim = dim3(kSelThreads);
     cfg.dynamicSmemBytes = 0;
-    if (cudaLaunchKernelEx(&cfg, decode_select_kernel, a) != cudaSuccess) return HILS_ERR_CUDA;
+    {
+        const int nw = (s.T - 1) / kS <= 4096 ? 4 : 16;
+        const size_t need = sizeof(SelWarp) * nw > kSelLmBytes ? sizeof(SelWarp) * nw : kSelLmBytes;
+        cfg.blockDim = dim3(nw * 32);
+        cfg.dynamicSmemBytes = need;
+        if (cudaLaunchKernelEx(&cfg, decode_select_kernel, a) != cudaSuccess) return HILS_ERR_CUDA;
+    }
     trace_mark("decode_select", stream);
 
     cfg.gridDim = dim3(p.n_ctas);
