@@ -143,6 +143,40 @@ def test_decode_with_bias(impl):
     check_decode(cfg, inp, out, lse, sel, bias=bias)
 
 
+@pytest.mark.parametrize("L", [8192, 64 * 3000, 64 * 5000])      # 127 / 2999 / 4999 candidate chunks
+def test_decode_ties_and_clustered_scores_pick_the_lower_chunk_ids(L):
+    """Equal and two-valued group scores: the exact tie rule decides the whole selection (Eq. surrogate
+    top-k with ties to the lower chunk id); both kernel sets must return exactly the expected ids."""
+    cfg = wl.CONFIGS[3].scaled(B=1, Hq=8, Hkv=2, L=L, K=24, seed=47, n_needles=0)
+    inp = wl.make_decode_inputs(cfg, "cpu", seq_lens=torch.tensor([L], dtype=torch.int32))
+    ncand = (L - 1) // cfg.S
+    # (a) all scores equal
+    inp_a = dict(inp)
+    inp_a["q"] = torch.zeros_like(inp["q"])
+    # (b) two score levels: chunks with c % 5 == 2 score 16, the rest 0
+    lm = torch.zeros_like(inp["landmarks"])
+    lm[:, :, 2::5, 0] = 4.0
+    q = torch.zeros_like(inp["q"])
+    q[..., 0] = 4.0
+    inp_b = dict(inp, landmarks=lm, q=q)
+    hi = [c for c in range(ncand) if c % 5 == 2]
+    lo = [c for c in range(ncand) if c % 5 != 2]
+    exp_b = sorted(hi[:cfg.K] + lo[:max(0, cfg.K - len(hi))])
+    # (c) as (b) but only 10 chunks on the upper level: the cut runs through the crowded lower level
+    lm_c = torch.zeros_like(inp["landmarks"])
+    top10 = [7 + 11 * j for j in range(10)]
+    lm_c[:, :, top10, 0] = 4.0
+    inp_c = dict(inp, landmarks=lm_c, q=q)
+    rest = [c for c in range(ncand) if c not in top10]
+    exp_c = sorted(top10 + rest[:cfg.K - 10])
+    for impl in ("generic", "fast"):
+        for case, expect in ((inp_a, list(range(cfg.K))), (inp_b, exp_b), (inp_c, exp_c)):
+            _, _, sel = run_decode(cfg, case, impl)
+            got = sel.cpu().numpy()
+            for g in range(cfg.Hkv):
+                assert got[0, g].tolist() == expect, (impl, L, g)
+
+
 def test_decode_invalid_seq_len_sets_status_without_fault():
     cfg = wl.CONFIGS[3].scaled(B=2, L=1024, K=4, seed=46)
     inp = wl.make_decode_inputs(cfg, "cpu", seq_lens=torch.tensor([1024, 512], dtype=torch.int32))
