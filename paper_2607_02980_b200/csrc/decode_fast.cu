@@ -21,10 +21,10 @@ constexpr int kD = 128;
 constexpr int kS = 64;
 constexpr int kScoreThreads = 256;
 constexpr int kScoreChunksPerCta = 256;      // 8 warps x 2 iterations x 16 chunks
-constexpr int kStages = 5;
+constexpr int kStages = 6;
 constexpr int kStageBytes = 2 * kS * kD * 2; // K tile + V tile
-constexpr int kMaxItems = 2048;
-constexpr int kConsumerWarps = 5;       // == kStages: a stage is always consumed by the same warp, so no
+constexpr int kMaxItems = 1024;
+constexpr int kConsumerWarps = 6;       // == kStages: a stage is always consumed by the same warp, so no
                                         // waiter can ever be more than one mbarrier phase away from its stage
 static_assert(kStages % kConsumerWarps == 0, "stage ownership must be fixed per consumer warp");
 constexpr int kAttendThreads = (kConsumerWarps + 1) * 32;
@@ -708,7 +708,12 @@ decode_attend_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
         if (n_sel >= 0 && part_idx < a.max_parts) {
             float* dst = a.part + (static_cast<long long>(pair) * a.max_parts + part_idx) * G * kD;
             for (int x = tid; x < G * kD; x += kConsumerWarps * 32)
-                dst[x] = ((sm.red[0][x] + sm.red[1][x]) + (sm.red[2][x] + sm.red[3][x])) + sm.red[4][x];
+                {
+                float acc = 0.f;
+#pragma unroll
+                for (int w = 0; w < kConsumerWarps; ++w) acc += sm.red[w][x];      // fixed order: deterministic
+                dst[x] = acc;
+            }
         }
         __threadfence();
         asm volatile("bar.sync 1, %0;" ::"r"(kConsumerWarps * 32));
