@@ -38,8 +38,7 @@ constexpr int kMmaWarp = kProdWarp0 + kProdThreads / 32;
 constexpr float kLog2e = 1.4426950408889634f;
 
 struct AtcSmem {
-    uint64_t kraw_full;       // TMA of the K and V rows landed
-    uint64_t kv_ready[2];     // K tile (with landmark row) and V usable by the MMA
+    uint64_t kv_ready[2];     // K tile and V landed (TMA bytes) and the landmark row written (one arrival): usable by the MMA
     uint64_t kv_empty[2];     // every MMA that reads this K/V buffer has completed
     uint64_t q_full[kQSlots]; // gathered Q rows landed and fenced (one arrival per producer warp)
     uint64_t q_empty[kQSlots];// the S MMA that reads this Q tile has completed
@@ -104,10 +103,9 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
     const long long hi = t_begin + static_cast<long long>(blockIdx.x + 1) * n_tiles / gridDim.x;
 
     if (tid == 0) {
-        mbar_init(&sm.kraw_full, 1);
         for (int i = 0; i < kQSlots; ++i) { mbar_init(&sm.q_full[i], 4); mbar_init(&sm.q_empty[i], 1); }
         for (int i = 0; i < 2; ++i) {
-            mbar_init(&sm.kv_ready[i], 1);
+            mbar_init(&sm.kv_ready[i], 2);          // the TMA issuer's arrive.expect_tx + the landmark writer
             mbar_init(&sm.kv_empty[i], 1);
             mbar_init(&sm.s_full[i], 1);
             mbar_init(&sm.s_empty[i], 4);
@@ -173,33 +171,39 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                 e_next = e_next2;
                 if (ti + 2 < nb) e_next2 = a.entries[sm.recs[ti + 2].z + min(ptid >> 2, sm.recs[ti + 2].w - 1)];
                 if (pair != cur_pair || c != cur_c) {
-                    // ---- new chunk: make its K/V usable
+                    // ---- new chunk: its K/V go to buffer cc & 1.  Nobody here waits for the copies: they complete on
+                    //      kv_ready, which only the MMA warp waits for, so the Q gathers below overlap them.
                     const uint32_t cbuf = cc & 1u;
-                    if (ptid == 0 && !next_issued) {
-                        if (cc >= 2 && !mbar_wait(&sm.kv_empty[cbuf], ((cc >> 1) - 1) & 1)) dead = true;
+                    if (pw == 0) {
+                        if (lane == 0 && !next_issued) {
+                            if (cc >= 2 && !mbar_wait(&sm.kv_empty[cbuf], ((cc >> 1) - 1) & 1)) dead = true;
+                            if (!dead) {
+                                const int row = pair * s.T + c * kS;
+                                mbar_expect_tx(&sm.kv_ready[cbuf], 2 * 8192 + kVBytes);
+                                tma_load_2d(kbuf + cbuf * kKBytes, &map_k, &sm.kv_ready[cbuf], 0, row);
+                                tma_load_2d(kbuf + cbuf * kKBytes + kNS * 128, &map_k, &sm.kv_ready[cbuf], 64, row);
+                                tma_load_2d(vbuf + cbuf * kVBytes, &map_v, &sm.kv_ready[cbuf], 0, row);
+                                tma_load_2d(vbuf + cbuf * kVBytes + 8192, &map_v, &sm.kv_ready[cbuf], 64, row);
+                            }
+                        }
+                        next_issued = false;
+                        dead = __shfl_sync(kFullMask, dead ? 1 : 0, 0) != 0;
                         if (!dead) {
-                            const int row = pair * s.T + c * kS;
-                            mbar_expect_tx(&sm.kraw_full, 2 * 8192 + kVBytes);
-                            tma_load_2d(kbuf + cbuf * kKBytes, &map_k, &sm.kraw_full, 0, row);
-                            tma_load_2d(kbuf + cbuf * kKBytes + kNS * 128, &map_k, &sm.kraw_full, 64, row);
-                            tma_load_2d(vbuf + cbuf * kVBytes, &map_v, &sm.kraw_full, 0, row);
-                            tma_load_2d(vbuf + cbuf * kVBytes + 8192, &map_v, &sm.kraw_full, 64, row);
+                            // landmark row (key 64) of both K-blocks: the buffer is free (its previous user's MMAs are
+                            // done) and TMA never writes this row.  V stays as TMA writes it (keys x dims): the second
+                            // MMA reads it as an MN-major operand; keys past the end of the sequence hold other rows'
+                            // data (or TMA zero fill) and meet probabilities of 0.
+                            if (lane < 16) {
+                                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                                if (c < s.C) v = *reinterpret_cast<const uint4*>(a.lm + (static_cast<long long>(pair) * s.C + c) * kD + lane * 8);
+                                *reinterpret_cast<uint4*>(kbuf + cbuf * kKBytes + (lane >> 3) * (kNS * 128) + swz128(64, lane & 7)) = v;
+                            }
+                            fence_proxy_async_smem();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(&sm.kv_ready[cbuf]);
                         }
                     }
-                    next_issued = false;
-                    if (!dead && !mbar_wait(&sm.kraw_full, cc & 1)) dead = true;
-                    if (dead) break;
-                    // landmark row (key 64) of both K-blocks
-                    if (ptid < 16) {
-                        uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                        if (c < s.C) v = *reinterpret_cast<const uint4*>(a.lm + (static_cast<long long>(pair) * s.C + c) * kD + ptid * 8);
-                        *reinterpret_cast<uint4*>(kbuf + cbuf * kKBytes + (ptid >> 3) * (kNS * 128) + swz128(64, ptid & 7)) = v;
-                    }
-                    // V stays as TMA wrote it (keys x dims): the second MMA reads it as an MN-major operand.  Keys past
-                    // the end of the sequence hold other rows' data (or TMA zero fill) and meet probabilities of 0.
-                    fence_proxy_async_smem();
-                    producer_barrier();
-                    if (ptid == 0) mbar_arrive(&sm.kv_ready[cbuf]);
+                    if (dead || *reinterpret_cast<volatile int*>(&sm.abort_flag)) { dead = true; break; }
                     cur_pair = pair;
                     cur_c = c;
                     ++cc;
@@ -220,11 +224,11 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                     const uint32_t nbuf = cc & 1u;
                     if (tj < nb && (cc < 2 || mbar_try_wait(&sm.kv_empty[nbuf], ((cc >> 1) - 1) & 1))) {
                         const int row = sm.recs[tj].x * s.T + sm.recs[tj].y * kS;
-                        mbar_expect_tx(&sm.kraw_full, 2 * 8192 + kVBytes);
-                        tma_load_2d(kbuf + nbuf * kKBytes, &map_k, &sm.kraw_full, 0, row);
-                        tma_load_2d(kbuf + nbuf * kKBytes + kNS * 128, &map_k, &sm.kraw_full, 64, row);
-                        tma_load_2d(vbuf + nbuf * kVBytes, &map_v, &sm.kraw_full, 0, row);
-                        tma_load_2d(vbuf + nbuf * kVBytes + 8192, &map_v, &sm.kraw_full, 64, row);
+                        mbar_expect_tx(&sm.kv_ready[nbuf], 2 * 8192 + kVBytes);
+                        tma_load_2d(kbuf + nbuf * kKBytes, &map_k, &sm.kv_ready[nbuf], 0, row);
+                        tma_load_2d(kbuf + nbuf * kKBytes + kNS * 128, &map_k, &sm.kv_ready[nbuf], 64, row);
+                        tma_load_2d(vbuf + nbuf * kVBytes, &map_v, &sm.kv_ready[nbuf], 0, row);
+                        tma_load_2d(vbuf + nbuf * kVBytes + 8192, &map_v, &sm.kv_ready[nbuf], 64, row);
                         next_issued = true;
                     }
                 }
@@ -269,7 +273,11 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                 if (lane == 0) mbar_arrive(&sm.q_full[(tc - 1) % kQSlots]);
             }
             if (dead && lane == 0) { set_status(a.status, kDevTimeout); atomicExch(&sm.abort_flag, 1); }
-            if (ptid == 0 && next_issued) mbar_wait(&sm.kraw_full, cc & 1);       // own copy in flight: let it land
+            if (ptid == 0 && next_issued) {
+                // (only after a timeout) a requested chunk was never taken up: complete its barrier, let the copy land
+                mbar_arrive(&sm.kv_ready[cc & 1u]);
+                mbar_wait(&sm.kv_ready[cc & 1u], (cc >> 1) & 1);
+            }
         } else if (warp == kMmaWarp) {
             // ================================================================ MMA issuer
             if (lane == 0) {
