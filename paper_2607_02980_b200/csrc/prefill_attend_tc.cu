@@ -10,7 +10,7 @@
 //            are contiguous there, so every epilogue warp hands its 32 rows to one TMA store per half.
 // Warp roles: 0-7 epilogue (warps 0-3 take even tiles, 4-7 odd tiles; a warp reads the TMEM lane quarter
 // warp % 4), 8-11 producers (cp.async gather of Q rows, TMA of K/V), 12 MMA issue.
-// S/P/O are double buffered, three gathered Q tiles are in flight, K/V is double buffered per chunk.
+// S/P/O are double buffered, three gathered Q tiles are in flight, K tiles are double and V tiles triple buffered.
 #include "internal.h"
 #include "tma.cuh"
 
@@ -29,6 +29,7 @@ constexpr int kQBytes = kRows * kD * 2;         // 32 KB
 constexpr int kPBytes = kRows * 128;            // 16 KB
 constexpr int kBatch = 128;                     // tile records cached per batch
 constexpr int kQSlots = 3;                      // gathered Q tiles in flight
+constexpr int kVBufs = 3;                       // V tiles in flight (K: 2)
 constexpr int kMetaSlots = 8;                   // ring of tile descriptors (producers are < 8 tiles ahead of the epilogue)
 constexpr int kProdThreads = 128;
 constexpr int kEpiThreads = 256;
@@ -38,8 +39,12 @@ constexpr int kMmaWarp = kProdWarp0 + kProdThreads / 32;
 constexpr float kLog2e = 1.4426950408889634f;
 
 struct AtcSmem {
-    uint64_t kv_ready[2];     // K tile and V landed (TMA bytes) and the landmark row written (one arrival): usable by the MMA
-    uint64_t kv_empty[2];     // every MMA that reads this K/V buffer has completed
+    // K tiles live in a ring of 2 (free again after the chunk's last S MMA), V tiles in a ring of kVBufs (free after
+    // its last P V MMA, about one epilogue phase later)
+    uint64_t k_ready[2];      // K tile landed (TMA bytes) and the landmark row written (one arrival)
+    uint64_t v_ready[kVBufs]; // V tile landed
+    uint64_t k_empty[2];      // every S MMA that reads this K buffer has completed
+    uint64_t v_empty[kVBufs]; // every P V MMA that reads this V buffer has completed
     uint64_t q_full[kQSlots]; // gathered Q rows landed and fenced (one arrival per producer warp)
     uint64_t q_empty[kQSlots];// the S MMA that reads this Q tile has completed
     uint64_t s_full[2];       // S = Q K^T in tensor memory
@@ -90,8 +95,8 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
     extern __shared__ uint8_t smem_raw[];
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* kbuf = base;                                   // [2][kKBytes]
-    uint8_t* vbuf = kbuf + 2 * kKBytes;                     // [2][kVBytes]
-    uint8_t* qbuf = vbuf + 2 * kVBytes;                     // [kQSlots][kQBytes]
+    uint8_t* vbuf = kbuf + 2 * kKBytes;                     // [kVBufs][kVBytes]
+    uint8_t* qbuf = vbuf + kVBufs * kVBytes;                     // [kQSlots][kQBytes]
     uint8_t* pbuf = qbuf + kQSlots * kQBytes;               // [2][kPBytes]
     AtcSmem& sm = *reinterpret_cast<AtcSmem*>(pbuf + 2 * kPBytes);
 
@@ -104,9 +109,10 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
 
     if (tid == 0) {
         for (int i = 0; i < kQSlots; ++i) { mbar_init(&sm.q_full[i], 4); mbar_init(&sm.q_empty[i], 1); }
+        for (int i = 0; i < kVBufs; ++i) { mbar_init(&sm.v_ready[i], 1); mbar_init(&sm.v_empty[i], 1); }
         for (int i = 0; i < 2; ++i) {
-            mbar_init(&sm.kv_ready[i], 2);          // the TMA issuer's arrive.expect_tx + the landmark writer
-            mbar_init(&sm.kv_empty[i], 1);
+            mbar_init(&sm.k_ready[i], 2);           // the TMA issuer's arrive.expect_tx + the landmark writer
+            mbar_init(&sm.k_empty[i], 1);
             mbar_init(&sm.s_full[i], 1);
             mbar_init(&sm.s_empty[i], 4);
             mbar_init(&sm.p_full[i], 4);
@@ -173,17 +179,19 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                 if (pair != cur_pair || c != cur_c) {
                     // ---- new chunk: its K/V go to buffer cc & 1.  Nobody here waits for the copies: they complete on
                     //      kv_ready, which only the MMA warp waits for, so the Q gathers below overlap them.
-                    const uint32_t cbuf = cc & 1u;
+                    const uint32_t cbuf = cc & 1u, vb = cc % kVBufs;
                     if (pw == 0) {
                         if (lane == 0 && !next_issued) {
-                            if (cc >= 2 && !mbar_wait(&sm.kv_empty[cbuf], ((cc >> 1) - 1) & 1)) dead = true;
+                            if (cc >= 2 && !mbar_wait(&sm.k_empty[cbuf], ((cc >> 1) - 1) & 1)) dead = true;
+                            if (!dead && cc >= kVBufs && !mbar_wait(&sm.v_empty[vb], ((cc / kVBufs) - 1) & 1)) dead = true;
                             if (!dead) {
                                 const int row = pair * s.T + c * kS;
-                                mbar_expect_tx(&sm.kv_ready[cbuf], 2 * 8192 + kVBytes);
-                                tma_load_2d(kbuf + cbuf * kKBytes, &map_k, &sm.kv_ready[cbuf], 0, row);
-                                tma_load_2d(kbuf + cbuf * kKBytes + kNS * 128, &map_k, &sm.kv_ready[cbuf], 64, row);
-                                tma_load_2d(vbuf + cbuf * kVBytes, &map_v, &sm.kv_ready[cbuf], 0, row);
-                                tma_load_2d(vbuf + cbuf * kVBytes + 8192, &map_v, &sm.kv_ready[cbuf], 64, row);
+                                mbar_expect_tx(&sm.k_ready[cbuf], 2 * 8192);
+                                tma_load_2d(kbuf + cbuf * kKBytes, &map_k, &sm.k_ready[cbuf], 0, row);
+                                tma_load_2d(kbuf + cbuf * kKBytes + kNS * 128, &map_k, &sm.k_ready[cbuf], 64, row);
+                                mbar_expect_tx(&sm.v_ready[vb], kVBytes);
+                                tma_load_2d(vbuf + vb * kVBytes, &map_v, &sm.v_ready[vb], 0, row);
+                                tma_load_2d(vbuf + vb * kVBytes + 8192, &map_v, &sm.v_ready[vb], 64, row);
                             }
                         }
                         next_issued = false;
@@ -200,7 +208,7 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                             }
                             fence_proxy_async_smem();
                             __syncwarp();
-                            if (lane == 0) mbar_arrive(&sm.kv_ready[cbuf]);
+                            if (lane == 0) mbar_arrive(&sm.k_ready[cbuf]);
                         }
                     }
                     if (dead || *reinterpret_cast<volatile int*>(&sm.abort_flag)) { dead = true; break; }
@@ -221,14 +229,16 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                 // ---- look ahead (producer thread 0): request the next chunk's K/V as soon as its buffer is free
                 if (ptid == 0 && !next_issued) {
                     const int tj = sm.cfirst[ck + 1];          // first tile of the next run (nb if none)
-                    const uint32_t nbuf = cc & 1u;
-                    if (tj < nb && (cc < 2 || mbar_try_wait(&sm.kv_empty[nbuf], ((cc >> 1) - 1) & 1))) {
+                    const uint32_t nbuf = cc & 1u, nvb = cc % kVBufs;
+                    if (tj < nb && (cc < 2 || mbar_try_wait(&sm.k_empty[nbuf], ((cc >> 1) - 1) & 1)) &&
+                        (cc < kVBufs || mbar_try_wait(&sm.v_empty[nvb], ((cc / kVBufs) - 1) & 1))) {
                         const int row = sm.recs[tj].x * s.T + sm.recs[tj].y * kS;
-                        mbar_expect_tx(&sm.kv_ready[nbuf], 2 * 8192 + kVBytes);
-                        tma_load_2d(kbuf + nbuf * kKBytes, &map_k, &sm.kv_ready[nbuf], 0, row);
-                        tma_load_2d(kbuf + nbuf * kKBytes + kNS * 128, &map_k, &sm.kv_ready[nbuf], 64, row);
-                        tma_load_2d(vbuf + nbuf * kVBytes, &map_v, &sm.kv_ready[nbuf], 0, row);
-                        tma_load_2d(vbuf + nbuf * kVBytes + 8192, &map_v, &sm.kv_ready[nbuf], 64, row);
+                        mbar_expect_tx(&sm.k_ready[nbuf], 2 * 8192);
+                        tma_load_2d(kbuf + nbuf * kKBytes, &map_k, &sm.k_ready[nbuf], 0, row);
+                        tma_load_2d(kbuf + nbuf * kKBytes + kNS * 128, &map_k, &sm.k_ready[nbuf], 64, row);
+                        mbar_expect_tx(&sm.v_ready[nvb], kVBytes);
+                        tma_load_2d(vbuf + nvb * kVBytes, &map_v, &sm.v_ready[nvb], 0, row);
+                        tma_load_2d(vbuf + nvb * kVBytes + 8192, &map_v, &sm.v_ready[nvb], 64, row);
                         next_issued = true;
                     }
                 }
@@ -275,8 +285,9 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
             if (dead && lane == 0) { set_status(a.status, kDevTimeout); atomicExch(&sm.abort_flag, 1); }
             if (ptid == 0 && next_issued) {
                 // (only after a timeout) a requested chunk was never taken up: complete its barrier, let the copy land
-                mbar_arrive(&sm.kv_ready[cc & 1u]);
-                mbar_wait(&sm.kv_ready[cc & 1u], (cc >> 1) & 1);
+                mbar_arrive(&sm.k_ready[cc & 1u]);
+                mbar_wait(&sm.k_ready[cc & 1u], (cc >> 1) & 1);
+                mbar_wait(&sm.v_ready[cc % kVBufs], (cc / kVBufs) & 1);
             }
         } else if (warp == kMmaWarp) {
             // ================================================================ MMA issuer
@@ -285,7 +296,7 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                 constexpr uint32_t idesc_o = umma_idesc_bf16(kRows, kD) | kUmmaBMnMajor;
                 uint32_t cc = ccount;
                 int cur_pair = -1, cur_c = -1;
-                uint32_t cbuf_of[2] = {0u, 0u};        // K/V buffer used by the tile in S/P/O slot i
+                uint32_t vbuf_of[2] = {0u, 0u};        // V buffer used by the tile in S/P/O slot i
                 bool ok = true;
                 // Two in-order queues (S MMAs, O MMAs) served by polling: an O MMA whose probabilities are
                 // ready is never held up by a Q tile that has not arrived yet, and vice versa.
@@ -298,12 +309,14 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                         const int4 rec = sm.recs[ns];
                         const bool newc = rec.x != cur_pair || rec.y != cur_c;
                         bool ready = mbar_try_wait(&sm.q_full[qs], (tcv / kQSlots) & 1);
-                        if (ready && newc) ready = mbar_try_wait(&sm.kv_ready[cc & 1u], (cc >> 1) & 1);
+                        if (ready && newc)
+                            ready = mbar_try_wait(&sm.k_ready[cc & 1u], (cc >> 1) & 1) &&
+                                    mbar_try_wait(&sm.v_ready[cc % kVBufs], (cc / kVBufs) & 1);
                         if (ready && tcv >= 2) ready = mbar_try_wait(&sm.s_empty[sl], ((tcv >> 1) - 1) & 1);
                         if (ready) {
                             if (newc) { cur_pair = rec.x; cur_c = rec.y; ++cc; }
                             const uint32_t cb = (cc - 1) & 1u;
-                            cbuf_of[sl] = cb;
+                            vbuf_of[sl] = (cc - 1) % kVBufs;
                             tc_fence_after_sync();
                             const uint32_t qa = smem_u32(qbuf + qs * kQBytes), ka = smem_u32(kbuf + cb * kKBytes);
 #pragma unroll
@@ -312,25 +325,27 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                                           umma_desc_k128(ka + (ks >> 2) * (kNS * 128) + (ks & 3) * 32), idesc_s, ks > 0 ? 1u : 0u);
                             umma_commit(&sm.s_full[sl]);
                             umma_commit(&sm.q_empty[qs]);
+                            // last tile of its chunk in this batch: the K buffer is free once these MMAs are done
+                            if (ns + 1 >= nb || sm.recs[ns + 1].x != rec.x || sm.recs[ns + 1].y != rec.y) umma_commit(&sm.k_empty[cb]);
                             ++ns;
                             progressed = true;
                         }
                     }
                     if (no < ns) {
-                        const uint32_t tcv = tcount + no, sl = tcv & 1u, cb = cbuf_of[sl];
+                        const uint32_t tcv = tcount + no, sl = tcv & 1u, vb = vbuf_of[sl];
                         bool ready = mbar_try_wait(&sm.p_full[sl], (tcv >> 1) & 1);
                         if (ready && tcv >= 2) ready = mbar_try_wait(&sm.o_empty[sl], ((tcv >> 1) - 1) & 1);
                         if (ready) {
                             tc_fence_after_sync();
-                            const uint32_t pa = smem_u32(pbuf + sl * kPBytes), va = smem_u32(vbuf + cb * kVBytes);
+                            const uint32_t pa = smem_u32(pbuf + sl * kPBytes), va = smem_u32(vbuf + vb * kVBytes);
 #pragma unroll
                             for (int ks = 0; ks < 4; ++ks)      // 16 keys per step = two 8-row groups of V
                                 umma_bf16(tmem_base + 256 + sl * 128, umma_desc_k128(pa + ks * 32),
                                           umma_desc_mn128(va + ks * 2048, 8192u, 1024u), idesc_o, ks > 0 ? 1u : 0u);
                             umma_commit(&sm.o_full[sl]);
-                            // last tile of its chunk in this batch: the K/V buffer is free once these MMAs are done
+                            // last tile of its chunk in this batch: the V buffer is free once these MMAs are done
                             const bool last = no + 1 >= nb || sm.recs[no + 1].x != sm.recs[no].x || sm.recs[no + 1].y != sm.recs[no].y;
-                            if (last) umma_commit(&sm.kv_empty[cb]);
+                            if (last) umma_commit(&sm.v_empty[vb]);
                             ++no;
                             progressed = true;
                         }
@@ -470,7 +485,7 @@ int launch_prefill_attend_tc(const Shape& s, const void* q, const void* maps, co
                              const float* bias, const int* entries, const void* tiles, const int* n_tiles, float* lam,
                              int* status, int i0, cudaStream_t stream) {
     const CUtensorMap* m = static_cast<const CUtensorMap*>(maps);
-    const size_t smem = 2 * kKBytes + 2 * kVBytes + kQSlots * kQBytes + 2 * kPBytes + sizeof(AtcSmem) + 1024;
+    const size_t smem = 2 * kKBytes + kVBufs * kVBytes + kQSlots * kQBytes + 2 * kPBytes + sizeof(AtcSmem) + 1024;
     static bool attr_done = false;
     if (!attr_done) {
         if (cudaFuncSetAttribute(prefill_attend_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
