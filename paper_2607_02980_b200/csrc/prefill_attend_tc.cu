@@ -166,6 +166,8 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
             int cur_pair = -1, cur_c = -1;
             int ck = -1;                       // ordinal of the current chunk run within the batch
             bool next_issued = false;          // (producer thread 0) K/V of the upcoming chunk already requested
+            uint4 lm_next = make_uint4(0u, 0u, 0u, 0u);   // (producer lanes 0-15) landmark piece of the next run, fetched a run ahead
+            bool lm_next_ok = false;
             bool dead = false;
             // entry of this thread's row for the upcoming tile, fetched one tile ahead
             int e_next = a.entries[sm.recs[0].z + min(ptid >> 2, sm.recs[0].w - 1)];
@@ -202,9 +204,19 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                             // MMA reads it as an MN-major operand; keys past the end of the sequence hold other rows'
                             // data (or TMA zero fill) and meet probabilities of 0.
                             if (lane < 16) {
-                                uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                                if (c < s.C) v = *reinterpret_cast<const uint4*>(a.lm + (static_cast<long long>(pair) * s.C + c) * kD + lane * 8);
+                                uint4 v = lm_next;
+                                if (!lm_next_ok) {
+                                    v = make_uint4(0u, 0u, 0u, 0u);
+                                    if (c < s.C) v = *reinterpret_cast<const uint4*>(a.lm + (static_cast<long long>(pair) * s.C + c) * kD + lane * 8);
+                                }
                                 *reinterpret_cast<uint4*>(kbuf + cbuf * kKBytes + (lane >> 3) * (kNS * 128) + swz128(64, lane & 7)) = v;
+                                // the next run's landmark, so that its load is not waited for at the next switch
+                                lm_next_ok = ck + 2 < sm.nchunks;
+                                if (lm_next_ok) {
+                                    const int4 r1 = sm.recs[sm.cfirst[ck + 2]];
+                                    lm_next = make_uint4(0u, 0u, 0u, 0u);
+                                    if (r1.y < s.C) lm_next = *reinterpret_cast<const uint4*>(a.lm + (static_cast<long long>(r1.x) * s.C + r1.y) * kD + lane * 8);
+                                }
                             }
                             fence_proxy_async_smem();
                             __syncwarp();
