@@ -49,6 +49,7 @@ def _load():
         _lib = ctypes.CDLL(_SO)
         _lib.hils_oracle_rows.restype = ctypes.c_int
         _lib.hils_oracle_num_threads.restype = ctypes.c_int
+        _lib.hils_oracle_landmarks.restype = ctypes.c_int
     return _lib
 
 
@@ -158,3 +159,27 @@ def hils_decode(q, k_cache, v_cache, landmarks, bias, seq_lens, *, S: int, K: in
     return hils_rows(qn.reshape(B, Hq, 1, d), k_cache, v_cache, landmarks, bias, S=S, K=K, W=W,
                      scale=scale, row_b=np.arange(B, dtype=np.int32), row_qi=np.zeros(B, dtype=np.int32),
                      row_pos=seq - 1, sel_idx=sel_idx, group_mode=group_mode, want_alpha=want_alpha)
+
+
+def hils_landmarks(lq, k, seq_lens=None, *, S: int, scale: float = 0.0):
+    """Chunk summaries of Proposition 3.1 (Eq. prop_q_c): k'_c = Attn(q'_c, K_c, K_c), b'_c = entropy.
+
+    lq [B,Hl,C,d] learnable chunk queries, k [B,Hkv,T,d] keys (both fp32 or both bf16), seq_lens [B] or None.
+    Returns (landmarks [B,Hl,C,d], bias [B,Hl,C]) as float64 numpy arrays.
+    """
+    lib = _load()
+    in_bf16 = int(_is_bf16(lq) and _is_bf16(k))
+    conv = _raw_bf16 if in_bf16 else _f32
+    lq = conv(lq); k = conv(k)
+    B, Hl, C, d = lq.shape
+    _, Hkv, T, _ = k.shape
+    sl = None if seq_lens is None else np.ascontiguousarray(
+        seq_lens.detach().cpu().numpy() if hasattr(seq_lens, "detach") else seq_lens, dtype=np.int32)
+    p = _Params(B, Hl, Hkv, Hl, 0, T, C, d, S, 1, 1, float(scale), 0, in_bf16)
+    lm = np.zeros((B, Hl, C, d), dtype=np.float64)
+    bias = np.zeros((B, Hl, C), dtype=np.float64)
+    rc = lib.hils_oracle_landmarks(ctypes.byref(p), ctypes.c_void_p(lq.ctypes.data), ctypes.c_void_p(k.ctypes.data),
+                                   _ptr(sl, ctypes.c_int32), _ptr(lm, ctypes.c_double), _ptr(bias, ctypes.c_double))
+    if rc != 0:
+        raise ValueError("hils_oracle_landmarks rejected its arguments (rc=%d)" % rc)
+    return lm, bias

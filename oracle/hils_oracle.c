@@ -32,6 +32,9 @@
  * or raw bf16 arrays, widened exactly to fp64 element by element; all
  * arithmetic is fp64 with libm exp/log.
  *
+ * hils_oracle_landmarks (bottom of the file) is the step upstream of the operator: the
+ * chunk summary of Proposition 3.1 (Eq. prop_q_c), pinned by tests/test_landmark_pins.py.
+ *
  * Pinned by tests/test_oracle_pins.py (closed forms, invariants, library
  * attention on reductions, an independent dense-weight brute force).  The paper
  * prints no worked numeric example, so absolute values against the authors'
@@ -262,4 +265,69 @@ int hils_oracle_num_threads(void) {
 #else
     return 1;
 #endif
+}
+
+
+/*
+ * Chunk summaries of Proposition 3.1 (Eq. LogSumExp linearization / Eq. prop_q_c).
+ * For sequence b, landmark head hl (its KV head is hl / (Hl / Hkv)) and chunk c, with the chunk's
+ * keys k_j, j in [c*S, min((c+1)*S, len_b)) and its learnable query q'_c = lq[b, hl, c, :]:
+ *     s_j = scale * q'_c . k_j,   p = softmax_j(s),
+ *     k'_c = sum_j p_j k_j                      (Attn(q'_c, K_c, K_c)),
+ *     b'_c = - sum_j p_j log p_j                (entropy of p).
+ * A chunk without tokens gets k' = 0, b' = 0.  The paper defines the summary for complete chunks; a
+ * partial last chunk uses the tokens it has (reading: the softmax runs over the tokens present).
+ *
+ * lq [B,Hl,C,d] and k [B,Hkv,T,d] are fp32 or raw bf16 (in_bf16); seq_lens [B] or NULL (= T);
+ * out_landmarks [B,Hl,C,d] and out_bias [B,Hl,C] are doubles.  Returns 0, or -1 for bad arguments.
+ */
+int hils_oracle_landmarks(const hils_oracle_params *p, const void *lq, const void *k, const int32_t *seq_lens,
+                          double *out_landmarks, double *out_bias) {
+    if (!p || !lq || !k || !out_landmarks || !out_bias) return -1;
+    if (p->B < 1 || p->Hkv < 1 || p->Hl < 1 || p->Hl % p->Hkv != 0 || p->d < 1 || p->S < 1 || p->C < 0 || p->T < 0)
+        return -1;
+    const int per = p->Hl / p->Hkv;
+    const double scale = p->scale > 0 ? p->scale : 1.0 / sqrt((double)p->d);
+    const long total = (long)p->B * p->Hl * p->C;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(static)
+#endif
+    for (long x = 0; x < total; ++x) {
+        const int c = (int)(x % p->C);
+        const int hl = (int)((x / p->C) % p->Hl);
+        const int b = (int)(x / ((long)p->C * p->Hl));
+        const int hkv = hl / per;
+        long len = seq_lens ? seq_lens[b] : p->T;
+        if (len > p->T) len = p->T;
+        const long j0 = (long)c * p->S;
+        long j1 = j0 + p->S;
+        if (j1 > len) j1 = len;
+        double *kp = out_landmarks + (size_t)x * p->d;
+        for (int e = 0; e < p->d; ++e) kp[e] = 0.0;
+        out_bias[x] = 0.0;
+        if (j1 <= j0) continue;
+        const size_t qoff = (size_t)x * p->d;
+        const size_t koff = ((size_t)b * p->Hkv + hkv) * (size_t)p->T * p->d;
+        const int n = (int)(j1 - j0);
+        double *s = (double *)malloc(sizeof(double) * (size_t)n);
+        double m = -INFINITY;
+        for (int j = 0; j < n; ++j) {
+            double acc = 0.0;
+            for (int e = 0; e < p->d; ++e)
+                acc += ld(lq, qoff + e, p->in_bf16) * ld(k, koff + (size_t)(j0 + j) * p->d + e, p->in_bf16);
+            s[j] = scale * acc;
+            if (s[j] > m) m = s[j];
+        }
+        double z = 0.0;
+        for (int j = 0; j < n; ++j) z += exp(s[j] - m);
+        double ent = 0.0;
+        for (int j = 0; j < n; ++j) {
+            const double pj = exp(s[j] - m) / z;
+            if (pj > 0.0) ent -= pj * log(pj);
+            for (int e = 0; e < p->d; ++e) kp[e] += pj * ld(k, koff + (size_t)(j0 + j) * p->d + e, p->in_bf16);
+        }
+        out_bias[x] = ent;
+        free(s);
+    }
+    return 0;
 }
