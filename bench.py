@@ -282,6 +282,31 @@ def roofline_for(w, kernel_ms, peaks):
                 algorithmic_flops=algo)
 
 
+def bench_landmark_summary(hils, w, peaks, iters=10):
+    """The chunk-summary kernel (Proposition 3.1) on the workload's K tensor: every chunk of every KV head once.
+    HBM-bound; algorithmic bytes = K read once + the learnable queries read + the summaries written."""
+    cfg = w.cfg
+    k = w.inp["k"]
+    lq = wl.make_landmark_queries(cfg, k.device)
+    lm = torch.empty_like(lq)
+    bias = torch.empty(lq.shape[:3], dtype=torch.float32, device=k.device)
+    for _ in range(3):
+        hils.hils_landmark_summary(lq, k, cfg.S, landmarks=lm, bias=bias)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(iters + 1)]
+    torch.cuda.synchronize()
+    ev[0].record()
+    for i in range(iters):
+        hils.hils_landmark_summary(lq, k, cfg.S, landmarks=lm, bias=bias)
+        ev[i + 1].record()
+    torch.cuda.synchronize()
+    ms = float(np.mean([ev[i].elapsed_time(ev[i + 1]) for i in range(iters)]))
+    nbytes = k.numel() * k.element_size() + 2 * lq.numel() * lq.element_size() + bias.numel() * 4
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    return {"metric": "landmark_summary_algorithmic_GBps", "value": gbs, "unit": "GB/s", "ms": ms,
+            "algorithmic_bytes": nbytes, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"],
+            "l2_policy": "K tensor of %.0f MB > 126 MB L2, read once per call" % (k.numel() * k.element_size() / 1e6)}
+
+
 # ----------------------------------------------------------------------------- CPU oracle legs
 def oracle_sample(cfg, inp_cpu, budget_rows):
     """Times the oracle, as it stands, on a bounded sample of the workload.  Returns (value, sample, secs)."""
@@ -505,6 +530,9 @@ def main():
                     ent["frac_of_nominal_2250_TFLOPs"] = ent["value"] / 2250.0
                 extras[name] = ent
                 launches += hils.last_launch_count() * (max(3, args.steps) + 3)
+                if name in ("cfg2", "cfg3"):
+                    extras["landmark_summary_" + name] = bench_landmark_summary(hils, ew, peaks)
+                    launches += 13
                 del ew
                 torch.cuda.empty_cache()
             except Exception as exc:  # keep the primary line even if an extra fails

@@ -130,6 +130,29 @@ int hils_decode_noalloc(const hils_params* params, const void* q, const void* k_
                         const void* landmarks, const float* bias, const int32_t* seq_lens,
                         void* out, float* lse, int32_t* sel_idx, int32_t* device_status, void* stream);
 
+/* Chunk summaries -- the step upstream of the operator (Proposition 3.1, Eq. LogSumExp linearization /
+ * Eq. prop_q_c).  For every sequence b, landmark head hl (its KV head is hl / (Hl / Hkv)) and chunk
+ * c in [chunk_begin, chunk_begin + chunk_count), with the chunk's keys k_j, j in [c*S, min((c+1)*S, len_b))
+ * and its learnable query q'_c = landmark_queries[b, hl, c, :]:
+ *     s_j = scale * q'_c . k_j,   p = softmax_j(s),
+ *     landmarks[b, hl, c, :] = k'_c = sum_j p_j k_j        (Attn(q'_c, K_c, K_c)),
+ *     bias[b, hl, c]         = b'_c = - sum_j p_j log p_j  (entropy of p),
+ * i.e. the `landmarks` / `bias` inputs of hils_prefill and hils_decode.  A chunk without tokens gets
+ * zeros; a partial last chunk uses the tokens it has.  Serving code calls this for the chunk that has
+ * just been completed (chunk_count = 1); prefill calls it for all chunks (chunk_count <= 0 means "up to C").
+ *
+ *   landmark_queries [B, Hl, C, d]  DEVICE, params->dtype
+ *   k                [B, Hkv, T, d] DEVICE, params->dtype, T = params->T_max if > 0, else params->L
+ *   seq_lens         [B] int32 DEVICE or NULL (NULL: every sequence holds T tokens)
+ *   landmarks        [B, Hl, C, d]  DEVICE, params->dtype (written for the requested chunks only)
+ *   bias             [B, Hl, C] fp32 DEVICE (same)
+ * Uses of params: B, Hkv, Hl, C, d, chunk_size (<= 128), scale, dtype, T_max / L; d a multiple of 32, <= 256.
+ * Needs no workspace; one kernel is enqueued on `stream`.  Errors: HILS_ERR_INVALID_ARG (null pointer, bad
+ * range or size), HILS_ERR_ALIGNMENT, HILS_ERR_UNSUPPORTED (d or chunk size outside the limits), HILS_ERR_CUDA. */
+int hils_landmark_summary(const hils_params* params, const void* landmark_queries, const void* k,
+                          const int32_t* seq_lens, int32_t chunk_begin, int32_t chunk_count, void* landmarks,
+                          float* bias, void* stream);
+
 /* Bytes of device memory the *_host entry points need for staging (inputs + outputs + workspace). */
 size_t hils_host_arena_bytes(const hils_params* params, int is_decode);
 

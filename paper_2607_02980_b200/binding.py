@@ -24,6 +24,7 @@ EXPORTS = [
     "hils_workspace_bytes", "hils_prefill", "hils_decode", "hils_host_arena_bytes",
     "hils_prefill_host", "hils_decode_host", "hils_poll_status", "hils_last_launch_count",
     "hils_status_string", "hils_version", "hils_trace_enable", "hils_trace_read", "hils_decode_noalloc",
+    "hils_landmark_summary",
 ]
 
 
@@ -69,6 +70,8 @@ def load_library() -> ctypes.CDLL:
     lib.hils_decode_host.argtypes = [pp, vp, vp, vp, vp, f32p, i32p, vp, f32p, i32p, vp, ctypes.c_size_t, vp]
     lib.hils_decode_noalloc.restype = ctypes.c_int
     lib.hils_decode_noalloc.argtypes = [pp, vp, vp, vp, vp, f32p, i32p, vp, f32p, i32p, i32p, vp]
+    lib.hils_landmark_summary.restype = ctypes.c_int
+    lib.hils_landmark_summary.argtypes = [pp, vp, vp, i32p, ctypes.c_int32, ctypes.c_int32, vp, f32p, vp]
     lib.hils_poll_status.restype = ctypes.c_int
     lib.hils_poll_status.argtypes = [vp, vp]
     lib.hils_last_launch_count.restype = ctypes.c_int
@@ -248,6 +251,37 @@ def hils_decode_noalloc(q, k_cache, v_cache, landmarks, seq_lens, chunk_size: in
     if rc != 0:
         raise HilsError(rc, "hils_decode_noalloc")
     return out, lse, sel_idx
+
+
+def hils_landmark_summary(landmark_queries, k, chunk_size: int, *, seq_lens=None, scale: float = 0.0,
+                          chunk_begin: int = 0, chunk_count: int = 0, landmarks=None, bias=None, stream=None):
+    """Chunk summaries of Proposition 3.1: landmarks k'_c = Attn(q'_c, K_c, K_c) and bias b'_c = entropy.
+
+    landmark_queries [B,Hl,C,d] and k [B,Hkv,T,d] are CUDA tensors of one dtype; seq_lens [B] int32 or None.
+    Computes the chunks [chunk_begin, chunk_begin + chunk_count) (chunk_count <= 0: up to C) into `landmarks`
+    [B,Hl,C,d] / `bias` [B,Hl,C] (allocated, zero-filled, when not passed).  Returns (landmarks, bias).
+    """
+    lib = load_library()
+    B, Hl, C, d = landmark_queries.shape
+    Hkv, T = k.shape[1], k.shape[2]
+    dt = landmark_queries.dtype
+    _check(landmark_queries, "landmark_queries", (B, Hl, C, d), dt, True)
+    _check(k, "k", (B, Hkv, T, d), dt, True)
+    if seq_lens is not None:
+        _check(seq_lens, "seq_lens", (B,), torch.int32, True)
+    if landmarks is None:
+        landmarks = torch.zeros((B, Hl, C, d), dtype=dt, device=k.device)
+    if bias is None:
+        bias = torch.zeros((B, Hl, C), dtype=torch.float32, device=k.device)
+    _check(landmarks, "landmarks", (B, Hl, C, d), dt, True)
+    _check(bias, "bias", (B, Hl, C), torch.float32, True)
+    p = make_params(B=B, Hq=Hl, Hkv=Hkv, Hl=Hl, L=0, T_max=T, C=C, d=d, chunk_size=chunk_size, top_k=1,
+                    window=1, scale=scale, dtype=_dtype_code(k), impl="auto")
+    rc = lib.hils_landmark_summary(ctypes.byref(p), _ptr(landmark_queries), _ptr(k), _ptr(seq_lens),
+                                   int(chunk_begin), int(chunk_count), _ptr(landmarks), _ptr(bias), _stream_ptr(stream))
+    if rc != 0:
+        raise HilsError(rc, "hils_landmark_summary")
+    return landmarks, bias
 
 
 class HostRunner:

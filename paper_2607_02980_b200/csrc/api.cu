@@ -244,6 +244,35 @@ int hils_decode_noalloc(const hils_params* params, const void* q, const void* k_
     return HILS_OK;
 }
 
+int hils_landmark_summary(const hils_params* params, const void* landmark_queries, const void* k,
+                          const int32_t* seq_lens, int32_t chunk_begin, int32_t chunk_count, void* landmarks,
+                          float* bias, void* stream) {
+    g_last_launches = 0;
+    const hils_params* p = params;
+    if (!p || !landmark_queries || !k || !landmarks || !bias) return HILS_ERR_INVALID_ARG;
+    if (p->B < 1 || p->Hkv < 1 || p->Hl < 1 || p->Hl % p->Hkv != 0 || p->C < 1 || p->d < 1 || p->chunk_size < 1)
+        return HILS_ERR_INVALID_ARG;
+    if (p->dtype != HILS_F32 && p->dtype != HILS_BF16) return HILS_ERR_INVALID_ARG;
+    const long long T = p->T_max > 0 ? p->T_max : p->L;
+    if (T < 1 || !(p->scale >= 0.f)) return HILS_ERR_INVALID_ARG;
+    if (chunk_begin < 0 || chunk_begin > p->C) return HILS_ERR_INVALID_ARG;
+    const int cn = chunk_count <= 0 ? p->C - chunk_begin : chunk_count;
+    if (cn > p->C - chunk_begin) return HILS_ERR_INVALID_ARG;
+    if (!aligned16(landmark_queries) || !aligned16(k) || !aligned16(landmarks) ||
+        (reinterpret_cast<uintptr_t>(bias) & 3u) || (seq_lens && (reinterpret_cast<uintptr_t>(seq_lens) & 3u)))
+        return HILS_ERR_ALIGNMENT;
+    if (!landmark_summary_supports(p->d, p->chunk_size)) return HILS_ERR_UNSUPPORTED;
+    const float scale = p->scale > 0.f ? p->scale : 1.0f / sqrtf(static_cast<float>(p->d));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    trace_begin(st);
+    const int n = launch_landmark_summary(p->dtype, p->B, p->Hkv, p->Hl, p->C, p->d, p->chunk_size, T, scale,
+                                          landmark_queries, k, seq_lens, chunk_begin, cn, landmarks, bias, st);
+    if (n < 0) return n;
+    trace_mark("landmark_summary", st);
+    g_last_launches = n;
+    return HILS_OK;
+}
+
 size_t hils_host_arena_bytes(const hils_params* params, int is_decode) {
     ArenaLayout a;
     if (arena_layout(params, is_decode, &a) != HILS_OK || a.ws_b == 0) return 0;

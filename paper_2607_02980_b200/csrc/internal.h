@@ -55,6 +55,12 @@ int launch_prefill_attend_tc(const Shape& s, const void* q, const void* maps, co
                              const float* bias, const int* entries, const void* tiles, const int* n_tiles, float* lam,
                              int* status, int i0, cudaStream_t stream);
 
+// Chunk summaries (Proposition 3.1): landmarks / bias of the chunks [c0, c0 + cn) from their learnable queries.
+bool landmark_summary_supports(int d, int S);
+int launch_landmark_summary(int dtype, int B, int Hkv, int Hl, int C, int d, int S, long long T, float scale,
+                            const void* lq, const void* k, const int32_t* seq_lens, int c0, int cn, void* landmarks,
+                            float* bias, cudaStream_t stream);
+
 int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream);
 bool prefill_fast_supports(const Shape& s, int dtype);
 size_t prefill_fast_scratch_bytes(const Shape& s);

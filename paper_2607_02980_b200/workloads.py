@@ -116,6 +116,22 @@ def _draw_landmarks(cfg: HilsConfig, k: torch.Tensor, gen, device) -> torch.Tens
     return out
 
 
+def make_landmark_queries(cfg: HilsConfig, device="cpu", Hl: Optional[int] = None, C: Optional[int] = None) -> torch.Tensor:
+    """Seeded learnable chunk queries q'_c [B, Hl, C, d] for the chunk-summary step (stand-ins for the query
+    vectors of trained landmark tokens): N(0, 1) in the config dtype, times sqrt(d) for the fp32 config whose
+    keys are N(0, 1)/sqrt(d), so that the scores inside a chunk have a standard deviation of about 1."""
+    dev = torch.device(device)
+    Hl = cfg.Hkv if Hl is None else Hl
+    C = cfg.C if C is None else C
+    gen = _gen(cfg.seed, 7, dev)
+    mul = math.sqrt(cfg.d) if cfg.dtype == "f32" else 1.0
+    out = torch.empty((cfg.B, Hl, C, cfg.d), dtype=cfg.torch_dtype(), device=dev)
+    for b in range(cfg.B):
+        for h in range(Hl):
+            out[b, h].copy_(_randn((C, cfg.d), gen, dev) * mul)
+    return out
+
+
 def _needle_dirs(lm_bh: torch.Tensor, idx: torch.Tensor) -> torch.Tensor:
     """3 * k'_n / ||k'_n|| for the landmark rows `idx` of one (b, KV head)."""
     rows = lm_bh.float()[idx]
