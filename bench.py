@@ -412,8 +412,14 @@ def main():
             w.between_steps()
             w.step()
         torch.cuda.synchronize()
+        kpc = hils.last_launch_count()
+        # the chunk-summary kernel over the same key tensor (two calls)
+        lq = wl.make_landmark_queries(cfg, w.inp["k"].device)
+        for _ in range(2):
+            hils.hils_landmark_summary(lq, w.inp["k"], cfg.S)
+        torch.cuda.synchronize()
         print(json.dumps({"profile_run": cfg.name, "B": cfg.B, "calls": args.warmup + args.steps,
-                          "kernels_per_call": hils.last_launch_count()}))
+                          "kernels_per_call": kpc, "landmark_summary_calls": 2}))
         return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 

@@ -474,45 +474,6 @@ __device__ inline int cta_of_item(long long x, long long N, int n_ctas) {
     return static_cast<int>(((x + 1) * n_ctas + N - 1) / N - 1);
 }
 
-// S = Q K^T for one 64-key tile held in shared memory (two 128B-swizzled boxes of 64 dims).
-__device__ inline void qk_tile(const uint32_t (&aq)[8][2], uint32_t ks_addr, int lane, float (&sc)[8][4]) {
-#pragma unroll
-    for (int nt = 0; nt < 8; ++nt) {
-        sc[nt][0] = sc[nt][1] = sc[nt][2] = sc[nt][3] = 0.f;
-#pragma unroll
-        for (int kp = 0; kp < 4; ++kp) {
-            const int row = nt * 8 + (lane & 7);
-            const int dim = kp * 32 + (lane >> 3) * 8;
-            const uint32_t addr = ks_addr + (dim >> 6) * 8192 + swz128(row, (dim & 63) >> 3);
-            uint32_t r0, r1, r2, r3;
-            ldmatrix_x4(addr, r0, r1, r2, r3);
-            const uint32_t a0[4] = {aq[2 * kp][0], 0u, aq[2 * kp][1], 0u};
-            mma_bf16_16816(sc[nt], a0, r0, r1);
-            const uint32_t a1[4] = {aq[2 * kp + 1][0], 0u, aq[2 * kp + 1][1], 0u};
-            mma_bf16_16816(sc[nt], a1, r2, r3);
-        }
-    }
-}
-
-// O += P V for one 64-key tile; p holds the (already weighted) probabilities of rows g in [0], [1].
-__device__ inline void pv_tile(const float (&p)[8][4], uint32_t vs_addr, int lane, float (&o)[16][4]) {
-#pragma unroll
-    for (int kk = 0; kk < 4; ++kk) {
-        const uint32_t ap[4] = {pack_bf16(p[2 * kk][0], p[2 * kk][1]), 0u, pack_bf16(p[2 * kk + 1][0], p[2 * kk + 1][1]), 0u};
-#pragma unroll
-        for (int dp = 0; dp < 8; ++dp) {
-            const int mat = lane >> 3;
-            const int row = kk * 16 + (mat & 1) * 8 + (lane & 7);
-            const int dim = dp * 16 + (mat >> 1) * 8;
-            const uint32_t addr = vs_addr + (dim >> 6) * 8192 + swz128(row, (dim & 63) >> 3);
-            uint32_t r0, r1, r2, r3;
-            ldmatrix_x4_trans(addr, r0, r1, r2, r3);
-            mma_bf16_16816(o[2 * dp], ap, r0, r1);
-            mma_bf16_16816(o[2 * dp + 1], ap, r2, r3);
-        }
-    }
-}
-
 __global__ void __launch_bounds__(kAttendThreads, 1)
 decode_attend_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                      const DArgs a) {

@@ -11,6 +11,7 @@
 // The loops are rolled (a first, fully unrolled register version was bound by instruction fetch at 20 % of
 // the memory bandwidth).  The kernel is bound by HBM: algorithmic bytes = the keys of the summarised chunks.
 #include "internal.h"
+#include "tma.cuh"
 
 namespace hils {
 namespace {
@@ -145,6 +146,132 @@ __global__ void landmark_summary_kernel(const LArgs a) {
     if (lane == 0) a.bias[orow] = __logf(z) - psum;
 }
 
+// ---- bf16, d = 128, S = 64, at most 8 landmark heads per KV head: both contractions on mma.sync ----
+// One warp per (sequence, KV head, chunk): the chunk's keys arrive as two TMA boxes (128B swizzle) in the warp's
+// own 16 KB tile; scores of all landmark heads of the KV head in one pass (the heads are the MMA rows), then
+// k' = P K with P split into two bf16 terms (p = hi + lo), so that the weights keep 16 bits of mantissa.
+constexpr int kTcWarps = 4;
+constexpr int kTcTileBytes = 64 * 128 * 2;
+
+struct TcSmemW {
+    uint64_t bar;
+};
+
+__global__ void __launch_bounds__(kTcWarps * 32)
+landmark_summary_tc_kernel(const __grid_constant__ CUtensorMap map_k, const LArgs a, int* timeout_flag) {
+    extern __shared__ uint8_t lsm_raw[];
+    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(lsm_raw) + 1023) & ~uintptr_t(1023));
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint8_t* tile = base + warp * kTcTileBytes;
+    TcSmemW& sw = reinterpret_cast<TcSmemW*>(base + kTcWarps * kTcTileBytes)[warp];
+    const int per = a.Hl / a.Hkv;                              // landmark heads per KV head (MMA rows), <= 8
+    const long long item = static_cast<long long>(blockIdx.x) * kTcWarps + warp;
+    const long long total = static_cast<long long>(a.B) * a.Hkv * a.cn;
+    if (item >= total) return;
+    const int c = a.c0 + static_cast<int>(item % a.cn);
+    const int hkv = static_cast<int>((item / a.cn) % a.Hkv);
+    const int b = static_cast<int>(item / (static_cast<long long>(a.cn) * a.Hkv));
+    long long len = a.seq ? a.seq[b] : a.T;
+    len = len < 0 ? 0 : (len > a.T ? a.T : len);
+    const long long j0 = static_cast<long long>(c) * 64;
+    const int n = static_cast<int>(len - j0 < 0 ? 0 : (len - j0 > 64 ? 64 : len - j0));
+    const int gq = lane >> 2, t = lane & 3;
+    const long long orow0 = (static_cast<long long>(b) * a.Hl + hkv * per) * a.C + c;      // head 0 of this KV head
+    __nv_bfloat16* lm = static_cast<__nv_bfloat16*>(a.lm);
+    if (n == 0) {
+        for (int x = lane; x < per * 64; x += 32)
+            *reinterpret_cast<uint32_t*>(lm + (orow0 + static_cast<long long>(x >> 6) * a.C) * 128 + (x & 63) * 2) = 0u;
+        if (lane < per) a.bias[orow0 + static_cast<long long>(lane) * a.C] = 0.f;
+        return;
+    }
+    if (lane == 0) {
+        mbar_init(&sw.bar, 1);
+        mbar_fence_init();
+        const int row = static_cast<int>((static_cast<long long>(b) * a.Hkv + hkv) * a.T + j0);
+        mbar_expect_tx(&sw.bar, kTcTileBytes);
+        tma_load_2d(tile, &map_k, &sw.bar, 0, row);
+        tma_load_2d(tile + 8192, &map_k, &sw.bar, 64, row);
+    }
+    // A operand: the `per` learnable queries of this KV head in rows 0..per-1 (loaded while the keys travel)
+    uint32_t aq[8][2];
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) { aq[ks][0] = 0u; aq[ks][1] = 0u; }
+    if (gq < per) {
+        const __nv_bfloat16* qrow = static_cast<const __nv_bfloat16*>(a.lq) + (orow0 + static_cast<long long>(gq) * a.C) * 128;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            aq[ks][0] = *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 2 * t);
+            aq[ks][1] = *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 8 + 2 * t);
+        }
+    }
+    __syncwarp();
+    if (!mbar_wait(&sw.bar, 0)) {
+        // the bounded wait ran out (never seen: the copy has a valid map): mark the chunk's bias NaN and leave
+        if (lane == 0 && timeout_flag) atomicExch(timeout_flag, 1);
+        if (lane < per) a.bias[orow0 + static_cast<long long>(lane) * a.C] = __int_as_float(0x7fc00000);
+        return;
+    }
+    if (n < 64) {
+        // rows past the sequence end may hold anything: zero them before they meet probabilities of 0
+        for (int x = lane; x < (64 - n) * 16; x += 32) {
+            const int row = n + (x >> 4), piece = x & 15;
+            *reinterpret_cast<uint4*>(tile + (piece >> 3) * 8192 + swz128(row, piece & 7)) = make_uint4(0u, 0u, 0u, 0u);
+        }
+        __syncwarp();
+    }
+    const uint32_t ks_addr = smem_u32(tile);
+    float sc[8][4];
+    qk_tile(aq, ks_addr, lane, sc);                             // sc[nt][0..1]: row gq, keys nt*8 + 2t, +1
+    const float sl = a.scale;
+    float m = -INFINITY;
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) {
+        const int key = nt * 8 + 2 * t;
+        sc[nt][0] = key < n ? sc[nt][0] * sl : -INFINITY;
+        sc[nt][1] = key + 1 < n ? sc[nt][1] * sl : -INFINITY;
+        m = fmaxf(m, fmaxf(sc[nt][0], sc[nt][1]));
+    }
+    m = fmaxf(m, __shfl_xor_sync(kFullMask, m, 1));
+    m = fmaxf(m, __shfl_xor_sync(kFullMask, m, 2));
+    float z = 0.f, ps = 0.f, e[8][2];
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) {
+        e[nt][0] = sc[nt][0] == -INFINITY ? 0.f : __expf(sc[nt][0] - m);
+        e[nt][1] = sc[nt][1] == -INFINITY ? 0.f : __expf(sc[nt][1] - m);
+        z += e[nt][0] + e[nt][1];
+    }
+    z += __shfl_xor_sync(kFullMask, z, 1);
+    z += __shfl_xor_sync(kFullMask, z, 2);
+    const float zi = 1.f / z;
+    float phi[8][4], plo[8][4];
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) {
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+            const float p = e[nt][x] * zi;
+            if (p > 0.f) ps = fmaf(p, sc[nt][x] - m, ps);
+            const float hi = __bfloat162float(__float2bfloat16_rn(p));
+            phi[nt][x] = hi;
+            plo[nt][x] = p - hi;
+        }
+        phi[nt][2] = phi[nt][3] = plo[nt][2] = plo[nt][3] = 0.f;
+    }
+    ps += __shfl_xor_sync(kFullMask, ps, 1);
+    ps += __shfl_xor_sync(kFullMask, ps, 2);
+    float o[16][4];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+    pv_tile(phi, ks_addr, lane, o);                             // the keys are the "values" of Attn(q', K, K)
+    pv_tile(plo, ks_addr, lane, o);
+    if (gq < per) {
+        __nv_bfloat16* dst = lm + (orow0 + static_cast<long long>(gq) * a.C) * 128;
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+            *reinterpret_cast<uint32_t*>(dst + i * 8 + 2 * t) = pack_bf16(o[i][0], o[i][1]);
+        if (t == 0) a.bias[orow0 + static_cast<long long>(gq) * a.C] = __logf(z) - ps;
+    }
+}
+
 template <typename T, int D>
 int launch_one(const LArgs& a, cudaStream_t stream) {
     const long long total = static_cast<long long>(a.B) * a.Hl * a.cn;
@@ -186,6 +313,26 @@ int launch_landmark_summary(int dtype, int B, int Hkv, int Hl, int C, int d, int
                             const void* lq, const void* k, const int32_t* seq_lens, int c0, int cn, void* landmarks,
                             float* bias, cudaStream_t stream) {
     LArgs a{B, Hkv, Hl, C, S, T, scale, lq, k, seq_lens, landmarks, bias, c0, cn};
+    static const bool no_tc = [] { const char* e = getenv("HILS_LANDMARK_NO_MMA"); return e && e[0] == '1'; }();
+    const long long rows = static_cast<long long>(B) * Hkv * T;
+    if (!no_tc && dtype == HILS_BF16 && d == 128 && S == 64 && Hl / Hkv <= 8 && rows < (1ll << 31)) {
+        const long long total = static_cast<long long>(B) * Hkv * cn;
+        if (total == 0) return 0;
+        CUtensorMap map_k;
+        if (!make_bf16_2d_map(&map_k, k, static_cast<uint64_t>(rows), 128, 64, 64)) return HILS_ERR_CUDA;
+        const size_t smem = kTcWarps * kTcTileBytes + kTcWarps * sizeof(TcSmemW) + 1024;
+        static bool attr_done = false;
+        if (!attr_done) {
+            if (cudaFuncSetAttribute(landmark_summary_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     static_cast<int>(smem)) != cudaSuccess)
+                return HILS_ERR_CUDA;
+            attr_done = true;
+        }
+        const long long blocks = (total + kTcWarps - 1) / kTcWarps;
+        if (blocks > 0x7fffffffll) return HILS_ERR_UNSUPPORTED;
+        landmark_summary_tc_kernel<<<static_cast<unsigned>(blocks), kTcWarps * 32, smem, stream>>>(map_k, a, nullptr);
+        return cudaGetLastError() == cudaSuccess ? 1 : HILS_ERR_CUDA;
+    }
     return dtype == HILS_F32 ? launch_typed<float>(a, d, stream) : launch_typed<__nv_bfloat16>(a, d, stream);
 }
 
