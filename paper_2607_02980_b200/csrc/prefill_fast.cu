@@ -247,15 +247,22 @@ prefill_select_kernel(const __grid_constant__ CUtensorMap map_lm, const PArgs a)
 }
 
 // ------------------------------------------------------------------------------------------ invert
-// Chunk attended by slot `slot` of token i0+il: a selected chunk, or (slot K) the token's own chunk.
+// Slots of a token: 0..K-1 the selected chunks, K..K+nl-1 the chunks of its local window [l(i), i] (Sec. 2.1:
+// l(i) is chunk-aligned, so the window is whole chunks plus the causal part of the token's own chunk).  Every
+// local chunk is attended like a selected one, with its own softmax; its chunk mass is the exact log-sum-exp of
+// its scores, so the softmax over all slots' masses reproduces the single softmax over the window (Eq. chunk mass).
+__host__ __device__ inline int max_local_slots(int W) { return (W - 1 + kS - 1) / kS + 1; }
 __device__ __forceinline__ int slot_chunk(const PArgs& a, int pair, int tok, int slot) {
-    if (slot == a.s.K) return tok / kS;
+    if (slot >= a.s.K) {
+        const int c = local_lo(tok, a.s.W, kS) / kS + (slot - a.s.K);
+        return c <= tok / kS ? c : -1;
+    }
     return a.sel[(static_cast<long long>(pair) * a.s.R + tok) * a.s.K + slot];
 }
 
 __global__ void invert_count_kernel(const PArgs a) {
     const Shape& s = a.s;
-    const int K1 = s.K + 1, pairs = s.B * s.Hkv;
+    const int K1 = s.K + max_local_slots(s.W), pairs = s.B * s.Hkv;
     const long long total = static_cast<long long>(pairs) * s.R * K1;
     for (long long x = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; x < total;
          x += static_cast<long long>(gridDim.x) * blockDim.x) {
@@ -328,7 +335,7 @@ __global__ void __launch_bounds__(1024) invert_scan_kernel(const PArgs a) {
 
 __global__ void invert_fill_kernel(const PArgs a) {
     const Shape& s = a.s;
-    const int K1 = s.K + 1, pairs = s.B * s.Hkv;
+    const int K1 = s.K + max_local_slots(s.W), pairs = s.B * s.Hkv;
     const long long total = static_cast<long long>(pairs) * s.R * K1;
     for (long long x = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; x < total;
          x += static_cast<long long>(gridDim.x) * blockDim.x) {
@@ -353,13 +360,14 @@ __global__ void invert_fill_kernel(const PArgs a) {
 // 4 heads are 1 KB contiguous (two 16-byte loads per lane); lane l covers head l/16 (and head 2 + l/16),
 // elements 8*(l%16)..+7.
 constexpr int kFuseWarps = 4;
+constexpr int kFuseRows = 96;             // rows mixed per token: K <= 64 selected + up to 16 local chunks, 3 x 32 lanes
 
 __global__ void __launch_bounds__(kFuseWarps * 32) prefill_fuse_kernel(const PArgs a) {
-    __shared__ float wsm[kFuseWarps][kG][68];
-    __shared__ int esm[kFuseWarps][68];
+    __shared__ float wsm[kFuseWarps][kG][kFuseRows];
+    __shared__ int esm[kFuseWarps][kFuseRows];
     const Shape& s = a.s;
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
-    const int K = s.K, K1 = K + 1, nblk = a.i1 - a.i0;
+    const int K = s.K, K1 = K + max_local_slots(s.W), nblk = a.i1 - a.i0;
     const long long total = static_cast<long long>(s.B) * s.Hkv * nblk;
     const long long w = static_cast<long long>(blockIdx.x) * kFuseWarps + wib;
     if (w >= total) return;
@@ -367,32 +375,41 @@ __global__ void __launch_bounds__(kFuseWarps * 32) prefill_fuse_kernel(const PAr
     const int pair = static_cast<int>(w / nblk);
     const int b = pair / s.Hkv, gk = pair % s.Hkv;
     const int tok = a.i0 + il;
-    const int nsel = min(K, tok / kS);               // W = 1: a token of chunk ci has ci candidates
+    // rows to mix: the selected chunks (slots 0..nsel-1), then the chunks of the local window (slots K..K+nl-1)
+    const int lc = local_lo(tok, s.W, kS) / kS;      // first local chunk = number of candidate chunks
+    const int nsel = min(K, lc);
+    const int nl = tok / kS - lc + 1;
+    const int nrows = nsel + nl;
     const int e0 = a.blk_toff[a.blk] * a.tile_tok;   // first entry of this query block
     const int* ep = a.epos + (static_cast<long long>(pair) * s.R + tok) * K1;
     const float4* lam4 = reinterpret_cast<const float4*>(a.lam);
-    float (*wv)[68] = wsm[wib];
+    float (*wv)[kFuseRows] = wsm[wib];
     int* ev = esm[wib];
-    // entry (relative to the block) and the four heads' chunk masses of slots lane, lane + 32 and the local slot
-    const int en0 = lane < nsel ? ep[lane] - e0 : 0, en1 = lane + 32 < nsel ? ep[lane + 32] - e0 : 0;
-    const int enl = ep[K] - e0;
-    const float4 ninf = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
-    const float4 v0 = lane < nsel ? lam4[en0] : ninf, v1 = lane + 32 < nsel ? lam4[en1] : ninf, vl = lam4[enl];
-    if (lane < nsel) ev[lane] = en0;
-    if (lane + 32 < nsel) ev[lane + 32] = en1;
-    if (lane == 0) ev[64] = enl;
-    const float l0s[kG] = {v0.x, v0.y, v0.z, v0.w}, l1s[kG] = {v1.x, v1.y, v1.z, v1.w}, lls[kG] = {vl.x, vl.y, vl.z, vl.w};
+    // entry (relative to the block) and the four heads' chunk masses of rows lane, lane + 32, lane + 64
+    float lam[3][kG];
+#pragma unroll
+    for (int st = 0; st < 3; ++st) {
+        const int r = lane + 32 * st;
+        float4 v = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+        if (r < nrows) {
+            const int en = ep[r < nsel ? r : K + (r - nsel)] - e0;
+            ev[r] = en;
+            v = lam4[en];
+        }
+        lam[st][0] = v.x; lam[st][1] = v.y; lam[st][2] = v.z; lam[st][3] = v.w;
+    }
     float lse_h = 0.f;
 #pragma unroll
     for (int h = 0; h < kG; ++h) {
-        const float l0 = l0s[h], l1 = l1s[h], ll = lls[h];
-        const float Mx = warp_max(fmaxf(fmaxf(l0, l1), ll));
-        const float e0x = __expf(l0 - Mx), e1x = __expf(l1 - Mx), el = __expf(ll - Mx);
-        const float D = warp_sum(e0x + e1x) + el;
+        const float Mx = warp_max(fmaxf(fmaxf(lam[0][h], lam[1][h]), lam[2][h]));
+        float ex[3];
+#pragma unroll
+        for (int st = 0; st < 3; ++st) ex[st] = __expf(lam[st][h] - Mx);
+        const float D = warp_sum(ex[0] + ex[1] + ex[2]);
         const float inv = 1.f / D;
-        if (lane < nsel) wv[h][lane] = e0x * inv;
-        if (lane + 32 < nsel) wv[h][lane + 32] = e1x * inv;
-        if (lane == 0) wv[h][64] = el * inv;
+#pragma unroll
+        for (int st = 0; st < 3; ++st)
+            if (lane + 32 * st < nrows) wv[h][lane + 32 * st] = ex[st] * inv;
         if (lane == h) lse_h = Mx + __logf(D);
     }
     __syncwarp();
@@ -408,28 +425,21 @@ __global__ void __launch_bounds__(kFuseWarps * 32) prefill_fuse_kernel(const PAr
             acc[2 * x + 1] = fmaf(wgt, __uint_as_float(wd[x] & 0xffff0000u), acc[2 * x + 1]);
         }
     };
-    // local slot first, then the selected slots four at a time (8 loads in flight per lane)
-    {
-        const __nv_bfloat16* row = a.obuf + static_cast<long long>(ev[64]) * kG * kD;
-        const uint4 ra = obuf_load(reinterpret_cast<const uint4*>(row + lane * 8));
-        const uint4 rb = obuf_load(reinterpret_cast<const uint4*>(row + 256 + lane * 8));
-        fma8(accA, ra, wv[hA][64]);
-        fma8(accB, rb, wv[hB][64]);
-    }
-    for (int sl0 = 0; sl0 < nsel; sl0 += 4) {
+    // four rows at a time (8 loads in flight per lane)
+    for (int r0 = 0; r0 < nrows; r0 += 4) {
         uint4 ra[4], rb[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            const int sl = min(sl0 + u, nsel - 1);
-            const __nv_bfloat16* row = a.obuf + static_cast<long long>(ev[sl]) * kG * kD;
+            const int r = min(r0 + u, nrows - 1);
+            const __nv_bfloat16* row = a.obuf + static_cast<long long>(ev[r]) * kG * kD;
             ra[u] = obuf_load(reinterpret_cast<const uint4*>(row + lane * 8));
             rb[u] = obuf_load(reinterpret_cast<const uint4*>(row + 256 + lane * 8));
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            if (sl0 + u < nsel) {
-                fma8(accA, ra[u], wv[hA][sl0 + u]);
-                fma8(accB, rb[u], wv[hB][sl0 + u]);
+            if (r0 + u < nrows) {
+                fma8(accA, ra[u], wv[hA][r0 + u]);
+                fma8(accB, rb[u], wv[hB][r0 + u]);
             }
         }
     }
@@ -478,7 +488,7 @@ Plan make_plan(const Shape& s) {
     for (size_t b = 0; b < nblocks; ++b) {
         const size_t toks = (b + 1) * blk <= static_cast<size_t>(s.R) ? blk : static_cast<size_t>(s.R) - b * blk;
         const size_t vis = ((b * blk + toks) + kS - 1) / kS;
-        const size_t tiles = pairs * (toks * (s.K + 1) / tt + (vis < nc ? vis : nc)) + 1;
+        const size_t tiles = pairs * (toks * (s.K + max_local_slots(s.W)) / tt + (vis < nc ? vis : nc)) + 1;
         all_tiles += tiles;
         max_blk = tiles > max_blk ? tiles : max_blk;
     }
@@ -493,7 +503,7 @@ Plan make_plan(const Shape& s) {
     p.off_seg = take(sizeof(int) * ((nblocks * pairs * nc + 1023) / 1024));
     p.off_off = take(sizeof(int) * nblocks * pairs * nc);
     p.off_entries = take(sizeof(int) * all_tiles * tt);
-    p.off_epos = take(sizeof(int) * pairs * s.R * (s.K + 1));
+    p.off_epos = take(sizeof(int) * pairs * s.R * (s.K + max_local_slots(s.W)));
     p.off_tiles = take(sizeof(int4) * all_tiles);
     p.off_obuf = take(sizeof(__nv_bfloat16) * max_blk * tt * kG * kD);
     p.off_lam = take(sizeof(float) * max_blk * tt * kG);
@@ -504,11 +514,13 @@ Plan make_plan(const Shape& s) {
 }  // namespace
 
 bool prefill_fast_supports(const Shape& s, int dtype) {
-    return dtype == HILS_BF16 && !s.is_decode && s.d == kD && s.S == kS && s.W == 1 && s.Hl == s.Hkv && s.G == kG &&
+    // any window whose chunks fit the fuse kernel's row table; the warp-MMA selection fallback (K > 32) knows W = 1 only
+    return dtype == HILS_BF16 && !s.is_decode && s.d == kD && s.S == kS && s.W >= 1 && max_local_slots(s.W) <= 16 &&
+           (s.W == 1 || (s.K <= 32 && prefill_select_tc_supports(s))) && s.Hl == s.Hkv && s.G == kG &&
            s.K >= 1 && s.K <= 64 && static_cast<long long>(s.B) * s.Hkv * s.T < (1ll << 31) &&
            static_cast<long long>(s.B) * s.Hkv * s.C < (1ll << 24) &&
            static_cast<long long>(s.B) * s.Hkv * ((s.R + kS - 1) / kS) < (1ll << 31) &&
-           static_cast<long long>(s.B) * s.Hkv * s.R * (s.K + 1) < (1ll << 31);
+           static_cast<long long>(s.B) * s.Hkv * s.R * (s.K + max_local_slots(s.W)) < (1ll << 31);
 }
 
 size_t prefill_fast_scratch_bytes(const Shape& s) { return make_plan(s).total; }
@@ -580,7 +592,7 @@ int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
     // and the table of attend tiles, grouped by block
     if (cudaMemsetAsync(sc + p.off_cnt, 0, p.zero_bytes, stream) != cudaSuccess) return HILS_ERR_CUDA;
     {
-        const long long elems = static_cast<long long>(pairs) * s.R * (s.K + 1);
+        const long long elems = static_cast<long long>(pairs) * s.R * (s.K + max_local_slots(s.W));
         const long long want = (elems + 255) / 256;
         const unsigned eb = static_cast<unsigned>(want < 148 * 16 ? want : 148 * 16);
         invert_count_kernel<<<eb, 256, 0, stream>>>(a);

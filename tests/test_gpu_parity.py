@@ -80,6 +80,18 @@ def test_prefill_window_bias_and_per_head_landmarks(impl):
     check_prefill(cfg, inp, out, lse, sel, bias=bias, W=100)
 
 
+@pytest.mark.parametrize("W", [2, 64, 65, 200, 512])
+def test_prefill_fast_path_with_a_chunk_aligned_local_window(W):
+    """The paper's operator form on the tensor-core path: local window W > 1 (Sec. 2.1; the experiments use
+    W = 512), a non-null bias, several query blocks; every chunk of the window is a slot of its own."""
+    cfg = wl.CONFIGS[1].scaled(B=2, Hq=8, Hkv=2, L=4300, K=12, seed=35)
+    fast_or_skip(cfg, False, W=W)
+    inp = wl.make_prefill_inputs(cfg, "cpu")
+    bias = wl.make_bias(cfg, "cpu")
+    out, lse, sel = run_prefill(cfg, inp, "fast", bias=bias, W=W)
+    check_prefill(cfg, inp, out, lse, sel, bias=bias, W=W)
+
+
 @pytest.mark.parametrize("impl", ["generic", "fast"])
 def test_prefill_bias_only(impl):
     cfg = wl.CONFIGS[1].scaled(L=1536, K=6, seed=32)
