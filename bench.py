@@ -59,11 +59,13 @@ def load_peaks():
 
 
 # ----------------------------------------------------------------------------- algorithmic work
-def prefill_flops(cfg):
-    """(gathered FLOP, scoring FLOP) of one prefill call with W = 1."""
+def prefill_flops(cfg, W=1):
+    """(gathered FLOP, scoring FLOP) of one prefill call: per position, QK^T and PV over the min(K, candidates)
+    selected chunks and the local window [l(i), i], l(i) = max(0, floor((i - W + 1) / S)) * S (Sec. 2.1)."""
     i = np.arange(cfg.L, dtype=np.float64)
-    ci = np.floor(i / cfg.S)
-    gathered = 4.0 * cfg.d * (np.minimum(cfg.K, ci) * cfg.S + (i % cfg.S) + 1)
+    lo = np.maximum(0.0, np.floor((i - W + 1) / cfg.S)) * cfg.S
+    ci = lo / cfg.S                                                     # candidate chunks
+    gathered = 4.0 * cfg.d * (np.minimum(cfg.K, ci) * cfg.S + (i - lo) + 1)
     scoring = 2.0 * cfg.d * ci
     return float(gathered.sum()) * cfg.Hq * cfg.B, float(scoring.sum()) * cfg.Hq * cfg.B
 
@@ -137,19 +139,21 @@ def pick_cfg(name):
     return wl.CONFIGS[idx]
 
 
-def params_for(hils, cfg, decode, impl="auto"):
+def params_for(hils, cfg, decode, impl="auto", window=1):
     return hils.make_params(B=cfg.B, Hq=cfg.Hq, Hkv=cfg.Hkv, Hl=cfg.Hkv, L=0 if decode else cfg.L, T_max=cfg.L,
-                            C=cfg.C, d=cfg.d, chunk_size=cfg.S, top_k=cfg.K, window=1,
+                            C=cfg.C, d=cfg.d, chunk_size=cfg.S, top_k=cfg.K, window=window,
                             dtype=0 if cfg.dtype == "f32" else 1, impl=impl)
 
 
 class Workload:
     """Device-resident inputs/outputs of one configuration and the call that runs one step."""
 
-    def __init__(self, hils, cfg, device, n_query_sets=8):
+    def __init__(self, hils, cfg, device, n_query_sets=8, window=1, with_bias=False):
         self.hils, self.cfg, self.dev = hils, cfg, device
         self.decode = cfg.mode == "decode"
-        self.p = params_for(hils, cfg, self.decode)
+        self.window = window                     # prefill only; > 1 = the paper's operator form (Sec. 2.1)
+        self.bias = wl.make_bias(cfg, device) if with_bias else None
+        self.p = params_for(hils, cfg, self.decode, window=window)
         self.ws = hils.alloc_workspace(self.p, self.decode, device)
         if self.decode:
             self.inp = wl.make_decode_inputs(cfg, device)
@@ -168,7 +172,7 @@ class Workload:
             self.out = torch.empty_like(self.inp["q"])
             self.lse = torch.empty((cfg.B, cfg.Hq, cfg.L), dtype=torch.float32, device=device)
             self.sel = torch.empty((cfg.B, cfg.Hkv, cfg.L, cfg.K), dtype=torch.int32, device=device)
-            self.work, self.work_aux = prefill_flops(cfg)
+            self.work, self.work_aux = prefill_flops(cfg, window)
             self.unit, self.metric = "TFLOP/s", "hils_prefill_effective_TFLOPs"
         # L2 flush between decode steps: write 256 MB, then read another 256 MB so that the timed kernels
         # start from an L2 full of clean lines (dirty lines would be written back under them)
@@ -184,8 +188,8 @@ class Workload:
             self.hils.hils_decode(q, i["k"], i["v"], i["landmarks"], i["seq_lens"], self.cfg.S, self.cfg.K,
                                   out=self.out, lse=self.lse, sel_idx=self.sel, workspace=self.ws)
         else:
-            self.hils.hils_prefill(i["q"], i["k"], i["v"], i["landmarks"], self.cfg.S, self.cfg.K,
-                                   out=self.out, lse=self.lse, sel_idx=self.sel, workspace=self.ws)
+            self.hils.hils_prefill(i["q"], i["k"], i["v"], i["landmarks"], self.cfg.S, self.cfg.K, bias=self.bias,
+                                   window=self.window, out=self.out, lse=self.lse, sel_idx=self.sel, workspace=self.ws)
 
     def between_steps(self):
         if self.flush is not None:
@@ -540,6 +544,18 @@ def main():
                     extras["landmark_summary_" + name] = bench_landmark_summary(hils, ew, peaks)
                     launches += 13
                 del ew
+                if name == "cfg2":
+                    # the paper's operator form (Sec. 2.1 / experiments): local window W = 512 and a non-null bias
+                    torch.cuda.empty_cache()
+                    pw = Workload(hils, pick_cfg(name), dev, window=512, with_bias=True)
+                    pms, _ = time_steps(pw, max(3, args.steps), 3, barrier)
+                    pk = kernel_times(pw, 3, barrier)
+                    extras["cfg2_window512_bias"] = {
+                        "metric": pw.metric, "value": pw.rate(float(np.mean(pms)) * 1e-3), "unit": pw.unit,
+                        "ms_per_step": float(np.mean(pms)), "kernel_ms": pk, "window": 512, "bias": True,
+                        "frac_of_measured_bf16_burst": pw.rate(float(np.mean(pms)) * 1e-3) / peaks["bf16_tflops"]}
+                    launches += hils.last_launch_count() * (max(3, args.steps) + 6)
+                    del pw
                 torch.cuda.empty_cache()
             except Exception as exc:  # keep the primary line even if an extra fails
                 extras[name] = {"error": repr(exc)}
