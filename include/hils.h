@@ -116,7 +116,7 @@ int hils_decode(const hils_params* params, const void* q, const void* k_cache, c
  *  - Limit: 256 + hils_workspace_bytes(params, 1) must fit in 8 MiB, otherwise HILS_ERR_WORKSPACE is
  *    returned before anything is launched (both benchmark decode shapes fit: B=64 x 64K tokens with
  *    K=32 needs about 5.3 MiB, B=4 x 1M tokens with K=64 about 2.5 MiB).  Shapes outside the
- *    bandwidth-tuned decode kernels (bf16, d=128, chunk 64, window 1, one landmark per KV head,
+ *    bandwidth-tuned decode kernels (bf16, d=128, chunk 64, window <= 897, one landmark per KV head,
  *    at most 8 query heads per KV head) return HILS_ERR_UNSUPPORTED.
  *  - The first call on each device looks up the array's device address (with that device current);
  *    make that first call outside any stream capture.

@@ -1,4 +1,5 @@
-// Bandwidth-tuned decode kernels: bf16, d = 128, S = 64, G <= 8, one landmark per KV head, W = 1.
+// Bandwidth-tuned decode kernels: bf16, d = 128, S = 64, G <= 8, one landmark per KV head, any local window of
+// up to 16 chunks (W <= 897).
 //
 //   decode_score   streams the landmarks of every (sequence, KV head) once with 128-bit loads and
 //                  scores them against the G query heads with warp MMA (landmark rows are the A
@@ -49,11 +50,18 @@ struct DArgs {
     int* pair_n;       // [pairs]       number of selected chunks, -1 = invalid sequence length
     int* done;         // [pairs]       slots finished (zeroed by the selection)
     float* part;       // [pairs, max_parts, G, 128] weighted partial sums
-    float* loc_o;      // [pairs, G, 128] local-branch output
-    float* loc_lam;    // [pairs, G]      log Z_swa
+    float* loc_o;      // [pairs, NL, G, 128] outputs of the chunks of the local window (NL = max_local_slots(W))
+    float* loc_lam;    // [pairs, NL, G]      their log masses (together: log Z_swa)
     int max_parts;
     int n_ctas;
 };
+
+// The local window [l(i), i] of the query at i = seq_len - 1 (Sec. 2.1) is whole chunks plus the causal part of the
+// query's own chunk: chunks lc .. ci, at most max_local_slots(W) of them.  Each is attended like a selected chunk,
+// with its own softmax; its mass is the exact log-sum-exp of its scores, so mixing by the masses reproduces the
+// single softmax over the window (Eq. chunk mass).  Candidates for selection are the chunks 0 .. lc - 1.
+__host__ __device__ inline int max_local_slots(int W) { return (W - 1 + kS - 1) / kS + 1; }
+__device__ __forceinline__ int first_local_chunk(int seq, int W) { return local_lo(seq - 1, W, kS) / kS; }
 
 // ------------------------------------------------------------------------------------------ select
 // Exact top-K as a tree of warp-level selections.  A warp stages up to kSelCap candidates (ordered score
@@ -375,7 +383,7 @@ __global__ void __launch_bounds__(kScoreThreads) decode_score_kernel(const DArgs
     const int b = pair / s.Hkv, g = pair % s.Hkv;
     const int seq = a.seq_lens[b];
     if (seq < 1 || seq > s.T) return;
-    const int ncand = (seq - 1) / kS;
+    const int ncand = first_local_chunk(seq, s.W);
     const int c_begin = blockIdx.x * kScoreChunksPerCta;
     if (c_begin >= ncand) return;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -454,7 +462,7 @@ __global__ void __launch_bounds__(512) decode_select_kernel(const DArgs a) {
         return;
     }
     pdl_wait();                                        // group scores of decode_score are visible
-    select_pair(a, pair, (seq - 1) / kS, sh, sel_dyn, nt >> 5);
+    select_pair(a, pair, first_local_chunk(seq, s.W), sh, sel_dyn, nt >> 5);
     pdl_launch_dependents();
 }
 
@@ -482,7 +490,7 @@ decode_attend_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
     AttendSmem& sm = *reinterpret_cast<AttendSmem*>(ring + kStages * kStageBytes);
     const Shape& s = a.s;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int K = s.K, G = s.G, slots = K + 1;
+    const int K = s.K, G = s.G, NL = max_local_slots(s.W), slots = K + NL;
     const long long N = static_cast<long long>(s.B) * s.Hkv * slots;
     const long long lo = (static_cast<long long>(blockIdx.x) * N) / a.n_ctas;
     const long long hi = (static_cast<long long>(blockIdx.x + 1) * N) / a.n_ctas;
@@ -505,9 +513,12 @@ decode_attend_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
             if (slot < K) {
                 c = slot < n ? a.sel[static_cast<long long>(pair) * K + slot] : -1;
             } else {
+                // slot K + r: chunk lc + r of the local window; only the query's own chunk can be partial
                 const int seq = a.seq_lens[pair / s.Hkv];
-                c = (seq - 1) / kS;
-                nv = (seq - 1) % kS + 1;
+                const int ci = (seq - 1) / kS;
+                c = first_local_chunk(seq, s.W) + (slot - K);
+                if (c > ci) c = -1;
+                else if (c == ci) nv = (seq - 1) % kS + 1;
             }
         }
         sm.item_chunk[j] = c;
@@ -643,11 +654,11 @@ decode_attend_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
                     for (int i = 0; i < 16; ++i) ol[i][0] = ol[i][1] = ol[i][2] = ol[i][3] = 0.f;
                     pv_tile(sc, vs_addr, lane, ol);
                     if (gq < G) {
-                        float* dst = a.loc_o + (static_cast<long long>(pair) * G + gq) * kD;
+                        float* dst = a.loc_o + ((static_cast<long long>(pair) * NL + (slot - K)) * G + gq) * kD;
 #pragma unroll
                         for (int i = 0; i < 16; ++i)
                             *reinterpret_cast<float2*>(dst + i * 8 + 2 * t) = make_float2(ol[i][0], ol[i][1]);
-                        if (t == 0) a.loc_lam[pair * G + gq] = m * s.scale + __logf(z);
+                        if (t == 0) a.loc_lam[(pair * NL + (slot - K)) * G + gq] = m * s.scale + __logf(z);
                     }
                     if (nv < kS) fence_proxy_async_smem();
                 }
@@ -689,25 +700,35 @@ decode_attend_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
             __threadfence();
             const int last_cta = cta_of_item(pair_end - 1, N, a.n_ctas);
             const int nparts = min(a.max_parts, last_cta - first_cta + 1);
+            const int seq_b = a.seq_lens[b];
+            const int nl = (seq_b - 1) / kS - first_local_chunk(seq_b, s.W) + 1;
             for (int x = tid; x < G * kD; x += kConsumerWarps * 32) {
                 const int h = x / kD;
                 float A = 0.f;
                 const float* src = a.part + static_cast<long long>(pair) * a.max_parts * G * kD + x;
                 for (int pidx = 0; pidx < nparts; ++pidx) A += __ldcg(src + static_cast<long long>(pidx) * G * kD);
-                const float lam_loc = __ldcg(a.loc_lam + pair * G + h);
-                const float ol = __ldcg(a.loc_o + static_cast<long long>(pair) * G * kD + x);
-                float res, lse;
-                if (n_sel == 0) {
-                    res = ol;
-                    lse = lam_loc;
-                } else {
-                    const float R = a.Rh[pair * G + h], E = a.Eh[pair * G + h];
-                    const float Rp = fmaxf(lam_loc, R);
-                    const float wl = __expf(lam_loc - Rp), ws = __expf(R - Rp);
-                    const float den = wl + ws * E;
-                    res = (wl * ol + ws * A) / den;
-                    lse = Rp + __logf(den);
+                // selected part first, then the chunks of the local window (masses lam_r, outputs o_r) folded in
+                // one at a time with a running maximum (fixed order: deterministic)
+                float Mx = -INFINITY, den = 0.f, num = 0.f;
+                if (n_sel > 0) {
+                    Mx = a.Rh[pair * G + h];
+                    den = a.Eh[pair * G + h];
+                    num = A;
                 }
+                const float* lam_p = a.loc_lam + pair * NL * G + h;
+                const float* o_p = a.loc_o + static_cast<long long>(pair) * NL * G * kD + x;
+#pragma unroll 2
+                for (int r = 0; r < nl; ++r) {
+                    const float lam = __ldcg(lam_p + r * G);
+                    const float ol = __ldcg(o_p + static_cast<long long>(r) * G * kD);
+                    const float nm = fmaxf(Mx, lam);
+                    const float f = __expf(Mx - nm), wl = __expf(lam - nm);
+                    den = fmaf(den, f, wl);
+                    num = fmaf(num, f, wl * ol);
+                    Mx = nm;
+                }
+                const float res = num / den;
+                const float lse = Mx + __logf(den);
                 const long long orow = static_cast<long long>(b) * s.Hq + g * G + h;
                 a.out[orow * kD + (x % kD)] = __float2bfloat16_rn(res);
                 if ((x % kD) == 0) a.lse[orow] = lse;
@@ -738,14 +759,15 @@ int sm_count() {
 Plan make_plan(const Shape& s, int n_sm) {
     Plan p;
     const long long pairs = static_cast<long long>(s.B) * s.Hkv;
-    const long long N = pairs * (s.K + 1);
+    const int slots = s.K + max_local_slots(s.W);
+    const long long N = pairs * slots;
     long long ctas = n_sm;
     if ((N + ctas - 1) / ctas + 1 > kMaxItems) ctas = (N + kMaxItems - 2) / (kMaxItems - 1);
     if (ctas > N) ctas = N;
     p.n_ctas = static_cast<int>(ctas);
     const long long per = N / ctas;                               // every CTA gets per or per+1 items
-    p.max_parts = static_cast<int>((s.K + 1 + per - 1) / per) + 1;
-    if (p.max_parts > s.K + 1) p.max_parts = s.K + 1;
+    p.max_parts = static_cast<int>((slots + per - 1) / per) + 1;
+    if (p.max_parts > slots) p.max_parts = slots;
     p.Cpad = (s.C + 63) / 64 * 64;
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = (off + bytes + 255) / 256 * 256; return o; };
@@ -756,8 +778,8 @@ Plan make_plan(const Shape& s, int n_sm) {
     p.off_n = take(sizeof(int) * pairs);
     p.off_done = take(sizeof(int) * pairs);
     p.off_part = take(sizeof(float) * pairs * p.max_parts * s.G * kD);
-    p.off_loco = take(sizeof(float) * pairs * s.G * kD);
-    p.off_loclam = take(sizeof(float) * pairs * s.G);
+    p.off_loco = take(sizeof(float) * pairs * max_local_slots(s.W) * s.G * kD);
+    p.off_loclam = take(sizeof(float) * pairs * max_local_slots(s.W) * s.G);
     p.total = off;
     return p;
 }
@@ -765,7 +787,7 @@ Plan make_plan(const Shape& s, int n_sm) {
 }  // namespace
 
 bool decode_fast_supports(const Shape& s, int dtype) {
-    return dtype == HILS_BF16 && s.is_decode && s.d == kD && s.S == kS && s.W == 1 && s.Hl == s.Hkv && s.G <= 8 &&
+    return dtype == HILS_BF16 && s.is_decode && s.d == kD && s.S == kS && s.W >= 1 && max_local_slots(s.W) <= 16 && s.Hl == s.Hkv && s.G <= 8 &&
            s.K >= 1 && s.K <= 128 && static_cast<long long>(s.B) * s.Hkv * s.T < (1ll << 31) &&
            static_cast<long long>(s.B) * s.Hkv <= 65535;
 }

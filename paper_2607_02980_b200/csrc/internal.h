@@ -42,7 +42,7 @@ size_t decode_fast_scratch_bytes(const Shape& s);
 int launch_decode_noalloc(const Shape& s, const Tensors& t, int32_t* device_status, cudaStream_t stream);
 size_t decode_noalloc_capacity();
 
-// tcgen05 scoring + top-K for prefill (bf16, d = 128, S = 64, G = 4, W = 1, K <= 32).
+// tcgen05 scoring + top-K for prefill (bf16, d = 128, S = 64, G = 4, K <= 32, any W).
 bool prefill_select_tc_supports(const Shape& s);
 int launch_prefill_select_tc(const Shape& s, const void* q, const void* landmarks, const float* bias, int32_t* sel,
                              int* status, cudaStream_t stream);

@@ -189,6 +189,19 @@ def test_decode_ties_and_clustered_scores_pick_the_lower_chunk_ids(L):
                 assert got[0, g].tolist() == expect, (impl, L, g)
 
 
+@pytest.mark.parametrize("W", [2, 64, 65, 200, 512])
+def test_decode_fast_path_with_a_chunk_aligned_local_window(W):
+    """The paper's operator form in decode: local window W > 1 (the experiments use W = 512) and a bias; the
+    chunks of the window are extra slots of the persistent attend kernel, mixed by their exact masses."""
+    cfg = wl.CONFIGS[3].scaled(B=6, L=4096, K=8, seed=48)
+    fast_or_skip(cfg, True, W=W)
+    seq = [4096, 4095, 1, 63, 2049, 640]
+    inp = wl.make_decode_inputs(cfg, "cpu", seq_lens=torch.tensor(seq, dtype=torch.int32))
+    bias = wl.make_bias(cfg, "cpu")
+    out, lse, sel = run_decode(cfg, inp, "fast", bias=bias, W=W)
+    check_decode(cfg, inp, out, lse, sel, bias=bias, W=W)
+
+
 def test_decode_invalid_seq_len_sets_status_without_fault():
     cfg = wl.CONFIGS[3].scaled(B=2, L=1024, K=4, seed=46)
     inp = wl.make_decode_inputs(cfg, "cpu", seq_lens=torch.tensor([1024, 512], dtype=torch.int32))
