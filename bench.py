@@ -286,6 +286,40 @@ def roofline_for(w, kernel_ms, peaks):
                 algorithmic_flops=algo)
 
 
+def bench_paged_decode(hils, w, peaks, iters=10):
+    """The decode workload again through hils_decode_paged: the same caches cut into pages of one chunk each,
+    shuffled (a random block table).  Same algorithmic bytes as the contiguous run."""
+    cfg, i = w.cfg, w.inp
+    B, Hkv, T, d = i["k"].shape
+    C, S = T // cfg.S, cfg.S
+    gen = torch.Generator(device=i["k"].device).manual_seed(991)
+    perm = torch.randperm(B * C, generator=gen, device=i["k"].device)
+    table = perm.reshape(B, C).to(torch.int32)
+
+    def pages(x):
+        src = x.view(B, Hkv, C, S, d).permute(0, 2, 1, 3, 4).reshape(B * C, Hkv, S, d)
+        out = torch.empty_like(src)
+        out[perm] = src                        # page perm[b*C + c] holds chunk c of sequence b
+        return out
+
+    kp, vp = pages(i["k"]), pages(i["v"])
+    ms = []
+    for it in range(iters + 3):
+        q = w.queries[it % len(w.queries)]
+        w.between_steps()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        hils.hils_decode_paged(q, kp, vp, i["landmarks"], table, i["seq_lens"], cfg.S, cfg.K, out=w.out, lse=w.lse,
+                               sel_idx=w.sel, workspace=w.ws)
+        e1.record()
+        torch.cuda.synchronize()
+        if it >= 3:
+            ms.append(e0.elapsed_time(e1))
+    m = float(np.mean(ms))
+    return {"metric": w.metric, "value": w.rate(m * 1e-3), "unit": w.unit, "ms_per_step": m,
+            "frac_of_measured_hbm": w.rate(m * 1e-3) / peaks["hbm_gbs"], "pages": int(B * C), "page_tokens": S}
+
+
 def bench_landmark_summary(hils, w, peaks, iters=10):
     """The chunk-summary kernel (Proposition 3.1) on the workload's K tensor: every chunk of every KV head once.
     HBM-bound; algorithmic bytes = K read once + the learnable queries read + the summaries written."""
@@ -543,6 +577,9 @@ def main():
                 if name in ("cfg2", "cfg3"):
                     extras["landmark_summary_" + name] = bench_landmark_summary(hils, ew, peaks)
                     launches += 13
+                if name == "cfg3":
+                    extras["cfg3_paged"] = bench_paged_decode(hils, ew, peaks)
+                    launches += 3 * 13
                 del ew
                 if name == "cfg2":
                     # the paper's operator form (Sec. 2.1 / experiments): local window W = 512 and a non-null bias

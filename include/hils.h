@@ -130,6 +130,20 @@ int hils_decode_noalloc(const hils_params* params, const void* q, const void* k_
                         const void* landmarks, const float* bias, const int32_t* seq_lens,
                         void* out, float* lse, int32_t* sel_idx, int32_t* device_status, void* stream);
 
+/* hils_decode over PAGED caches with page = chunk (the serving layout of Sec. 7.1: one KV page per chunk).
+ * Same operator, same outputs as hils_decode; only the addressing of K and V differs:
+ *   k_pages, v_pages [num_pages, Hkv, S, d]  DEVICE: page p holds S consecutive tokens of one sequence for all KV heads
+ *   block_table      [B, C] int32 DEVICE: page of logical chunk c of sequence b (read for the chunks that are
+ *                    attended: c <= (seq_lens[b]-1)/S); params->C is its row length, params->T_max = C * S
+ *   landmarks, bias  stay logical: [B, Hl, C, d] / [B, Hl, C]
+ * A page id outside [0, num_pages) sets the device status to HILS_ERR_DEVICE_INDEX and the chunk is skipped.
+ * Supported by the bandwidth-tuned decode kernels only (bf16, d = 128, S = 64, one landmark per KV head, at most 8
+ * query heads per KV head); other shapes return HILS_ERR_UNSUPPORTED.  Workspace as for hils_decode. */
+int hils_decode_paged(const hils_params* params, const void* q, const void* k_pages, const void* v_pages,
+                      const void* landmarks, const float* bias, const int32_t* block_table, int32_t num_pages,
+                      const int32_t* seq_lens, void* out, float* lse, int32_t* sel_idx, void* workspace,
+                      size_t workspace_bytes, void* stream);
+
 /* Chunk summaries -- the step upstream of the operator (Proposition 3.1, Eq. LogSumExp linearization /
  * Eq. prop_q_c).  For every sequence b, landmark head hl (its KV head is hl / (Hl / Hkv)) and chunk
  * c in [chunk_begin, chunk_begin + chunk_count), with the chunk's keys k_j, j in [c*S, min((c+1)*S, len_b))

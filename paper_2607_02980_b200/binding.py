@@ -24,7 +24,7 @@ EXPORTS = [
     "hils_workspace_bytes", "hils_prefill", "hils_decode", "hils_host_arena_bytes",
     "hils_prefill_host", "hils_decode_host", "hils_poll_status", "hils_last_launch_count",
     "hils_status_string", "hils_version", "hils_trace_enable", "hils_trace_read", "hils_decode_noalloc",
-    "hils_landmark_summary",
+    "hils_landmark_summary", "hils_decode_paged",
 ]
 
 
@@ -70,6 +70,9 @@ def load_library() -> ctypes.CDLL:
     lib.hils_decode_host.argtypes = [pp, vp, vp, vp, vp, f32p, i32p, vp, f32p, i32p, vp, ctypes.c_size_t, vp]
     lib.hils_decode_noalloc.restype = ctypes.c_int
     lib.hils_decode_noalloc.argtypes = [pp, vp, vp, vp, vp, f32p, i32p, vp, f32p, i32p, i32p, vp]
+    lib.hils_decode_paged.restype = ctypes.c_int
+    lib.hils_decode_paged.argtypes = [pp, vp, vp, vp, vp, f32p, i32p, ctypes.c_int32, i32p, vp, f32p, i32p, vp,
+                                      ctypes.c_size_t, vp]
     lib.hils_landmark_summary.restype = ctypes.c_int
     lib.hils_landmark_summary.argtypes = [pp, vp, vp, i32p, ctypes.c_int32, ctypes.c_int32, vp, f32p, vp]
     lib.hils_poll_status.restype = ctypes.c_int
@@ -250,6 +253,37 @@ def hils_decode_noalloc(q, k_cache, v_cache, landmarks, seq_lens, chunk_size: in
                                  _ptr(device_status), _stream_ptr(stream))
     if rc != 0:
         raise HilsError(rc, "hils_decode_noalloc")
+    return out, lse, sel_idx
+
+
+def hils_decode_paged(q, k_pages, v_pages, landmarks, block_table, seq_lens, chunk_size: int, top_k: int, stream=None, *,
+                      bias=None, window: int = 1, scale: float = 0.0, out=None, lse=None, sel_idx=None, workspace=None):
+    """hils_decode over paged caches with page = chunk: k_pages, v_pages [num_pages, Hkv, S, d], block_table [B, C]
+    int32 (page of every logical chunk); landmarks / bias stay logical.  Returns (out, lse, sel_idx)."""
+    lib = load_library()
+    B, Hq, d = q.shape
+    P, Hkv, S, _ = k_pages.shape
+    Hl, C = landmarks.shape[1], landmarks.shape[2]
+    dt = q.dtype
+    _check(q, "q", (B, Hq, d), dt, True)
+    _check(k_pages, "k_pages", (P, Hkv, chunk_size, d), dt, True)
+    _check(v_pages, "v_pages", (P, Hkv, chunk_size, d), dt, True)
+    _check(landmarks, "landmarks", (B, Hl, C, d), dt, True)
+    _check(block_table, "block_table", (B, C), torch.int32, True)
+    _check(seq_lens, "seq_lens", (B,), torch.int32, True)
+    if bias is not None:
+        _check(bias, "bias", (B, Hl, C), torch.float32, True)
+    p = make_params(B=B, Hq=Hq, Hkv=Hkv, Hl=Hl, L=0, T_max=C * chunk_size, C=C, d=d, chunk_size=chunk_size,
+                    top_k=top_k, window=window, scale=scale, dtype=_dtype_code(q), impl="auto")
+    ws = alloc_workspace(p, True, q.device) if workspace is None else workspace
+    out = torch.empty((B, Hq, d), dtype=dt, device=q.device) if out is None else out
+    lse = torch.empty((B, Hq), dtype=torch.float32, device=q.device) if lse is None else lse
+    sel_idx = torch.empty((B, Hkv, top_k), dtype=torch.int32, device=q.device) if sel_idx is None else sel_idx
+    rc = lib.hils_decode_paged(ctypes.byref(p), _ptr(q), _ptr(k_pages), _ptr(v_pages), _ptr(landmarks), _ptr(bias),
+                               _ptr(block_table), int(P), _ptr(seq_lens), _ptr(out), _ptr(lse), _ptr(sel_idx),
+                               _ptr(ws), ws.numel() * ws.element_size(), _stream_ptr(stream))
+    if rc != 0:
+        raise HilsError(rc, "hils_decode_paged")
     return out, lse, sel_idx
 
 

@@ -100,7 +100,7 @@ size_t scratch_bytes(const Shape& s, Path path) {
 
 int run(const hils_params* p, int is_decode, const void* q, const void* k, const void* v, const void* lm,
         const float* bias, const int32_t* seq_lens, void* out, float* lse, int32_t* sel, void* ws,
-        size_t ws_bytes, void* stream_v) {
+        size_t ws_bytes, void* stream_v, const int32_t* block_table = nullptr, int num_pages = 0) {
     g_last_launches = 0;
     Shape s;
     int rc = make_shape(p, is_decode, &s);
@@ -113,11 +113,19 @@ int run(const hils_params* p, int is_decode, const void* q, const void* k, const
     Path path;
     rc = pick_path(s, p, &path);
     if (rc != HILS_OK) return rc;
+    if (block_table) {
+        // paged caches: only the TMA decode kernels address K / V through a page table
+        if (path != Path::DecodeFast) return HILS_ERR_UNSUPPORTED;
+        if (num_pages < 1 || static_cast<long long>(num_pages) * s.Hkv * s.S >= (1ll << 31)) return HILS_ERR_INVALID_ARG;
+        if (reinterpret_cast<uintptr_t>(block_table) & 3u) return HILS_ERR_ALIGNMENT;
+    }
     const size_t need = kStatusBytes + scratch_bytes(s, path);
     if (!ws || ws_bytes < need) return HILS_ERR_WORKSPACE;
     if (!aligned16(ws)) return HILS_ERR_ALIGNMENT;
     Tensors t{q, k, v, lm, bias, seq_lens, out, lse, sel, static_cast<int*>(ws),
               static_cast<char*>(ws) + kStatusBytes, ws_bytes - kStatusBytes};
+    t.block_table = block_table;
+    t.num_pages = num_pages;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     trace_begin(stream);
     int n;
@@ -219,6 +227,15 @@ int hils_decode(const hils_params* params, const void* q, const void* k_cache, c
                 int32_t* sel_idx, void* workspace, size_t workspace_bytes, void* stream) {
     return run(params, 1, q, k_cache, v_cache, landmarks, bias, seq_lens, out, lse, sel_idx, workspace,
                workspace_bytes, stream);
+}
+
+int hils_decode_paged(const hils_params* params, const void* q, const void* k_pages, const void* v_pages,
+                      const void* landmarks, const float* bias, const int32_t* block_table, int32_t num_pages,
+                      const int32_t* seq_lens, void* out, float* lse, int32_t* sel_idx, void* workspace,
+                      size_t workspace_bytes, void* stream) {
+    if (!block_table) return HILS_ERR_INVALID_ARG;
+    return run(params, 1, q, k_pages, v_pages, landmarks, bias, seq_lens, out, lse, sel_idx, workspace, workspace_bytes,
+               stream, block_table, num_pages);
 }
 
 int hils_decode_noalloc(const hils_params* params, const void* q, const void* k_cache, const void* v_cache,

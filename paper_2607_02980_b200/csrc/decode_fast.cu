@@ -54,6 +54,8 @@ struct DArgs {
     float* loc_lam;    // [pairs, NL, G]      their log masses (together: log Z_swa)
     int max_parts;
     int n_ctas;
+    const int32_t* block_table;   // paged caches: [B, C] page of every logical chunk, or NULL (contiguous caches)
+    int num_pages;
 };
 
 // The local window [l(i), i] of the query at i = seq_len - 1 (Sec. 2.1) is whole chunks plus the causal part of the
@@ -471,7 +473,8 @@ struct AttendSmem {
     uint64_t full[kStages];
     uint64_t empty[kStages];
     int item_chunk[kMaxItems];     // chunk id, or -1 for an empty slot
-    int item_nvalid[kMaxItems];    // valid rows (64, or fewer for the partial local chunk)
+    int item_row[kMaxItems];       // first row of the chunk in the K / V tensor maps
+    uint8_t item_nvalid[kMaxItems];// valid rows (64, or fewer for the partial local chunk)
     float red[kConsumerWarps][8 * kD];
     int flag;
     int dead;                      // a bounded wait ran out: every consumer warp leaves at the next barrier
@@ -521,8 +524,23 @@ decode_attend_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
                 else if (c == ci) nv = (seq - 1) % kS + 1;
             }
         }
+        int row = 0;
+        if (c >= 0) {
+            if (a.block_table) {
+                const int page = a.block_table[static_cast<long long>(pair / s.Hkv) * s.C + c];
+                if (page < 0 || page >= a.num_pages) {       // flag it and skip the chunk
+                    set_status(a.status, kDevBadIndex);
+                    c = -1;
+                } else {
+                    row = (page * s.Hkv + pair % s.Hkv) * kS;
+                }
+            } else {
+                row = pair * s.T + c * kS;
+            }
+        }
         sm.item_chunk[j] = c;
-        sm.item_nvalid[j] = nv;
+        sm.item_row[j] = row;
+        sm.item_nvalid[j] = static_cast<uint8_t>(nv);
     }
     __syncthreads();
     if (nitems == 0) return;
@@ -538,8 +556,7 @@ decode_attend_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
                 }
                 const int c = sm.item_chunk[j];
                 if (c < 0) { mbar_arrive(&sm.full[st]); continue; }
-                const int pair = static_cast<int>((lo + j) / slots);
-                const int row = pair * s.T + c * kS;
+                const int row = sm.item_row[j];
                 uint8_t* dst = ring + st * kStageBytes;
                 mbar_expect_tx(&sm.full[st], kStageBytes);
                 tma_load_2d(dst, &map_k, &sm.full[st], 0, row);
@@ -824,9 +841,11 @@ int launch_decode_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
     a.loc_lam = reinterpret_cast<float*>(sc + p.off_loclam);
     a.max_parts = p.max_parts;
     a.n_ctas = p.n_ctas;
+    a.block_table = t.block_table;
+    a.num_pages = t.num_pages;
 
     CUtensorMap map_k, map_v;
-    const uint64_t rows = static_cast<uint64_t>(pairs) * s.T;
+    const uint64_t rows = t.block_table ? static_cast<uint64_t>(t.num_pages) * s.Hkv * kS : static_cast<uint64_t>(pairs) * s.T;
     if (!make_bf16_2d_map(&map_k, t.k, rows, kD, 64, kS) || !make_bf16_2d_map(&map_v, t.v, rows, kD, 64, kS))
         return HILS_ERR_CUDA;
 

@@ -22,6 +22,10 @@ struct Tensors {
     int* status;               // device status word
     void* scratch;             // workspace past the status block
     size_t scratch_bytes;
+    // paged decode (page = chunk): k, v are [num_pages, Hkv, S, d] and block_table [B, C] maps a sequence's
+    // logical chunk to its page; NULL = contiguous caches
+    const int32_t* block_table = nullptr;
+    int num_pages = 0;
 };
 
 // Optional per-kernel timing: when tracing is on (hils_trace_enable), every launcher calls
