@@ -130,6 +130,20 @@ int hils_decode_noalloc(const hils_params* params, const void* q, const void* k_
                         const void* landmarks, const float* bias, const int32_t* seq_lens,
                         void* out, float* lse, int32_t* sel_idx, int32_t* device_status, void* stream);
 
+/* hils_prefill for a SLICE of a sequence: the L query tokens sit at positions pos0 .. pos0 + L - 1 of sequences
+ * whose caches already hold at least pos0 + L tokens (chunked prefill; with small L, multi-token decode as used by
+ * speculative decoding).  Same operator: query row r is treated exactly like position pos0 + r of hils_prefill.
+ *   q, out   [B, Hq, L, d]      lse [B, Hq, L]      sel_idx [B, Hkv, L, K]
+ *   k, v     [B, Hkv, T, d]     T = params->T_max >= pos0 + L (row j is the token at position j)
+ *   landmarks [B, Hl, C, d], bias [B, Hl, C]: rows of all chunks left of the last query's window
+ * pos0 = 0 with T_max = L is hils_prefill.  The workspace depends on pos0: size it with
+ * hils_prefill_at_workspace_bytes (0 = unsupported or invalid).  Errors as hils_prefill; pos0 < 0 or
+ * pos0 + L > T_max returns HILS_ERR_INVALID_ARG. */
+size_t hils_prefill_at_workspace_bytes(const hils_params* params, int64_t pos0);
+int hils_prefill_at(const hils_params* params, const void* q, const void* k, const void* v, const void* landmarks,
+                    const float* bias, int64_t pos0, void* out, float* lse, int32_t* sel_idx, void* workspace,
+                    size_t workspace_bytes, void* stream);
+
 /* hils_decode over PAGED caches with page = chunk (the serving layout of Sec. 7.1: one KV page per chunk).
  * Same operator, same outputs as hils_decode; only the addressing of K and V differs:
  *   k_pages, v_pages [num_pages, Hkv, S, d]  DEVICE: page p holds S consecutive tokens of one sequence for all KV heads

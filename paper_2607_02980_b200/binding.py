@@ -24,7 +24,7 @@ EXPORTS = [
     "hils_workspace_bytes", "hils_prefill", "hils_decode", "hils_host_arena_bytes",
     "hils_prefill_host", "hils_decode_host", "hils_poll_status", "hils_last_launch_count",
     "hils_status_string", "hils_version", "hils_trace_enable", "hils_trace_read", "hils_decode_noalloc",
-    "hils_landmark_summary", "hils_decode_paged",
+    "hils_landmark_summary", "hils_decode_paged", "hils_prefill_at", "hils_prefill_at_workspace_bytes",
 ]
 
 
@@ -70,6 +70,10 @@ def load_library() -> ctypes.CDLL:
     lib.hils_decode_host.argtypes = [pp, vp, vp, vp, vp, f32p, i32p, vp, f32p, i32p, vp, ctypes.c_size_t, vp]
     lib.hils_decode_noalloc.restype = ctypes.c_int
     lib.hils_decode_noalloc.argtypes = [pp, vp, vp, vp, vp, f32p, i32p, vp, f32p, i32p, i32p, vp]
+    lib.hils_prefill_at.restype = ctypes.c_int
+    lib.hils_prefill_at.argtypes = [pp, vp, vp, vp, vp, f32p, ctypes.c_int64, vp, f32p, i32p, vp, ctypes.c_size_t, vp]
+    lib.hils_prefill_at_workspace_bytes.restype = ctypes.c_size_t
+    lib.hils_prefill_at_workspace_bytes.argtypes = [pp, ctypes.c_int64]
     lib.hils_decode_paged.restype = ctypes.c_int
     lib.hils_decode_paged.argtypes = [pp, vp, vp, vp, vp, f32p, i32p, ctypes.c_int32, i32p, vp, f32p, i32p, vp,
                                       ctypes.c_size_t, vp]
@@ -253,6 +257,37 @@ def hils_decode_noalloc(q, k_cache, v_cache, landmarks, seq_lens, chunk_size: in
                                  _ptr(device_status), _stream_ptr(stream))
     if rc != 0:
         raise HilsError(rc, "hils_decode_noalloc")
+    return out, lse, sel_idx
+
+
+def hils_prefill_at(q, k, v, landmarks, chunk_size: int, top_k: int, pos0: int, stream=None, *, bias=None,
+                    window: int = 1, scale: float = 0.0, impl: str = "auto", out=None, lse=None, sel_idx=None):
+    """hils_prefill for the L query tokens at positions pos0 .. pos0 + L - 1 of sequences whose caches k, v
+    [B,Hkv,T,d] hold at least pos0 + L tokens (chunked prefill / multi-token decode).  Returns (out, lse, sel_idx)."""
+    lib = load_library()
+    B, Hq, L, d = q.shape
+    Hkv, T = k.shape[1], k.shape[2]
+    Hl, C = landmarks.shape[1], landmarks.shape[2]
+    dt = q.dtype
+    _check(q, "q", (B, Hq, L, d), dt, True)
+    _check(k, "k", (B, Hkv, T, d), dt, True)
+    _check(v, "v", (B, Hkv, T, d), dt, True)
+    _check(landmarks, "landmarks", (B, Hl, C, d), dt, True)
+    if bias is not None:
+        _check(bias, "bias", (B, Hl, C), torch.float32, True)
+    p = make_params(B=B, Hq=Hq, Hkv=Hkv, Hl=Hl, L=L, T_max=T, C=C, d=d, chunk_size=chunk_size, top_k=top_k,
+                    window=window, scale=scale, dtype=_dtype_code(q), impl=impl)
+    nbytes = int(lib.hils_prefill_at_workspace_bytes(ctypes.byref(p), int(pos0)))
+    if nbytes == 0:
+        raise HilsError(-2, "hils_prefill_at_workspace_bytes")
+    ws = torch.zeros(nbytes, dtype=torch.uint8, device=q.device)
+    out = torch.empty((B, Hq, L, d), dtype=dt, device=q.device) if out is None else out
+    lse = torch.empty((B, Hq, L), dtype=torch.float32, device=q.device) if lse is None else lse
+    sel_idx = torch.empty((B, Hkv, L, top_k), dtype=torch.int32, device=q.device) if sel_idx is None else sel_idx
+    rc = lib.hils_prefill_at(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(landmarks), _ptr(bias), int(pos0),
+                             _ptr(out), _ptr(lse), _ptr(sel_idx), _ptr(ws), nbytes, _stream_ptr(stream))
+    if rc != 0:
+        raise HilsError(rc, "hils_prefill_at")
     return out, lse, sel_idx
 
 

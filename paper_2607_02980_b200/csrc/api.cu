@@ -41,7 +41,7 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline size_t elem_bytes(int dtype) { return dtype == HILS_F32 ? 4 : 2; }
 
 // Fills `s` from the public parameters; returns a status.
-int make_shape(const hils_params* p, int is_decode, Shape* s) {
+int make_shape(const hils_params* p, int is_decode, Shape* s, long long pos0 = 0) {
     if (!p) return HILS_ERR_INVALID_ARG;
     if (p->B < 1 || p->Hq < 1 || p->Hkv < 1 || p->d < 1 || p->chunk_size < 1 || p->top_k < 1 || p->window < 1)
         return HILS_ERR_INVALID_ARG;
@@ -54,6 +54,7 @@ int make_shape(const hils_params* p, int is_decode, Shape* s) {
     s->d = p->d; s->S = p->chunk_size; s->K = p->top_k; s->W = p->window;
     s->scale = p->scale > 0.f ? p->scale : 1.0f / sqrtf(static_cast<float>(p->d));
     s->is_decode = is_decode;
+    s->pos0 = 0;
     if (is_decode) {
         if (p->T_max < 1) return HILS_ERR_INVALID_ARG;
         s->R = 1;
@@ -62,11 +63,12 @@ int make_shape(const hils_params* p, int is_decode, Shape* s) {
         if (p->L < 1) return HILS_ERR_INVALID_ARG;
         s->R = p->L;
         s->T = p->T_max > 0 ? p->T_max : p->L;
-        if (s->T < p->L) return HILS_ERR_INVALID_ARG;
+        if (pos0 < 0 || pos0 + p->L > s->T) return HILS_ERR_INVALID_ARG;      // the cache holds the queries' tokens
+        s->pos0 = static_cast<int>(pos0);
     }
     s->C = p->C > 0 ? p->C : s->T / s->S;
     // every candidate chunk of the last position must have a landmark row
-    const int last = is_decode ? s->T - 1 : p->L - 1;
+    const int last = is_decode ? s->T - 1 : s->pos0 + p->L - 1;
     const int max_cand = local_lo(last, s->W, s->S) / s->S;
     if (s->C < max_cand) return HILS_ERR_INVALID_ARG;
     return HILS_OK;
@@ -100,10 +102,10 @@ size_t scratch_bytes(const Shape& s, Path path) {
 
 int run(const hils_params* p, int is_decode, const void* q, const void* k, const void* v, const void* lm,
         const float* bias, const int32_t* seq_lens, void* out, float* lse, int32_t* sel, void* ws,
-        size_t ws_bytes, void* stream_v, const int32_t* block_table = nullptr, int num_pages = 0) {
+        size_t ws_bytes, void* stream_v, const int32_t* block_table = nullptr, int num_pages = 0, long long pos0 = 0) {
     g_last_launches = 0;
     Shape s;
-    int rc = make_shape(p, is_decode, &s);
+    int rc = make_shape(p, is_decode, &s, pos0);
     if (rc != HILS_OK) return rc;
     if (!q || !k || !v || !lm || !out || !lse || !sel || (is_decode && !seq_lens)) return HILS_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(lm) || !aligned16(out) ||
@@ -227,6 +229,21 @@ int hils_decode(const hils_params* params, const void* q, const void* k_cache, c
                 int32_t* sel_idx, void* workspace, size_t workspace_bytes, void* stream) {
     return run(params, 1, q, k_cache, v_cache, landmarks, bias, seq_lens, out, lse, sel_idx, workspace,
                workspace_bytes, stream);
+}
+
+int hils_prefill_at(const hils_params* params, const void* q, const void* k, const void* v, const void* landmarks,
+                    const float* bias, int64_t pos0, void* out, float* lse, int32_t* sel_idx, void* workspace,
+                    size_t workspace_bytes, void* stream) {
+    return run(params, 0, q, k, v, landmarks, bias, nullptr, out, lse, sel_idx, workspace, workspace_bytes, stream,
+               nullptr, 0, pos0);
+}
+
+size_t hils_prefill_at_workspace_bytes(const hils_params* params, int64_t pos0) {
+    Shape s;
+    if (make_shape(params, 0, &s, pos0) != HILS_OK) return 0;
+    Path path;
+    if (pick_path(s, params, &path) != HILS_OK) return 0;
+    return kStatusBytes + align_up(scratch_bytes(s, path), 256);
 }
 
 int hils_decode_paged(const hils_params* params, const void* q, const void* k_pages, const void* v_pages,

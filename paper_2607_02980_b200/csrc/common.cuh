@@ -24,6 +24,8 @@ struct Shape {
     int d, S, K, W;
     float scale;
     int is_decode;
+    int pos0;       // prefill: sequence position of query row 0 (rows are the tokens pos0 .. pos0 + R - 1 of a cache
+                    // of T tokens); 0 for a whole-sequence prefill
 };
 
 __host__ __device__ inline int floordiv_i(int a, int b) {

@@ -26,7 +26,7 @@ struct GArgs {
 
 // Position of query row r of sequence b, or -1 if the decode length is invalid.
 __device__ inline int row_position(const GArgs& a, int b, int r) {
-    if (!a.s.is_decode) return r;
+    if (!a.s.is_decode) return a.s.pos0 + r;
     const int n = a.seq_lens[b];
     if (n < 1 || n > a.s.T) return -1;
     return n - 1;

@@ -395,7 +395,7 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                 const int e = sm.tile_ent[ms][tk];
                 const int il = e >> 8, slot = e & 255;
                 const bool local = slot >= s.K;                            // a chunk of the local window: mass = its exact log-sum-exp
-                const int lim = local ? a.i0 + il - c * kS : kS - 1;        // last visible key of the chunk
+                const int lim = local ? s.pos0 + a.i0 + il - c * kS : kS - 1;   // last visible key of the chunk
                 float zi;
                 {
                     float v[64];

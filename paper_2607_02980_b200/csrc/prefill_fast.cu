@@ -255,8 +255,9 @@ prefill_select_kernel(const __grid_constant__ CUtensorMap map_lm, const PArgs a)
 __host__ __device__ inline int max_local_slots(int W) { return (W - 1 + kS - 1) / kS + 1; }
 __device__ __forceinline__ int slot_chunk(const PArgs& a, int pair, int tok, int slot) {
     if (slot >= a.s.K) {
-        const int c = local_lo(tok, a.s.W, kS) / kS + (slot - a.s.K);
-        return c <= tok / kS ? c : -1;
+        const int pos = a.s.pos0 + tok;
+        const int c = local_lo(pos, a.s.W, kS) / kS + (slot - a.s.K);
+        return c <= pos / kS ? c : -1;
     }
     return a.sel[(static_cast<long long>(pair) * a.s.R + tok) * a.s.K + slot];
 }
@@ -377,9 +378,10 @@ __global__ void __launch_bounds__(kFuseWarps * 32) prefill_fuse_kernel(const PAr
     const int b = pair / s.Hkv, gk = pair % s.Hkv;
     const int tok = a.i0 + il;
     // rows to mix: the selected chunks (slots 0..nsel-1), then the chunks of the local window (slots K..K+nl-1)
-    const int lc = local_lo(tok, s.W, kS) / kS;      // first local chunk = number of candidate chunks
+    const int pos = s.pos0 + tok;                    // sequence position of this query row
+    const int lc = local_lo(pos, s.W, kS) / kS;      // first local chunk = number of candidate chunks
     const int nsel = min(K, lc);
-    const int nl = tok / kS - lc + 1;
+    const int nl = pos / kS - lc + 1;
     const int nrows = nsel + nl;
     const int e0 = a.blk_toff[a.blk] * a.tile_tok;   // first entry of this query block
     const int* ep = a.epos + (static_cast<long long>(pair) * s.R + tok) * K1;
@@ -479,7 +481,8 @@ Plan make_plan(const Shape& s) {
     const size_t pairs = static_cast<size_t>(s.B) * s.Hkv;
     const size_t blk = static_cast<size_t>(s.R < kQB ? (s.R + kS - 1) / kS * kS : kQB);
     p.qb = static_cast<int>(blk);
-    const size_t nc = static_cast<size_t>(s.C > (s.R + kS - 1) / kS ? s.C : (s.R + kS - 1) / kS);
+    const size_t nchunks = (static_cast<size_t>(s.pos0) + s.R + kS - 1) / kS;     // chunks the queries can touch
+    const size_t nc = static_cast<size_t>(s.C) > nchunks ? static_cast<size_t>(s.C) : nchunks;
     p.nc = static_cast<int>(nc);
     const size_t nblocks = (static_cast<size_t>(s.R) + blk - 1) / blk;
     p.n_blocks = static_cast<int>(nblocks);
@@ -488,7 +491,7 @@ Plan make_plan(const Shape& s) {
     size_t all_tiles = 0, max_blk = 0;
     for (size_t b = 0; b < nblocks; ++b) {
         const size_t toks = (b + 1) * blk <= static_cast<size_t>(s.R) ? blk : static_cast<size_t>(s.R) - b * blk;
-        const size_t vis = ((b * blk + toks) + kS - 1) / kS;
+        const size_t vis = ((s.pos0 + b * blk + toks) + kS - 1) / kS;
         const size_t tiles = pairs * (toks * (s.K + max_local_slots(s.W)) / tt + (vis < nc ? vis : nc)) + 1;
         all_tiles += tiles;
         max_blk = tiles > max_blk ? tiles : max_blk;
@@ -517,10 +520,10 @@ Plan make_plan(const Shape& s) {
 bool prefill_fast_supports(const Shape& s, int dtype) {
     // any window whose chunks fit the fuse kernel's row table; the warp-MMA selection fallback (K > 32) knows W = 1 only
     return dtype == HILS_BF16 && !s.is_decode && s.d == kD && s.S == kS && s.W >= 1 && max_local_slots(s.W) <= 16 &&
-           (s.W == 1 || (s.K <= 32 && prefill_select_tc_supports(s))) && s.Hl == s.Hkv && s.G == kG &&
+           ((s.W == 1 && s.pos0 == 0) || (s.K <= 32 && prefill_select_tc_supports(s))) && s.Hl == s.Hkv && s.G == kG &&
            s.K >= 1 && s.K <= 64 && static_cast<long long>(s.B) * s.Hkv * s.T < (1ll << 31) &&
            static_cast<long long>(s.B) * s.Hkv * s.C < (1ll << 24) &&
-           static_cast<long long>(s.B) * s.Hkv * ((s.R + kS - 1) / kS) < (1ll << 31) &&
+           static_cast<long long>(s.B) * s.Hkv * ((s.pos0 + s.R + kS - 1) / kS) < (1ll << 31) &&
            static_cast<long long>(s.B) * s.Hkv * s.R * (s.K + max_local_slots(s.W)) < (1ll << 31);
 }
 

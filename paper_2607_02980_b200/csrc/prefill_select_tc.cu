@@ -136,7 +136,7 @@ prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     const int b = pair / s.Hkv, gk = pair % s.Hkv;
     // candidates of a token = the chunks left of its local window (Sec. 2.1); the tile's last token has the most
     const int last_tok = min(s.R, (ti + 1) * kTileTok) - 1;
-    const int ncand_max = local_lo(last_tok, s.W, kS) / kS;
+    const int ncand_max = local_lo(s.pos0 + last_tok, s.W, kS) / kS;
     const int nsteps = (ncand_max + kS - 1) / kS;
     const int K = s.K;
 
@@ -214,7 +214,7 @@ prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         // ------------------------------------------------------------------ epilogue: one token per thread
         const int row = warp * 32 + lane;
         const int tok = ti * kTileTok + row;
-        const int my_ncand = local_lo(tok, s.W, kS) / kS;
+        const int my_ncand = local_lo(s.pos0 + tok, s.W, kS) / kS;
         const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
         unsigned long long* mytop = lists + tid;           // sorted top list: entry e at mytop[e * 128], 0 = empty
         unsigned long long* myq = queue + tid;             // append buffer of raw (score bits, chunk id) pairs
