@@ -1,6 +1,8 @@
 // C ABI of the HiLS library: argument validation, kernel-set dispatch, host-buffer variants.
 #include <string.h>
 
+#include <mutex>
+
 #include "internal.h"
 
 namespace hils {
@@ -25,6 +27,8 @@ void trace_begin(cudaStream_t stream) {
     t.n = 0;
     if (t.enabled && t.have_events) cudaEventRecord(t.ev[0], stream);
 }
+
+bool trace_active() { return g_trace.enabled && g_trace.have_events; }
 
 void trace_mark(const char* name, cudaStream_t stream) {
     Trace& t = g_trace;
@@ -171,6 +175,123 @@ int arena_layout(const hils_params* p, int is_decode, ArenaLayout* a) {
     return HILS_OK;
 }
 
+// ---- pipelined host-buffer prefill -------------------------------------------------------------------------
+// The operator is causal, so a block of query tokens needs only the inputs up to its own end: blocks of
+// kHostBlock tokens are copied in, computed (the slice entry point) and copied out on three internal streams,
+// and the transfers of neighbouring blocks overlap each other (PCIe is full duplex) and the kernels.
+constexpr int kHostBlock = 4096;
+
+struct HostPipe {
+    bool ok = false;
+    cudaStream_t in = nullptr, cmp = nullptr, out = nullptr;
+    cudaEvent_t fork = nullptr, in_done[2] = {nullptr, nullptr}, cmp_done[2] = {nullptr, nullptr},
+                out_done[2] = {nullptr, nullptr}, tail[3] = {nullptr, nullptr, nullptr};
+};
+std::mutex g_pipe_mutex;       // the events are shared: calls that enqueue through the pipe are serialised on the host
+HostPipe g_pipe[64];
+
+HostPipe* host_pipe() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    HostPipe& hp = g_pipe[dev];
+    if (!hp.ok) {
+        auto mk = [](cudaEvent_t* e) { return cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess; };
+        if (cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaStreamCreateWithFlags(&hp.cmp, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking) != cudaSuccess)
+            return nullptr;
+        bool good = mk(&hp.fork);
+        for (int i = 0; i < 2; ++i) good = good && mk(&hp.in_done[i]) && mk(&hp.cmp_done[i]) && mk(&hp.out_done[i]);
+        for (int i = 0; i < 3; ++i) good = good && mk(&hp.tail[i]);
+        if (!good) return nullptr;
+        hp.ok = true;
+    }
+    return &hp;
+}
+
+// Returns HILS_OK, an error, or 1 when the pipelined form does not apply (the caller then takes the plain path).
+int run_host_prefill_pipelined(const hils_params* p, const ArenaLayout& full, const void* q, const void* k,
+                               const void* v, const void* lm, const float* bias, void* out, float* lse, int32_t* sel,
+                               char* base, void* stream_v) {
+    static const bool off = [] { const char* e = getenv("HILS_HOST_PIPELINE"); return e && e[0] == '0'; }();
+    if (off || p->L < 2 * kHostBlock || (p->T_max > 0 && p->T_max != p->L) || trace_active()) return 1;
+    Shape s;
+    if (make_shape(p, 0, &s) != HILS_OK) return 1;
+    const size_t eb = elem_bytes(p->dtype);
+    const int L = p->L, nb = (L + kHostBlock - 1) / kHostBlock;
+    hils_params bp = *p;
+    bp.T_max = L;
+    bp.L = kHostBlock;
+    const size_t ws_b = hils_prefill_at_workspace_bytes(&bp, static_cast<int64_t>(nb - 1) * kHostBlock);
+    if (ws_b == 0) return 1;
+    // layout inside the caller's arena: workspace, K, V, landmarks, bias, then two slots of per-block q / out / lse / sel
+    const size_t rowsq = static_cast<size_t>(s.B) * s.Hq, rowskv = static_cast<size_t>(s.B) * s.Hkv;
+    const size_t q_blk = rowsq * kHostBlock * s.d * eb, lse_blk = rowsq * kHostBlock * 4;
+    const size_t sel_blk = rowskv * kHostBlock * s.K * 4;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
+    const size_t a_ws = take(ws_b), a_k = take(full.kv_b), a_v = take(full.kv_b), a_lm = take(full.lm_b), a_bias = take(full.bias_b);
+    size_t a_q[2], a_out[2], a_lse[2], a_sel[2];
+    for (int i = 0; i < 2; ++i) { a_q[i] = take(q_blk); a_out[i] = take(q_blk); a_lse[i] = take(lse_blk); a_sel[i] = take(sel_blk); }
+    if (o > full.total) return 1;
+
+    std::lock_guard<std::mutex> lock(g_pipe_mutex);
+    HostPipe* hp = host_pipe();
+    if (!hp) return 1;
+    cudaStream_t user = static_cast<cudaStream_t>(stream_v);
+    bool ok = cudaEventRecord(hp->fork, user) == cudaSuccess;
+    ok = ok && cudaStreamWaitEvent(hp->in, hp->fork, 0) == cudaSuccess && cudaStreamWaitEvent(hp->cmp, hp->fork, 0) == cudaSuccess &&
+         cudaStreamWaitEvent(hp->out, hp->fork, 0) == cudaSuccess;
+    // the status word at the arena's head stays as the caller left it; landmarks and bias go first
+    ok = ok && cudaMemcpyAsync(base + a_lm, lm, full.lm_b, cudaMemcpyHostToDevice, hp->in) == cudaSuccess;
+    if (bias) ok = ok && cudaMemcpyAsync(base + a_bias, bias, full.bias_b, cudaMemcpyHostToDevice, hp->in) == cudaSuccess;
+    if (!ok) return HILS_ERR_CUDA;
+    int launches = 0;
+    const size_t tok_b = static_cast<size_t>(s.d) * eb;                  // bytes per token row
+    for (int b = 0; b < nb; ++b) {
+        const int i0 = b * kHostBlock, len = (L - i0 < kHostBlock) ? L - i0 : kHostBlock, sl = b & 1;
+        // ---- copy in: this block's K / V rows into the device caches, its queries into slot sl
+        if (b >= 2) ok = ok && cudaStreamWaitEvent(hp->in, hp->cmp_done[sl], 0) == cudaSuccess;
+        ok = ok && cudaMemcpy2DAsync(base + a_k + i0 * tok_b, L * tok_b, static_cast<const char*>(k) + i0 * tok_b, L * tok_b,
+                                     len * tok_b, rowskv, cudaMemcpyHostToDevice, hp->in) == cudaSuccess;
+        ok = ok && cudaMemcpy2DAsync(base + a_v + i0 * tok_b, L * tok_b, static_cast<const char*>(v) + i0 * tok_b, L * tok_b,
+                                     len * tok_b, rowskv, cudaMemcpyHostToDevice, hp->in) == cudaSuccess;
+        ok = ok && cudaMemcpy2DAsync(base + a_q[sl], len * tok_b, static_cast<const char*>(q) + i0 * tok_b, L * tok_b,
+                                     len * tok_b, rowsq, cudaMemcpyHostToDevice, hp->in) == cudaSuccess;
+        ok = ok && cudaEventRecord(hp->in_done[sl], hp->in) == cudaSuccess;
+        // ---- compute
+        ok = ok && cudaStreamWaitEvent(hp->cmp, hp->in_done[sl], 0) == cudaSuccess;
+        if (b >= 2) ok = ok && cudaStreamWaitEvent(hp->cmp, hp->out_done[sl], 0) == cudaSuccess;
+        if (!ok) return HILS_ERR_CUDA;
+        bp.L = len;
+        const int rc = run(&bp, 0, base + a_q[sl], base + a_k, base + a_v, base + a_lm,
+                           bias ? reinterpret_cast<const float*>(base + a_bias) : nullptr, nullptr, base + a_out[sl],
+                           reinterpret_cast<float*>(base + a_lse[sl]), reinterpret_cast<int32_t*>(base + a_sel[sl]),
+                           base + a_ws, ws_b, hp->cmp, nullptr, 0, i0);
+        if (rc != HILS_OK) return rc;
+        launches += g_last_launches;
+        ok = ok && cudaEventRecord(hp->cmp_done[sl], hp->cmp) == cudaSuccess;
+        // ---- copy out
+        ok = ok && cudaStreamWaitEvent(hp->out, hp->cmp_done[sl], 0) == cudaSuccess;
+        ok = ok && cudaMemcpy2DAsync(static_cast<char*>(out) + i0 * tok_b, L * tok_b, base + a_out[sl], len * tok_b, len * tok_b,
+                                     rowsq, cudaMemcpyDeviceToHost, hp->out) == cudaSuccess;
+        ok = ok && cudaMemcpy2DAsync(reinterpret_cast<char*>(lse) + static_cast<size_t>(i0) * 4, static_cast<size_t>(L) * 4,
+                                     base + a_lse[sl], static_cast<size_t>(len) * 4, static_cast<size_t>(len) * 4, rowsq,
+                                     cudaMemcpyDeviceToHost, hp->out) == cudaSuccess;
+        const size_t selrow = static_cast<size_t>(s.K) * 4;
+        ok = ok && cudaMemcpy2DAsync(reinterpret_cast<char*>(sel) + i0 * selrow, L * selrow, base + a_sel[sl], len * selrow,
+                                     len * selrow, rowskv, cudaMemcpyDeviceToHost, hp->out) == cudaSuccess;
+        ok = ok && cudaEventRecord(hp->out_done[sl], hp->out) == cudaSuccess;
+        if (!ok) return HILS_ERR_CUDA;
+    }
+    // ---- join: the caller's stream continues after everything enqueued here
+    ok = ok && cudaEventRecord(hp->tail[0], hp->in) == cudaSuccess && cudaEventRecord(hp->tail[1], hp->cmp) == cudaSuccess &&
+         cudaEventRecord(hp->tail[2], hp->out) == cudaSuccess;
+    for (int i = 0; i < 3; ++i) ok = ok && cudaStreamWaitEvent(user, hp->tail[i], 0) == cudaSuccess;
+    g_last_launches = launches;
+    return ok ? HILS_OK : HILS_ERR_CUDA;
+}
+
 int run_host(const hils_params* p, int is_decode, const void* q, const void* k, const void* v, const void* lm,
              const float* bias, const int32_t* seq_lens, void* out, float* lse, int32_t* sel, void* arena,
              size_t arena_bytes, void* stream_v) {
@@ -182,6 +303,10 @@ int run_host(const hils_params* p, int is_decode, const void* q, const void* k, 
     if (reinterpret_cast<uintptr_t>(arena) & 255u) return HILS_ERR_ALIGNMENT;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     char* base = static_cast<char*>(arena);
+    if (!is_decode) {
+        rc = run_host_prefill_pipelined(p, a, q, k, v, lm, bias, out, lse, sel, base, stream_v);
+        if (rc != 1) return rc;
+    }
     bool ok = true;
     ok &= cudaMemcpyAsync(base + a.q, q, a.q_b, cudaMemcpyHostToDevice, stream) == cudaSuccess;
     ok &= cudaMemcpyAsync(base + a.k, k, a.kv_b, cudaMemcpyHostToDevice, stream) == cudaSuccess;

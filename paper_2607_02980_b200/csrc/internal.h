@@ -33,6 +33,7 @@ struct Tensors {
 // time between consecutive marks is that kernel's device time.  Off by default (no events).
 void trace_begin(cudaStream_t stream);
 void trace_mark(const char* name, cudaStream_t stream);
+bool trace_active();
 
 // Each launcher returns the number of kernels it enqueued, or a negative hils_status.
 int launch_generic(const Shape& s, int dtype, const Tensors& t, cudaStream_t stream);

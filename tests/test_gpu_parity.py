@@ -242,3 +242,21 @@ def test_host_entry_points_match_device_entry_points():
     torch.cuda.synchronize()
     assert torch.equal(hs, s.cpu())
     assert (ho.float() - o.cpu().float()).abs().max() <= 1e-2
+
+
+def test_pipelined_host_prefill_matches_the_device_entry_point():
+    """Long sequences through hils_prefill_host are copied, computed and copied back in blocks of 4096 tokens on
+    internal streams; the result must be the device entry point's, twice in a row (buffer slots are reused)."""
+    cfg = wl.CONFIGS[1].scaled(B=2, Hq=8, Hkv=2, L=2 * 4096 + 808, K=12, seed=51)
+    inp = wl.make_prefill_inputs(cfg, "cpu")
+    bias = wl.make_bias(cfg, "cpu")
+    out, lse, sel = run_prefill(cfg, inp, "auto", bias=bias)
+    p = hils.make_params(B=cfg.B, Hq=cfg.Hq, Hkv=cfg.Hkv, Hl=cfg.Hkv, L=cfg.L, T_max=cfg.L, C=cfg.C, d=cfg.d,
+                         chunk_size=cfg.S, top_k=cfg.K, dtype=1, impl="auto")
+    runner = hils.HostRunner(p, False, DEV)
+    pinned = {k: v.pin_memory() for k, v in inp.items()}
+    for _ in range(2):
+        ho, hl, hs = runner.run(pinned["q"], pinned["k"], pinned["v"], pinned["landmarks"], bias=bias.pin_memory())
+        torch.cuda.synchronize()
+        assert torch.equal(hs, sel.cpu())
+        assert torch.equal(ho, out.cpu()) and torch.equal(hl, lse.cpu())
