@@ -74,3 +74,70 @@ def test_cfg3_batched_decode_sampled_sequences():
 
 def test_cfg4_ultralong_decode_sampled_sequences():
     print(decode_full(wl.CONFIGS[4], [1, 3]))
+
+
+def test_cfg2_shape_with_the_papers_window_and_bias_sampled_rows():
+    """cfg2's shape in the paper's operator form (W = 512, bias), the configuration bench.py reports as
+    extra.cfg2_window512_bias, on sampled rows."""
+    cfg = wl.CONFIGS[2]
+    inp = wl.make_prefill_inputs(cfg, DEV)
+    bias = wl.make_bias(cfg, DEV)
+    out, lse, sel = hils.hils_prefill(inp["q"], inp["k"], inp["v"], inp["landmarks"], cfg.S, cfg.K, bias=bias, window=512)
+    torch.cuda.synchronize()
+    rows = wl.sample_rows(cfg, 2048).numpy()
+    ridx = torch.as_tensor(rows, device=DEV)
+    cpu = {k: v.cpu() for k, v in inp.items()}
+    B, Hq, _, d = out.shape
+    full_out = torch.zeros((B, Hq, cfg.L, d), dtype=torch.float32)
+    full_lse = torch.zeros((B, Hq, cfg.L), dtype=torch.float32)
+    full_sel = torch.full((B, cfg.Hkv, cfg.L, cfg.K), -1, dtype=torch.int32)
+    r = torch.as_tensor(rows)
+    full_out[:, :, r] = out[:, :, ridx].float().cpu()
+    full_lse[:, :, r] = lse[:, :, ridx].cpu()
+    full_sel[:, :, r] = sel[:, :, ridx].cpu()
+    print(check_prefill(cfg, cpu, full_out, full_lse, full_sel, rows=rows, bias=bias.cpu(), W=512))
+
+
+def test_cfg3_paged_and_windowed_decode_sampled_sequences():
+    """cfg3 through hils_decode_paged (shuffled pages, as bench.py's extra.cfg3_paged) with W = 512 and bias:
+    identical to the contiguous entry point on every sequence, and the oracle on sampled ones."""
+    cfg = wl.CONFIGS[3]
+    inp = wl.make_decode_inputs(cfg, DEV)
+    bias = wl.make_bias(cfg, DEV)
+    B, Hkv, T, d = inp["k"].shape
+    C, S = T // cfg.S, cfg.S
+    perm = torch.randperm(B * C, generator=torch.Generator(device=DEV).manual_seed(3), device=DEV)
+
+    def pages(x):
+        src = x.view(B, Hkv, C, S, d).permute(0, 2, 1, 3, 4).reshape(B * C, Hkv, S, d)
+        dst = torch.empty_like(src)
+        dst[perm] = src
+        return dst
+
+    table = perm.reshape(B, C).to(torch.int32)
+    out_c, lse_c, sel_c = hils.hils_decode(inp["q"], inp["k"], inp["v"], inp["landmarks"], inp["seq_lens"], cfg.S, cfg.K,
+                                           bias=bias, window=512)
+    out_p, lse_p, sel_p = hils.hils_decode_paged(inp["q"], pages(inp["k"]), pages(inp["v"]), inp["landmarks"], table,
+                                                 inp["seq_lens"], cfg.S, cfg.K, bias=bias, window=512)
+    torch.cuda.synchronize()
+    assert torch.equal(sel_p, sel_c) and torch.equal(out_p, out_c) and torch.equal(lse_p, lse_c)
+    s = torch.as_tensor([0, 17, 63], device=DEV)
+    cpu = {k: v[s].cpu() for k, v in inp.items()}
+    print(check_decode(cfg.scaled(B=3), cpu, out_p[s], lse_p[s], sel_p[s], bias=bias[s].cpu(), W=512))
+
+
+def test_landmark_summary_on_the_cfg3_key_cache_sampled_sequences():
+    """The chunk-summary kernel on the full 8.6 GB key cache (the launch bench.py times); sampled sequences against
+    the oracle, all of them finite and with entropies in [0, log S]."""
+    import oracle
+    cfg = wl.CONFIGS[3]
+    inp = wl.make_decode_inputs(cfg, DEV)
+    lq = wl.make_landmark_queries(cfg, DEV)
+    lm, b = hils.hils_landmark_summary(lq, inp["k"], cfg.S, seq_lens=inp["seq_lens"])
+    torch.cuda.synchronize()
+    assert torch.isfinite(lm.float()).all() and (b >= -1e-5).all() and (b <= np.log(cfg.S) + 1e-4).all()
+    for bi in (0, 31, 63):
+        ref_lm, ref_b = oracle.hils_landmarks(lq[bi:bi + 1].cpu(), inp["k"][bi:bi + 1].cpu(),
+                                              seq_lens=inp["seq_lens"][bi:bi + 1].cpu(), S=cfg.S)
+        assert np.abs(lm[bi:bi + 1].float().cpu().numpy() - ref_lm).max() <= 2e-2
+        assert np.abs(b[bi:bi + 1].cpu().numpy() - ref_b).max() <= 2e-5
