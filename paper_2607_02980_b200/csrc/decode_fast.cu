@@ -323,30 +323,37 @@ __device__ void select_pair(const DArgs& a, int pair, int ncand, SelShared& sh, 
     //     landmark rows and the G queries are staged in shared memory with one round of 16-byte
     //     loads, then every thread computes (chunk, head) dot products
     __nv_bfloat16 (*lm_s)[kD + 8] = reinterpret_cast<__nv_bfloat16 (*)[kD + 8]>(dyn);
-    const __nv_bfloat16* lm = a.lm + static_cast<long long>(pair) * s.C * kD;
+    const int per = s.Hl / s.Hkv;                        // landmark rows per chunk: 1, or one per query head (G)
+    const long long lrow0 = (static_cast<long long>(b) * s.Hl + g * per) * s.C;      // landmark head 0 of this KV head
     const __nv_bfloat16* qg = a.q + (static_cast<long long>(b) * s.Hq + g * G) * kD;
     for (int x = tid; x < G * 16; x += NT)
         *reinterpret_cast<uint4*>(&sh.q_s[x >> 4][(x & 15) * 8]) = *reinterpret_cast<const uint4*>(qg + (x >> 4) * kD + (x & 15) * 8);
-    for (int t0 = 0; t0 < n; t0 += 64) {
-        const int nt = min(64, n - t0);
+    const int tstep = 64 / per;                          // selected chunks staged per round (64 landmark rows)
+    for (int t0 = 0; t0 < n; t0 += tstep) {
+        const int nt = min(tstep, n - t0);
         __syncthreads();
-        for (int x0 = 0; x0 < nt * 16; x0 += 4 * NT) {       // four 16-byte loads in flight per thread
+        // staged row (t * per + hh): landmark head hh of selected chunk t0 + t
+        for (int x0 = 0; x0 < nt * per * 16; x0 += 4 * NT) {       // four 16-byte loads in flight per thread
             uint4 v[4];
 #pragma unroll
             for (int r = 0; r < 4; ++r) {
                 const int x = x0 + r * NT + tid;
-                if (x < nt * 16) v[r] = *reinterpret_cast<const uint4*>(lm + static_cast<long long>(sel_s[t0 + (x >> 4)]) * kD + (x & 15) * 8);
+                if (x < nt * per * 16) {
+                    const int row = x >> 4, tt = row / per, hh = row % per;
+                    v[r] = *reinterpret_cast<const uint4*>(a.lm + (lrow0 + static_cast<long long>(hh) * s.C + sel_s[t0 + tt]) * kD + (x & 15) * 8);
+                }
             }
 #pragma unroll
             for (int r = 0; r < 4; ++r) {
                 const int x = x0 + r * NT + tid;
-                if (x < nt * 16) *reinterpret_cast<uint4*>(&lm_s[x >> 4][(x & 15) * 8]) = v[r];
+                if (x < nt * per * 16) *reinterpret_cast<uint4*>(&lm_s[x >> 4][(x & 15) * 8]) = v[r];
             }
         }
         __syncthreads();
         for (int x = tid; x < nt * G; x += NT) {
             const int t = x / G, h = x % G;
-            const __nv_bfloat16* lr = lm_s[t];
+            const int hh = per == 1 ? 0 : h;             // the landmark head this query head scores against
+            const __nv_bfloat16* lr = lm_s[t * per + hh];
             const __nv_bfloat16* qr = sh.q_s[h];
             float acc = 0.f;
 #pragma unroll 8
@@ -356,7 +363,7 @@ __device__ void select_pair(const DArgs& a, int pair, int ncand, SelShared& sh, 
                 acc = fmaf(lv.x, qv.x, acc);
                 acc = fmaf(lv.y, qv.y, acc);
             }
-            const float bb = a.bias ? a.bias[static_cast<long long>(pair) * s.C + sel_s[t0 + t]] : 0.f;
+            const float bb = a.bias ? a.bias[lrow0 + static_cast<long long>(hh) * s.C + sel_s[t0 + t]] : 0.f;
             sh.lam_s[h][t0 + t] = acc * s.scale + bb;
         }
     }
@@ -401,46 +408,62 @@ __global__ void __launch_bounds__(kScoreThreads) decode_score_kernel(const DArgs
 #pragma unroll
         for (int kb = 0; kb < 4; ++kb) qf[kb] = *reinterpret_cast<const uint4*>(qrow + kb * 32 + t * 8);
     }
-    const __nv_bfloat16* lm = a.lm + static_cast<long long>(pair) * s.C * kD;
-    const float* bias = a.bias ? a.bias + static_cast<long long>(pair) * s.C : nullptr;
+    // One landmark per KV head (per = 1: all heads score the same row), or one per query head (per = G, App. C:
+    // k'_c in R^{G x d}): then head hh scores only its own landmark row and only column hh of the MMA is kept.
+    const int per = s.Hl / s.Hkv;
     float* u = a.u + static_cast<long long>(pair) * a.Cpad;
-
-    uint4 x[2][2][4];
     int c0[2];
+    float best[2][2];
 #pragma unroll
     for (int it = 0; it < 2; ++it) {
         c0[it] = c_begin + (warp * 2 + it) * 16;
-        if (c0[it] < ncand) {
-            const int r0 = min(c0[it] + gq, ncand - 1), r1 = min(c0[it] + gq + 8, ncand - 1);
+        best[it][0] = best[it][1] = -INFINITY;
+    }
+    for (int hh = 0; hh < per; ++hh) {
+        const long long lrow = (static_cast<long long>(b) * s.Hl + g * per + hh) * s.C;
+        const __nv_bfloat16* lm = a.lm + lrow * kD;
+        const float* bias = a.bias ? a.bias + lrow : nullptr;
+        uint4 x[2][2][4];
+#pragma unroll
+        for (int it = 0; it < 2; ++it) {
+            if (c0[it] < ncand) {
+                const int r0 = min(c0[it] + gq, ncand - 1), r1 = min(c0[it] + gq + 8, ncand - 1);
+#pragma unroll
+                for (int kb = 0; kb < 4; ++kb) {
+                    x[it][0][kb] = __ldg(reinterpret_cast<const uint4*>(lm + static_cast<long long>(r0) * kD + kb * 32 + t * 8));
+                    x[it][1][kb] = __ldg(reinterpret_cast<const uint4*>(lm + static_cast<long long>(r1) * kD + kb * 32 + t * 8));
+                }
+            }
+        }
+#pragma unroll
+        for (int it = 0; it < 2; ++it) {
+            if (c0[it] >= ncand) continue;
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int kb = 0; kb < 4; ++kb) {
-                x[it][0][kb] = __ldg(reinterpret_cast<const uint4*>(lm + static_cast<long long>(r0) * kD + kb * 32 + t * 8));
-                x[it][1][kb] = __ldg(reinterpret_cast<const uint4*>(lm + static_cast<long long>(r1) * kD + kb * 32 + t * 8));
+                const uint32_t a1[4] = {x[it][0][kb].x, x[it][1][kb].x, x[it][0][kb].y, x[it][1][kb].y};
+                mma_bf16_16816(acc, a1, qf[kb].x, qf[kb].y);
+                const uint32_t a2[4] = {x[it][0][kb].z, x[it][1][kb].z, x[it][0][kb].w, x[it][1][kb].w};
+                mma_bf16_16816(acc, a2, qf[kb].z, qf[kb].w);
             }
+            // acc[0..1]: chunk c0+gq, heads 2t, 2t+1; acc[2..3]: chunk c0+gq+8
+            const bool h0 = per == 1 ? 2 * t < s.G : 2 * t == hh, h1 = per == 1 ? 2 * t + 1 < s.G : 2 * t + 1 == hh;
+            float m0 = fmaxf(h0 ? acc[0] : -INFINITY, h1 ? acc[1] : -INFINITY);
+            float m1 = fmaxf(h0 ? acc[2] : -INFINITY, h1 ? acc[3] : -INFINITY);
+            m0 = fmaxf(m0, __shfl_xor_sync(kFullMask, m0, 1));
+            m1 = fmaxf(m1, __shfl_xor_sync(kFullMask, m1, 1));
+            m0 = fmaxf(m0, __shfl_xor_sync(kFullMask, m0, 2));
+            m1 = fmaxf(m1, __shfl_xor_sync(kFullMask, m1, 2));
+            const int ca = c0[it] + gq, cb = ca + 8;
+            best[it][0] = fmaxf(best[it][0], m0 * s.scale + ((bias && ca < ncand) ? bias[ca] : 0.f));
+            best[it][1] = fmaxf(best[it][1], m1 * s.scale + ((bias && cb < ncand) ? bias[cb] : 0.f));
         }
     }
 #pragma unroll
     for (int it = 0; it < 2; ++it) {
-        if (c0[it] >= ncand) continue;
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-        for (int kb = 0; kb < 4; ++kb) {
-            const uint32_t a1[4] = {x[it][0][kb].x, x[it][1][kb].x, x[it][0][kb].y, x[it][1][kb].y};
-            mma_bf16_16816(acc, a1, qf[kb].x, qf[kb].y);
-            const uint32_t a2[4] = {x[it][0][kb].z, x[it][1][kb].z, x[it][0][kb].w, x[it][1][kb].w};
-            mma_bf16_16816(acc, a2, qf[kb].z, qf[kb].w);
-        }
-        // acc[0..1]: chunk c0+gq, heads 2t, 2t+1; acc[2..3]: chunk c0+gq+8
-        const bool h0 = 2 * t < s.G, h1 = 2 * t + 1 < s.G;
-        float m0 = fmaxf(h0 ? acc[0] : -INFINITY, h1 ? acc[1] : -INFINITY);
-        float m1 = fmaxf(h0 ? acc[2] : -INFINITY, h1 ? acc[3] : -INFINITY);
-        m0 = fmaxf(m0, __shfl_xor_sync(kFullMask, m0, 1));
-        m1 = fmaxf(m1, __shfl_xor_sync(kFullMask, m1, 1));
-        m0 = fmaxf(m0, __shfl_xor_sync(kFullMask, m0, 2));
-        m1 = fmaxf(m1, __shfl_xor_sync(kFullMask, m1, 2));
         const int ca = c0[it] + gq, cb = ca + 8;
-        if (t == 0 && ca < ncand) u[ca] = m0 * s.scale + (bias ? bias[ca] : 0.f);
-        if (t == 1 && cb < ncand) u[cb] = m1 * s.scale + (bias ? bias[cb] : 0.f);
+        if (t == 0 && ca < ncand) u[ca] = best[it][0];
+        if (t == 1 && cb < ncand) u[cb] = best[it][1];
     }
     pdl_launch_dependents();
 }
@@ -804,7 +827,7 @@ Plan make_plan(const Shape& s, int n_sm) {
 }  // namespace
 
 bool decode_fast_supports(const Shape& s, int dtype) {
-    return dtype == HILS_BF16 && s.is_decode && s.d == kD && s.S == kS && s.W >= 1 && max_local_slots(s.W) <= 16 && s.Hl == s.Hkv && s.G <= 8 &&
+    return dtype == HILS_BF16 && s.is_decode && s.d == kD && s.S == kS && s.W >= 1 && max_local_slots(s.W) <= 16 && (s.Hl == s.Hkv || s.Hl == s.Hq) && s.G <= 8 &&
            s.K >= 1 && s.K <= 128 && static_cast<long long>(s.B) * s.Hkv * s.T < (1ll << 31) &&
            static_cast<long long>(s.B) * s.Hkv <= 65535;
 }

@@ -202,6 +202,20 @@ def test_decode_fast_path_with_a_chunk_aligned_local_window(W):
     check_decode(cfg, inp, out, lse, sel, bias=bias, W=W)
 
 
+@pytest.mark.parametrize("W", [1, 200])
+def test_decode_fast_path_with_one_landmark_per_query_head(W):
+    """App. C: in GQA the chunk summary has one row per query head (k'_c in R^{G x d}); every head scores its own
+    landmark, the group score is still the maximum over the heads."""
+    cfg = wl.CONFIGS[3].scaled(B=4, L=4096, K=8, seed=52)
+    fast_or_skip(cfg, True, W=W, Hl=cfg.Hq)
+    inp = wl.make_decode_inputs(cfg, "cpu", seq_lens=torch.tensor([4096, 3000, 130, 65], dtype=torch.int32))
+    g = torch.Generator().manual_seed(9)
+    inp["landmarks"] = (torch.randn((cfg.B, cfg.Hq, cfg.C, cfg.d), generator=g) * 0.7).to(torch.bfloat16)
+    bias = torch.rand((cfg.B, cfg.Hq, cfg.C), generator=g) * float(np.log(cfg.S))
+    out, lse, sel = run_decode(cfg, inp, "fast", bias=bias, W=W)
+    check_decode(cfg, inp, out, lse, sel, bias=bias, W=W)
+
+
 def test_decode_invalid_seq_len_sets_status_without_fault():
     cfg = wl.CONFIGS[3].scaled(B=2, L=1024, K=4, seed=46)
     inp = wl.make_decode_inputs(cfg, "cpu", seq_lens=torch.tensor([1024, 512], dtype=torch.int32))
