@@ -166,8 +166,20 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
             int cur_pair = -1, cur_c = -1;
             int ck = -1;                       // ordinal of the current chunk run within the batch
             bool next_issued = false;          // (producer thread 0) K/V of the upcoming chunk already requested
-            uint4 lm_next = make_uint4(0u, 0u, 0u, 0u);   // (producer lanes 0-15) landmark piece of the next run, fetched a run ahead
+            // landmark pieces of the next run, fetched a run ahead: piece x = lane + 32 r of the `per` landmark rows
+            // (16 pieces each; per = 1: lanes 0-15, r = 0 only)
+            uint4 lm_next[2] = {make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u)};
             bool lm_next_ok = false;
+            const int per = s.Hl / s.Hkv;      // landmark rows per chunk: 1, or one per query head (App. C)
+            auto lm_piece = [&](int pr, int ch, int x) {
+                // 16-byte piece x % 16 of landmark head x / 16 of KV-head pair pr, chunk ch
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                if (ch < s.C) {
+                    const long long lrow = (static_cast<long long>(pr / s.Hkv) * s.Hl + (pr % s.Hkv) * per + (x >> 4)) * s.C + ch;
+                    v = *reinterpret_cast<const uint4*>(a.lm + lrow * kD + (x & 15) * 8);
+                }
+                return v;
+            };
             bool dead = false;
             // entry of this thread's row for the upcoming tile, fetched one tile ahead
             int e_next = a.entries[sm.recs[0].z + min(ptid >> 2, sm.recs[0].w - 1)];
@@ -203,21 +215,21 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                             // done) and TMA never writes this row.  V stays as TMA writes it (keys x dims): the second
                             // MMA reads it as an MN-major operand; keys past the end of the sequence hold other rows'
                             // data (or TMA zero fill) and meet probabilities of 0.
-                            if (lane < 16) {
-                                uint4 v = lm_next;
-                                if (!lm_next_ok) {
-                                    v = make_uint4(0u, 0u, 0u, 0u);
-                                    if (c < s.C) v = *reinterpret_cast<const uint4*>(a.lm + (static_cast<long long>(pair) * s.C + c) * kD + lane * 8);
-                                }
-                                *reinterpret_cast<uint4*>(kbuf + cbuf * kKBytes + (lane >> 3) * (kNS * 128) + swz128(64, lane & 7)) = v;
-                                // the next run's landmark, so that its load is not waited for at the next switch
-                                lm_next_ok = ck + 2 < sm.nchunks;
-                                if (lm_next_ok) {
-                                    const int4 r1 = sm.recs[sm.cfirst[ck + 2]];
-                                    lm_next = make_uint4(0u, 0u, 0u, 0u);
-                                    if (r1.y < s.C) lm_next = *reinterpret_cast<const uint4*>(a.lm + (static_cast<long long>(r1.x) * s.C + r1.y) * kD + lane * 8);
+                            // key rows 64 .. 64 + per - 1: the chunk's landmark(s)
+                            const bool have_next = ck + 2 < sm.nchunks;
+                            const int4 r1 = have_next ? sm.recs[sm.cfirst[ck + 2]] : make_int4(0, 0, 0, 0);
+#pragma unroll
+                            for (int r = 0; r < 2; ++r) {
+                                const int x = lane + 32 * r;
+                                if (x < per * 16) {
+                                    const uint4 v = lm_next_ok ? lm_next[r] : lm_piece(pair, c, x);
+                                    const int pc = x & 15;
+                                    *reinterpret_cast<uint4*>(kbuf + cbuf * kKBytes + (pc >> 3) * (kNS * 128) + swz128(64 + (x >> 4), pc & 7)) = v;
+                                    // the next run's landmark, so that its load is not waited for at the next switch
+                                    if (have_next) lm_next[r] = lm_piece(r1.x, r1.y, x);
                                 }
                             }
+                            lm_next_ok = have_next;
                             fence_proxy_async_smem();
                             __syncwarp();
                             if (lane == 0) mbar_arrive(&sm.k_ready[cbuf]);
@@ -400,7 +412,11 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                 {
                     float v[64];
                     tmem_ld64(t_lane + sl * 128, v);
-                    const float lmk = tmem_ld1(t_lane + sl * 128 + 64);
+                    // surrogate score column: the landmark of this row's head (key 64 + hd) or the shared one (key 64)
+                    const int lh = (s.Hl == s.Hkv) ? 0 : hd;
+                    float lm4[4];
+                    tmem_ld4(t_lane + sl * 128 + 64, lm4);           // warp-uniform address; the lane picks its column
+                    const float lmk = lh == 0 ? lm4[0] : (lh == 1 ? lm4[1] : (lh == 2 ? lm4[2] : lm4[3]));
                     tc_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&sm.s_empty[sl]);
@@ -434,7 +450,8 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                     }
                     zi = 1.f / z;
                     // chunk mass of the row (rows of a ragged tile's padding land in the list's padding)
-                    const float bb = (a.bias && c < s.C) ? a.bias[static_cast<long long>(pair) * s.C + c] : 0.f;
+                    const float bb = (a.bias && c < s.C)
+                        ? a.bias[(static_cast<long long>(pair / s.Hkv) * s.Hl + (pair % s.Hkv) * (s.Hl / s.Hkv) + lh) * s.C + c] : 0.f;
                     a.lam[orow0 + row] = local ? m * s.scale + __logf(z) : lmk * s.scale + bb;
                 }
                 fence_proxy_async_smem();

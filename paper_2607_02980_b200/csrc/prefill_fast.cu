@@ -520,7 +520,8 @@ Plan make_plan(const Shape& s) {
 bool prefill_fast_supports(const Shape& s, int dtype) {
     // any window whose chunks fit the fuse kernel's row table; the warp-MMA selection fallback (K > 32) knows W = 1 only
     return dtype == HILS_BF16 && !s.is_decode && s.d == kD && s.S == kS && s.W >= 1 && max_local_slots(s.W) <= 16 &&
-           ((s.W == 1 && s.pos0 == 0) || (s.K <= 32 && prefill_select_tc_supports(s))) && s.Hl == s.Hkv && s.G == kG &&
+           ((s.W == 1 && s.pos0 == 0 && s.Hl == s.Hkv) || (s.K <= 32 && prefill_select_tc_supports(s))) &&
+           (s.Hl == s.Hkv || s.Hl == s.Hq) && s.G == kG &&
            s.K >= 1 && s.K <= 64 && static_cast<long long>(s.B) * s.Hkv * s.T < (1ll << 31) &&
            static_cast<long long>(s.B) * s.Hkv * s.C < (1ll << 24) &&
            static_cast<long long>(s.B) * s.Hkv * ((s.pos0 + s.R + kS - 1) / kS) < (1ll << 31) &&

@@ -116,7 +116,9 @@ __device__ __noinline__ float merge_buffer(unsigned long long* mytop, const unsi
 }
 
 // N = length of the per-token top list and of the append buffer: 16 for K <= 16, else 32.
-template <int N>
+// PERHEAD: one landmark row (and bias) per query head (App. C) instead of one per KV head.  A template parameter, not
+// a run-time branch: the scan loop's code has to stay small (the kernel is sensitive to instruction fetch).
+template <int N, bool PERHEAD>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_lm,
                          const TcArgs a) {
@@ -139,6 +141,7 @@ prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     const int ncand_max = local_lo(s.pos0 + last_tok, s.W, kS) / kS;
     const int nsteps = (ncand_max + kS - 1) / kS;
     const int K = s.K;
+    constexpr int per = PERHEAD ? kG : 1;     // landmark rows per chunk
 
     if (tid == 0) {
         mbar_init(&sm.q_full, 1);
@@ -163,15 +166,18 @@ prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 tma_load_2d(qs + h * 32768, &map_q, &sm.q_full, 0, row);
                 tma_load_2d(qs + h * 32768 + 16384, &map_q, &sm.q_full, 64, row);
             }
+            // landmark tiles in ring order: step it, landmark head hh (per = 1: one tile per step for all heads;
+            // per = G: one tile per query head, App. C)
             int issued = 0;
-            for (int it = 0; it < nsteps; ++it) {
-                const int st = it % kLmStages;
-                if (it >= kLmStages && !mbar_wait(&sm.empty[st], ((it / kLmStages) - 1) & 1)) {
+            const int ntiles = nsteps * per;
+            for (int n = 0; n < ntiles; ++n) {
+                const int st = n % kLmStages, it = n / per, hh = n % per;
+                if (n >= kLmStages && !mbar_wait(&sm.empty[st], ((n / kLmStages) - 1) & 1)) {
                     set_status(a.status, kDevTimeout);
                     break;
                 }
                 uint8_t* dst = lms + st * kLmStageBytes;
-                const int row = pair * s.C + it * kS;
+                const int row = ((b * s.Hl + gk * per + hh)) * s.C + it * kS;
                 mbar_expect_tx(&sm.full[st], kLmStageBytes);
                 tma_load_2d(dst, &map_lm, &sm.full[st], 0, row);
                 tma_load_2d(dst + 8192, &map_lm, &sm.full[st], 64, row);
@@ -179,33 +185,52 @@ prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             }
             // own copies in flight: every issued stage and the query tile must have landed before exit
             mbar_wait(&sm.q_full, 0);
-            for (int it = max(0, issued - kLmStages); it < issued; ++it)
-                mbar_wait(&sm.full[it % kLmStages], (it / kLmStages) & 1);
+            for (int n = max(0, issued - kLmStages); n < issued; ++n)
+                mbar_wait(&sm.full[n % kLmStages], (n / kLmStages) & 1);
         }
     } else if (warp == 5) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0 && nsteps > 0) {
             constexpr uint32_t idesc = umma_idesc_bf16(kTileTok, kS);
             bool ok = mbar_wait(&sm.q_full, 0);
-            for (int it = 0; it < nsteps && ok; ++it) {
-                const int st = it % kLmStages, buf = it & 1;
-                ok = mbar_wait(&sm.full[st], (it / kLmStages) & 1);
-                if (ok && it >= 2) ok = mbar_wait(&sm.tmem_empty[buf], ((it >> 1) - 1) & 1);
-                if (!ok) break;
-                tc_fence_after_sync();
-                const uint32_t lm_addr = smem_u32(lms + st * kLmStageBytes);
+            // S_h = Q_h x landmark tile^T (M = 128 tokens, N = 64 chunks, K = 128) into head h's 64 columns
+            auto issue_head = [&](uint32_t d_tmem, uint32_t q_addr, uint32_t lm_addr) {
 #pragma unroll
-                for (int h = 0; h < kG; ++h) {
-                    const uint32_t d_tmem = tmem_base + buf * 256 + h * kS;
-                    const uint32_t q_addr = smem_u32(qs + h * 32768);
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks) {
-                        const uint64_t da = umma_desc_k128(q_addr + (ks >> 2) * 16384 + (ks & 3) * 32);
-                        const uint64_t db = umma_desc_k128(lm_addr + (ks >> 2) * 8192 + (ks & 3) * 32);
-                        umma_bf16(d_tmem, da, db, idesc, ks > 0 ? 1u : 0u);
-                    }
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint64_t da = umma_desc_k128(q_addr + (ks >> 2) * 16384 + (ks & 3) * 32);
+                    const uint64_t db = umma_desc_k128(lm_addr + (ks >> 2) * 8192 + (ks & 3) * 32);
+                    umma_bf16(d_tmem, da, db, idesc, ks > 0 ? 1u : 0u);
                 }
-                umma_commit(&sm.empty[st]);            // landmark stage reusable once these MMAs are done
+            };
+            const uint32_t q0 = smem_u32(qs);
+            for (int it = 0; it < nsteps && ok; ++it) {
+                const int buf = it & 1;
+                if (it >= 2) ok = mbar_wait(&sm.tmem_empty[buf], ((it >> 1) - 1) & 1);
+                if (!ok) break;
+                if (per == 1) {
+                    // one landmark tile for the four query heads
+                    const int st = it % kLmStages;
+                    ok = mbar_wait(&sm.full[st], (it / kLmStages) & 1);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const uint32_t lm_addr = smem_u32(lms + st * kLmStageBytes);
+#pragma unroll
+                    for (int h = 0; h < kG; ++h) issue_head(tmem_base + buf * 256 + h * kS, q0 + h * 32768, lm_addr);
+                    umma_commit(&sm.empty[st]);        // landmark stage reusable once these MMAs are done
+                } else {
+                    // one landmark tile per query head (App. C), in ring order
+#pragma unroll
+                    for (int h = 0; h < kG; ++h) {
+                        const int n = it * kG + h, st = n % kLmStages;
+                        if (ok) ok = mbar_wait(&sm.full[st], (n / kLmStages) & 1);
+                        if (ok) {
+                            tc_fence_after_sync();
+                            issue_head(tmem_base + buf * 256 + h * kS, q0 + h * 32768, smem_u32(lms + st * kLmStageBytes));
+                            umma_commit(&sm.empty[st]);
+                        }
+                    }
+                    if (!ok) break;
+                }
                 umma_commit(&sm.tmem_full[buf]);       // scores of this step readable
             }
             if (!ok) set_status(a.status, kDevTimeout);
@@ -218,7 +243,8 @@ prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
         unsigned long long* mytop = lists + tid;           // sorted top list: entry e at mytop[e * 128], 0 = empty
         unsigned long long* myq = queue + tid;             // append buffer of raw (score bits, chunk id) pairs
-        const float* bias = a.bias ? a.bias + static_cast<long long>(pair) * s.C : nullptr;
+        // bias rows of this KV head's landmark heads (per = 1: one row, shared by the four query heads)
+        const float* bias = a.bias ? a.bias + (static_cast<long long>(b) * s.Hl + gk * per) * s.C : nullptr;
         float tau_f = -INFINITY;           // score of the K-th best key so far: the filter of the scan
         int qn = 0;
         bool ok = true;
@@ -242,18 +268,33 @@ prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 const uint32_t col = t_lane + buf * 256 + cb * 16;
                 tmem_ld16x4(col, col + kS, col + 2 * kS, col + 3 * kS, r);
                 const int c0 = it * kS + cb * 16;
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const int c = c0 + j;
-                    float u = fmaxf(fmaxf(r[0][j], r[1][j]), fmaxf(r[2][j], r[3][j])) * s.scale;
-                    if (bias) u += bias[min(c, s.C - 1)];
-                    // first filter on the score alone (ties pass and are settled on the full key when draining);
-                    // branch-free append: the slot is written always and kept only when the candidate passes
+                // first filter on the score alone (ties pass and are settled on the full key when merging);
+                // branch-free append: the slot is written always and kept only when the candidate passes
+                auto offer = [&](float u, int c, int j) {
                     const bool pass = u >= tau_f && (!tail || c < my_ncand);
                     myq[qn * kTileTok] = (static_cast<unsigned long long>(__float_as_uint(u)) << 32) | static_cast<uint32_t>(c);
                     qn += pass ? 1 : 0;
                     // at most 8 appends between checks: a buffer never overflows
                     if ((j & 7) == 7 && __any_sync(kFullMask, qn > N - 8)) compact();
+                };
+                if (PERHEAD && bias != nullptr) {
+                    // every head adds its own bias before the maximum over the group (App. C); kept apart from
+                    // the common loop below, whose code must stay small
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const int c = c0 + j, cc = min(c, s.C - 1);
+                        offer(fmaxf(fmaxf(fmaf(r[0][j], s.scale, bias[cc]), fmaf(r[1][j], s.scale, bias[s.C + cc])),
+                                    fmaxf(fmaf(r[2][j], s.scale, bias[2 * s.C + cc]), fmaf(r[3][j], s.scale, bias[3 * s.C + cc]))),
+                              c, j);
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const int c = c0 + j;
+                        float u = fmaxf(fmaxf(r[0][j], r[1][j]), fmaxf(r[2][j], r[3][j])) * s.scale;
+                        if (bias) u += bias[min(c, s.C - 1)];
+                        offer(u, c, j);
+                    }
                 }
             }
             tc_fence_before_sync();
@@ -295,15 +336,19 @@ int launch_prefill_select_tc(const Shape& s, const void* q, const void* landmark
     const int pairs = s.B * s.Hkv;
     CUtensorMap map_q, map_lm;
     if (!make_bf16_2d_map(&map_q, q, static_cast<uint64_t>(s.B) * s.Hq * s.R, kD, 64, kTileTok) ||
-        !make_bf16_2d_map(&map_lm, landmarks, static_cast<uint64_t>(pairs) * s.C, kD, 64, kS))
+        !make_bf16_2d_map(&map_lm, landmarks, static_cast<uint64_t>(s.B) * s.Hl * s.C, kD, 64, kS))
         return HILS_ERR_CUDA;
     const size_t smem = kQBytes + kLmStages * kLmStageBytes + sizeof(unsigned long long) * 2 * kMaxK * kTileTok +
                         sizeof(TcSmem) + 1024;
     static bool attr_done = false;
     if (!attr_done) {
-        if (cudaFuncSetAttribute(prefill_select_tc_kernel<16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(prefill_select_tc_kernel<16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(smem)) != cudaSuccess ||
-            cudaFuncSetAttribute(prefill_select_tc_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            cudaFuncSetAttribute(prefill_select_tc_kernel<32, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(smem)) != cudaSuccess ||
+            cudaFuncSetAttribute(prefill_select_tc_kernel<16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(smem)) != cudaSuccess ||
+            cudaFuncSetAttribute(prefill_select_tc_kernel<32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(smem)) != cudaSuccess)
             return HILS_ERR_CUDA;
         attr_done = true;
@@ -311,8 +356,14 @@ int launch_prefill_select_tc(const Shape& s, const void* q, const void* landmark
     TcArgs a{s, bias, sel, status};
     const int tiles = (s.R + kTileTok - 1) / kTileTok;
     const unsigned grid = static_cast<unsigned>(pairs) * tiles;
-    if (s.K <= 16) prefill_select_tc_kernel<16><<<grid, kThreads, smem, stream>>>(map_q, map_lm, a);
-    else prefill_select_tc_kernel<32><<<grid, kThreads, smem, stream>>>(map_q, map_lm, a);
+    const bool perhead = s.Hl != s.Hkv;
+    if (s.K <= 16) {
+        if (perhead) prefill_select_tc_kernel<16, true><<<grid, kThreads, smem, stream>>>(map_q, map_lm, a);
+        else prefill_select_tc_kernel<16, false><<<grid, kThreads, smem, stream>>>(map_q, map_lm, a);
+    } else {
+        if (perhead) prefill_select_tc_kernel<32, true><<<grid, kThreads, smem, stream>>>(map_q, map_lm, a);
+        else prefill_select_tc_kernel<32, false><<<grid, kThreads, smem, stream>>>(map_q, map_lm, a);
+    }
     if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
     return 1;
 }

@@ -273,6 +273,19 @@ __device__ __forceinline__ void tmem_ld64(uint32_t taddr, float (&r)[64]) {
 #pragma unroll
     for (int i = 0; i < 64; ++i) r[i] = __uint_as_float(v[i]);
 }
+// four consecutive fp32 columns of this thread's tensor-memory lane (the address is warp-uniform: lane-dependent
+// choices are made on the loaded values)
+__device__ __forceinline__ void tmem_ld4(uint32_t taddr, float (&r)[4]) {
+    uint32_t v[4];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0,%1,%2,%3}, [%4];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3])
+        : "r"(taddr)
+        : "memory");
+#pragma unroll
+    for (int i = 0; i < 4; ++i) r[i] = __uint_as_float(v[i]);
+}
 // one fp32 column of this thread's tensor-memory lane
 __device__ __forceinline__ float tmem_ld1(uint32_t taddr) {
     uint32_t v;

@@ -92,6 +92,20 @@ def test_prefill_fast_path_with_a_chunk_aligned_local_window(W):
     check_prefill(cfg, inp, out, lse, sel, bias=bias, W=W)
 
 
+@pytest.mark.parametrize("W", [1, 200])
+def test_prefill_fast_path_with_one_landmark_per_query_head(W):
+    """App. C on the tensor-core path: every query head scores its own landmark row and adds its own bias; the
+    group score is the maximum over the heads; the fusion weight of a row uses its own head's score."""
+    cfg = wl.CONFIGS[1].scaled(B=2, Hq=8, Hkv=2, L=4300, K=12, seed=36)
+    fast_or_skip(cfg, False, W=W, Hl=cfg.Hq)
+    inp = wl.make_prefill_inputs(cfg, "cpu")
+    g = torch.Generator().manual_seed(11)
+    inp["landmarks"] = (torch.randn((cfg.B, cfg.Hq, cfg.C, cfg.d), generator=g) * 0.7).to(torch.bfloat16)
+    bias = torch.rand((cfg.B, cfg.Hq, cfg.C), generator=g) * float(np.log(cfg.S))
+    out, lse, sel = run_prefill(cfg, inp, "fast", bias=bias, W=W)
+    check_prefill(cfg, inp, out, lse, sel, bias=bias, W=W)
+
+
 @pytest.mark.parametrize("impl", ["generic", "fast"])
 def test_prefill_bias_only(impl):
     cfg = wl.CONFIGS[1].scaled(L=1536, K=6, seed=32)
