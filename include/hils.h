@@ -116,7 +116,7 @@ int hils_decode(const hils_params* params, const void* q, const void* k_cache, c
  *  - Limit: 256 + hils_workspace_bytes(params, 1) must fit in 8 MiB, otherwise HILS_ERR_WORKSPACE is
  *    returned before anything is launched (both benchmark decode shapes fit: B=64 x 64K tokens with
  *    K=32 needs about 5.3 MiB, B=4 x 1M tokens with K=64 about 2.5 MiB).  Shapes outside the
- *    bandwidth-tuned decode kernels (bf16, d=128, chunk 64, window <= 897, one landmark per KV head,
+ *    bandwidth-tuned decode kernels (bf16, d=128, chunk 64, window <= 897, one landmark per KV or per query head,
  *    at most 8 query heads per KV head) return HILS_ERR_UNSUPPORTED.
  *  - The first call on each device looks up the array's device address (with that device current);
  *    make that first call outside any stream capture.
@@ -151,7 +151,7 @@ int hils_prefill_at(const hils_params* params, const void* q, const void* k, con
  *                    attended: c <= (seq_lens[b]-1)/S); params->C is its row length, params->T_max = C * S
  *   landmarks, bias  stay logical: [B, Hl, C, d] / [B, Hl, C]
  * A page id outside [0, num_pages) sets the device status to HILS_ERR_DEVICE_INDEX and the chunk is skipped.
- * Supported by the bandwidth-tuned decode kernels only (bf16, d = 128, S = 64, one landmark per KV head, at most 8
+ * Supported by the bandwidth-tuned decode kernels only (bf16, d = 128, S = 64, at most 8
  * query heads per KV head); other shapes return HILS_ERR_UNSUPPORTED.  Workspace as for hils_decode. */
 int hils_decode_paged(const hils_params* params, const void* q, const void* k_pages, const void* v_pages,
                       const void* landmarks, const float* bias, const int32_t* block_table, int32_t num_pages,

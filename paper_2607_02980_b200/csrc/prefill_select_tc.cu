@@ -262,40 +262,40 @@ prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             if (!ok) break;
             tc_fence_after_sync();
             const bool tail = (it + 1) * kS > my_ncand;     // only the last step holds chunks this token may not see
+            // 8 candidates x 4 heads per round: a short loop body (the code has to stay resident close to the core)
 #pragma unroll 1
-            for (int cb = 0; cb < 4; ++cb) {
-                float r[4][16];
-                const uint32_t col = t_lane + buf * 256 + cb * 16;
-                tmem_ld16x4(col, col + kS, col + 2 * kS, col + 3 * kS, r);
-                const int c0 = it * kS + cb * 16;
+            for (int cb = 0; cb < 8; ++cb) {
+                float r[4][8];
+                const uint32_t col = t_lane + buf * 256 + cb * 8;
+                tmem_ld8x4(col, col + kS, col + 2 * kS, col + 3 * kS, r);
+                const int c0 = it * kS + cb * 8;
                 // first filter on the score alone (ties pass and are settled on the full key when merging);
                 // branch-free append: the slot is written always and kept only when the candidate passes
-                auto offer = [&](float u, int c, int j) {
+                auto offer = [&](float u, int c) {
                     const bool pass = u >= tau_f && (!tail || c < my_ncand);
                     myq[qn * kTileTok] = (static_cast<unsigned long long>(__float_as_uint(u)) << 32) | static_cast<uint32_t>(c);
                     qn += pass ? 1 : 0;
-                    // at most 8 appends between checks: a buffer never overflows
-                    if ((j & 7) == 7 && __any_sync(kFullMask, qn > N - 8)) compact();
                 };
                 if (PERHEAD && bias != nullptr) {
-                    // every head adds its own bias before the maximum over the group (App. C); kept apart from
-                    // the common loop below, whose code must stay small
+                    // every head adds its own bias before the maximum over the group (App. C)
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
+                    for (int j = 0; j < 8; ++j) {
                         const int c = c0 + j, cc = min(c, s.C - 1);
                         offer(fmaxf(fmaxf(fmaf(r[0][j], s.scale, bias[cc]), fmaf(r[1][j], s.scale, bias[s.C + cc])),
                                     fmaxf(fmaf(r[2][j], s.scale, bias[2 * s.C + cc]), fmaf(r[3][j], s.scale, bias[3 * s.C + cc]))),
-                              c, j);
+                              c);
                     }
                 } else {
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
+                    for (int j = 0; j < 8; ++j) {
                         const int c = c0 + j;
                         float u = fmaxf(fmaxf(r[0][j], r[1][j]), fmaxf(r[2][j], r[3][j])) * s.scale;
                         if (bias) u += bias[min(c, s.C - 1)];
-                        offer(u, c, j);
+                        offer(u, c);
                     }
                 }
+                // at most 8 appends between checks: a buffer never overflows
+                if (__any_sync(kFullMask, qn > N - 8)) compact();
             }
             tc_fence_before_sync();
             __syncwarp();
