@@ -50,6 +50,7 @@ def _load():
         _lib.hils_oracle_rows.restype = ctypes.c_int
         _lib.hils_oracle_num_threads.restype = ctypes.c_int
         _lib.hils_oracle_landmarks.restype = ctypes.c_int
+        _lib.hils_oracle_rows_routed.restype = ctypes.c_int
     return _lib
 
 
@@ -80,7 +81,7 @@ def _ptr(a: Optional[np.ndarray], ct):
 
 def hils_rows(q, k, v, landmarks, bias, *, S: int, K: int, W: int = 1, scale: float = 0.0,
               row_b, row_qi, row_pos, sel_idx=None, attend: bool = True, group_mode: int = 0,
-              want_alpha: bool = False):
+              want_alpha: bool = False, q_route=None):
     """Run the oracle on a list of query rows.
 
     q [B,Hq,Lq,d]; k,v [B,Hkv,T,d]; landmarks [B,Hl,C,d]; bias [B,Hl,C] or None.
@@ -93,6 +94,10 @@ def hils_rows(q, k, v, landmarks, bias, *, S: int, K: int, W: int = 1, scale: fl
     in_bf16 = int(all(_is_bf16(t) for t in (q, k, v, landmarks)))
     conv = _raw_bf16 if in_bf16 else _f32
     q = conv(q); k = conv(k); v = conv(v); landmarks = conv(landmarks)
+    # routing query (Eq. Q-Cal): replaces q in the surrogate scores only; same shape and dtype as q
+    qr = None if q_route is None else conv(q_route)
+    if qr is not None and qr.shape != q.shape:
+        raise ValueError("q_route must have the shape of q")
     bias_a = None if bias is None else _f32(bias)
     B, Hq, Lq, d = q.shape
     _, Hkv, T, _ = k.shape
@@ -112,8 +117,9 @@ def hils_rows(q, k, v, landmarks, bias, *, S: int, K: int, W: int = 1, scale: fl
     out = np.zeros((n, Hq, d), dtype=np.float64) if attend else None
     lse = np.zeros((n, Hq), dtype=np.float64) if attend else None
     alpha = np.zeros((n, Hq, K + 1), dtype=np.float64) if (attend and want_alpha) else None
-    rc = lib.hils_oracle_rows(
-        ctypes.byref(p), ctypes.c_void_p(q.ctypes.data), ctypes.c_void_p(k.ctypes.data),
+    rc = lib.hils_oracle_rows_routed(
+        ctypes.byref(p), ctypes.c_void_p(q.ctypes.data), ctypes.c_void_p(None if qr is None else qr.ctypes.data),
+        ctypes.c_void_p(k.ctypes.data),
         ctypes.c_void_p(v.ctypes.data), ctypes.c_void_p(landmarks.ctypes.data), _ptr(bias_a, ctypes.c_float),
         ctypes.c_int64(n), _ptr(row_b, ctypes.c_int32), _ptr(row_qi, ctypes.c_int32),
         _ptr(row_pos, ctypes.c_int64), ctypes.c_int(sel_mode), ctypes.c_int(1 if attend else 0),
@@ -128,7 +134,7 @@ def hils_rows(q, k, v, landmarks, bias, *, S: int, K: int, W: int = 1, scale: fl
 
 
 def hils_prefill(q, k, v, landmarks, bias=None, *, S: int, K: int, W: int = 1, scale: float = 0.0,
-                 rows=None, sel_idx=None, group_mode: int = 0, want_alpha: bool = False):
+                 rows=None, sel_idx=None, group_mode: int = 0, want_alpha: bool = False, q_route=None):
     """Prefill oracle: every position (or the positions in ``rows``) of every sequence.
 
     Returns arrays shaped [B, n_rows, ...]: sel_idx [B,n,Hkv,K], margin [B,n,Hkv],
@@ -143,12 +149,12 @@ def hils_prefill(q, k, v, landmarks, bias=None, *, S: int, K: int, W: int = 1, s
         sel_idx = np.asarray(sel_idx).reshape(B * n, -1, K)
     res = hils_rows(q, k, v, landmarks, bias, S=S, K=K, W=W, scale=scale, row_b=row_b,
                     row_qi=row_pos.astype(np.int32), row_pos=row_pos, sel_idx=sel_idx,
-                    group_mode=group_mode, want_alpha=want_alpha)
+                    group_mode=group_mode, want_alpha=want_alpha, q_route=q_route)
     return {key: val.reshape((B, n) + val.shape[1:]) for key, val in res.items() if val is not None}
 
 
 def hils_decode(q, k_cache, v_cache, landmarks, bias, seq_lens, *, S: int, K: int, W: int = 1,
-                scale: float = 0.0, sel_idx=None, group_mode: int = 0, want_alpha: bool = False):
+                scale: float = 0.0, sel_idx=None, group_mode: int = 0, want_alpha: bool = False, q_route=None):
     """Decode oracle: one query per sequence at position seq_lens[b]-1 (its own k,v are in the cache).
 
     q [B,Hq,d].  Returns sel_idx [B,Hkv,K], margin [B,Hkv], out [B,Hq,d], lse [B,Hq].
@@ -156,9 +162,12 @@ def hils_decode(q, k_cache, v_cache, landmarks, bias, seq_lens, *, S: int, K: in
     qn = q if _is_bf16(q) else _f32(q)
     B, Hq, d = qn.shape
     seq = np.asarray(seq_lens.cpu() if hasattr(seq_lens, "cpu") else seq_lens, dtype=np.int64)
+    qr = None
+    if q_route is not None:
+        qr = (q_route if _is_bf16(q_route) else _f32(q_route)).reshape(B, Hq, 1, d)
     return hils_rows(qn.reshape(B, Hq, 1, d), k_cache, v_cache, landmarks, bias, S=S, K=K, W=W,
                      scale=scale, row_b=np.arange(B, dtype=np.int32), row_qi=np.zeros(B, dtype=np.int32),
-                     row_pos=seq - 1, sel_idx=sel_idx, group_mode=group_mode, want_alpha=want_alpha)
+                     row_pos=seq - 1, sel_idx=sel_idx, group_mode=group_mode, want_alpha=want_alpha, q_route=qr)
 
 
 def hils_landmarks(lq, k, seq_lens=None, *, S: int, scale: float = 0.0):

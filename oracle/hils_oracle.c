@@ -129,8 +129,11 @@ static double attend_span(const void *q, size_t iq, const void *k, const void *v
  * out [n_rows, Hq, d]; lse [n_rows, Hq]; alpha [n_rows, Hq, K+1] (selected slots, then local).
  * Returns 0, or -1 on bad arguments.
  */
-int hils_oracle_rows(const hils_oracle_params *p,
-                     const void *q, const void *k, const void *v,
+/* q_route: the routing query q-hat of Eq. (Q-Cal) (q-hat = q + W_up W_down h, computed upstream), same shape as q;
+ * it replaces q in the surrogate scores s^h_c only (selection and fusion weights), never in the token-level
+ * attention.  NULL means q-hat = q. */
+static int rows_impl(const hils_oracle_params *p,
+                     const void *q, const void *q_route, const void *k, const void *v,
                      const void *landmarks, const float *bias,
                      int64_t n_rows, const int32_t *row_b, const int32_t *row_qi,
                      const int64_t *row_pos,
@@ -138,6 +141,7 @@ int hils_oracle_rows(const hils_oracle_params *p,
                      int32_t *sel_idx, double *margin,
                      double *out, double *lse, double *alpha)
 {
+    const void *qs = q_route ? q_route : q;
     if (!p || p->Hq % p->Hkv != 0 || (p->Hl != p->Hkv && p->Hl != p->Hq) || p->S <= 0 ||
         p->K < 0 || p->W < 1 || !sel_idx)
         return -1;
@@ -171,7 +175,7 @@ int hils_oracle_rows(const hils_oracle_params *p,
             const size_t iq = (((size_t)b * p->Hq + h) * p->Lq + row_qi[r]) * d;
             for (int c = 0; c < ncand; ++c) {
                 const size_t ilm = (((size_t)b * p->Hl + hl) * p->C + c) * d;
-                double s = scale * dotx(q, iq, landmarks, ilm, d, bf);
+                double s = scale * dotx(qs, iq, landmarks, ilm, d, bf);
                 if (bias) s += (double)bias[((size_t)b * p->Hl + hl) * p->C + c];
                 shat[rr * ncand + c] = s;
             }
@@ -267,6 +271,32 @@ int hils_oracle_num_threads(void) {
 #endif
 }
 
+
+int hils_oracle_rows(const hils_oracle_params *p,
+                     const void *q, const void *k, const void *v,
+                     const void *landmarks, const float *bias,
+                     int64_t n_rows, const int32_t *row_b, const int32_t *row_qi,
+                     const int64_t *row_pos,
+                     int sel_mode, int do_attend,
+                     int32_t *sel_idx, double *margin,
+                     double *out, double *lse, double *alpha)
+{
+    return rows_impl(p, q, NULL, k, v, landmarks, bias, n_rows, row_b, row_qi, row_pos, sel_mode, do_attend, sel_idx,
+                     margin, out, lse, alpha);
+}
+
+int hils_oracle_rows_routed(const hils_oracle_params *p,
+                            const void *q, const void *q_route, const void *k, const void *v,
+                            const void *landmarks, const float *bias,
+                            int64_t n_rows, const int32_t *row_b, const int32_t *row_qi,
+                            const int64_t *row_pos,
+                            int sel_mode, int do_attend,
+                            int32_t *sel_idx, double *margin,
+                            double *out, double *lse, double *alpha)
+{
+    return rows_impl(p, q, q_route, k, v, landmarks, bias, n_rows, row_b, row_qi, row_pos, sel_mode, do_attend,
+                     sel_idx, margin, out, lse, alpha);
+}
 
 /*
  * Chunk summaries of Proposition 3.1 (Eq. LogSumExp linearization / Eq. prop_q_c).

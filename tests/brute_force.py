@@ -9,13 +9,16 @@ from the C oracle on purpose.  Used only to pin the oracle.
 import numpy as np
 
 
-def brute_force_prefill(q, k, v, landmarks, bias, S, K, W=1, scale=None):
+def brute_force_prefill(q, k, v, landmarks, bias, S, K, W=1, scale=None, q_route=None):
     """q [Hq,L,d], k,v [Hkv,L,d], landmarks [Hl,C,d], bias [Hl,C] or None (one sequence).
+
+    q_route [Hq,L,d] or None: the routing query of Eq. (Q-Cal); it takes q's place in the surrogate scores only.
 
     Returns (out [Hq,L,d], lse [Hq,L], sel list-of-lists [Hkv][L] (ascending ids), weights [Hq,L,L]).
     """
     q = np.asarray(q, np.float64); k = np.asarray(k, np.float64); v = np.asarray(v, np.float64)
     landmarks = np.asarray(landmarks, np.float64)
+    qhat = q if q_route is None else np.asarray(q_route, np.float64)
     Hq, L, d = q.shape
     Hkv = k.shape[0]
     Hl = landmarks.shape[0]
@@ -32,7 +35,7 @@ def brute_force_prefill(q, k, v, landmarks, bias, S, K, W=1, scale=None):
                 h = g * G + r
                 hl = h if Hl == Hq else g
                 for c in range(ncand):
-                    shat[r, c] = scale * (q[h, i] @ landmarks[hl, c]) + (0.0 if bias is None else bias[hl, c])
+                    shat[r, c] = scale * (qhat[h, i] @ landmarks[hl, c]) + (0.0 if bias is None else bias[hl, c])
             u = shat.max(axis=0) if ncand > 0 else np.zeros(0)
             order = sorted(range(ncand), key=lambda c: (-u[c], c))
             chosen = sorted(order[:K])

@@ -378,3 +378,33 @@ def test_normalised_group_mode_is_available_and_differs_only_in_selection():
     b = oracle.hils_prefill(q, k, v, lm, None, S=S, K=K, group_mode=1)
     assert (a["sel_idx"] == b["sel_idx"]).all()
     np.testing.assert_allclose(a["out"], b["out"], atol=0)
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# Routing query (Eq. Q-Cal): q-hat replaces q in the surrogate scores only
+def test_routing_query_equal_to_q_changes_nothing_and_a_different_one_only_moves_scores():
+    rng = np.random.default_rng(77)
+    B, Hq, Hkv, L, d, S, K = 1, 4, 2, 96, 8, 8, 3
+    q = rng.standard_normal((B, Hq, L, d)).astype(np.float32)
+    qr = rng.standard_normal((B, Hq, L, d)).astype(np.float32)
+    k = rng.standard_normal((B, Hkv, L, d)).astype(np.float32)
+    v = rng.standard_normal((B, Hkv, L, d)).astype(np.float32)
+    lm = rng.standard_normal((B, Hkv, L // S, d)).astype(np.float32)
+    bias = rng.random((B, Hkv, L // S)).astype(np.float32)
+    base = oracle.hils_prefill(q, k, v, lm, bias, S=S, K=K)
+    same = oracle.hils_prefill(q, k, v, lm, bias, S=S, K=K, q_route=q)
+    assert (same["sel_idx"] == base["sel_idx"]).all() and np.array_equal(same["out"], base["out"])
+    # a different routing query: the independent brute force (dense weights from App. C) agrees ...
+    routed = oracle.hils_prefill(q, k, v, lm, bias, S=S, K=K, q_route=qr)
+    bo, blse, bsel, _ = brute_force_prefill(q[0], k[0], v[0], lm[0], bias[0], S, K, q_route=qr[0])
+    assert np.allclose(routed["out"][0].transpose(1, 0, 2), bo, atol=1e-10)
+    assert np.allclose(routed["lse"][0].T, blse, atol=1e-10)
+    for g in range(Hkv):
+        for i in range(L):
+            got = [c for c in routed["sel_idx"][0, i, g] if c >= 0]
+            assert got == bsel[g][i]
+    # ... the selection is the one q-hat alone would make, and rows without candidates (first chunk) do not move
+    alone = oracle.hils_prefill(qr, k, v, lm, bias, S=S, K=K)
+    assert (routed["sel_idx"] == alone["sel_idx"]).all()
+    assert np.array_equal(routed["out"][:, :S], base["out"][:, :S])
+    assert not np.allclose(routed["out"][:, S * (K + 2):], base["out"][:, S * (K + 2):])
