@@ -130,6 +130,19 @@ int hils_decode_noalloc(const hils_params* params, const void* q, const void* k_
                         const void* landmarks, const float* bias, const int32_t* seq_lens,
                         void* out, float* lse, int32_t* sel_idx, int32_t* device_status, void* stream);
 
+/* The operators with a separate ROUTING QUERY q-hat (Eq. Q-Cal: q-hat = q + W_up W_down h, computed upstream by
+ * the model).  q_route has the shape, dtype and alignment of q; it takes q's place in the surrogate scores
+ * s^h_c = scale * q-hat^h . k'_c + b'_c -- i.e. in the selection and in the fusion weights -- and nowhere else
+ * (token-level attention inside the selected chunks and the local window uses q).  Everything else as
+ * hils_prefill / hils_decode, same workspace. */
+int hils_prefill_routed(const hils_params* params, const void* q, const void* q_route, const void* k, const void* v,
+                        const void* landmarks, const float* bias, void* out, float* lse, int32_t* sel_idx,
+                        void* workspace, size_t workspace_bytes, void* stream);
+int hils_decode_routed(const hils_params* params, const void* q, const void* q_route, const void* k_cache,
+                       const void* v_cache, const void* landmarks, const float* bias, const int32_t* seq_lens,
+                       void* out, float* lse, int32_t* sel_idx, void* workspace, size_t workspace_bytes,
+                       void* stream);
+
 /* hils_prefill for a SLICE of a sequence: the L query tokens sit at positions pos0 .. pos0 + L - 1 of sequences
  * whose caches already hold at least pos0 + L tokens (chunked prefill; with small L, multi-token decode as used by
  * speculative decoding).  Same operator: query row r is treated exactly like position pos0 + r of hils_prefill.

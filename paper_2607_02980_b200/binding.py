@@ -25,6 +25,7 @@ EXPORTS = [
     "hils_prefill_host", "hils_decode_host", "hils_poll_status", "hils_last_launch_count",
     "hils_status_string", "hils_version", "hils_trace_enable", "hils_trace_read", "hils_decode_noalloc",
     "hils_landmark_summary", "hils_decode_paged", "hils_prefill_at", "hils_prefill_at_workspace_bytes",
+    "hils_prefill_routed", "hils_decode_routed",
 ]
 
 
@@ -70,6 +71,10 @@ def load_library() -> ctypes.CDLL:
     lib.hils_decode_host.argtypes = [pp, vp, vp, vp, vp, f32p, i32p, vp, f32p, i32p, vp, ctypes.c_size_t, vp]
     lib.hils_decode_noalloc.restype = ctypes.c_int
     lib.hils_decode_noalloc.argtypes = [pp, vp, vp, vp, vp, f32p, i32p, vp, f32p, i32p, i32p, vp]
+    lib.hils_prefill_routed.restype = ctypes.c_int
+    lib.hils_prefill_routed.argtypes = [pp, vp, vp, vp, vp, vp, f32p, vp, f32p, i32p, vp, ctypes.c_size_t, vp]
+    lib.hils_decode_routed.restype = ctypes.c_int
+    lib.hils_decode_routed.argtypes = [pp, vp, vp, vp, vp, vp, f32p, i32p, vp, f32p, i32p, vp, ctypes.c_size_t, vp]
     lib.hils_prefill_at.restype = ctypes.c_int
     lib.hils_prefill_at.argtypes = [pp, vp, vp, vp, vp, f32p, ctypes.c_int64, vp, f32p, i32p, vp, ctypes.c_size_t, vp]
     lib.hils_prefill_at_workspace_bytes.restype = ctypes.c_size_t
@@ -155,8 +160,9 @@ def _stream_ptr(stream) -> ctypes.c_void_p:
 
 
 def hils_prefill(q, k, v, landmarks, chunk_size: int, top_k: int, out=None, lse=None, sel_idx=None, stream=None, *,
-                 bias=None, window: int = 1, scale: float = 0.0, impl: str = "auto", workspace=None):
+                 bias=None, window: int = 1, scale: float = 0.0, impl: str = "auto", workspace=None, q_route=None):
     """HiLS prefill on CUDA tensors: q [B,Hq,L,d], k,v [B,Hkv,L,d], landmarks [B,Hl,C,d].
+    q_route (optional, shape of q): the routing query of Eq. (Q-Cal), used for the surrogate scores only.
 
     Returns (out [B,Hq,L,d], lse [B,Hq,L] fp32, sel_idx [B,Hkv,L,K] int32).  Asynchronous on the
     given (default: current) CUDA stream.
@@ -181,8 +187,14 @@ def hils_prefill(q, k, v, landmarks, chunk_size: int, top_k: int, out=None, lse=
     p = make_params(B=B, Hq=Hq, Hkv=Hkv, Hl=Hl, L=L, T_max=T, C=C, d=d, chunk_size=chunk_size, top_k=top_k,
                     window=window, scale=scale, dtype=_dtype_code(q), impl=impl)
     ws = alloc_workspace(p, False, q.device) if workspace is None else workspace
-    rc = lib.hils_prefill(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(landmarks), _ptr(bias), _ptr(out),
-                          _ptr(lse), _ptr(sel_idx), _ptr(ws), ws.numel(), _stream_ptr(stream))
+    if q_route is not None:
+        _check(q_route, "q_route", (B, Hq, L, d), dt, True)
+        rc = lib.hils_prefill_routed(ctypes.byref(p), _ptr(q), _ptr(q_route), _ptr(k), _ptr(v), _ptr(landmarks),
+                                     _ptr(bias), _ptr(out), _ptr(lse), _ptr(sel_idx), _ptr(ws), ws.numel(),
+                                     _stream_ptr(stream))
+    else:
+        rc = lib.hils_prefill(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(landmarks), _ptr(bias), _ptr(out),
+                              _ptr(lse), _ptr(sel_idx), _ptr(ws), ws.numel(), _stream_ptr(stream))
     if rc != 0:
         raise HilsError(rc, "hils_prefill")
     return out, lse, sel_idx
@@ -190,7 +202,7 @@ def hils_prefill(q, k, v, landmarks, chunk_size: int, top_k: int, out=None, lse=
 
 def hils_decode(q, k_cache, v_cache, landmarks, seq_lens, chunk_size: int, top_k: int, out=None, lse=None,
                 sel_idx=None, stream=None, *, bias=None, window: int = 1, scale: float = 0.0, impl: str = "auto",
-                workspace=None):
+                workspace=None, q_route=None):
     """HiLS single-token decode: q [B,Hq,d], caches [B,Hkv,T_max,d], seq_lens [B] int32 (CUDA).
 
     Returns (out [B,Hq,d], lse [B,Hq], sel_idx [B,Hkv,K])."""
@@ -215,9 +227,15 @@ def hils_decode(q, k_cache, v_cache, landmarks, seq_lens, chunk_size: int, top_k
     p = make_params(B=B, Hq=Hq, Hkv=Hkv, Hl=Hl, L=0, T_max=T, C=C, d=d, chunk_size=chunk_size, top_k=top_k,
                     window=window, scale=scale, dtype=_dtype_code(q), impl=impl)
     ws = alloc_workspace(p, True, q.device) if workspace is None else workspace
-    rc = lib.hils_decode(ctypes.byref(p), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(landmarks), _ptr(bias),
-                         _ptr(seq_lens), _ptr(out), _ptr(lse), _ptr(sel_idx), _ptr(ws), ws.numel(),
-                         _stream_ptr(stream))
+    if q_route is not None:
+        _check(q_route, "q_route", tuple(q.shape), q.dtype, True)
+        rc = lib.hils_decode_routed(ctypes.byref(p), _ptr(q), _ptr(q_route), _ptr(k_cache), _ptr(v_cache), _ptr(landmarks),
+                                    _ptr(bias), _ptr(seq_lens), _ptr(out), _ptr(lse), _ptr(sel_idx), _ptr(ws), ws.numel(),
+                                    _stream_ptr(stream))
+    else:
+        rc = lib.hils_decode(ctypes.byref(p), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(landmarks), _ptr(bias),
+                             _ptr(seq_lens), _ptr(out), _ptr(lse), _ptr(sel_idx), _ptr(ws), ws.numel(),
+                             _stream_ptr(stream))
     if rc != 0:
         raise HilsError(rc, "hils_decode")
     return out, lse, sel_idx

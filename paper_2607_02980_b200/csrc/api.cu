@@ -106,7 +106,8 @@ size_t scratch_bytes(const Shape& s, Path path) {
 
 int run(const hils_params* p, int is_decode, const void* q, const void* k, const void* v, const void* lm,
         const float* bias, const int32_t* seq_lens, void* out, float* lse, int32_t* sel, void* ws,
-        size_t ws_bytes, void* stream_v, const int32_t* block_table = nullptr, int num_pages = 0, long long pos0 = 0) {
+        size_t ws_bytes, void* stream_v, const int32_t* block_table = nullptr, int num_pages = 0, long long pos0 = 0,
+        const void* q_route = nullptr) {
     g_last_launches = 0;
     Shape s;
     int rc = make_shape(p, is_decode, &s, pos0);
@@ -132,6 +133,8 @@ int run(const hils_params* p, int is_decode, const void* q, const void* k, const
               static_cast<char*>(ws) + kStatusBytes, ws_bytes - kStatusBytes};
     t.block_table = block_table;
     t.num_pages = num_pages;
+    if (q_route && !aligned16(q_route)) return HILS_ERR_ALIGNMENT;
+    t.q_route = q_route;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_v);
     trace_begin(stream);
     int n;
@@ -354,6 +357,23 @@ int hils_decode(const hils_params* params, const void* q, const void* k_cache, c
                 int32_t* sel_idx, void* workspace, size_t workspace_bytes, void* stream) {
     return run(params, 1, q, k_cache, v_cache, landmarks, bias, seq_lens, out, lse, sel_idx, workspace,
                workspace_bytes, stream);
+}
+
+int hils_prefill_routed(const hils_params* params, const void* q, const void* q_route, const void* k, const void* v,
+                        const void* landmarks, const float* bias, void* out, float* lse, int32_t* sel_idx,
+                        void* workspace, size_t workspace_bytes, void* stream) {
+    if (!q_route) return HILS_ERR_INVALID_ARG;
+    return run(params, 0, q, k, v, landmarks, bias, nullptr, out, lse, sel_idx, workspace, workspace_bytes, stream,
+               nullptr, 0, 0, q_route);
+}
+
+int hils_decode_routed(const hils_params* params, const void* q, const void* q_route, const void* k_cache,
+                       const void* v_cache, const void* landmarks, const float* bias, const int32_t* seq_lens,
+                       void* out, float* lse, int32_t* sel_idx, void* workspace, size_t workspace_bytes,
+                       void* stream) {
+    if (!q_route) return HILS_ERR_INVALID_ARG;
+    return run(params, 1, q, k_cache, v_cache, landmarks, bias, seq_lens, out, lse, sel_idx, workspace,
+               workspace_bytes, stream, nullptr, 0, 0, q_route);
 }
 
 int hils_prefill_at(const hils_params* params, const void* q, const void* k, const void* v, const void* landmarks,

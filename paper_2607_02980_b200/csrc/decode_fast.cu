@@ -34,6 +34,7 @@ constexpr float kLog2e = 1.4426950408889634f;
 struct DArgs {
     Shape s;
     const __nv_bfloat16* q;
+    const __nv_bfloat16* q_route;  // routing query for the surrogate scores (= q unless a separate one was given)
     const __nv_bfloat16* lm;
     const float* bias;
     const int32_t* seq_lens;
@@ -325,7 +326,7 @@ __device__ void select_pair(const DArgs& a, int pair, int ncand, SelShared& sh, 
     __nv_bfloat16 (*lm_s)[kD + 8] = reinterpret_cast<__nv_bfloat16 (*)[kD + 8]>(dyn);
     const int per = s.Hl / s.Hkv;                        // landmark rows per chunk: 1, or one per query head (G)
     const long long lrow0 = (static_cast<long long>(b) * s.Hl + g * per) * s.C;      // landmark head 0 of this KV head
-    const __nv_bfloat16* qg = a.q + (static_cast<long long>(b) * s.Hq + g * G) * kD;
+    const __nv_bfloat16* qg = a.q_route + (static_cast<long long>(b) * s.Hq + g * G) * kD;     // fusion scores: q-hat
     for (int x = tid; x < G * 16; x += NT)
         *reinterpret_cast<uint4*>(&sh.q_s[x >> 4][(x & 15) * 8]) = *reinterpret_cast<const uint4*>(qg + (x >> 4) * kD + (x & 15) * 8);
     const int tstep = 64 / per;                          // selected chunks staged per round (64 landmark rows)
@@ -404,7 +405,7 @@ __global__ void __launch_bounds__(kScoreThreads) decode_score_kernel(const DArgs
 #pragma unroll
     for (int kb = 0; kb < 4; ++kb) qf[kb] = make_uint4(0u, 0u, 0u, 0u);
     if (gq < s.G) {
-        const __nv_bfloat16* qrow = a.q + (static_cast<long long>(b) * s.Hq + g * s.G + gq) * kD;
+        const __nv_bfloat16* qrow = a.q_route + (static_cast<long long>(b) * s.Hq + g * s.G + gq) * kD;
 #pragma unroll
         for (int kb = 0; kb < 4; ++kb) qf[kb] = *reinterpret_cast<const uint4*>(qrow + kb * 32 + t * 8);
     }
@@ -845,6 +846,7 @@ int launch_decode_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
     DArgs a;
     a.s = s;
     a.q = static_cast<const __nv_bfloat16*>(t.q);
+    a.q_route = static_cast<const __nv_bfloat16*>(t.q_route ? t.q_route : t.q);
     a.lm = static_cast<const __nv_bfloat16*>(t.landmarks);
     a.bias = t.bias;
     a.seq_lens = t.seq_lens;

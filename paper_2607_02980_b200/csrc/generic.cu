@@ -13,6 +13,7 @@ constexpr int kWarpsPerBlock = 4;
 struct GArgs {
     Shape s;
     const void* q;
+    const void* q_route;   // routing query for the surrogate scores (= q unless a separate one was given)
     const void* k;
     const void* v;
     const void* lm;
@@ -75,7 +76,7 @@ generic_select_kernel(const GArgs a) {
     const int ncand = local_lo(pos, s.W, s.S) / s.S;
     const int d = s.d, G = s.G;
     float* sq = smem + static_cast<size_t>(wib) * G * d;        // [G][d] queries of the group
-    const T* q = static_cast<const T*>(a.q);
+    const T* q = static_cast<const T*>(a.q_route);       // selection scores use the routing query
     for (int x = lane; x < G * d; x += 32) {
         const int rr = x / d, t = x % d;
         sq[x] = to_f32(q[((static_cast<long long>(b) * s.Hq + g * G + rr) * s.R + r) * d + t]);
@@ -210,9 +211,11 @@ generic_attend_kernel(const GArgs a) {
     }
     const int lo = local_lo(pos, s.W, s.S);
     const int ncand = lo / s.S;
-    float* sq = smem + static_cast<size_t>(wib) * d;
+    float* sq = smem + static_cast<size_t>(wib) * 2 * d;        // attention query, then routing query
+    float* sr = sq + d;
     const T* q = static_cast<const T*>(a.q) + orow * d;
-    for (int t = lane; t < d; t += 32) sq[t] = to_f32(q[t]);
+    const T* qr = static_cast<const T*>(a.q_route) + orow * d;
+    for (int t = lane; t < d; t += 32) { sq[t] = to_f32(q[t]); sr[t] = to_f32(qr[t]); }
     __syncwarp();
 
     const T* kg = static_cast<const T*>(a.k) + (static_cast<long long>(b) * s.Hkv + g) * s.T * d;
@@ -238,7 +241,7 @@ generic_attend_kernel(const GArgs a) {
             continue;
         }
         float dotp = 0.f;
-        for (int x = lane; x < d; x += 32) dotp = fmaf(sq[x], to_f32(lm[static_cast<long long>(c) * d + x]), dotp);
+        for (int x = lane; x < d; x += 32) dotp = fmaf(sr[x], to_f32(lm[static_cast<long long>(c) * d + x]), dotp);
         float lam = warp_sum(dotp) * s.scale;
         if (bias) lam += bias[c];
         attend_span<T, NE>(sq, kg, vg, c * s.S, (c + 1) * s.S, d, s.scale, lane, m, Z, part);
@@ -265,7 +268,7 @@ int launch_typed(const GArgs& a, cudaStream_t stream) {
     const unsigned sel_blocks = static_cast<unsigned>((sel_warps + kWarpsPerBlock - 1) / kWarpsPerBlock);
     const unsigned att_blocks = static_cast<unsigned>((att_warps + kWarpsPerBlock - 1) / kWarpsPerBlock);
     const size_t sel_smem = sizeof(float) * kWarpsPerBlock * s.G * s.d;
-    const size_t att_smem = sizeof(float) * kWarpsPerBlock * s.d;
+    const size_t att_smem = sizeof(float) * kWarpsPerBlock * 2 * s.d;
     const int nr = (s.K + 31) / 32;
     if (nr <= 1) generic_select_kernel<T, 1><<<sel_blocks, kWarpsPerBlock * 32, sel_smem, stream>>>(a);
     else if (nr == 2) generic_select_kernel<T, 2><<<sel_blocks, kWarpsPerBlock * 32, sel_smem, stream>>>(a);
@@ -290,7 +293,7 @@ bool generic_supports(const Shape& s) {
 
 int launch_generic(const Shape& s, int dtype, const Tensors& t, cudaStream_t stream) {
     if (!generic_supports(s)) return HILS_ERR_UNSUPPORTED;
-    GArgs a{s, t.q, t.k, t.v, t.landmarks, t.bias, t.seq_lens, t.out, t.lse, t.sel_idx, t.status};
+    GArgs a{s, t.q, t.q_route ? t.q_route : t.q, t.k, t.v, t.landmarks, t.bias, t.seq_lens, t.out, t.lse, t.sel_idx, t.status};
     if (dtype == HILS_F32) return launch_typed<float>(a, stream);
     return launch_typed<__nv_bfloat16>(a, stream);
 }

@@ -26,6 +26,8 @@ struct Tensors {
     // logical chunk to its page; NULL = contiguous caches
     const int32_t* block_table = nullptr;
     int num_pages = 0;
+    // routing query q-hat (Eq. Q-Cal), same shape as q: used for the surrogate scores only; NULL = q
+    const void* q_route = nullptr;
 };
 
 // Optional per-kernel timing: when tracing is on (hils_trace_enable), every launcher calls

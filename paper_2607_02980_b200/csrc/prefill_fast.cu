@@ -355,6 +355,40 @@ __global__ void invert_fill_kernel(const PArgs a) {
     }
 }
 
+// ------------------------------------------------------------------------------------------ routed scores
+// With a separate routing query q-hat (Eq. Q-Cal) the chunk mass of a selected slot is scale * q-hat . k'_c + b'_c,
+// not the q . k'_c that the attend kernel read off its score tile: this kernel overwrites those masses.  One CTA
+// per tile, one warp per entry at a time; lane l covers dimensions 4l .. 4l+3.  Local slots keep their masses.
+__global__ void __launch_bounds__(128) prefill_route_scores_kernel(const PArgs a) {
+    const Shape& s = a.s;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int t_begin = a.blk_toff[a.blk];
+    const int tile = t_begin + static_cast<int>(blockIdx.x);
+    if (tile >= a.blk_toff[a.blk + 1]) return;
+    const int4 rec = a.tiles[tile];
+    const int pair = rec.x, c = rec.y, first = rec.z, ntok = rec.w;
+    if (c >= s.C) return;
+    const int b = pair / s.Hkv, gk = pair % s.Hkv, per = s.Hl / s.Hkv;
+    const int e0 = t_begin * a.tile_tok;
+    for (int ei = warp; ei < ntok; ei += 4) {
+        const int e = a.entries[first + ei];
+        const int tok = a.i0 + (e >> 8), slot = e & 255;
+        if (slot >= s.K) continue;
+#pragma unroll
+        for (int h = 0; h < kG; ++h) {
+            const long long lrow = (static_cast<long long>(b) * s.Hl + gk * per + (per == 1 ? 0 : h)) * s.C + c;
+            const uint2 qv = *reinterpret_cast<const uint2*>(a.q + ((static_cast<long long>(b) * s.Hq + gk * kG + h) * s.R + tok) * kD + lane * 4);
+            const uint2 lv = *reinterpret_cast<const uint2*>(a.lm + lrow * kD + lane * 4);
+            float dotp = __uint_as_float(qv.x << 16) * __uint_as_float(lv.x << 16);
+            dotp = fmaf(__uint_as_float(qv.x & 0xffff0000u), __uint_as_float(lv.x & 0xffff0000u), dotp);
+            dotp = fmaf(__uint_as_float(qv.y << 16), __uint_as_float(lv.y << 16), dotp);
+            dotp = fmaf(__uint_as_float(qv.y & 0xffff0000u), __uint_as_float(lv.y & 0xffff0000u), dotp);
+            dotp = warp_sum(dotp);
+            if (lane == 0) a.lam[static_cast<long long>(first - e0 + ei) * kG + h] = dotp * s.scale + (a.bias ? a.bias[lrow] : 0.f);
+        }
+    }
+}
+
 // ------------------------------------------------------------------------------------------ fuse
 // One warp per (sequence, KV head, token): softmax over {surrogate scores of the selected chunks} U
 // {log Z_swa} per head (Eq. HiLS weights, inter-chunk factor) and the weighted sum of the rows that
@@ -537,7 +571,8 @@ int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
     char* sc = static_cast<char*>(t.scratch);
     PArgs a;
     a.s = s;
-    a.q = static_cast<const __nv_bfloat16*>(t.q);
+    // PArgs::q feeds the selection fallback and the routed-score kernel: the routing query (q itself unless given)
+    a.q = static_cast<const __nv_bfloat16*>(t.q_route ? t.q_route : t.q);
     a.lm = static_cast<const __nv_bfloat16*>(t.landmarks);
     a.bias = t.bias;
     a.out = static_cast<__nv_bfloat16*>(t.out);
@@ -584,7 +619,7 @@ int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
     int launches = 0;
     const int tiles_per_seq = (s.R + kS - 1) / kS;
     if (prefill_select_tc_supports(s) && !g_force_mma_select) {
-        const int rc = launch_prefill_select_tc(s, t.q, t.landmarks, t.bias, t.sel_idx, t.status, stream);
+        const int rc = launch_prefill_select_tc(s, a.q, t.landmarks, t.bias, t.sel_idx, t.status, stream);
         if (rc < 0) return rc;
     } else {
         prefill_select_kernel<<<static_cast<unsigned>(pairs) * tiles_per_seq, 160, sel_smem, stream>>>(map_lm, a);
@@ -621,6 +656,13 @@ int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
             if (rc < 0) return rc;
         }
         trace_mark("prefill_attend", stream);
+        if (t.q_route) {
+            const int ntl = (p.max_blk_tiles);
+            prefill_route_scores_kernel<<<static_cast<unsigned>(ntl), 128, 0, stream>>>(a);
+            if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
+            trace_mark("prefill_route_scores", stream);
+            ++launches;
+        }
         const long long fuse_warps = static_cast<long long>(pairs) * nblk;
         prefill_fuse_kernel<<<static_cast<unsigned>((fuse_warps + kFuseWarps - 1) / kFuseWarps), kFuseWarps * 32, 0, stream>>>(a);
         if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
