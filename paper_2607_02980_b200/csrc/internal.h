@@ -51,8 +51,10 @@ size_t decode_noalloc_capacity();
 
 // tcgen05 scoring + top-K for prefill (bf16, d = 128, S = 64, G = 4, K <= 32, any W).
 bool prefill_select_tc_supports(const Shape& s);
+// cnt (optional): [query blocks][pairs][nc] entry counts per chunk, accumulated by the kernel (zeroed by the
+// caller) when qb is a multiple of 128; returns 2 instead of 1 when it did so.
 int launch_prefill_select_tc(const Shape& s, const void* q, const void* landmarks, const float* bias, int32_t* sel,
-                             int* status, cudaStream_t stream);
+                             int* status, int* cnt, int qb, int nc, cudaStream_t stream);
 
 // tcgen05 chunk-major attention over the tile table built by the invert kernels (32-token tiles).
 int attend_tc_tile_tokens();

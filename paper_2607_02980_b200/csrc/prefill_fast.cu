@@ -618,9 +618,13 @@ int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
 
     int launches = 0;
     const int tiles_per_seq = (s.R + kS - 1) / kS;
+    // counters of the inverse index start at zero; the tcgen05 selection kernel fills the per-chunk entry counts itself
+    if (cudaMemsetAsync(sc + p.off_cnt, 0, p.zero_bytes, stream) != cudaSuccess) return HILS_ERR_CUDA;
+    bool counted = false;
     if (prefill_select_tc_supports(s) && !g_force_mma_select) {
-        const int rc = launch_prefill_select_tc(s, a.q, t.landmarks, t.bias, t.sel_idx, t.status, stream);
+        const int rc = launch_prefill_select_tc(s, a.q, t.landmarks, t.bias, t.sel_idx, t.status, a.cnt, a.qb, a.nc, stream);
         if (rc < 0) return rc;
+        counted = rc == 2;
     } else {
         prefill_select_kernel<<<static_cast<unsigned>(pairs) * tiles_per_seq, 160, sel_smem, stream>>>(map_lm, a);
         if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
@@ -630,19 +634,21 @@ int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
 
     // inverse index for every query block at once: per-(block, pair, chunk) lists of (token, slot) entries
     // and the table of attend tiles, grouped by block
-    if (cudaMemsetAsync(sc + p.off_cnt, 0, p.zero_bytes, stream) != cudaSuccess) return HILS_ERR_CUDA;
     {
         const long long elems = static_cast<long long>(pairs) * s.R * (s.K + max_local_slots(s.W));
         const long long want = (elems + 255) / 256;
         const unsigned eb = static_cast<unsigned>(want < 148 * 16 ? want : 148 * 16);
-        invert_count_kernel<<<eb, 256, 0, stream>>>(a);
+        if (!counted) {
+            invert_count_kernel<<<eb, 256, 0, stream>>>(a);
+            ++launches;
+        }
         const unsigned nseg = static_cast<unsigned>((static_cast<long long>(p.n_blocks) * pairs * p.nc + 1023) / 1024);
         invert_segsum_kernel<<<nseg, 1024, 0, stream>>>(a);
         invert_scan_kernel<<<nseg, 1024, 0, stream>>>(a);
         invert_fill_kernel<<<eb, 256, 0, stream>>>(a);
         if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
         trace_mark("prefill_invert", stream);
-        launches += 4;
+        launches += 3;
     }
     for (int i0 = 0, blk = 0; i0 < s.R; i0 += a.qb, ++blk) {
         a.i0 = i0;

@@ -31,6 +31,10 @@ struct TcArgs {
     const float* bias;
     int32_t* sel;
     int* status;
+    // optional: per-(query block, pair, chunk) counts of the (token, slot) entries that attend each chunk -- the
+    // first step of the inverse index, taken here because the selections are at hand (NULL: not wanted)
+    int* cnt;
+    int qb, nc;        // tokens per query block (a multiple of the 128-token tile), chunk slots per pair in cnt
 };
 
 struct TcSmem {
@@ -317,6 +321,32 @@ prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             }
             for (int e = cnt; e < K; ++e) sel[e] = -1;
         }
+        if (a.cnt) {
+            // chunk histogram of this tile's entries (selected chunks + the chunks of each token's local window) in the
+            // landmark ring's shared memory (every MMA that read it has completed), then one global add per used bin
+            int* hist = reinterpret_cast<int*>(lms);
+            const bool in_smem = a.nc * static_cast<int>(sizeof(int)) <= kLmStages * kLmStageBytes;
+            int* gcnt = a.cnt + (static_cast<long long>(ti * kTileTok / a.qb) * pairs + pair) * a.nc;
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (in_smem) {
+                for (int x = tid; x < a.nc; x += kTileTok) hist[x] = 0;
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+            }
+            if (tok < s.R) {
+                int* dst = in_smem ? hist : gcnt;
+                for (int e = 0; e < K; ++e) {
+                    const unsigned long long key = mytop[e * kTileTok];
+                    if (key != 0ull) atomicAdd(dst + key_chunk(key), 1);
+                }
+                const int pos = s.pos0 + tok;
+                for (int c = local_lo(pos, s.W, kS) / kS; c <= pos / kS; ++c) atomicAdd(dst + c, 1);
+            }
+            if (in_smem) {
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                for (int x = tid; x < a.nc; x += kTileTok)
+                    if (hist[x]) atomicAdd(gcnt + x, hist[x]);
+            }
+        }
     }
 
     tc_fence_before_sync();
@@ -332,7 +362,7 @@ bool prefill_select_tc_supports(const Shape& s) {
 }
 
 int launch_prefill_select_tc(const Shape& s, const void* q, const void* landmarks, const float* bias, int32_t* sel,
-                             int* status, cudaStream_t stream) {
+                             int* status, int* cnt, int qb, int nc, cudaStream_t stream) {
     const int pairs = s.B * s.Hkv;
     CUtensorMap map_q, map_lm;
     if (!make_bf16_2d_map(&map_q, q, static_cast<uint64_t>(s.B) * s.Hq * s.R, kD, 64, kTileTok) ||
@@ -353,7 +383,7 @@ int launch_prefill_select_tc(const Shape& s, const void* q, const void* landmark
             return HILS_ERR_CUDA;
         attr_done = true;
     }
-    TcArgs a{s, bias, sel, status};
+    TcArgs a{s, bias, sel, status, (cnt && qb % kTileTok == 0) ? cnt : nullptr, qb, nc};
     const int tiles = (s.R + kTileTok - 1) / kTileTok;
     const unsigned grid = static_cast<unsigned>(pairs) * tiles;
     const bool perhead = s.Hl != s.Hkv;
@@ -365,7 +395,7 @@ int launch_prefill_select_tc(const Shape& s, const void* q, const void* landmark
         else prefill_select_tc_kernel<32, false><<<grid, kThreads, smem, stream>>>(map_q, map_lm, a);
     }
     if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
-    return 1;
+    return a.cnt ? 2 : 1;
 }
 
 }  // namespace hils
