@@ -102,11 +102,6 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
 
     const Shape& s = a.s;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    // a.n_tiles points at {first tile of this query block, first tile of the next one}
-    const int t_begin = a.n_tiles[0], n_tiles = a.n_tiles[1] - t_begin;
-    const long long lo = t_begin + static_cast<long long>(blockIdx.x) * n_tiles / gridDim.x;
-    const long long hi = t_begin + static_cast<long long>(blockIdx.x + 1) * n_tiles / gridDim.x;
-
     if (tid == 0) {
         for (int i = 0; i < kQSlots; ++i) { mbar_init(&sm.q_full[i], 4); mbar_init(&sm.q_empty[i], 1); }
         for (int i = 0; i < kVBufs; ++i) { mbar_init(&sm.v_ready[i], 1); mbar_init(&sm.v_empty[i], 1); }
@@ -136,6 +131,15 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = sm.tmem_base;
+
+    // Everything above touched only this CTA's own shared and tensor memory, so it may overlap the tail of the
+    // previous kernel of the stream (the fusion of the previous query block, which still reads the partial outputs
+    // this kernel overwrites, or the inverse-index kernels).  From here on their results are needed.
+    pdl_wait();
+    // a.n_tiles points at {first tile of this query block, first tile of the next one}
+    const int t_begin = a.n_tiles[0], n_tiles = a.n_tiles[1] - t_begin;
+    const long long lo = t_begin + static_cast<long long>(blockIdx.x) * n_tiles / gridDim.x;
+    const long long hi = t_begin + static_cast<long long>(blockIdx.x + 1) * n_tiles / gridDim.x;
 
     // running counters (identical in every role): tiles and chunk loads processed so far by this CTA
     uint32_t tcount = 0, ccount = 0;
@@ -524,7 +528,8 @@ int launch_prefill_attend_tc(const Shape& s, const void* q, const void* maps, co
     }
     AtcArgs a{s, static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(landmarks), bias, entries,
               static_cast<const int4*>(tiles), n_tiles, lam, status, i0};
-    prefill_attend_tc_kernel<<<148, kThreads, smem, stream>>>(m[0], m[1], m[2], a);
+    if (launch_pdl(prefill_attend_tc_kernel, dim3(148), dim3(kThreads), smem, stream, m[0], m[1], m[2], a) != cudaSuccess)
+        return HILS_ERR_CUDA;
     if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
     return 1;
 }

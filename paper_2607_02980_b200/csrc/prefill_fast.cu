@@ -282,6 +282,7 @@ __global__ void invert_count_kernel(const PArgs a) {
 // tile-aligned range of entries.
 __global__ void __launch_bounds__(1024) invert_segsum_kernel(const PArgs a) {
     __shared__ int wsum[32];
+    pdl_wait();
     const int n = a.s.B * a.s.Hkv * a.nc * a.n_blocks;
     const int x = blockIdx.x * 1024 + threadIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     int ct = x < n ? (a.cnt[x] + a.tile_tok - 1) / a.tile_tok : 0;
@@ -300,6 +301,7 @@ __global__ void __launch_bounds__(1024) invert_segsum_kernel(const PArgs a) {
 __global__ void __launch_bounds__(1024) invert_scan_kernel(const PArgs a) {
     __shared__ int wsum_t[32];
     __shared__ int wpre[32];
+    pdl_wait();
     const Shape& s = a.s;
     const int per_blk = s.B * s.Hkv * a.nc;
     const int n = per_blk * a.n_blocks;
@@ -336,6 +338,7 @@ __global__ void __launch_bounds__(1024) invert_scan_kernel(const PArgs a) {
 }
 
 __global__ void invert_fill_kernel(const PArgs a) {
+    pdl_wait();
     const Shape& s = a.s;
     const int K1 = s.K + max_local_slots(s.W), pairs = s.B * s.Hkv;
     const long long total = static_cast<long long>(pairs) * s.R * K1;
@@ -360,6 +363,7 @@ __global__ void invert_fill_kernel(const PArgs a) {
 // not the q . k'_c that the attend kernel read off its score tile: this kernel overwrites those masses.  One CTA
 // per tile, one warp per entry at a time; lane l covers dimensions 4l .. 4l+3.  Local slots keep their masses.
 __global__ void __launch_bounds__(128) prefill_route_scores_kernel(const PArgs a) {
+    pdl_wait();
     const Shape& s = a.s;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int t_begin = a.blk_toff[a.blk];
@@ -401,6 +405,7 @@ constexpr int kFuseRows = 96;             // rows mixed per token: K <= 64 selec
 __global__ void __launch_bounds__(kFuseWarps * 32) prefill_fuse_kernel(const PArgs a) {
     __shared__ float wsm[kFuseWarps][kG][kFuseRows];
     __shared__ int esm[kFuseWarps][kFuseRows];
+    pdl_wait();
     const Shape& s = a.s;
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     const int K = s.K, K1 = K + max_local_slots(s.W), nblk = a.i1 - a.i0;
@@ -643,10 +648,13 @@ int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
             ++launches;
         }
         const unsigned nseg = static_cast<unsigned>((static_cast<long long>(p.n_blocks) * pairs * p.nc + 1023) / 1024);
-        invert_segsum_kernel<<<nseg, 1024, 0, stream>>>(a);
-        invert_scan_kernel<<<nseg, 1024, 0, stream>>>(a);
-        invert_fill_kernel<<<eb, 256, 0, stream>>>(a);
-        if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
+        // From here on every kernel of the call is launched so that its launch and prologue overlap the previous
+        // kernel's tail; each of them waits for its predecessors' results before its first dependent access.  None
+        // triggers its dependents early: CTAs of the next kernel parked beside a running attend kernel cost 5 %.
+        if (launch_pdl(invert_segsum_kernel, dim3(nseg), dim3(1024), 0, stream, a) != cudaSuccess ||
+            launch_pdl(invert_scan_kernel, dim3(nseg), dim3(1024), 0, stream, a) != cudaSuccess ||
+            launch_pdl(invert_fill_kernel, dim3(eb), dim3(256), 0, stream, a) != cudaSuccess)
+            return HILS_ERR_CUDA;
         trace_mark("prefill_invert", stream);
         launches += 3;
     }
@@ -664,14 +672,15 @@ int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
         trace_mark("prefill_attend", stream);
         if (t.q_route) {
             const int ntl = (p.max_blk_tiles);
-            prefill_route_scores_kernel<<<static_cast<unsigned>(ntl), 128, 0, stream>>>(a);
-            if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
+            if (launch_pdl(prefill_route_scores_kernel, dim3(static_cast<unsigned>(ntl)), dim3(128), 0, stream, a) != cudaSuccess)
+                return HILS_ERR_CUDA;
             trace_mark("prefill_route_scores", stream);
             ++launches;
         }
         const long long fuse_warps = static_cast<long long>(pairs) * nblk;
-        prefill_fuse_kernel<<<static_cast<unsigned>((fuse_warps + kFuseWarps - 1) / kFuseWarps), kFuseWarps * 32, 0, stream>>>(a);
-        if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
+        if (launch_pdl(prefill_fuse_kernel, dim3(static_cast<unsigned>((fuse_warps + kFuseWarps - 1) / kFuseWarps)),
+                       dim3(kFuseWarps * 32), 0, stream, a) != cudaSuccess)
+            return HILS_ERR_CUDA;
         trace_mark("prefill_fuse", stream);
         launches += 2;
     }

@@ -181,6 +181,25 @@ __device__ __forceinline__ void pv_tile(const float (&p)[8][4], uint32_t vs_addr
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// Host side: launch `kernel` so that it may become resident while the previous kernel of the stream drains.
+// Every kernel launched this way calls pdl_wait() before it touches anything an earlier kernel wrote (and
+// before it calls pdl_launch_dependents()), which keeps the chain of dependencies transitive.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              Args&&... args) {
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // ---- 5th-generation tensor cores (tcgen05): tensor-memory allocation, MMA issue, commit, loads ----
 
 // Instruction descriptor of tcgen05.mma.kind::f16 for bf16 x bf16 -> fp32, both operands K-major.
