@@ -192,3 +192,41 @@ def hils_landmarks(lq, k, seq_lens=None, *, S: int, scale: float = 0.0):
     if rc != 0:
         raise ValueError("hils_oracle_landmarks rejected its arguments (rc=%d)" % rc)
     return lm, bias
+
+
+def chunk_overlap(sel_idx, M: int):
+    """Chunk-id overlap among blocks of M adjacent queries (Sec. "Chunk Overlap", Eq. Overlap).
+
+    sel_idx: integer array [..., L, K], the selected chunk ids of L consecutive queries (-1 = empty slot).
+    Queries r*M .. r*M + M - 1 form block r; a trailing block holds the L mod M queries that are left.
+    For every block, written out with Python sets:
+        total   = sum over its queries m of |I_m|
+        union   = | union over m of I_m |                       (the chunks a packed kernel loads once)
+        reused  = | union  intersected with  the previous block's union |   (0 for block 0: inter-block reuse)
+        overlap = (M K - union) / ((M - 1) K)    as the equation has it, for blocks of M queries that each hold
+                  K chunks; NaN for any other block (fewer than K candidates, or the short trailing block)
+    Returns a dict of arrays [..., ceil(L / M)]: int64 total / union / reused, float64 overlap.
+    """
+    sel = np.asarray(sel_idx)
+    assert M >= 1 and sel.ndim >= 2
+    lead, (L, K) = sel.shape[:-2], sel.shape[-2:]
+    flat = sel.reshape((-1, L, K))
+    nblk = (L + M - 1) // M
+    total = np.zeros((flat.shape[0], nblk), np.int64)
+    union = np.zeros_like(total)
+    reused = np.zeros_like(total)
+    overlap = np.full((flat.shape[0], nblk), np.nan, np.float64)
+    for x in range(flat.shape[0]):
+        prev = set()
+        for r in range(nblk):
+            sets = [set(int(c) for c in flat[x, i] if c >= 0) for i in range(r * M, min(L, r * M + M))]
+            u = set().union(*sets)
+            total[x, r] = sum(len(s) for s in sets)
+            union[x, r] = len(u)
+            reused[x, r] = len(u & prev)
+            if M > 1 and len(sets) == M and all(len(s) == K for s in sets):
+                overlap[x, r] = (M * K - len(u)) / ((M - 1) * K)
+            prev = u
+    shape = lead + (nblk,)
+    return {"total": total.reshape(shape), "union": union.reshape(shape), "reused": reused.reshape(shape),
+            "overlap": overlap.reshape(shape)}

@@ -26,6 +26,12 @@ Value recipe:
                   N(0, I) query on the landmark direction), so that selection
                   has margin.
 
+    structured overlap (optional, `overlap_block=M`): adjacent queries of a
+                  real model retrieve largely the same chunks (Sec. "Chunk
+                  Overlap": up to 80-93 % shared).  One base query per block
+                  of M adjacent tokens and head, q_i = base + noise * N(0,1);
+                  no needles.  The other tensors are unchanged.
+
 Every tensor has its own generator seeded with seed*1000 + tensor_id, so a
 tensor does not change when another one is added or resized.
 """
@@ -138,7 +144,8 @@ def _needle_dirs(lm_bh: torch.Tensor, idx: torch.Tensor) -> torch.Tensor:
     return 3.0 * rows / rows.norm(dim=-1, keepdim=True).clamp_min(1e-20)
 
 
-def make_prefill_inputs(cfg: HilsConfig, device="cpu") -> Dict[str, torch.Tensor]:
+def make_prefill_inputs(cfg: HilsConfig, device="cpu", overlap_block: int = 0,
+                        overlap_noise: float = 0.3) -> Dict[str, torch.Tensor]:
     assert cfg.mode == "prefill"
     dev = torch.device(device)
     k = _draw_kv(cfg, _gen(cfg.seed, 1, dev), dev)
@@ -151,10 +158,15 @@ def make_prefill_inputs(cfg: HilsConfig, device="cpu") -> Dict[str, torch.Tensor
     G = cfg.G
     pos = torch.arange(cfg.L, device=dev)
     ci = pos // cfg.S                         # number of complete past chunks of each row
+    gb = _gen(cfg.seed, 8, dev)
     for b in range(cfg.B):
         for g in range(cfg.Hkv):
             qg = _randn((G, cfg.L, cfg.d), gq, dev) * mul
-            if cfg.n_needles > 0:
+            if overlap_block > 1:
+                nblk = (cfg.L + overlap_block - 1) // overlap_block
+                base = _randn((G, nblk, cfg.d), gb, dev) * mul
+                qg = base.repeat_interleave(overlap_block, dim=1)[:, :cfg.L] + overlap_noise * qg
+            elif cfg.n_needles > 0:
                 ok = ci >= cfg.n_needles      # rows with enough past chunks to plant into
                 u = torch.rand((cfg.n_needles, cfg.L), generator=gn, device=dev)
                 chosen = []
