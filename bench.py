@@ -148,7 +148,7 @@ def params_for(hils, cfg, decode, impl="auto", window=1):
 class Workload:
     """Device-resident inputs/outputs of one configuration and the call that runs one step."""
 
-    def __init__(self, hils, cfg, device, n_query_sets=8, window=1, with_bias=False):
+    def __init__(self, hils, cfg, device, n_query_sets=8, window=1, with_bias=False, overlap_block=0):
         self.hils, self.cfg, self.dev = hils, cfg, device
         self.decode = cfg.mode == "decode"
         self.window = window                     # prefill only; > 1 = the paper's operator form (Sec. 2.1)
@@ -168,7 +168,7 @@ class Workload:
             self.work, self.work_aux = lm_b + kv_b, kv_b
             self.unit, self.metric = "GB/s", "hils_decode_algorithmic_GBps"
         else:
-            self.inp = wl.make_prefill_inputs(cfg, device)
+            self.inp = wl.make_prefill_inputs(cfg, device, overlap_block=overlap_block)
             self.out = torch.empty_like(self.inp["q"])
             self.lse = torch.empty((cfg.B, cfg.Hq, cfg.L), dtype=torch.float32, device=device)
             self.sel = torch.empty((cfg.B, cfg.Hkv, cfg.L, cfg.K), dtype=torch.int32, device=device)
@@ -343,6 +343,32 @@ def bench_landmark_summary(hils, w, peaks, iters=10):
     return {"metric": "landmark_summary_algorithmic_GBps", "value": gbs, "unit": "GB/s", "ms": ms,
             "algorithmic_bytes": nbytes, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"],
             "l2_policy": "K tensor of %.0f MB > 126 MB L2, read once per call" % (k.numel() * k.element_size() / 1e6)}
+
+
+def bench_chunk_overlap(hils, w, peaks, M=16, iters=10):
+    """Chunk-id overlap of blocks of M adjacent queries (Sec. "Chunk Overlap", Eq. Overlap) on the selection the
+    workload's last prefill wrote: the statistics, and the kernel's time against reading sel_idx once."""
+    cfg, sel = w.cfg, w.sel
+    stats, ov = hils.hils_chunk_overlap(sel, M, cfg.C)
+    for _ in range(2):
+        hils.hils_chunk_overlap(sel, M, cfg.C, stats=stats, overlap=ov)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(iters + 1)]
+    torch.cuda.synchronize()
+    ev[0].record()
+    for i in range(iters):
+        hils.hils_chunk_overlap(sel, M, cfg.C, stats=stats, overlap=ov)
+        ev[i + 1].record()
+    torch.cuda.synchronize()
+    ms = float(np.mean([ev[i].elapsed_time(ev[i + 1]) for i in range(iters)]))
+    st = stats.cpu().numpy().astype(np.int64)
+    o = ov.cpu().numpy()
+    full = st[..., 3] == 1
+    nbytes = sel.numel() * 4 + stats.numel() * 4 + ov.numel() * 4
+    return {"block_queries": M, "top_k": cfg.K, "blocks": int(full.size), "full_blocks": int(full.sum()),
+            "mean_overlap": float(o[full].mean()), "mean_union_chunks": float(st[..., 1][full].mean()),
+            "reused_from_previous_block": float(st[..., 2][..., 1:].sum() / max(1, st[..., 1][..., 1:].sum())),
+            "ms": ms, "algorithmic_bytes": nbytes, "GBps": nbytes / (ms * 1e-3) / 1e9,
+            "frac_of_measured_hbm": nbytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
 
 
 # ----------------------------------------------------------------------------- CPU oracle legs
@@ -580,8 +606,22 @@ def main():
                 if name == "cfg3":
                     extras["cfg3_paged"] = bench_paged_decode(hils, ew, peaks)
                     launches += 3 * 13
+                if name == "cfg2":
+                    extras["cfg2_chunk_overlap_iid_queries"] = bench_chunk_overlap(hils, ew, peaks)
+                    launches += 13
                 del ew
                 if name == "cfg2":
+                    # adjacent queries that retrieve mostly the same chunks, as the paper measures on a trained model
+                    torch.cuda.empty_cache()
+                    sw = Workload(hils, pick_cfg(name), dev, overlap_block=16)
+                    sms, _ = time_steps(sw, max(3, args.steps), 3, barrier)
+                    extras["cfg2_structured_overlap"] = {
+                        "metric": sw.metric, "value": sw.rate(float(np.mean(sms)) * 1e-3), "unit": sw.unit,
+                        "ms_per_step": float(np.mean(sms)), "kernel_ms": kernel_times(sw, 3, barrier),
+                        "queries": "one base query per 16 adjacent tokens + 0.3 N(0,1)",
+                        "chunk_overlap": bench_chunk_overlap(hils, sw, peaks)}
+                    launches += hils.last_launch_count() * (max(3, args.steps) + 6) + 13
+                    del sw
                     # the paper's operator form (Sec. 2.1 / experiments): local window W = 512 and a non-null bias
                     torch.cuda.empty_cache()
                     pw = Workload(hils, pick_cfg(name), dev, window=512, with_bias=True)

@@ -194,6 +194,25 @@ int hils_landmark_summary(const hils_params* params, const void* landmark_querie
                           const int32_t* seq_lens, int32_t chunk_begin, int32_t chunk_count, void* landmarks,
                           float* bias, void* stream);
 
+/* Chunk-id overlap among adjacent queries (Sec. "Chunk Overlap", Eq. Overlap) -- the statistic behind packing M
+ * adjacent queries over the union of their chunks.  Queries r*M .. r*M + M - 1 of one (sequence, KV head) pair
+ * form block r (M = block_queries; a trailing block holds the L mod M queries left); I_m is the set of chunk
+ * ids in the K slots of its m-th query (ids outside [0, C), e.g. the -1 of an empty slot, are skipped).
+ *
+ *   sel_idx  [B, Hkv, L, K] int32 DEVICE, as written by hils_prefill / hils_prefill_at (L = params->L,
+ *            K = params->top_k, C = params->C)
+ *   stats    [B, Hkv, nblk, 4] int32 DEVICE, 16-byte aligned, nblk = ceil(L / M); per block
+ *              [0] total  = sum_m |I_m|
+ *              [1] union  = |union_m I_m|           (chunks a packed kernel loads once for the block)
+ *              [2] reused = |union  intersected with  the previous block's union|   (0 for block 0)
+ *              [3] full   = 1 if the block has M queries holding K chunks each, else 0
+ *   overlap  [B, Hkv, nblk] fp32 DEVICE or NULL: (M K - union) / ((M - 1) K) where full = 1 and M > 1,
+ *            NaN elsewhere (the equation is stated for M queries of K chunks)
+ * Uses of params: B, Hkv, L, C (<= 2^19), top_k.  Needs no workspace; one kernel is enqueued on `stream`.
+ * Errors: HILS_ERR_INVALID_ARG, HILS_ERR_ALIGNMENT, HILS_ERR_UNSUPPORTED (C too large), HILS_ERR_CUDA. */
+int hils_chunk_overlap(const hils_params* params, const int32_t* sel_idx, int32_t block_queries, int32_t* stats,
+                       float* overlap, void* stream);
+
 /* Bytes of device memory the *_host entry points need for staging (inputs + outputs + workspace). */
 size_t hils_host_arena_bytes(const hils_params* params, int is_decode);
 

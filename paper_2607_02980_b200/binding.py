@@ -25,7 +25,7 @@ EXPORTS = [
     "hils_prefill_host", "hils_decode_host", "hils_poll_status", "hils_last_launch_count",
     "hils_status_string", "hils_version", "hils_trace_enable", "hils_trace_read", "hils_decode_noalloc",
     "hils_landmark_summary", "hils_decode_paged", "hils_prefill_at", "hils_prefill_at_workspace_bytes",
-    "hils_prefill_routed", "hils_decode_routed",
+    "hils_prefill_routed", "hils_decode_routed", "hils_chunk_overlap",
 ]
 
 
@@ -84,6 +84,8 @@ def load_library() -> ctypes.CDLL:
                                       ctypes.c_size_t, vp]
     lib.hils_landmark_summary.restype = ctypes.c_int
     lib.hils_landmark_summary.argtypes = [pp, vp, vp, i32p, ctypes.c_int32, ctypes.c_int32, vp, f32p, vp]
+    lib.hils_chunk_overlap.restype = ctypes.c_int
+    lib.hils_chunk_overlap.argtypes = [pp, i32p, ctypes.c_int32, i32p, f32p, vp]
     lib.hils_poll_status.restype = ctypes.c_int
     lib.hils_poll_status.argtypes = [vp, vp]
     lib.hils_last_launch_count.restype = ctypes.c_int
@@ -369,6 +371,32 @@ def hils_landmark_summary(landmark_queries, k, chunk_size: int, *, seq_lens=None
     if rc != 0:
         raise HilsError(rc, "hils_landmark_summary")
     return landmarks, bias
+
+
+def hils_chunk_overlap(sel_idx, block_queries: int, num_chunks: int, *, stats=None, overlap=None, stream=None):
+    """Chunk-id overlap of blocks of `block_queries` adjacent queries (Sec. "Chunk Overlap", Eq. Overlap).
+
+    sel_idx [B,Hkv,L,K] int32 CUDA tensor as written by hils_prefill; num_chunks = C bounds the chunk ids.
+    Returns (stats [B,Hkv,nblk,4] int32: total, union, reused, full; overlap [B,Hkv,nblk] fp32, NaN where the
+    equation does not apply), nblk = ceil(L / block_queries).
+    """
+    lib = load_library()
+    B, Hkv, L, K = sel_idx.shape
+    _check(sel_idx, "sel_idx", (B, Hkv, L, K), torch.int32, True)
+    nblk = (L + int(block_queries) - 1) // max(int(block_queries), 1)
+    if stats is None:
+        stats = torch.empty((B, Hkv, nblk, 4), dtype=torch.int32, device=sel_idx.device)
+    if overlap is None:
+        overlap = torch.empty((B, Hkv, nblk), dtype=torch.float32, device=sel_idx.device)
+    _check(stats, "stats", (B, Hkv, nblk, 4), torch.int32, True)
+    _check(overlap, "overlap", (B, Hkv, nblk), torch.float32, True)
+    p = make_params(B=B, Hq=Hkv, Hkv=Hkv, Hl=Hkv, L=L, T_max=0, C=int(num_chunks), d=1, chunk_size=1, top_k=K,
+                    window=1, scale=0.0, dtype=0, impl="auto")
+    rc = lib.hils_chunk_overlap(ctypes.byref(p), _ptr(sel_idx), int(block_queries), _ptr(stats), _ptr(overlap),
+                                _stream_ptr(stream))
+    if rc != 0:
+        raise HilsError(rc, "hils_chunk_overlap")
+    return stats, overlap
 
 
 class HostRunner:

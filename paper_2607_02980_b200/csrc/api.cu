@@ -452,6 +452,27 @@ int hils_landmark_summary(const hils_params* params, const void* landmark_querie
     return HILS_OK;
 }
 
+int hils_chunk_overlap(const hils_params* params, const int32_t* sel_idx, int32_t block_queries, int32_t* stats,
+                       float* overlap, void* stream) {
+    g_last_launches = 0;
+    const hils_params* p = params;
+    if (!p || !sel_idx || !stats) return HILS_ERR_INVALID_ARG;
+    if (p->B < 1 || p->Hkv < 1 || p->L < 1 || p->C < 1 || p->top_k < 1 || block_queries < 1)
+        return HILS_ERR_INVALID_ARG;
+    if (static_cast<long long>(block_queries) * p->top_k > (1ll << 24)) return HILS_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(sel_idx) & 3u) || (reinterpret_cast<uintptr_t>(stats) & 15u) ||
+        (overlap && (reinterpret_cast<uintptr_t>(overlap) & 3u)))
+        return HILS_ERR_ALIGNMENT;
+    if (!chunk_overlap_supports(p->C)) return HILS_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    trace_begin(st);
+    const int n = launch_chunk_overlap(p->B * p->Hkv, p->L, p->top_k, p->C, block_queries, sel_idx, stats, overlap, st);
+    if (n < 0) return n;
+    trace_mark("chunk_overlap", st);
+    g_last_launches = n;
+    return HILS_OK;
+}
+
 size_t hils_host_arena_bytes(const hils_params* params, int is_decode) {
     ArenaLayout a;
     if (arena_layout(params, is_decode, &a) != HILS_OK || a.ws_b == 0) return 0;

@@ -70,6 +70,11 @@ int launch_landmark_summary(int dtype, int B, int Hkv, int Hl, int C, int d, int
                             const void* lq, const void* k, const int32_t* seq_lens, int c0, int cn, void* landmarks,
                             float* bias, cudaStream_t stream);
 
+// Chunk-id overlap of blocks of M adjacent queries (Sec. "Chunk Overlap"): stats [pairs, nblk, 4], overlap [pairs, nblk].
+bool chunk_overlap_supports(int C);
+int launch_chunk_overlap(int pairs, int R, int K, int C, int M, const int32_t* sel, int32_t* stats, float* overlap,
+                         cudaStream_t stream);
+
 int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream);
 bool prefill_fast_supports(const Shape& s, int dtype);
 size_t prefill_fast_scratch_bytes(const Shape& s);
