@@ -51,6 +51,7 @@ def _load():
         _lib.hils_oracle_num_threads.restype = ctypes.c_int
         _lib.hils_oracle_landmarks.restype = ctypes.c_int
         _lib.hils_oracle_rows_routed.restype = ctypes.c_int
+        _lib.hils_oracle_backward.restype = ctypes.c_int
     return _lib
 
 
@@ -192,6 +193,42 @@ def hils_landmarks(lq, k, seq_lens=None, *, S: int, scale: float = 0.0):
     if rc != 0:
         raise ValueError("hils_oracle_landmarks rejected its arguments (rc=%d)" % rc)
     return lm, bias
+
+
+def hils_backward(q, k, v, landmarks, bias, sel_idx, dout, *, S: int, K: int, W: int = 1, scale: float = 0.0,
+                  pos0: int = 0):
+    """Gradients of a scalar loss through `out` of the operator (chain rule on Eq. HiLS weights, selection fixed).
+
+    q, dout [B,Hq,Lq,d]; k, v [B,Hkv,T,d]; landmarks [B,Hl,C,d]; bias [B,Hl,C] or None; sel_idx [B,Hkv,Lq,K]
+    as the forward wrote it; query row r sits at position pos0 + r.  dout is taken as float64.
+    Returns dict(dq, dk, dv, dlandmarks, dbias) of float64 arrays shaped like q, k, v, landmarks, bias.
+    """
+    lib = _load()
+    in_bf16 = int(all(_is_bf16(t) for t in (q, k, v, landmarks)))
+    conv = _raw_bf16 if in_bf16 else _f32
+    q = conv(q); k = conv(k); v = conv(v); landmarks = conv(landmarks)
+    bias_a = None if bias is None else _f32(bias)
+    B, Hq, Lq, d = q.shape
+    _, Hkv, T, _ = k.shape
+    _, Hl, C, _ = landmarks.shape
+    sel = np.ascontiguousarray(sel_idx.detach().cpu().numpy() if hasattr(sel_idx, "detach") else sel_idx,
+                               dtype=np.int32)
+    assert sel.shape == (B, Hkv, Lq, K)
+    do = np.ascontiguousarray(dout.detach().cpu().double().numpy() if hasattr(dout, "detach") else dout,
+                              dtype=np.float64)
+    assert do.shape == (B, Hq, Lq, d)
+    p = _Params(B, Hq, Hkv, Hl, Lq, T, C, d, S, K, W, float(scale), 0, in_bf16)
+    res = {"dq": np.zeros((B, Hq, Lq, d)), "dk": np.zeros((B, Hkv, T, d)), "dv": np.zeros((B, Hkv, T, d)),
+           "dlandmarks": np.zeros((B, Hl, C, d)), "dbias": np.zeros((B, Hl, C))}
+    rc = lib.hils_oracle_backward(
+        ctypes.byref(p), ctypes.c_void_p(q.ctypes.data), ctypes.c_void_p(k.ctypes.data),
+        ctypes.c_void_p(v.ctypes.data), ctypes.c_void_p(landmarks.ctypes.data), _ptr(bias_a, ctypes.c_float),
+        _ptr(sel, ctypes.c_int32), ctypes.c_int64(pos0), _ptr(do, ctypes.c_double),
+        _ptr(res["dq"], ctypes.c_double), _ptr(res["dk"], ctypes.c_double), _ptr(res["dv"], ctypes.c_double),
+        _ptr(res["dlandmarks"], ctypes.c_double), _ptr(res["dbias"], ctypes.c_double))
+    if rc != 0:
+        raise ValueError("hils_oracle_backward rejected its arguments (rc=%d)" % rc)
+    return res
 
 
 def chunk_overlap(sel_idx, M: int):

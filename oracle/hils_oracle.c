@@ -361,3 +361,155 @@ int hils_oracle_landmarks(const hils_oracle_params *p, const void *lq, const voi
     }
     return 0;
 }
+
+/*
+ * Backward of the operator: the gradient of a scalar loss through `out`, given dout = dLoss/dout.
+ *
+ * The paper states that the retrieval scores sit inside the forward attention weights so that the language-model
+ * loss trains the landmarks (Sec. 3.2, below Eq. HiLS weights), but prints no backward equations: what follows is
+ * the chain rule applied, step by step, to the forward above, with the selected set I held fixed (top-K has no
+ * derivative) and q-hat = q.  For one query head (position i, head h), with slots t = selected chunks and the
+ * local span, p_tj the softmax inside slot t, o_t = sum_j p_tj v_j, lambda_t the slot's log mass
+ * (s^h_c = scale q.k'_c + b'_c for a selected chunk, log Z_swa = log sum_j exp(s_j) for the local span),
+ * alpha = softmax_t(lambda), out = sum_t alpha_t o_t:
+ *
+ *   d alpha_t   = dout . o_t
+ *   d lambda_t  = alpha_t (d alpha_t - sum_u alpha_u d alpha_u)            (softmax over the slots)
+ *   d o_t       = alpha_t dout
+ *   d v_j      += p_tj d o_t                                               (o_t = sum_j p_tj v_j)
+ *   d p_tj      = d o_t . v_j
+ *   d s_tj      = p_tj (d p_tj - sum_l p_tl d p_tl)                        (softmax inside the slot)
+ *   local span only:  d s_tj += d lambda_t p_tj                            (lambda_loc = logsumexp_j s_j)
+ *   selected chunk c: d q += scale d lambda_t k'_c,  d k'_c += scale d lambda_t q,  d b'_c += d lambda_t
+ *   d q += scale sum_j d s_tj k_j,   d k_j += scale d s_tj q               (s_tj = scale q . k_j)
+ *
+ * Pinned by tests/test_backward_pins.py: central finite differences of the forward oracle in every input,
+ * library autograd on the rows that reduce to causal softmax attention, and the K = 1 two-branch mix.
+ *
+ * Layouts: q, dout, dq [B, Hq, Lq, d]; k, v, dk, dv [B, Hkv, T, d]; landmarks, dlm [B, Hl, C, d];
+ * bias, dbias [B, Hl, C]; sel_idx [B, Hkv, Lq, K] (ascending, -1 padded, as the forward wrote it).
+ * Query row r sits at position pos0 + r.  The five gradient arrays are overwritten.  Returns 0 or -1.
+ */
+int hils_oracle_backward(const hils_oracle_params *p, const void *q, const void *k, const void *v,
+                         const void *landmarks, const float *bias, const int32_t *sel_idx, int64_t pos0,
+                         const double *dout, double *dq, double *dk, double *dv, double *dlm, double *dbias)
+{
+    if (!p || p->Hq % p->Hkv != 0 || (p->Hl != p->Hkv && p->Hl != p->Hq) || p->S <= 0 || p->K < 0 ||
+        p->W < 1 || !sel_idx || !dout || !dq || !dk || !dv || !dlm || !dbias || pos0 < 0)
+        return -1;
+    const int G = p->Hq / p->Hkv, d = p->d, S = p->S, K = p->K, bf = p->in_bf16;
+    const double scale = p->scale > 0 ? p->scale : 1.0 / sqrt((double)d);
+    memset(dq, 0, sizeof(double) * (size_t)p->B * p->Hq * p->Lq * d);
+    memset(dk, 0, sizeof(double) * (size_t)p->B * p->Hkv * p->T * d);
+    memset(dv, 0, sizeof(double) * (size_t)p->B * p->Hkv * p->T * d);
+    memset(dlm, 0, sizeof(double) * (size_t)p->B * p->Hl * p->C * d);
+    memset(dbias, 0, sizeof(double) * (size_t)p->B * p->Hl * p->C);
+    int status = 0;
+
+    /* one (sequence, KV group) per thread: its slices of dk, dv, dlm, dbias belong to it alone */
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int pair = 0; pair < p->B * p->Hkv; ++pair) {
+        const int b = pair / p->Hkv, g = pair % p->Hkv;
+        const size_t ikv = ((size_t)b * p->Hkv + g) * (size_t)p->T * d;
+        const size_t max_span = (size_t)S * ((size_t)(p->W + S - 1) / S + 1);
+        double *pr = (double *)malloc(sizeof(double) * (size_t)(K + 1) * max_span);   /* p_tj          */
+        double *o = (double *)malloc(sizeof(double) * (size_t)(K + 1) * d);           /* o_t           */
+        double *lam = (double *)malloc(sizeof(double) * (size_t)(K + 1));
+        double *alpha = (double *)malloc(sizeof(double) * (size_t)(K + 1));
+        double *dalpha = (double *)malloc(sizeof(double) * (size_t)(K + 1));
+        double *dp = (double *)malloc(sizeof(double) * max_span);
+        long *lo_t = (long *)malloc(sizeof(long) * (size_t)(K + 1));
+        long *n_t = (long *)malloc(sizeof(long) * (size_t)(K + 1));
+        int *chunk_t = (int *)malloc(sizeof(int) * (size_t)(K + 1));
+
+        for (int r = 0; r < p->Lq; ++r) {
+            const long i = (long)(pos0 + r);
+            long lo = floordiv(i - p->W + 1, S) * S;
+            if (lo < 0) lo = 0;
+            const int ncand = (int)(lo / S);
+            if (i >= p->T || ncand > p->C) { status = -1; continue; }
+            const int32_t *sel = sel_idx + (((size_t)b * p->Hkv + g) * p->Lq + r) * K;
+
+            for (int rr = 0; rr < G; ++rr) {
+                const int h = g * G + rr;
+                const int hl = (p->Hl == p->Hq) ? h : g;
+                const size_t iq = (((size_t)b * p->Hq + h) * p->Lq + r) * d;
+                const double *dor = dout + iq;
+
+                /* ---- forward, keeping what the derivative needs */
+                int nslot = 0;
+                for (int t = 0; t < K; ++t) {
+                    const int c = sel[t];
+                    if (c < 0) continue;
+                    if (c >= ncand) { status = -1; continue; }
+                    chunk_t[nslot] = c; lo_t[nslot] = (long)c * S; n_t[nslot] = S;
+                    const size_t ilm = (((size_t)b * p->Hl + hl) * p->C + c) * d;
+                    lam[nslot] = scale * dotx(q, iq, landmarks, ilm, d, bf);
+                    if (bias) lam[nslot] += (double)bias[((size_t)b * p->Hl + hl) * p->C + c];
+                    ++nslot;
+                }
+                chunk_t[nslot] = -1; lo_t[nslot] = lo; n_t[nslot] = i + 1 - lo;        /* the local span */
+                ++nslot;
+                for (int t = 0; t < nslot; ++t) {
+                    double *pt = pr + (size_t)t * max_span, *ot = o + (size_t)t * d;
+                    double m = -INFINITY, Z = 0.0;
+                    for (long j = 0; j < n_t[t]; ++j) {
+                        pt[j] = scale * dotx(q, iq, k, ikv + (size_t)(lo_t[t] + j) * d, d, bf);
+                        if (pt[j] > m) m = pt[j];
+                    }
+                    for (long j = 0; j < n_t[t]; ++j) { pt[j] = exp(pt[j] - m); Z += pt[j]; }
+                    for (int x = 0; x < d; ++x) ot[x] = 0.0;
+                    for (long j = 0; j < n_t[t]; ++j) {
+                        pt[j] /= Z;
+                        for (int x = 0; x < d; ++x) ot[x] += pt[j] * ld(v, ikv + (size_t)(lo_t[t] + j) * d + x, bf);
+                    }
+                    if (chunk_t[t] < 0) lam[t] = m + log(Z);
+                }
+                double Mx = -INFINITY, Dn = 0.0;
+                for (int t = 0; t < nslot; ++t) if (lam[t] > Mx) Mx = lam[t];
+                for (int t = 0; t < nslot; ++t) Dn += exp(lam[t] - Mx);
+                for (int t = 0; t < nslot; ++t) alpha[t] = exp(lam[t] - Mx) / Dn;
+
+                /* ---- backward */
+                double mix = 0.0;                                   /* sum_u alpha_u d alpha_u */
+                for (int t = 0; t < nslot; ++t) {
+                    dalpha[t] = 0.0;
+                    for (int x = 0; x < d; ++x) dalpha[t] += dor[x] * o[(size_t)t * d + x];
+                    mix += alpha[t] * dalpha[t];
+                }
+                double *dqr = dq + iq;
+                for (int t = 0; t < nslot; ++t) {
+                    const double *pt = pr + (size_t)t * max_span;
+                    const double dlam = alpha[t] * (dalpha[t] - mix);
+                    double inner = 0.0;                             /* sum_l p_tl d p_tl */
+                    for (long j = 0; j < n_t[t]; ++j) {
+                        dp[j] = 0.0;
+                        for (int x = 0; x < d; ++x)
+                            dp[j] += alpha[t] * dor[x] * ld(v, ikv + (size_t)(lo_t[t] + j) * d + x, bf);
+                        inner += pt[j] * dp[j];
+                    }
+                    for (long j = 0; j < n_t[t]; ++j) {
+                        const size_t row = ikv + (size_t)(lo_t[t] + j) * d;
+                        double ds = pt[j] * (dp[j] - inner);
+                        if (chunk_t[t] < 0) ds += dlam * pt[j];
+                        for (int x = 0; x < d; ++x) {
+                            dv[row + x] += pt[j] * alpha[t] * dor[x];
+                            dqr[x] += scale * ds * ld(k, row + x, bf);
+                            dk[row + x] += scale * ds * ld(q, iq + x, bf);
+                        }
+                    }
+                    if (chunk_t[t] >= 0) {
+                        const size_t ilm = (((size_t)b * p->Hl + hl) * p->C + chunk_t[t]) * d;
+                        for (int x = 0; x < d; ++x) {
+                            dqr[x] += scale * dlam * ld(landmarks, ilm + x, bf);
+                            dlm[ilm + x] += scale * dlam * ld(q, iq + x, bf);
+                        }
+                        dbias[((size_t)b * p->Hl + hl) * p->C + chunk_t[t]] += dlam;
+                    }
+                }
+            }
+        }
+        free(pr); free(o); free(lam); free(alpha); free(dalpha); free(dp); free(lo_t); free(n_t); free(chunk_t);
+    }
+    return status;
+}
