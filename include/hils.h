@@ -213,6 +213,34 @@ int hils_landmark_summary(const hils_params* params, const void* landmark_querie
 int hils_chunk_overlap(const hils_params* params, const int32_t* sel_idx, int32_t block_queries, int32_t* stats,
                        float* overlap, void* stream);
 
+/* Backward of hils_prefill through `out` (training; Sec. 3.2: the retrieval scores sit inside the forward
+ * weights, so the loss reaches the landmarks).  The paper prints no backward equations; this is the chain rule
+ * on Eq. (HiLS weights) / App. C with the selected set held fixed (top-K has no derivative), the routing query
+ * equal to q, and no gradient through `lse`.  With alpha_c = exp(s^h_c - lse), p_j the softmax inside a slot,
+ * w_j the final weight of key j (alpha_c p_j in a selected chunk, exp(s_j - lse) in the local span),
+ * g_c = dout . o_c and D = dout . out:
+ *     d s_j = w_j (dout . v_j - g_c)   (selected chunk)        d s_j = w_j (dout . v_j - D)   (local span)
+ *     d lambda_c = alpha_c (g_c - D)
+ *     dv_j += w_j dout,  dq += scale d s_j k_j,  dk_j += scale d s_j q,
+ *     dq += scale d lambda_c k'_c,  dlandmarks_c += scale d lambda_c q,  dbias_c += d lambda_c.
+ *
+ *   q, k, v, landmarks, bias   as given to hils_prefill (params likewise)
+ *   out, lse, sel_idx          as hils_prefill wrote them (out in params->dtype)
+ *   dout            [B, Hq, L, d]   DEVICE, params->dtype: dLoss/dout
+ *   dq              [B, Hq, L, d]   fp32 DEVICE, overwritten
+ *   dk, dv          [B, Hkv, T, d]  fp32 DEVICE, overwritten (zeroed by the call, then accumulated)
+ *   dlandmarks      [B, Hl, C, d]   fp32 DEVICE, same
+ *   dbias           [B, Hl, C]      fp32 DEVICE or NULL, same
+ * All gradient pointers 16-byte aligned (dbias 4).  Sums over queries are accumulated with fp32 atomics, so
+ * the last bits of dk, dv, dlandmarks, dbias may differ from run to run.  Workspace:
+ * hils_prefill_backward_workspace_bytes (0 = unsupported shape); its head is the status word of
+ * hils_poll_status.  Errors as for hils_prefill. */
+size_t hils_prefill_backward_workspace_bytes(const hils_params* params);
+int hils_prefill_backward(const hils_params* params, const void* q, const void* k, const void* v,
+                          const void* landmarks, const float* bias, const void* out, const float* lse,
+                          const int32_t* sel_idx, const void* dout, float* dq, float* dk, float* dv,
+                          float* dlandmarks, float* dbias, void* workspace, size_t workspace_bytes, void* stream);
+
 /* Bytes of device memory the *_host entry points need for staging (inputs + outputs + workspace). */
 size_t hils_host_arena_bytes(const hils_params* params, int is_decode);
 

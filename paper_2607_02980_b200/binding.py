@@ -25,7 +25,8 @@ EXPORTS = [
     "hils_prefill_host", "hils_decode_host", "hils_poll_status", "hils_last_launch_count",
     "hils_status_string", "hils_version", "hils_trace_enable", "hils_trace_read", "hils_decode_noalloc",
     "hils_landmark_summary", "hils_decode_paged", "hils_prefill_at", "hils_prefill_at_workspace_bytes",
-    "hils_prefill_routed", "hils_decode_routed", "hils_chunk_overlap",
+    "hils_prefill_routed", "hils_decode_routed", "hils_chunk_overlap", "hils_prefill_backward",
+    "hils_prefill_backward_workspace_bytes",
 ]
 
 
@@ -84,6 +85,11 @@ def load_library() -> ctypes.CDLL:
                                       ctypes.c_size_t, vp]
     lib.hils_landmark_summary.restype = ctypes.c_int
     lib.hils_landmark_summary.argtypes = [pp, vp, vp, i32p, ctypes.c_int32, ctypes.c_int32, vp, f32p, vp]
+    lib.hils_prefill_backward_workspace_bytes.restype = ctypes.c_size_t
+    lib.hils_prefill_backward_workspace_bytes.argtypes = [pp]
+    lib.hils_prefill_backward.restype = ctypes.c_int
+    lib.hils_prefill_backward.argtypes = [pp, vp, vp, vp, vp, f32p, vp, f32p, i32p, vp, f32p, f32p, f32p, f32p, f32p,
+                                          vp, ctypes.c_size_t, vp]
     lib.hils_chunk_overlap.restype = ctypes.c_int
     lib.hils_chunk_overlap.argtypes = [pp, i32p, ctypes.c_int32, i32p, f32p, vp]
     lib.hils_poll_status.restype = ctypes.c_int
@@ -371,6 +377,49 @@ def hils_landmark_summary(landmark_queries, k, chunk_size: int, *, seq_lens=None
     if rc != 0:
         raise HilsError(rc, "hils_landmark_summary")
     return landmarks, bias
+
+
+def hils_prefill_backward(q, k, v, landmarks, chunk_size: int, top_k: int, out, lse, sel_idx, dout, *, bias=None,
+                          window: int = 1, scale: float = 0.0, impl: str = "auto", workspace=None, stream=None):
+    """Gradients of a loss through `out` of hils_prefill (selection fixed): dout [B,Hq,L,d] in q's dtype;
+    out, lse, sel_idx as hils_prefill returned them.
+
+    Returns (dq [B,Hq,L,d], dk, dv [B,Hkv,T,d], dlandmarks [B,Hl,C,d], dbias [B,Hl,C] or None), all fp32.
+    """
+    lib = load_library()
+    B, Hq, L, d = q.shape
+    Hkv, T = k.shape[1], k.shape[2]
+    Hl, C = landmarks.shape[1], landmarks.shape[2]
+    dt = q.dtype
+    _check(q, "q", (B, Hq, L, d), dt, True)
+    _check(k, "k", (B, Hkv, T, d), dt, True)
+    _check(v, "v", (B, Hkv, T, d), dt, True)
+    _check(landmarks, "landmarks", (B, Hl, C, d), dt, True)
+    _check(out, "out", (B, Hq, L, d), dt, True)
+    _check(dout, "dout", (B, Hq, L, d), dt, True)
+    _check(lse, "lse", (B, Hq, L), torch.float32, True)
+    _check(sel_idx, "sel_idx", (B, Hkv, L, top_k), torch.int32, True)
+    if bias is not None:
+        _check(bias, "bias", (B, Hl, C), torch.float32, True)
+    f32 = dict(dtype=torch.float32, device=q.device)
+    dq = torch.empty((B, Hq, L, d), **f32)
+    dk = torch.empty((B, Hkv, T, d), **f32)
+    dv = torch.empty((B, Hkv, T, d), **f32)
+    dlm = torch.empty((B, Hl, C, d), **f32)
+    dbias = torch.empty((B, Hl, C), **f32) if bias is not None else None
+    p = make_params(B=B, Hq=Hq, Hkv=Hkv, Hl=Hl, L=L, T_max=T, C=C, d=d, chunk_size=chunk_size, top_k=top_k,
+                    window=window, scale=scale, dtype=_dtype_code(q), impl=impl)
+    if workspace is None:
+        n = int(lib.hils_prefill_backward_workspace_bytes(ctypes.byref(p)))
+        if n == 0:
+            raise HilsError(-2, "hils_prefill_backward_workspace_bytes")
+        workspace = torch.zeros(n, dtype=torch.uint8, device=q.device)
+    rc = lib.hils_prefill_backward(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(landmarks), _ptr(bias), _ptr(out),
+                                   _ptr(lse), _ptr(sel_idx), _ptr(dout), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dlm),
+                                   _ptr(dbias), _ptr(workspace), workspace.numel(), _stream_ptr(stream))
+    if rc != 0:
+        raise HilsError(rc, "hils_prefill_backward")
+    return dq, dk, dv, dlm, dbias
 
 
 def hils_chunk_overlap(sel_idx, block_queries: int, num_chunks: int, *, stats=None, overlap=None, stream=None):

@@ -452,6 +452,51 @@ int hils_landmark_summary(const hils_params* params, const void* landmark_querie
     return HILS_OK;
 }
 
+size_t hils_prefill_backward_workspace_bytes(const hils_params* params) {
+    Shape s;
+    if (make_shape(params, 0, &s) != HILS_OK) return 0;
+    if (!generic_supports(s)) return 0;
+    return kStatusBytes;
+}
+
+int hils_prefill_backward(const hils_params* params, const void* q, const void* k, const void* v,
+                          const void* landmarks, const float* bias, const void* out, const float* lse,
+                          const int32_t* sel_idx, const void* dout, float* dq, float* dk, float* dv,
+                          float* dlandmarks, float* dbias, void* workspace, size_t workspace_bytes, void* stream) {
+    g_last_launches = 0;
+    const hils_params* p = params;
+    Shape s;
+    int rc = make_shape(p, 0, &s);
+    if (rc != HILS_OK) return rc;
+    if (!q || !k || !v || !landmarks || !out || !lse || !sel_idx || !dout || !dq || !dk || !dv || !dlandmarks)
+        return HILS_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(landmarks) || !aligned16(out) ||
+        !aligned16(dout) || !aligned16(dq) || !aligned16(dk) || !aligned16(dv) || !aligned16(dlandmarks) ||
+        (reinterpret_cast<uintptr_t>(lse) & 3u) || (reinterpret_cast<uintptr_t>(sel_idx) & 3u) ||
+        (bias && (reinterpret_cast<uintptr_t>(bias) & 3u)) || (dbias && (reinterpret_cast<uintptr_t>(dbias) & 3u)))
+        return HILS_ERR_ALIGNMENT;
+    if (!generic_supports(s)) return HILS_ERR_UNSUPPORTED;
+    const size_t need = hils_prefill_backward_workspace_bytes(p);
+    if (!workspace || workspace_bytes < need) return HILS_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return HILS_ERR_ALIGNMENT;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // the four shared gradients are accumulated: they start at zero (dq is written whole)
+    const size_t kv = static_cast<size_t>(s.B) * s.Hkv * s.T * s.d * sizeof(float);
+    const size_t lmb = static_cast<size_t>(s.B) * s.Hl * s.C * sizeof(float);
+    if (cudaMemsetAsync(dk, 0, kv, st) != cudaSuccess || cudaMemsetAsync(dv, 0, kv, st) != cudaSuccess ||
+        cudaMemsetAsync(dlandmarks, 0, lmb * s.d, st) != cudaSuccess ||
+        (dbias && cudaMemsetAsync(dbias, 0, lmb, st) != cudaSuccess))
+        return HILS_ERR_CUDA;
+    BackwardTensors t{q, k, v, landmarks, bias, out, lse, sel_idx, dout, dq, dk, dv, dlandmarks, dbias,
+                      static_cast<int*>(workspace), static_cast<char*>(workspace) + kStatusBytes,
+                      workspace_bytes - kStatusBytes};
+    trace_begin(st);
+    const int n = launch_backward_generic(s, p->dtype, t, st);
+    if (n < 0) return n;
+    g_last_launches = n;
+    return HILS_OK;
+}
+
 int hils_chunk_overlap(const hils_params* params, const int32_t* sel_idx, int32_t block_queries, int32_t* stats,
                        float* overlap, void* stream) {
     g_last_launches = 0;

@@ -70,6 +70,28 @@ int launch_landmark_summary(int dtype, int B, int Hkv, int Hl, int C, int d, int
                             const void* lq, const void* k, const int32_t* seq_lens, int c0, int cn, void* landmarks,
                             float* bias, cudaStream_t stream);
 
+// Backward through `out` (selection fixed): inputs of the forward, what it wrote, dout; fp32 gradients.
+struct BackwardTensors {
+    const void* q;
+    const void* k;
+    const void* v;
+    const void* landmarks;
+    const float* bias;
+    const void* out;
+    const float* lse;
+    const int32_t* sel_idx;
+    const void* dout;
+    float* dq;
+    float* dk;
+    float* dv;
+    float* dlandmarks;
+    float* dbias;              // may be NULL
+    int* status;
+    void* scratch;
+    size_t scratch_bytes;
+};
+int launch_backward_generic(const Shape& s, int dtype, const BackwardTensors& t, cudaStream_t stream);
+
 // Chunk-id overlap of blocks of M adjacent queries (Sec. "Chunk Overlap"): stats [pairs, nblk, 4], overlap [pairs, nblk].
 bool chunk_overlap_supports(int C);
 int launch_chunk_overlap(int pairs, int R, int K, int C, int M, const int32_t* sel, int32_t* stats, float* overlap,
