@@ -455,7 +455,9 @@ int hils_landmark_summary(const hils_params* params, const void* landmark_querie
 size_t hils_prefill_backward_workspace_bytes(const hils_params* params) {
     Shape s;
     if (make_shape(params, 0, &s) != HILS_OK) return 0;
-    if (!generic_supports(s)) return 0;
+    const bool fast = params->impl != HILS_IMPL_GENERIC && prefill_backward_fast_supports(s, params->dtype);
+    if (fast) return kStatusBytes + prefill_backward_fast_scratch_bytes(s);
+    if (params->impl == HILS_IMPL_FAST || !generic_supports(s)) return 0;
     return kStatusBytes;
 }
 
@@ -475,7 +477,8 @@ int hils_prefill_backward(const hils_params* params, const void* q, const void* 
         (reinterpret_cast<uintptr_t>(lse) & 3u) || (reinterpret_cast<uintptr_t>(sel_idx) & 3u) ||
         (bias && (reinterpret_cast<uintptr_t>(bias) & 3u)) || (dbias && (reinterpret_cast<uintptr_t>(dbias) & 3u)))
         return HILS_ERR_ALIGNMENT;
-    if (!generic_supports(s)) return HILS_ERR_UNSUPPORTED;
+    const bool fast = p->impl != HILS_IMPL_GENERIC && prefill_backward_fast_supports(s, p->dtype);
+    if (!fast && (p->impl == HILS_IMPL_FAST || !generic_supports(s))) return HILS_ERR_UNSUPPORTED;
     const size_t need = hils_prefill_backward_workspace_bytes(p);
     if (!workspace || workspace_bytes < need) return HILS_ERR_WORKSPACE;
     if (!aligned16(workspace)) return HILS_ERR_ALIGNMENT;
@@ -491,7 +494,15 @@ int hils_prefill_backward(const hils_params* params, const void* q, const void* 
                       static_cast<int*>(workspace), static_cast<char*>(workspace) + kStatusBytes,
                       workspace_bytes - kStatusBytes};
     trace_begin(st);
-    const int n = launch_backward_generic(s, p->dtype, t, st);
+    int n;
+    if (fast) {
+        // dq is accumulated too on this path (one reduction per slot of a row)
+        if (cudaMemsetAsync(dq, 0, static_cast<size_t>(s.B) * s.Hq * s.R * s.d * sizeof(float), st) != cudaSuccess)
+            return HILS_ERR_CUDA;
+        n = launch_prefill_backward_fast(s, t, st);
+    } else {
+        n = launch_backward_generic(s, p->dtype, t, st);
+    }
     if (n < 0) return n;
     g_last_launches = n;
     return HILS_OK;

@@ -1,0 +1,509 @@
+// Backward of the HiLS operator for the benchmark shapes (bf16, d = 128, S = 64, four query heads per KV head,
+// one landmark per KV head): chunk-major like the forward attend kernel, so that d k and d v of a chunk are
+// accumulated on chip over all the queries that attend it.  Formulas: see backward.cu / the C header.
+//
+// The tiles of the forward's inverse index are reused: a tile is 32 (token, slot) entries x 4 heads = 128 query
+// rows against one 64-key chunk.  A CTA of 8 warps walks a contiguous range of a query block's tiles.  Per tile
+//   phase 1 (warp w owns rows 16w .. 16w+15):  S = Q K^T and T = dO V^T on mma.sync (bf16 -> fp32), the slot's
+//           softmax statistics with quad shuffles, w_j and d s_j; d s and w go to shared memory as bf16;
+//           d Q = d S K (+ the landmark term) is added to dq with vector reductions;
+//   phase 2 (warp w owns dims 16w .. 16w+15):  d K += d S^T Q and d V += W^T dO, contractions over the 128 rows,
+//           accumulated in registers over the run of tiles of one chunk and added to dk / dv when the run ends;
+//           d landmark and d bias of the chunk likewise.
+// K and V of the chunk arrive by TMA (128-byte swizzle), Q and dO rows by cp.async into the same swizzled layout,
+// so that every MMA operand is read with ldmatrix.
+#include "internal.h"
+#include "tma.cuh"
+
+namespace hils {
+namespace {
+
+constexpr int kD = 128;
+constexpr int kS = 64;
+constexpr int kG = 4;
+constexpr int kBfThreads = 256;
+constexpr int kRows = 128;                 // rows of a tile: 32 entries x 4 heads, row = entry * 4 + head
+constexpr int kKBytes = kS * kD * 2;       // 16 KB: two swizzled boxes of 64 dims x 64 keys
+constexpr int kQBytes = kRows * kD * 2;    // 32 KB: two swizzled boxes of 64 dims x 128 rows
+constexpr int kDsBytes = kRows * kS * 2;   // 16 KB: one swizzled box of 64 keys x 128 rows
+
+struct BfArgs {
+    Shape s;
+    const __nv_bfloat16* q;
+    const __nv_bfloat16* dout;
+    const __nv_bfloat16* lm;
+    const float* bias;
+    const float* lse;
+    const float* dsum;        // [B, Hq, R] dout . out
+    const int* entries;
+    const int4* tiles;
+    const int* blk_range;     // {first tile of this query block, first tile of the next}
+    float* dq;
+    float* dk;
+    float* dv;
+    float* dlm;
+    float* dbias;
+    int* status;
+    int i0;                   // first token of the query block
+};
+
+struct BfSmem {
+    uint64_t kv_bar;
+    float lmf[kD];            // the chunk's landmark
+    float dlam[kRows];        // scale * d lambda of each row (0 for local-window and padding rows)
+    float row_lse[kRows];
+    float row_dsum[kRows];
+    int row_orow[kRows];      // (sequence, head, token) row of q / dout / dq, -1 = padding row
+    int row_limit[kRows];     // last valid key column of the row (63 = whole chunk, -1 = none)
+    int row_local[kRows];
+    float bias_c;
+    int abort_flag;
+};
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void red_add_v2(float* p, float x, float y) {
+    asm volatile("red.global.add.v2.f32 [%0], {%1, %2};" ::"l"(p), "f"(x), "f"(y) : "memory");
+}
+
+// Per-row dot products with dout: D = dout . out (one warp per row, 4 dims per lane).
+__global__ void backward_dsum_kernel(const __nv_bfloat16* dout, const __nv_bfloat16* out, float* dsum, long long rows) {
+    const long long row = static_cast<long long>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (row >= rows) return;
+    const int lane = threadIdx.x & 31;
+    const uint2 a = *reinterpret_cast<const uint2*>(dout + row * kD + lane * 4);
+    const uint2 b = *reinterpret_cast<const uint2*>(out + row * kD + lane * 4);
+    const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&a);
+    const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&b);
+    float acc = 0.f;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const float2 x = __bfloat1622float2(pa[i]), y = __bfloat1622float2(pb[i]);
+        acc = fmaf(x.x, y.x, acc);
+        acc = fmaf(x.y, y.y, acc);
+    }
+    acc = warp_sum(acc);
+    if (lane == 0) dsum[row] = acc;
+}
+
+// A fragments (16 rows x 128 dims) of a [128 rows][128 dims] tile stored as two swizzled boxes of 64 dims.
+__device__ __forceinline__ void load_a_frags(uint32_t tile_addr, int r0, int lane, uint32_t (&a)[8][4]) {
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+        const int row = r0 + (lane & 7) + ((lane >> 3) & 1) * 8;
+        const int dim = ks * 16 + (lane >> 4) * 8;
+        ldmatrix_x4(tile_addr + (dim >> 6) * (kRows * 128) + swz128(row, (dim & 63) >> 3), a[ks][0], a[ks][1], a[ks][2],
+                    a[ks][3]);
+    }
+}
+
+// C[16 x 64] = A[16 x 128] B^T, B = a [64 keys][128 dims] tile (two swizzled boxes of 64 dims, 8192 bytes apart).
+__device__ __forceinline__ void rows_times_keys(const uint32_t (&a)[8][4], uint32_t keys_addr, int lane, float (&c)[8][4]) {
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) {
+        c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0.f;
+#pragma unroll
+        for (int kp = 0; kp < 4; ++kp) {
+            const int row = nt * 8 + (lane & 7);
+            const int dim = kp * 32 + (lane >> 3) * 8;
+            uint32_t r0, r1, r2, r3;
+            ldmatrix_x4(keys_addr + (dim >> 6) * 8192 + swz128(row, (dim & 63) >> 3), r0, r1, r2, r3);
+            mma_bf16_16816(c[nt], a[2 * kp], r0, r1);
+            mma_bf16_16816(c[nt], a[2 * kp + 1], r2, r3);
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kBfThreads, 1)
+prefill_backward_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                            const BfArgs a) {
+    extern __shared__ uint8_t bf_raw[];
+    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(bf_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* kbuf = base;
+    uint8_t* vbuf = kbuf + kKBytes;
+    uint8_t* qbuf = vbuf + kKBytes;
+    uint8_t* dobuf = qbuf + kQBytes;
+    uint8_t* dsbuf = dobuf + kQBytes;
+    uint8_t* wbuf = dsbuf + kDsBytes;
+    BfSmem& sm = *reinterpret_cast<BfSmem*>(wbuf + kDsBytes);
+
+    const Shape& s = a.s;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t4 = lane & 3;
+    const int t_begin = a.blk_range[0], n_tiles = a.blk_range[1] - t_begin;
+    const long long lo = t_begin + static_cast<long long>(blockIdx.x) * n_tiles / gridDim.x;
+    const long long hi = t_begin + static_cast<long long>(blockIdx.x + 1) * n_tiles / gridDim.x;
+
+    if (tid == 0) {
+        mbar_init(&sm.kv_bar, 1);
+        mbar_fence_init();
+        sm.abort_flag = 0;
+        tma_prefetch_desc(&map_k);
+        tma_prefetch_desc(&map_v);
+    }
+    __syncthreads();
+
+    const uint32_t k_addr = smem_u32(kbuf), v_addr = smem_u32(vbuf), q_addr = smem_u32(qbuf), do_addr = smem_u32(dobuf);
+    const uint32_t ds_addr = smem_u32(dsbuf), w_addr = smem_u32(wbuf);
+    uint32_t kv_phase = 0;
+    int cur_pair = -1, cur_c = -1;
+    float dk_acc[4][2][4], dv_acc[4][2][4];
+    float lm_acc = 0.f, bias_acc = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 2; ++j)
+#pragma unroll
+            for (int x = 0; x < 4; ++x) dk_acc[i][j][x] = dv_acc[i][j][x] = 0.f;
+
+    // adds the finished chunk's register accumulators to dk, dv, dlandmarks, dbias and clears them
+    auto flush = [&]() {
+        if (cur_pair < 0) return;
+        const int b = cur_pair / s.Hkv, gk = cur_pair % s.Hkv;
+        const long long kvrow0 = static_cast<long long>(cur_pair) * s.T;
+#pragma unroll
+        for (int mt = 0; mt < 4; ++mt)
+#pragma unroll
+            for (int n2 = 0; n2 < 2; ++n2) {
+                const int dim = warp * 16 + n2 * 8 + 2 * t4;
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    const int key = cur_c * kS + mt * 16 + g + hh * 8;
+                    if (key < s.T) {
+                        red_add_v2(a.dk + (kvrow0 + key) * kD + dim, dk_acc[mt][n2][2 * hh], dk_acc[mt][n2][2 * hh + 1]);
+                        red_add_v2(a.dv + (kvrow0 + key) * kD + dim, dv_acc[mt][n2][2 * hh], dv_acc[mt][n2][2 * hh + 1]);
+                    }
+                    dk_acc[mt][n2][2 * hh] = dk_acc[mt][n2][2 * hh + 1] = 0.f;
+                    dv_acc[mt][n2][2 * hh] = dv_acc[mt][n2][2 * hh + 1] = 0.f;
+                }
+            }
+        lm_acc += __shfl_xor_sync(kFullMask, lm_acc, 16);
+        if (cur_c < s.C) {
+            const long long lrow = (static_cast<long long>(b) * s.Hl + gk) * s.C + cur_c;
+            if (lane < 16) atomicAdd(a.dlm + lrow * kD + warp * 16 + lane, lm_acc);
+            if (warp == 0 && lane == 0 && a.dbias) atomicAdd(a.dbias + lrow, bias_acc / s.scale);
+        }
+        lm_acc = 0.f;
+        bias_acc = 0.f;
+    };
+
+    for (long long tile = lo; tile < hi; ++tile) {
+        const int4 rec = a.tiles[tile];
+        const int pair = rec.x, c = rec.y, first = rec.z, ntok = rec.w;
+        const bool newc = pair != cur_pair || c != cur_c;
+        if (newc) {
+            flush();
+            cur_pair = pair;
+            cur_c = c;
+        }
+        const int b = pair / s.Hkv, gk = pair % s.Hkv;
+        __syncthreads();                        // the previous tile's readers are done with every buffer
+
+        if (tid < kRows) {
+            const int e = tid >> 2, h = tid & 3;
+            int orow = -1, limit = -1, local = 0;
+            float lse = 0.f, dsum = 0.f;
+            if (e < ntok) {
+                const int ent = a.entries[first + e];
+                const int tok = a.i0 + (ent >> 8), slot = ent & 255;
+                orow = (b * s.Hq + gk * kG + h) * s.R + tok;
+                local = slot >= s.K ? 1 : 0;
+                limit = local ? min(kS - 1, s.pos0 + tok - c * kS) : kS - 1;
+                lse = a.lse[orow];
+                dsum = a.dsum[orow];
+            }
+            sm.row_orow[tid] = orow;
+            sm.row_limit[tid] = limit;
+            sm.row_local[tid] = local;
+            sm.row_lse[tid] = lse;
+            sm.row_dsum[tid] = dsum;
+        } else if (newc) {
+            const int x = tid - kRows;
+            const long long lrow = (static_cast<long long>(b) * s.Hl + gk) * s.C + c;
+            sm.lmf[x] = c < s.C ? __bfloat162float(a.lm[lrow * kD + x]) : 0.f;
+            if (x == 0) sm.bias_c = (a.bias && c < s.C) ? a.bias[lrow] : 0.f;
+        }
+        if (newc && tid == 0) {
+            const int row = pair * s.T + c * kS;
+            mbar_expect_tx(&sm.kv_bar, 2 * kKBytes);
+            tma_load_2d(kbuf, &map_k, &sm.kv_bar, 0, row);
+            tma_load_2d(kbuf + 8192, &map_k, &sm.kv_bar, 64, row);
+            tma_load_2d(vbuf, &map_v, &sm.kv_bar, 0, row);
+            tma_load_2d(vbuf + 8192, &map_v, &sm.kv_bar, 64, row);
+        }
+        __syncthreads();                        // row table visible
+
+        {   // gather: thread -> (row, 64-dim half) of Q and of dO; padding rows are zero
+            const int row = tid >> 1, half = tid & 1;
+            const int orow = sm.row_orow[row];
+            if (orow >= 0) {
+                const __nv_bfloat16* qs = a.q + static_cast<long long>(orow) * kD + half * 64;
+                const __nv_bfloat16* ds = a.dout + static_cast<long long>(orow) * kD + half * 64;
+#pragma unroll
+                for (int p = 0; p < 8; ++p) {
+                    cp_async16(q_addr + half * (kRows * 128) + swz128(row, p), qs + p * 8);
+                    cp_async16(do_addr + half * (kRows * 128) + swz128(row, p), ds + p * 8);
+                }
+            } else {
+#pragma unroll
+                for (int p = 0; p < 8; ++p) {
+                    *reinterpret_cast<uint4*>(qbuf + half * (kRows * 128) + swz128(row, p)) = make_uint4(0u, 0u, 0u, 0u);
+                    *reinterpret_cast<uint4*>(dobuf + half * (kRows * 128) + swz128(row, p)) = make_uint4(0u, 0u, 0u, 0u);
+                }
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+        }
+        if (newc) {
+            if (!mbar_wait(&sm.kv_bar, kv_phase)) {
+                sm.abort_flag = 1;
+                if (lane == 0) set_status(a.status, kDevTimeout);
+            }
+            kv_phase ^= 1u;
+        }
+        __syncthreads();                        // Q, dO, K, V are in shared memory
+        if (sm.abort_flag) break;
+
+        // ------------------------------------------------------------------ phase 1: rows 16 warp .. 16 warp + 15
+        const int r0 = warp * 16;
+        const int rA = r0 + g, rB = rA + 8;
+        float lamA, lamB;
+        {   // surrogate score of each row: two lanes per row, 64 dims each
+            const int row = r0 + (lane >> 1), half = lane & 1;
+            float acc = 0.f;
+#pragma unroll
+            for (int p = 0; p < 8; ++p) {
+                const uint4 v = *reinterpret_cast<const uint4*>(qbuf + half * (kRows * 128) + swz128(row, p));
+                const __nv_bfloat162* pv = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float2 x = __bfloat1622float2(pv[i]);
+                    acc = fmaf(x.x, sm.lmf[half * 64 + p * 8 + 2 * i], acc);
+                    acc = fmaf(x.y, sm.lmf[half * 64 + p * 8 + 2 * i + 1], acc);
+                }
+            }
+            acc += __shfl_xor_sync(kFullMask, acc, 1);
+            const float lam = acc * s.scale + sm.bias_c;
+            lamA = __shfl_sync(kFullMask, lam, 2 * g);
+            lamB = __shfl_sync(kFullMask, lam, 2 * (g + 8));
+        }
+
+        float sc[8][4], tc[8][4];
+        {
+            uint32_t af[8][4];
+            load_a_frags(q_addr, r0, lane, af);
+            rows_times_keys(af, k_addr, lane, sc);
+            load_a_frags(do_addr, r0, lane, af);
+            rows_times_keys(af, v_addr, lane, tc);
+        }
+
+        float dlam2[2];
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+            const int row = hh ? rB : rA;
+            const int limit = sm.row_limit[row];
+            const bool local = sm.row_local[row] != 0;
+            const float lse = sm.row_lse[row], dsum = sm.row_dsum[row], lam = hh ? lamB : lamA;
+            // the slot's own softmax statistics: computed for every row (the quad shuffles must not sit in a
+            // branch that differs between the rows of a warp), used by the rows of selected chunks only
+            float m = -INFINITY;
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt) m = fmaxf(m, fmaxf(sc[nt][2 * hh], sc[nt][2 * hh + 1]));
+            m = fmaxf(m, __shfl_xor_sync(kFullMask, m, 1));
+            m = fmaxf(m, __shfl_xor_sync(kFullMask, m, 2));
+            m *= s.scale;
+            float Z = 0.f, gt = 0.f;
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt)
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    const float e = __expf(sc[nt][2 * hh + i] * s.scale - m);
+                    Z += e;
+                    gt = fmaf(e, tc[nt][2 * hh + i], gt);
+                }
+            Z += __shfl_xor_sync(kFullMask, Z, 1);
+            Z += __shfl_xor_sync(kFullMask, Z, 2);
+            gt += __shfl_xor_sync(kFullMask, gt, 1);
+            gt += __shfl_xor_sync(kFullMask, gt, 2);
+            float shift = lse, sub = dsum, dl = 0.f;
+            if (!local) {
+                const float gc = gt / Z;
+                const float alpha = __expf(lam - lse);
+                shift = m + __logf(Z) - (lam - lse);
+                sub = gc;
+                dl = limit >= 0 ? alpha * (gc - dsum) * s.scale : 0.f;
+            }
+            dlam2[hh] = dl;
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt)
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    const int col = nt * 8 + 2 * t4 + i;
+                    const float w = col <= limit ? __expf(sc[nt][2 * hh + i] * s.scale - shift) : 0.f;
+                    sc[nt][2 * hh + i] = w * (tc[nt][2 * hh + i] - sub) * s.scale;     // d s_j (times scale)
+                    tc[nt][2 * hh + i] = w;                                           // w_j
+                }
+        }
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt) {
+            *reinterpret_cast<uint32_t*>(dsbuf + swz128(rA, nt) + 4 * t4) = pack_bf16(sc[nt][0], sc[nt][1]);
+            *reinterpret_cast<uint32_t*>(dsbuf + swz128(rB, nt) + 4 * t4) = pack_bf16(sc[nt][2], sc[nt][3]);
+            *reinterpret_cast<uint32_t*>(wbuf + swz128(rA, nt) + 4 * t4) = pack_bf16(tc[nt][0], tc[nt][1]);
+            *reinterpret_cast<uint32_t*>(wbuf + swz128(rB, nt) + 4 * t4) = pack_bf16(tc[nt][2], tc[nt][3]);
+        }
+        if (t4 == 0) {
+            sm.dlam[rA] = dlam2[0];
+            sm.dlam[rB] = dlam2[1];
+        }
+
+        {   // d Q = d S K + d lambda k' for the warp's 16 rows
+            float o[16][4];
+#pragma unroll
+            for (int nt = 0; nt < 16; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+                const uint32_t af[4] = {pack_bf16(sc[2 * kk][0], sc[2 * kk][1]), pack_bf16(sc[2 * kk][2], sc[2 * kk][3]),
+                                        pack_bf16(sc[2 * kk + 1][0], sc[2 * kk + 1][1]),
+                                        pack_bf16(sc[2 * kk + 1][2], sc[2 * kk + 1][3])};
+#pragma unroll
+                for (int dp = 0; dp < 8; ++dp) {
+                    const int mat = lane >> 3;
+                    const int row = kk * 16 + (mat & 1) * 8 + (lane & 7);
+                    const int dim = dp * 16 + (mat >> 1) * 8;
+                    uint32_t r0v, r1v, r2v, r3v;
+                    ldmatrix_x4_trans(k_addr + (dim >> 6) * 8192 + swz128(row, (dim & 63) >> 3), r0v, r1v, r2v, r3v);
+                    mma_bf16_16816(o[2 * dp], af, r0v, r1v);
+                    mma_bf16_16816(o[2 * dp + 1], af, r2v, r3v);
+                }
+            }
+            const int orowA = sm.row_orow[rA], orowB = sm.row_orow[rB];
+#pragma unroll
+            for (int nt = 0; nt < 16; ++nt) {
+                const int col = nt * 8 + 2 * t4;
+                const float l0 = sm.lmf[col], l1 = sm.lmf[col + 1];
+                if (orowA >= 0)
+                    red_add_v2(a.dq + static_cast<long long>(orowA) * kD + col, fmaf(dlam2[0], l0, o[nt][0]),
+                               fmaf(dlam2[0], l1, o[nt][1]));
+                if (orowB >= 0)
+                    red_add_v2(a.dq + static_cast<long long>(orowB) * kD + col, fmaf(dlam2[1], l0, o[nt][2]),
+                               fmaf(dlam2[1], l1, o[nt][3]));
+            }
+        }
+        __syncthreads();                        // d S, W and d lambda of all 128 rows are in shared memory
+
+        // ------------------------------------------------------------------ phase 2: dims 16 warp .. 16 warp + 15
+#pragma unroll 2
+        for (int ks = 0; ks < 8; ++ks) {
+            const int mat = lane >> 3;
+            uint32_t bq[4], bo[4];
+            {
+                const int row = ks * 16 + (mat & 1) * 8 + (lane & 7);
+                const int dim = warp * 16 + (mat >> 1) * 8;
+                const uint32_t off = (dim >> 6) * (kRows * 128) + swz128(row, (dim & 63) >> 3);
+                ldmatrix_x4_trans(q_addr + off, bq[0], bq[1], bq[2], bq[3]);
+                ldmatrix_x4_trans(do_addr + off, bo[0], bo[1], bo[2], bo[3]);
+            }
+#pragma unroll
+            for (int mt = 0; mt < 4; ++mt) {
+                const int row = ks * 16 + (mat >> 1) * 8 + (lane & 7);
+                const uint32_t off = swz128(row, 2 * mt + (mat & 1));
+                uint32_t ad[4], aw[4];
+                ldmatrix_x4_trans(ds_addr + off, ad[0], ad[1], ad[2], ad[3]);
+                ldmatrix_x4_trans(w_addr + off, aw[0], aw[1], aw[2], aw[3]);
+                mma_bf16_16816(dk_acc[mt][0], ad, bq[0], bq[1]);
+                mma_bf16_16816(dk_acc[mt][1], ad, bq[2], bq[3]);
+                mma_bf16_16816(dv_acc[mt][0], aw, bo[0], bo[1]);
+                mma_bf16_16816(dv_acc[mt][1], aw, bo[2], bo[3]);
+            }
+        }
+        {   // d landmark: sum over rows of (scale d lambda_r) q_r, lane -> (dim, half of the rows)
+            const int dim = warp * 16 + (lane & 15), half = lane >> 4;
+            const uint8_t* col = qbuf + (dim >> 6) * (kRows * 128) + (dim & 7) * 2;
+            const int piece = (dim & 63) >> 3;
+            float acc = 0.f;
+#pragma unroll 8
+            for (int r = half * 64; r < half * 64 + 64; ++r) {
+                const float dl = sm.dlam[r];
+                const __nv_bfloat16 x = *reinterpret_cast<const __nv_bfloat16*>(col + swz128(r, piece));
+                acc = fmaf(dl, __bfloat162float(x), acc);
+            }
+            lm_acc += acc;
+            if (warp == 0) {
+                const float v = sm.dlam[lane] + sm.dlam[lane + 32] + sm.dlam[lane + 64] + sm.dlam[lane + 96];
+                bias_acc += warp_sum(v);
+            }
+        }
+    }
+    flush();
+}
+
+}  // namespace
+
+bool prefill_backward_fast_supports(const Shape& s, int dtype) {
+    return prefill_fast_supports(s, dtype) && s.Hl == s.Hkv && s.K + 17 <= 255 &&
+           static_cast<long long>(s.B) * s.Hq * s.R < (1ll << 31);
+}
+
+namespace {
+size_t dsum_bytes(const Shape& s) { return (static_cast<size_t>(s.B) * s.Hq * s.R * sizeof(float) + 255) / 256 * 256; }
+}
+
+size_t prefill_backward_fast_scratch_bytes(const Shape& s) { return dsum_bytes(s) + inverse_index_bytes(s); }
+
+int launch_prefill_backward_fast(const Shape& s, const BackwardTensors& t, cudaStream_t stream) {
+    if (t.scratch_bytes < prefill_backward_fast_scratch_bytes(s)) return HILS_ERR_WORKSPACE;
+    char* sc = static_cast<char*>(t.scratch);
+    float* dsum = reinterpret_cast<float*>(sc);
+    const long long rows = static_cast<long long>(s.B) * s.Hq * s.R;
+    int launches = 0;
+    backward_dsum_kernel<<<static_cast<unsigned>((rows + 7) / 8), 256, 0, stream>>>(
+        static_cast<const __nv_bfloat16*>(t.dout), static_cast<const __nv_bfloat16*>(t.out), dsum, rows);
+    if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
+    trace_mark("backward_dsum", stream);
+    ++launches;
+
+    InverseIndex ix;
+    const int rc = build_inverse_index(s, t.sel_idx, sc + dsum_bytes(s), t.scratch_bytes - dsum_bytes(s), &ix, stream);
+    if (rc < 0) return rc;
+    launches += rc;
+
+    CUtensorMap map_k, map_v;
+    const uint64_t kv_rows = static_cast<uint64_t>(s.B) * s.Hkv * s.T;
+    if (!make_bf16_2d_map(&map_k, t.k, kv_rows, kD, 64, kS) || !make_bf16_2d_map(&map_v, t.v, kv_rows, kD, 64, kS))
+        return HILS_ERR_CUDA;
+    const size_t smem = 2 * kKBytes + 2 * kQBytes + 2 * kDsBytes + sizeof(BfSmem) + 1024;
+    static bool attr_done = false;
+    if (!attr_done) {
+        if (cudaFuncSetAttribute(prefill_backward_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(smem)) != cudaSuccess)
+            return HILS_ERR_CUDA;
+        attr_done = true;
+    }
+    BfArgs a;
+    a.s = s;
+    a.q = static_cast<const __nv_bfloat16*>(t.q);
+    a.dout = static_cast<const __nv_bfloat16*>(t.dout);
+    a.lm = static_cast<const __nv_bfloat16*>(t.landmarks);
+    a.bias = t.bias;
+    a.lse = t.lse;
+    a.dsum = dsum;
+    a.entries = ix.entries;
+    a.tiles = ix.tiles;
+    a.dq = t.dq;
+    a.dk = t.dk;
+    a.dv = t.dv;
+    a.dlm = t.dlandmarks;
+    a.dbias = t.dbias;
+    a.status = t.status;
+    for (int blk = 0; blk < ix.n_blocks; ++blk) {
+        a.blk_range = ix.blk_toff + blk;
+        a.i0 = blk * ix.qb;
+        prefill_backward_mma_kernel<<<148, kBfThreads, smem, stream>>>(map_k, map_v, a);
+        if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
+        trace_mark("backward_attend", stream);
+        ++launches;
+    }
+    return launches;
+}
+
+}  // namespace hils

@@ -70,6 +70,20 @@ int launch_landmark_summary(int dtype, int B, int Hkv, int Hl, int C, int d, int
                             const void* lq, const void* k, const int32_t* seq_lens, int c0, int cn, void* landmarks,
                             float* bias, cudaStream_t stream);
 
+// Chunk-major index of a selection (the structure the prefill attend kernel walks): for every query block of
+// `qb` tokens, (sequence, KV head) pair and chunk, the (token, slot) entries that attend that chunk, padded to
+// tiles of `tile_tok` entries.  entries[e] = ((token - block start) << 8) | slot, slot >= K = local-window chunk;
+// tiles[t] = {pair, chunk, first entry, entries in the tile}; blk_toff[b] = first tile of query block b.
+struct InverseIndex {
+    int qb, nc, n_blocks, max_tiles, tile_tok;
+    const int* entries;
+    const int4* tiles;
+    const int* blk_toff;
+};
+size_t inverse_index_bytes(const Shape& s);
+int build_inverse_index(const Shape& s, const int32_t* sel, void* scratch, size_t bytes, InverseIndex* ix,
+                        cudaStream_t stream);
+
 // Backward through `out` (selection fixed): inputs of the forward, what it wrote, dout; fp32 gradients.
 struct BackwardTensors {
     const void* q;
@@ -91,6 +105,10 @@ struct BackwardTensors {
     size_t scratch_bytes;
 };
 int launch_backward_generic(const Shape& s, int dtype, const BackwardTensors& t, cudaStream_t stream);
+// chunk-major mma.sync path for the benchmark shapes (bf16, d = 128, S = 64, G = 4, Hl = Hkv)
+bool prefill_backward_fast_supports(const Shape& s, int dtype);
+size_t prefill_backward_fast_scratch_bytes(const Shape& s);
+int launch_prefill_backward_fast(const Shape& s, const BackwardTensors& t, cudaStream_t stream);
 
 // Chunk-id overlap of blocks of M adjacent queries (Sec. "Chunk Overlap"): stats [pairs, nblk, 4], overlap [pairs, nblk].
 bool chunk_overlap_supports(int C);

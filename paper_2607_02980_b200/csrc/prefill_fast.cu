@@ -569,6 +569,54 @@ bool prefill_fast_supports(const Shape& s, int dtype) {
 
 size_t prefill_fast_scratch_bytes(const Shape& s) { return make_plan(s).total; }
 
+// The inverse index on its own (the backward pass walks the same chunk-major tiles): per-(query block, pair, chunk)
+// entry lists and the tile table, built from a selection that is already in memory.
+size_t inverse_index_bytes(const Shape& s) { return make_plan(s).off_obuf; }
+
+int build_inverse_index(const Shape& s, const int32_t* sel, void* scratch, size_t bytes, InverseIndex* ix,
+                        cudaStream_t stream) {
+    const Plan p = make_plan(s);
+    if (bytes < p.off_obuf) return HILS_ERR_WORKSPACE;
+    const int pairs = s.B * s.Hkv;
+    char* sc = static_cast<char*>(scratch);
+    PArgs a = {};
+    a.s = s;
+    a.sel = const_cast<int32_t*>(sel);
+    a.cnt = reinterpret_cast<int*>(sc + p.off_cnt);
+    a.cursor = reinterpret_cast<int*>(sc + p.off_cursor);
+    a.blk_toff = reinterpret_cast<int*>(sc + p.off_ntiles);
+    a.n_blocks = p.n_blocks;
+    a.seg_tiles = reinterpret_cast<int*>(sc + p.off_seg);
+    a.off = reinterpret_cast<int*>(sc + p.off_off);
+    a.entries = reinterpret_cast<int*>(sc + p.off_entries);
+    a.epos = reinterpret_cast<int*>(sc + p.off_epos);
+    a.tiles = reinterpret_cast<int4*>(sc + p.off_tiles);
+    a.max_tiles = p.max_tiles;
+    a.qb = p.qb;
+    a.nc = p.nc;
+    a.tile_tok = attend_tc_tile_tokens();
+    if (cudaMemsetAsync(sc + p.off_cnt, 0, p.zero_bytes, stream) != cudaSuccess) return HILS_ERR_CUDA;
+    const long long elems = static_cast<long long>(pairs) * s.R * (s.K + max_local_slots(s.W));
+    const long long want = (elems + 255) / 256;
+    const unsigned eb = static_cast<unsigned>(want < 148 * 16 ? want : 148 * 16);
+    const unsigned nseg = static_cast<unsigned>((static_cast<long long>(p.n_blocks) * pairs * p.nc + 1023) / 1024);
+    invert_count_kernel<<<eb, 256, 0, stream>>>(a);
+    invert_segsum_kernel<<<nseg, 1024, 0, stream>>>(a);
+    invert_scan_kernel<<<nseg, 1024, 0, stream>>>(a);
+    invert_fill_kernel<<<eb, 256, 0, stream>>>(a);
+    if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
+    trace_mark("backward_invert", stream);
+    ix->qb = p.qb;
+    ix->nc = p.nc;
+    ix->n_blocks = p.n_blocks;
+    ix->max_tiles = p.max_tiles;
+    ix->tile_tok = a.tile_tok;
+    ix->entries = a.entries;
+    ix->tiles = a.tiles;
+    ix->blk_toff = a.blk_toff;
+    return 4;
+}
+
 int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
     const Plan p = make_plan(s);
     if (t.scratch_bytes < p.total) return HILS_ERR_WORKSPACE;

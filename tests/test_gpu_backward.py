@@ -66,6 +66,33 @@ def test_backward_matches_oracle(name):
     compare(grads, ref, cfg.dtype)
 
 
+FAST_CASES = {
+    "bf16_gqa": CASES["bf16_gqa"],
+    "bf16_window": CASES["bf16_window"],
+    # more than one query block of 4096 tokens, ragged tiles, runs of a chunk split across CTAs
+    # (K = 2 keeps the single-threaded oracle, one thread per (sequence, KV head), under a minute)
+    "bf16_two_query_blocks": (wl.CONFIGS[1].scaled(B=1, Hq=4, Hkv=1, L=4400, K=2, seed=207), None, 1, True),
+    "bf16_window_512": (wl.CONFIGS[1].scaled(B=1, Hq=8, Hkv=2, L=1500, K=5, seed=208), None, 512, True),
+}
+
+
+@pytest.mark.parametrize("name", list(FAST_CASES))
+def test_tensor_core_backward_matches_oracle(name):
+    cfg, Hl, W, with_bias = FAST_CASES[name]
+    grads, ref = run_case(cfg, Hl, W, with_bias, impl="fast")
+    assert hils.last_launch_count() >= 6          # dsum + 4 index kernels + one backward kernel per query block
+    compare(grads, ref, cfg.dtype)
+
+
+def test_fast_path_refuses_shapes_it_does_not_take():
+    cfg = wl.CONFIGS[0].scaled(L=128, seed=209)   # fp32
+    inp = {n: t.to(DEV) for n, t in wl.make_prefill_inputs(cfg, "cpu").items()}
+    out, lse, sel = hils.hils_prefill(inp["q"], inp["k"], inp["v"], inp["landmarks"], cfg.S, cfg.K)
+    with pytest.raises(hils.HilsError):
+        hils.hils_prefill_backward(inp["q"], inp["k"], inp["v"], inp["landmarks"], cfg.S, cfg.K, out, lse, sel,
+                                   torch.ones_like(inp["q"]), impl="fast")
+
+
 def test_missing_arguments_are_refused():
     cfg = wl.CONFIGS[0].scaled(L=128, seed=206)
     inp = {n: t.to(DEV) for n, t in wl.make_prefill_inputs(cfg, "cpu").items()}
