@@ -345,6 +345,43 @@ def bench_landmark_summary(hils, w, peaks, iters=10):
             "l2_policy": "K tensor of %.0f MB > 126 MB L2, read once per call" % (k.numel() * k.element_size() / 1e6)}
 
 
+class BackwardWorkload:
+    """hils_prefill_backward on a prefill workload's tensors (its forward has run: out, lse, sel_idx are set)."""
+
+    def __init__(self, w):
+        self.hils, self.w = w.hils, w
+        self.dout = torch.randn(w.inp["q"].shape, generator=torch.Generator(device=w.dev).manual_seed(77),
+                                device=w.dev, dtype=torch.float32).to(w.inp["q"].dtype)
+        self.flush = None
+        # five matrix products per (row, selected key) against the forward's two
+        self.work = 2.5 * w.work
+
+    def between_steps(self):
+        pass
+
+    def step(self):
+        w, i = self.w, self.w.inp
+        self.grads = self.hils.hils_prefill_backward(i["q"], i["k"], i["v"], i["landmarks"], w.cfg.S, w.cfg.K, w.out,
+                                                     w.lse, w.sel, self.dout, bias=w.bias, window=w.window)
+
+
+def bench_backward(hils, w, peaks, steps, barrier):
+    """The backward pass on the workload (gradients through `out`, selection fixed): whole-call time and the
+    per-kernel split.  FLOP = 2.5 x the forward's gathered-attention FLOP (S, dO V^T, dQ, dK, dV)."""
+    bw = BackwardWorkload(w)
+    ms, _ = time_steps(bw, steps, 3, barrier)
+    km = kernel_times(bw, 3, barrier)
+    t = float(np.mean(ms))
+    val = bw.work / (t * 1e-3) / 1e12
+    n_launch = hils.last_launch_count()
+    del bw
+    return {"metric": "hils_prefill_backward_effective_TFLOPs", "value": val, "unit": "TFLOP/s", "ms_per_step": t,
+            "median_ms": float(np.median(ms)), "kernel_ms": km, "launches_per_step": n_launch,
+            "frac_of_measured_bf16_burst": val / peaks["bf16_tflops"],
+            "inputs": "larger than L2: q, dout, out %.0f MB each; dq fp32 %.0f MB" % (
+                w.inp["q"].numel() * 2 / 1e6, w.inp["q"].numel() * 4 / 1e6)}
+
+
 def bench_chunk_overlap(hils, w, peaks, M=16, iters=10):
     """Chunk-id overlap of blocks of M adjacent queries (Sec. "Chunk Overlap", Eq. Overlap) on the selection the
     workload's last prefill wrote: the statistics, and the kernel's time against reading sel_idx once."""
@@ -482,8 +519,16 @@ def main():
         for _ in range(2):
             hils.hils_landmark_summary(lq, w.inp["k"], cfg.S)
         torch.cuda.synchronize()
+        bwd_calls = 0
+        if not w.decode and cfg.dtype == "bf16":
+            # the backward pass over the same tensors (two calls)
+            bw = BackwardWorkload(w)
+            for _ in range(2):
+                bw.step()
+            torch.cuda.synchronize()
+            bwd_calls = 2
         print(json.dumps({"profile_run": cfg.name, "B": cfg.B, "calls": args.warmup + args.steps,
-                          "kernels_per_call": kpc, "landmark_summary_calls": 2}))
+                          "kernels_per_call": kpc, "landmark_summary_calls": 2, "backward_calls": bwd_calls}))
         return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -580,6 +625,12 @@ def main():
     # ---- other configurations (reported beside, never instead of, the primary workload)
     if not args.no_extra and world == 1:
         extras = {}
+        if not w.decode and cfg.dtype == "bf16":
+            try:
+                extras[args.workload + "_backward"] = bench_backward(hils, w, peaks, max(3, args.steps), barrier)
+                launches += extras[args.workload + "_backward"]["launches_per_step"] * (max(3, args.steps) + 6)
+            except Exception as exc:
+                extras[args.workload + "_backward"] = {"error": repr(exc)}
         del w
         torch.cuda.empty_cache()
         for name in ("cfg2", "cfg3", "cfg4", "cfg0"):
@@ -609,6 +660,8 @@ def main():
                 if name == "cfg2":
                     extras["cfg2_chunk_overlap_iid_queries"] = bench_chunk_overlap(hils, ew, peaks)
                     launches += 13
+                    extras["cfg2_backward"] = bench_backward(hils, ew, peaks, 3, barrier)
+                    launches += extras["cfg2_backward"]["launches_per_step"] * 9
                 del ew
                 if name == "cfg2":
                     # adjacent queries that retrieve mostly the same chunks, as the paper measures on a trained model

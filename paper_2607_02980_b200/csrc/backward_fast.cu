@@ -51,11 +51,12 @@ struct BfSmem {
     uint64_t kv_bar;
     float lmf[kD];            // the chunk's landmark
     float dlam[kRows];        // scale * d lambda of each row (0 for local-window and padding rows)
-    float row_lse[kRows];
-    float row_dsum[kRows];
-    int row_orow[kRows];      // (sequence, head, token) row of q / dout / dq, -1 = padding row
-    int row_limit[kRows];     // last valid key column of the row (63 = whole chunk, -1 = none)
-    int row_local[kRows];
+    // row tables of the tile in work and of the next one
+    float row_lse[2][kRows];
+    float row_dsum[2][kRows];
+    int row_orow[2][kRows];   // (sequence, head, token) row of q / dout / dq, -1 = padding row
+    int row_limit[2][kRows];  // last valid key column of the row (63 = whole chunk, -1 = none)
+    int row_local[2][kRows];
     float bias_c;
     int abort_flag;
 };
@@ -87,30 +88,36 @@ __global__ void backward_dsum_kernel(const __nv_bfloat16* dout, const __nv_bfloa
     if (lane == 0) dsum[row] = acc;
 }
 
-// A fragments (16 rows x 128 dims) of a [128 rows][128 dims] tile stored as two swizzled boxes of 64 dims.
-__device__ __forceinline__ void load_a_frags(uint32_t tile_addr, int r0, int lane, uint32_t (&a)[8][4]) {
+// C[16 x 64] = A[16 x 128] B^T.  A = rows r0 .. r0+15 of a [128 rows][128 dims] tile (two swizzled boxes of 64
+// dims, kRows * 128 bytes apart), B = a [64 keys][128 dims] tile (two swizzled boxes, 8192 bytes apart).
+// The 32-dim step is the outer loop so that consecutive MMAs go to different accumulators (the instructions are
+// issued in program order; a chain on one accumulator would wait for each result).
+__device__ __forceinline__ void rows_times_keys(uint32_t rows_addr, int r0, uint32_t keys_addr, int lane, float (&c)[8][4]) {
 #pragma unroll
-    for (int ks = 0; ks < 8; ++ks) {
-        const int row = r0 + (lane & 7) + ((lane >> 3) & 1) * 8;
-        const int dim = ks * 16 + (lane >> 4) * 8;
-        ldmatrix_x4(tile_addr + (dim >> 6) * (kRows * 128) + swz128(row, (dim & 63) >> 3), a[ks][0], a[ks][1], a[ks][2],
-                    a[ks][3]);
-    }
-}
-
-// C[16 x 64] = A[16 x 128] B^T, B = a [64 keys][128 dims] tile (two swizzled boxes of 64 dims, 8192 bytes apart).
-__device__ __forceinline__ void rows_times_keys(const uint32_t (&a)[8][4], uint32_t keys_addr, int lane, float (&c)[8][4]) {
+    for (int nt = 0; nt < 8; ++nt) c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0.f;
 #pragma unroll
-    for (int nt = 0; nt < 8; ++nt) {
-        c[nt][0] = c[nt][1] = c[nt][2] = c[nt][3] = 0.f;
+    for (int kp = 0; kp < 4; ++kp) {
+        uint32_t a0[4], a1[4];
+        {
+            const int row = r0 + (lane & 7) + ((lane >> 3) & 1) * 8;
+            const int dim = kp * 32 + (lane >> 4) * 8;
+            ldmatrix_x4(rows_addr + (dim >> 6) * (kRows * 128) + swz128(row, (dim & 63) >> 3), a0[0], a0[1], a0[2], a0[3]);
+            ldmatrix_x4(rows_addr + ((dim + 16) >> 6) * (kRows * 128) + swz128(row, ((dim + 16) & 63) >> 3), a1[0], a1[1],
+                        a1[2], a1[3]);
+        }
 #pragma unroll
-        for (int kp = 0; kp < 4; ++kp) {
-            const int row = nt * 8 + (lane & 7);
-            const int dim = kp * 32 + (lane >> 3) * 8;
-            uint32_t r0, r1, r2, r3;
-            ldmatrix_x4(keys_addr + (dim >> 6) * 8192 + swz128(row, (dim & 63) >> 3), r0, r1, r2, r3);
-            mma_bf16_16816(c[nt], a[2 * kp], r0, r1);
-            mma_bf16_16816(c[nt], a[2 * kp + 1], r2, r3);
+        for (int ng = 0; ng < 2; ++ng) {
+            uint32_t b[4][4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int row = (ng * 4 + i) * 8 + (lane & 7);
+                const int dim = kp * 32 + (lane >> 3) * 8;
+                ldmatrix_x4(keys_addr + (dim >> 6) * 8192 + swz128(row, (dim & 63) >> 3), b[i][0], b[i][1], b[i][2], b[i][3]);
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) mma_bf16_16816(c[ng * 4 + i], a0, b[i][0], b[i][1]);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) mma_bf16_16816(c[ng * 4 + i], a1, b[i][2], b[i][3]);
         }
     }
 }
@@ -122,9 +129,9 @@ prefill_backward_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(bf_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* kbuf = base;
     uint8_t* vbuf = kbuf + kKBytes;
-    uint8_t* qbuf = vbuf + kKBytes;
-    uint8_t* dobuf = qbuf + kQBytes;
-    uint8_t* dsbuf = dobuf + kQBytes;
+    uint8_t* qbuf0 = vbuf + kKBytes;             // [2][kQBytes]: the tile in work and the next one
+    uint8_t* dobuf0 = qbuf0 + 2 * kQBytes;       // [2][kQBytes]
+    uint8_t* dsbuf = dobuf0 + 2 * kQBytes;
     uint8_t* wbuf = dsbuf + kDsBytes;
     BfSmem& sm = *reinterpret_cast<BfSmem*>(wbuf + kDsBytes);
 
@@ -143,7 +150,7 @@ prefill_backward_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     }
     __syncthreads();
 
-    const uint32_t k_addr = smem_u32(kbuf), v_addr = smem_u32(vbuf), q_addr = smem_u32(qbuf), do_addr = smem_u32(dobuf);
+    const uint32_t k_addr = smem_u32(kbuf), v_addr = smem_u32(vbuf);
     const uint32_t ds_addr = smem_u32(dsbuf), w_addr = smem_u32(wbuf);
     uint32_t kv_phase = 0;
     int cur_pair = -1, cur_c = -1;
@@ -187,82 +194,114 @@ prefill_backward_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
         bias_acc = 0.f;
     };
 
-    for (long long tile = lo; tile < hi; ++tile) {
-        const int4 rec = a.tiles[tile];
-        const int pair = rec.x, c = rec.y, first = rec.z, ntok = rec.w;
-        const bool newc = pair != cur_pair || c != cur_c;
-        if (newc) {
-            flush();
-            cur_pair = pair;
-            cur_c = c;
-        }
+    // Requests the chunk's K and V (TMA, thread 0) and reads its landmark and bias (threads 128..255).  Called when
+    // nobody reads the previous chunk's copies any more.
+    auto issue_chunk = [&](int pair, int c) {
         const int b = pair / s.Hkv, gk = pair % s.Hkv;
-        __syncthreads();                        // the previous tile's readers are done with every buffer
-
-        if (tid < kRows) {
-            const int e = tid >> 2, h = tid & 3;
-            int orow = -1, limit = -1, local = 0;
-            float lse = 0.f, dsum = 0.f;
-            if (e < ntok) {
-                const int ent = a.entries[first + e];
-                const int tok = a.i0 + (ent >> 8), slot = ent & 255;
-                orow = (b * s.Hq + gk * kG + h) * s.R + tok;
-                local = slot >= s.K ? 1 : 0;
-                limit = local ? min(kS - 1, s.pos0 + tok - c * kS) : kS - 1;
-                lse = a.lse[orow];
-                dsum = a.dsum[orow];
-            }
-            sm.row_orow[tid] = orow;
-            sm.row_limit[tid] = limit;
-            sm.row_local[tid] = local;
-            sm.row_lse[tid] = lse;
-            sm.row_dsum[tid] = dsum;
-        } else if (newc) {
-            const int x = tid - kRows;
-            const long long lrow = (static_cast<long long>(b) * s.Hl + gk) * s.C + c;
-            sm.lmf[x] = c < s.C ? __bfloat162float(a.lm[lrow * kD + x]) : 0.f;
-            if (x == 0) sm.bias_c = (a.bias && c < s.C) ? a.bias[lrow] : 0.f;
-        }
-        if (newc && tid == 0) {
+        if (tid == 0) {
             const int row = pair * s.T + c * kS;
             mbar_expect_tx(&sm.kv_bar, 2 * kKBytes);
             tma_load_2d(kbuf, &map_k, &sm.kv_bar, 0, row);
             tma_load_2d(kbuf + 8192, &map_k, &sm.kv_bar, 64, row);
             tma_load_2d(vbuf, &map_v, &sm.kv_bar, 0, row);
             tma_load_2d(vbuf + 8192, &map_v, &sm.kv_bar, 64, row);
+        } else if (tid >= kRows) {
+            const int x = tid - kRows;
+            const long long lrow = (static_cast<long long>(b) * s.Hl + gk) * s.C + c;
+            sm.lmf[x] = c < s.C ? __bfloat162float(a.lm[lrow * kD + x]) : 0.f;
+            if (x == 0) sm.bias_c = (a.bias && c < s.C) ? a.bias[lrow] : 0.f;
         }
-        __syncthreads();                        // row table visible
-
-        {   // gather: thread -> (row, 64-dim half) of Q and of dO; padding rows are zero
-            const int row = tid >> 1, half = tid & 1;
-            const int orow = sm.row_orow[row];
-            if (orow >= 0) {
-                const __nv_bfloat16* qs = a.q + static_cast<long long>(orow) * kD + half * 64;
-                const __nv_bfloat16* ds = a.dout + static_cast<long long>(orow) * kD + half * 64;
+    };
+    // Starts the gather of a tile's Q and dO rows into buffer `par` (thread -> row tid / 2, 64-dim half tid & 1;
+    // padding rows are zero) and returns what the row table needs; store_row() writes it once the loads are back.
+    struct RowInfo { int orow, limit, local; float lse, dsum; };
+    // entry of this thread's row in a tile (read two tiles ahead of its use, so that no tile waits for it)
+    auto load_entry = [&](const int4 rec) { return (tid >> 3) < rec.w ? a.entries[rec.z + (tid >> 3)] : 0; };
+    auto issue_tile = [&](const int4 rec, int ent, int par) {
+        const int pair = rec.x, c = rec.y, ntok = rec.w;
+        const int b = pair / s.Hkv, gk = pair % s.Hkv;
+        const int row = tid >> 1, half = tid & 1, e = row >> 2, h = row & 3;
+        RowInfo ri{-1, -1, 0, 0.f, 0.f};
+        uint8_t* qb = qbuf0 + par * kQBytes + half * (kRows * 128);
+        uint8_t* db = dobuf0 + par * kQBytes + half * (kRows * 128);
+        if (e < ntok) {
+            const int tok = a.i0 + (ent >> 8), slot = ent & 255;
+            ri.orow = (b * s.Hq + gk * kG + h) * s.R + tok;
+            ri.local = slot >= s.K ? 1 : 0;
+            ri.limit = ri.local ? min(kS - 1, s.pos0 + tok - c * kS) : kS - 1;
+            const __nv_bfloat16* qs = a.q + static_cast<long long>(ri.orow) * kD + half * 64;
+            const __nv_bfloat16* ds = a.dout + static_cast<long long>(ri.orow) * kD + half * 64;
+            const uint32_t qa = smem_u32(qb), da = smem_u32(db);
 #pragma unroll
-                for (int p = 0; p < 8; ++p) {
-                    cp_async16(q_addr + half * (kRows * 128) + swz128(row, p), qs + p * 8);
-                    cp_async16(do_addr + half * (kRows * 128) + swz128(row, p), ds + p * 8);
-                }
-            } else {
-#pragma unroll
-                for (int p = 0; p < 8; ++p) {
-                    *reinterpret_cast<uint4*>(qbuf + half * (kRows * 128) + swz128(row, p)) = make_uint4(0u, 0u, 0u, 0u);
-                    *reinterpret_cast<uint4*>(dobuf + half * (kRows * 128) + swz128(row, p)) = make_uint4(0u, 0u, 0u, 0u);
-                }
+            for (int p = 0; p < 8; ++p) {
+                cp_async16(qa + swz128(row, p), qs + p * 8);
+                cp_async16(da + swz128(row, p), ds + p * 8);
             }
-            asm volatile("cp.async.commit_group;" ::: "memory");
-            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            if (half == 0) {
+                ri.lse = a.lse[ri.orow];
+                ri.dsum = a.dsum[ri.orow];
+            }
+        } else {
+#pragma unroll
+            for (int p = 0; p < 8; ++p) {
+                *reinterpret_cast<uint4*>(qb + swz128(row, p)) = make_uint4(0u, 0u, 0u, 0u);
+                *reinterpret_cast<uint4*>(db + swz128(row, p)) = make_uint4(0u, 0u, 0u, 0u);
+            }
         }
-        if (newc) {
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        return ri;
+    };
+    auto store_row = [&](const RowInfo& ri, int par) {
+        if ((tid & 1) == 0) {
+            const int row = tid >> 1;
+            sm.row_orow[par][row] = ri.orow;
+            sm.row_limit[par][row] = ri.limit;
+            sm.row_local[par][row] = ri.local;
+            sm.row_lse[par][row] = ri.lse;
+            sm.row_dsum[par][row] = ri.dsum;
+        }
+    };
+
+    const int4 no_tile = make_int4(-1, -1, 0, 0);
+    int4 rec = no_tile, nrec = no_tile, n2rec = no_tile;       // this tile, the next one, the one after
+    int nent = 0;                                              // this thread's entry in the next tile
+    bool kv_issued = false;
+    if (lo < hi) {
+        rec = a.tiles[lo];
+        if (lo + 1 < hi) nrec = a.tiles[lo + 1];
+        if (lo + 2 < hi) n2rec = a.tiles[lo + 2];
+        issue_chunk(rec.x, rec.y);
+        kv_issued = true;
+        store_row(issue_tile(rec, load_entry(rec), 0), 0);
+        nent = load_entry(nrec);
+    }
+    for (long long tile = lo; tile < hi; ++tile) {
+        const int par = static_cast<int>(tile - lo) & 1;
+        const int pair = rec.x, c = rec.y;
+        cur_pair = pair;
+        cur_c = c;
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        if (kv_issued) {
             if (!mbar_wait(&sm.kv_bar, kv_phase)) {
                 sm.abort_flag = 1;
                 if (lane == 0) set_status(a.status, kDevTimeout);
             }
             kv_phase ^= 1u;
+            kv_issued = false;
         }
-        __syncthreads();                        // Q, dO, K, V are in shared memory
+        __syncthreads();                        // this tile's Q, dO, row table, K, V, landmark are in shared memory;
+                                                // the previous tile's readers are done with the other buffers
         if (sm.abort_flag) break;
+        // the next tile's rows start to arrive while this one is computed
+        const bool has_next = tile + 1 < hi;
+        RowInfo nri{-1, -1, 0, 0.f, 0.f};
+        if (has_next) nri = issue_tile(nrec, nent, par ^ 1);
+        // metadata of the tiles after the next: in registers by the time they are needed
+        const int n2ent = load_entry(n2rec);
+        const int4 n3rec = tile + 3 < hi ? a.tiles[tile + 3] : no_tile;
+        const bool next_new = has_next && (nrec.x != pair || nrec.y != c);
+        const uint8_t* qbuf = qbuf0 + par * kQBytes;
+        const uint32_t q_addr = smem_u32(qbuf), do_addr = smem_u32(dobuf0 + par * kQBytes);
 
         // ------------------------------------------------------------------ phase 1: rows 16 warp .. 16 warp + 15
         const int r0 = warp * 16;
@@ -289,21 +328,16 @@ prefill_backward_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
         }
 
         float sc[8][4], tc[8][4];
-        {
-            uint32_t af[8][4];
-            load_a_frags(q_addr, r0, lane, af);
-            rows_times_keys(af, k_addr, lane, sc);
-            load_a_frags(do_addr, r0, lane, af);
-            rows_times_keys(af, v_addr, lane, tc);
-        }
+        rows_times_keys(q_addr, r0, k_addr, lane, sc);
+        rows_times_keys(do_addr, r0, v_addr, lane, tc);
 
         float dlam2[2];
 #pragma unroll
         for (int hh = 0; hh < 2; ++hh) {
             const int row = hh ? rB : rA;
-            const int limit = sm.row_limit[row];
-            const bool local = sm.row_local[row] != 0;
-            const float lse = sm.row_lse[row], dsum = sm.row_dsum[row], lam = hh ? lamB : lamA;
+            const int limit = sm.row_limit[par][row];
+            const bool local = sm.row_local[par][row] != 0;
+            const float lse = sm.row_lse[par][row], dsum = sm.row_dsum[par][row], lam = hh ? lamB : lamA;
             // the slot's own softmax statistics: computed for every row (the quad shuffles must not sit in a
             // branch that differs between the rows of a warp), used by the rows of selected chunks only
             float m = -INFINITY;
@@ -376,7 +410,7 @@ prefill_backward_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
                     mma_bf16_16816(o[2 * dp + 1], af, r2v, r3v);
                 }
             }
-            const int orowA = sm.row_orow[rA], orowB = sm.row_orow[rB];
+            const int orowA = sm.row_orow[par][rA], orowB = sm.row_orow[par][rB];
 #pragma unroll
             for (int nt = 0; nt < 16; ++nt) {
                 const int col = nt * 8 + 2 * t4;
@@ -389,7 +423,12 @@ prefill_backward_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
                                fmaf(dlam2[1], l1, o[nt][3]));
             }
         }
+        if (has_next) store_row(nri, par ^ 1);
         __syncthreads();                        // d S, W and d lambda of all 128 rows are in shared memory
+        if (next_new) {                         // K, V and the landmark are not read in phase 2: fetch the next chunk's
+            issue_chunk(nrec.x, nrec.y);
+            kv_issued = true;
+        }
 
         // ------------------------------------------------------------------ phase 2: dims 16 warp .. 16 warp + 15
 #pragma unroll 2
@@ -433,8 +472,13 @@ prefill_backward_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
                 bias_acc += warp_sum(v);
             }
         }
+        if (!has_next || next_new) flush();
+        rec = nrec;
+        nrec = n2rec;
+        nent = n2ent;
+        n2rec = n3rec;
     }
-    flush();
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
 
 }  // namespace
@@ -471,7 +515,7 @@ int launch_prefill_backward_fast(const Shape& s, const BackwardTensors& t, cudaS
     const uint64_t kv_rows = static_cast<uint64_t>(s.B) * s.Hkv * s.T;
     if (!make_bf16_2d_map(&map_k, t.k, kv_rows, kD, 64, kS) || !make_bf16_2d_map(&map_v, t.v, kv_rows, kD, 64, kS))
         return HILS_ERR_CUDA;
-    const size_t smem = 2 * kKBytes + 2 * kQBytes + 2 * kDsBytes + sizeof(BfSmem) + 1024;
+    const size_t smem = 2 * kKBytes + 4 * kQBytes + 2 * kDsBytes + sizeof(BfSmem) + 1024;
     static bool attr_done = false;
     if (!attr_done) {
         if (cudaFuncSetAttribute(prefill_backward_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
