@@ -422,6 +422,37 @@ def hils_prefill_backward(q, k, v, landmarks, chunk_size: int, top_k: int, out, 
     return dq, dk, dv, dlm, dbias
 
 
+class _HilsAttentionFn(torch.autograd.Function):
+    """hils_prefill / hils_prefill_backward as one differentiable op (argument marshalling only: both passes run
+    in the library's kernels).  The selection is a constant of the backward pass; lse and sel_idx are returned
+    without gradient."""
+
+    @staticmethod
+    def forward(ctx, q, k, v, landmarks, bias, chunk_size, top_k, window, scale):
+        out, lse, sel = hils_prefill(q, k, v, landmarks, chunk_size, top_k, bias=bias, window=window, scale=scale)
+        ctx.save_for_backward(q, k, v, landmarks, bias if bias is not None else q.new_empty(0), out, lse, sel)
+        ctx.has_bias = bias is not None
+        ctx.cfg = (chunk_size, top_k, window, scale)
+        ctx.mark_non_differentiable(lse, sel)
+        return out, lse, sel
+
+    @staticmethod
+    def backward(ctx, dout, _dlse, _dsel):
+        q, k, v, landmarks, bias, out, lse, sel = ctx.saved_tensors
+        chunk_size, top_k, window, scale = ctx.cfg
+        dq, dk, dv, dlm, db = hils_prefill_backward(q, k, v, landmarks, chunk_size, top_k, out, lse, sel,
+                                                    dout.contiguous(), bias=bias if ctx.has_bias else None,
+                                                    window=window, scale=scale)
+        return (dq.to(q.dtype), dk.to(k.dtype), dv.to(v.dtype), dlm.to(landmarks.dtype),
+                db if ctx.has_bias else None, None, None, None, None)
+
+
+def hils_attention(q, k, v, landmarks, chunk_size: int, top_k: int, *, bias=None, window: int = 1, scale: float = 0.0):
+    """Differentiable HiLS prefill for training: returns (out, lse, sel_idx); gradients flow through `out` to
+    q, k, v, landmarks and bias (cast to the inputs' dtypes)."""
+    return _HilsAttentionFn.apply(q, k, v, landmarks, bias, chunk_size, top_k, window, scale)
+
+
 def hils_chunk_overlap(sel_idx, block_queries: int, num_chunks: int, *, stats=None, overlap=None, stream=None):
     """Chunk-id overlap of blocks of `block_queries` adjacent queries (Sec. "Chunk Overlap", Eq. Overlap).
 

@@ -93,6 +93,26 @@ def test_fast_path_refuses_shapes_it_does_not_take():
                                    torch.ones_like(inp["q"]), impl="fast")
 
 
+def test_autograd_wrapper_routes_both_passes_through_the_library():
+    cfg = wl.CONFIGS[1].scaled(B=1, Hq=8, Hkv=2, L=512, K=4, seed=210)
+    inp = wl.make_prefill_inputs(cfg, "cpu")
+    bias = torch.randn(inp["landmarks"].shape[:3], generator=torch.Generator().manual_seed(3)) * 0.5
+    dout = torch.randn(inp["q"].shape, generator=torch.Generator().manual_seed(4)).to(torch.bfloat16)
+    leaves = {n: t.to(DEV).requires_grad_(True) for n, t in inp.items()}
+    bg = bias.to(DEV).requires_grad_(True)
+    out, lse, sel = hils.hils_attention(leaves["q"], leaves["k"], leaves["v"], leaves["landmarks"], cfg.S, cfg.K, bias=bg)
+    assert not lse.requires_grad and not sel.requires_grad
+    (out.float() * dout.to(DEV).float()).sum().backward()
+    ref = oracle.hils_backward(inp["q"], inp["k"], inp["v"], inp["landmarks"], bias, sel.cpu(), dout.float(),
+                               S=cfg.S, K=cfg.K)
+    got = (leaves["q"].grad, leaves["k"].grad, leaves["v"].grad, leaves["landmarks"].grad, bg.grad)
+    for g, n in zip(got, ("dq", "dk", "dv", "dlandmarks", "dbias")):
+        assert g is not None
+        r = ref[n]
+        # the wrapper rounds the gradients to the inputs' dtype (bf16) on top of the kernel's own error
+        assert np.abs(g.float().cpu().numpy() - r).max() <= 2.5e-2 * np.abs(r).max(), n
+
+
 def test_missing_arguments_are_refused():
     cfg = wl.CONFIGS[0].scaled(L=128, seed=206)
     inp = {n: t.to(DEV) for n, t in wl.make_prefill_inputs(cfg, "cpu").items()}
