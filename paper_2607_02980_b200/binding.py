@@ -287,7 +287,8 @@ def hils_decode_noalloc(q, k_cache, v_cache, landmarks, seq_lens, chunk_size: in
 
 
 def hils_prefill_at(q, k, v, landmarks, chunk_size: int, top_k: int, pos0: int, stream=None, *, bias=None,
-                    window: int = 1, scale: float = 0.0, impl: str = "auto", out=None, lse=None, sel_idx=None):
+                    window: int = 1, scale: float = 0.0, impl: str = "auto", out=None, lse=None, sel_idx=None,
+                    workspace=None):
     """hils_prefill for the L query tokens at positions pos0 .. pos0 + L - 1 of sequences whose caches k, v
     [B,Hkv,T,d] hold at least pos0 + L tokens (chunked prefill / multi-token decode).  Returns (out, lse, sel_idx)."""
     lib = load_library()
@@ -306,7 +307,10 @@ def hils_prefill_at(q, k, v, landmarks, chunk_size: int, top_k: int, pos0: int, 
     nbytes = int(lib.hils_prefill_at_workspace_bytes(ctypes.byref(p), int(pos0)))
     if nbytes == 0:
         raise HilsError(-2, "hils_prefill_at_workspace_bytes")
-    ws = torch.zeros(nbytes, dtype=torch.uint8, device=q.device)
+    if workspace is None:
+        workspace = torch.empty(nbytes, dtype=torch.uint8, device=q.device)
+        workspace[:256].zero_()                   # only the status block has to start at zero
+    ws = workspace
     out = torch.empty((B, Hq, L, d), dtype=dt, device=q.device) if out is None else out
     lse = torch.empty((B, Hq, L), dtype=torch.float32, device=q.device) if lse is None else lse
     sel_idx = torch.empty((B, Hkv, L, top_k), dtype=torch.int32, device=q.device) if sel_idx is None else sel_idx
@@ -413,7 +417,8 @@ def hils_prefill_backward(q, k, v, landmarks, chunk_size: int, top_k: int, out, 
         n = int(lib.hils_prefill_backward_workspace_bytes(ctypes.byref(p)))
         if n == 0:
             raise HilsError(-2, "hils_prefill_backward_workspace_bytes")
-        workspace = torch.zeros(n, dtype=torch.uint8, device=q.device)
+        workspace = torch.empty(n, dtype=torch.uint8, device=q.device)
+        workspace[:256].zero_()
     rc = lib.hils_prefill_backward(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(landmarks), _ptr(bias), _ptr(out),
                                    _ptr(lse), _ptr(sel_idx), _ptr(dout), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dlm),
                                    _ptr(dbias), _ptr(workspace), workspace.numel(), _stream_ptr(stream))

@@ -531,7 +531,10 @@ Plan make_plan(const Shape& s) {
     for (size_t b = 0; b < nblocks; ++b) {
         const size_t toks = (b + 1) * blk <= static_cast<size_t>(s.R) ? blk : static_cast<size_t>(s.R) - b * blk;
         const size_t vis = ((s.pos0 + b * blk + toks) + kS - 1) / kS;
-        const size_t tiles = pairs * (toks * (s.K + max_local_slots(s.W)) / tt + (vis < nc ? vis : nc)) + 1;
+        // (and never more than its entries: a list that exists holds at least one)
+        const size_t ents = pairs * toks * (s.K + max_local_slots(s.W));
+        const size_t ragged = pairs * (toks * (s.K + max_local_slots(s.W)) / tt + (vis < nc ? vis : nc));
+        const size_t tiles = (ents < ragged ? ents : ragged) + 1;
         all_tiles += tiles;
         max_blk = tiles > max_blk ? tiles : max_blk;
     }
