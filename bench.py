@@ -320,6 +320,40 @@ def bench_paged_decode(hils, w, peaks, iters=10):
             "frac_of_measured_hbm": w.rate(m * 1e-3) / peaks["hbm_gbs"], "pages": int(B * C), "page_tokens": S}
 
 
+def bench_multi_token_decode(hils, w, peaks, M=4, iters=10):
+    """M new tokens per sequence in one hils_decode_multi call on the decode workload's caches (the caches hold
+    them already).  Bytes = M single-token decodes' algorithmic bytes (every token scans the landmarks and
+    gathers its own chunks); tokens of a sequence that retrieve the same chunk find it in L2."""
+    cfg, i = w.cfg, w.inp
+    q = torch.stack([w.queries[m % len(w.queries)] for m in range(M)], dim=1).contiguous()     # [B, M, Hq, d]
+    out = torch.empty_like(q)
+    lse = torch.empty((cfg.B, M, cfg.Hq), dtype=torch.float32, device=q.device)
+    sel = torch.empty((cfg.B, M, cfg.Hkv, cfg.K), dtype=torch.int32, device=q.device)
+    import ctypes
+    n = hils.load_library().hils_decode_multi_workspace_bytes(ctypes.byref(w.p), M)
+    ws = torch.zeros(n, dtype=torch.uint8, device=q.device)
+
+    def call():
+        hils.hils_decode_multi(q, i["k"], i["v"], i["landmarks"], i["seq_lens"], cfg.S, cfg.K, out=out, lse=lse,
+                               sel_idx=sel, workspace=ws)
+    for _ in range(3):
+        w.between_steps()
+        call()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(iters)]
+    torch.cuda.synchronize()
+    for a, b in ev:
+        w.between_steps()
+        a.record()
+        call()
+        b.record()
+    torch.cuda.synchronize()
+    ms = float(np.mean([a.elapsed_time(b) for a, b in ev]))
+    return {"metric": "hils_decode_algorithmic_GBps", "tokens_per_seq": M, "ms_per_step": ms, "ms_per_token": ms / M,
+            "value": M * w.work / (ms * 1e-3) / 1e9, "unit": "GB/s",
+            "frac_of_measured_hbm": M * w.work / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+            "l2_policy": "L2 flushed between calls; tokens of one sequence share landmark rows within a call"}
+
+
 def bench_landmark_summary(hils, w, peaks, iters=10):
     """The chunk-summary kernel (Proposition 3.1) on the workload's K tensor: every chunk of every KV head once.
     HBM-bound; algorithmic bytes = K read once + the learnable queries read + the summaries written."""
@@ -656,6 +690,8 @@ def main():
                     launches += 13
                 if name == "cfg3":
                     extras["cfg3_paged"] = bench_paged_decode(hils, ew, peaks)
+                    launches += 3 * 13
+                    extras["cfg3_multi_token_decode"] = bench_multi_token_decode(hils, ew, peaks)
                     launches += 3 * 13
                 if name == "cfg2":
                     extras["cfg2_chunk_overlap_iid_queries"] = bench_chunk_overlap(hils, ew, peaks)

@@ -171,6 +171,27 @@ int hils_decode_paged(const hils_params* params, const void* q, const void* k_pa
                       const int32_t* seq_lens, void* out, float* lse, int32_t* sel_idx, void* workspace,
                       size_t workspace_bytes, void* stream);
 
+/* Multi-token decode: M = tokens_per_seq new tokens per sequence in one call (speculative decoding, verification
+ * of draft tokens; Sec. "Hardware-Efficient Kernel Design" names it as a use of packing adjacent queries).  The
+ * caches already hold all M new tokens; token m of sequence b sits at position seq_lens[b] - M + m and is
+ * treated exactly like a single-token hils_decode at length seq_lens[b] - M + m + 1: the call runs the decode
+ * kernels over B * M queries that share the caches, landmarks and bias of their sequence.
+ *
+ *   q        [B, M, Hq, d]     DEVICE        out     [B, M, Hq, d]
+ *   lse      [B, M, Hq] fp32                 sel_idx [B, M, Hkv, K] int32
+ *   seq_lens [B] int32 DEVICE: lengths INCLUDING the M new tokens (a sequence with seq_lens[b] < M has tokens
+ *            at negative positions: those queries get zero output and the device status is set)
+ *   k_cache, v_cache, landmarks, bias: as for hils_decode ([B, ...], params->B = B); with block_table != NULL
+ *            they are page pools addressed as in hils_decode_paged ([B, C] table, shared by the M queries)
+ * Supported by the bandwidth-tuned decode kernels only (bf16, d = 128, S = 64, at most 8 query heads per KV
+ * head): other shapes, and params->impl = HILS_IMPL_GENERIC, return HILS_ERR_UNSUPPORTED (use hils_prefill_at).
+ * Workspace: hils_decode_multi_workspace_bytes(params, M).  Errors as for hils_decode. */
+size_t hils_decode_multi_workspace_bytes(const hils_params* params, int32_t tokens_per_seq);
+int hils_decode_multi(const hils_params* params, int32_t tokens_per_seq, const void* q, const void* k_cache,
+                      const void* v_cache, const void* landmarks, const float* bias, const int32_t* block_table,
+                      int32_t num_pages, const int32_t* seq_lens, void* out, float* lse, int32_t* sel_idx,
+                      void* workspace, size_t workspace_bytes, void* stream);
+
 /* Chunk summaries -- the step upstream of the operator (Proposition 3.1, Eq. LogSumExp linearization /
  * Eq. prop_q_c).  For every sequence b, landmark head hl (its KV head is hl / (Hl / Hkv)) and chunk
  * c in [chunk_begin, chunk_begin + chunk_count), with the chunk's keys k_j, j in [c*S, min((c+1)*S, len_b))

@@ -26,7 +26,7 @@ EXPORTS = [
     "hils_status_string", "hils_version", "hils_trace_enable", "hils_trace_read", "hils_decode_noalloc",
     "hils_landmark_summary", "hils_decode_paged", "hils_prefill_at", "hils_prefill_at_workspace_bytes",
     "hils_prefill_routed", "hils_decode_routed", "hils_chunk_overlap", "hils_prefill_backward",
-    "hils_prefill_backward_workspace_bytes",
+    "hils_prefill_backward_workspace_bytes", "hils_decode_multi", "hils_decode_multi_workspace_bytes",
 ]
 
 
@@ -90,6 +90,11 @@ def load_library() -> ctypes.CDLL:
     lib.hils_prefill_backward.restype = ctypes.c_int
     lib.hils_prefill_backward.argtypes = [pp, vp, vp, vp, vp, f32p, vp, f32p, i32p, vp, f32p, f32p, f32p, f32p, f32p,
                                           vp, ctypes.c_size_t, vp]
+    lib.hils_decode_multi_workspace_bytes.restype = ctypes.c_size_t
+    lib.hils_decode_multi_workspace_bytes.argtypes = [pp, ctypes.c_int32]
+    lib.hils_decode_multi.restype = ctypes.c_int
+    lib.hils_decode_multi.argtypes = [pp, ctypes.c_int32, vp, vp, vp, vp, f32p, i32p, ctypes.c_int32, i32p, vp, f32p,
+                                      i32p, vp, ctypes.c_size_t, vp]
     lib.hils_chunk_overlap.restype = ctypes.c_int
     lib.hils_chunk_overlap.argtypes = [pp, i32p, ctypes.c_int32, i32p, f32p, vp]
     lib.hils_poll_status.restype = ctypes.c_int
@@ -482,6 +487,55 @@ def hils_chunk_overlap(sel_idx, block_queries: int, num_chunks: int, *, stats=No
     if rc != 0:
         raise HilsError(rc, "hils_chunk_overlap")
     return stats, overlap
+
+
+def hils_decode_multi(q, k_cache, v_cache, landmarks, seq_lens, chunk_size: int, top_k: int, stream=None, *,
+                      bias=None, window: int = 1, scale: float = 0.0, block_table=None, out=None, lse=None,
+                      sel_idx=None, workspace=None):
+    """Multi-token decode: q [B,M,Hq,d], the M newest tokens of every sequence (already in the caches; seq_lens [B]
+    counts them).  Caches [B,Hkv,T,d], or page pools [P,Hkv,S,d] with block_table [B,C].
+    Returns (out [B,M,Hq,d], lse [B,M,Hq], sel_idx [B,M,Hkv,K])."""
+    lib = load_library()
+    B, M, Hq, d = q.shape
+    Hkv = k_cache.shape[1]
+    Hl, C = landmarks.shape[1], landmarks.shape[2]
+    dt = q.dtype
+    _check(q, "q", (B, M, Hq, d), dt, True)
+    _check(landmarks, "landmarks", (B, Hl, C, d), dt, True)
+    _check(seq_lens, "seq_lens", (B,), torch.int32, True)
+    num_pages = 0
+    if block_table is None:
+        T = k_cache.shape[2]
+        _check(k_cache, "k_cache", (B, Hkv, T, d), dt, True)
+        _check(v_cache, "v_cache", (B, Hkv, T, d), dt, True)
+    else:
+        num_pages = k_cache.shape[0]
+        T = C * chunk_size
+        _check(k_cache, "k_pages", (num_pages, Hkv, chunk_size, d), dt, True)
+        _check(v_cache, "v_pages", (num_pages, Hkv, chunk_size, d), dt, True)
+        _check(block_table, "block_table", (B, C), torch.int32, True)
+    if bias is not None:
+        _check(bias, "bias", (B, Hl, C), torch.float32, True)
+    out = torch.empty_like(q) if out is None else out
+    lse = torch.empty((B, M, Hq), dtype=torch.float32, device=q.device) if lse is None else lse
+    sel_idx = torch.empty((B, M, Hkv, top_k), dtype=torch.int32, device=q.device) if sel_idx is None else sel_idx
+    _check(out, "out", (B, M, Hq, d), dt, True)
+    _check(lse, "lse", (B, M, Hq), torch.float32, True)
+    _check(sel_idx, "sel_idx", (B, M, Hkv, top_k), torch.int32, True)
+    p = make_params(B=B, Hq=Hq, Hkv=Hkv, Hl=Hl, L=0, T_max=T, C=C, d=d, chunk_size=chunk_size, top_k=top_k,
+                    window=window, scale=scale, dtype=_dtype_code(q), impl="auto")
+    if workspace is None:
+        n = int(lib.hils_decode_multi_workspace_bytes(ctypes.byref(p), int(M)))
+        if n == 0:
+            raise HilsError(-2, "hils_decode_multi_workspace_bytes")
+        workspace = torch.empty(n, dtype=torch.uint8, device=q.device)
+        workspace[:256].zero_()
+    rc = lib.hils_decode_multi(ctypes.byref(p), int(M), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(landmarks),
+                               _ptr(bias), _ptr(block_table), int(num_pages), _ptr(seq_lens), _ptr(out), _ptr(lse),
+                               _ptr(sel_idx), _ptr(workspace), workspace.numel(), _stream_ptr(stream))
+    if rc != 0:
+        raise HilsError(rc, "hils_decode_multi")
+    return out, lse, sel_idx
 
 
 class HostRunner:

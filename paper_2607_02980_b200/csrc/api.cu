@@ -59,6 +59,7 @@ int make_shape(const hils_params* p, int is_decode, Shape* s, long long pos0 = 0
     s->scale = p->scale > 0.f ? p->scale : 1.0f / sqrtf(static_cast<float>(p->d));
     s->is_decode = is_decode;
     s->pos0 = 0;
+    s->qps = 1;
     if (is_decode) {
         if (p->T_max < 1) return HILS_ERR_INVALID_ARG;
         s->R = 1;
@@ -107,11 +108,17 @@ size_t scratch_bytes(const Shape& s, Path path) {
 int run(const hils_params* p, int is_decode, const void* q, const void* k, const void* v, const void* lm,
         const float* bias, const int32_t* seq_lens, void* out, float* lse, int32_t* sel, void* ws,
         size_t ws_bytes, void* stream_v, const int32_t* block_table = nullptr, int num_pages = 0, long long pos0 = 0,
-        const void* q_route = nullptr) {
+        const void* q_route = nullptr, int qps = 1) {
     g_last_launches = 0;
     Shape s;
     int rc = make_shape(p, is_decode, &s, pos0);
     if (rc != HILS_OK) return rc;
+    if (qps != 1) {
+        // multi-token decode: qps queries per sequence, run as B * qps decode queries over shared caches
+        if (!is_decode || qps < 1 || static_cast<long long>(s.B) * qps > (1 << 24)) return HILS_ERR_INVALID_ARG;
+        s.B *= qps;
+        s.qps = qps;
+    }
     if (!q || !k || !v || !lm || !out || !lse || !sel || (is_decode && !seq_lens)) return HILS_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(lm) || !aligned16(out) ||
         (reinterpret_cast<uintptr_t>(lse) & 3u) || (reinterpret_cast<uintptr_t>(sel) & 3u) ||
@@ -120,6 +127,7 @@ int run(const hils_params* p, int is_decode, const void* q, const void* k, const
     Path path;
     rc = pick_path(s, p, &path);
     if (rc != HILS_OK) return rc;
+    if (qps != 1 && path != Path::DecodeFast) return HILS_ERR_UNSUPPORTED;     // shared caches: TMA decode kernels only
     if (block_table) {
         // paged caches: only the TMA decode kernels address K / V through a page table
         if (path != Path::DecodeFast) return HILS_ERR_UNSUPPORTED;
@@ -398,6 +406,26 @@ int hils_decode_paged(const hils_params* params, const void* q, const void* k_pa
     if (!block_table) return HILS_ERR_INVALID_ARG;
     return run(params, 1, q, k_pages, v_pages, landmarks, bias, seq_lens, out, lse, sel_idx, workspace, workspace_bytes,
                stream, block_table, num_pages);
+}
+
+size_t hils_decode_multi_workspace_bytes(const hils_params* params, int32_t tokens_per_seq) {
+    Shape s;
+    if (tokens_per_seq < 1 || make_shape(params, 1, &s) != HILS_OK) return 0;
+    if (static_cast<long long>(s.B) * tokens_per_seq > (1 << 24)) return 0;
+    s.B *= tokens_per_seq;
+    s.qps = tokens_per_seq;
+    if (params->impl == HILS_IMPL_GENERIC || !decode_fast_supports(s, params->dtype)) return 0;
+    return kStatusBytes + align_up(decode_fast_scratch_bytes(s), 256);
+}
+
+int hils_decode_multi(const hils_params* params, int32_t tokens_per_seq, const void* q, const void* k_cache,
+                      const void* v_cache, const void* landmarks, const float* bias, const int32_t* block_table,
+                      int32_t num_pages, const int32_t* seq_lens, void* out, float* lse, int32_t* sel_idx,
+                      void* workspace, size_t workspace_bytes, void* stream) {
+    if (tokens_per_seq < 1) return HILS_ERR_INVALID_ARG;
+    if (params && params->impl == HILS_IMPL_GENERIC) return HILS_ERR_UNSUPPORTED;
+    return run(params, 1, q, k_cache, v_cache, landmarks, bias, seq_lens, out, lse, sel_idx, workspace, workspace_bytes,
+               stream, block_table, num_pages, 0, nullptr, tokens_per_seq);
 }
 
 int hils_decode_noalloc(const hils_params* params, const void* q, const void* k_cache, const void* v_cache,

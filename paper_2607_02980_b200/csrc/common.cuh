@@ -26,6 +26,8 @@ struct Shape {
     int is_decode;
     int pos0;       // prefill: sequence position of query row 0 (rows are the tokens pos0 .. pos0 + R - 1 of a cache
                     // of T tokens); 0 for a whole-sequence prefill
+    int qps;        // decode: queries per sequence (multi-token decode).  B then counts queries: query b belongs to
+                    // cache sequence b / qps and is its token number b % qps of the qps newest ones; 1 otherwise
 };
 
 __host__ __device__ inline int floordiv_i(int a, int b) {

@@ -64,6 +64,11 @@ struct DArgs {
 // with its own softmax; its mass is the exact log-sum-exp of its scores, so mixing by the masses reproduces the
 // single softmax over the window (Eq. chunk mass).  Candidates for selection are the chunks 0 .. lc - 1.
 __host__ __device__ inline int max_local_slots(int W) { return (W - 1 + kS - 1) / kS + 1; }
+// Multi-token decode: query b of the call sees the cache of sequence b / qps up to and including its own token.
+__device__ __forceinline__ int query_seq_len(const DArgs& a, int b) {
+    const int q = a.s.qps;
+    return q == 1 ? a.seq_lens[b] : a.seq_lens[b / q] - (q - 1) + b % q;
+}
 __device__ __forceinline__ int first_local_chunk(int seq, int W) { return local_lo(seq - 1, W, kS) / kS; }
 
 // ------------------------------------------------------------------------------------------ select
@@ -325,7 +330,7 @@ __device__ void select_pair(const DArgs& a, int pair, int ncand, SelShared& sh, 
     //     loads, then every thread computes (chunk, head) dot products
     __nv_bfloat16 (*lm_s)[kD + 8] = reinterpret_cast<__nv_bfloat16 (*)[kD + 8]>(dyn);
     const int per = s.Hl / s.Hkv;                        // landmark rows per chunk: 1, or one per query head (G)
-    const long long lrow0 = (static_cast<long long>(b) * s.Hl + g * per) * s.C;      // landmark head 0 of this KV head
+    const long long lrow0 = (static_cast<long long>(b / s.qps) * s.Hl + g * per) * s.C;      // landmark head 0 of this KV head
     const __nv_bfloat16* qg = a.q_route + (static_cast<long long>(b) * s.Hq + g * G) * kD;     // fusion scores: q-hat
     for (int x = tid; x < G * 16; x += NT)
         *reinterpret_cast<uint4*>(&sh.q_s[x >> 4][(x & 15) * 8]) = *reinterpret_cast<const uint4*>(qg + (x >> 4) * kD + (x & 15) * 8);
@@ -391,7 +396,7 @@ __global__ void __launch_bounds__(kScoreThreads) decode_score_kernel(const DArgs
     const Shape& s = a.s;
     const int pair = blockIdx.y;
     const int b = pair / s.Hkv, g = pair % s.Hkv;
-    const int seq = a.seq_lens[b];
+    const int seq = query_seq_len(a, b);
     if (seq < 1 || seq > s.T) return;
     const int ncand = first_local_chunk(seq, s.W);
     const int c_begin = blockIdx.x * kScoreChunksPerCta;
@@ -421,7 +426,7 @@ __global__ void __launch_bounds__(kScoreThreads) decode_score_kernel(const DArgs
         best[it][0] = best[it][1] = -INFINITY;
     }
     for (int hh = 0; hh < per; ++hh) {
-        const long long lrow = (static_cast<long long>(b) * s.Hl + g * per + hh) * s.C;
+        const long long lrow = (static_cast<long long>(b / s.qps) * s.Hl + g * per + hh) * s.C;
         const __nv_bfloat16* lm = a.lm + lrow * kD;
         const float* bias = a.bias ? a.bias + lrow : nullptr;
         uint4 x[2][2][4];
@@ -477,7 +482,7 @@ __global__ void __launch_bounds__(512) decode_select_kernel(const DArgs a) {
     const Shape& s = a.s;
     const int pair = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
     const int b = pair / s.Hkv, g = pair % s.Hkv;
-    const int seq = a.seq_lens[b];
+    const int seq = query_seq_len(a, b);
     if (seq < 1 || seq > s.T) {
         // invalid length: flag it, emit empty outputs
         if (tid == 0) { set_status(a.status, kDevBadIndex); a.pair_n[pair] = -1; a.done[pair] = 0; }
@@ -541,7 +546,7 @@ decode_attend_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
                 c = slot < n ? a.sel[static_cast<long long>(pair) * K + slot] : -1;
             } else {
                 // slot K + r: chunk lc + r of the local window; only the query's own chunk can be partial
-                const int seq = a.seq_lens[pair / s.Hkv];
+                const int seq = query_seq_len(a, pair / s.Hkv);
                 const int ci = (seq - 1) / kS;
                 c = first_local_chunk(seq, s.W) + (slot - K);
                 if (c > ci) c = -1;
@@ -551,7 +556,7 @@ decode_attend_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
         int row = 0;
         if (c >= 0) {
             if (a.block_table) {
-                const int page = a.block_table[static_cast<long long>(pair / s.Hkv) * s.C + c];
+                const int page = a.block_table[static_cast<long long>(pair / s.Hkv / s.qps) * s.C + c];
                 if (page < 0 || page >= a.num_pages) {       // flag it and skip the chunk
                     set_status(a.status, kDevBadIndex);
                     c = -1;
@@ -559,7 +564,7 @@ decode_attend_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
                     row = (page * s.Hkv + pair % s.Hkv) * kS;
                 }
             } else {
-                row = pair * s.T + c * kS;
+                row = ((pair / s.Hkv / s.qps) * s.Hkv + pair % s.Hkv) * s.T + c * kS;
             }
         }
         sm.item_chunk[j] = c;
@@ -741,7 +746,7 @@ decode_attend_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
             __threadfence();
             const int last_cta = cta_of_item(pair_end - 1, N, a.n_ctas);
             const int nparts = min(a.max_parts, last_cta - first_cta + 1);
-            const int seq_b = a.seq_lens[b];
+            const int seq_b = query_seq_len(a, b);
             const int nl = (seq_b - 1) / kS - first_local_chunk(seq_b, s.W) + 1;
             for (int x = tid; x < G * kD; x += kConsumerWarps * 32) {
                 const int h = x / kD;
@@ -870,7 +875,8 @@ int launch_decode_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
     a.num_pages = t.num_pages;
 
     CUtensorMap map_k, map_v;
-    const uint64_t rows = t.block_table ? static_cast<uint64_t>(t.num_pages) * s.Hkv * kS : static_cast<uint64_t>(pairs) * s.T;
+    const uint64_t rows = t.block_table ? static_cast<uint64_t>(t.num_pages) * s.Hkv * kS
+                                        : static_cast<uint64_t>(pairs / s.qps) * s.T;
     if (!make_bf16_2d_map(&map_k, t.k, rows, kD, 64, kS) || !make_bf16_2d_map(&map_v, t.v, rows, kD, 64, kS))
         return HILS_ERR_CUDA;
 
