@@ -270,8 +270,9 @@ size_t hils_host_arena_bytes(const hils_params* params, int is_decode);
  * runs, and out / lse / sel_idx are copied back, all enqueued on `stream`.  The call returns
  * without synchronising: results are valid once the stream has been synchronised.  The arena's
  * first 256 bytes are the status word (zero them once). */
-/* Sequences of at least 8192 tokens go through hils_prefill_host in blocks of 4096 tokens (the operator is causal:
- * a block needs only the inputs up to its own end): copy-in, kernels (hils_prefill_at) and copy-out of
+/* Sequences of at least 8192 tokens go through hils_prefill_host in blocks of 4096 tokens, the last 4096 cut into
+ * 1/2, 1/4, 1/4 (the operator is causal: a block needs only the inputs up to its own end; the last block's
+ * kernels and copy-out overlap nothing, so it is kept short): copy-in, kernels (hils_prefill_at) and copy-out of
  * neighbouring blocks overlap on three internal streams, created on first use, that fork from and join `stream`;
  * calls that take this route are serialised on the host by a mutex (their events are shared).  Results are those
  * of hils_prefill.  HILS_HOST_PIPELINE=0 in the environment keeps the single-stream form. */

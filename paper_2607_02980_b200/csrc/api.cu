@@ -2,6 +2,7 @@
 #include <string.h>
 
 #include <mutex>
+#include <vector>
 
 #include "internal.h"
 
@@ -190,7 +191,10 @@ int arena_layout(const hils_params* p, int is_decode, ArenaLayout* a) {
 // The operator is causal, so a block of query tokens needs only the inputs up to its own end: blocks of
 // kHostBlock tokens are copied in, computed (the slice entry point) and copied out on three internal streams,
 // and the transfers of neighbouring blocks overlap each other (PCIe is full duplex) and the kernels.
-constexpr int kHostBlock = 4096;
+#ifndef HILS_HOST_BLOCK
+#define HILS_HOST_BLOCK 4096
+#endif
+constexpr int kHostBlock = HILS_HOST_BLOCK;
 
 struct HostPipe {
     bool ok = false;
@@ -229,12 +233,34 @@ int run_host_prefill_pipelined(const hils_params* p, const ArenaLayout& full, co
     Shape s;
     if (make_shape(p, 0, &s) != HILS_OK) return 1;
     const size_t eb = elem_bytes(p->dtype);
-    const int L = p->L, nb = (L + kHostBlock - 1) / kHostBlock;
+    const int L = p->L;
+    // Block schedule: kHostBlock tokens each, the last stretch in shrinking pieces (1/2, 1/4, 1/4): what cannot
+    // overlap anything is the last block's compute and copy-out, so that block is kept short.
+    std::vector<int> blk_i0, blk_len;
+    {
+        int i0 = 0;
+        while (L - i0 > kHostBlock) { blk_i0.push_back(i0); blk_len.push_back(kHostBlock); i0 += kHostBlock; }
+        const int rem = L - i0;
+        const int half = (rem / 2 + 63) / 64 * 64, quarter = (rem / 4 + 63) / 64 * 64;
+        int cuts[3] = {half, quarter, rem};
+        for (int c = 0; c < 3 && i0 < L; ++c) {
+            const int len = c == 2 ? L - i0 : (cuts[c] < L - i0 ? cuts[c] : L - i0);
+            if (len <= 0) continue;
+            blk_i0.push_back(i0);
+            blk_len.push_back(len);
+            i0 += len;
+        }
+    }
+    const int nb = static_cast<int>(blk_i0.size());
     hils_params bp = *p;
     bp.T_max = L;
-    bp.L = kHostBlock;
-    const size_t ws_b = hils_prefill_at_workspace_bytes(&bp, static_cast<int64_t>(nb - 1) * kHostBlock);
-    if (ws_b == 0) return 1;
+    size_t ws_b = 0;
+    for (int b = 0; b < nb; ++b) {
+        bp.L = blk_len[b];
+        const size_t need = hils_prefill_at_workspace_bytes(&bp, blk_i0[b]);
+        if (need == 0) return 1;
+        ws_b = need > ws_b ? need : ws_b;
+    }
     // layout inside the caller's arena: workspace, K, V, landmarks, bias, then two slots of per-block q / out / lse / sel
     const size_t rowsq = static_cast<size_t>(s.B) * s.Hq, rowskv = static_cast<size_t>(s.B) * s.Hkv;
     const size_t q_blk = rowsq * kHostBlock * s.d * eb, lse_blk = rowsq * kHostBlock * 4;
@@ -260,7 +286,7 @@ int run_host_prefill_pipelined(const hils_params* p, const ArenaLayout& full, co
     int launches = 0;
     const size_t tok_b = static_cast<size_t>(s.d) * eb;                  // bytes per token row
     for (int b = 0; b < nb; ++b) {
-        const int i0 = b * kHostBlock, len = (L - i0 < kHostBlock) ? L - i0 : kHostBlock, sl = b & 1;
+        const int i0 = blk_i0[b], len = blk_len[b], sl = b & 1;
         // ---- copy in: this block's K / V rows into the device caches, its queries into slot sl
         if (b >= 2) ok = ok && cudaStreamWaitEvent(hp->in, hp->cmp_done[sl], 0) == cudaSuccess;
         ok = ok && cudaMemcpy2DAsync(base + a_k + i0 * tok_b, L * tok_b, static_cast<const char*>(k) + i0 * tok_b, L * tok_b,
