@@ -140,6 +140,8 @@ DECODE_SMALL = {
     "bf16_k_ge_chunks": (wl.CONFIGS[3].scaled(B=3, L=2048, K=64, seed=42), [2048, 1000, 65]),
     "bf16_cfg4_like": (wl.CONFIGS[4].scaled(B=2, L=32768, K=64, seed=43), [32768, 32700]),
     "f32_g1_d64": (wl.CONFIGS[0].scaled(mode="decode", B=4, L=1024, K=4, seed=44), [1024, 1, 64, 500]),
+    # long candidate lists whose length is 1 / 0 / 15 past a multiple of 16
+    "bf16_long_candidate_lists": (wl.CONFIGS[3].scaled(B=3, L=65536, K=8, seed=50), [65536, 64 * 640 + 5, 64 * 625 + 64]),
     # many (sequence, KV head) pairs: every persistent CTA walks several pairs and wraps its TMA ring
     "bf16_many_pairs": (wl.CONFIGS[3].scaled(B=64, L=2048, K=16, seed=49),
                         [2048 - 37 * (i % 11) - (1 if i % 3 == 0 else 0) for i in range(64)]),
@@ -166,6 +168,27 @@ def test_decode_with_bias(impl):
     inp = wl.make_decode_inputs(cfg, "cpu", seq_lens=torch.tensor([8192, 8000, 4097], dtype=torch.int32))
     bias = wl.make_bias(cfg, "cpu")
     out, lse, sel = run_decode(cfg, inp, impl, bias=bias)
+    check_decode(cfg, inp, out, lse, sel, bias=bias)
+
+
+def test_decode_selection_reaches_the_last_candidates_of_long_lists():
+    """Long candidate lists with a bias that forces the very last candidate chunk and the one 16 before it into
+    the selection (the ends of the warps' slices of the list)."""
+    cfg = wl.CONFIGS[3].scaled(B=2, L=65536, K=8, seed=51)
+    fast_or_skip(cfg, True)
+    seq = [64 * 641 + 3, 64 * 655 + 64]                 # 641 and 655 candidate chunks
+    inp = wl.make_decode_inputs(cfg, "cpu", seq_lens=torch.tensor(seq, dtype=torch.int32))
+    bias = torch.zeros((cfg.B, cfg.Hkv, cfg.C), dtype=torch.float32)
+    for b, n in enumerate(seq):
+        ncand = (n - 1) // cfg.S
+        bias[b, :, ncand - 1] = 50.0
+        bias[b, :, ncand - 17] = 50.0
+    out, lse, sel = run_decode(cfg, inp, "fast", bias=bias)
+    got = sel.cpu().numpy()
+    for b, n in enumerate(seq):
+        ncand = (n - 1) // cfg.S
+        assert (got[b] == ncand - 1).any(axis=-1).all() and (got[b] == ncand - 17).any(axis=-1).all()
+        assert (got[b] < ncand).all()
     check_decode(cfg, inp, out, lse, sel, bias=bias)
 
 
