@@ -553,6 +553,13 @@ def main():
         for _ in range(2):
             hils.hils_landmark_summary(lq, w.inp["k"], cfg.S)
         torch.cuda.synchronize()
+        ov_calls = 0
+        if not w.decode:
+            # the chunk-overlap statistic of the selection just written (two calls)
+            for _ in range(2):
+                hils.hils_chunk_overlap(w.sel, 16, cfg.C)
+            torch.cuda.synchronize()
+            ov_calls = 2
         bwd_calls = 0
         if not w.decode and cfg.dtype == "bf16":
             # the backward pass over the same tensors (two calls)
@@ -562,7 +569,8 @@ def main():
             torch.cuda.synchronize()
             bwd_calls = 2
         print(json.dumps({"profile_run": cfg.name, "B": cfg.B, "calls": args.warmup + args.steps,
-                          "kernels_per_call": kpc, "landmark_summary_calls": 2, "backward_calls": bwd_calls}))
+                          "kernels_per_call": kpc, "landmark_summary_calls": 2, "chunk_overlap_calls": ov_calls,
+                          "backward_calls": bwd_calls}))
         return
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
