@@ -84,6 +84,15 @@ def test_tensor_core_backward_matches_oracle(name):
     compare(grads, ref, cfg.dtype)
 
 
+def test_auto_dispatch_falls_back_to_the_generic_kernel_for_per_head_landmarks():
+    """One landmark per query head (App. C) is outside the tensor-core backward: `auto` must take the generic
+    kernel and still match the oracle (bf16)."""
+    cfg = wl.CONFIGS[1].scaled(B=1, Hq=8, Hkv=2, L=448, K=4, seed=211)
+    grads, ref = run_case(cfg, 8, 1, True, impl="auto")
+    assert hils.last_launch_count() == 1
+    compare(grads, ref, cfg.dtype)
+
+
 def test_fast_path_refuses_shapes_it_does_not_take():
     cfg = wl.CONFIGS[0].scaled(L=128, seed=209)   # fp32
     inp = {n: t.to(DEV) for n, t in wl.make_prefill_inputs(cfg, "cpu").items()}
