@@ -516,12 +516,12 @@ int launch_prefill_backward_fast(const Shape& s, const BackwardTensors& t, cudaS
     if (!make_bf16_2d_map(&map_k, t.k, kv_rows, kD, 64, kS) || !make_bf16_2d_map(&map_v, t.v, kv_rows, kD, 64, kS))
         return HILS_ERR_CUDA;
     const size_t smem = 2 * kKBytes + 4 * kQBytes + 2 * kDsBytes + sizeof(BfSmem) + 1024;
-    static bool attr_done = false;
-    if (!attr_done) {
+    static PerDeviceOnce attr_once;
+    if (attr_once.pending()) {
         if (cudaFuncSetAttribute(prefill_backward_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(smem)) != cudaSuccess)
             return HILS_ERR_CUDA;
-        attr_done = true;
+        attr_once.done();
     }
     BfArgs a;
     a.s = s;

@@ -881,14 +881,14 @@ int launch_decode_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
         return HILS_ERR_CUDA;
 
     const size_t attend_smem = kStages * kStageBytes + sizeof(AttendSmem) + 1024;
-    static bool attr_done = false;
-    if (!attr_done) {
+    static PerDeviceOnce attr_once;
+    if (attr_once.pending()) {
         if (cudaFuncSetAttribute(decode_attend_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(attend_smem)) != cudaSuccess ||
             cudaFuncSetAttribute(decode_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(sizeof(SelWarp) * 16)) != cudaSuccess)
             return HILS_ERR_CUDA;
-        attr_done = true;
+        attr_once.done();
     }
 
     const int nseg = (s.C + kScoreChunksPerCta - 1) / kScoreChunksPerCta;

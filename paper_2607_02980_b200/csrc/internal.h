@@ -30,6 +30,18 @@ struct Tensors {
     const void* q_route = nullptr;
 };
 
+// Kernel attributes (the opt-in dynamic shared-memory size) belong to a device: a launcher sets them the first time
+// it runs on each device of the process.  pending() is true until done() has been called on the current device.
+struct PerDeviceOnce {
+    bool set[64] = {};
+    static int device() {
+        int d = 0;
+        return (cudaGetDevice(&d) == cudaSuccess && d >= 0 && d < 64) ? d : -1;
+    }
+    bool pending() const { const int d = device(); return d < 0 || !set[d]; }
+    void done() { const int d = device(); if (d >= 0) set[d] = true; }
+};
+
 // Optional per-kernel timing: when tracing is on (hils_trace_enable), every launcher calls
 // trace_mark(name) after each kernel it enqueues; an event is recorded on the stream so that the
 // time between consecutive marks is that kernel's device time.  Off by default (no events).

@@ -321,12 +321,12 @@ int launch_landmark_summary(int dtype, int B, int Hkv, int Hl, int C, int d, int
         CUtensorMap map_k;
         if (!make_bf16_2d_map(&map_k, k, static_cast<uint64_t>(rows), 128, 64, 64)) return HILS_ERR_CUDA;
         const size_t smem = kTcWarps * kTcTileBytes + kTcWarps * sizeof(TcSmemW) + 1024;
-        static bool attr_done = false;
-        if (!attr_done) {
+        static PerDeviceOnce attr_once;
+        if (attr_once.pending()) {
             if (cudaFuncSetAttribute(landmark_summary_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      static_cast<int>(smem)) != cudaSuccess)
                 return HILS_ERR_CUDA;
-            attr_done = true;
+            attr_once.done();
         }
         const long long blocks = (total + kTcWarps - 1) / kTcWarps;
         if (blocks > 0x7fffffffll) return HILS_ERR_UNSUPPORTED;

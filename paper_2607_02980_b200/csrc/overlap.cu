@@ -147,12 +147,12 @@ int launch_chunk_overlap(int pairs, int R, int K, int C, int M, const int32_t* s
     if (ctas > 0x7fffffffll) return HILS_ERR_UNSUPPORTED;
     const size_t smem = per_warp * wpc;
     if (smem > 48 * 1024) {
-        static bool attr_done = false;
-        if (!attr_done) {
+        static PerDeviceOnce attr_once;
+        if (attr_once.pending()) {
             if (cudaFuncSetAttribute(chunk_overlap_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024) !=
                 cudaSuccess)
                 return HILS_ERR_CUDA;
-            attr_done = true;
+            attr_once.done();
         }
     }
     chunk_overlap_kernel<<<static_cast<unsigned>(ctas), wpc * 32, smem, stream>>>(a);

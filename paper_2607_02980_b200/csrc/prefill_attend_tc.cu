@@ -519,12 +519,12 @@ int launch_prefill_attend_tc(const Shape& s, const void* q, const void* maps, co
                              int* status, int i0, cudaStream_t stream) {
     const CUtensorMap* m = static_cast<const CUtensorMap*>(maps);
     const size_t smem = 2 * kKBytes + kVBufs * kVBytes + kQSlots * kQBytes + 2 * kPBytes + sizeof(AtcSmem) + 1024;
-    static bool attr_done = false;
-    if (!attr_done) {
+    static PerDeviceOnce attr_once;
+    if (attr_once.pending()) {
         if (cudaFuncSetAttribute(prefill_attend_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(smem)) != cudaSuccess)
             return HILS_ERR_CUDA;
-        attr_done = true;
+        attr_once.done();
     }
     AtcArgs a{s, static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(landmarks), bias, entries,
               static_cast<const int4*>(tiles), n_tiles, lam, status, i0};

@@ -663,13 +663,13 @@ int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
         return HILS_ERR_CUDA;
 
     const size_t sel_smem = kSelStages * kSelStageBytes + 64 + sizeof(unsigned long long) * 64 * (s.K + 1) + 1024;
-    static bool attr_done = false;
-    if (!attr_done) {
+    static PerDeviceOnce attr_once;
+    if (attr_once.pending()) {
         const size_t sel_max = kSelStages * kSelStageBytes + 64 + sizeof(unsigned long long) * 64 * 65 + 1024;
         if (cudaFuncSetAttribute(prefill_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(sel_max)) != cudaSuccess)
             return HILS_ERR_CUDA;
-        attr_done = true;
+        attr_once.done();
     }
 
     int launches = 0;

@@ -370,8 +370,8 @@ int launch_prefill_select_tc(const Shape& s, const void* q, const void* landmark
         return HILS_ERR_CUDA;
     const size_t smem = kQBytes + kLmStages * kLmStageBytes + sizeof(unsigned long long) * 2 * kMaxK * kTileTok +
                         sizeof(TcSmem) + 1024;
-    static bool attr_done = false;
-    if (!attr_done) {
+    static PerDeviceOnce attr_once;
+    if (attr_once.pending()) {
         if (cudaFuncSetAttribute(prefill_select_tc_kernel<16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(smem)) != cudaSuccess ||
             cudaFuncSetAttribute(prefill_select_tc_kernel<32, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -381,7 +381,7 @@ int launch_prefill_select_tc(const Shape& s, const void* q, const void* landmark
             cudaFuncSetAttribute(prefill_select_tc_kernel<32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(smem)) != cudaSuccess)
             return HILS_ERR_CUDA;
-        attr_done = true;
+        attr_once.done();
     }
     TcArgs a{s, bias, sel, status, (cnt && qb % kTileTok == 0) ? cnt : nullptr, qb, nc};
     const int tiles = (s.R + kTileTok - 1) / kTileTok;
