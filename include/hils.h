@@ -17,6 +17,13 @@
  *              softmax({s^h_c : c selected} U {log Z_swa}) -- per head.
  *              lse = log( sum_c exp(s^h_c) + Z_swa ).
  *
+ * Around the operator (each documented at its declaration): the chunk summaries that produce
+ * landmarks / bias (Proposition 3.1, hils_landmark_summary); the operator on a slice of a sequence, on paged
+ * caches, with a separate routing query (Eq. Q-Cal) and for several new tokens per sequence
+ * (hils_prefill_at, hils_decode_paged, hils_*_routed, hils_decode_multi); the overlap statistic of adjacent
+ * queries (Sec. "Chunk Overlap", hils_chunk_overlap); the backward pass through `out`
+ * (hils_prefill_backward); host-buffer variants and an allocation-free decode.
+ *
  * Conventions
  *   - Every pointer is a DEVICE pointer owned by the caller unless the entry point says HOST.
  *   - The library never allocates, frees or synchronises (except where stated); all work is
