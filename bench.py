@@ -435,7 +435,12 @@ def bench_chunk_overlap(hils, w, peaks, M=16, iters=10):
     o = ov.cpu().numpy()
     full = st[..., 3] == 1
     nbytes = sel.numel() * 4 + stats.numel() * 4 + ov.numel() * 4
+    # the paper's left panel of Fig. chunk_overlap: what the final M queries load of the chunks they can see
+    visible = max(0, (cfg.L - 1 - w.window + 1) // cfg.S) if w.window > 1 else (cfg.L - 1) // cfg.S
+    last_union = float(st[..., -1, 1].mean())
     return {"block_queries": M, "top_k": cfg.K, "blocks": int(full.size), "full_blocks": int(full.sum()),
+            "final_block_union_chunks": last_union, "final_block_visible_chunks": visible,
+            "final_block_loaded_fraction": last_union / max(1, visible),
             "mean_overlap": float(o[full].mean()), "mean_union_chunks": float(st[..., 1][full].mean()),
             "reused_from_previous_block": float(st[..., 2][..., 1:].sum() / max(1, st[..., 1][..., 1:].sum())),
             "ms": ms, "algorithmic_bytes": nbytes, "GBps": nbytes / (ms * 1e-3) / 1e9,

@@ -267,3 +267,9 @@ def chunk_overlap(sel_idx, M: int):
     shape = lead + (nblk,)
     return {"total": total.reshape(shape), "union": union.reshape(shape), "reused": reused.reshape(shape),
             "overlap": overlap.reshape(shape)}
+
+
+def loaded_fraction(union_size, visible_chunks):
+    """Share of the visible historical chunks that a block of adjacent queries loads (Sec. "Chunk Overlap", the
+    percentages of Fig. chunk_overlap, left): union size / visible pool."""
+    return np.asarray(union_size, dtype=np.float64) / np.asarray(visible_chunks, dtype=np.float64)

@@ -74,3 +74,39 @@ def test_single_query_blocks_have_no_ratio():
     sel = np.arange(12).reshape(3, 4)
     r = oracle.chunk_overlap(sel, 1)
     assert r["union"].tolist() == [4, 4, 4] and np.isnan(r["overlap"]).all()
+
+
+def test_loaded_fraction_and_overlap_against_the_numbers_the_paper_prints():
+    """Fig. chunk_overlap (left) as described in the text: pool 57 -> union 43.6 is 76.4 %, pool 1032 -> union 102.1
+    is 9.9 %; and by Eq. Overlap a union of 102.1 of M K = 512 slots is an overlap of (512 - 102.1) / 480 = 0.854,
+    inside the 80-93 % the section reports."""
+    import os
+    rows, consts = [], {}
+    with open(os.path.join(os.path.dirname(__file__), "golden", "chunk_overlap_loaded_fraction.txt")) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            kv = dict(t.split("=") for t in line.split())
+            if "pool" in kv:
+                rows.append(kv)
+            else:
+                consts.update(kv)
+    assert len(rows) == 2 and consts == {"M": "16", "K": "32"}
+    for r in rows:
+        frac = oracle.loaded_fraction(float(r["union"]), float(r["pool"]))
+        assert abs(100.0 * frac - float(r["fraction_pct"])) <= 0.15          # printed to one decimal
+    # a block whose 16 queries (K = 32) cover exactly 102 distinct chunks: the oracle's Eq. Overlap
+    M, K = int(consts["M"]), int(consts["K"])
+    sel = np.zeros((M, K), np.int64)
+    ids = iter(range(32, 102))
+    for m in range(M):
+        sel[m] = np.arange(K)                                    # 32 chunks shared by all
+    for m in range(M):                                           # 70 more distinct chunks spread over the queries
+        for s in range(K - 1, K - 1 - 5, -1):
+            nxt = next(ids, None)
+            if nxt is not None:
+                sel[m, s] = nxt
+    sel.sort(axis=1)
+    r = oracle.chunk_overlap(sel, M)
+    assert r["union"].tolist() == [102] and abs(r["overlap"][0] - (M * K - 102) / ((M - 1) * K)) < 1e-15
+    assert 0.80 <= r["overlap"][0] <= 0.93
