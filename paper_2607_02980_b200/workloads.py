@@ -30,7 +30,10 @@ Value recipe:
                   real model retrieve largely the same chunks (Sec. "Chunk
                   Overlap": up to 80-93 % shared).  One base query per block
                   of M adjacent tokens and head, q_i = base + noise * N(0,1);
-                  no needles.  The other tensors are unchanged.
+                  no needles.  The other tensors are unchanged.  With
+                  `overlap_drift=rho` the base queries of consecutive blocks
+                  form an AR(1) sequence (inter-block reuse, 92.8 % in the
+                  paper's measurement).
 
 Every tensor has its own generator seeded with seed*1000 + tensor_id, so a
 tensor does not change when another one is added or resized.
@@ -145,7 +148,7 @@ def _needle_dirs(lm_bh: torch.Tensor, idx: torch.Tensor) -> torch.Tensor:
 
 
 def make_prefill_inputs(cfg: HilsConfig, device="cpu", overlap_block: int = 0,
-                        overlap_noise: float = 0.3) -> Dict[str, torch.Tensor]:
+                        overlap_noise: float = 0.3, overlap_drift: float = 0.0) -> Dict[str, torch.Tensor]:
     assert cfg.mode == "prefill"
     dev = torch.device(device)
     k = _draw_kv(cfg, _gen(cfg.seed, 1, dev), dev)
@@ -165,6 +168,12 @@ def make_prefill_inputs(cfg: HilsConfig, device="cpu", overlap_block: int = 0,
             if overlap_block > 1:
                 nblk = (cfg.L + overlap_block - 1) // overlap_block
                 base = _randn((G, nblk, cfg.d), gb, dev) * mul
+                if overlap_drift > 0.0:
+                    # slowly drifting base queries: base_r = rho * base_{r-1} + sqrt(1 - rho^2) * N(0,1), so that a
+                    # block also shares most of its chunks with the block before it (the paper measures 92.8 %)
+                    rho, fresh = overlap_drift, math.sqrt(1.0 - overlap_drift * overlap_drift)
+                    for r in range(1, nblk):
+                        base[:, r] = rho * base[:, r - 1] + fresh * base[:, r]
                 qg = base.repeat_interleave(overlap_block, dim=1)[:, :cfg.L] + overlap_noise * qg
             elif cfg.n_needles > 0:
                 ok = ci >= cfg.n_needles      # rows with enough past chunks to plant into
