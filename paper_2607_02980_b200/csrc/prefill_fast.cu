@@ -503,22 +503,34 @@ const bool g_force_mma_select = [] {
     const char* e = getenv("HILS_FORCE_MMA_SELECT");
     return e != nullptr && e[0] == '1';
 }();
-// HILS_PREFILL_QB overrides the query-block length (multiple of 64, for tuning runs).
-const int kQB = [] {
+// HILS_PREFILL_QB overrides the query-block length (multiple of 64, for tuning runs); 0 = choose per call.
+const int kQBEnv = [] {
     const char* e = getenv("HILS_PREFILL_QB");
     const int v = e ? atoi(e) : 0;
-    return (v >= 64 && v % 64 == 0 && v <= (1 << 20)) ? v : kQBDefault;
+    return (v >= 64 && v % 64 == 0 && v <= (1 << 20)) ? v : 0;
 }();
+// Tokens per query block.  A block's tokens that selected a chunk form that chunk's list; lists of about 500 entries
+// (16 tiles) amortise the chunk's K/V load and the ragged last tile, and a list holds about block * K / (visible
+// chunks ~ L / 2S) entries: block ~ 4 L / K, between 4096 (the gathered Q rows of a block stay in L2) and 8192
+// (16384 gains another 0.7 % on 128K tokens for twice the partial-output buffer).
+int pick_query_block(const Shape& s) {
+    if (kQBEnv) return kQBEnv;
+    const long long want = 4ll * (static_cast<long long>(s.pos0) + s.R) / (s.K > 0 ? s.K : 1);
+    int qb = kQBDefault;
+    while (qb < want && qb < 2 * kQBDefault) qb *= 2;
+    return qb;
+}
 struct Plan {
     int qb, nc, n_blocks, max_tiles, max_blk_tiles;
     size_t off_cnt, off_cursor, off_ntiles, zero_bytes, off_seg, off_off, off_entries, off_epos, off_tiles, off_obuf, off_lam,
         total;
 };
 
-Plan make_plan(const Shape& s) {
+Plan make_plan(const Shape& s, int qb_fixed = 0) {
     Plan p;
     const size_t pairs = static_cast<size_t>(s.B) * s.Hkv;
-    const size_t blk = static_cast<size_t>(s.R < kQB ? (s.R + kS - 1) / kS * kS : kQB);
+    const int QB = qb_fixed > 0 ? qb_fixed : pick_query_block(s);
+    const size_t blk = static_cast<size_t>(s.R < QB ? (s.R + kS - 1) / kS * kS : QB);
     p.qb = static_cast<int>(blk);
     const size_t nchunks = (static_cast<size_t>(s.pos0) + s.R + kS - 1) / kS;     // chunks the queries can touch
     const size_t nc = static_cast<size_t>(s.C) > nchunks ? static_cast<size_t>(s.C) : nchunks;
@@ -574,11 +586,12 @@ size_t prefill_fast_scratch_bytes(const Shape& s) { return make_plan(s).total; }
 
 // The inverse index on its own (the backward pass walks the same chunk-major tiles): per-(query block, pair, chunk)
 // entry lists and the tile table, built from a selection that is already in memory.
-size_t inverse_index_bytes(const Shape& s) { return make_plan(s).off_obuf; }
+// (query blocks of kQBDefault tokens: the fp32 dq rows a block accumulates into have to stay in L2)
+size_t inverse_index_bytes(const Shape& s) { return make_plan(s, kQBEnv ? kQBEnv : kQBDefault).off_obuf; }
 
 int build_inverse_index(const Shape& s, const int32_t* sel, void* scratch, size_t bytes, InverseIndex* ix,
                         cudaStream_t stream) {
-    const Plan p = make_plan(s);
+    const Plan p = make_plan(s, kQBEnv ? kQBEnv : kQBDefault);
     if (bytes < p.off_obuf) return HILS_ERR_WORKSPACE;
     const int pairs = s.B * s.Hkv;
     char* sc = static_cast<char*>(scratch);
