@@ -71,10 +71,12 @@ int launch_prefill_select_tc(const Shape& s, const void* q, const void* landmark
 // tcgen05 chunk-major attention over the tile table built by the invert kernels (32-token tiles).
 int attend_tc_tile_tokens();
 // maps: CUtensorMap[3] = K, V ([pairs*T, 128] bf16, boxes of 64 x 64) and the partial-output buffer
-// ([entries of a block * 4 heads, 128] bf16, boxes of 64 x 32), all with the 128-byte swizzle.
+// ([entries of a block * 4 heads, 128] bf16, boxes of 64 x 32), all with the 128-byte swizzle.  whole = 1: the
+// partial-output buffer and lam hold every query block of the call (rows indexed by global entry), else one block;
+// n_run consecutive query blocks (n_tiles[0 .. n_run]) of qb tokens are walked by one launch.
 int launch_prefill_attend_tc(const Shape& s, const void* q, const void* maps, const void* landmarks,
                              const float* bias, const int* entries, const void* tiles, const int* n_tiles, float* lam,
-                             int* status, int i0, cudaStream_t stream);
+                             int* status, int i0, int whole, int n_run, int qb, cudaStream_t stream);
 
 // Chunk summaries (Proposition 3.1): landmarks / bias of the chunks [c0, c0 + cn) from their learnable queries.
 bool landmark_summary_supports(int d, int S);

@@ -73,6 +73,9 @@ struct AtcArgs {
     float* lam;
     int* status;
     int i0;
+    int whole;        // 1: the output buffers cover every query block of the call (rows indexed by global entry)
+    int n_run;        // query blocks this launch walks one after the other (> 1 only with whole = 1)
+    int qb;           // tokens per query block
 };
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
@@ -136,13 +139,16 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
     // previous kernel of the stream (the fusion of the previous query block, which still reads the partial outputs
     // this kernel overwrites, or the inverse-index kernels).  From here on their results are needed.
     pdl_wait();
-    // a.n_tiles points at {first tile of this query block, first tile of the next one}
-    const int t_begin = a.n_tiles[0], n_tiles = a.n_tiles[1] - t_begin;
-    const long long lo = t_begin + static_cast<long long>(blockIdx.x) * n_tiles / gridDim.x;
-    const long long hi = t_begin + static_cast<long long>(blockIdx.x + 1) * n_tiles / gridDim.x;
-
     // running counters (identical in every role): tiles and chunk loads processed so far by this CTA
     uint32_t tcount = 0, ccount = 0;
+
+    // a.n_tiles[blk], a.n_tiles[blk + 1]: first tile of query block blk and of the next one.  A launch that walks
+    // several blocks takes them in order, so that the CTAs stay on the same block (its gathered Q rows stay in L2).
+    for (int blk = 0; blk < a.n_run; ++blk) {
+    const int t_begin = a.n_tiles[blk], n_tiles = a.n_tiles[blk + 1] - t_begin;
+    const int i0 = a.i0 + blk * a.qb;
+    const long long lo = t_begin + static_cast<long long>(blockIdx.x) * n_tiles / gridDim.x;
+    const long long hi = t_begin + static_cast<long long>(blockIdx.x + 1) * n_tiles / gridDim.x;
 
     for (long long b0 = lo; b0 < hi; b0 += kBatch) {
         const int nb = static_cast<int>(min(static_cast<long long>(kBatch), hi - b0));
@@ -277,9 +283,9 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                     // thread ptid owns row ptid for the address table
                     const int tk = ptid >> 2, hd = ptid & 3;
                     const int bb = pair / s.Hkv, gk = pair % s.Hkv;
-                    sm.rowptr[rb][ptid] = a.q + ((static_cast<long long>(bb) * s.Hq + gk * kG + hd) * s.R + a.i0 + (e >> 8)) * kD;
+                    sm.rowptr[rb][ptid] = a.q + ((static_cast<long long>(bb) * s.Hq + gk * kG + hd) * s.R + i0 + (e >> 8)) * kD;
                     if (hd == 0) sm.tile_ent[ms][tk] = e;
-                    if (ptid == 0) { sm.tile_meta[ms][0] = pair; sm.tile_meta[ms][1] = c; sm.tile_meta[ms][2] = ntok; sm.tile_meta[ms][3] = rec.z - t_begin * kTok; }
+                    if (ptid == 0) { sm.tile_meta[ms][0] = pair; sm.tile_meta[ms][1] = c; sm.tile_meta[ms][2] = ntok; sm.tile_meta[ms][3] = rec.z - (a.whole ? 0 : t_begin * kTok); }
                     producer_barrier();
                     const uint32_t qaddr = smem_u32(qbuf + qs * kQBytes);
                     const int p16 = lane & 15;
@@ -411,7 +417,7 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                 const int e = sm.tile_ent[ms][tk];
                 const int il = e >> 8, slot = e & 255;
                 const bool local = slot >= s.K;                            // a chunk of the local window: mass = its exact log-sum-exp
-                const int lim = local ? s.pos0 + a.i0 + il - c * kS : kS - 1;   // last visible key of the chunk
+                const int lim = local ? s.pos0 + i0 + il - c * kS : kS - 1;   // last visible key of the chunk
                 float zi;
                 {
                     float v[64];
@@ -503,6 +509,8 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
         __syncthreads();
         if (sm.abort_flag) break;
     }
+    if (sm.abort_flag) break;
+    }
 
     tc_fence_before_sync();
     __syncthreads();
@@ -516,7 +524,7 @@ int attend_tc_tile_tokens() { return kTok; }
 
 int launch_prefill_attend_tc(const Shape& s, const void* q, const void* maps, const void* landmarks,
                              const float* bias, const int* entries, const void* tiles, const int* n_tiles, float* lam,
-                             int* status, int i0, cudaStream_t stream) {
+                             int* status, int i0, int whole, int n_run, int qb, cudaStream_t stream) {
     const CUtensorMap* m = static_cast<const CUtensorMap*>(maps);
     const size_t smem = 2 * kKBytes + kVBufs * kVBytes + kQSlots * kQBytes + 2 * kPBytes + sizeof(AtcSmem) + 1024;
     static PerDeviceOnce attr_once;
@@ -527,7 +535,7 @@ int launch_prefill_attend_tc(const Shape& s, const void* q, const void* maps, co
         attr_once.done();
     }
     AtcArgs a{s, static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(landmarks), bias, entries,
-              static_cast<const int4*>(tiles), n_tiles, lam, status, i0};
+              static_cast<const int4*>(tiles), n_tiles, lam, status, i0, whole, n_run, qb};
     if (launch_pdl(prefill_attend_tc_kernel, dim3(148), dim3(kThreads), smem, stream, m[0], m[1], m[2], a) != cudaSuccess)
         return HILS_ERR_CUDA;
     if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;

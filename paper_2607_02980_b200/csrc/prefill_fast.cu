@@ -60,6 +60,7 @@ struct PArgs {
     int nc;                 // chunk slots per pair in cnt/off/...: max(C, ceil(L / S))
     int tile_tok;           // entries per attend tile
     int max_tiles;
+    int whole;              // obuf / lam cover all query blocks (indexed by global entry): one fuse launch per call
 };
 
 // ------------------------------------------------------------------------------------------ select
@@ -373,7 +374,7 @@ __global__ void __launch_bounds__(128) prefill_route_scores_kernel(const PArgs a
     const int pair = rec.x, c = rec.y, first = rec.z, ntok = rec.w;
     if (c >= s.C) return;
     const int b = pair / s.Hkv, gk = pair % s.Hkv, per = s.Hl / s.Hkv;
-    const int e0 = t_begin * a.tile_tok;
+    const int e0 = a.whole ? 0 : t_begin * a.tile_tok;
     for (int ei = warp; ei < ntok; ei += 4) {
         const int e = a.entries[first + ei];
         const int tok = a.i0 + (e >> 8), slot = e & 255;
@@ -422,7 +423,7 @@ __global__ void __launch_bounds__(kFuseWarps * 32) prefill_fuse_kernel(const PAr
     const int nsel = min(K, lc);
     const int nl = pos / kS - lc + 1;
     const int nrows = nsel + nl;
-    const int e0 = a.blk_toff[a.blk] * a.tile_tok;   // first entry of this query block
+    const int e0 = a.whole ? 0 : a.blk_toff[a.blk] * a.tile_tok;   // first entry of this query block
     const int* ep = a.epos + (static_cast<long long>(pair) * s.R + tok) * K1;
     const float4* lam4 = reinterpret_cast<const float4*>(a.lam);
     float (*wv)[kFuseRows] = wsm[wib];
@@ -521,9 +522,9 @@ int pick_query_block(const Shape& s) {
     return qb;
 }
 struct Plan {
-    int qb, nc, n_blocks, max_tiles, max_blk_tiles;
+    int qb, nc, n_blocks, max_tiles, max_blk_tiles, whole;
     size_t off_cnt, off_cursor, off_ntiles, zero_bytes, off_seg, off_off, off_entries, off_epos, off_tiles, off_obuf, off_lam,
-        total;
+        total, obuf_tiles;
 };
 
 Plan make_plan(const Shape& s, int qb_fixed = 0) {
@@ -563,8 +564,13 @@ Plan make_plan(const Shape& s, int qb_fixed = 0) {
     p.off_entries = take(sizeof(int) * all_tiles * tt);
     p.off_epos = take(sizeof(int) * pairs * s.R * (s.K + max_local_slots(s.W)));
     p.off_tiles = take(sizeof(int4) * all_tiles);
-    p.off_obuf = take(sizeof(__nv_bfloat16) * max_blk * tt * kG * kD);
-    p.off_lam = take(sizeof(float) * max_blk * tt * kG);
+    // Partial outputs of all query blocks at once while that stays under 4 GB: the fusion then runs as one launch
+    // over the whole call instead of one per block (each launch pays its ramp and its last wave).
+    p.whole = (nblocks > 1 && all_tiles * tt * kG * kD * sizeof(__nv_bfloat16) <= (4ull << 30)) ? 1 : 0;
+    const size_t obuf_tiles = p.whole ? all_tiles : max_blk;
+    p.obuf_tiles = obuf_tiles;
+    p.off_obuf = take(sizeof(__nv_bfloat16) * obuf_tiles * tt * kG * kD);
+    p.off_lam = take(sizeof(float) * obuf_tiles * tt * kG);
     p.total = off;
     return p;
 }
@@ -666,13 +672,14 @@ int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
     a.tile_tok = attend_tc_tile_tokens();
     a.i0 = 0;
     a.i1 = 0;
+    a.whole = p.whole;
 
     // K, V: boxes of 64 dims x 64 keys; partial outputs: boxes of 64 dims x 32 rows (one epilogue warp's rows)
     CUtensorMap map_k, map_v, map_lm, map_o;
     const uint64_t kv_rows = static_cast<uint64_t>(pairs) * s.T;
     if (!make_bf16_2d_map(&map_k, t.k, kv_rows, kD, 64, kS) || !make_bf16_2d_map(&map_v, t.v, kv_rows, kD, 64, kS) ||
         !make_bf16_2d_map(&map_lm, t.landmarks, static_cast<uint64_t>(pairs) * s.C, kD, 64, kS) ||
-        !make_bf16_2d_map(&map_o, a.obuf, static_cast<uint64_t>(p.max_blk_tiles) * a.tile_tok * kG, kD, 64, 32))
+        !make_bf16_2d_map(&map_o, a.obuf, static_cast<uint64_t>(p.obuf_tiles) * a.tile_tok * kG, kD, 64, 32))
         return HILS_ERR_CUDA;
 
     const size_t sel_smem = kSelStages * kSelStageBytes + 64 + sizeof(unsigned long long) * 64 * (s.K + 1) + 1024;
@@ -726,14 +733,16 @@ int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
         a.i0 = i0;
         a.i1 = s.R < i0 + a.qb ? s.R : i0 + a.qb;
         a.blk = blk;
-        const int nblk = a.i1 - a.i0;
-        {
+        if (!a.whole || blk == 0) {
+            // one launch per query block, or a single launch that walks all of them (whole-call output buffers)
             const CUtensorMap maps[3] = {map_k, map_v, map_o};
             const int rc = launch_prefill_attend_tc(s, t.q, maps, t.landmarks, t.bias, a.entries, a.tiles,
-                                                    a.blk_toff + blk, a.lam, t.status, a.i0, stream);
+                                                    a.blk_toff + blk, a.lam, t.status, a.i0, a.whole,
+                                                    a.whole ? p.n_blocks : 1, a.qb, stream);
             if (rc < 0) return rc;
+            trace_mark("prefill_attend", stream);
+            ++launches;
         }
-        trace_mark("prefill_attend", stream);
         if (t.q_route) {
             const int ntl = (p.max_blk_tiles);
             if (launch_pdl(prefill_route_scores_kernel, dim3(static_cast<unsigned>(ntl)), dim3(128), 0, stream, a) != cudaSuccess)
@@ -741,12 +750,17 @@ int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
             trace_mark("prefill_route_scores", stream);
             ++launches;
         }
-        const long long fuse_warps = static_cast<long long>(pairs) * nblk;
+        if (a.whole) {
+            // one fusion launch after the last block's attend, over every token of the call
+            if (a.i1 < s.R) continue;
+            a.i0 = 0;
+        }
+        const long long fuse_warps = static_cast<long long>(pairs) * (a.i1 - a.i0);
         if (launch_pdl(prefill_fuse_kernel, dim3(static_cast<unsigned>((fuse_warps + kFuseWarps - 1) / kFuseWarps)),
                        dim3(kFuseWarps * 32), 0, stream, a) != cudaSuccess)
             return HILS_ERR_CUDA;
         trace_mark("prefill_fuse", stream);
-        launches += 2;
+        ++launches;
     }
     return launches;
 }
