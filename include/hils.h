@@ -88,7 +88,10 @@ typedef struct hils_params {
 
 /* Bytes of device scratch hils_prefill (is_decode = 0) or hils_decode (is_decode = 1) needs for
  * these parameters.  Returns 0 if the parameters are invalid.  The first 256 bytes hold the
- * device status word; the caller must zero them once after allocation. */
+ * device status word; the caller must zero them once after allocation.
+ * Prefill on the tensor-core path keeps per-(token, retrieved chunk) partial outputs in the workspace:
+ * (K + window chunks) * Hq * d * 2 bytes per token, for all tokens of the call while that is at most 4 GiB
+ * (2.3 GB for 16K tokens, 32 heads, K = 16), else for one block of 4096-8192 tokens at a time. */
 size_t hils_workspace_bytes(const hils_params* params, int is_decode);
 
 /* Prefill: Eq. (surrogate top-k) + Eq. (HiLS weights) (GQA form: App. C) for all L positions of
