@@ -12,6 +12,8 @@
 //           d landmark and d bias of the chunk likewise.
 // K and V of the chunk arrive by TMA (128-byte swizzle), Q and dO rows by cp.async into the same swizzled layout,
 // so that every MMA operand is read with ldmatrix.
+#include <stdlib.h>
+
 #include "internal.h"
 #include "tma.cuh"
 
@@ -481,6 +483,401 @@ prefill_backward_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
     asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
 
+struct BtSmem {               // shared state of the tcgen05 variant
+    uint64_t kv_bar, st_bar, dq_bar;
+    uint32_t tmem_base;
+    float lmf[2][kD];         // the landmark of the chunk in work and of the next one
+    float bias_c[2];
+    float dlam[kRows];
+    float row_lse[2][kRows];
+    float row_dsum[2][kRows];
+    int row_orow[2][kRows];
+    int row_limit[2][kRows];
+    int row_local[2][kRows];
+    int abort_flag;
+};
+__device__ __forceinline__ void red_add_v4(float* p, float x, float y, float z, float w) {
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(x), "f"(y), "f"(z), "f"(w) : "memory");
+}
+
+__global__ void __launch_bounds__(kBfThreads, 1)
+prefill_backward_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                            const BfArgs a) {
+    extern __shared__ uint8_t bf_raw[];
+    uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(bf_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* kbuf = base;
+    uint8_t* vbuf = kbuf + kKBytes;
+    uint8_t* qbuf0 = vbuf + kKBytes;             // [2][kQBytes]: the tile in work and the next one
+    uint8_t* dobuf0 = qbuf0 + 2 * kQBytes;       // [2][kQBytes]
+    uint8_t* dsbuf = dobuf0 + 2 * kQBytes;
+    uint8_t* wbuf = dsbuf + kDsBytes;
+    BtSmem& sm = *reinterpret_cast<BtSmem*>(wbuf + kDsBytes);
+
+    const Shape& s = a.s;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t4 = lane & 3;
+    const int t_begin = a.blk_range[0], n_tiles = a.blk_range[1] - t_begin;
+    const long long lo = t_begin + static_cast<long long>(blockIdx.x) * n_tiles / gridDim.x;
+    const long long hi = t_begin + static_cast<long long>(blockIdx.x + 1) * n_tiles / gridDim.x;
+
+    if (tid == 0) {
+        mbar_init(&sm.kv_bar, 1);
+        mbar_init(&sm.st_bar, 1);
+        mbar_init(&sm.dq_bar, 1);
+        mbar_fence_init();
+        sm.abort_flag = 0;
+        tma_prefetch_desc(&map_k);
+        tma_prefetch_desc(&map_v);
+    }
+    if (warp == 0) tmem_alloc(&sm.tmem_base, 512);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = sm.tmem_base;
+    const uint32_t t_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);     // this warp's 32 rows
+    // tensor-memory columns: S = Q K^T at 0..63, T = dO V^T at 64..127, dQ at 128..255
+    uint32_t st_phase = 0, dq_phase = 0;
+    int cpar = 0;                                      // which copy of the landmark / bias belongs to the chunk in work
+
+    const uint32_t k_addr = smem_u32(kbuf), v_addr = smem_u32(vbuf);
+    const uint32_t ds_addr = smem_u32(dsbuf), w_addr = smem_u32(wbuf);
+    uint32_t kv_phase = 0;
+    int cur_pair = -1, cur_c = -1;
+    float dk_acc[4][2][4], dv_acc[4][2][4];
+    float lm_acc = 0.f, bias_acc = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 2; ++j)
+#pragma unroll
+            for (int x = 0; x < 4; ++x) dk_acc[i][j][x] = dv_acc[i][j][x] = 0.f;
+
+    // adds the finished chunk's register accumulators to dk, dv, dlandmarks, dbias and clears them
+    auto flush = [&]() {
+        if (cur_pair < 0) return;
+        const int b = cur_pair / s.Hkv, gk = cur_pair % s.Hkv;
+        const long long kvrow0 = static_cast<long long>(cur_pair) * s.T;
+#pragma unroll
+        for (int mt = 0; mt < 4; ++mt)
+#pragma unroll
+            for (int n2 = 0; n2 < 2; ++n2) {
+                const int dim = warp * 16 + n2 * 8 + 2 * t4;
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    const int key = cur_c * kS + mt * 16 + g + hh * 8;
+                    if (key < s.T) {
+                        red_add_v2(a.dk + (kvrow0 + key) * kD + dim, dk_acc[mt][n2][2 * hh], dk_acc[mt][n2][2 * hh + 1]);
+                        red_add_v2(a.dv + (kvrow0 + key) * kD + dim, dv_acc[mt][n2][2 * hh], dv_acc[mt][n2][2 * hh + 1]);
+                    }
+                    dk_acc[mt][n2][2 * hh] = dk_acc[mt][n2][2 * hh + 1] = 0.f;
+                    dv_acc[mt][n2][2 * hh] = dv_acc[mt][n2][2 * hh + 1] = 0.f;
+                }
+            }
+        lm_acc += __shfl_xor_sync(kFullMask, lm_acc, 16);
+        if (cur_c < s.C) {
+            const long long lrow = (static_cast<long long>(b) * s.Hl + gk) * s.C + cur_c;
+            if (lane < 16) atomicAdd(a.dlm + lrow * kD + warp * 16 + lane, lm_acc);
+            if (warp == 0 && lane == 0 && a.dbias) atomicAdd(a.dbias + lrow, bias_acc / s.scale);
+        }
+        lm_acc = 0.f;
+        bias_acc = 0.f;
+    };
+
+    // Requests the chunk's K and V (TMA, thread 0) and reads its landmark and bias (threads 128..255).  Called when
+    // nobody reads the previous chunk's copies any more.
+    auto issue_chunk = [&](int pair, int c, int cp) {
+        const int b = pair / s.Hkv, gk = pair % s.Hkv;
+        if (tid == kRows) {
+            const int row = pair * s.T + c * kS;
+            mbar_expect_tx(&sm.kv_bar, 2 * kKBytes);
+            tma_load_2d(kbuf, &map_k, &sm.kv_bar, 0, row);
+            tma_load_2d(kbuf + 8192, &map_k, &sm.kv_bar, 64, row);
+            tma_load_2d(vbuf, &map_v, &sm.kv_bar, 0, row);
+            tma_load_2d(vbuf + 8192, &map_v, &sm.kv_bar, 64, row);
+        }
+        if (tid >= kRows) {
+            const int x = tid - kRows;
+            const long long lrow = (static_cast<long long>(b) * s.Hl + gk) * s.C + c;
+            sm.lmf[cp][x] = c < s.C ? __bfloat162float(a.lm[lrow * kD + x]) : 0.f;
+            if (x == 0) sm.bias_c[cp] = (a.bias && c < s.C) ? a.bias[lrow] : 0.f;
+        }
+    };
+    // Starts the gather of a tile's Q and dO rows into buffer `par` (thread -> row tid / 2, 64-dim half tid & 1;
+    // padding rows are zero) and returns what the row table needs; store_row() writes it once the loads are back.
+    struct RowInfo { int orow, limit, local; float lse, dsum; };
+    // entry of this thread's row in a tile (read two tiles ahead of its use, so that no tile waits for it)
+    auto load_entry = [&](const int4 rec) { return (tid >> 3) < rec.w ? a.entries[rec.z + (tid >> 3)] : 0; };
+    auto issue_tile = [&](const int4 rec, int ent, int par) {
+        const int pair = rec.x, c = rec.y, ntok = rec.w;
+        const int b = pair / s.Hkv, gk = pair % s.Hkv;
+        const int row = tid >> 1, half = tid & 1, e = row >> 2, h = row & 3;
+        RowInfo ri{-1, -1, 0, 0.f, 0.f};
+        uint8_t* qb = qbuf0 + par * kQBytes + half * (kRows * 128);
+        uint8_t* db = dobuf0 + par * kQBytes + half * (kRows * 128);
+        if (e < ntok) {
+            const int tok = a.i0 + (ent >> 8), slot = ent & 255;
+            ri.orow = (b * s.Hq + gk * kG + h) * s.R + tok;
+            ri.local = slot >= s.K ? 1 : 0;
+            ri.limit = ri.local ? min(kS - 1, s.pos0 + tok - c * kS) : kS - 1;
+            const __nv_bfloat16* qs = a.q + static_cast<long long>(ri.orow) * kD + half * 64;
+            const __nv_bfloat16* ds = a.dout + static_cast<long long>(ri.orow) * kD + half * 64;
+            const uint32_t qa = smem_u32(qb), da = smem_u32(db);
+#pragma unroll
+            for (int p = 0; p < 8; ++p) {
+                cp_async16(qa + swz128(row, p), qs + p * 8);
+                cp_async16(da + swz128(row, p), ds + p * 8);
+            }
+            if (half == 0) {
+                ri.lse = a.lse[ri.orow];
+                ri.dsum = a.dsum[ri.orow];
+            }
+        } else {
+#pragma unroll
+            for (int p = 0; p < 8; ++p) {
+                *reinterpret_cast<uint4*>(qb + swz128(row, p)) = make_uint4(0u, 0u, 0u, 0u);
+                *reinterpret_cast<uint4*>(db + swz128(row, p)) = make_uint4(0u, 0u, 0u, 0u);
+            }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        return ri;
+    };
+    auto store_row = [&](const RowInfo& ri, int par) {
+        if ((tid & 1) == 0) {
+            const int row = tid >> 1;
+            sm.row_orow[par][row] = ri.orow;
+            sm.row_limit[par][row] = ri.limit;
+            sm.row_local[par][row] = ri.local;
+            sm.row_lse[par][row] = ri.lse;
+            sm.row_dsum[par][row] = ri.dsum;
+        }
+    };
+
+    const int4 no_tile = make_int4(-1, -1, 0, 0);
+    int4 rec = no_tile, nrec = no_tile, n2rec = no_tile;       // this tile, the next one, the one after
+    int nent = 0;                                              // this thread's entry in the next tile
+    bool kv_issued = false;
+    if (lo < hi) {
+        rec = a.tiles[lo];
+        if (lo + 1 < hi) nrec = a.tiles[lo + 1];
+        if (lo + 2 < hi) n2rec = a.tiles[lo + 2];
+        issue_chunk(rec.x, rec.y, 0);
+        kv_issued = true;
+        store_row(issue_tile(rec, load_entry(rec), 0), 0);
+        nent = load_entry(nrec);
+    }
+    for (long long tile = lo; tile < hi; ++tile) {
+        const int par = static_cast<int>(tile - lo) & 1;
+        const int pair = rec.x, c = rec.y;
+        cur_pair = pair;
+        cur_c = c;
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        fence_proxy_async_smem();                   // the gathered rows are read by the tensor cores (async proxy)
+        if (kv_issued) {
+            if (!mbar_wait(&sm.kv_bar, kv_phase)) {
+                sm.abort_flag = 1;
+                if (lane == 0) set_status(a.status, kDevTimeout);
+            }
+            kv_phase ^= 1u;
+            kv_issued = false;
+        }
+        __syncthreads();                        // this tile's Q, dO, row table, K, V, landmark are in shared memory;
+                                                // the previous tile's readers are done with the other buffers
+        if (sm.abort_flag) break;
+        // the next tile's rows start to arrive while this one is computed
+        const bool has_next = tile + 1 < hi;
+        RowInfo nri{-1, -1, 0, 0.f, 0.f};
+        if (has_next) nri = issue_tile(nrec, nent, par ^ 1);
+        // metadata of the tiles after the next: in registers by the time they are needed
+        const int n2ent = load_entry(n2rec);
+        const int4 n3rec = tile + 3 < hi ? a.tiles[tile + 3] : no_tile;
+        const bool next_new = has_next && (nrec.x != pair || nrec.y != c);
+        const uint8_t* qbuf = qbuf0 + par * kQBytes;
+        const uint32_t q_addr = smem_u32(qbuf), do_addr = smem_u32(dobuf0 + par * kQBytes);
+
+        // ------------------------------------------------------------------ S = Q K^T and T = dO V^T on tcgen05
+        const uint32_t ds_a = smem_u32(dsbuf);
+        if (tid == 0) {
+            constexpr uint32_t idesc_st = umma_idesc_bf16(kRows, kS);
+            tc_fence_after_sync();
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks)
+                umma_bf16(tmem_base, umma_desc_k128(q_addr + (ks >> 2) * (kRows * 128) + (ks & 3) * 32),
+                          umma_desc_k128(k_addr + (ks >> 2) * 8192 + (ks & 3) * 32), idesc_st, ks > 0 ? 1u : 0u);
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks)
+                umma_bf16(tmem_base + 64, umma_desc_k128(do_addr + (ks >> 2) * (kRows * 128) + (ks & 3) * 32),
+                          umma_desc_k128(v_addr + (ks >> 2) * 8192 + (ks & 3) * 32), idesc_st, ks > 0 ? 1u : 0u);
+            umma_commit(&sm.st_bar);
+        }
+        // ------------------------------------------------------------------ phase 1: warps 0-3, one row per thread
+        if (warp < 4) {
+            const int row = tid;
+            const int limit = sm.row_limit[par][row];
+            const bool local = sm.row_local[par][row] != 0;
+            const float lse = sm.row_lse[par][row], dsum = sm.row_dsum[par][row];
+            // surrogate score of the row (its own Q row against the landmark) while the MMAs run
+            float lam = 0.f;
+#pragma unroll
+            for (int half = 0; half < 2; ++half)
+#pragma unroll
+                for (int pc = 0; pc < 8; ++pc) {
+                    const uint4 v = *reinterpret_cast<const uint4*>(qbuf + half * (kRows * 128) + swz128(row, pc));
+                    const __nv_bfloat162* pv = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const float2 x = __bfloat1622float2(pv[i]);
+                        lam = fmaf(x.x, sm.lmf[cpar][half * 64 + pc * 8 + 2 * i], lam);
+                        lam = fmaf(x.y, sm.lmf[cpar][half * 64 + pc * 8 + 2 * i + 1], lam);
+                    }
+                }
+            lam = lam * s.scale + sm.bias_c[cpar];
+            if (!mbar_wait(&sm.st_bar, st_phase)) {
+                sm.abort_flag = 1;
+                if (lane == 0) set_status(a.status, kDevTimeout);
+            }
+            tc_fence_after_sync();
+            float sv[64], tv[64];
+            tmem_ld64(t_lane, sv);
+            tmem_ld64(t_lane + 64, tv);
+            float m = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < 64; ++j) m = fmaxf(m, sv[j]);
+            m *= s.scale;
+            float Z = 0.f, gt = 0.f;
+#pragma unroll
+            for (int j = 0; j < 64; ++j) {
+                const float e = __expf(sv[j] * s.scale - m);
+                Z += e;
+                gt = fmaf(e, tv[j], gt);
+            }
+            float shift = lse, sub = dsum, dl = 0.f;
+            if (!local) {
+                const float gc = gt / Z;
+                const float alpha = __expf(lam - lse);
+                shift = m + __logf(Z) - (lam - lse);
+                sub = gc;
+                dl = limit >= 0 ? alpha * (gc - dsum) * s.scale : 0.f;
+            }
+#pragma unroll
+            for (int j = 0; j < 64; ++j) {
+                const float w = j <= limit ? __expf(sv[j] * s.scale - shift) : 0.f;
+                sv[j] = w * (tv[j] - sub) * s.scale;       // d s_j (times scale)
+                tv[j] = w;                                 // w_j
+            }
+#pragma unroll
+            for (int pc = 0; pc < 8; ++pc) {
+                *reinterpret_cast<uint4*>(dsbuf + swz128(row, pc)) =
+                    make_uint4(pack_bf16(sv[8 * pc], sv[8 * pc + 1]), pack_bf16(sv[8 * pc + 2], sv[8 * pc + 3]),
+                               pack_bf16(sv[8 * pc + 4], sv[8 * pc + 5]), pack_bf16(sv[8 * pc + 6], sv[8 * pc + 7]));
+                *reinterpret_cast<uint4*>(wbuf + swz128(row, pc)) =
+                    make_uint4(pack_bf16(tv[8 * pc], tv[8 * pc + 1]), pack_bf16(tv[8 * pc + 2], tv[8 * pc + 3]),
+                               pack_bf16(tv[8 * pc + 4], tv[8 * pc + 5]), pack_bf16(tv[8 * pc + 6], tv[8 * pc + 7]));
+            }
+            sm.dlam[row] = dl;
+            fence_proxy_async_smem();               // d S is an operand of the d Q MMA
+            tc_fence_before_sync();
+        }
+        st_phase ^= 1u;
+        if (has_next) store_row(nri, par ^ 1);
+        __syncthreads();                        // d S, W and d lambda of all 128 rows are in shared memory
+        if (tid == 0) {
+            // d Q = d S K: A = d S as written above (K-major, 64 keys), B = the chunk's K tile read MN-major
+            constexpr uint32_t idesc_dq = umma_idesc_bf16(kRows, kD) | kUmmaBMnMajor;
+            tc_fence_after_sync();
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)
+                umma_bf16(tmem_base + 128, umma_desc_k128(ds_a + ks * 32), umma_desc_mn128(k_addr + ks * 2048, 8192u, 1024u),
+                          idesc_dq, ks > 0 ? 1u : 0u);
+            umma_commit(&sm.dq_bar);
+        }
+
+        // ------------------------------------------------------------------ phase 2: dims 16 warp .. 16 warp + 15
+#pragma unroll 2
+        for (int ks = 0; ks < 8; ++ks) {
+            const int mat = lane >> 3;
+            uint32_t bq[4], bo[4];
+            {
+                const int row = ks * 16 + (mat & 1) * 8 + (lane & 7);
+                const int dim = warp * 16 + (mat >> 1) * 8;
+                const uint32_t off = (dim >> 6) * (kRows * 128) + swz128(row, (dim & 63) >> 3);
+                ldmatrix_x4_trans(q_addr + off, bq[0], bq[1], bq[2], bq[3]);
+                ldmatrix_x4_trans(do_addr + off, bo[0], bo[1], bo[2], bo[3]);
+            }
+#pragma unroll
+            for (int mt = 0; mt < 4; ++mt) {
+                const int row = ks * 16 + (mat >> 1) * 8 + (lane & 7);
+                const uint32_t off = swz128(row, 2 * mt + (mat & 1));
+                uint32_t ad[4], aw[4];
+                ldmatrix_x4_trans(ds_addr + off, ad[0], ad[1], ad[2], ad[3]);
+                ldmatrix_x4_trans(w_addr + off, aw[0], aw[1], aw[2], aw[3]);
+                mma_bf16_16816(dk_acc[mt][0], ad, bq[0], bq[1]);
+                mma_bf16_16816(dk_acc[mt][1], ad, bq[2], bq[3]);
+                mma_bf16_16816(dv_acc[mt][0], aw, bo[0], bo[1]);
+                mma_bf16_16816(dv_acc[mt][1], aw, bo[2], bo[3]);
+            }
+        }
+        {   // d landmark: sum over rows of (scale d lambda_r) q_r, lane -> (dim, half of the rows)
+            const int dim = warp * 16 + (lane & 15), half = lane >> 4;
+            const uint8_t* col = qbuf + (dim >> 6) * (kRows * 128) + (dim & 7) * 2;
+            const int piece = (dim & 63) >> 3;
+            float acc = 0.f;
+#pragma unroll 8
+            for (int r = half * 64; r < half * 64 + 64; ++r) {
+                const float dl = sm.dlam[r];
+                const __nv_bfloat16 x = *reinterpret_cast<const __nv_bfloat16*>(col + swz128(r, piece));
+                acc = fmaf(dl, __bfloat162float(x), acc);
+            }
+            lm_acc += acc;
+            if (warp == 0) {
+                const float v = sm.dlam[lane] + sm.dlam[lane + 32] + sm.dlam[lane + 64] + sm.dlam[lane + 96];
+                bias_acc += warp_sum(v);
+            }
+        }
+        // ------------------------------------------------------------------ d Q read-out: warps 4-7, one row per thread
+        if (warp >= 4) {
+            const int row = (warp - 4) * 32 + lane;
+            if (!mbar_wait(&sm.dq_bar, dq_phase)) {
+                sm.abort_flag = 1;
+                if (lane == 0) set_status(a.status, kDevTimeout);
+            }
+            tc_fence_after_sync();
+            const int orow = sm.row_orow[par][row];
+            const float dl = sm.dlam[row];
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                float o[64];
+                tmem_ld64(t_lane + 128 + half * 64, o);
+                if (orow >= 0) {
+                    float* dst = a.dq + static_cast<long long>(orow) * kD + half * 64;
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float* l = &sm.lmf[cpar][half * 64 + 4 * i];
+                        red_add_v4(dst + 4 * i, fmaf(dl, l[0], o[4 * i]), fmaf(dl, l[1], o[4 * i + 1]),
+                                   fmaf(dl, l[2], o[4 * i + 2]), fmaf(dl, l[3], o[4 * i + 3]));
+                    }
+                }
+            }
+            tc_fence_before_sync();
+            // every MMA that read the chunk's K and V has completed: the next chunk's copies may land
+            if (next_new) issue_chunk(nrec.x, nrec.y, cpar ^ 1);
+        }
+        dq_phase ^= 1u;
+        if (next_new) {
+            kv_issued = true;
+            cpar ^= 1;
+        }
+        if (!has_next || next_new) flush();
+        rec = nrec;
+        nrec = n2rec;
+        nent = n2ent;
+        n2rec = n3rec;
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    if (warp == 0) tmem_dealloc(tmem_base, 512);
+}
+
 }  // namespace
 
 bool prefill_backward_fast_supports(const Shape& s, int dtype) {
@@ -515,10 +912,14 @@ int launch_prefill_backward_fast(const Shape& s, const BackwardTensors& t, cudaS
     const uint64_t kv_rows = static_cast<uint64_t>(s.B) * s.Hkv * s.T;
     if (!make_bf16_2d_map(&map_k, t.k, kv_rows, kD, 64, kS) || !make_bf16_2d_map(&map_v, t.v, kv_rows, kD, 64, kS))
         return HILS_ERR_CUDA;
-    const size_t smem = 2 * kKBytes + 4 * kQBytes + 2 * kDsBytes + sizeof(BfSmem) + 1024;
+    const size_t smem = 2 * kKBytes + 4 * kQBytes + 2 * kDsBytes + sizeof(BtSmem) + 1024;
+    // HILS_BACKWARD_MMA_SYNC=1: the warp-level variant (every product on mma.sync) instead of the tcgen05 one
+    static const bool warp_mma = [] { const char* e = getenv("HILS_BACKWARD_MMA_SYNC"); return e && e[0] == '1'; }();
     static PerDeviceOnce attr_once;
     if (attr_once.pending()) {
         if (cudaFuncSetAttribute(prefill_backward_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(smem)) != cudaSuccess ||
+            cudaFuncSetAttribute(prefill_backward_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(smem)) != cudaSuccess)
             return HILS_ERR_CUDA;
         attr_once.done();
@@ -542,7 +943,8 @@ int launch_prefill_backward_fast(const Shape& s, const BackwardTensors& t, cudaS
     for (int blk = 0; blk < ix.n_blocks; ++blk) {
         a.blk_range = ix.blk_toff + blk;
         a.i0 = blk * ix.qb;
-        prefill_backward_mma_kernel<<<148, kBfThreads, smem, stream>>>(map_k, map_v, a);
+        if (warp_mma) prefill_backward_mma_kernel<<<148, kBfThreads, smem, stream>>>(map_k, map_v, a);
+        else prefill_backward_tc_kernel<<<148, kBfThreads, smem, stream>>>(map_k, map_v, a);
         if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
         trace_mark("backward_attend", stream);
         ++launches;
