@@ -537,6 +537,34 @@ prefill_backward_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __gr
     // tensor-memory columns: S = Q K^T at 0..63, T = dO V^T at 64..127, dQ at 128..255
     uint32_t st_phase = 0, dq_phase = 0;
     int cpar = 0;                                      // which copy of the landmark / bias belongs to the chunk in work
+    bool st_issued = false;                            // S / T MMAs of the tile at the loop top were issued a tile early
+    // read-out of d Q one tile late (warps 4-7), beside the next tile's row statistics (warps 0-3)
+    int ro_orow = -1, ro_cpar = 0;
+    float ro_dl = 0.f;
+    bool ro_pending = false;
+    auto read_out = [&]() {
+        // thread = row (warps 4-7): d Q row from tensor memory + d lambda k', added to dq
+        if (!mbar_wait(&sm.dq_bar, dq_phase ^ 1u)) {
+            sm.abort_flag = 1;
+            if (lane == 0) set_status(a.status, kDevTimeout);
+        }
+        tc_fence_after_sync();
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            float o[64];
+            tmem_ld64(t_lane + 128 + half * 64, o);
+            if (ro_orow >= 0) {
+                float* dst = a.dq + static_cast<long long>(ro_orow) * kD + half * 64;
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const float* l = &sm.lmf[ro_cpar][half * 64 + 4 * i];
+                    red_add_v4(dst + 4 * i, fmaf(ro_dl, l[0], o[4 * i]), fmaf(ro_dl, l[1], o[4 * i + 1]),
+                               fmaf(ro_dl, l[2], o[4 * i + 2]), fmaf(ro_dl, l[3], o[4 * i + 3]));
+                }
+            }
+        }
+        tc_fence_before_sync();
+    };
 
     const uint32_t k_addr = smem_u32(kbuf), v_addr = smem_u32(vbuf);
     const uint32_t ds_addr = smem_u32(dsbuf), w_addr = smem_u32(wbuf);
@@ -695,19 +723,23 @@ prefill_backward_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __gr
 
         // ------------------------------------------------------------------ S = Q K^T and T = dO V^T on tcgen05
         const uint32_t ds_a = smem_u32(dsbuf);
-        if (tid == 0) {
+        auto issue_st = [&](uint32_t qa, uint32_t da) {          // one thread: S = Q K^T, T = dO V^T
             constexpr uint32_t idesc_st = umma_idesc_bf16(kRows, kS);
             tc_fence_after_sync();
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks)
-                umma_bf16(tmem_base, umma_desc_k128(q_addr + (ks >> 2) * (kRows * 128) + (ks & 3) * 32),
+                umma_bf16(tmem_base, umma_desc_k128(qa + (ks >> 2) * (kRows * 128) + (ks & 3) * 32),
                           umma_desc_k128(k_addr + (ks >> 2) * 8192 + (ks & 3) * 32), idesc_st, ks > 0 ? 1u : 0u);
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks)
-                umma_bf16(tmem_base + 64, umma_desc_k128(do_addr + (ks >> 2) * (kRows * 128) + (ks & 3) * 32),
+                umma_bf16(tmem_base + 64, umma_desc_k128(da + (ks >> 2) * (kRows * 128) + (ks & 3) * 32),
                           umma_desc_k128(v_addr + (ks >> 2) * 8192 + (ks & 3) * 32), idesc_st, ks > 0 ? 1u : 0u);
             umma_commit(&sm.st_bar);
-        }
+        };
+        if (tid == 0 && !st_issued) issue_st(q_addr, do_addr);
+        // the previous tile's d Q leaves tensor memory while this tile's statistics are computed
+        if (warp >= 4 && ro_pending) read_out();
+        ro_pending = false;
         // ------------------------------------------------------------------ phase 1: warps 0-3, one row per thread
         if (warp < 4) {
             const int row = tid;
@@ -763,6 +795,10 @@ prefill_backward_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __gr
                 sv[j] = w * (tv[j] - sub) * s.scale;       // d s_j (times scale)
                 tv[j] = w;                                 // w_j
             }
+            if (tile > lo && !mbar_wait(&sm.dq_bar, dq_phase ^ 1u)) {        // the previous d Q MMA still reads d S
+                sm.abort_flag = 1;
+                if (lane == 0) set_status(a.status, kDevTimeout);
+            }
 #pragma unroll
             for (int pc = 0; pc < 8; ++pc) {
                 *reinterpret_cast<uint4*>(dsbuf + swz128(row, pc)) =
@@ -778,7 +814,18 @@ prefill_backward_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __gr
         }
         st_phase ^= 1u;
         if (has_next) store_row(nri, par ^ 1);
+        if (has_next && !next_new) {
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            fence_proxy_async_smem();
+        }
         __syncthreads();                        // d S, W and d lambda of all 128 rows are in shared memory
+        if (warp >= 4) {                        // what the deferred read-out of this tile needs
+            const int row = (warp - 4) * 32 + lane;
+            ro_orow = sm.row_orow[par][row];
+            ro_dl = sm.dlam[row];
+            ro_cpar = cpar;
+        }
+        ro_pending = true;
         if (tid == 0) {
             // d Q = d S K: A = d S as written above (K-major, 64 keys), B = the chunk's K tile read MN-major
             constexpr uint32_t idesc_dq = umma_idesc_bf16(kRows, kD) | kUmmaBMnMajor;
@@ -788,7 +835,12 @@ prefill_backward_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __gr
                 umma_bf16(tmem_base + 128, umma_desc_k128(ds_a + ks * 32), umma_desc_mn128(k_addr + ks * 2048, 8192u, 1024u),
                           idesc_dq, ks > 0 ? 1u : 0u);
             umma_commit(&sm.dq_bar);
+            // same chunk next: its S and T can start now (their operands are in place, S / T of this tile were read)
+            if (has_next && !next_new)
+                issue_st(smem_u32(qbuf0 + (par ^ 1) * kQBytes), smem_u32(dobuf0 + (par ^ 1) * kQBytes));
         }
+        st_issued = has_next && !next_new;
+        dq_phase ^= 1u;
 
         // ------------------------------------------------------------------ phase 2: dims 16 warp .. 16 warp + 15
 #pragma unroll 2
@@ -832,35 +884,14 @@ prefill_backward_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __gr
                 bias_acc += warp_sum(v);
             }
         }
-        // ------------------------------------------------------------------ d Q read-out: warps 4-7, one row per thread
-        if (warp >= 4) {
-            const int row = (warp - 4) * 32 + lane;
-            if (!mbar_wait(&sm.dq_bar, dq_phase)) {
+        // the next chunk's K, V and landmark may land once every MMA on this chunk has completed: its d Q is the last
+        if (next_new && warp >= 4) {
+            if (!mbar_wait(&sm.dq_bar, dq_phase ^ 1u)) {
                 sm.abort_flag = 1;
                 if (lane == 0) set_status(a.status, kDevTimeout);
             }
-            tc_fence_after_sync();
-            const int orow = sm.row_orow[par][row];
-            const float dl = sm.dlam[row];
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                float o[64];
-                tmem_ld64(t_lane + 128 + half * 64, o);
-                if (orow >= 0) {
-                    float* dst = a.dq + static_cast<long long>(orow) * kD + half * 64;
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const float* l = &sm.lmf[cpar][half * 64 + 4 * i];
-                        red_add_v4(dst + 4 * i, fmaf(dl, l[0], o[4 * i]), fmaf(dl, l[1], o[4 * i + 1]),
-                                   fmaf(dl, l[2], o[4 * i + 2]), fmaf(dl, l[3], o[4 * i + 3]));
-                    }
-                }
-            }
-            tc_fence_before_sync();
-            // every MMA that read the chunk's K and V has completed: the next chunk's copies may land
-            if (next_new) issue_chunk(nrec.x, nrec.y, cpar ^ 1);
+            issue_chunk(nrec.x, nrec.y, cpar ^ 1);
         }
-        dq_phase ^= 1u;
         if (next_new) {
             kv_issued = true;
             cpar ^= 1;
@@ -872,6 +903,7 @@ prefill_backward_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __gr
         n2rec = n3rec;
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
+    if (warp >= 4 && ro_pending && !sm.abort_flag) read_out();
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
