@@ -484,7 +484,7 @@ prefill_backward_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
 }
 
 struct BtSmem {               // shared state of the tcgen05 variant
-    uint64_t kv_bar, st_bar, dq_bar;
+    uint64_t kv_bar, st_bar, dq_bar, p2_bar;
     uint32_t tmem_base;
     float lmf[2][kD];         // the landmark of the chunk in work and of the next one
     float bias_c[2];
@@ -496,6 +496,10 @@ struct BtSmem {               // shared state of the tcgen05 variant
     int row_local[2][kRows];
     int abort_flag;
 };
+constexpr uint32_t kUmmaAMnMajor = 1u << 15;     // instruction-descriptor bit: A operand is MN-major
+__device__ __forceinline__ void red_add_f32(float* p, float x) {
+    asm volatile("red.global.add.f32 [%0], %1;" ::"l"(p), "f"(x) : "memory");
+}
 __device__ __forceinline__ void red_add_v4(float* p, float x, float y, float z, float w) {
     asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(x), "f"(y), "f"(z), "f"(w) : "memory");
 }
@@ -523,6 +527,7 @@ prefill_backward_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __gr
         mbar_init(&sm.kv_bar, 1);
         mbar_init(&sm.st_bar, 1);
         mbar_init(&sm.dq_bar, 1);
+        mbar_init(&sm.p2_bar, 1);
         mbar_fence_init();
         sm.abort_flag = 0;
         tma_prefetch_desc(&map_k);
@@ -534,8 +539,10 @@ prefill_backward_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __gr
     tc_fence_after_sync();
     const uint32_t tmem_base = sm.tmem_base;
     const uint32_t t_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);     // this warp's 32 rows
-    // tensor-memory columns: S = Q K^T at 0..63, T = dO V^T at 64..127, dQ at 128..255
-    uint32_t st_phase = 0, dq_phase = 0;
+    // tensor-memory columns: S = Q K^T at 0..63, T = dO V^T at 64..127, dQ at 128..255,
+    // dK^T (dims x keys) at 256..319, dV^T at 320..383
+    uint32_t st_phase = 0, dq_phase = 0, p2_phase = 0;
+    bool run_acc = false;                              // the chunk's dK^T / dV^T accumulators hold earlier tiles
     int cpar = 0;                                      // which copy of the landmark / bias belongs to the chunk in work
     bool st_issued = false;                            // S / T MMAs of the tile at the loop top were issued a tile early
     // read-out of d Q one tile late (warps 4-7), beside the next tile's row statistics (warps 0-3)
@@ -570,36 +577,32 @@ prefill_backward_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __gr
     const uint32_t ds_addr = smem_u32(dsbuf), w_addr = smem_u32(wbuf);
     uint32_t kv_phase = 0;
     int cur_pair = -1, cur_c = -1;
-    float dk_acc[4][2][4], dv_acc[4][2][4];
     float lm_acc = 0.f, bias_acc = 0.f;
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int j = 0; j < 2; ++j)
-#pragma unroll
-            for (int x = 0; x < 4; ++x) dk_acc[i][j][x] = dv_acc[i][j][x] = 0.f;
 
-    // adds the finished chunk's register accumulators to dk, dv, dlandmarks, dbias and clears them
+    // Adds the finished chunk's accumulators to dk, dv, dlandmarks, dbias.  dK^T and dV^T sit in tensor memory with a
+    // lane per dimension: warps 0-3 read dK^T, warps 4-7 dV^T (64 keys each), a reduction of 32 consecutive
+    // dimensions per key and warp.  Called by every thread after the chunk's last MMAs were issued.
     auto flush = [&]() {
         if (cur_pair < 0) return;
         const int b = cur_pair / s.Hkv, gk = cur_pair % s.Hkv;
         const long long kvrow0 = static_cast<long long>(cur_pair) * s.T;
+        if (!mbar_wait(&sm.p2_bar, p2_phase ^ 1u)) {
+            sm.abort_flag = 1;
+            if (lane == 0) set_status(a.status, kDevTimeout);
+        }
+        tc_fence_after_sync();
+        {
+            float acc[64];
+            tmem_ld64(t_lane + 256 + (warp >= 4 ? 64 : 0), acc);
+            float* dst = (warp >= 4 ? a.dv : a.dk) + kvrow0 * kD + (warp & 3) * 32 + lane;
 #pragma unroll
-        for (int mt = 0; mt < 4; ++mt)
-#pragma unroll
-            for (int n2 = 0; n2 < 2; ++n2) {
-                const int dim = warp * 16 + n2 * 8 + 2 * t4;
-#pragma unroll
-                for (int hh = 0; hh < 2; ++hh) {
-                    const int key = cur_c * kS + mt * 16 + g + hh * 8;
-                    if (key < s.T) {
-                        red_add_v2(a.dk + (kvrow0 + key) * kD + dim, dk_acc[mt][n2][2 * hh], dk_acc[mt][n2][2 * hh + 1]);
-                        red_add_v2(a.dv + (kvrow0 + key) * kD + dim, dv_acc[mt][n2][2 * hh], dv_acc[mt][n2][2 * hh + 1]);
-                    }
-                    dk_acc[mt][n2][2 * hh] = dk_acc[mt][n2][2 * hh + 1] = 0.f;
-                    dv_acc[mt][n2][2 * hh] = dv_acc[mt][n2][2 * hh + 1] = 0.f;
-                }
+            for (int j = 0; j < 64; ++j) {
+                const int key = cur_c * kS + j;
+                if (key < s.T) red_add_f32(dst + static_cast<long long>(key) * kD, acc[j]);
             }
+        }
+        tc_fence_before_sync();
+        run_acc = false;
         lm_acc += __shfl_xor_sync(kFullMask, lm_acc, 16);
         if (cur_c < s.C) {
             const long long lrow = (static_cast<long long>(b) * s.Hl + gk) * s.C + cur_c;
@@ -699,6 +702,11 @@ prefill_backward_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __gr
         cur_c = c;
         asm volatile("cp.async.wait_group 0;" ::: "memory");
         fence_proxy_async_smem();                   // the gathered rows are read by the tensor cores (async proxy)
+        // the previous tile's dK / dV MMAs read its Q, dO rows and d S, W: all of them are overwritten from here on
+        if (tile > lo && !mbar_wait(&sm.p2_bar, p2_phase ^ 1u)) {
+            sm.abort_flag = 1;
+            if (lane == 0) set_status(a.status, kDevTimeout);
+        }
         if (kv_issued) {
             if (!mbar_wait(&sm.kv_bar, kv_phase)) {
                 sm.abort_flag = 1;
@@ -795,10 +803,6 @@ prefill_backward_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __gr
                 sv[j] = w * (tv[j] - sub) * s.scale;       // d s_j (times scale)
                 tv[j] = w;                                 // w_j
             }
-            if (tile > lo && !mbar_wait(&sm.dq_bar, dq_phase ^ 1u)) {        // the previous d Q MMA still reads d S
-                sm.abort_flag = 1;
-                if (lane == 0) set_status(a.status, kDevTimeout);
-            }
 #pragma unroll
             for (int pc = 0; pc < 8; ++pc) {
                 *reinterpret_cast<uint4*>(dsbuf + swz128(row, pc)) =
@@ -835,38 +839,29 @@ prefill_backward_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __gr
                 umma_bf16(tmem_base + 128, umma_desc_k128(ds_a + ks * 32), umma_desc_mn128(k_addr + ks * 2048, 8192u, 1024u),
                           idesc_dq, ks > 0 ? 1u : 0u);
             umma_commit(&sm.dq_bar);
+            // dK^T += Q^T dS and dV^T += dO^T W: contractions over the tile's 128 rows; A = the Q / dO rows read MN-major
+            // (dimension contiguous, the two 64-dim boxes 16 KB apart), B = d S / W read MN-major (key contiguous)
+            constexpr uint32_t idesc_kv = umma_idesc_bf16(kD, kS) | kUmmaAMnMajor | kUmmaBMnMajor;
+            const uint32_t w_a = smem_u32(wbuf);
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                const uint32_t accf = (run_acc || ks > 0) ? 1u : 0u;
+                umma_bf16(tmem_base + 256, umma_desc_mn128(q_addr + ks * 2048, kRows * 128, 1024u),
+                          umma_desc_mn128(ds_a + ks * 2048, 8192u, 1024u), idesc_kv, accf);
+                umma_bf16(tmem_base + 320, umma_desc_mn128(do_addr + ks * 2048, kRows * 128, 1024u),
+                          umma_desc_mn128(w_a + ks * 2048, 8192u, 1024u), idesc_kv, accf);
+            }
+            umma_commit(&sm.p2_bar);
             // same chunk next: its S and T can start now (their operands are in place, S / T of this tile were read)
             if (has_next && !next_new)
                 issue_st(smem_u32(qbuf0 + (par ^ 1) * kQBytes), smem_u32(dobuf0 + (par ^ 1) * kQBytes));
         }
         st_issued = has_next && !next_new;
         dq_phase ^= 1u;
+        p2_phase ^= 1u;
+        run_acc = true;
 
-        // ------------------------------------------------------------------ phase 2: dims 16 warp .. 16 warp + 15
-#pragma unroll 2
-        for (int ks = 0; ks < 8; ++ks) {
-            const int mat = lane >> 3;
-            uint32_t bq[4], bo[4];
-            {
-                const int row = ks * 16 + (mat & 1) * 8 + (lane & 7);
-                const int dim = warp * 16 + (mat >> 1) * 8;
-                const uint32_t off = (dim >> 6) * (kRows * 128) + swz128(row, (dim & 63) >> 3);
-                ldmatrix_x4_trans(q_addr + off, bq[0], bq[1], bq[2], bq[3]);
-                ldmatrix_x4_trans(do_addr + off, bo[0], bo[1], bo[2], bo[3]);
-            }
-#pragma unroll
-            for (int mt = 0; mt < 4; ++mt) {
-                const int row = ks * 16 + (mat >> 1) * 8 + (lane & 7);
-                const uint32_t off = swz128(row, 2 * mt + (mat & 1));
-                uint32_t ad[4], aw[4];
-                ldmatrix_x4_trans(ds_addr + off, ad[0], ad[1], ad[2], ad[3]);
-                ldmatrix_x4_trans(w_addr + off, aw[0], aw[1], aw[2], aw[3]);
-                mma_bf16_16816(dk_acc[mt][0], ad, bq[0], bq[1]);
-                mma_bf16_16816(dk_acc[mt][1], ad, bq[2], bq[3]);
-                mma_bf16_16816(dv_acc[mt][0], aw, bo[0], bo[1]);
-                mma_bf16_16816(dv_acc[mt][1], aw, bo[2], bo[3]);
-            }
-        }
+        // ------------------------------------------------------------------ d landmark, d bias (CUDA cores)
         {   // d landmark: sum over rows of (scale d lambda_r) q_r, lane -> (dim, half of the rows)
             const int dim = warp * 16 + (lane & 15), half = lane >> 4;
             const uint8_t* col = qbuf + (dim >> 6) * (kRows * 128) + (dim & 7) * 2;
