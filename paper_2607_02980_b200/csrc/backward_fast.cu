@@ -556,24 +556,32 @@ prefill_backward_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __gr
             if (lane == 0) set_status(a.status, kDevTimeout);
         }
         tc_fence_after_sync();
+        float o0[64], o1[64];
+        tmem_ld64x2(t_lane + 128, t_lane + 192, o0, o1);
+        if (ro_orow >= 0) {
+            float* dst = a.dq + static_cast<long long>(ro_orow) * kD;
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            float o[64];
-            tmem_ld64(t_lane + 128 + half * 64, o);
-            if (ro_orow >= 0) {
-                float* dst = a.dq + static_cast<long long>(ro_orow) * kD + half * 64;
+            for (int i = 0; i < 16; ++i) {
+                const float* l = &sm.lmf[ro_cpar][4 * i];
+                red_add_v4(dst + 4 * i, fmaf(ro_dl, l[0], o0[4 * i]), fmaf(ro_dl, l[1], o0[4 * i + 1]),
+                           fmaf(ro_dl, l[2], o0[4 * i + 2]), fmaf(ro_dl, l[3], o0[4 * i + 3]));
+            }
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const float* l = &sm.lmf[ro_cpar][half * 64 + 4 * i];
-                    red_add_v4(dst + 4 * i, fmaf(ro_dl, l[0], o[4 * i]), fmaf(ro_dl, l[1], o[4 * i + 1]),
-                               fmaf(ro_dl, l[2], o[4 * i + 2]), fmaf(ro_dl, l[3], o[4 * i + 3]));
-                }
+            for (int i = 0; i < 16; ++i) {
+                const float* l = &sm.lmf[ro_cpar][64 + 4 * i];
+                red_add_v4(dst + 64 + 4 * i, fmaf(ro_dl, l[0], o1[4 * i]), fmaf(ro_dl, l[1], o1[4 * i + 1]),
+                           fmaf(ro_dl, l[2], o1[4 * i + 2]), fmaf(ro_dl, l[3], o1[4 * i + 3]));
             }
         }
         tc_fence_before_sync();
     };
 
     const uint32_t k_addr = smem_u32(kbuf), v_addr = smem_u32(vbuf);
+    const uint64_t dk0 = umma_desc_k128(k_addr), dv0 = umma_desc_k128(v_addr);                 // K, V as K-major operands
+    const uint64_t dkmn0 = umma_desc_mn128(k_addr, 8192u, 1024u);                               // K as an MN-major operand
+    const uint64_t dds0 = umma_desc_k128(smem_u32(dsbuf));                                      // d S, K-major (d Q)
+    const uint64_t ddsmn0 = umma_desc_mn128(smem_u32(dsbuf), 8192u, 1024u);                     // d S, W MN-major (dK, dV)
+    const uint64_t dwmn0 = umma_desc_mn128(smem_u32(wbuf), 8192u, 1024u);
     const uint32_t ds_addr = smem_u32(dsbuf), w_addr = smem_u32(wbuf);
     uint32_t kv_phase = 0;
     int cur_pair = -1, cur_c = -1;
@@ -603,11 +611,10 @@ prefill_backward_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __gr
         }
         tc_fence_before_sync();
         run_acc = false;
-        lm_acc += __shfl_xor_sync(kFullMask, lm_acc, 16);
-        if (cur_c < s.C) {
+        if (cur_c < s.C && warp >= 4) {
             const long long lrow = (static_cast<long long>(b) * s.Hl + gk) * s.C + cur_c;
-            if (lane < 16) atomicAdd(a.dlm + lrow * kD + warp * 16 + lane, lm_acc);
-            if (warp == 0 && lane == 0 && a.dbias) atomicAdd(a.dbias + lrow, bias_acc / s.scale);
+            atomicAdd(a.dlm + lrow * kD + (warp - 4) * 32 + lane, lm_acc);
+            if (warp == 4 && lane == 0 && a.dbias) atomicAdd(a.dbias + lrow, bias_acc / s.scale);
         }
         lm_acc = 0.f;
         bias_acc = 0.f;
@@ -730,18 +737,20 @@ prefill_backward_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __gr
         const uint32_t q_addr = smem_u32(qbuf), do_addr = smem_u32(dobuf0 + par * kQBytes);
 
         // ------------------------------------------------------------------ S = Q K^T and T = dO V^T on tcgen05
-        const uint32_t ds_a = smem_u32(dsbuf);
+        // (a descriptor's start address is its low field in units of 16 bytes: a later k-step is the first one's
+        // descriptor plus the byte offset / 16; nothing here comes near a carry out of the field)
         auto issue_st = [&](uint32_t qa, uint32_t da) {          // one thread: S = Q K^T, T = dO V^T
             constexpr uint32_t idesc_st = umma_idesc_bf16(kRows, kS);
             tc_fence_after_sync();
+            const uint64_t dq0 = umma_desc_k128(qa), dd0 = umma_desc_k128(da);
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks)
-                umma_bf16(tmem_base, umma_desc_k128(qa + (ks >> 2) * (kRows * 128) + (ks & 3) * 32),
-                          umma_desc_k128(k_addr + (ks >> 2) * 8192 + (ks & 3) * 32), idesc_st, ks > 0 ? 1u : 0u);
+                umma_bf16(tmem_base, dq0 + (((ks >> 2) * (kRows * 128) + (ks & 3) * 32) >> 4),
+                          dk0 + (((ks >> 2) * 8192 + (ks & 3) * 32) >> 4), idesc_st, ks > 0 ? 1u : 0u);
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks)
-                umma_bf16(tmem_base + 64, umma_desc_k128(da + (ks >> 2) * (kRows * 128) + (ks & 3) * 32),
-                          umma_desc_k128(v_addr + (ks >> 2) * 8192 + (ks & 3) * 32), idesc_st, ks > 0 ? 1u : 0u);
+                umma_bf16(tmem_base + 64, dd0 + (((ks >> 2) * (kRows * 128) + (ks & 3) * 32) >> 4),
+                          dv0 + (((ks >> 2) * 8192 + (ks & 3) * 32) >> 4), idesc_st, ks > 0 ? 1u : 0u);
             umma_commit(&sm.st_bar);
         };
         if (tid == 0 && !st_issued) issue_st(q_addr, do_addr);
@@ -776,32 +785,49 @@ prefill_backward_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __gr
             }
             tc_fence_after_sync();
             float sv[64], tv[64];
-            tmem_ld64(t_lane, sv);
-            tmem_ld64(t_lane + 64, tv);
-            float m = -INFINITY;
+            tmem_ld64x2(t_lane, t_lane + 64, sv, tv);
+            // One exponential per key: e_j = exp(x_j - m) over the row's visible keys (x = scale s, four partial
+            // maxima / sums so that no chain of 64 dependent operations forms); the final weights are e_j times one
+            // factor per row: alpha / Z in a selected chunk, exp(m - lse) in the local span.
+            const float c2 = s.scale * 1.4426950408889634f;         // scale * log2(e)
+            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-            for (int j = 0; j < 64; ++j) m = fmaxf(m, sv[j]);
-            m *= s.scale;
-            float Z = 0.f, gt = 0.f;
+            for (int j = 0; j < 64; ++j) mx[j & 3] = fmaxf(mx[j & 3], j <= limit ? sv[j] : -INFINITY);
+            float m = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+            if (limit < 0) m = 0.f;                                 // padding row
+            const float m2 = m * c2;
+            float Zp[4] = {0.f, 0.f, 0.f, 0.f}, gp[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int j = 0; j < 64; ++j) {
-                const float e = __expf(sv[j] * s.scale - m);
-                Z += e;
-                gt = fmaf(e, tv[j], gt);
+                float e;
+                asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(fmaf(sv[j], c2, -m2)));
+                e = j <= limit ? e : 0.f;
+                sv[j] = e;
+                Zp[j & 3] += e;
+                gp[j & 3] = fmaf(e, tv[j], gp[j & 3]);
             }
-            float shift = lse, sub = dsum, dl = 0.f;
+            const float Z = (Zp[0] + Zp[1]) + (Zp[2] + Zp[3]), gt = (gp[0] + gp[1]) + (gp[2] + gp[3]);
+            m *= s.scale;
+            float f, sub = dsum, dl = 0.f;
             if (!local) {
                 const float gc = gt / Z;
                 const float alpha = __expf(lam - lse);
-                shift = m + __logf(Z) - (lam - lse);
+                f = alpha / Z;
                 sub = gc;
                 dl = limit >= 0 ? alpha * (gc - dsum) * s.scale : 0.f;
+            } else {
+                f = __expf(m - lse);
             }
+            if (limit < 0) {                                        // padding row: Z = 0, nothing may leak a NaN
+                f = 0.f;
+                sub = 0.f;
+            }
+            const float fs = f * s.scale;
 #pragma unroll
             for (int j = 0; j < 64; ++j) {
-                const float w = j <= limit ? __expf(sv[j] * s.scale - shift) : 0.f;
-                sv[j] = w * (tv[j] - sub) * s.scale;       // d s_j (times scale)
-                tv[j] = w;                                 // w_j
+                const float e = sv[j];
+                sv[j] = e * fs * (tv[j] - sub);            // d s_j (times scale)
+                tv[j] = e * f;                             // w_j
             }
 #pragma unroll
             for (int pc = 0; pc < 8; ++pc) {
@@ -836,20 +862,17 @@ prefill_backward_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __gr
             tc_fence_after_sync();
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks)
-                umma_bf16(tmem_base + 128, umma_desc_k128(ds_a + ks * 32), umma_desc_mn128(k_addr + ks * 2048, 8192u, 1024u),
-                          idesc_dq, ks > 0 ? 1u : 0u);
+                umma_bf16(tmem_base + 128, dds0 + ((ks * 32) >> 4), dkmn0 + ((ks * 2048) >> 4), idesc_dq, ks > 0 ? 1u : 0u);
             umma_commit(&sm.dq_bar);
             // dK^T += Q^T dS and dV^T += dO^T W: contractions over the tile's 128 rows; A = the Q / dO rows read MN-major
             // (dimension contiguous, the two 64-dim boxes 16 KB apart), B = d S / W read MN-major (key contiguous)
             constexpr uint32_t idesc_kv = umma_idesc_bf16(kD, kS) | kUmmaAMnMajor | kUmmaBMnMajor;
-            const uint32_t w_a = smem_u32(wbuf);
+            const uint64_t dqmn0 = umma_desc_mn128(q_addr, kRows * 128, 1024u), ddmn0 = umma_desc_mn128(do_addr, kRows * 128, 1024u);
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
                 const uint32_t accf = (run_acc || ks > 0) ? 1u : 0u;
-                umma_bf16(tmem_base + 256, umma_desc_mn128(q_addr + ks * 2048, kRows * 128, 1024u),
-                          umma_desc_mn128(ds_a + ks * 2048, 8192u, 1024u), idesc_kv, accf);
-                umma_bf16(tmem_base + 320, umma_desc_mn128(do_addr + ks * 2048, kRows * 128, 1024u),
-                          umma_desc_mn128(w_a + ks * 2048, 8192u, 1024u), idesc_kv, accf);
+                umma_bf16(tmem_base + 256, dqmn0 + ((ks * 2048) >> 4), ddsmn0 + ((ks * 2048) >> 4), idesc_kv, accf);
+                umma_bf16(tmem_base + 320, ddmn0 + ((ks * 2048) >> 4), dwmn0 + ((ks * 2048) >> 4), idesc_kv, accf);
             }
             umma_commit(&sm.p2_bar);
             // same chunk next: its S and T can start now (their operands are in place, S / T of this tile were read)
@@ -862,19 +885,20 @@ prefill_backward_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __gr
         run_acc = true;
 
         // ------------------------------------------------------------------ d landmark, d bias (CUDA cores)
-        {   // d landmark: sum over rows of (scale d lambda_r) q_r, lane -> (dim, half of the rows)
-            const int dim = warp * 16 + (lane & 15), half = lane >> 4;
+        if (warp >= 4) {
+            // d landmark: sum over rows of (scale d lambda_r) q_r.  Warp w - 4 owns dims 32 (w - 4) .. +31 (one per
+            // lane) and walks all 128 rows; the partial sums stay in a register until the chunk ends.
+            const int dim = (warp - 4) * 32 + lane;
             const uint8_t* col = qbuf + (dim >> 6) * (kRows * 128) + (dim & 7) * 2;
             const int piece = (dim & 63) >> 3;
-            float acc = 0.f;
+            float acc0 = 0.f, acc1 = 0.f;
 #pragma unroll 8
-            for (int r = half * 64; r < half * 64 + 64; ++r) {
-                const float dl = sm.dlam[r];
-                const __nv_bfloat16 x = *reinterpret_cast<const __nv_bfloat16*>(col + swz128(r, piece));
-                acc = fmaf(dl, __bfloat162float(x), acc);
+            for (int r = 0; r < kRows; r += 2) {
+                acc0 = fmaf(sm.dlam[r], __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(col + swz128(r, piece))), acc0);
+                acc1 = fmaf(sm.dlam[r + 1], __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(col + swz128(r + 1, piece))), acc1);
             }
-            lm_acc += acc;
-            if (warp == 0) {
+            lm_acc += acc0 + acc1;
+            if (warp == 4) {
                 const float v = sm.dlam[lane] + sm.dlam[lane + 32] + sm.dlam[lane + 64] + sm.dlam[lane + 96];
                 bias_acc += warp_sum(v);
             }
