@@ -486,7 +486,7 @@ prefill_backward_mma_kernel(const __grid_constant__ CUtensorMap map_k, const __g
 struct BtSmem {               // shared state of the tcgen05 variant
     uint64_t kv_bar, st_bar, dq_bar, p2_bar;
     uint32_t tmem_base;
-    float lmf[2][kD];         // the landmark of the chunk in work and of the next one
+    alignas(16) float lmf[2][kD];   // the landmark of the chunk in work and of the next one
     float bias_c[2];
     float dlam[kRows];
     float row_lse[2][kRows];
@@ -764,21 +764,27 @@ prefill_backward_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __gr
             const bool local = sm.row_local[par][row] != 0;
             const float lse = sm.row_lse[par][row], dsum = sm.row_dsum[par][row];
             // surrogate score of the row (its own Q row against the landmark) while the MMAs run
-            float lam = 0.f;
+            float lam = 0.f, lam2 = 0.f;
 #pragma unroll
             for (int half = 0; half < 2; ++half)
 #pragma unroll
                 for (int pc = 0; pc < 8; ++pc) {
                     const uint4 v = *reinterpret_cast<const uint4*>(qbuf + half * (kRows * 128) + swz128(row, pc));
                     const __nv_bfloat162* pv = reinterpret_cast<const __nv_bfloat162*>(&v);
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const float2 x = __bfloat1622float2(pv[i]);
-                        lam = fmaf(x.x, sm.lmf[cpar][half * 64 + pc * 8 + 2 * i], lam);
-                        lam = fmaf(x.y, sm.lmf[cpar][half * 64 + pc * 8 + 2 * i + 1], lam);
-                    }
+                    const float4 l0 = *reinterpret_cast<const float4*>(&sm.lmf[cpar][half * 64 + pc * 8]);
+                    const float4 l1 = *reinterpret_cast<const float4*>(&sm.lmf[cpar][half * 64 + pc * 8 + 4]);
+                    const float2 x0 = __bfloat1622float2(pv[0]), x1 = __bfloat1622float2(pv[1]);
+                    const float2 x2 = __bfloat1622float2(pv[2]), x3 = __bfloat1622float2(pv[3]);
+                    lam = fmaf(x0.x, l0.x, lam);
+                    lam2 = fmaf(x0.y, l0.y, lam2);
+                    lam = fmaf(x1.x, l0.z, lam);
+                    lam2 = fmaf(x1.y, l0.w, lam2);
+                    lam = fmaf(x2.x, l1.x, lam);
+                    lam2 = fmaf(x2.y, l1.y, lam2);
+                    lam = fmaf(x3.x, l1.z, lam);
+                    lam2 = fmaf(x3.y, l1.w, lam2);
                 }
-            lam = lam * s.scale + sm.bias_c[cpar];
+            lam = (lam + lam2) * s.scale + sm.bias_c[cpar];
             if (!mbar_wait(&sm.st_bar, st_phase)) {
                 sm.abort_flag = 1;
                 if (lane == 0) set_status(a.status, kDevTimeout);
