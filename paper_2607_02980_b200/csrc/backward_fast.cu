@@ -644,38 +644,58 @@ prefill_backward_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __gr
     struct RowInfo { int orow, limit, local; float lse, dsum; };
     // entry of this thread's row in a tile (read two tiles ahead of its use, so that no tile waits for it)
     auto load_entry = [&](const int4 rec) { return (tid >> 3) < rec.w ? a.entries[rec.z + (tid >> 3)] : 0; };
-    auto issue_tile = [&](const int4 rec, int ent, int par) {
+    // Gather of a tile's Q and dO rows.  Eight consecutive lanes fetch the eight 16-byte pieces of one 128-byte
+    // half row, so every request covers whole lines; a group of eight lanes owns one entry = its four heads' rows.
+    // The copies are requested in four parts (head g in part g), spread over the computation of the tile before.
+    struct Gather { const __nv_bfloat16* qs; const __nv_bfloat16* ds; uint32_t qa, da; int row0; bool valid; };
+    auto gather_part = [&](const Gather& gt, int g) {
+        if (gt.valid) {
+            const int row = gt.row0 + g, pc = tid & 7;
+            const long long src = static_cast<long long>(g) * s.R * kD;          // head g of the entry's token
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                cp_async16(gt.qa + half * (kRows * 128) + swz128(row, pc), gt.qs + src + half * 64);
+                cp_async16(gt.da + half * (kRows * 128) + swz128(row, pc), gt.ds + src + half * 64);
+            }
+        }
+    };
+    auto issue_tile = [&](const int4 rec, int ent, int par, Gather* defer = nullptr) {
         const int pair = rec.x, c = rec.y, ntok = rec.w;
         const int b = pair / s.Hkv, gk = pair % s.Hkv;
-        const int row = tid >> 1, half = tid & 1, e = row >> 2, h = row & 3;
+        const int row = tid >> 1, e = tid >> 3, h = row & 3;               // e = the entry of row tid / 2 as well
         RowInfo ri{-1, -1, 0, 0.f, 0.f};
-        uint8_t* qb = qbuf0 + par * kQBytes + half * (kRows * 128);
-        uint8_t* db = dobuf0 + par * kQBytes + half * (kRows * 128);
+        uint8_t* qb = qbuf0 + par * kQBytes;
+        uint8_t* db = dobuf0 + par * kQBytes;
         if (e < ntok) {
             const int tok = a.i0 + (ent >> 8), slot = ent & 255;
-            ri.orow = (b * s.Hq + gk * kG + h) * s.R + tok;
+            const int orow0 = (b * s.Hq + gk * kG) * s.R + tok;            // head 0 of the entry
+            ri.orow = orow0 + h * s.R;
             ri.local = slot >= s.K ? 1 : 0;
             ri.limit = ri.local ? min(kS - 1, s.pos0 + tok - c * kS) : kS - 1;
-            const __nv_bfloat16* qs = a.q + static_cast<long long>(ri.orow) * kD + half * 64;
-            const __nv_bfloat16* ds = a.dout + static_cast<long long>(ri.orow) * kD + half * 64;
-            const uint32_t qa = smem_u32(qb), da = smem_u32(db);
+            const Gather gt{a.q + static_cast<long long>(orow0) * kD + (tid & 7) * 8,
+                            a.dout + static_cast<long long>(orow0) * kD + (tid & 7) * 8, smem_u32(qb), smem_u32(db), e * 4, true};
+            if (defer) {
+                *defer = gt;
+                gather_part(gt, 0);
+            } else {
 #pragma unroll
-            for (int p = 0; p < 8; ++p) {
-                cp_async16(qa + swz128(row, p), qs + p * 8);
-                cp_async16(da + swz128(row, p), ds + p * 8);
+                for (int g4 = 0; g4 < 4; ++g4) gather_part(gt, g4);
             }
-            if (half == 0) {
+            if ((tid & 1) == 0) {
                 ri.lse = a.lse[ri.orow];
                 ri.dsum = a.dsum[ri.orow];
             }
         } else {
+            // padding entry: its four rows are zero
 #pragma unroll
-            for (int p = 0; p < 8; ++p) {
-                *reinterpret_cast<uint4*>(qb + swz128(row, p)) = make_uint4(0u, 0u, 0u, 0u);
-                *reinterpret_cast<uint4*>(db + swz128(row, p)) = make_uint4(0u, 0u, 0u, 0u);
-            }
+            for (int g4 = 0; g4 < 4; ++g4)
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    *reinterpret_cast<uint4*>(qb + half * (kRows * 128) + swz128(e * 4 + g4, tid & 7)) = make_uint4(0u, 0u, 0u, 0u);
+                    *reinterpret_cast<uint4*>(db + half * (kRows * 128) + swz128(e * 4 + g4, tid & 7)) = make_uint4(0u, 0u, 0u, 0u);
+                }
         }
-        asm volatile("cp.async.commit_group;" ::: "memory");
+        if (!defer) asm volatile("cp.async.commit_group;" ::: "memory");
         return ri;
     };
     auto store_row = [&](const RowInfo& ri, int par) {
@@ -728,7 +748,8 @@ prefill_backward_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __gr
         // the next tile's rows start to arrive while this one is computed
         const bool has_next = tile + 1 < hi;
         RowInfo nri{-1, -1, 0, 0.f, 0.f};
-        if (has_next) nri = issue_tile(nrec, nent, par ^ 1);
+        Gather gth{nullptr, nullptr, 0u, 0u, 0, false};
+        if (has_next) nri = issue_tile(nrec, nent, par ^ 1, &gth);
         // metadata of the tiles after the next: in registers by the time they are needed
         const int n2ent = load_entry(n2rec);
         const int4 n3rec = tile + 3 < hi ? a.tiles[tile + 3] : no_tile;
@@ -755,7 +776,12 @@ prefill_backward_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __gr
         };
         if (tid == 0 && !st_issued) issue_st(q_addr, do_addr);
         // the previous tile's d Q leaves tensor memory while this tile's statistics are computed
-        if (warp >= 4 && ro_pending) read_out();
+        if (warp >= 4) {
+            gather_part(gth, 1);
+            if (ro_pending) read_out();
+            gather_part(gth, 2);
+            gather_part(gth, 3);
+        }
         ro_pending = false;
         // ------------------------------------------------------------------ phase 1: warps 0-3, one row per thread
         if (warp < 4) {
@@ -785,6 +811,7 @@ prefill_backward_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __gr
                     lam2 = fmaf(x3.y, l1.w, lam2);
                 }
             lam = (lam + lam2) * s.scale + sm.bias_c[cpar];
+            gather_part(gth, 1);
             if (!mbar_wait(&sm.st_bar, st_phase)) {
                 sm.abort_flag = 1;
                 if (lane == 0) set_status(a.status, kDevTimeout);
@@ -792,6 +819,7 @@ prefill_backward_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __gr
             tc_fence_after_sync();
             float sv[64], tv[64];
             tmem_ld64x2(t_lane, t_lane + 64, sv, tv);
+            gather_part(gth, 2);
             // One exponential per key: e_j = exp(x_j - m) over the row's visible keys (x = scale s, four partial
             // maxima / sums so that no chain of 64 dependent operations forms); the final weights are e_j times one
             // factor per row: alpha / Z in a selected chunk, exp(m - lse) in the local span.
@@ -812,6 +840,7 @@ prefill_backward_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __gr
                 Zp[j & 3] += e;
                 gp[j & 3] = fmaf(e, tv[j], gp[j & 3]);
             }
+            gather_part(gth, 3);
             const float Z = (Zp[0] + Zp[1]) + (Zp[2] + Zp[3]), gt = (gp[0] + gp[1]) + (gp[2] + gp[3]);
             m *= s.scale;
             float f, sub = dsum, dl = 0.f;
@@ -850,6 +879,7 @@ prefill_backward_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __gr
         }
         st_phase ^= 1u;
         if (has_next) store_row(nri, par ^ 1);
+        asm volatile("cp.async.commit_group;" ::: "memory");
         if (has_next && !next_new) {
             asm volatile("cp.async.wait_group 0;" ::: "memory");
             fence_proxy_async_smem();
