@@ -3,15 +3,19 @@
 // accumulated on chip over all the queries that attend it.  Formulas: see backward.cu / the C header.
 //
 // The tiles of the forward's inverse index are reused: a tile is 32 (token, slot) entries x 4 heads = 128 query
-// rows against one 64-key chunk.  A CTA of 8 warps walks a contiguous range of a query block's tiles.  Per tile
-//   phase 1 (warp w owns rows 16w .. 16w+15):  S = Q K^T and T = dO V^T on mma.sync (bf16 -> fp32), the slot's
-//           softmax statistics with quad shuffles, w_j and d s_j; d s and w go to shared memory as bf16;
-//           d Q = d S K (+ the landmark term) is added to dq with vector reductions;
-//   phase 2 (warp w owns dims 16w .. 16w+15):  d K += d S^T Q and d V += W^T dO, contractions over the 128 rows,
-//           accumulated in registers over the run of tiles of one chunk and added to dk / dv when the run ends;
-//           d landmark and d bias of the chunk likewise.
-// K and V of the chunk arrive by TMA (128-byte swizzle), Q and dO rows by cp.async into the same swizzled layout,
-// so that every MMA operand is read with ldmatrix.
+// rows against one 64-key chunk.  A CTA of 8 warps walks a contiguous range of a query block's tiles.  K and V of
+// the chunk arrive by TMA (128-byte swizzle), Q and dO rows by cp.async into the same swizzled layout.
+//
+// prefill_backward_tc_kernel (default): every product on the 5th-generation tensor cores, accumulators in tensor
+//   memory.  S = Q K^T and T = dO V^T (K-major operands); warps 0-3 read one row each with tcgen05.ld, compute the
+//   slot's softmax statistics thread-locally and write d S and W rows to shared memory as bf16; d Q = d S K (K read
+//   MN-major); dK^T += Q^T d S and dV^T += dO^T W with both operands MN-major (the row tiles as they sit in shared
+//   memory), accumulated in tensor memory over the tiles of a chunk.  Warps 4-7 read d Q of the previous tile out
+//   beside the next tile's statistics (+ the landmark term, vector reductions into dq) and compute d landmark and
+//   d bias; one thread issues the MMAs.
+// prefill_backward_mma_kernel (HILS_BACKWARD_MMA_SYNC=1): the first version, every product on mma.sync with
+//   ldmatrix operands: phase 1, warp = 16 rows: S, T, statistics with quad shuffles, d Q; phase 2, warp = 16 dims:
+//   d K += d S^T Q, d V += W^T dO in registers across the tiles of a chunk.
 #include <stdlib.h>
 
 #include "internal.h"
