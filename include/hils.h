@@ -262,6 +262,9 @@ int hils_chunk_overlap(const hils_params* params, const int32_t* sel_idx, int32_
  *   dk, dv          [B, Hkv, T, d]  fp32 DEVICE, overwritten (zeroed by the call, then accumulated)
  *   dlandmarks      [B, Hl, C, d]   fp32 DEVICE, same
  *   dbias           [B, Hl, C]      fp32 DEVICE or NULL, same
+ * bf16 with d = 128, chunk_size = 64, four query heads per KV head and one landmark per KV head runs on the
+ * 5th-generation tensor cores (chunk-major, accumulators in tensor memory); every other supported shape on
+ * CUDA cores (params->impl selects as for hils_prefill).
  * All gradient pointers 16-byte aligned (dbias 4).  Sums over queries are accumulated with fp32 atomics, so
  * the last bits of dk, dv, dlandmarks, dbias may differ from run to run.  Workspace:
  * hils_prefill_backward_workspace_bytes (0 = unsupported shape); its head is the status word of
