@@ -430,18 +430,21 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                     tc_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&sm.s_empty[sl]);
-                    float m = -INFINITY;
+                    // four independent chains for the maximum and for the sum: the row is one thread's work and a
+                    // single chain of 64 dependent operations is what the warp would otherwise wait on
+                    float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
                     if (__any_sync(kFullMask, local)) {
 #pragma unroll
                         for (int j = 0; j < 64; ++j) {
                             if (j > lim) v[j] = -INFINITY;
-                            m = fmaxf(m, v[j]);
+                            mx[j & 3] = fmaxf(mx[j & 3], v[j]);
                         }
                     } else {
 #pragma unroll
-                        for (int j = 0; j < 64; ++j) m = fmaxf(m, v[j]);
+                        for (int j = 0; j < 64; ++j) mx[j & 3] = fmaxf(mx[j & 3], v[j]);
                     }
-                    float z = 0.f;
+                    const float m = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+                    float zp[4] = {0.f, 0.f, 0.f, 0.f};
                     const float ms2 = m * sl2;
                     // this warp's rows of the slot staged the previous tile's output: its store must have read them
                     if (lane == 0) bulk_wait_read<0>();
@@ -453,11 +456,12 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                         for (int j = 0; j < 4; ++j) {
                             const float p0 = ex2_approx(fmaf(v[pc * 8 + 2 * j], sl2, -ms2));
                             const float p1 = ex2_approx(fmaf(v[pc * 8 + 2 * j + 1], sl2, -ms2));
-                            z += p0 + p1;
+                            zp[j] += p0 + p1;
                             pk[j] = pack_bf16(p0, p1);
                         }
                         *reinterpret_cast<uint4*>(pslot + swz128(row, pc)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                     }
+                    const float z = (zp[0] + zp[1]) + (zp[2] + zp[3]);
                     zi = 1.f / z;
                     // chunk mass of the row (rows of a ragged tile's padding land in the list's padding)
                     const float bb = (a.bias && c < s.C)
