@@ -2,15 +2,20 @@
 //
 // A tile is 32 (token, slot) entries of one chunk x 4 heads = 128 query rows (one TMEM lane each).
 // Per tile:  S = Q K_c^T (M=128, N=80: 64 keys + the chunk's landmark as key 64, K=128) -> tensor memory;
-//            each epilogue thread owns one row: mask (local rows are causal), the chunk's own softmax
-//            (Eq. HiLS weights, intra-chunk factor), P as bf16 back to shared memory;
-//            O = P V_c (M=128, N=128, K=64, V read as an MN-major operand exactly as TMA wrote it) -> tensor memory;
+//            each softmax thread owns one row: mask (local rows are causal), the chunk's own softmax
+//            (Eq. HiLS weights, intra-chunk factor), P as bf16 pairs into tensor memory (32 columns behind the
+//            slot's scores: shared memory carries neither the write nor the read of P);
+//            O = P V_c (M=128, N=128, K=64; A = P from tensor memory, V read from shared memory as an MN-major
+//            operand exactly as TMA wrote it) -> tensor memory;
 //            normalised bf16 rows and the row's chunk mass (surrogate score, or log Z_swa for the
 //            local branch) go to the buffers that prefill_fuse mixes, in entry order: a tile's 128 rows
-//            are contiguous there, so every epilogue warp hands its 32 rows to one TMA store per half.
-// Warp roles: 0-7 epilogue (warps 0-3 take even tiles, 4-7 odd tiles; a warp reads the TMEM lane quarter
-// warp % 4), 8-11 producers (cp.async gather of Q rows, TMA of K/V), 12 MMA issue.
+//            are contiguous there, so every output warp hands its 32 rows to one TMA store per half.
+// Warp roles: 0-3 softmax of every tile, 4-7 output of every tile (a warp reads the TMEM lane quarter warp % 4; the
+// softmax of a tile never waits for the tile's own P V, and 1 / row sum passes through a small ring in shared
+// memory), 8-11 producers (cp.async gather of Q rows, TMA of K/V), 12 MMA issue.
 // S/P/O are double buffered, three gathered Q tiles are in flight, K tiles are double and V tiles triple buffered.
+// What bounds the kernel is the shared-memory port: the MMA operands (Q 32 KB + K 20 KB + V 16 KB per tile), the
+// gathered Q rows (32 KB) and the output staging (32 KB in, 32 KB out) all pass through it.
 #include "internal.h"
 #include "tma.cuh"
 
@@ -27,12 +32,13 @@ constexpr int kKBytes = kNS * 128 * 2;          // two 64-dim K-blocks of 80 row
 constexpr int kVBytes = kS * kD * 2;            // two boxes of 64 keys x 64 dims
 constexpr int kQBytes = kRows * kD * 2;         // 32 KB
 constexpr int kPBytes = kRows * 128;            // 16 KB
+constexpr int kPCol = 96;                       // probabilities (bf16 pairs, 32 columns) behind the slot's 80 score columns
 constexpr int kBatch = 128;                     // tile records cached per batch
 constexpr int kQSlots = 3;                      // gathered Q tiles in flight
 constexpr int kVBufs = 3;                       // V tiles in flight (K: 2)
 constexpr int kMetaSlots = 8;                   // ring of tile descriptors (producers are < 8 tiles ahead of the epilogue)
 constexpr int kProdThreads = 128;
-constexpr int kEpiThreads = 256;
+constexpr int kEpiThreads = 256;                // a softmax group and an output group of 128 threads
 constexpr int kThreads = kEpiThreads + kProdThreads + 32;
 constexpr int kProdWarp0 = kEpiThreads / 32;
 constexpr int kMmaWarp = kProdWarp0 + kProdThreads / 32;
@@ -49,7 +55,7 @@ struct AtcSmem {
     uint64_t q_empty[kQSlots];// the S MMA that reads this Q tile has completed
     uint64_t s_full[2];       // S = Q K^T in tensor memory
     uint64_t s_empty[2];      // epilogue has read S
-    uint64_t p_full[2];       // P written to shared memory and fenced
+    uint64_t p_full[2];       // P written to tensor memory
     uint64_t o_full[2];       // O = P V in tensor memory
     uint64_t o_empty[2];      // epilogue has read O
     uint32_t tmem_base;
@@ -58,6 +64,7 @@ struct AtcSmem {
     int tile_meta[kMetaSlots][4];     // pair, chunk, tokens, first entry relative to the query block
     const __nv_bfloat16* rowptr[2][kRows];
     int4 recs[kBatch];
+    float zinv[4][kRows];             // 1 / row sum of the tiles in flight (softmax group -> output group)
     int nchunks;                      // distinct (pair, chunk) runs in the current batch
     uint8_t cfirst[kBatch + 4];       // first tile (batch index) of each run; cfirst[nchunks] = tiles in the batch
 };
@@ -100,8 +107,8 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
     uint8_t* kbuf = base;                                   // [2][kKBytes]
     uint8_t* vbuf = kbuf + 2 * kKBytes;                     // [kVBufs][kVBytes]
     uint8_t* qbuf = vbuf + kVBufs * kVBytes;                     // [kQSlots][kQBytes]
-    uint8_t* pbuf = qbuf + kQSlots * kQBytes;               // [2][kPBytes]
-    AtcSmem& sm = *reinterpret_cast<AtcSmem*>(pbuf + 2 * kPBytes);
+    uint8_t* obuf = qbuf + kQSlots * kQBytes;               // [2][kPBytes]: staging of the output rows being stored
+    AtcSmem& sm = *reinterpret_cast<AtcSmem*>(obuf + 2 * kPBytes);
 
     const Shape& s = a.s;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -264,8 +271,8 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                 if (ptid == 0 && !next_issued) {
                     const int tj = sm.cfirst[ck + 1];          // first tile of the next run (nb if none)
                     const uint32_t nbuf = cc & 1u, nvb = cc % kVBufs;
-                    if (tj < nb && (cc < 2 || mbar_try_wait(&sm.k_empty[nbuf], ((cc >> 1) - 1) & 1)) &&
-                        (cc < kVBufs || mbar_try_wait(&sm.v_empty[nvb], ((cc / kVBufs) - 1) & 1))) {
+                    if (tj < nb && (cc < 2 || mbar_test_wait(&sm.k_empty[nbuf], ((cc >> 1) - 1) & 1)) &&
+                        (cc < kVBufs || mbar_test_wait(&sm.v_empty[nvb], ((cc / kVBufs) - 1) & 1))) {
                         const int row = sm.recs[tj].x * s.T + sm.recs[tj].y * kS;
                         mbar_expect_tx(&sm.k_ready[nbuf], 2 * 8192);
                         tma_load_2d(kbuf + nbuf * kKBytes, &map_k, &sm.k_ready[nbuf], 0, row);
@@ -342,11 +349,11 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                         const uint32_t tcv = tcount + ns, sl = tcv & 1u, qs = tcv % kQSlots;
                         const int4 rec = sm.recs[ns];
                         const bool newc = rec.x != cur_pair || rec.y != cur_c;
-                        bool ready = mbar_try_wait(&sm.q_full[qs], (tcv / kQSlots) & 1);
+                        bool ready = mbar_test_wait(&sm.q_full[qs], (tcv / kQSlots) & 1);
                         if (ready && newc)
-                            ready = mbar_try_wait(&sm.k_ready[cc & 1u], (cc >> 1) & 1) &&
-                                    mbar_try_wait(&sm.v_ready[cc % kVBufs], (cc / kVBufs) & 1);
-                        if (ready && tcv >= 2) ready = mbar_try_wait(&sm.s_empty[sl], ((tcv >> 1) - 1) & 1);
+                            ready = mbar_test_wait(&sm.k_ready[cc & 1u], (cc >> 1) & 1) &&
+                                    mbar_test_wait(&sm.v_ready[cc % kVBufs], (cc / kVBufs) & 1);
+                        if (ready && tcv >= 2) ready = mbar_test_wait(&sm.s_empty[sl], ((tcv >> 1) - 1) & 1);
                         if (ready) {
                             if (newc) { cur_pair = rec.x; cur_c = rec.y; ++cc; }
                             const uint32_t cb = (cc - 1) & 1u;
@@ -367,15 +374,17 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                     }
                     if (no < ns) {
                         const uint32_t tcv = tcount + no, sl = tcv & 1u, vb = vbuf_of[sl];
-                        bool ready = mbar_try_wait(&sm.p_full[sl], (tcv >> 1) & 1);
-                        if (ready && tcv >= 2) ready = mbar_try_wait(&sm.o_empty[sl], ((tcv >> 1) - 1) & 1);
+                        bool ready = mbar_test_wait(&sm.p_full[sl], (tcv >> 1) & 1);
+                        if (ready && tcv >= 2) ready = mbar_test_wait(&sm.o_empty[sl], ((tcv >> 1) - 1) & 1);
                         if (ready) {
                             tc_fence_after_sync();
-                            const uint32_t pa = smem_u32(pbuf + sl * kPBytes), va = smem_u32(vbuf + vb * kVBytes);
+                            const uint32_t va = smem_u32(vbuf + vb * kVBytes);
+                            // P from tensor memory (columns kPCol.. of the slot: 8 columns = 16 keys per step), V from
+                            // shared memory, 16 keys per step = two 8-row groups
 #pragma unroll
-                            for (int ks = 0; ks < 4; ++ks)      // 16 keys per step = two 8-row groups of V
-                                umma_bf16(tmem_base + 256 + sl * 128, umma_desc_k128(pa + ks * 32),
-                                          umma_desc_mn128(va + ks * 2048, 8192u, 1024u), idesc_o, ks > 0 ? 1u : 0u);
+                            for (int ks = 0; ks < 4; ++ks)
+                                umma_bf16_ts(tmem_base + 256 + sl * 128, tmem_base + sl * 128 + kPCol + ks * 8,
+                                             umma_desc_mn128(va + ks * 2048, 8192u, 1024u), idesc_o, ks > 0 ? 1u : 0u);
                             umma_commit(&sm.o_full[sl]);
                             // last tile of its chunk in this batch: the V buffer is free once these MMAs are done
                             const bool last = no + 1 >= nb || sm.recs[no + 1].x != sm.recs[no].x || sm.recs[no + 1].y != sm.recs[no].y;
@@ -395,31 +404,27 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
             }
         } else {
             // ================================================================ epilogue: one row per thread
-            const int grp = warp >> 2;                       // tiles of parity grp, S/P/O slot grp
+            // Group 0 turns every tile's scores into probabilities, group 1 takes every tile's O = P V out of tensor
+            // memory: the softmax of a tile never waits for the tile's own P V.
+            const int grp = warp >> 2;
             const int row = (warp & 3) * 32 + lane;
-            const int tk = row >> 2, hd = row & 3;
             const uint32_t t_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-            const float sl2 = s.scale * kLog2e;
-            const uint32_t sl = static_cast<uint32_t>(grp);
-            uint8_t* pslot = pbuf + sl * kPBytes;
-            const uint64_t pol = l2_policy_evict_first();
             bool ok = true;
-            for (int ti = 0; ti < nb && ok; ++ti) {
-                const uint32_t tcv = tcount + ti;
-                if ((tcv & 1u) != sl) continue;
-                // ---------------- scores -> probabilities
-                ok = mbar_wait(&sm.s_full[sl], (tcv >> 1) & 1);
-                if (!ok) break;
-                tc_fence_after_sync();
-                const uint32_t ms = tcv % kMetaSlots;
-                const int pair = sm.tile_meta[ms][0], c = sm.tile_meta[ms][1];
-                const int orow0 = sm.tile_meta[ms][3] * kG;          // first row of the tile in the output buffers
-                const int e = sm.tile_ent[ms][tk];
-                const int il = e >> 8, slot = e & 255;
-                const bool local = slot >= s.K;                            // a chunk of the local window: mass = its exact log-sum-exp
-                const int lim = local ? s.pos0 + i0 + il - c * kS : kS - 1;   // last visible key of the chunk
-                float zi;
-                {
+            if (grp == 0) {
+                const int tk = row >> 2, hd = row & 3;
+                const float sl2 = s.scale * kLog2e;
+                for (int ti = 0; ti < nb && ok; ++ti) {
+                    const uint32_t tcv = tcount + ti, sl = tcv & 1u;
+                    ok = mbar_wait(&sm.s_full[sl], (tcv >> 1) & 1);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const uint32_t ms = tcv % kMetaSlots;
+                    const int pair = sm.tile_meta[ms][0], c = sm.tile_meta[ms][1];
+                    const int orow0 = sm.tile_meta[ms][3] * kG;          // first row of the tile in the output buffers
+                    const int e = sm.tile_ent[ms][tk];
+                    const int il = e >> 8, slot = e & 255;
+                    const bool local = slot >= s.K;                            // a chunk of the local window: mass = its exact log-sum-exp
+                    const int lim = local ? s.pos0 + i0 + il - c * kS : kS - 1;   // last visible key of the chunk
                     float v[64];
                     tmem_ld64(t_lane + sl * 128, v);
                     // surrogate score column: the landmark of this row's head (key 64 + hd) or the shared one (key 64)
@@ -446,64 +451,80 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                     const float m = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
                     float zp[4] = {0.f, 0.f, 0.f, 0.f};
                     const float ms2 = m * sl2;
-                    // this warp's rows of the slot staged the previous tile's output: its store must have read them
-                    if (lane == 0) bulk_wait_read<0>();
-                    __syncwarp();
+                    // the P V product of this slot's previous tile must have read its probabilities
+                    if (tcv >= 2) {
+                        ok = mbar_wait(&sm.o_full[sl], ((tcv >> 1) - 1) & 1);
+                        if (!ok) break;
+                    }
 #pragma unroll
-                    for (int pc = 0; pc < 8; ++pc) {
-                        uint32_t pk[4];
+                    for (int pc = 0; pc < 4; ++pc) {
+                        uint32_t pk[8];
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const float p0 = ex2_approx(fmaf(v[pc * 8 + 2 * j], sl2, -ms2));
-                            const float p1 = ex2_approx(fmaf(v[pc * 8 + 2 * j + 1], sl2, -ms2));
-                            zp[j] += p0 + p1;
+                        for (int j = 0; j < 8; ++j) {
+                            const float p0 = ex2_approx(fmaf(v[pc * 16 + 2 * j], sl2, -ms2));
+                            const float p1 = ex2_approx(fmaf(v[pc * 16 + 2 * j + 1], sl2, -ms2));
+                            zp[j & 3] += p0 + p1;
                             pk[j] = pack_bf16(p0, p1);
                         }
-                        *reinterpret_cast<uint4*>(pslot + swz128(row, pc)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        tmem_st8(t_lane + sl * 128 + kPCol + pc * 8, pk);
                     }
                     const float z = (zp[0] + zp[1]) + (zp[2] + zp[3]);
-                    zi = 1.f / z;
+                    // read by the output group after this tile's P V.  The ring's slot was last read for the tile
+                    // four back, before the output group released that tile's accumulator; the P V waited for
+                    // above could only be issued after that release.
+                    sm.zinv[tcv & 3u][row] = 1.f / z;
                     // chunk mass of the row (rows of a ragged tile's padding land in the list's padding)
                     const float bb = (a.bias && c < s.C)
                         ? a.bias[(static_cast<long long>(pair / s.Hkv) * s.Hl + (pair % s.Hkv) * (s.Hl / s.Hkv) + lh) * s.C + c] : 0.f;
                     a.lam[orow0 + row] = local ? m * s.scale + __logf(z) : lmk * s.scale + bb;
+                    tmem_wait_st();
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sm.p_full[sl]);
                 }
-                fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&sm.p_full[sl]);
-                // ---------------- O = P V -> normalised bf16 rows
-                ok = mbar_wait(&sm.o_full[sl], (tcv >> 1) & 1);
-                if (!ok) break;
-                tc_fence_after_sync();
-                // P has been consumed: the warp's 32 rows of its slot (4 KB, swizzled as the output map expects) stage
-                // the output, 64 columns at a time; one TMA store per half writes 32 full rows
-                uint8_t* wstg = pslot + (warp & 3) * 4096;
+            } else {
+                // ---------------- O = P V -> normalised bf16 rows: the warp's 32 rows of the staging buffer (4 KB,
+                // swizzled as the output map expects) take 64 columns at a time; one TMA store per half writes 32
+                // full rows
+                const uint64_t pol = l2_policy_evict_first();
+                uint8_t* wstg = obuf + (warp & 3) * 4096;            // columns 0..63; + kPBytes: columns 64..127
+                for (int ti = 0; ti < nb && ok; ++ti) {
+                    const uint32_t tcv = tcount + ti, sl = tcv & 1u;
+                    ok = mbar_wait(&sm.o_full[sl], (tcv >> 1) & 1);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const int orow0 = sm.tile_meta[tcv % kMetaSlots][3] * kG;
+                    const float zi = sm.zinv[tcv & 3u][row];
 #pragma unroll 1
-                for (int hb = 0; hb < 2; ++hb) {
-                    uint32_t pk[32];
-                    {
-                        float v[64];
-                        tmem_ld64(t_lane + 256 + sl * 128 + hb * 64, v);
+                    for (int hb = 0; hb < 2; ++hb) {
+                        uint32_t pk[32];
+                        {
+                            float v[64];
+                            tmem_ld64(t_lane + 256 + sl * 128 + hb * 64, v);
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) pk[j] = pack_bf16(v[2 * j] * zi, v[2 * j + 1] * zi);
-                    }
-                    if (hb == 1) {
-                        if (lane == 0) bulk_wait_read<0>();
-                        __syncwarp();
-                    }
+                            for (int j = 0; j < 32; ++j) pk[j] = pack_bf16(v[2 * j] * zi, v[2 * j + 1] * zi);
+                        }
+                        if (hb == 0) {
+                            // the previous tile's stores (lane 0: columns 0..63, lane 1: 64..127) must have read the staging rows
+                            if (lane < 2) bulk_wait_read<0>();
+                            __syncwarp();
+                        } else {
+                            // the accumulator (and the ring slot of 1 / row sum) is free for the slot's next tile
+                            tc_fence_before_sync();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(&sm.o_empty[sl]);
+                        }
 #pragma unroll
-                    for (int pc = 0; pc < 8; ++pc)
-                        *reinterpret_cast<uint4*>(pslot + swz128(row, pc)) = make_uint4(pk[4 * pc], pk[4 * pc + 1], pk[4 * pc + 2], pk[4 * pc + 3]);
+                        for (int pc = 0; pc < 8; ++pc)
+                            *reinterpret_cast<uint4*>(obuf + hb * kPBytes + swz128(row, pc)) = make_uint4(pk[4 * pc], pk[4 * pc + 1], pk[4 * pc + 2], pk[4 * pc + 3]);
+                    }
                     fence_proxy_async_smem();
                     __syncwarp();
-                    if (lane == 0) {
-                        tma_store_2d(&map_o, wstg, hb * 64, orow0 + (warp & 3) * 32, pol);
+                    if (lane < 2) {
+                        tma_store_2d(&map_o, wstg + lane * kPBytes, lane * 64, orow0 + (warp & 3) * 32, pol);
                         bulk_commit();
                     }
                 }
-                tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&sm.o_empty[sl]);
             }
             if (!ok && lane == 0) { set_status(a.status, kDevTimeout); atomicExch(&sm.abort_flag, 1); }
         }
