@@ -37,7 +37,7 @@ from paper_2607_02980_b200 import workloads as wl
 # captures summarised under profiles/.  The decode captures ran a reduced batch (8 of 64 sequences for cfg3, 1 of 4
 # for cfg4); traffic is proportional to the number of (sequence, KV head) pairs and is scaled to the full launch.
 NCU_TRAFFIC_BYTES = {
-    ("cfg1", "prefill_attend"): int((660.4 + 2276.0) * 1e6),   # the one launch that walks all four query blocks
+    ("cfg1", "prefill_attend"): int((654.3 + 2270.9) * 1e6),   # the one launch that walks all four query blocks
     ("cfg3", "decode_attend"): int(70.5e6 * 8),
     ("cfg4", "decode_attend"): int(17.1e6 * 4),
     ("cfg4", "decode_score"): int(33.57e6 * 4),
