@@ -5,10 +5,14 @@
 // tcgen05.mma (M = 128 tokens, N = 64 chunks, K = 128) once per head into tensor memory, double
 // buffered; the four epilogue warps own one token per thread (token = TMEM lane), read the four
 // heads' scores, take the group max (App. C) and keep the token's exact running top-K
-// (Eq. surrogate top-k; equal scores go to the lower chunk id): candidates that beat the current
-// K-th score are appended to a private buffer; when a buffer of the warp fills up, every thread sorts
-// its buffer with a register bitonic network and merges it into its sorted top list, which raises the
-// threshold.  The number of such merges grows with log(candidates / K), not with the candidates.
+// (Eq. surrogate top-k; equal scores go to the lower chunk id).  A token's candidates that beat its current
+// K-th best score are appended, in arrival order = ascending chunk id, to its pool in shared memory; the N best
+// SCORES so far stay sorted in registers.  When a pool of the warp may fill up, every thread sorts the scores
+// appended since the last time (register bitonic network on 32-bit values: one max and one min per
+// compare-exchange), merges them into its sorted list, reads the new K-th best score off it and filters its pool
+// in place: everything above that score and the earliest of those equal to it, exactly K entries, still in
+// ascending chunk order -- which is the order the selection is written in.  The number of such compactions grows
+// with log(candidates / K), not with the candidates.
 #include "internal.h"
 #include "tma.cuh"
 
@@ -46,9 +50,10 @@ struct TcSmem {
     uint32_t tmem_base;
 };
 
-// Sorts N keys in registers, largest first (bitonic network, fully unrolled: static register indices).
+// Sorts N scores in registers, largest first (bitonic network, fully unrolled: static register indices; a
+// compare-exchange is one max and one min).
 template <int N>
-__device__ __forceinline__ void bitonic_sort_desc(unsigned long long (&a)[N]) {
+__device__ __forceinline__ void bitonic_sort_desc(float (&a)[N]) {
     constexpr int kLog = N == 32 ? 5 : 4;
 #pragma unroll
     for (int ks = 1; ks <= kLog; ++ks) {
@@ -61,18 +66,17 @@ __device__ __forceinline__ void bitonic_sort_desc(unsigned long long (&a)[N]) {
                 const int l = i ^ j;
                 if (l > i) {
                     const bool desc = (i & k) == 0;
-                    const unsigned long long x = a[i], y = a[l];
-                    const bool sw = desc ? (x < y) : (x > y);
-                    a[i] = sw ? y : x;
-                    a[l] = sw ? x : y;
+                    const float hi = fmaxf(a[i], a[l]), lo = fminf(a[i], a[l]);
+                    a[i] = desc ? hi : lo;
+                    a[l] = desc ? lo : hi;
                 }
             }
         }
     }
 }
-// Sorts a bitonic sequence of N keys, largest first.
+// Sorts a bitonic sequence of N scores, largest first.
 template <int N>
-__device__ __forceinline__ void bitonic_merge_desc(unsigned long long (&a)[N]) {
+__device__ __forceinline__ void bitonic_merge_desc(float (&a)[N]) {
     constexpr int kLog = N == 32 ? 5 : 4;
 #pragma unroll
     for (int js = kLog - 1; js >= 0; --js) {
@@ -81,45 +85,15 @@ __device__ __forceinline__ void bitonic_merge_desc(unsigned long long (&a)[N]) {
         for (int i = 0; i < N; ++i) {
             const int l = i ^ j;
             if (l > i) {
-                const unsigned long long x = a[i], y = a[l];
-                const bool sw = x < y;
-                a[i] = sw ? y : x;
-                a[l] = sw ? x : y;
+                const float hi = fmaxf(a[i], a[l]), lo = fminf(a[i], a[l]);
+                a[i] = hi;
+                a[l] = lo;
             }
         }
     }
 }
 
-// Merges a thread's append buffer (qn raw (score bits, chunk id) pairs at myq[e * 128]) into its sorted top list
-// (mytop[e * 128], largest first, 0 = empty): exact keys, register bitonic sort of the buffer, the N largest of
-// both lists, sorted again.  Returns the score of the K-th best key (-inf while fewer than K are known).
-// One copy of this code per N (not inlined: it is a few thousand instructions).
-template <int N>
-__device__ __noinline__ float merge_buffer(unsigned long long* mytop, const unsigned long long* myq, int qn, int K) {
-    unsigned long long kb[N];
-#pragma unroll
-    for (int e = 0; e < N; ++e) {
-        const unsigned long long raw = myq[e * kTileTok];
-        const unsigned long long key =
-            select_key(__uint_as_float(static_cast<uint32_t>(raw >> 32)), static_cast<int>(raw & 0xffffffffull));
-        kb[e] = e < qn ? key : 0ull;
-    }
-    bitonic_sort_desc<N>(kb);
-#pragma unroll
-    for (int e = 0; e < N / 2; ++e) {
-        const unsigned long long x = kb[e], y = kb[N - 1 - e];
-        const unsigned long long t0 = mytop[e * kTileTok], t1 = mytop[(N - 1 - e) * kTileTok];
-        kb[e] = t0 > y ? t0 : y;
-        kb[N - 1 - e] = t1 > x ? t1 : x;
-    }
-    bitonic_merge_desc<N>(kb);
-#pragma unroll
-    for (int e = 0; e < N; ++e) mytop[e * kTileTok] = kb[e];
-    const unsigned long long tau = mytop[(K - 1) * kTileTok];
-    return tau ? key_to_float(static_cast<uint32_t>(tau >> 32)) : -INFINITY;
-}
-
-// N = length of the per-token top list and of the append buffer: 16 for K <= 16, else 32.
+// N = length of the per-token sorted score list and room for appended candidates: 16 for K <= 16, else 32.
 // PERHEAD: one landmark row (and bias) per query head (App. C) instead of one per KV head.  A template parameter, not
 // a run-time branch: the scan loop's code has to stay small (the kernel is sensitive to instruction fetch).
 template <int N, bool PERHEAD>
@@ -129,9 +103,8 @@ prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     extern __shared__ uint8_t smem_raw[];
     uint8_t* qs = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* lms = qs + kQBytes;
-    unsigned long long* lists = reinterpret_cast<unsigned long long*>(lms + kLmStages * kLmStageBytes);
-    unsigned long long* queue = lists + kMaxK * kTileTok;
-    TcSmem& sm = *reinterpret_cast<TcSmem*>(queue + kMaxK * kTileTok);
+    unsigned long long* lists = reinterpret_cast<unsigned long long*>(lms + kLmStages * kLmStageBytes);   // [2 kMaxK][128]
+    TcSmem& sm = *reinterpret_cast<TcSmem*>(lists + 2 * kMaxK * kTileTok);
 
     const Shape& s = a.s;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -245,20 +218,18 @@ prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         const int tok = ti * kTileTok + row;
         const int my_ncand = local_lo(s.pos0 + tok, s.W, kS) / kS;
         const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
-        unsigned long long* mytop = lists + tid;           // sorted top list: entry e at mytop[e * 128], 0 = empty
-        unsigned long long* myq = queue + tid;             // append buffer of raw (score bits, chunk id) pairs
+        // The token's pool of raw (score bits, chunk id) pairs in arrival order = ascending chunk id: entry e at
+        // pool[e * 128]; the first `kept` entries survived the last compaction (at most K), the rest were appended
+        // since (at most N).
+        unsigned long long* pool = lists + tid;
         // bias rows of this KV head's landmark heads (per = 1: one row, shared by the four query heads)
         const float* bias = a.bias ? a.bias + (static_cast<long long>(b) * s.Hl + gk * per) * s.C : nullptr;
-        float tau_f = -INFINITY;           // score of the K-th best key so far: the filter of the scan
-        int qn = 0;
-        bool ok = true;
+        float tau_f = -INFINITY;           // score of the K-th best candidate so far: the filter of the scan
+        float best[N];                     // the N best scores so far, largest first (-inf = none)
 #pragma unroll
-        for (int e = 0; e < N; ++e) mytop[e * kTileTok] = 0ull;
-
-        auto compact = [&]() {
-            tau_f = merge_buffer<N>(mytop, myq, qn, K);
-            qn = 0;
-        };
+        for (int e = 0; e < N; ++e) best[e] = -INFINITY;
+        int cnt = 0, kept = 0;
+        bool ok = true;
 
         for (int it = 0; it < nsteps && ok; ++it) {
             const int buf = it & 1;
@@ -273,12 +244,13 @@ prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 const uint32_t col = t_lane + buf * 256 + cb * 8;
                 tmem_ld8x4(col, col + kS, col + 2 * kS, col + 3 * kS, r);
                 const int c0 = it * kS + cb * 8;
-                // first filter on the score alone (ties pass and are settled on the full key when merging);
-                // branch-free append: the slot is written always and kept only when the candidate passes
+                // Filter on the score: a candidate that only EQUALS the K-th best score so far loses to the K
+                // candidates at or above it, which all have lower chunk ids.  Branch-free append: the slot is
+                // written always and kept only when the candidate passes.
                 auto offer = [&](float u, int c) {
-                    const bool pass = u >= tau_f && (!tail || c < my_ncand);
-                    myq[qn * kTileTok] = (static_cast<unsigned long long>(__float_as_uint(u)) << 32) | static_cast<uint32_t>(c);
-                    qn += pass ? 1 : 0;
+                    const bool pass = u > tau_f && (!tail || c < my_ncand);
+                    pool[cnt * kTileTok] = (static_cast<unsigned long long>(__float_as_uint(u)) << 32) | static_cast<uint32_t>(c);
+                    cnt += pass ? 1 : 0;
                 };
                 if (PERHEAD && bias != nullptr) {
                     // every head adds its own bias before the maximum over the group (App. C)
@@ -286,7 +258,7 @@ prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                     for (int j = 0; j < 8; ++j) {
                         const int c = c0 + j, cc = min(c, s.C - 1);
                         offer(fmaxf(fmaxf(fmaf(r[0][j], s.scale, bias[cc]), fmaf(r[1][j], s.scale, bias[s.C + cc])),
-                                    fmaxf(fmaf(r[2][j], s.scale, bias[2 * s.C + cc]), fmaf(r[3][j], s.scale, bias[3 * s.C + cc]))),
+                                    fmaxf(fmaf(r[2][j], s.scale, bias[2 * s.C + cc]), fmaf(r[3][j], s.scale, bias[3 * s.C + cc]))) + 0.0f,
                               c);
                     }
                 } else {
@@ -295,31 +267,63 @@ prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                         const int c = c0 + j;
                         float u = fmaxf(fmaxf(r[0][j], r[1][j]), fmaxf(r[2][j], r[3][j])) * s.scale;
                         if (bias) u += bias[min(c, s.C - 1)];
-                        offer(u, c);
+                        offer(u + 0.0f, c);                    // -0 folds into +0: scores compare as numbers
                     }
                 }
-                // at most 8 appends between checks: a buffer never overflows
-                if (__any_sync(kFullMask, qn > N - 8)) compact();
+                // Compaction (one call site: the code is large): when a row of the warp may overflow on the next
+                // round (at most 8 appends between checks), and once after the last round.
+                const bool last_round = it + 1 == nsteps && cb == 7;
+                if (__any_sync(kFullMask, cnt - kept > N - 8) || last_round) {
+                    // the N best scores of (best so far) + (appended since): sort the new ones, take the larger of
+                    // the i-th best old and the i-th worst new, sort that bitonic sequence
+                    float nw[N];
+#pragma unroll
+                    for (int e = 0; e < N; ++e) {
+                        const unsigned long long raw = pool[(kept + e) * kTileTok];
+                        nw[e] = kept + e < cnt ? __uint_as_float(static_cast<uint32_t>(raw >> 32)) : -INFINITY;
+                    }
+                    bitonic_sort_desc<N>(nw);
+#pragma unroll
+                    for (int e = 0; e < N; ++e) best[e] = fmaxf(best[e], nw[N - 1 - e]);
+                    bitonic_merge_desc<N>(best);
+                    // the K-th best = the smallest of the first K (written so that the list stays in registers:
+                    // picking entry K - 1 would index it dynamically)
+                    float tau = INFINITY;
+#pragma unroll
+                    for (int e = 0; e < N; ++e) tau = fminf(tau, e < K ? best[e] : INFINITY);
+                    if (tau > -INFINITY) {
+                        // exactly K survive: every score above tau, and the earliest of those equal to it
+                        int above = 0;
+#pragma unroll
+                        for (int e = 0; e < N; ++e) above += (e < K && best[e] > tau) ? 1 : 0;
+                        int ties = K - above, w = 0;
+#pragma unroll 4
+                        for (int e = 0; e < cnt; ++e) {
+                            const unsigned long long raw = pool[e * kTileTok];
+                            const float sc = __uint_as_float(static_cast<uint32_t>(raw >> 32));
+                            const bool tie = sc == tau && ties > 0;
+                            const bool keep = sc > tau || tie;
+                            ties -= tie ? 1 : 0;
+                            pool[w * kTileTok] = raw;          // w <= e: in place, order preserved
+                            w += keep ? 1 : 0;
+                        }
+                        cnt = w;
+                    }
+                    kept = cnt;
+                    tau_f = tau;
+                }
             }
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm.tmem_empty[buf]);
         }
         if (!ok && lane == 0) set_status(a.status, kDevTimeout);
-        compact();
 
-        // the first K entries of the top list (0 = none), emitted as ascending chunk ids, -1 padded
+        // the survivors are the selection, already in ascending chunk order; -1 padded
         if (tok < s.R) {
             int32_t* sel = a.sel + (static_cast<long long>(pair) * s.R + tok) * K;
-            int cnt = 0;
-            for (int e = 0; e < K; ++e) cnt += mytop[e * kTileTok] != 0ull ? 1 : 0;
-            for (int e = 0; e < cnt; ++e) {
-                const int id = key_chunk(mytop[e * kTileTok]);
-                int rank = 0;
-                for (int j = 0; j < cnt; ++j) rank += key_chunk(mytop[j * kTileTok]) < id ? 1 : 0;
-                sel[rank] = id;
-            }
-            for (int e = cnt; e < K; ++e) sel[e] = -1;
+            for (int e = 0; e < K; ++e)
+                sel[e] = e < cnt ? static_cast<int32_t>(pool[e * kTileTok] & 0xffffffffull) : -1;
         }
         if (a.cnt) {
             // chunk histogram of this tile's entries (selected chunks + the chunks of each token's local window) in the
@@ -334,10 +338,7 @@ prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             }
             if (tok < s.R) {
                 int* dst = in_smem ? hist : gcnt;
-                for (int e = 0; e < K; ++e) {
-                    const unsigned long long key = mytop[e * kTileTok];
-                    if (key != 0ull) atomicAdd(dst + key_chunk(key), 1);
-                }
+                for (int e = 0; e < cnt; ++e) atomicAdd(dst + static_cast<int>(pool[e * kTileTok] & 0xffffffffull), 1);
                 const int pos = s.pos0 + tok;
                 for (int c = local_lo(pos, s.W, kS) / kS; c <= pos / kS; ++c) atomicAdd(dst + c, 1);
             }

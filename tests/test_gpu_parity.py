@@ -135,6 +135,32 @@ def test_prefill_ties_go_to_lower_chunk_and_runs_are_deterministic():
     assert (a[0].float() - b[0].float()).abs().max() <= 1e-2
 
 
+@pytest.mark.parametrize("K", [8, 24])
+def test_prefill_two_level_scores_cut_through_the_crowded_level(K):
+    """Two-valued group scores in prefill: a few chunks on the upper level, every other chunk tied on the lower
+    one, so the exact tie rule (lower chunk id) decides most of the selection, for tokens early and late in a
+    long sequence (the late ones go through several compactions of the running top-K)."""
+    cfg = wl.CONFIGS[1].scaled(Hq=8, Hkv=2, L=8192, K=K, seed=34, n_needles=0)
+    inp = wl.make_prefill_inputs(cfg, "cpu")
+    upper = [5 + 9 * j for j in range(6)]                       # chunks 5, 14, ..., 50
+    lm = torch.zeros_like(inp["landmarks"])
+    lm[:, :, upper, 0] = 4.0
+    q = torch.zeros_like(inp["q"])
+    q[..., 0] = 4.0
+    case = dict(inp, landmarks=lm, q=q)
+    for impl in ("generic", "auto"):
+        _, _, sel = run_prefill(cfg, case, impl)
+        got = sel.cpu().numpy()
+        for i in (63, 64 * 4 + 1, 64 * 30, 64 * 51 + 7, 64 * 100, 8191):
+            ncand = i // cfg.S                                  # W = 1: the chunks before the token's own
+            hi = [c for c in upper if c < ncand]
+            lo = [c for c in range(ncand) if c not in upper]
+            exp = sorted(hi[:K] + lo[:max(0, K - len(hi))])
+            exp = exp + [-1] * (K - len(exp))
+            for g in range(cfg.Hkv):
+                assert got[0, g, i].tolist() == exp, (impl, K, i, g)
+
+
 DECODE_SMALL = {
     "bf16_ragged": (wl.CONFIGS[3].scaled(B=6, L=4096, K=8, seed=41), [4096, 4095, 1, 63, 2049, 640]),
     "bf16_k_ge_chunks": (wl.CONFIGS[3].scaled(B=3, L=2048, K=64, seed=42), [2048, 1000, 65]),
