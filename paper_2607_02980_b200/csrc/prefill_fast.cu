@@ -441,6 +441,16 @@ __global__ void __launch_bounds__(kFuseWarps * 32) prefill_fuse_kernel(const PAr
         }
         lam[st][0] = v.x; lam[st][1] = v.y; lam[st][2] = v.z; lam[st][3] = v.w;
     }
+    // the first four rows are requested before the weights are worked out (their addresses need only the entries)
+    __syncwarp();
+    uint4 ra[4], rb[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        const int r = min(u, nrows - 1);
+        const __nv_bfloat16* row = a.obuf + static_cast<long long>(ev[r]) * kG * kD;
+        ra[u] = obuf_load(reinterpret_cast<const uint4*>(row + lane * 8));
+        rb[u] = obuf_load(reinterpret_cast<const uint4*>(row + 256 + lane * 8));
+    }
     float lse_h = 0.f;
 #pragma unroll
     for (int h = 0; h < kG; ++h) {
@@ -470,13 +480,14 @@ __global__ void __launch_bounds__(kFuseWarps * 32) prefill_fuse_kernel(const PAr
     };
     // four rows at a time (8 loads in flight per lane)
     for (int r0 = 0; r0 < nrows; r0 += 4) {
-        uint4 ra[4], rb[4];
+        if (r0 > 0) {
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int r = min(r0 + u, nrows - 1);
-            const __nv_bfloat16* row = a.obuf + static_cast<long long>(ev[r]) * kG * kD;
-            ra[u] = obuf_load(reinterpret_cast<const uint4*>(row + lane * 8));
-            rb[u] = obuf_load(reinterpret_cast<const uint4*>(row + 256 + lane * 8));
+            for (int u = 0; u < 4; ++u) {
+                const int r = min(r0 + u, nrows - 1);
+                const __nv_bfloat16* row = a.obuf + static_cast<long long>(ev[r]) * kG * kD;
+                ra[u] = obuf_load(reinterpret_cast<const uint4*>(row + lane * 8));
+                rb[u] = obuf_load(reinterpret_cast<const uint4*>(row + 256 + lane * 8));
+            }
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
