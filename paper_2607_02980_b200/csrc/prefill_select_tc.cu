@@ -27,6 +27,7 @@ constexpr int kLmStages = 2;
 constexpr int kLmStageBytes = kS * kD * 2;          // 64 landmark rows = two 8 KB K-blocks
 constexpr int kQBytes = kG * kTileTok * kD * 2;     // 128 KB
 constexpr int kMaxK = 32;
+constexpr int kRoom = 32;                           // candidates a pool takes between two compactions
 constexpr int kThreads = 192;                       // 4 epilogue warps, 1 TMA warp, 1 MMA warp
 constexpr uint32_t kTmemCols = 512;                 // 2 buffers x 4 heads x 64 columns
 
@@ -93,7 +94,8 @@ __device__ __forceinline__ void bitonic_merge_desc(float (&a)[N]) {
     }
 }
 
-// N = length of the per-token sorted score list and room for appended candidates: 16 for K <= 16, else 32.
+// N = length of the per-token sorted score list: 16 for K <= 16, else 32; a pool has room for kRoom = 32 candidates
+// appended between two compactions (fewer, larger compactions are cheaper than more, smaller ones).
 // PERHEAD: one landmark row (and bias) per query head (App. C) instead of one per KV head.  A template parameter, not
 // a run-time branch: the scan loop's code has to stay small (the kernel is sensitive to instruction fetch).
 template <int N, bool PERHEAD>
@@ -220,7 +222,7 @@ prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
         const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
         // The token's pool of raw (score bits, chunk id) pairs in arrival order = ascending chunk id: entry e at
         // pool[e * 128]; the first `kept` entries survived the last compaction (at most K), the rest were appended
-        // since (at most N).
+        // since (at most kRoom).
         unsigned long long* pool = lists + tid;
         // bias rows of this KV head's landmark heads (per = 1: one row, shared by the four query heads)
         const float* bias = a.bias ? a.bias + (static_cast<long long>(b) * s.Hl + gk * per) * s.C : nullptr;
@@ -273,16 +275,16 @@ prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 // Compaction (one call site: the code is large): when a row of the warp may overflow on the next
                 // round (at most 8 appends between checks), and once after the last round.
                 const bool last_round = it + 1 == nsteps && cb == 7;
-                if (__any_sync(kFullMask, cnt - kept > N - 8) || last_round) {
+                if (__any_sync(kFullMask, cnt - kept > kRoom - 8) || last_round) {
                     // the N best scores of (best so far) + (appended since): sort the new ones, take the larger of
                     // the i-th best old and the i-th worst new, sort that bitonic sequence
-                    float nw[N];
+                    float nw[kRoom];
 #pragma unroll
-                    for (int e = 0; e < N; ++e) {
+                    for (int e = 0; e < kRoom; ++e) {
                         const unsigned long long raw = pool[(kept + e) * kTileTok];
                         nw[e] = kept + e < cnt ? __uint_as_float(static_cast<uint32_t>(raw >> 32)) : -INFINITY;
                     }
-                    bitonic_sort_desc<N>(nw);
+                    bitonic_sort_desc<kRoom>(nw);
 #pragma unroll
                     for (int e = 0; e < N; ++e) best[e] = fmaxf(best[e], nw[N - 1 - e]);
                     bitonic_merge_desc<N>(best);
