@@ -425,12 +425,12 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                     const int il = e >> 8, slot = e & 255;
                     const bool local = slot >= s.K;                            // a chunk of the local window: mass = its exact log-sum-exp
                     const int lim = local ? s.pos0 + i0 + il - c * kS : kS - 1;   // last visible key of the chunk
+                    // the 64 key scores and the surrogate score columns: the landmark of this row's head (key 64 + hd)
+                    // or the shared one (key 64); warp-uniform addresses, the lane picks its column
                     float v[64];
-                    tmem_ld64(t_lane + sl * 128, v);
-                    // surrogate score column: the landmark of this row's head (key 64 + hd) or the shared one (key 64)
                     const int lh = (s.Hl == s.Hkv) ? 0 : hd;
                     float lm4[4];
-                    tmem_ld4(t_lane + sl * 128 + 64, lm4);           // warp-uniform address; the lane picks its column
+                    tmem_ld64_4(t_lane + sl * 128, t_lane + sl * 128 + 64, v, lm4);
                     const float lmk = lh == 0 ? lm4[0] : (lh == 1 ? lm4[1] : (lh == 2 ? lm4[2] : lm4[3]));
                     tc_fence_before_sync();
                     __syncwarp();
