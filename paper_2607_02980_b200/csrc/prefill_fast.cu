@@ -338,24 +338,37 @@ __global__ void __launch_bounds__(1024) invert_scan_kernel(const PArgs a) {
     }
 }
 
+// A warp takes one slot of 32 consecutive tokens: neighbouring tokens mostly hold the same chunk in a slot (the
+// local window's chunks always, the selected ones whenever adjacent queries agree), so the lanes that target the
+// same list are served by ONE add on its cursor: the lowest such lane reserves room for all of them.
 __global__ void invert_fill_kernel(const PArgs a) {
     pdl_wait();
     const Shape& s = a.s;
     const int K1 = s.K + max_local_slots(s.W), pairs = s.B * s.Hkv;
-    const long long total = static_cast<long long>(pairs) * s.R * K1;
-    for (long long x = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; x < total;
-         x += static_cast<long long>(gridDim.x) * blockDim.x) {
-        const int slot = static_cast<int>(x % K1);
-        const int tok = static_cast<int>((x / K1) % s.R);
-        const int pair = static_cast<int>(x / (static_cast<long long>(K1) * s.R));
-        const int c = slot_chunk(a, pair, tok, slot);
-        int pos = -1;
-        if (c >= 0) {
-            const long long idx = (static_cast<long long>(tok / a.qb) * pairs + pair) * a.nc + c;
-            pos = a.off[idx] + atomicAdd(&a.cursor[idx], 1);
-            if (pos < a.max_tiles * a.tile_tok) a.entries[pos] = ((tok % a.qb) << 8) | slot;
+    const int lane = threadIdx.x & 31;
+    const int tblocks = (s.R + 31) / 32;
+    const long long total = static_cast<long long>(pairs) * tblocks * K1;
+    const long long nwarps = static_cast<long long>(gridDim.x) * (blockDim.x >> 5);
+    for (long long w = static_cast<long long>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5); w < total; w += nwarps) {
+        const int slot = static_cast<int>(w % K1);
+        const int tb = static_cast<int>((w / K1) % tblocks);
+        const int pair = static_cast<int>(w / (static_cast<long long>(K1) * tblocks));
+        const int tok = tb * 32 + lane;
+        const int c = tok < s.R ? slot_chunk(a, pair, tok, slot) : -1;
+        const long long idx = c >= 0 ? (static_cast<long long>(tok / a.qb) * pairs + pair) * a.nc + c : -1 - lane;
+        const unsigned same = __match_any_sync(kFullMask, idx);
+        const int leader = __ffs(same) - 1;
+        int base = 0;
+        if (c >= 0 && lane == leader) base = a.off[idx] + atomicAdd(&a.cursor[idx], __popc(same));
+        base = __shfl_sync(kFullMask, base, leader);
+        if (tok < s.R) {
+            int pos = -1;
+            if (c >= 0) {
+                pos = base + __popc(same & ((1u << lane) - 1u));
+                if (pos < a.max_tiles * a.tile_tok) a.entries[pos] = ((tok % a.qb) << 8) | slot;
+            }
+            a.epos[(static_cast<long long>(pair) * s.R + tok) * K1 + slot] = pos;
         }
-        a.epos[x] = pos;
     }
 }
 
