@@ -1,6 +1,7 @@
 // Landmark scoring + exact top-K for prefill on the 5th-generation tensor cores (tcgen05 + TMEM).
 //
-// One CTA per (sequence, KV head, 128-token tile).  The tile's queries (4 heads x 128 tokens x 128 d)
+// One persistent CTA per SM walks (sequence, KV head, 128-token tile) triples, heavy tiles first; the next tile's
+// queries and first scores are fetched and computed while the epilogue finishes the previous tile.  The tile's queries (4 heads x 128 tokens x 128 d)
 // stay in shared memory; landmark tiles of 64 chunks stream through a TMA ring.  One thread issues
 // tcgen05.mma (M = 128 tokens, N = 64 chunks, K = 128) once per head into tensor memory, double
 // buffered; the four epilogue warps own one token per thread (token = TMEM lane), read the four
@@ -43,12 +44,14 @@ struct TcArgs {
 };
 
 struct TcSmem {
+    uint64_t q_empty;          // every MMA of the tile has completed: its query tile may be overwritten
     uint64_t q_full;
     uint64_t full[kLmStages];
     uint64_t empty[kLmStages];
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
     uint32_t tmem_base;
+    int abort;                 // a bounded wait of an epilogue thread ran out: every epilogue warp leaves after the tile
 };
 
 // Sorts N scores in registers, largest first (bitonic network, fully unrolled: static register indices; a
@@ -112,18 +115,25 @@ prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int pairs = s.B * s.Hkv;
     const int tiles_per_seq = (s.R + kTileTok - 1) / kTileTok;
-    const int ti = tiles_per_seq - 1 - static_cast<int>(blockIdx.x) / pairs;     // heavy tiles first
-    const int pair = static_cast<int>(blockIdx.x) % pairs;
-    const int b = pair / s.Hkv, gk = pair % s.Hkv;
-    // candidates of a token = the chunks left of its local window (Sec. 2.1); the tile's last token has the most
-    const int last_tok = min(s.R, (ti + 1) * kTileTok) - 1;
-    const int ncand_max = local_lo(s.pos0 + last_tok, s.W, kS) / kS;
-    const int nsteps = (ncand_max + kS - 1) / kS;
+    const int n_tiles = pairs * tiles_per_seq;
     const int K = s.K;
     constexpr int per = PERHEAD ? kG : 1;     // landmark rows per chunk
+    // A CTA walks the tiles blockIdx.x, blockIdx.x + gridDim.x, ... (heavy tiles first): the query tile and the first
+    // scores of the next tile are fetched and computed while the epilogue still finishes the previous one.  Every
+    // role derives the same tile sequence; tiles without candidates touch no barrier.
+    auto tile_of = [&](int idx, int& ti, int& pair, int& nsteps) {
+        ti = tiles_per_seq - 1 - idx / pairs;
+        pair = idx % pairs;
+        // candidates of a token = the chunks left of its local window (Sec. 2.1); the tile's last token has the most
+        const int last_tok = min(s.R, (ti + 1) * kTileTok) - 1;
+        const int ncand_max = local_lo(s.pos0 + last_tok, s.W, kS) / kS;
+        nsteps = (ncand_max + kS - 1) / kS;
+    };
 
     if (tid == 0) {
         mbar_init(&sm.q_full, 1);
+        mbar_init(&sm.q_empty, 1);
+        sm.abort = 0;
         for (int i = 0; i < kLmStages; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(&sm.tmem_full[i], 1); mbar_init(&sm.tmem_empty[i], 4); }
         mbar_fence_init();
@@ -138,40 +148,48 @@ prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 
     if (warp == 4) {
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0 && nsteps > 0) {
-            mbar_expect_tx(&sm.q_full, kQBytes);
-            for (int h = 0; h < kG; ++h) {
-                const int row = (b * s.Hq + gk * kG + h) * s.R + ti * kTileTok;
-                tma_load_2d(qs + h * 32768, &map_q, &sm.q_full, 0, row);
-                tma_load_2d(qs + h * 32768 + 16384, &map_q, &sm.q_full, 64, row);
-            }
-            // landmark tiles in ring order: step it, landmark head hh (per = 1: one tile per step for all heads;
-            // per = G: one tile per query head, App. C)
-            int issued = 0;
-            const int ntiles = nsteps * per;
-            for (int n = 0; n < ntiles; ++n) {
-                const int st = n % kLmStages, it = n / per, hh = n % per;
-                if (n >= kLmStages && !mbar_wait(&sm.empty[st], ((n / kLmStages) - 1) & 1)) {
-                    set_status(a.status, kDevTimeout);
-                    break;
+        if (lane == 0) {
+            uint32_t n_lm = 0;            // landmark tiles requested so far, over all tiles of this CTA
+            int tn = 0;                   // tiles with candidates so far
+            bool ok = true;
+            for (int idx = blockIdx.x; idx < n_tiles && ok; idx += gridDim.x) {
+                int ti, pair, nsteps;
+                tile_of(idx, ti, pair, nsteps);
+                if (nsteps == 0) continue;
+                const int b = pair / s.Hkv, gk = pair % s.Hkv;
+                if (tn > 0) ok = mbar_wait(&sm.q_empty, (tn - 1) & 1);
+                if (!ok) break;
+                mbar_expect_tx(&sm.q_full, kQBytes);
+                for (int h = 0; h < kG; ++h) {
+                    const int row = (b * s.Hq + gk * kG + h) * s.R + ti * kTileTok;
+                    tma_load_2d(qs + h * 32768, &map_q, &sm.q_full, 0, row);
+                    tma_load_2d(qs + h * 32768 + 16384, &map_q, &sm.q_full, 64, row);
                 }
-                uint8_t* dst = lms + st * kLmStageBytes;
-                const int row = ((b * s.Hl + gk * per + hh)) * s.C + it * kS;
-                mbar_expect_tx(&sm.full[st], kLmStageBytes);
-                tma_load_2d(dst, &map_lm, &sm.full[st], 0, row);
-                tma_load_2d(dst + 8192, &map_lm, &sm.full[st], 64, row);
-                ++issued;
+                // landmark tiles in ring order: step it, landmark head hh (per = 1: one tile per step for all heads;
+                // per = G: one tile per query head, App. C)
+                const int ntiles = nsteps * per;
+                for (int n = 0; n < ntiles && ok; ++n, ++n_lm) {
+                    const int st = n_lm % kLmStages, it = n / per, hh = n % per;
+                    if (n_lm >= kLmStages) ok = mbar_wait(&sm.empty[st], ((n_lm / kLmStages) - 1) & 1);
+                    if (!ok) break;
+                    uint8_t* dst = lms + st * kLmStageBytes;
+                    const int row = ((b * s.Hl + gk * per + hh)) * s.C + it * kS;
+                    mbar_expect_tx(&sm.full[st], kLmStageBytes);
+                    tma_load_2d(dst, &map_lm, &sm.full[st], 0, row);
+                    tma_load_2d(dst + 8192, &map_lm, &sm.full[st], 64, row);
+                }
+                ++tn;
             }
-            // own copies in flight: every issued stage and the query tile must have landed before exit
-            mbar_wait(&sm.q_full, 0);
-            for (int n = max(0, issued - kLmStages); n < issued; ++n)
+            if (!ok) set_status(a.status, kDevTimeout);
+            // own copies in flight: the last query tile and the last stages must have landed before exit
+            if (tn > 0) mbar_wait(&sm.q_full, (tn - 1) & 1);
+            for (uint32_t n = n_lm > kLmStages ? n_lm - kLmStages : 0; n < n_lm; ++n)
                 mbar_wait(&sm.full[n % kLmStages], (n / kLmStages) & 1);
         }
     } else if (warp == 5) {
         // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0 && nsteps > 0) {
+        if (lane == 0) {
             constexpr uint32_t idesc = umma_idesc_bf16(kTileTok, kS);
-            bool ok = mbar_wait(&sm.q_full, 0);
             // S_h = Q_h x landmark tile^T (M = 128 tokens, N = 64 chunks, K = 128) into head h's 64 columns
             auto issue_head = [&](uint32_t d_tmem, uint32_t q_addr, uint32_t lm_addr) {
 #pragma unroll
@@ -182,44 +200,63 @@ prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 }
             };
             const uint32_t q0 = smem_u32(qs);
-            for (int it = 0; it < nsteps && ok; ++it) {
-                const int buf = it & 1;
-                if (it >= 2) ok = mbar_wait(&sm.tmem_empty[buf], ((it >> 1) - 1) & 1);
-                if (!ok) break;
-                if (per == 1) {
-                    // one landmark tile for the four query heads
-                    const int st = it % kLmStages;
-                    ok = mbar_wait(&sm.full[st], (it / kLmStages) & 1);
+            uint32_t n_lm = 0, n_step = 0;     // landmark tiles / steps so far, over all tiles of this CTA
+            int tn = 0;
+            bool ok = true;
+            for (int idx = blockIdx.x; idx < n_tiles && ok; idx += gridDim.x) {
+                int ti, pair, nsteps;
+                tile_of(idx, ti, pair, nsteps);
+                if (nsteps == 0) continue;
+                ok = mbar_wait(&sm.q_full, tn & 1);
+                for (int it = 0; it < nsteps && ok; ++it, ++n_step) {
+                    const uint32_t buf = n_step & 1u;
+                    if (n_step >= 2) ok = mbar_wait(&sm.tmem_empty[buf], ((n_step >> 1) - 1) & 1);
                     if (!ok) break;
-                    tc_fence_after_sync();
-                    const uint32_t lm_addr = smem_u32(lms + st * kLmStageBytes);
+                    if (per == 1) {
+                        // one landmark tile for the four query heads
+                        const uint32_t st = n_lm % kLmStages;
+                        ok = mbar_wait(&sm.full[st], (n_lm / kLmStages) & 1);
+                        if (!ok) break;
+                        tc_fence_after_sync();
+                        const uint32_t lm_addr = smem_u32(lms + st * kLmStageBytes);
 #pragma unroll
-                    for (int h = 0; h < kG; ++h) issue_head(tmem_base + buf * 256 + h * kS, q0 + h * 32768, lm_addr);
-                    umma_commit(&sm.empty[st]);        // landmark stage reusable once these MMAs are done
-                } else {
-                    // one landmark tile per query head (App. C), in ring order
+                        for (int h = 0; h < kG; ++h) issue_head(tmem_base + buf * 256 + h * kS, q0 + h * 32768, lm_addr);
+                        umma_commit(&sm.empty[st]);        // landmark stage reusable once these MMAs are done
+                        ++n_lm;
+                    } else {
+                        // one landmark tile per query head (App. C), in ring order
 #pragma unroll
-                    for (int h = 0; h < kG; ++h) {
-                        const int n = it * kG + h, st = n % kLmStages;
-                        if (ok) ok = mbar_wait(&sm.full[st], (n / kLmStages) & 1);
-                        if (ok) {
-                            tc_fence_after_sync();
-                            issue_head(tmem_base + buf * 256 + h * kS, q0 + h * 32768, smem_u32(lms + st * kLmStageBytes));
-                            umma_commit(&sm.empty[st]);
+                        for (int h = 0; h < kG; ++h) {
+                            const uint32_t st = n_lm % kLmStages;
+                            if (ok) ok = mbar_wait(&sm.full[st], (n_lm / kLmStages) & 1);
+                            if (ok) {
+                                tc_fence_after_sync();
+                                issue_head(tmem_base + buf * 256 + h * kS, q0 + h * 32768, smem_u32(lms + st * kLmStageBytes));
+                                umma_commit(&sm.empty[st]);
+                                ++n_lm;
+                            }
                         }
+                        if (!ok) break;
                     }
-                    if (!ok) break;
+                    umma_commit(&sm.tmem_full[buf]);       // scores of this step readable
                 }
-                umma_commit(&sm.tmem_full[buf]);       // scores of this step readable
+                if (ok) umma_commit(&sm.q_empty);          // the query tile may be replaced once all of these are done
+                ++tn;
             }
             if (!ok) set_status(a.status, kDevTimeout);
         }
     } else {
         // ------------------------------------------------------------------ epilogue: one token per thread
         const int row = warp * 32 + lane;
+        const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
+        uint32_t n_step = 0;               // steps so far, over all tiles of this CTA
+        bool ok = true;
+        for (int idx = blockIdx.x; idx < n_tiles; idx += gridDim.x) {
+        int ti, pair, nsteps;
+        tile_of(idx, ti, pair, nsteps);
+        const int b = pair / s.Hkv, gk = pair % s.Hkv;
         const int tok = ti * kTileTok + row;
         const int my_ncand = local_lo(s.pos0 + tok, s.W, kS) / kS;
-        const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
         // The token's pool of raw (score bits, chunk id) pairs in arrival order = ascending chunk id: entry e at
         // pool[e * 128]; the first `kept` entries survived the last compaction (at most K), the rest were appended
         // since (at most kRoom).
@@ -231,11 +268,10 @@ prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 #pragma unroll
         for (int e = 0; e < N; ++e) best[e] = -INFINITY;
         int cnt = 0, kept = 0;
-        bool ok = true;
 
-        for (int it = 0; it < nsteps && ok; ++it) {
-            const int buf = it & 1;
-            ok = mbar_wait(&sm.tmem_full[buf], (it >> 1) & 1);
+        for (int it = 0; it < nsteps && ok; ++it, ++n_step) {
+            const uint32_t buf = n_step & 1u;
+            ok = mbar_wait(&sm.tmem_full[buf], (n_step >> 1) & 1);
             if (!ok) break;
             tc_fence_after_sync();
             const bool tail = (it + 1) * kS > my_ncand;     // only the last step holds chunks this token may not see
@@ -319,19 +355,24 @@ prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm.tmem_empty[buf]);
         }
-        if (!ok && lane == 0) set_status(a.status, kDevTimeout);
+        // (after a timeout the thread still walks through the tile's barriers; every warp leaves together below)
+        if (!ok) { set_status(a.status, kDevTimeout); *reinterpret_cast<volatile int*>(&sm.abort) = 1; }
 
         // the survivors are the selection, already in ascending chunk order; -1 padded
+        int ids[N];
+#pragma unroll
+        for (int e = 0; e < N; ++e) ids[e] = e < cnt ? static_cast<int>(pool[e * kTileTok] & 0xffffffffull) : -1;
         if (tok < s.R) {
             int32_t* sel = a.sel + (static_cast<long long>(pair) * s.R + tok) * K;
-            for (int e = 0; e < K; ++e)
-                sel[e] = e < cnt ? static_cast<int32_t>(pool[e * kTileTok] & 0xffffffffull) : -1;
+#pragma unroll
+            for (int e = 0; e < N; ++e)
+                if (e < K) sel[e] = ids[e];
         }
         if (a.cnt) {
             // chunk histogram of this tile's entries (selected chunks + the chunks of each token's local window) in the
-            // landmark ring's shared memory (every MMA that read it has completed), then one global add per used bin
-            int* hist = reinterpret_cast<int*>(lms);
-            const bool in_smem = a.nc * static_cast<int>(sizeof(int)) <= kLmStages * kLmStageBytes;
+            // pools' shared memory (every thread holds its ids in registers by now), then one global add per used bin
+            int* hist = reinterpret_cast<int*>(lists);
+            const bool in_smem = a.nc * sizeof(int) <= sizeof(unsigned long long) * 2 * kMaxK * kTileTok;
             int* gcnt = a.cnt + (static_cast<long long>(ti * kTileTok / a.qb) * pairs + pair) * a.nc;
             asm volatile("bar.sync 1, 128;" ::: "memory");
             if (in_smem) {
@@ -340,7 +381,9 @@ prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             }
             if (tok < s.R) {
                 int* dst = in_smem ? hist : gcnt;
-                for (int e = 0; e < cnt; ++e) atomicAdd(dst + static_cast<int>(pool[e * kTileTok] & 0xffffffffull), 1);
+#pragma unroll
+                for (int e = 0; e < N; ++e)
+                    if (ids[e] >= 0) atomicAdd(dst + ids[e], 1);
                 const int pos = s.pos0 + tok;
                 for (int c = local_lo(pos, s.W, kS) / kS; c <= pos / kS; ++c) atomicAdd(dst + c, 1);
             }
@@ -349,6 +392,10 @@ prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
                 for (int x = tid; x < a.nc; x += kTileTok)
                     if (hist[x]) atomicAdd(gcnt + x, hist[x]);
             }
+        }
+        // the pools' memory (histogram) is free for the next tile; after a timeout every warp leaves here
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (*reinterpret_cast<volatile int*>(&sm.abort)) break;
         }
     }
 
@@ -388,7 +435,8 @@ int launch_prefill_select_tc(const Shape& s, const void* q, const void* landmark
     }
     TcArgs a{s, bias, sel, status, (cnt && qb % kTileTok == 0) ? cnt : nullptr, qb, nc};
     const int tiles = (s.R + kTileTok - 1) / kTileTok;
-    const unsigned grid = static_cast<unsigned>(pairs) * tiles;
+    const unsigned all_tiles = static_cast<unsigned>(pairs) * tiles;
+    const unsigned grid = all_tiles < 148u ? all_tiles : 148u;       // one persistent CTA per SM
     const bool perhead = s.Hl != s.Hkv;
     if (s.K <= 16) {
         if (perhead) prefill_select_tc_kernel<16, true><<<grid, kThreads, smem, stream>>>(map_q, map_lm, a);
