@@ -337,7 +337,8 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                 constexpr uint32_t idesc_o = umma_idesc_bf16(kRows, kD) | kUmmaBMnMajor;
                 uint32_t cc = ccount;
                 int cur_pair = -1, cur_c = -1;
-                uint32_t vbuf_of[2] = {0u, 0u};        // V buffer used by the tile in S/P/O slot i
+                uint32_t vbuf_of0 = 0u, vbuf_of1 = 0u;     // V buffer used by the tile in S/P/O slot 0 / 1 (two scalars: an
+                                                           // array indexed by the slot would live in local memory)
                 bool ok = true;
                 // Two in-order queues (S MMAs, O MMAs) served by polling: an O MMA whose probabilities are
                 // ready is never held up by a Q tile that has not arrived yet, and vice versa.
@@ -357,7 +358,7 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                         if (ready) {
                             if (newc) { cur_pair = rec.x; cur_c = rec.y; ++cc; }
                             const uint32_t cb = (cc - 1) & 1u;
-                            vbuf_of[sl] = (cc - 1) % kVBufs;
+                            if (sl) vbuf_of1 = (cc - 1) % kVBufs; else vbuf_of0 = (cc - 1) % kVBufs;
                             tc_fence_after_sync();
                             const uint32_t qa = smem_u32(qbuf + qs * kQBytes), ka = smem_u32(kbuf + cb * kKBytes);
 #pragma unroll
@@ -373,7 +374,7 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                         }
                     }
                     if (no < ns) {
-                        const uint32_t tcv = tcount + no, sl = tcv & 1u, vb = vbuf_of[sl];
+                        const uint32_t tcv = tcount + no, sl = tcv & 1u, vb = sl ? vbuf_of1 : vbuf_of0;
                         bool ready = mbar_test_wait(&sm.p_full[sl], (tcv >> 1) & 1);
                         if (ready && tcv >= 2) ready = mbar_test_wait(&sm.o_empty[sl], ((tcv >> 1) - 1) & 1);
                         if (ready) {
