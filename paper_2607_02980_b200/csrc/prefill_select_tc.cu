@@ -335,15 +335,23 @@ prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
 #pragma unroll
                         for (int e = 0; e < N; ++e) above += (e < K && best[e] > tau) ? 1 : 0;
                         int ties = K - above, w = 0;
-#pragma unroll 4
-                        for (int e = 0; e < cnt; ++e) {
-                            const unsigned long long raw = pool[e * kTileTok];
-                            const float sc = __uint_as_float(static_cast<uint32_t>(raw >> 32));
-                            const bool tie = sc == tau && ties > 0;
-                            const bool keep = sc > tau || tie;
-                            ties -= tie ? 1 : 0;
-                            pool[w * kTileTok] = raw;          // w <= e: in place, order preserved
-                            w += keep ? 1 : 0;
+                        // eight entries per round: their loads go out together (slots past cnt hold old entries or
+                        // nothing that matters: their stores land at or behind w and are overwritten or ignored)
+#pragma unroll 1
+                        for (int e0 = 0; e0 < cnt; e0 += 8) {
+                            unsigned long long raw[8];
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) raw[j] = pool[(e0 + j) * kTileTok];
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                const float sc = __uint_as_float(static_cast<uint32_t>(raw[j] >> 32));
+                                const bool valid = e0 + j < cnt;
+                                const bool tie = valid && sc == tau && ties > 0;
+                                const bool keep = valid && (sc > tau || tie);
+                                ties -= tie ? 1 : 0;
+                                if (valid) pool[w * kTileTok] = raw[j];   // w <= e: in place, order preserved
+                                w += keep ? 1 : 0;
+                            }
                         }
                         cnt = w;
                     }
