@@ -275,38 +275,44 @@ prefill_select_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid
             if (!ok) break;
             tc_fence_after_sync();
             const bool tail = (it + 1) * kS > my_ncand;     // only the last step holds chunks this token may not see
-            // 8 candidates x 4 heads per round: a short loop body (the code has to stay resident close to the core)
+            // 8 candidates per round (a short loop body: the code has to stay resident close to the core); the group
+            // scores of 16 candidates are read from tensor memory and reduced over the heads every other round
+            float u16[16];
 #pragma unroll 1
             for (int cb = 0; cb < 8; ++cb) {
-                float r[4][8];
-                const uint32_t col = t_lane + buf * 256 + cb * 8;
-                tmem_ld8x4(col, col + kS, col + 2 * kS, col + 3 * kS, r);
+                if ((cb & 1) == 0) {
+                    float r[4][16];
+                    const uint32_t col = t_lane + buf * 256 + cb * 8;
+                    tmem_ld16x4(col, col + kS, col + 2 * kS, col + 3 * kS, r);
+                    const int cbase = it * kS + cb * 8;
+                    if (PERHEAD && bias != nullptr) {
+                        // every head adds its own bias before the maximum over the group (App. C)
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const int cc = min(cbase + j, s.C - 1);
+                            u16[j] = fmaxf(fmaxf(fmaf(r[0][j], s.scale, bias[cc]), fmaf(r[1][j], s.scale, bias[s.C + cc])),
+                                           fmaxf(fmaf(r[2][j], s.scale, bias[2 * s.C + cc]), fmaf(r[3][j], s.scale, bias[3 * s.C + cc]))) + 0.0f;
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            float u = fmaxf(fmaxf(r[0][j], r[1][j]), fmaxf(r[2][j], r[3][j])) * s.scale;
+                            if (bias) u += bias[min(cbase + j, s.C - 1)];
+                            u16[j] = u + 0.0f;                 // -0 folds into +0: scores compare as numbers
+                        }
+                    }
+                }
                 const int c0 = it * kS + cb * 8;
                 // Filter on the score: a candidate that only EQUALS the K-th best score so far loses to the K
                 // candidates at or above it, which all have lower chunk ids.  Branch-free append: the slot is
                 // written always and kept only when the candidate passes.
-                auto offer = [&](float u, int c) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float u = (cb & 1) ? u16[8 + j] : u16[j];
+                    const int c = c0 + j;
                     const bool pass = u > tau_f && (!tail || c < my_ncand);
                     pool[cnt * kTileTok] = (static_cast<unsigned long long>(__float_as_uint(u)) << 32) | static_cast<uint32_t>(c);
                     cnt += pass ? 1 : 0;
-                };
-                if (PERHEAD && bias != nullptr) {
-                    // every head adds its own bias before the maximum over the group (App. C)
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const int c = c0 + j, cc = min(c, s.C - 1);
-                        offer(fmaxf(fmaxf(fmaf(r[0][j], s.scale, bias[cc]), fmaf(r[1][j], s.scale, bias[s.C + cc])),
-                                    fmaxf(fmaf(r[2][j], s.scale, bias[2 * s.C + cc]), fmaf(r[3][j], s.scale, bias[3 * s.C + cc]))) + 0.0f,
-                              c);
-                    }
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const int c = c0 + j;
-                        float u = fmaxf(fmaxf(r[0][j], r[1][j]), fmaxf(r[2][j], r[3][j])) * s.scale;
-                        if (bias) u += bias[min(c, s.C - 1)];
-                        offer(u + 0.0f, c);                    // -0 folds into +0: scores compare as numbers
-                    }
                 }
                 // Compaction (one call site: the code is large): when a row of the warp may overflow on the next
                 // round (at most 8 appends between checks), and once after the last round.
