@@ -23,6 +23,19 @@ thread_local Trace g_trace;
 
 }  // namespace
 
+int sm_count() {
+    // per device, looked up once; 148 (B200) where no device answers, e.g. a workspace-size query on a host without a GPU
+    static int cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
 void trace_begin(cudaStream_t stream) {
     Trace& t = g_trace;
     t.n = 0;

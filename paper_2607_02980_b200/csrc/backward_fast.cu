@@ -1034,8 +1034,8 @@ int launch_prefill_backward_fast(const Shape& s, const BackwardTensors& t, cudaS
     for (int blk = 0; blk < ix.n_blocks; ++blk) {
         a.blk_range = ix.blk_toff + blk;
         a.i0 = blk * ix.qb;
-        if (warp_mma) prefill_backward_mma_kernel<<<148, kBfThreads, smem, stream>>>(map_k, map_v, a);
-        else prefill_backward_tc_kernel<<<148, kBfThreads, smem, stream>>>(map_k, map_v, a);
+        if (warp_mma) prefill_backward_mma_kernel<<<sm_count(), kBfThreads, smem, stream>>>(map_k, map_v, a);
+        else prefill_backward_tc_kernel<<<sm_count(), kBfThreads, smem, stream>>>(map_k, map_v, a);
         if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
         trace_mark("backward_attend", stream);
         ++launches;

@@ -791,17 +791,6 @@ struct Plan {
     size_t off_u, off_wgt, off_R, off_E, off_n, off_done, off_part, off_loco, off_loclam, total;
 };
 
-int sm_count() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-            n = 148;
-        if (n <= 0) n = 148;
-    }
-    return n;
-}
-
 Plan make_plan(const Shape& s, int n_sm) {
     Plan p;
     const long long pairs = static_cast<long long>(s.B) * s.Hkv;
@@ -840,11 +829,15 @@ bool decode_fast_supports(const Shape& s, int dtype) {
 
 size_t decode_fast_scratch_bytes(const Shape& s) {
     // sized for the largest CTA count the launcher may use, independent of the device queried at run time
-    return make_plan(s, 148).total > make_plan(s, 1).total ? make_plan(s, 148).total : make_plan(s, 1).total;
+    // the larger of the layouts for this device's SM count, a B200's 148 and a single CTA
+    size_t n = make_plan(s, 148).total;
+    const size_t n1 = make_plan(s, 1).total, nd = make_plan(s, sm_count()).total;
+    n = n1 > n ? n1 : n;
+    return nd > n ? nd : n;
 }
 
 int launch_decode_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
-    const Plan p = make_plan(s, 148);
+    const Plan p = make_plan(s, sm_count());
     if (t.scratch_bytes < p.total) return HILS_ERR_WORKSPACE;
     const int pairs = s.B * s.Hkv;
     char* sc = static_cast<char*>(t.scratch);

@@ -42,6 +42,9 @@ struct PerDeviceOnce {
     void done() { const int d = device(); if (d >= 0) set[d] = true; }
 };
 
+// Streaming multiprocessors of the current device: the grid of every persistent kernel (one CTA per SM).
+int sm_count();
+
 // Optional per-kernel timing: when tracing is on (hils_trace_enable), every launcher calls
 // trace_mark(name) after each kernel it enqueues; an event is recorded on the stream so that the
 // time between consecutive marks is that kernel's device time.  Off by default (no events).

@@ -138,7 +138,7 @@ int launch_chunk_overlap(int pairs, int R, int K, int C, int M, const int32_t* s
     int wpc = static_cast<int>(kOvSmemBudget / per_warp);
     wpc = wpc < 1 ? 1 : (wpc > kOvMaxWarps ? kOvMaxWarps : wpc);
     // enough runs for 32 warps per SM; a run never shorter than 8 blocks (each run re-reads one block to start)
-    const int want_runs = (148 * 32 + pairs - 1) / pairs;
+    const int want_runs = (sm_count() * 32 + pairs - 1) / pairs;
     int per = (a.nblk + want_runs - 1) / want_runs;
     if (per < 8) per = 8;
     a.blocks_per_run = per;

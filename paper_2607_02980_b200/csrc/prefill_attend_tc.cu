@@ -3,19 +3,21 @@
 // A tile is 32 (token, slot) entries of one chunk x 4 heads = 128 query rows (one TMEM lane each).
 // Per tile:  S = Q K_c^T (M=128, N=80: 64 keys + the chunk's landmark as key 64, K=128) -> tensor memory;
 //            each softmax thread owns one row: mask (local rows are causal), the chunk's own softmax
-//            (Eq. HiLS weights, intra-chunk factor), P as bf16 pairs into tensor memory (32 columns behind the
-//            slot's scores: shared memory carries neither the write nor the read of P);
+//            (Eq. HiLS weights, intra-chunk factor), normalised P as bf16 pairs into tensor memory (32 columns behind
+//            the slot's scores: shared memory carries neither the write nor the read of P);
 //            O = P V_c (M=128, N=128, K=64; A = P from tensor memory, V read from shared memory as an MN-major
 //            operand exactly as TMA wrote it) -> tensor memory;
-//            normalised bf16 rows and the row's chunk mass (surrogate score, or log Z_swa for the
+//            bf16 rows and the row's chunk mass (surrogate score, or log Z_swa for the
 //            local branch) go to the buffers that prefill_fuse mixes, in entry order: a tile's 128 rows
 //            are contiguous there, so every output warp hands its 32 rows to one TMA store per half.
-// Warp roles: 0-3 softmax of every tile, 4-7 output of every tile (a warp reads the TMEM lane quarter warp % 4; the
-// softmax of a tile never waits for the tile's own P V, and 1 / row sum passes through a small ring in shared
-// memory), 8-11 producers (cp.async gather of Q rows, TMA of K/V), 12 MMA issue.
+// Warp roles: 0-3 and 4-7 two softmax groups (tiles alternate between them; a warp reads the TMEM lane quarter
+// warp % 4), 8-11 output group, 12-15 query gather, 16 K/V loader, 17 MMA issue.
+// The gather: a warp's cp.async requests complete at the latency of a loaded L2 and a warp keeps only so many in
+// flight, so the rate grows with the number of gathering warps (measured alone: 1 warp 1500 cycles per 32 KB tile, 2
+// warps 840, 4 and more 480; inside this kernel about three times that).  TMA boxes of one entry (512 B) cost about
+// 86 cycles each and 1-D bulk copies of one row 54: both slower.  More than four gather warps need per-group register
+// budgets (setmaxnreg), which measured slower (1.08 ms against 0.73 ms on the 16K-token benchmark shape).
 // S/P/O are double buffered, three gathered Q tiles are in flight, K tiles are double and V tiles triple buffered.
-// What bounds the kernel is the shared-memory port: the MMA operands (Q 32 KB + K 20 KB + V 16 KB per tile), the
-// gathered Q rows (32 KB) and the output staging (32 KB in, 32 KB out) all pass through it.
 #include "internal.h"
 #include "tma.cuh"
 
@@ -36,12 +38,14 @@ constexpr int kPCol = 96;                       // probabilities (bf16 pairs, 32
 constexpr int kBatch = 128;                     // tile records cached per batch
 constexpr int kQSlots = 3;                      // gathered Q tiles in flight
 constexpr int kVBufs = 3;                       // V tiles in flight (K: 2)
-constexpr int kMetaSlots = 8;                   // ring of tile descriptors (producers are < 8 tiles ahead of the epilogue)
-constexpr int kProdThreads = 128;
-constexpr int kEpiThreads = 256;                // a softmax group and an output group of 128 threads
-constexpr int kThreads = kEpiThreads + kProdThreads + 32;
-constexpr int kProdWarp0 = kEpiThreads / 32;
-constexpr int kMmaWarp = kProdWarp0 + kProdThreads / 32;
+constexpr int kMetaSlots = 8;                   // ring of tile descriptors (the loader is < 8 tiles ahead of the output group)
+constexpr int kSoftThreads = 256;               // two softmax groups of 128 threads
+constexpr int kOutWarp0 = kSoftThreads / 32;    // 8
+constexpr int kGatherWarps = 4;
+constexpr int kGatherWarp0 = kOutWarp0 + 4;     // 12 .. 15
+constexpr int kLoadWarp = kGatherWarp0 + kGatherWarps;   // 16
+constexpr int kMmaWarp = kLoadWarp + 1;         // 17
+constexpr int kThreads = (kMmaWarp + 1) * 32;   // 576
 constexpr float kLog2e = 1.4426950408889634f;
 
 struct AtcSmem {
@@ -51,20 +55,18 @@ struct AtcSmem {
     uint64_t v_ready[kVBufs]; // V tile landed
     uint64_t k_empty[2];      // every S MMA that reads this K buffer has completed
     uint64_t v_empty[kVBufs]; // every P V MMA that reads this V buffer has completed
-    uint64_t q_full[kQSlots]; // gathered Q rows landed and fenced (one arrival per producer warp)
+    uint64_t q_full[kQSlots]; // gathered Q rows landed (TMA bytes)
     uint64_t q_empty[kQSlots];// the S MMA that reads this Q tile has completed
     uint64_t s_full[2];       // S = Q K^T in tensor memory
-    uint64_t s_empty[2];      // epilogue has read S
+    uint64_t s_empty[2];      // the slot's softmax group has read S
     uint64_t p_full[2];       // P written to tensor memory
     uint64_t o_full[2];       // O = P V in tensor memory
-    uint64_t o_empty[2];      // epilogue has read O
+    uint64_t o_empty[2];      // the output group has read O
     uint32_t tmem_base;
     int abort_flag;
     int tile_ent[kMetaSlots][kTok];   // entries of the tiles in flight
     int tile_meta[kMetaSlots][4];     // pair, chunk, tokens, first entry relative to the query block
-    const __nv_bfloat16* rowptr[2][kRows];
     int4 recs[kBatch];
-    float zinv[4][kRows];             // 1 / row sum of the tiles in flight (softmax group -> output group)
     int nchunks;                      // distinct (pair, chunk) runs in the current batch
     uint8_t cfirst[kBatch + 4];       // first tile (batch index) of each run; cfirst[nchunks] = tiles in the batch
 };
@@ -97,7 +99,6 @@ __device__ __forceinline__ float ex2_approx(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-__device__ __forceinline__ void producer_barrier() { asm volatile("bar.sync 2, %0;" ::"n"(kProdThreads) : "memory"); }
 
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
@@ -106,14 +107,14 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
     uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* kbuf = base;                                   // [2][kKBytes]
     uint8_t* vbuf = kbuf + 2 * kKBytes;                     // [kVBufs][kVBytes]
-    uint8_t* qbuf = vbuf + kVBufs * kVBytes;                     // [kQSlots][kQBytes]
+    uint8_t* qbuf = vbuf + kVBufs * kVBytes;                // [kQSlots][kQBytes]
     uint8_t* obuf = qbuf + kQSlots * kQBytes;               // [2][kPBytes]: staging of the output rows being stored
     AtcSmem& sm = *reinterpret_cast<AtcSmem*>(obuf + 2 * kPBytes);
 
     const Shape& s = a.s;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
-        for (int i = 0; i < kQSlots; ++i) { mbar_init(&sm.q_full[i], 4); mbar_init(&sm.q_empty[i], 1); }
+        for (int i = 0; i < kQSlots; ++i) { mbar_init(&sm.q_full[i], kGatherWarps); mbar_init(&sm.q_empty[i], 1); }
         for (int i = 0; i < kVBufs; ++i) { mbar_init(&sm.v_ready[i], 1); mbar_init(&sm.v_empty[i], 1); }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&sm.k_ready[i], 2);           // the TMA issuer's arrive.expect_tx + the landmark writer
@@ -146,165 +147,90 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
     // previous kernel of the stream (the fusion of the previous query block, which still reads the partial outputs
     // this kernel overwrites, or the inverse-index kernels).  From here on their results are needed.
     pdl_wait();
-    // running counters (identical in every role): tiles and chunk loads processed so far by this CTA
-    uint32_t tcount = 0, ccount = 0;
 
-    // a.n_tiles[blk], a.n_tiles[blk + 1]: first tile of query block blk and of the next one.  A launch that walks
-    // several blocks takes them in order, so that the CTAs stay on the same block (its gathered Q rows stay in L2).
-    for (int blk = 0; blk < a.n_run; ++blk) {
-    const int t_begin = a.n_tiles[blk], n_tiles = a.n_tiles[blk + 1] - t_begin;
-    const int i0 = a.i0 + blk * a.qb;
-    const long long lo = t_begin + static_cast<long long>(blockIdx.x) * n_tiles / gridDim.x;
-    const long long hi = t_begin + static_cast<long long>(blockIdx.x + 1) * n_tiles / gridDim.x;
-
-    for (long long b0 = lo; b0 < hi; b0 += kBatch) {
-        const int nb = static_cast<int>(min(static_cast<long long>(kBatch), hi - b0));
-        for (int x = tid; x < nb; x += kThreads) sm.recs[x] = a.tiles[b0 + x];
-        __syncthreads();
-        if (sm.abort_flag) break;
-        if (warp == 0) {
-            // table of chunk runs: where each run of tiles of one (pair, chunk) starts
-            int basec = 0;
-            for (int w = 0; w < kBatch / 32; ++w) {
-                const int x = w * 32 + lane;
-                const bool nw = x < nb && (x == 0 || sm.recs[x].x != sm.recs[x - 1].x || sm.recs[x].y != sm.recs[x - 1].y);
-                const unsigned m = __ballot_sync(kFullMask, nw);
-                if (nw) sm.cfirst[basec + __popc(m & ((1u << lane) - 1u))] = static_cast<uint8_t>(x);
-                basec += __popc(m);
-            }
-            if (lane == 0) { sm.cfirst[basec] = static_cast<uint8_t>(nb); sm.nchunks = basec; }
-        }
-        __syncthreads();
-
-        if (warp >= kProdWarp0 && warp < kMmaWarp) {
-            // ================================================================ producers (128 threads)
-            const int ptid = tid - kEpiThreads, pw = warp - kProdWarp0;
-            uint32_t tc = tcount, cc = ccount;
-            int cur_pair = -1, cur_c = -1;
-            int ck = -1;                       // ordinal of the current chunk run within the batch
-            bool next_issued = false;          // (producer thread 0) K/V of the upcoming chunk already requested
-            // landmark pieces of the next run, fetched a run ahead: piece x = lane + 32 r of the `per` landmark rows
-            // (16 pieces each; per = 1: lanes 0-15, r = 0 only)
-            uint4 lm_next[2] = {make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u)};
-            bool lm_next_ok = false;
-            const int per = s.Hl / s.Hkv;      // landmark rows per chunk: 1, or one per query head (App. C)
-            auto lm_piece = [&](int pr, int ch, int x) {
-                // 16-byte piece x % 16 of landmark head x / 16 of KV-head pair pr, chunk ch
-                uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                if (ch < s.C) {
-                    const long long lrow = (static_cast<long long>(pr / s.Hkv) * s.Hl + (pr % s.Hkv) * per + (x >> 4)) * s.C + ch;
-                    v = *reinterpret_cast<const uint4*>(a.lm + lrow * kD + (x & 15) * 8);
+    // Every role walks the same batches of tiles.  a.n_tiles[blk], a.n_tiles[blk + 1]: first tile of query block blk
+    // and of the next one; a launch that walks several blocks takes them in order, so that the CTAs stay on the same
+    // block (its gathered Q rows stay in L2).  The walk is instantiated once per role.
+    // body(nb, tcount, ccount, t_begin, i0): nb tiles cached in sm.recs, the CTA's running tile and chunk-run counters.
+    auto walk = [&](auto&& body) {
+        uint32_t tcount = 0, ccount = 0;
+        for (int blk = 0; blk < a.n_run; ++blk) {
+            const int t_begin = a.n_tiles[blk], n_tiles = a.n_tiles[blk + 1] - t_begin;
+            const int i0 = a.i0 + blk * a.qb;
+            const long long lo = t_begin + static_cast<long long>(blockIdx.x) * n_tiles / gridDim.x;
+            const long long hi = t_begin + static_cast<long long>(blockIdx.x + 1) * n_tiles / gridDim.x;
+            for (long long b0 = lo; b0 < hi; b0 += kBatch) {
+                const int nb = static_cast<int>(min(static_cast<long long>(kBatch), hi - b0));
+                for (int x = tid; x < nb; x += kThreads) sm.recs[x] = a.tiles[b0 + x];
+                __syncthreads();
+                if (sm.abort_flag) return;
+                if (warp == 0) {
+                    // table of chunk runs: where each run of tiles of one (pair, chunk) starts
+                    int basec = 0;
+                    for (int w = 0; w < kBatch / 32; ++w) {
+                        const int x = w * 32 + lane;
+                        const bool nw = x < nb && (x == 0 || sm.recs[x].x != sm.recs[x - 1].x || sm.recs[x].y != sm.recs[x - 1].y);
+                        const unsigned m = __ballot_sync(kFullMask, nw);
+                        if (nw) sm.cfirst[basec + __popc(m & ((1u << lane) - 1u))] = static_cast<uint8_t>(x);
+                        basec += __popc(m);
+                    }
+                    if (lane == 0) { sm.cfirst[basec] = static_cast<uint8_t>(nb); sm.nchunks = basec; }
                 }
-                return v;
-            };
+                __syncthreads();
+                body(nb, tcount, ccount, t_begin, i0);
+                // every role advances the shared counters identically
+                tcount += static_cast<uint32_t>(nb);
+                ccount += static_cast<uint32_t>(sm.nchunks);
+                __syncthreads();
+                if (sm.abort_flag) return;
+            }
+        }
+    };
+
+    auto gather_role = [&]() {
+        // ================================================================ Q gather (four warps)
+        // The tile's 128 rows (entry-major, head-minor) are 64 cp.async instructions of two 256-byte rows (a half-warp
+        // each, both of one entry); warp gw issues numbers 16 gw .. 16 gw + 15.  Lane l < 8 holds entry 8 gw + l and
+        // hands its token to the warp by a uniform shuffle: no address table, no barrier between the gather warps.
+        const int gw = warp - kGatherWarp0;
+        constexpr int kPerWarp = 64 / kGatherWarps;
+        const int j0 = gw * kPerWarp, j1 = j0 + kPerWarp;
+        const int e0 = j0 >> 1;                                      // first entry this warp touches
+        const int el = min(e0 + (lane & 7), kTok - 1);
+        const bool owns = lane < 8 && 2 * (e0 + lane) >= j0 && 2 * (e0 + lane) < j1;   // this lane records its entry
+        const int p16 = lane & 15, hh = lane >> 4;
+        const long long hstride = static_cast<long long>(s.R) * kD;
+        walk([&](int nb, uint32_t tcount, uint32_t, int t_begin, int i0) {
+            uint32_t tc = tcount;
             bool dead = false;
-            // entry of this thread's row for the upcoming tile, fetched one tile ahead
-            int e_next = a.entries[sm.recs[0].z + min(ptid >> 2, sm.recs[0].w - 1)];
-            int e_next2 = nb > 1 ? a.entries[sm.recs[1].z + min(ptid >> 2, sm.recs[1].w - 1)] : 0;
+            // this lane's entry of the upcoming tiles, fetched two tiles ahead
+            int e_next = a.entries[sm.recs[0].z + min(el, sm.recs[0].w - 1)];
+            int e_next2 = nb > 1 ? a.entries[sm.recs[1].z + min(el, sm.recs[1].w - 1)] : 0;
             for (int ti = 0; ti < nb; ++ti) {
                 const int4 rec = sm.recs[ti];
-                const int pair = rec.x, c = rec.y, ntok = rec.w;
+                const int pair = rec.x, ntok = rec.w;
                 const int e = e_next;
                 e_next = e_next2;
-                if (ti + 2 < nb) e_next2 = a.entries[sm.recs[ti + 2].z + min(ptid >> 2, sm.recs[ti + 2].w - 1)];
-                if (pair != cur_pair || c != cur_c) {
-                    // ---- new chunk: its K/V go to buffer cc & 1.  Nobody here waits for the copies: they complete on
-                    //      kv_ready, which only the MMA warp waits for, so the Q gathers below overlap them.
-                    const uint32_t cbuf = cc & 1u, vb = cc % kVBufs;
-                    if (pw == 0) {
-                        if (lane == 0 && !next_issued) {
-                            if (cc >= 2 && !mbar_wait(&sm.k_empty[cbuf], ((cc >> 1) - 1) & 1)) dead = true;
-                            if (!dead && cc >= kVBufs && !mbar_wait(&sm.v_empty[vb], ((cc / kVBufs) - 1) & 1)) dead = true;
-                            if (!dead) {
-                                const int row = pair * s.T + c * kS;
-                                mbar_expect_tx(&sm.k_ready[cbuf], 2 * 8192);
-                                tma_load_2d(kbuf + cbuf * kKBytes, &map_k, &sm.k_ready[cbuf], 0, row);
-                                tma_load_2d(kbuf + cbuf * kKBytes + kNS * 128, &map_k, &sm.k_ready[cbuf], 64, row);
-                                mbar_expect_tx(&sm.v_ready[vb], kVBytes);
-                                tma_load_2d(vbuf + vb * kVBytes, &map_v, &sm.v_ready[vb], 0, row);
-                                tma_load_2d(vbuf + vb * kVBytes + 8192, &map_v, &sm.v_ready[vb], 64, row);
-                            }
-                        }
-                        next_issued = false;
-                        dead = __shfl_sync(kFullMask, dead ? 1 : 0, 0) != 0;
-                        if (!dead) {
-                            // landmark row (key 64) of both K-blocks: the buffer is free (its previous user's MMAs are
-                            // done) and TMA never writes this row.  V stays as TMA writes it (keys x dims): the second
-                            // MMA reads it as an MN-major operand; keys past the end of the sequence hold other rows'
-                            // data (or TMA zero fill) and meet probabilities of 0.
-                            // key rows 64 .. 64 + per - 1: the chunk's landmark(s)
-                            const bool have_next = ck + 2 < sm.nchunks;
-                            const int4 r1 = have_next ? sm.recs[sm.cfirst[ck + 2]] : make_int4(0, 0, 0, 0);
-#pragma unroll
-                            for (int r = 0; r < 2; ++r) {
-                                const int x = lane + 32 * r;
-                                if (x < per * 16) {
-                                    const uint4 v = lm_next_ok ? lm_next[r] : lm_piece(pair, c, x);
-                                    const int pc = x & 15;
-                                    *reinterpret_cast<uint4*>(kbuf + cbuf * kKBytes + (pc >> 3) * (kNS * 128) + swz128(64 + (x >> 4), pc & 7)) = v;
-                                    // the next run's landmark, so that its load is not waited for at the next switch
-                                    if (have_next) lm_next[r] = lm_piece(r1.x, r1.y, x);
-                                }
-                            }
-                            lm_next_ok = have_next;
-                            fence_proxy_async_smem();
-                            __syncwarp();
-                            if (lane == 0) mbar_arrive(&sm.k_ready[cbuf]);
-                        }
-                    }
-                    if (dead || *reinterpret_cast<volatile int*>(&sm.abort_flag)) { dead = true; break; }
-                    cur_pair = pair;
-                    cur_c = c;
-                    ++cc;
-                    ++ck;
-                    // warm L2 with the K/V rows of the run after the next one (the next one is requested below)
-                    if (ptid == 0 && ck + 2 < sm.nchunks) {
-                        const int4 r2 = sm.recs[sm.cfirst[ck + 2]];
-                        const int row2 = r2.x * s.T + r2.y * kS;
-                        tma_prefetch_l2_2d(&map_k, 0, row2);
-                        tma_prefetch_l2_2d(&map_k, 64, row2);
-                        tma_prefetch_l2_2d(&map_v, 0, row2);
-                        tma_prefetch_l2_2d(&map_v, 64, row2);
-                    }
-                }
-                // ---- look ahead (producer thread 0): request the next chunk's K/V as soon as its buffer is free
-                if (ptid == 0 && !next_issued) {
-                    const int tj = sm.cfirst[ck + 1];          // first tile of the next run (nb if none)
-                    const uint32_t nbuf = cc & 1u, nvb = cc % kVBufs;
-                    if (tj < nb && (cc < 2 || mbar_test_wait(&sm.k_empty[nbuf], ((cc >> 1) - 1) & 1)) &&
-                        (cc < kVBufs || mbar_test_wait(&sm.v_empty[nvb], ((cc / kVBufs) - 1) & 1))) {
-                        const int row = sm.recs[tj].x * s.T + sm.recs[tj].y * kS;
-                        mbar_expect_tx(&sm.k_ready[nbuf], 2 * 8192);
-                        tma_load_2d(kbuf + nbuf * kKBytes, &map_k, &sm.k_ready[nbuf], 0, row);
-                        tma_load_2d(kbuf + nbuf * kKBytes + kNS * 128, &map_k, &sm.k_ready[nbuf], 64, row);
-                        mbar_expect_tx(&sm.v_ready[nvb], kVBytes);
-                        tma_load_2d(vbuf + nvb * kVBytes, &map_v, &sm.v_ready[nvb], 0, row);
-                        tma_load_2d(vbuf + nvb * kVBytes + 8192, &map_v, &sm.v_ready[nvb], 64, row);
-                        next_issued = true;
-                    }
-                }
-                // ---- gather the tile's 128 query rows (token-major, head-minor) into the swizzled Q tile
-                const uint32_t qs = tc % kQSlots, ms = tc % kMetaSlots, rb = tc & 1u;
+                if (ti + 2 < nb) e_next2 = a.entries[sm.recs[ti + 2].z + min(el, sm.recs[ti + 2].w - 1)];
+                const uint32_t qs = tc % kQSlots, ms = tc % kMetaSlots;
                 if (tc >= kQSlots && !mbar_wait(&sm.q_empty[qs], ((tc / kQSlots) - 1) & 1)) { dead = true; break; }
+                if (*reinterpret_cast<volatile int*>(&sm.abort_flag)) { dead = true; break; }
+                if (owns) sm.tile_ent[ms][e0 + lane] = e;
+                if (gw == 0 && lane == 0) {
+                    sm.tile_meta[ms][0] = pair; sm.tile_meta[ms][1] = rec.y; sm.tile_meta[ms][2] = ntok;
+                    sm.tile_meta[ms][3] = rec.z - (a.whole ? 0 : t_begin * kTok);
+                }
                 {
-                    // thread ptid owns row ptid for the address table
-                    const int tk = ptid >> 2, hd = ptid & 3;
-                    const int bb = pair / s.Hkv, gk = pair % s.Hkv;
-                    sm.rowptr[rb][ptid] = a.q + ((static_cast<long long>(bb) * s.Hq + gk * kG + hd) * s.R + i0 + (e >> 8)) * kD;
-                    if (hd == 0) sm.tile_ent[ms][tk] = e;
-                    if (ptid == 0) { sm.tile_meta[ms][0] = pair; sm.tile_meta[ms][1] = c; sm.tile_meta[ms][2] = ntok; sm.tile_meta[ms][3] = rec.z - (a.whole ? 0 : t_begin * kTok); }
-                    producer_barrier();
-                    const uint32_t qaddr = smem_u32(qbuf + qs * kQBytes);
-                    const int p16 = lane & 15;
-                    const uint32_t koff = (p16 >> 3) * 16384;
-                    // all 16 source addresses first, then the 16 copies back to back
-                    const __nv_bfloat16* src[16];
+                    const uint32_t qaddr = smem_u32(qbuf + qs * kQBytes) + (p16 >> 3) * 16384;
+                    const __nv_bfloat16* qb0 = a.q + (static_cast<long long>(pair / s.Hkv) * s.Hq + (pair % s.Hkv) * kG + hh) * hstride +
+                                               static_cast<long long>(i0) * kD + p16 * 8;
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) src[j] = sm.rowptr[rb][pw * 32 + 2 * j + (lane >> 4)] + p16 * 8;
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const int row = pw * 32 + 2 * j + (lane >> 4);       // a half-warp copies one 256-byte row
-                        cp_async16(qaddr + koff + swz128(row, p16 & 7), src[j]);
+                    for (int jj = 0; jj < kPerWarp; ++jj) {
+                        const int j = j0 + jj;
+                        const int ej = __shfl_sync(kFullMask, e, (j >> 1) - e0);
+                        const int row = 2 * j + hh;
+                        const __nv_bfloat16* src = qb0 + (2 * j & 3) * hstride + static_cast<long long>(ej >> 8) * kD;
+                        cp_async16(qaddr + swz128(row, p16 & 7), src);
                     }
                     cp_async_commit();
                 }
@@ -324,21 +250,251 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                 if (lane == 0) mbar_arrive(&sm.q_full[(tc - 1) % kQSlots]);
             }
             if (dead && lane == 0) { set_status(a.status, kDevTimeout); atomicExch(&sm.abort_flag, 1); }
-            if (ptid == 0 && next_issued) {
-                // (only after a timeout) a requested chunk was never taken up: complete its barrier, let the copy land
-                mbar_arrive(&sm.k_ready[cc & 1u]);
-                mbar_wait(&sm.k_ready[cc & 1u], (cc >> 1) & 1);
-                mbar_wait(&sm.v_ready[cc % kVBufs], (cc / kVBufs) & 1);
+        });
+    };
+
+    // (called at the end of every role)
+    auto finish = [&]() {
+        tc_fence_before_sync();
+        __syncthreads();
+        tc_fence_after_sync();
+        if (warp == kMmaWarp) tmem_dealloc(tmem_base, 512);
+    };
+
+    if (warp < kOutWarp0) {
+        // ================================================================ softmax: one row per thread
+        // Group g (warps 4g .. 4g+3) turns the scores of the tiles in S/P/O slot g into probabilities: the two
+        // groups work on consecutive tiles at the same time.
+        const uint32_t grp = static_cast<uint32_t>(warp >> 2);
+        const int row = (warp & 3) * 32 + lane;
+        const uint32_t t_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16) + grp * 128;
+        const int tk = row >> 2, hd = row & 3;
+        const float sl2 = s.scale * kLog2e;
+        const int lh = (s.Hl == s.Hkv) ? 0 : hd;
+        walk([&](int nb, uint32_t tcount, uint32_t, int, int i0) {
+            bool ok = true;
+            for (int ti = static_cast<int>((grp ^ tcount) & 1u); ti < nb && ok; ti += 2) {
+                const uint32_t tcv = tcount + ti;                      // (tcv & 1) == grp
+                ok = mbar_wait(&sm.s_full[grp], (tcv >> 1) & 1);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t ms = tcv % kMetaSlots;
+                const int pair = sm.tile_meta[ms][0], c = sm.tile_meta[ms][1];
+                const int orow0 = sm.tile_meta[ms][3] * kG;          // first row of the tile in the output buffers
+                const int e = sm.tile_ent[ms][tk];
+                const int il = e >> 8, slot = e & 255;
+                const bool local = slot >= s.K;                            // a chunk of the local window: mass = its exact log-sum-exp
+                const int lim = local ? s.pos0 + i0 + il - c * kS : kS - 1;   // last visible key of the chunk
+                // the 64 key scores and the surrogate score columns: the landmark of this row's head (key 64 + hd)
+                // or the shared one (key 64); warp-uniform addresses, the lane picks its column
+                float v[64];
+                float lm4[4];
+                tmem_ld64_4(t_lane, t_lane + 64, v, lm4);
+                const float lmk = lh == 0 ? lm4[0] : (lh == 1 ? lm4[1] : (lh == 2 ? lm4[2] : lm4[3]));
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.s_empty[grp]);
+                if (__any_sync(kFullMask, local)) {
+#pragma unroll
+                    for (int j = 0; j < 64; ++j)
+                        if (j > lim) v[j] = -INFINITY;
+                }
+                // four independent chains of three-input maxima
+                float mx[4] = {v[0], v[1], v[2], v[3]};
+#pragma unroll
+                for (int j = 4; j < 60; j += 8) {
+                    mx[0] = fmax3(mx[0], v[j], v[j + 1]);
+                    mx[1] = fmax3(mx[1], v[j + 2], v[j + 3]);
+                    mx[2] = fmax3(mx[2], v[j + 4], v[j + 5]);
+                    mx[3] = fmax3(mx[3], v[j + 6], v[j + 7]);
+                }
+                mx[0] = fmax3(mx[0], v[60], v[61]);
+                mx[1] = fmax3(mx[1], v[62], v[63]);
+                const float m = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+                const float2 sl22 = make_float2(sl2, sl2);
+                const float2 nms2 = make_float2(-m * sl2, -m * sl2);
+                // exponentials in place, two lanes of arithmetic per instruction; four chains for the row sum
+                float2 zp[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const float2 x = __ffma2_rn(make_float2(v[2 * j], v[2 * j + 1]), sl22, nms2);
+                    v[2 * j] = ex2_approx(x.x);
+                    v[2 * j + 1] = ex2_approx(x.y);
+                    zp[j & 3] = __fadd2_rn(zp[j & 3], make_float2(v[2 * j], v[2 * j + 1]));
+                }
+                const float2 z2 = __fadd2_rn(__fadd2_rn(zp[0], zp[1]), __fadd2_rn(zp[2], zp[3]));
+                const float z = z2.x + z2.y;
+                const float zi = 1.f / z;
+                const float2 zi2 = make_float2(zi, zi);
+                // the P V product of this slot's previous tile must have read its probabilities
+                if (tcv >= 2) {
+                    ok = mbar_wait(&sm.o_full[grp], ((tcv >> 1) - 1) & 1);
+                    if (!ok) break;
+                }
+#pragma unroll
+                for (int pc = 0; pc < 4; ++pc) {
+                    uint32_t pk[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const float2 p = __fmul2_rn(make_float2(v[pc * 16 + 2 * j], v[pc * 16 + 2 * j + 1]), zi2);
+                        pk[j] = pack_bf16(p.x, p.y);
+                    }
+                    tmem_st8(t_lane + kPCol + pc * 8, pk);
+                }
+                // chunk mass of the row (rows of a ragged tile's padding land in the list's padding)
+                const float bb = (a.bias && c < s.C)
+                    ? a.bias[(static_cast<long long>(pair / s.Hkv) * s.Hl + (pair % s.Hkv) * (s.Hl / s.Hkv) + lh) * s.C + c] : 0.f;
+                a.lam[orow0 + row] = local ? m * s.scale + __logf(z) : lmk * s.scale + bb;
+                tmem_wait_st();
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.p_full[grp]);
             }
+            if (!ok && lane == 0) { set_status(a.status, kDevTimeout); atomicExch(&sm.abort_flag, 1); }
+        });
+        finish();
+    } else if (warp < kGatherWarp0) {
+        // ================================================================ output group: O = P V -> bf16 rows
+        // The warp's 32 rows of the staging buffer (4 KB, swizzled as the output map expects) take 64 columns at a
+        // time; one TMA store per half writes 32 full rows.
+        const int ow = warp - kOutWarp0;
+        const int row = ow * 32 + lane;
+        const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(ow * 32) << 16);
+        const uint64_t pol = l2_policy_evict_first();
+        uint8_t* wstg = obuf + ow * 4096;            // columns 0..63; + kPBytes: columns 64..127
+        walk([&](int nb, uint32_t tcount, uint32_t, int, int) {
+            bool ok = true;
+            for (int ti = 0; ti < nb && ok; ++ti) {
+                const uint32_t tcv = tcount + ti, sl = tcv & 1u;
+                ok = mbar_wait(&sm.o_full[sl], (tcv >> 1) & 1);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const int orow0 = sm.tile_meta[tcv % kMetaSlots][3] * kG;
+#pragma unroll 1
+                for (int hb = 0; hb < 2; ++hb) {
+                    uint32_t pk[32];
+                    {
+                        float v[64];
+                        tmem_ld64(t_lane + 256 + sl * 128 + hb * 64, v);
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) pk[j] = pack_bf16(v[2 * j], v[2 * j + 1]);
+                    }
+                    if (hb == 0) {
+                        // the previous tile's stores (lane 0: columns 0..63, lane 1: 64..127) must have read the staging rows
+                        if (lane < 2) bulk_wait_read<0>();
+                        __syncwarp();
+                    } else {
+                        // the accumulator is free for the slot's next tile
+                        tc_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&sm.o_empty[sl]);
+                    }
+#pragma unroll
+                    for (int pc = 0; pc < 8; ++pc)
+                        *reinterpret_cast<uint4*>(obuf + hb * kPBytes + swz128(row, pc)) = make_uint4(pk[4 * pc], pk[4 * pc + 1], pk[4 * pc + 2], pk[4 * pc + 3]);
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane < 2) {
+                    tma_store_2d(&map_o, wstg + lane * kPBytes, lane * 64, orow0 + ow * 32, pol);
+                    bulk_commit();
+                }
+            }
+            if (!ok && lane == 0) { set_status(a.status, kDevTimeout); atomicExch(&sm.abort_flag, 1); }
+        });
+        finish();
+    } else if (warp < kLoadWarp) {
+        gather_role();
+        finish();
+    } else {
+        if (warp == kLoadWarp) {
+            // ================================================================ K/V loader (one warp)
+            // One chunk run after the other: wait until the run's K and V buffers are free, request the tiles (they
+            // complete on k_ready / v_ready, which only the MMA warp waits for), write the landmark row(s).
+            const int per = s.Hl / s.Hkv;      // landmark rows per chunk: 1, or one per query head (App. C)
+            auto lm_piece = [&](int pr, int ch, int x) {
+                // 16-byte piece x % 16 of landmark head x / 16 of KV-head pair pr, chunk ch
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                if (ch < s.C) {
+                    const long long lrow = (static_cast<long long>(pr / s.Hkv) * s.Hl + (pr % s.Hkv) * per + (x >> 4)) * s.C + ch;
+                    v = *reinterpret_cast<const uint4*>(a.lm + lrow * kD + (x & 15) * 8);
+                }
+                return v;
+            };
+            walk([&](int, uint32_t, uint32_t ccount, int, int) {
+                const int nch = sm.nchunks;
+                bool dead = false;
+                // landmark pieces of the current run (piece x = lane + 32 r of the `per` rows, 16 pieces each),
+                // fetched a run ahead
+                uint4 lm_cur[2] = {make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u)};
+                if (nch > 0) {
+                    const int4 r0 = sm.recs[0];
+#pragma unroll
+                    for (int r = 0; r < 2; ++r)
+                        if (lane + 32 * r < per * 16) lm_cur[r] = lm_piece(r0.x, r0.y, lane + 32 * r);
+                }
+                for (int ck = 0; ck < nch; ++ck) {
+                    const uint32_t cc = ccount + static_cast<uint32_t>(ck);
+                    const int4 rec = sm.recs[sm.cfirst[ck]];
+                    const int pair = rec.x, c = rec.y;
+                    const uint32_t cbuf = cc & 1u, vb = cc % kVBufs;
+                    if (lane == 0) {
+                        if (cc >= 2 && !mbar_wait(&sm.k_empty[cbuf], ((cc >> 1) - 1) & 1)) dead = true;
+                        if (!dead && cc >= kVBufs && !mbar_wait(&sm.v_empty[vb], ((cc / kVBufs) - 1) & 1)) dead = true;
+                        if (!dead) {
+                            const int row = pair * s.T + c * kS;
+                            mbar_expect_tx(&sm.k_ready[cbuf], 2 * 8192);
+                            tma_load_2d(kbuf + cbuf * kKBytes, &map_k, &sm.k_ready[cbuf], 0, row);
+                            tma_load_2d(kbuf + cbuf * kKBytes + kNS * 128, &map_k, &sm.k_ready[cbuf], 64, row);
+                            mbar_expect_tx(&sm.v_ready[vb], kVBytes);
+                            tma_load_2d(vbuf + vb * kVBytes, &map_v, &sm.v_ready[vb], 0, row);
+                            tma_load_2d(vbuf + vb * kVBytes + 8192, &map_v, &sm.v_ready[vb], 64, row);
+                            // warm L2 with the K/V rows of the run after the next one
+                            if (ck + 2 < nch) {
+                                const int4 r2 = sm.recs[sm.cfirst[ck + 2]];
+                                const int row2 = r2.x * s.T + r2.y * kS;
+                                tma_prefetch_l2_2d(&map_k, 0, row2);
+                                tma_prefetch_l2_2d(&map_k, 64, row2);
+                                tma_prefetch_l2_2d(&map_v, 0, row2);
+                                tma_prefetch_l2_2d(&map_v, 64, row2);
+                            }
+                        }
+                    }
+                    dead = __shfl_sync(kFullMask, dead ? 1 : 0, 0) != 0;
+                    if (dead || *reinterpret_cast<volatile int*>(&sm.abort_flag)) { dead = true; break; }
+                    // landmark row(s) (keys 64 .. 64 + per - 1) of both K-blocks: the buffer is free (its previous
+                    // user's MMAs are done) and TMA never writes these rows.  V stays as TMA writes it (keys x dims):
+                    // the second MMA reads it as an MN-major operand; keys past the end of the sequence hold other
+                    // rows' data (or TMA zero fill) and meet probabilities of 0.
+                    const bool have_next = ck + 1 < nch;
+                    const int4 r1 = have_next ? sm.recs[sm.cfirst[ck + 1]] : make_int4(0, 0, 0, 0);
+#pragma unroll
+                    for (int r = 0; r < 2; ++r) {
+                        const int x = lane + 32 * r;
+                        if (x < per * 16) {
+                            const int pc = x & 15;
+                            *reinterpret_cast<uint4*>(kbuf + cbuf * kKBytes + (pc >> 3) * (kNS * 128) + swz128(64 + (x >> 4), pc & 7)) = lm_cur[r];
+                            if (have_next) lm_cur[r] = lm_piece(r1.x, r1.y, x);
+                        }
+                    }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sm.k_ready[cbuf]);
+                }
+                if (dead && lane == 0) { set_status(a.status, kDevTimeout); atomicExch(&sm.abort_flag, 1); }
+            });
         } else if (warp == kMmaWarp) {
             // ================================================================ MMA issuer
-            if (lane == 0) {
+            walk([&](int nb, uint32_t tcount, uint32_t ccount, int, int) {
+                if (lane != 0) return;
                 constexpr uint32_t idesc_s = umma_idesc_bf16(kRows, kNS);
                 constexpr uint32_t idesc_o = umma_idesc_bf16(kRows, kD) | kUmmaBMnMajor;
                 uint32_t cc = ccount;
                 int cur_pair = -1, cur_c = -1;
-                uint32_t vbuf_of0 = 0u, vbuf_of1 = 0u;     // V buffer used by the tile in S/P/O slot 0 / 1 (two scalars: an
-                                                           // array indexed by the slot would live in local memory)
+                // the P V queue follows the chunk runs on its own (its V buffer is the run's ordinal modulo kVBufs), so
+                // the score queue may run ahead of it as far as the S slots and the gathered Q tiles allow
+                uint32_t cco = ccount;
+                int cur_pair_o = -1, cur_c_o = -1;
                 bool ok = true;
                 // Two in-order queues (S MMAs, O MMAs) served by polling: an O MMA whose probabilities are
                 // ready is never held up by a Q tile that has not arrived yet, and vice versa.
@@ -346,7 +502,7 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                 uint32_t idle = 0;
                 while (no < nb && ok) {
                     bool progressed = false;
-                    if (ns < nb && ns < no + 2) {
+                    if (ns < nb) {
                         const uint32_t tcv = tcount + ns, sl = tcv & 1u, qs = tcv % kQSlots;
                         const int4 rec = sm.recs[ns];
                         const bool newc = rec.x != cur_pair || rec.y != cur_c;
@@ -358,7 +514,6 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                         if (ready) {
                             if (newc) { cur_pair = rec.x; cur_c = rec.y; ++cc; }
                             const uint32_t cb = (cc - 1) & 1u;
-                            if (sl) vbuf_of1 = (cc - 1) % kVBufs; else vbuf_of0 = (cc - 1) % kVBufs;
                             tc_fence_after_sync();
                             const uint32_t qa = smem_u32(qbuf + qs * kQBytes), ka = smem_u32(kbuf + cb * kKBytes);
 #pragma unroll
@@ -374,10 +529,13 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                         }
                     }
                     if (no < ns) {
-                        const uint32_t tcv = tcount + no, sl = tcv & 1u, vb = sl ? vbuf_of1 : vbuf_of0;
+                        const uint32_t tcv = tcount + no, sl = tcv & 1u;
                         bool ready = mbar_test_wait(&sm.p_full[sl], (tcv >> 1) & 1);
                         if (ready && tcv >= 2) ready = mbar_test_wait(&sm.o_empty[sl], ((tcv >> 1) - 1) & 1);
                         if (ready) {
+                            const int4 reco = sm.recs[no];
+                            if (reco.x != cur_pair_o || reco.y != cur_c_o) { cur_pair_o = reco.x; cur_c_o = reco.y; ++cco; }
+                            const uint32_t vb = (cco - 1) % kVBufs;
                             tc_fence_after_sync();
                             const uint32_t va = smem_u32(vbuf + vb * kVBytes);
                             // P from tensor memory (columns kPCol.. of the slot: 8 columns = 16 keys per step), V from
@@ -388,7 +546,7 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                                              umma_desc_mn128(va + ks * 2048, 8192u, 1024u), idesc_o, ks > 0 ? 1u : 0u);
                             umma_commit(&sm.o_full[sl]);
                             // last tile of its chunk in this batch: the V buffer is free once these MMAs are done
-                            const bool last = no + 1 >= nb || sm.recs[no + 1].x != sm.recs[no].x || sm.recs[no + 1].y != sm.recs[no].y;
+                            const bool last = no + 1 >= nb || sm.recs[no + 1].x != reco.x || sm.recs[no + 1].y != reco.y;
                             if (last) umma_commit(&sm.v_empty[vb]);
                             ++no;
                             progressed = true;
@@ -402,146 +560,10 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                     }
                 }
                 if (!ok) { set_status(a.status, kDevTimeout); atomicExch(&sm.abort_flag, 1); }
-            }
-        } else {
-            // ================================================================ epilogue: one row per thread
-            // Group 0 turns every tile's scores into probabilities, group 1 takes every tile's O = P V out of tensor
-            // memory: the softmax of a tile never waits for the tile's own P V.
-            const int grp = warp >> 2;
-            const int row = (warp & 3) * 32 + lane;
-            const uint32_t t_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-            bool ok = true;
-            if (grp == 0) {
-                const int tk = row >> 2, hd = row & 3;
-                const float sl2 = s.scale * kLog2e;
-                for (int ti = 0; ti < nb && ok; ++ti) {
-                    const uint32_t tcv = tcount + ti, sl = tcv & 1u;
-                    ok = mbar_wait(&sm.s_full[sl], (tcv >> 1) & 1);
-                    if (!ok) break;
-                    tc_fence_after_sync();
-                    const uint32_t ms = tcv % kMetaSlots;
-                    const int pair = sm.tile_meta[ms][0], c = sm.tile_meta[ms][1];
-                    const int orow0 = sm.tile_meta[ms][3] * kG;          // first row of the tile in the output buffers
-                    const int e = sm.tile_ent[ms][tk];
-                    const int il = e >> 8, slot = e & 255;
-                    const bool local = slot >= s.K;                            // a chunk of the local window: mass = its exact log-sum-exp
-                    const int lim = local ? s.pos0 + i0 + il - c * kS : kS - 1;   // last visible key of the chunk
-                    // the 64 key scores and the surrogate score columns: the landmark of this row's head (key 64 + hd)
-                    // or the shared one (key 64); warp-uniform addresses, the lane picks its column
-                    float v[64];
-                    const int lh = (s.Hl == s.Hkv) ? 0 : hd;
-                    float lm4[4];
-                    tmem_ld64_4(t_lane + sl * 128, t_lane + sl * 128 + 64, v, lm4);
-                    const float lmk = lh == 0 ? lm4[0] : (lh == 1 ? lm4[1] : (lh == 2 ? lm4[2] : lm4[3]));
-                    tc_fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&sm.s_empty[sl]);
-                    // four independent chains for the maximum and for the sum: the row is one thread's work and a
-                    // single chain of 64 dependent operations is what the warp would otherwise wait on
-                    float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-                    if (__any_sync(kFullMask, local)) {
-#pragma unroll
-                        for (int j = 0; j < 64; ++j) {
-                            if (j > lim) v[j] = -INFINITY;
-                            mx[j & 3] = fmaxf(mx[j & 3], v[j]);
-                        }
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 64; ++j) mx[j & 3] = fmaxf(mx[j & 3], v[j]);
-                    }
-                    const float m = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-                    float zp[4] = {0.f, 0.f, 0.f, 0.f};
-                    const float ms2 = m * sl2;
-                    // the P V product of this slot's previous tile must have read its probabilities
-                    if (tcv >= 2) {
-                        ok = mbar_wait(&sm.o_full[sl], ((tcv >> 1) - 1) & 1);
-                        if (!ok) break;
-                    }
-#pragma unroll
-                    for (int pc = 0; pc < 4; ++pc) {
-                        uint32_t pk[8];
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            const float p0 = ex2_approx(fmaf(v[pc * 16 + 2 * j], sl2, -ms2));
-                            const float p1 = ex2_approx(fmaf(v[pc * 16 + 2 * j + 1], sl2, -ms2));
-                            zp[j & 3] += p0 + p1;
-                            pk[j] = pack_bf16(p0, p1);
-                        }
-                        tmem_st8(t_lane + sl * 128 + kPCol + pc * 8, pk);
-                    }
-                    const float z = (zp[0] + zp[1]) + (zp[2] + zp[3]);
-                    // read by the output group after this tile's P V.  The ring's slot was last read for the tile
-                    // four back, before the output group released that tile's accumulator; the P V waited for
-                    // above could only be issued after that release.
-                    sm.zinv[tcv & 3u][row] = 1.f / z;
-                    // chunk mass of the row (rows of a ragged tile's padding land in the list's padding)
-                    const float bb = (a.bias && c < s.C)
-                        ? a.bias[(static_cast<long long>(pair / s.Hkv) * s.Hl + (pair % s.Hkv) * (s.Hl / s.Hkv) + lh) * s.C + c] : 0.f;
-                    a.lam[orow0 + row] = local ? m * s.scale + __logf(z) : lmk * s.scale + bb;
-                    tmem_wait_st();
-                    tc_fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&sm.p_full[sl]);
-                }
-            } else {
-                // ---------------- O = P V -> normalised bf16 rows: the warp's 32 rows of the staging buffer (4 KB,
-                // swizzled as the output map expects) take 64 columns at a time; one TMA store per half writes 32
-                // full rows
-                const uint64_t pol = l2_policy_evict_first();
-                uint8_t* wstg = obuf + (warp & 3) * 4096;            // columns 0..63; + kPBytes: columns 64..127
-                for (int ti = 0; ti < nb && ok; ++ti) {
-                    const uint32_t tcv = tcount + ti, sl = tcv & 1u;
-                    ok = mbar_wait(&sm.o_full[sl], (tcv >> 1) & 1);
-                    if (!ok) break;
-                    tc_fence_after_sync();
-                    const int orow0 = sm.tile_meta[tcv % kMetaSlots][3] * kG;
-                    const float zi = sm.zinv[tcv & 3u][row];
-#pragma unroll 1
-                    for (int hb = 0; hb < 2; ++hb) {
-                        uint32_t pk[32];
-                        {
-                            float v[64];
-                            tmem_ld64(t_lane + 256 + sl * 128 + hb * 64, v);
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) pk[j] = pack_bf16(v[2 * j] * zi, v[2 * j + 1] * zi);
-                        }
-                        if (hb == 0) {
-                            // the previous tile's stores (lane 0: columns 0..63, lane 1: 64..127) must have read the staging rows
-                            if (lane < 2) bulk_wait_read<0>();
-                            __syncwarp();
-                        } else {
-                            // the accumulator (and the ring slot of 1 / row sum) is free for the slot's next tile
-                            tc_fence_before_sync();
-                            __syncwarp();
-                            if (lane == 0) mbar_arrive(&sm.o_empty[sl]);
-                        }
-#pragma unroll
-                        for (int pc = 0; pc < 8; ++pc)
-                            *reinterpret_cast<uint4*>(obuf + hb * kPBytes + swz128(row, pc)) = make_uint4(pk[4 * pc], pk[4 * pc + 1], pk[4 * pc + 2], pk[4 * pc + 3]);
-                    }
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane < 2) {
-                        tma_store_2d(&map_o, wstg + lane * kPBytes, lane * 64, orow0 + (warp & 3) * 32, pol);
-                        bulk_commit();
-                    }
-                }
-            }
-            if (!ok && lane == 0) { set_status(a.status, kDevTimeout); atomicExch(&sm.abort_flag, 1); }
+            });
         }
-        // every role advances the shared counters identically
-        tcount += static_cast<uint32_t>(nb);
-        ccount += static_cast<uint32_t>(sm.nchunks);
-        __syncthreads();
-        if (sm.abort_flag) break;
+        finish();
     }
-    if (sm.abort_flag) break;
-    }
-
-    tc_fence_before_sync();
-    __syncthreads();
-    tc_fence_after_sync();
-    if (warp == kMmaWarp) tmem_dealloc(tmem_base, 512);
 }
 
 }  // namespace
@@ -562,7 +584,7 @@ int launch_prefill_attend_tc(const Shape& s, const void* q, const void* maps, co
     }
     AtcArgs a{s, static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(landmarks), bias, entries,
               static_cast<const int4*>(tiles), n_tiles, lam, status, i0, whole, n_run, qb};
-    if (launch_pdl(prefill_attend_tc_kernel, dim3(148), dim3(kThreads), smem, stream, m[0], m[1], m[2], a) != cudaSuccess)
+    if (launch_pdl(prefill_attend_tc_kernel, dim3(sm_count()), dim3(kThreads), smem, stream, m[0], m[1], m[2], a) != cudaSuccess)
         return HILS_ERR_CUDA;
     if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
     return 1;

@@ -644,7 +644,7 @@ int build_inverse_index(const Shape& s, const int32_t* sel, void* scratch, size_
     if (cudaMemsetAsync(sc + p.off_cnt, 0, p.zero_bytes, stream) != cudaSuccess) return HILS_ERR_CUDA;
     const long long elems = static_cast<long long>(pairs) * s.R * (s.K + max_local_slots(s.W));
     const long long want = (elems + 255) / 256;
-    const unsigned eb = static_cast<unsigned>(want < 148 * 16 ? want : 148 * 16);
+    const unsigned eb = static_cast<unsigned>(want < sm_count() * 16 ? want : sm_count() * 16);
     const unsigned nseg = static_cast<unsigned>((static_cast<long long>(p.n_blocks) * pairs * p.nc + 1023) / 1024);
     invert_count_kernel<<<eb, 256, 0, stream>>>(a);
     invert_segsum_kernel<<<nseg, 1024, 0, stream>>>(a);
@@ -737,7 +737,7 @@ int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
     {
         const long long elems = static_cast<long long>(pairs) * s.R * (s.K + max_local_slots(s.W));
         const long long want = (elems + 255) / 256;
-        const unsigned eb = static_cast<unsigned>(want < 148 * 16 ? want : 148 * 16);
+        const unsigned eb = static_cast<unsigned>(want < sm_count() * 16 ? want : sm_count() * 16);
         if (!counted) {
             invert_count_kernel<<<eb, 256, 0, stream>>>(a);
             ++launches;

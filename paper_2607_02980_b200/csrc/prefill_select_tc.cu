@@ -450,7 +450,8 @@ int launch_prefill_select_tc(const Shape& s, const void* q, const void* landmark
     TcArgs a{s, bias, sel, status, (cnt && qb % kTileTok == 0) ? cnt : nullptr, qb, nc};
     const int tiles = (s.R + kTileTok - 1) / kTileTok;
     const unsigned all_tiles = static_cast<unsigned>(pairs) * tiles;
-    const unsigned grid = all_tiles < 148u ? all_tiles : 148u;       // one persistent CTA per SM
+    const unsigned nsm = static_cast<unsigned>(sm_count());
+    const unsigned grid = all_tiles < nsm ? all_tiles : nsm;       // one persistent CTA per SM
     const bool perhead = s.Hl != s.Hkv;
     if (s.K <= 16) {
         if (perhead) prefill_select_tc_kernel<16, true><<<grid, kThreads, smem, stream>>>(map_q, map_lm, a);

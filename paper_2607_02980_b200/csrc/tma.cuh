@@ -445,4 +445,28 @@ inline bool make_bf16_2d_map(CUtensorMap* map, const void* base, uint64_t rows, 
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+
+// bf16 tensor [n2, n1, cols] (cols contiguous, pitches of cols and n1 * cols elements) -> map with box
+// {box_cols, box1, box2} and the 128-byte swizzle (box_cols * 2 bytes must be 128): the box's box1 * box2 rows land
+// as consecutive 128-byte rows in shared memory.
+inline bool make_bf16_3d_map(CUtensorMap* map, const void* base, uint64_t n2, uint64_t n1, uint64_t cols,
+                             uint32_t box_cols, uint32_t box1, uint32_t box2) {
+    EncodeTiledFn fn = get_encode_tiled();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {cols, n1, n2};
+    cuuint64_t strides[2] = {cols * 2, n1 * cols * 2};
+    cuuint32_t box[3] = {box_cols, box1, box2};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// packed pairs of fp32 (sm_100): one instruction per two lanes of a row's arithmetic
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
 }  // namespace hils
