@@ -4,8 +4,12 @@
 A "step" is one pass of the whole hot path (landmark scoring, group max, top-K selection, local
 attention, per-chunk attention, fusion) over one batch of seeded synthetic input, through the C ABI.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg1|cfg0|cfg2|cfg3|cfg4]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg0|cfg1|cfg3|cfg4]
                   [--impl ours|reference] [--no-extra] [--no-e2e] [--no-cpu-baseline]
+
+The default workload is cfg2, the largest single-GPU prefill configuration (L = 131072, K = 32); the decode half of
+the metric (cfg3, cfg4) and cfg1 are measured in the same run and carried in top-level fields of the JSON line
+(decode_cfg3_GBps, decode_cfg4_frac_of_measured_hbm, ...), with their per-kernel detail under "extra".
 
 Prefill workloads report effective TFLOP/s on the gathered FLOP (what the method must do, not what
 dense attention would); decode workloads report GB/s on the algorithmic bytes (landmarks scanned +
@@ -33,15 +37,20 @@ import torch
 
 from paper_2607_02980_b200 import workloads as wl
 
-# dram__bytes_read.sum + dram__bytes_write.sum PER LAUNCH of each workload's dominant kernel, from the ncu
-# captures summarised under profiles/.  The decode captures ran a reduced batch (8 of 64 sequences for cfg3, 1 of 4
-# for cfg4); traffic is proportional to the number of (sequence, KV head) pairs and is scaled to the full launch.
-NCU_TRAFFIC_BYTES = {
-    ("cfg1", "prefill_attend"): int((654.3 + 2270.9) * 1e6),   # the one launch that walks all four query blocks
-    ("cfg3", "decode_attend"): int(70.5e6 * 8),
-    ("cfg4", "decode_attend"): int(17.1e6 * 4),
-    ("cfg4", "decode_score"): int(33.57e6 * 4),
-}
+# dram__bytes_read.sum + dram__bytes_write.sum PER LAUNCH of each workload's dominant kernel come from the ncu
+# captures recorded in profiles/ncu_dram_traffic.json (kernel, bytes, what was captured, how it was scaled, when): a
+# kernel without a record there reports "traffic": null rather than a stale figure.
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "ncu_dram_traffic.json")
+
+
+def load_traffic(path=TRAFFIC_FILE):
+    """{(workload key, kernel name): record} from the committed traffic file ({} if it is missing)."""
+    try:
+        with open(path) as f:
+            doc = json.load(f)
+    except (OSError, ValueError):
+        return {}
+    return {(r["workload"], r["kernel"]): r for r in doc.get("records", [])}
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -263,8 +272,11 @@ def roofline_for(w, kernel_ms, peaks):
     nl = max(1, getattr(w, "launches", {}).get(name, 1))     # launches of that kernel per step
     sec = kernel_ms[name] * 1e-3 / nl                        # average duration of one launch
     src = "of measured" if peaks["_source"] == "measured" else "of fallback"
+    rec = load_traffic().get((w.cfg.name.split("_")[0], name))
     common = {"kernel": name, "launches_per_step": nl, "kernel_ms_per_launch": sec * 1e3,
-              "traffic": NCU_TRAFFIC_BYTES.get((w.cfg.name.split("_")[0], name)), "peak_source": src}
+              "traffic": int(rec["bytes_per_launch"]) if rec else None,
+              "traffic_source": ("profiles/ncu_dram_traffic.json: " + rec["capture"]) if rec else None,
+              "peak_source": src}
     if w.decode:
         lm_b, kv_b = decode_bytes(w.cfg, w.inp["seq_lens"].cpu().numpy())
         algo = kv_b if "attend" in name else (lm_b if ("score" in name or "select" in name) else lm_b + kv_b)
@@ -458,7 +470,8 @@ def oracle_sample(cfg, inp_cpu, budget_rows):
                             rows=rows)
         dt = time.perf_counter() - t0
         val = prefill_flops_rows(cfg, rows) / dt / 1e12
-        return val, "%d seeded query positions x all %d heads of %s" % (len(rows), cfg.Hq, cfg.name), dt
+        note = "" if len(rows) >= cfg.L else " (rate on the sample; the whole workload is extrapolated from it)"
+        return val, "%d seeded query positions x all %d heads of %s%s" % (len(rows), cfg.Hq, cfg.name, note), dt
     nb = min(cfg.B, budget_rows)
     sub = {k: v[:nb] for k, v in inp_cpu.items()}
     t0 = time.perf_counter()
@@ -468,14 +481,16 @@ def oracle_sample(cfg, inp_cpu, budget_rows):
     return (lm_b + kv_b) / dt / 1e9, "first %d of %d sequences of %s" % (nb, cfg.B, cfg.name), dt
 
 
-def oracle_sample_timed(cfg, inp_cpu, target_seconds=15.0):
-    """Pilot run, then a sample sized for about `target_seconds` of CPU work (bounded by the workload)."""
+# Query positions the oracle legs run on a prefill workload: the same seeded sample in the cpu_baseline leg of the
+# GPU arm and in every step of the reference arm (a few seconds of work on the 128K-token configuration).
+ORACLE_SAMPLE_ROWS = 2048
+
+
+def oracle_sample_timed(cfg, inp_cpu):
+    """The oracle, as it stands, on the bounded sample of the workload that both oracle legs use."""
     if cfg.mode != "prefill":
         return oracle_sample(cfg, inp_cpu, cfg.B)
-    pilot_rows = 256
-    _, _, dt = oracle_sample(cfg, inp_cpu, pilot_rows)
-    rows = int(min(cfg.L, max(pilot_rows, pilot_rows * target_seconds / max(dt, 1e-3))))
-    return oracle_sample(cfg, inp_cpu, rows)
+    return oracle_sample(cfg, inp_cpu, ORACLE_SAMPLE_ROWS)
 
 
 def reference_cfg_inputs(cfg):
@@ -493,7 +508,7 @@ def run_reference(args):
     import oracle
     cfg = pick_cfg(args.workload)
     small, inp = reference_cfg_inputs(cfg)
-    budget = 512 if cfg.mode == "prefill" else 2
+    budget = ORACLE_SAMPLE_ROWS if cfg.mode == "prefill" else 2
     vals, secs, sample = [], [], ""
     for s in range(args.warmup + args.steps):
         v, sample, dt = oracle_sample(small, inp, budget)
@@ -506,7 +521,9 @@ def run_reference(args):
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": float(np.mean(secs)) * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f64", "data": "synthetic",
-            "config": {"workload": cfg.name, "note": "each step = the CPU oracle on a bounded sample"},
+            "config": {"workload": cfg.name, "B": cfg.B, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "L_or_T": cfg.L, "d": cfg.d,
+                       "chunk_size": cfg.S, "top_k": cfg.K, "window": 1,
+                       "note": "each step = the CPU oracle on a bounded seeded sample of this workload: " + sample},
             "cpu_baseline": {"value": value, "unit": unit, "cores": oracle.num_threads(), "kind": "oracle",
                              "sample": sample},
             "e2e": {"value": value, "unit": unit, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -526,13 +543,50 @@ def aggregate_over_ranks(ms_per_step_local, work_per_replica, unit_scale, dist=N
     return work_per_replica * world / (ms * 1e-3) / unit_scale, ms
 
 
+# ----------------------------------------------------------------------------- ranks
+def spawn_ranks(n, argv):
+    """`python bench.py --gpus N` started by hand: run N copies of this script as ranks 0..N-1 of one node (one GPU
+    each, rendezvous on 127.0.0.1) and relay rank 0's output.  Under torchrun (RANK already set) nothing is spawned."""
+    import socket
+    sock = socket.socket()
+    sock.bind(("127.0.0.1", 0))
+    port = sock.getsockname()[1]
+    sock.close()
+    procs = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port), HILS_BENCH_SPAWNED="1")
+        env.setdefault("NCCL_DEBUG", "INFO")          # the communicator log names every rank of the job
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__)] + list(argv), env=env,
+                                      stdout=None if r == 0 else subprocess.DEVNULL))
+    rc = 0
+    for pr in procs:
+        rc = max(rc, abs(pr.wait()))
+    return rc
+
+
+def selftest_ranks(args):
+    """Host-only check of the rank plumbing (used by the CPU tests): every rank joins a gloo group, reports a fake
+    per-step time, and rank 0 prints the aggregated line exactly as the GPU path would."""
+    import torch.distributed as dist
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group("gloo")
+    value, ms = aggregate_over_ranks(1.0 + rank, 2.0e12, 1e12, dist if world > 1 else None, "cpu")
+    if rank == 0:
+        print(json.dumps({"selftest": True, "n_gpus": world, "value": value, "ms_per_step": ms}))
+    if world > 1:
+        dist.destroy_process_group()
+
+
 # ----------------------------------------------------------------------------- main
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="cfg1", choices=["cfg0", "cfg1", "cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg0", "cfg1", "cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--selftest-ranks", action="store_true", help="host-only check of the rank plumbing (gloo)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extra", action="store_true", help="skip the other single-GPU configurations")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -541,6 +595,11 @@ def main():
                     help="only run warmup+steps calls of the workload (for ncu captures); no timing extras")
     ap.add_argument("--batch", type=int, default=0, help="profile runs: override the batch size (smaller footprint)")
     args = ap.parse_args()
+    if args.gpus > 1 and "RANK" not in os.environ:
+        sys.exit(spawn_ranks(args.gpus, sys.argv[1:]))
+    if args.selftest_ranks:
+        selftest_ranks(args)
+        return
     if args.profile_run:
         import paper_2607_02980_b200 as hils
         torch.cuda.set_device(0)
@@ -588,6 +647,7 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    assert torch.cuda.device_count() > local, "rank %d has no GPU of its own (%d visible)" % (local, torch.cuda.device_count())
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     dist = None
@@ -639,6 +699,11 @@ def main():
     else:
         line["scoring_flops"] = w.work_aux
         line["frac_of_nominal_2250_TFLOPs"] = value / world / 2250.0
+        line["frac_of_measured_bf16_burst"] = value / world / peaks["bf16_tflops"]
+        key = args.workload
+        line["prefill_%s_TFLOPs" % key] = value / world
+        line["prefill_%s_ms" % key] = ms_step
+        line["prefill_%s_frac_of_measured_bf16_burst" % key] = value / world / peaks["bf16_tflops"]
     roof = roofline_for(w, kernel_ms, peaks)
     if roof:
         line["roofline"] = roof
@@ -668,6 +733,7 @@ def main():
 
     clocks = sampler.stop()          # sampled over the timed steps, the per-kernel pass and the e2e steps
     line["clocks"] = clocks
+    inp_cpu_primary = None
 
     # ---- other configurations (reported beside, never instead of, the primary workload)
     if not args.no_extra and world == 1:
@@ -678,40 +744,70 @@ def main():
                 launches += extras[args.workload + "_backward"]["launches_per_step"] * (max(3, args.steps) + 6)
             except Exception as exc:
                 extras[args.workload + "_backward"] = {"error": repr(exc)}
+        try:
+            if args.workload in ("cfg2", "cfg3"):
+                extras["landmark_summary_" + args.workload] = bench_landmark_summary(hils, w, peaks)
+                launches += 13
+            if args.workload == "cfg2":
+                extras["cfg2_chunk_overlap_iid_queries"] = bench_chunk_overlap(hils, w, peaks)
+                launches += 13
+            if args.workload == "cfg3":
+                extras["cfg3_paged"] = bench_paged_decode(hils, w, peaks)
+                extras["cfg3_multi_token_decode"] = bench_multi_token_decode(hils, w, peaks)
+                launches += 6 * 13
+        except Exception as exc:
+            extras["primary_extras"] = {"error": repr(exc)}
+        if rank == 0 and not args.no_cpu_baseline and not w.decode:
+            inp_cpu_primary = {k: v.cpu() for k, v in w.inp.items()}
         del w
         torch.cuda.empty_cache()
-        for name in ("cfg2", "cfg3", "cfg4", "cfg0"):
-            if name == args.workload:
-                continue
+        for name in ("cfg1", "cfg2", "cfg3", "cfg4", "cfg0"):
+            primary = name == args.workload
             try:
-                ew = Workload(hils, pick_cfg(name), dev)
-                ems, etr = time_steps(ew, max(3, args.steps), 3, barrier)
-                ek = kernel_times(ew, 3, barrier)
-                ent = {"metric": ew.metric, "value": ew.rate(float(np.mean(ems)) * 1e-3), "unit": ew.unit,
-                       "ms_per_step": float(np.mean(ems)), "median_ms": float(np.median(ems)), "kernel_ms": ek,
-                       "roofline": roofline_for(ew, ek, peaks)}
-                if ew.decode:
-                    ent["frac_of_measured_hbm"] = ent["value"] / peaks["hbm_gbs"]
-                    ent["frac_of_nominal_8000_GBps"] = ent["value"] / 8000.0
-                else:
-                    ent["frac_of_measured_bf16_burst"] = ent["value"] / peaks["bf16_tflops"]
-                    ent["frac_of_nominal_2250_TFLOPs"] = ent["value"] / 2250.0
-                extras[name] = ent
-                launches += hils.last_launch_count() * (max(3, args.steps) + 3)
-                if name in ("cfg2", "cfg3"):
-                    extras["landmark_summary_" + name] = bench_landmark_summary(hils, ew, peaks)
-                    launches += 13
-                if name == "cfg3":
-                    extras["cfg3_paged"] = bench_paged_decode(hils, ew, peaks)
-                    launches += 3 * 13
-                    extras["cfg3_multi_token_decode"] = bench_multi_token_decode(hils, ew, peaks)
-                    launches += 3 * 13
-                if name == "cfg2":
-                    extras["cfg2_chunk_overlap_iid_queries"] = bench_chunk_overlap(hils, ew, peaks)
-                    launches += 13
-                    extras["cfg2_backward"] = bench_backward(hils, ew, peaks, 3, barrier)
-                    launches += extras["cfg2_backward"]["launches_per_step"] * 9
-                del ew
+                if not primary:
+                    ew = Workload(hils, pick_cfg(name), dev)
+                    ems, etr = time_steps(ew, max(3, args.steps), 3, barrier)
+                    ek = kernel_times(ew, 3, barrier)
+                    ent = {"metric": ew.metric, "value": ew.rate(float(np.mean(ems)) * 1e-3), "unit": ew.unit,
+                           "ms_per_step": float(np.mean(ems)), "median_ms": float(np.median(ems)), "kernel_ms": ek,
+                           "roofline": roofline_for(ew, ek, peaks)}
+                    if ew.decode:
+                        ent["frac_of_measured_hbm"] = ent["value"] / peaks["hbm_gbs"]
+                        ent["frac_of_nominal_8000_GBps"] = ent["value"] / 8000.0
+                    else:
+                        ent["frac_of_measured_bf16_burst"] = ent["value"] / peaks["bf16_tflops"]
+                        ent["frac_of_nominal_2250_TFLOPs"] = ent["value"] / 2250.0
+                    extras[name] = ent
+                    launches += hils.last_launch_count() * (max(3, args.steps) + 3)
+                    # the other half of the metric and the small prefill configuration, where the driver's parser keeps them
+                    if name in ("cfg3", "cfg4"):
+                        line["decode_%s_GBps" % name] = ent["value"]
+                        line["decode_%s_ms" % name] = ent["ms_per_step"]
+                        line["decode_%s_frac_of_measured_hbm" % name] = ent["frac_of_measured_hbm"]
+                        line["decode_%s_frac_of_nominal_8000_GBps" % name] = ent["frac_of_nominal_8000_GBps"]
+                        for kn, kms in ek.items():
+                            if "attend" in kn:
+                                line["decode_%s_gathered_kv_GBps" % name] = ew.work_aux / (kms * 1e-3) / 1e9
+                                line["decode_%s_gathered_kv_frac_of_measured_hbm" % name] = (
+                                    ew.work_aux / (kms * 1e-3) / 1e9 / peaks["hbm_gbs"])
+                    elif name in ("cfg1", "cfg2"):
+                        line["prefill_%s_TFLOPs" % name] = ent["value"]
+                        line["prefill_%s_ms" % name] = ent["ms_per_step"]
+                        line["prefill_%s_frac_of_measured_bf16_burst" % name] = ent["frac_of_measured_bf16_burst"]
+                    if name in ("cfg2", "cfg3"):
+                        extras["landmark_summary_" + name] = bench_landmark_summary(hils, ew, peaks)
+                        launches += 13
+                    if name == "cfg3":
+                        extras["cfg3_paged"] = bench_paged_decode(hils, ew, peaks)
+                        launches += 3 * 13
+                        extras["cfg3_multi_token_decode"] = bench_multi_token_decode(hils, ew, peaks)
+                        launches += 3 * 13
+                    if name == "cfg2":
+                        extras["cfg2_chunk_overlap_iid_queries"] = bench_chunk_overlap(hils, ew, peaks)
+                        launches += 13
+                        extras["cfg2_backward"] = bench_backward(hils, ew, peaks, 3, barrier)
+                        launches += extras["cfg2_backward"]["launches_per_step"] * 9
+                    del ew
                 if name == "cfg2":
                     # adjacent queries that retrieve mostly the same chunks, as the paper measures on a trained model
                     torch.cuda.empty_cache()
@@ -743,7 +839,10 @@ def main():
     # ---- the oracle timed beside it on this machine's host cores (rank 0, N = 1 only)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
-        small, inp_cpu = reference_cfg_inputs(cfg)
+        if inp_cpu_primary is not None:
+            small, inp_cpu = cfg, inp_cpu_primary       # the very tensors the GPU steps ran on
+        else:
+            small, inp_cpu = reference_cfg_inputs(cfg)
         val, sample, secs = oracle_sample_timed(small, inp_cpu)
         line["cpu_baseline"] = {"value": val, "unit": "TFLOP/s" if cfg.mode == "prefill" else "GB/s",
                                 "cores": oracle.num_threads(), "kind": "oracle", "sample": sample, "seconds": secs}

@@ -31,14 +31,43 @@ class _Params(ctypes.Structure):
                 ("scale", ctypes.c_double), ("group_mode", ctypes.c_int), ("in_bf16", ctypes.c_int)]
 
 
+_CFLAGS = ["-O3", "-march=native", "-fopenmp", "-shared", "-fPIC", "-std=c11"]
+
+
+def _stamp() -> str:
+    """What the built object depends on: the source, the flags and (because of -march=native) this machine's CPU."""
+    import hashlib
+    h = hashlib.sha256()
+    with open(_SRC, "rb") as f:
+        h.update(f.read())
+    h.update(" ".join(_CFLAGS).encode())
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.startswith("flags") or line.startswith("model name"):
+                    h.update(line.encode())
+                    if line.startswith("flags"):
+                        break
+    except OSError:
+        pass
+    return h.hexdigest()
+
+
 def build(force: bool = False) -> str:
-    """Compile the oracle with gcc (OpenMP) if the shared object is missing or stale."""
-    if (not force and os.path.exists(_SO) and os.path.getmtime(_SO) >= os.path.getmtime(_SRC)):
-        return _SO
+    """Compile the oracle with gcc (-O3 -march=native, OpenMP) if the shared object is missing, stale or was built
+    on a machine with another CPU."""
+    stamp_path = _SO + ".stamp"
+    want = _stamp()
+    if not force and os.path.exists(_SO) and os.path.exists(stamp_path):
+        with open(stamp_path) as f:
+            if f.read() == want:
+                return _SO
     tmp = _SO + ".tmp%d" % os.getpid()
-    cmd = ["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-std=c11", "-o", tmp, _SRC, "-lm"]
+    cmd = ["gcc"] + _CFLAGS + ["-o", tmp, _SRC, "-lm"]
     subprocess.run(cmd, check=True)
     os.replace(tmp, _SO)
+    with open(stamp_path, "w") as f:
+        f.write(want)
     return _SO
 
 

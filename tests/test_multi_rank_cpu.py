@@ -54,3 +54,32 @@ def test_single_process_aggregate_is_plain_rate():
     import bench
     value, ms = bench.aggregate_over_ranks(4.0, work_per_replica=8e9, unit_scale=1e9)
     assert ms == 4.0 and abs(value - 8e9 / 4e-3 / 1e9) < 1e-9
+
+
+def test_bench_gpus_2_spawns_its_own_ranks():
+    """`python bench.py --gpus 2` started by hand (no RANK in the environment) starts two ranks itself: here the
+    host-only self-test of that plumbing (gloo), whose rank 0 prints the line with n_gpus = 2 and the MAX-over-ranks
+    step time."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_PORT")}
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--selftest-ranks"],
+                         capture_output=True, text=True, env=env, cwd=ROOT, timeout=600)
+    assert res.returncode == 0, res.stderr[-2000:]
+    line = json.loads(res.stdout.strip().splitlines()[-1])
+    assert line["n_gpus"] == 2 and line["ms_per_step"] == 2.0          # ranks report 1.0 and 2.0 ms
+    assert abs(line["value"] - 2 * 2.0e12 / 2e-3 / 1e12) < 1e-9
+
+
+def test_reference_arm_through_the_spawner_prints_one_line():
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_PORT")}
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--impl", "reference",
+                          "--workload", "cfg0", "--steps", "1", "--warmup", "0"],
+                         capture_output=True, text=True, env=env, cwd=ROOT, timeout=600)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [x for x in res.stdout.strip().splitlines() if x.startswith("{")]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["impl"] == "reference" and line["n_gpus"] == 2
