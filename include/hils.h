@@ -26,8 +26,10 @@
  *
  * Conventions
  *   - Every pointer is a DEVICE pointer owned by the caller unless the entry point says HOST.
- *   - The library never allocates, frees or synchronises (except where stated); all work is
- *     enqueued on `stream`.  Outputs are fully overwritten.
+ *   - The library never allocates, frees or synchronises; all work is enqueued on `stream`.  Outputs are fully
+ *     overwritten.  The exceptions say so at their declarations: hils_prefill_host / hils_decode_host (three
+ *     internal streams and ten events per device, created on first use, and a process-wide mutex around a call),
+ *     hils_trace_enable (1025 events on first use), hils_trace_read and hils_poll_status (they wait for the stream).
  *   - Tensors are contiguous, last dimension fastest, base pointers 16-byte aligned:
  *       q, out      [B, Hq, L, d]          (decode: [B, Hq, d])
  *       k, v        [B, Hkv, T, d]         T = L for prefill, T_max for decode
@@ -123,8 +125,8 @@ int hils_decode(const hils_params* params, const void* q, const void* k_cache, c
  * the process exits.  The caller still passes every input and output.
  *
  *  - Nothing is allocated or freed, by CUDA or otherwise, on any call.
- *  - Limit: 256 + hils_workspace_bytes(params, 1) must fit in 8 MiB, otherwise HILS_ERR_WORKSPACE is
- *    returned before anything is launched (both benchmark decode shapes fit: B=64 x 64K tokens with
+ *  - Limit: the decode workspace of the shape, hils_workspace_bytes(params, 1) (its 256-byte status block
+ *    included), must fit in 8 MiB, otherwise HILS_ERR_WORKSPACE is returned before anything is launched (both benchmark decode shapes fit: B=64 x 64K tokens with
  *    K=32 needs about 5.3 MiB, B=4 x 1M tokens with K=64 about 2.5 MiB).  Shapes outside the
  *    bandwidth-tuned decode kernels (bf16, d=128, chunk 64, window <= 897, one landmark per KV or per query head,
  *    at most 8 query heads per KV head) return HILS_ERR_UNSUPPORTED.

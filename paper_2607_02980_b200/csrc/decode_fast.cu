@@ -932,6 +932,8 @@ int launch_decode_noalloc(const Shape& s, const Tensors& t_in, int32_t* device_s
     if (dev < 0 || dev >= kMaxDevices) return HILS_ERR_UNSUPPORTED;
     // In host code `g_noalloc_scratch` is only a handle for the symbol, not an address a kernel can
     // use: the device address is looked up once per device, with that device current.
+    // (No lock around this cache: two host threads that make a device's first call at the same moment both look the
+    // address up and both store the same value.)
     static void* dev_ptr[kMaxDevices] = {};
     if (!dev_ptr[dev]) {
         void* p = nullptr;

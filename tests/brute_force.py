@@ -9,10 +9,13 @@ from the C oracle on purpose.  Used only to pin the oracle.
 import numpy as np
 
 
-def brute_force_prefill(q, k, v, landmarks, bias, S, K, W=1, scale=None, q_route=None):
+def brute_force_prefill(q, k, v, landmarks, bias, S, K, W=1, scale=None, q_route=None, group_mode=0):
     """q [Hq,L,d], k,v [Hkv,L,d], landmarks [Hl,C,d], bias [Hl,C] or None (one sequence).
 
     q_route [Hq,L,d] or None: the routing query of Eq. (Q-Cal); it takes q's place in the surrogate scores only.
+    group_mode 0: group score = max over the group's heads of the raw surrogate score (App. C);
+    group_mode 1: each head's scores are first turned into weights over the row's candidates (a softmax over the
+    candidate chunks), the group score is the largest weight any head gives the chunk (the wording of Sec. 4.1).
 
     Returns (out [Hq,L,d], lse [Hq,L], sel list-of-lists [Hkv][L] (ascending ids), weights [Hq,L,L]).
     """
@@ -36,7 +39,14 @@ def brute_force_prefill(q, k, v, landmarks, bias, S, K, W=1, scale=None, q_route
                 hl = h if Hl == Hq else g
                 for c in range(ncand):
                     shat[r, c] = scale * (qhat[h, i] @ landmarks[hl, c]) + (0.0 if bias is None else bias[hl, c])
-            u = shat.max(axis=0) if ncand > 0 else np.zeros(0)
+            if ncand == 0:
+                u = np.zeros(0)
+            elif group_mode == 0:
+                u = shat.max(axis=0)
+            else:
+                wgt = np.exp(shat)                            # raw exponentials: the inputs here are small
+                wgt = wgt / wgt.sum(axis=1, keepdims=True)
+                u = wgt.max(axis=0)
             order = sorted(range(ncand), key=lambda c: (-u[c], c))
             chosen = sorted(order[:K])
             sel[g][i] = chosen

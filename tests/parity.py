@@ -4,7 +4,9 @@ Acceptance:
   * sel_idx bit-exact, except rows where the oracle's K-th and (K+1)-th group scores differ by
     less than 1e-3 ("exempt" rows); a mismatch on a row with margin >= 1e-3 fails;
   * on exempt rows that differ, the GPU's selection must still be valid (ascending, distinct,
-    in range, right count) and `out` is compared with the oracle attending the GPU's selection;
+    in range, right count), it may differ from the oracle's only inside the tie band -- every chunk it took
+    scores at least (K-th best - 1e-3) and every chunk it left out at most (K-th best + 1e-3), with the group
+    scores recomputed here in fp64 -- and `out` is compared with the oracle attending the GPU's selection;
   * out: max-abs 1e-4 (fp32) / 2e-2 (bf16 inputs, fp32 accumulation, oracle output unrounded);
   * lse: 1e-4 (fp32) / 1e-3 (bf16).
 """
@@ -31,10 +33,45 @@ def check_selection_valid(sel_row, ncand, K):
     assert all(0 <= c < ncand for c in ids), "chunk id outside the candidate range"
 
 
-def compare_rows(dtype, K, S, W, ref, gpu_sel, gpu_out, gpu_lse, row_pos, rerun):
+def group_scores(q_row, lm, bias, ncand, scale=None):
+    """Per-head surrogate scores s[h, c] = scale * q^h . k'_c + b'_c (Eq. surrogate top-k) of one query row for the
+    candidates c < ncand, in fp64; the group score of App. C is their maximum over a KV group's heads.
+    q_row [Hq, d]; lm [Hl, C, d] with Hl = Hkv or Hq; bias [Hl, C] or None."""
+    q_row = np.asarray(q_row, np.float64)
+    lm = np.asarray(lm, np.float64)[:, :ncand]
+    Hq, d = q_row.shape
+    Hl = lm.shape[0]
+    scale = 1.0 / np.sqrt(d) if scale is None else scale
+    if Hl == Hq:
+        s = scale * np.einsum("hd,hcd->hc", q_row, lm)
+        if bias is not None:
+            s = s + np.asarray(bias, np.float64)[:, :ncand]
+    else:
+        G = Hq // Hl
+        s = scale * np.einsum("hd,hcd->hc", q_row, np.repeat(lm, G, axis=0))
+        if bias is not None:
+            s = s + np.repeat(np.asarray(bias, np.float64)[:, :ncand], G, axis=0)
+    return s
+
+
+def check_selection_in_tie_band(sel_row, u, K):
+    """sel_row: the GPU's chunk ids of one (row, KV group); u [ncand]: the group's scores.  Whatever differs from
+    the exact top-K must lie within MARGIN of the K-th best score."""
+    ncand = u.shape[0]
+    if ncand <= K:
+        return
+    kth = np.sort(u)[ncand - K]
+    taken = np.zeros(ncand, bool)
+    taken[[int(c) for c in sel_row if c >= 0]] = True
+    assert (u[taken] >= kth - MARGIN).all(), "took a chunk scoring %g below the K-th best %g" % (u[taken].min(), kth)
+    assert (u[~taken] <= kth + MARGIN).all(), "left out a chunk scoring %g above the K-th best %g" % (u[~taken].max(), kth)
+
+
+def compare_rows(dtype, K, S, W, ref, gpu_sel, gpu_out, gpu_lse, row_pos, rerun, scores=None):
     """ref: oracle dict indexed [n, ...]; gpu_*: numpy arrays indexed [n, Hkv|Hq, ...].
 
-    `rerun(rows_subset_indices, sel)` must return the oracle dict attending the given selection.
+    `rerun(rows_subset_indices, sel)` must return the oracle dict attending the given selection;
+    `scores(row_index, ncand)` the per-head surrogate scores [Hq, ncand] of that row (fp64).
     Returns a stats dict; raises AssertionError on a violation.
     """
     n, Hkv = gpu_sel.shape[0], gpu_sel.shape[1]
@@ -50,8 +87,11 @@ def compare_rows(dtype, K, S, W, ref, gpu_sel, gpu_out, gpu_lse, row_pos, rerun)
     if len(rows_m):
         for r in rows_m:
             lo = max(0, ((int(row_pos[r]) - W + 1) // S) * S)
+            sh = scores(r, lo // S) if (scores is not None and lo // S > K) else None
             for g in range(Hkv):
                 check_selection_valid(gpu_sel[r, g], lo // S, K)
+                if sh is not None and mism[r, g]:
+                    check_selection_in_tie_band(gpu_sel[r, g], sh[g * G:(g + 1) * G].max(axis=0), K)
         alt = rerun(rows_m, gpu_sel[rows_m])
         ref_out[rows_m] = alt["out"]
         ref_lse[rows_m] = alt["lse"]
@@ -87,7 +127,11 @@ def check_prefill(cfg, inp_cpu, out, lse, sel, rows=None, bias=None, W=1):
                                     rows=rows[idx], sel_idx=sel_sub[None])
             return {k_: v_[0] for k_, v_ in r.items()}
 
-        stats.append(compare_rows(cfg.dtype, cfg.K, cfg.S, W, refb, g_sel, g_out, g_lse, rows, rerun))
+        def scores(r, ncand, b=b):
+            return group_scores(inp_cpu["q"][b, :, int(rows[r])].float().numpy(), inp_cpu["landmarks"][b].float().numpy(),
+                                None if bias is None else _np(bias[b]), ncand)
+
+        stats.append(compare_rows(cfg.dtype, cfg.K, cfg.S, W, refb, g_sel, g_out, g_lse, rows, rerun, scores))
     return stats
 
 
@@ -102,4 +146,8 @@ def check_decode(cfg, inp_cpu, out, lse, sel, bias=None, W=1):
         return oracle.hils_decode(sub["q"], sub["k"], sub["v"], sub["landmarks"], bb, seq[idx], S=cfg.S, K=cfg.K,
                                   W=W, sel_idx=sel_sub)
 
-    return compare_rows(cfg.dtype, cfg.K, cfg.S, W, ref, sel.cpu().numpy(), _np(out), _np(lse), seq - 1, rerun)
+    def scores(r, ncand):
+        return group_scores(inp_cpu["q"][r].float().numpy(), inp_cpu["landmarks"][r].float().numpy(),
+                            None if bias is None else _np(bias[r]), ncand)
+
+    return compare_rows(cfg.dtype, cfg.K, cfg.S, W, ref, sel.cpu().numpy(), _np(out), _np(lse), seq - 1, rerun, scores)

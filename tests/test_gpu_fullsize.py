@@ -42,38 +42,48 @@ def check_prefill_rows(cfg, cpu, out, lse, sel, rows):
 
 def test_cfg1_gqa_bf16_prefill_16k_sampled_rows():
     args = prefill_full(wl.CONFIGS[1], 2048)
-    stats = check_prefill_rows(*args)
-    print(stats)
-    assert stats[0]["mismatch_rows"] <= stats[0]["exempt_rows"]
+    report("cfg1", check_prefill_rows(*args)[0])
 
 
 def test_cfg2_long_bf16_prefill_128k_sampled_rows():
     args = prefill_full(wl.CONFIGS[2], 4096)
-    stats = check_prefill_rows(*args)
-    print(stats)
+    report("cfg2", check_prefill_rows(*args)[0])
 
 
-def decode_full(cfg, seqs):
+def decode_full(cfg, per_batch):
+    """Every sequence of the configuration against the oracle, `per_batch` sequences' cache slabs on the host at a time."""
     inp = wl.make_decode_inputs(cfg, DEV)
     out, lse, sel = hils.hils_decode(inp["q"], inp["k"], inp["v"], inp["landmarks"], inp["seq_lens"], cfg.S, cfg.K)
     torch.cuda.synchronize()
-    s = torch.as_tensor(seqs, device=DEV)
-    cpu = {k: v[s].cpu() for k, v in inp.items()}
-    sub = cfg.scaled(B=len(seqs))
-    stats = check_decode(sub, cpu, out[s], lse[s], sel[s])
-    # every sequence: selection is valid and outputs are finite
     sel_c = sel.cpu().numpy()
     assert (sel_c >= 0).all() and (np.diff(sel_c, axis=-1) > 0).all() and (sel_c < cfg.C - 1).all()
     assert torch.isfinite(out.float()).all() and torch.isfinite(lse).all()
-    return stats
+    total = {"rows": 0, "exempt_rows": 0, "mismatch_rows": 0, "max_err_out": 0.0, "max_err_lse": 0.0}
+    for b0 in range(0, cfg.B, per_batch):
+        s = torch.arange(b0, min(cfg.B, b0 + per_batch), device=DEV)
+        cpu = {k: v[s].cpu() for k, v in inp.items()}
+        st = check_decode(cfg.scaled(B=len(s)), cpu, out[s], lse[s], sel[s])
+        for key in ("rows", "exempt_rows", "mismatch_rows"):
+            total[key] += st[key]
+        for key in ("max_err_out", "max_err_lse"):
+            total[key] = max(total[key], st[key])
+    assert total["rows"] == cfg.B
+    return total
 
 
-def test_cfg3_batched_decode_sampled_sequences():
-    print(decode_full(wl.CONFIGS[3], [0, 17, 42, 63]))
+def report(name, stats):
+    """Selections differ from the oracle's only on rows inside the 1e-3 tie band (compare_rows has already rejected any
+    other mismatch and any swap outside the band); the counts go to the test log."""
+    print("%s: %s" % (name, stats))
+    assert stats["mismatch_rows"] <= stats["exempt_rows"]
 
 
-def test_cfg4_ultralong_decode_sampled_sequences():
-    print(decode_full(wl.CONFIGS[4], [1, 3]))
+def test_cfg3_batched_decode_every_sequence():
+    report("cfg3", decode_full(wl.CONFIGS[3], 8))
+
+
+def test_cfg4_ultralong_decode_every_sequence():
+    report("cfg4", decode_full(wl.CONFIGS[4], 1))
 
 
 def test_cfg2_shape_with_the_papers_window_and_bias_sampled_rows():
@@ -95,7 +105,7 @@ def test_cfg2_shape_with_the_papers_window_and_bias_sampled_rows():
     full_out[:, :, r] = out[:, :, ridx].float().cpu()
     full_lse[:, :, r] = lse[:, :, ridx].cpu()
     full_sel[:, :, r] = sel[:, :, ridx].cpu()
-    print(check_prefill(cfg, cpu, full_out, full_lse, full_sel, rows=rows, bias=bias.cpu(), W=512))
+    report("cfg2 W=512 bias", check_prefill(cfg, cpu, full_out, full_lse, full_sel, rows=rows, bias=bias.cpu(), W=512)[0])
 
 
 def test_cfg3_paged_and_windowed_decode_sampled_sequences():
@@ -123,7 +133,7 @@ def test_cfg3_paged_and_windowed_decode_sampled_sequences():
     assert torch.equal(sel_p, sel_c) and torch.equal(out_p, out_c) and torch.equal(lse_p, lse_c)
     s = torch.as_tensor([0, 17, 63], device=DEV)
     cpu = {k: v[s].cpu() for k, v in inp.items()}
-    print(check_decode(cfg.scaled(B=3), cpu, out_p[s], lse_p[s], sel_p[s], bias=bias[s].cpu(), W=512))
+    report("cfg3 paged W=512 bias", check_decode(cfg.scaled(B=3), cpu, out_p[s], lse_p[s], sel_p[s], bias=bias[s].cpu(), W=512))
 
 
 def test_landmark_summary_on_the_cfg3_key_cache_sampled_sequences():

@@ -380,6 +380,29 @@ def test_normalised_group_mode_is_available_and_differs_only_in_selection():
     np.testing.assert_allclose(a["out"], b["out"], atol=0)
 
 
+@pytest.mark.parametrize("G,Hl_is_Hq,W,with_bias", [(2, False, 1, False), (4, False, 1, True), (4, True, 11, True),
+                                                     (2, True, 1, False)])
+def test_normalised_group_mode_matches_the_brute_force_for_several_heads(G, Hl_is_Hq, W, with_bias):
+    """The Sec. 4.1 reading (per-head softmax over the candidate chunks, then the maximum over the group's heads)
+    against the independent dense-weight program, for G > 1 where it differs from the App. C rule: same selection,
+    same outputs; and the two readings do pick different chunks somewhere on these inputs."""
+    S, K, Hkv, L = 4, 3, 2, 72
+    Hq = Hkv * G
+    q, k, v, lm, bias = rand_inputs(40 + G + W, Hq=Hq, Hkv=Hkv, L=L, d=8, S=S, Hl=Hq if Hl_is_Hq else Hkv,
+                                    amp=1.5, with_bias=with_bias)
+    res = oracle.hils_prefill(q, k, v, lm, bias, S=S, K=K, W=W, group_mode=1)
+    bo, blse, bsel, _ = brute_force_prefill(q[0], k[0], v[0], lm[0], None if bias is None else bias[0], S, K, W=W,
+                                            group_mode=1)
+    for g in range(Hkv):
+        for i in range(L):
+            got = [int(c) for c in res["sel_idx"][0, i, g] if c >= 0]
+            assert got == bsel[g][i], (g, i)
+    np.testing.assert_allclose(res["out"][0].transpose(1, 0, 2), bo, atol=1e-11)
+    np.testing.assert_allclose(res["lse"][0].T, blse, atol=1e-11)
+    raw = oracle.hils_prefill(q, k, v, lm, bias, S=S, K=K, W=W, group_mode=0)
+    assert (raw["sel_idx"] != res["sel_idx"]).any(), "inputs on which the two GQA readings agree pin nothing"
+
+
 # ---------------------------------------------------------------------------------------------------------------
 # Routing query (Eq. Q-Cal): q-hat replaces q in the surrogate scores only
 def test_routing_query_equal_to_q_changes_nothing_and_a_different_one_only_moves_scores():

@@ -9,6 +9,7 @@ import torch
 
 import paper_2607_02980_b200 as hils
 from paper_2607_02980_b200 import workloads as wl
+from parity import check_decode
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
@@ -31,13 +32,41 @@ def _run_pair(cfg, seq, query_set):
     assert torch.equal(sel, ref_sel)
     assert (out.float() - ref_out.float()).abs().max().item() <= TOL_OUT
     assert (lse - ref_lse).abs().max().item() <= TOL_LSE
+    return inp, out, lse, sel
 
 
 def test_noalloc_matches_hils_decode_on_two_calls_in_a_row():
     # first call: many pairs, ragged lengths (also leaves partial sums and counters behind)
     _run_pair(wl.CONFIGS[3].scaled(B=16, L=4096, K=16, seed=71), [4096 - 97 * i for i in range(16)], 0)
-    # second call: another shape and other queries over the same static scratch
-    _run_pair(wl.CONFIGS[4].scaled(B=2, L=16384, K=64, seed=72), [16384, 9001], 1)
+    # second call: another shape and other queries over the same static scratch; this one also against the CPU oracle
+    cfg = wl.CONFIGS[4].scaled(B=2, L=16384, K=64, seed=72)
+    inp, out, lse, sel = _run_pair(cfg, [16384, 9001], 1)
+    check_decode(cfg, inp, out, lse, sel)
+
+
+def test_noalloc_clears_the_status_word_a_failed_call_left_in_the_shared_array():
+    """A call with an impossible sequence length reports it through device_status (the bounds check skips the
+    sequence, nothing faults); the word it leaves in the static array must not show up in the next call's status."""
+    cfg = wl.CONFIGS[3].scaled(B=2, L=1024, K=4, seed=74)
+    inp = wl.make_decode_inputs(cfg, "cpu", seq_lens=torch.tensor([1024, 512], dtype=torch.int32))
+    g = {k: v.to(DEV) for k, v in inp.items()}
+    out = torch.empty_like(g["q"])
+    lse = torch.empty((cfg.B, cfg.Hq), dtype=torch.float32, device=DEV)
+    sel = torch.empty((cfg.B, cfg.Hkv, cfg.K), dtype=torch.int32, device=DEV)
+    status = torch.zeros((1,), dtype=torch.int32, device=DEV)
+    bad = torch.tensor([1024, 0], dtype=torch.int32, device=DEV)
+    hils.hils_decode_noalloc(g["q"], g["k"], g["v"], g["landmarks"], bad, cfg.S, cfg.K, out, lse, sel, device_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 2                  # bad index recorded, sequence skipped
+    assert (sel[1] == -1).all()
+    hils.hils_decode_noalloc(g["q"], g["k"], g["v"], g["landmarks"], g["seq_lens"], cfg.S, cfg.K, out, lse, sel,
+                             device_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    ref_out, ref_lse, ref_sel = hils.hils_decode(g["q"], g["k"], g["v"], g["landmarks"], g["seq_lens"], cfg.S, cfg.K)
+    assert torch.equal(sel, ref_sel)
+    assert (out.float() - ref_out.float()).abs().max().item() <= TOL_OUT
+    assert (lse - ref_lse).abs().max().item() <= TOL_LSE
 
 
 def test_noalloc_rejects_shapes_beyond_its_fixed_scratch():
