@@ -4,8 +4,8 @@
 //   decode_score   streams the landmarks of every (sequence, KV head) once with 128-bit loads and
 //                  scores them against the G query heads with warp MMA (landmark rows are the A
 //                  operand straight from global memory); writes the group score u_c = max_h s^h_c.
-//   decode_select  one CTA per (sequence, KV head): exact top-K of u (ties to the lower chunk id) as a tree
-//                  of warp-level selections (linear-bin histogram + exact ranks in the boundary bin),
+//   decode_select  one CTA per (sequence, KV head): exact top-K of u (ties to the lower chunk id) by radix
+//                  selection on the ordered score keys (8 bits per pass over keys cached in shared memory),
 //                  ascending ids, then the per-head surrogate scores of the selected chunks and the
 //                  fusion weights exp(s^h_c - max_c s^h_c).
 //   decode_attend  persistent CTAs over a flat list of (pair, slot) items; K/V chunks arrive through
@@ -14,6 +14,21 @@
 //                  finishes a pair last mixes the partial sums with the local branch (App. C).
 #include "internal.h"
 #include "tma.cuh"
+#ifdef X_STAMP
+namespace hils { __device__ unsigned long long g_dbg[16]; }
+__device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+#define STAMP_MIN(i) if (threadIdx.x == 0) atomicMin(&hils::g_dbg[i], gtime())
+#define STAMP_MAX(i) if (threadIdx.x == 0) atomicMax(&hils::g_dbg[i], gtime())
+extern "C" void hils_debug_stamps(unsigned long long* out, int reset) {
+    unsigned long long h[16];
+    cudaMemcpyFromSymbol(h, hils::g_dbg, sizeof(h));
+    for (int i = 0; i < 16; ++i) out[i] = h[i];
+    if (reset) { for (int i = 0; i < 16; ++i) h[i] = (i & 1) ? 0ull : ~0ull; cudaMemcpyToSymbol(hils::g_dbg, h, sizeof(h)); }
+}
+#else
+#define STAMP_MIN(i)
+#define STAMP_MAX(i)
+#endif
 
 namespace hils {
 namespace {
@@ -72,170 +87,104 @@ __device__ __forceinline__ int query_seq_len(const DArgs& a, int b) {
 __device__ __forceinline__ int first_local_chunk(int seq, int W) { return local_lo(seq - 1, W, kS) / kS; }
 
 // ------------------------------------------------------------------------------------------ select
-// Exact top-K as a tree of warp-level selections.  A warp stages up to kSelCap candidates (ordered score
-// key + chunk id) in its own shared-memory buffer, bins the scores linearly between the buffer's minimum
-// and maximum (128 warp-private counters), finds the bin that holds the K-th best, takes everything above
-// it and ranks the few candidates inside it exactly (score, then lower chunk id).  Level 1 runs one such
-// selection per warp over its slice of the pair's candidates; the survivor lists are then merged, kSelCap / K
-// lists per warp and round, until one list is left.  A member of the global top-K is in the top-K of every
-// subset that holds it, so the result is exact.  All loops are rolled on purpose: the code runs once per
-// CTA, so its size (instruction fetch), not its instruction count, sets the pace.
+// Exact top-K by radix selection on the ordered score keys, one CTA per (sequence, KV head) pair.  The K-th best key T
+// is found digit by digit (four passes of 8 bits, most significant first): every pass histograms the digit of the
+// candidates that still match the prefix found so far (one private histogram per warp: equal digits are the rule in
+// the leading, exponent, byte), sums the histograms and walks the 256 bins from the top until K candidates are
+// covered.  Chunks with a key above T are selected; of those equal to T as many as are still missing, lowest chunk ids
+// first -- if there are more than that, a second selection of the same kind runs on their ids.  The keys are cached
+// in shared memory after the first pass (they come from L2) when they fit.  Integer arithmetic throughout: exact and
+// independent of the thread count.
 constexpr int kSelMaxK = 128;
-constexpr int kSelCap = 1024 + kSelMaxK;     // staged candidates per warp: a slice round + carried survivors
-constexpr int kSelBins = 128;
-constexpr int kSelEdge = 64;                 // candidates of the boundary bin that are ranked pairwise
+constexpr int kSelMaxWarps = 32;
+constexpr int kSelKeyCap = 40960;            // keys cached in shared memory (160 KB); longer lists re-read the scores
 
-struct SelWarp {                             // one per warp, in dynamic shared memory
-    unsigned key[kSelCap];                   // ordered score keys (>= 1)
-    int id[kSelCap];                         // chunk ids
-    unsigned long long list[kSelMaxK];       // survivors (key << 32 | id), unordered
-    unsigned long long edge[kSelEdge];       // boundary-bin candidates (key << 32 | ~id)
-    int hist[kSelBins];
-    int cnt;                                 // entries of list
+struct SelState {
+    int hist[256];                           // summed histogram of the current pass
+    unsigned prefix, mask;                   // digits fixed so far
+    int remaining;                           // how many candidates matching the prefix are still wanted from the top
+    int equal;                               // candidates whose key equals the finished prefix
+    int nout;                                // selected so far
 };
 
-// Selects the best min(K, n) of the n staged candidates of w into w.list / w.cnt.
-__device__ __noinline__ void warp_select(SelWarp& w, int n, int K, int lane) {
-    int nout = 0;
-    if (n <= K) {
-        for (int i = lane; i < n; i += 32) w.list[i] = (static_cast<unsigned long long>(w.key[i]) << 32) | static_cast<unsigned>(w.id[i]);
-        nout = n;
-    } else {
-        unsigned kmax = 0u, kmin = 0xffffffffu;
-#pragma unroll 4
-        for (int i = lane; i < n; i += 32) { kmax = max(kmax, w.key[i]); kmin = min(kmin, w.key[i]); }
-        kmax = __reduce_max_sync(kFullMask, kmax);
-        kmin = __reduce_min_sync(kFullMask, kmin);
-        // monotone linear binning of the scores between the extremes
-        const float lo = key_to_float(kmin), hi = key_to_float(kmax);
-        const float inv = hi > lo ? static_cast<float>(kSelBins - 1) / (hi - lo) : 0.f;
-        for (int x = lane; x < kSelBins; x += 32) w.hist[x] = 0;
-        __syncwarp();
-#pragma unroll 4
-        for (int i = lane; i < n; i += 32)
-            atomicAdd(&w.hist[max(0, min(kSelBins - 1, static_cast<int>((key_to_float(w.key[i]) - lo) * inv)))], 1);
-        __syncwarp();
-        // boundary bin b*: the highest bin with count(bin >= b*) >= K; lane l owns bins 127-4l .. 124-4l
-        int tsum = 0;
-        for (int x = 0; x < 4; ++x) tsum += w.hist[kSelBins - 1 - 4 * lane - x];
-        int inc = tsum;
-        for (int o = 1; o < 32; o <<= 1) {
-            const int nn = __shfl_up_sync(kFullMask, inc, o);
-            if (lane >= o) inc += nn;
-        }
-        int cum = inc - tsum, bstar = -1, above = 0;
-        if (cum < K && inc >= K) {
-            for (int x = 0; x < 4 && bstar < 0; ++x) {
-                const int h = w.hist[kSelBins - 1 - 4 * lane - x];
-                if (cum + h >= K) { bstar = kSelBins - 1 - 4 * lane - x; above = cum; }
-                cum += h;
+// One selection: the `want`-th largest value of val(i) over the candidates i in [0, n) for which live(i) holds
+// (bits [top_bit, 0] are examined, 8 at a time).  Returns the value; `equal` = how many live candidates hold exactly
+// that value, `remaining` = how many of those are wanted.  Called by every thread of the CTA.
+template <typename Val, typename Live>
+__device__ unsigned radix_kth(SelState& st, int (*whist)[256], int n, int want, int top_shift, Val val, Live live,
+                          bool first_hist_ready = false) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, NT = blockDim.x, nw = NT >> 5;
+    if (tid == 0) { st.prefix = 0u; st.mask = 0u; st.remaining = want; }
+    if (!first_hist_ready)
+        for (int x = lane; x < 256; x += 32) whist[warp][x] = 0;
+    __syncthreads();
+    for (int shift = top_shift; shift >= 0; shift -= 8) {
+        const unsigned prefix = st.prefix, mask = st.mask;
+        if (!(first_hist_ready && shift == top_shift)) {
+            for (int i = tid; i < n; i += NT) {
+                if (!live(i)) continue;
+                const unsigned v = val(i);
+                if ((v & mask) == prefix) atomicAdd(&whist[warp][(v >> shift) & 255u], 1);
             }
         }
-        const int src = __ffs(__ballot_sync(kFullMask, bstar >= 0)) - 1;      // exactly one lane found it
-        bstar = __shfl_sync(kFullMask, bstar, src);
-        above = __shfl_sync(kFullMask, above, src);
-        const int quota = K - above;          // >= 1 candidates of the boundary bin survive
-        const int m = w.hist[bstar];          // its population (>= quota)
-        const bool rank_edge = m != quota && m <= kSelEdge;
-        // everything above the boundary bin survives; the boundary bin goes to the edge list (or survives whole)
-        int nedge = 0;
-#pragma unroll 2
-        for (int i0 = 0; i0 < n; i0 += 32) {
-            const int i = i0 + lane;
-            int bin = -1;
-            unsigned k = 0u;
-            int c = 0;
-            if (i < n) {
-                k = w.key[i];
-                c = w.id[i];
-                bin = max(0, min(kSelBins - 1, static_cast<int>((key_to_float(k) - lo) * inv)));
-            }
-            const bool tk = bin > bstar || (bin == bstar && m == quota);
-            const unsigned bt = __ballot_sync(kFullMask, tk);
-            if (tk) w.list[nout + __popc(bt & ((1u << lane) - 1u))] = (static_cast<unsigned long long>(k) << 32) | static_cast<unsigned>(c);
-            nout += __popc(bt);
-            const bool ed = bin == bstar && rank_edge;
-            const unsigned be = __ballot_sync(kFullMask, ed);
-            if (ed) w.edge[nedge + __popc(be & ((1u << lane) - 1u))] = (static_cast<unsigned long long>(k) << 32) | (0xffffffffu - static_cast<unsigned>(c));
-            nedge += __popc(be);
+        __syncthreads();
+        // sum of the warps' histograms (left zeroed for the next pass)
+        for (int x = tid; x < 256; x += NT) {
+            int sum = 0;
+#pragma unroll 8
+            for (int w = 0; w < nw; ++w) { sum += whist[w][x]; whist[w][x] = 0; }
+            st.hist[x] = sum;
         }
-        __syncwarp();
-        if (rank_edge) {
-            // pairwise ranks inside the boundary bin (full keys: score, then lower id)
-            for (int e0 = 0; e0 < m; e0 += 32) {
-                const int e = e0 + lane;
-                const unsigned long long mine = e < m ? w.edge[e] : 0ull;
-                int rank = 0;
-                for (int j = 0; j < m; ++j) rank += w.edge[j] > mine ? 1 : 0;
-                const bool tk = e < m && rank < quota;
-                const unsigned bt = __ballot_sync(kFullMask, tk);
-                if (tk) w.list[nout + __popc(bt & ((1u << lane) - 1u))] = (mine & 0xffffffff00000000ull) | (0xffffffffu - static_cast<unsigned>(mine & 0xffffffffull));
-                nout += __popc(bt);
+        __syncthreads();
+        if (warp == 0) {
+            // lane l owns bins 255 - 8 l .. 248 - 8 l; the digit is the highest bin d with count(bins >= d) >= remaining
+            const int rem = st.remaining;
+            int h8[8];
+            int tsum = 0;
+#pragma unroll
+            for (int x = 0; x < 8; ++x) { h8[x] = st.hist[255 - 8 * lane - x]; tsum += h8[x]; }
+            int inc = tsum;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int nn = __shfl_up_sync(kFullMask, inc, o);
+                if (lane >= o) inc += nn;
             }
-        } else if (m != quota) {
-            // crowded boundary bin (clustered or equal scores): bisection on its members' keys, one bit at a time,
-            // then the lowest chunk ids among the keys on the cut
-            unsigned prefix = 0u;
-            for (int bit = 31; bit >= 0; --bit) {
-                const unsigned cand = prefix | (1u << bit);
-                int cnt = 0;
-                for (int i = lane; i < n; i += 32) {
-                    const unsigned k = w.key[i];
-                    const int bin = max(0, min(kSelBins - 1, static_cast<int>((key_to_float(k) - lo) * inv)));
-                    cnt += (bin == bstar && k >= cand) ? 1 : 0;
+            int cum = inc - tsum;
+            if (cum < rem && inc >= rem) {          // exactly one lane
+#pragma unroll
+                for (int x = 0; x < 8; ++x) {
+                    if (cum < rem && cum + h8[x] >= rem) {
+                        st.prefix = prefix | (static_cast<unsigned>(255 - 8 * lane - x) << shift);
+                        st.mask = mask | (255u << shift);
+                        st.remaining = rem - cum;
+                        st.equal = h8[x];
+                    }
+                    cum += h8[x];
                 }
-                if (__reduce_add_sync(kFullMask, cnt) >= quota) prefix = cand;
-            }
-            int n_gt = 0;
-            for (int i = lane; i < n; i += 32) {
-                const unsigned k = w.key[i];
-                const int bin = max(0, min(kSelBins - 1, static_cast<int>((key_to_float(k) - lo) * inv)));
-                n_gt += (bin == bstar && k > prefix) ? 1 : 0;
-            }
-            n_gt = __reduce_add_sync(kFullMask, n_gt);
-            int q2 = quota - n_gt;            // members with key == prefix still to take, lowest ids first
-            int last_id = -1;
-            for (int i0 = 0; i0 < n; i0 += 32) {
-                const int i = i0 + lane;
-                unsigned k = 0u;
-                int bin = -1;
-                if (i < n) {
-                    k = w.key[i];
-                    bin = max(0, min(kSelBins - 1, static_cast<int>((key_to_float(k) - lo) * inv)));
-                }
-                const bool tk = bin == bstar && k > prefix;
-                const unsigned bt = __ballot_sync(kFullMask, tk);
-                if (tk) w.list[nout + __popc(bt & ((1u << lane) - 1u))] = (static_cast<unsigned long long>(k) << 32) | static_cast<unsigned>(w.id[i]);
-                nout += __popc(bt);
-            }
-            for (; q2 > 0; --q2) {
-                int best = 0x7fffffff;
-                for (int i = lane; i < n; i += 32) {
-                    const unsigned k = w.key[i];
-                    const int bin = max(0, min(kSelBins - 1, static_cast<int>((key_to_float(k) - lo) * inv)));
-                    if (bin == bstar && k == prefix && w.id[i] > last_id) best = min(best, w.id[i]);
-                }
-                best = static_cast<int>(__reduce_min_sync(kFullMask, static_cast<unsigned>(best)));
-                if (lane == 0) w.list[nout] = (static_cast<unsigned long long>(prefix) << 32) | static_cast<unsigned>(best);
-                ++nout;
-                last_id = best;
             }
         }
+        __syncthreads();
     }
-    __syncwarp();
-    if (lane == 0) w.cnt = nout;
+    return st.prefix;
 }
 
 struct SelShared {
     int sel_s[kSelMaxK];
+    int raw_s[kSelMaxK];                     // selected ids in arrival order
     float lam_s[8][kSelMaxK];
     alignas(16) __nv_bfloat16 q_s[8][kD + 8];
+    SelState st;
 };
 constexpr size_t kSelLmBytes = 64 * (kD + 8) * 2;          // staged landmark rows alias the selection buffers
+// dynamic shared memory of the selection: per-warp histograms, then the cached keys
+__host__ __device__ inline size_t sel_dyn_bytes(int nw, int ncached) {
+    const size_t need = static_cast<size_t>(nw) * 256 * sizeof(int) + static_cast<size_t>(ncached) * sizeof(unsigned);
+    return need > kSelLmBytes ? need : kSelLmBytes;
+}
 
 // Exact top-K of the group scores of one (sequence, KV head) pair (ties: lower chunk id), ascending ids,
 // then the per-head surrogate scores of the selected chunks and the fusion weights.  Called by every
-// thread of the pair's CTA (nw warps); dyn: nw SelWarp buffers.
+// thread of the pair's CTA (nw warps); dyn: nw histograms of 256 counters, then room for the cached keys.
 __device__ void select_pair(const DArgs& a, int pair, int ncand, SelShared& sh, uint8_t* dyn, int nw) {
     const Shape& s = a.s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -246,85 +195,74 @@ __device__ void select_pair(const DArgs& a, int pair, int ncand, SelShared& sh, 
     const int n = min(K, ncand);
     const float* u = a.u + static_cast<long long>(pair) * a.Cpad;
     int* sel_s = sh.sel_s;
-    SelWarp* sw = reinterpret_cast<SelWarp*>(dyn);
+    int (*whist)[256] = reinterpret_cast<int (*)[256]>(dyn);
+    unsigned* keys = reinterpret_cast<unsigned*>(dyn + static_cast<size_t>(nw) * 256 * sizeof(int));
+    const bool cached = ncand <= kSelKeyCap;
 
     if (ncand <= K) {
         for (int t = tid; t < K; t += NT) sel_s[t] = t < ncand ? t : -1;
         __syncthreads();
     } else {
-        // --- level 1: warp w owns the candidates [w * per, (w + 1) * per) and walks them in rounds of
-        //     kSelCap - K, carrying its survivors from round to round
-        {
-            SelWarp& w = sw[warp];
-            const int per = ((ncand + nw - 1) / nw + 31) & ~31;
-            const int cb = min(ncand, warp * per), ce = min(ncand, cb + per);
-            int nl = 0;
-            for (int r0 = cb; r0 < ce || r0 == cb; r0 += kSelCap - kSelMaxK) {
-                const int nr = max(0, min(ce - r0, kSelCap - kSelMaxK));
-                for (int i = lane; i < nl; i += 32) {
-                    const unsigned long long v = w.list[i];
-                    w.key[nr + i] = static_cast<unsigned>(v >> 32);
-                    w.id[nr + i] = static_cast<int>(v & 0xffffffffull);
+        if (cached) {
+            // the scores come from L2: sixteen loads in flight per thread; the histogram of the keys' leading byte
+            // (the first selection pass) is taken on the way
+            for (int x = tid & 31; x < 256; x += 32) whist[tid >> 5][x] = 0;
+            __syncwarp();
+            for (int i0 = 0; i0 < ncand; i0 += 16 * NT) {
+                float v[16];
+#pragma unroll
+                for (int x = 0; x < 16; ++x) {
+                    const int i = i0 + x * NT + tid;
+                    v[x] = i < ncand ? __ldcg(u + i) : 0.f;
                 }
-                // sixteen loads in flight per lane (the scores come from L2)
-                for (int i0 = 0; i0 < nr; i0 += 512) {
-                    float v[16];
 #pragma unroll
-                    for (int x = 0; x < 16; ++x) {
-                        const int i = i0 + x * 32 + lane;
-                        v[x] = i < nr ? __ldcg(u + r0 + i) : 0.f;
-                    }
-#pragma unroll
-                    for (int x = 0; x < 16; ++x) {
-                        const int i = i0 + x * 32 + lane;
-                        if (i < nr) { w.key[i] = max(1u, ordered_key(v[x])); w.id[i] = r0 + i; }
+                for (int x = 0; x < 16; ++x) {
+                    const int i = i0 + x * NT + tid;
+                    if (i < ncand) {
+                        const unsigned k = ordered_key(v[x]);
+                        keys[i] = k;
+                        atomicAdd(&whist[tid >> 5][k >> 24], 1);
                     }
                 }
-                __syncwarp();
-                warp_select(w, nr + nl, K, lane);
-                __syncwarp();
-                nl = w.cnt;
+            }
+            __syncthreads();
+        }
+        auto key_of = [&](int i) { return cached ? keys[i] : ordered_key(__ldcg(u + i)); };
+        // T = the K-th best score key; `quota` of the chunks that hold exactly T are still wanted
+        const unsigned T = radix_kth(sh.st, whist, ncand, K, 24, key_of, [](int) { return true; }, cached);
+        const int quota = sh.st.remaining, equal = sh.st.equal;
+        __syncthreads();
+        // more ties than places: the `quota` lowest chunk ids among them, i.e. the quota-th largest of ~id
+        unsigned idcut = 0u;                      // chunks with key == T and ~id >= idcut are taken
+        if (equal > quota) {
+            idcut = radix_kth(sh.st, whist, ncand, quota, 16, [](int i) { return 0x00ffffffu - static_cast<unsigned>(i); },
+                              [&](int i) { return key_of(i) == T; });
+            __syncthreads();
+        }
+        if (tid == 0) sh.st.nout = 0;
+        __syncthreads();
+        for (int i = tid; i < ncand; i += NT) {
+            const unsigned k = key_of(i);
+            if (k > T || (k == T && 0x00ffffffu - static_cast<unsigned>(i) >= idcut)) {
+                const int pos = atomicAdd(&sh.st.nout, 1);
+                if (pos < kSelMaxK) sh.raw_s[pos] = i;
             }
         }
         __syncthreads();
-        // --- merge rounds: warp g gathers the lists [g * fan, (g + 1) * fan) into its staging buffer (fan x K <= kSelCap).
-        //     A round reads lists that the previous round finished; it writes only the staging arrays and, after a
-        //     barrier, its own list.
-        int lists = nw;
-        const int fan = min(4, kSelCap / K);               // few lists per warp: short rounds on many warps
-        while (lists > 1) {
-            const int groups = (lists + fan - 1) / fan;
-            int tot = 0;
-            if (warp < groups) {
-                SelWarp& w = sw[warp];
-                for (int li = warp * fan; li < min(lists, (warp + 1) * fan); ++li) {
-                    const SelWarp& src = sw[li];
-                    const int cn = src.cnt;
-                    for (int i = lane; i < cn; i += 32) {
-                        const unsigned long long v = src.list[i];
-                        w.key[tot + i] = static_cast<unsigned>(v >> 32);
-                        w.id[tot + i] = static_cast<int>(v & 0xffffffffull);
-                    }
-                    tot += cn;
-                }
-            }
-            __syncthreads();                               // every list of this round has been read
-            if (warp < groups) warp_select(sw[warp], tot, K, lane);
-            __syncthreads();
-            lists = groups;
-        }
-        // --- ascending chunk ids: position = number of selected ids below mine
-        const unsigned long long* fin = sw[0].list;
-        for (int t = tid; t < n; t += NT) {
-            const int idt = static_cast<int>(fin[t] & 0xffffffffull);
+        // --- ascending chunk ids: position = number of selected ids below mine (eight lanes share an element)
+        for (int t0 = 0; t0 < n; t0 += NT / 8) {
+            const int t = t0 + (tid >> 3), part = tid & 7;
+            const int idt = t < n ? sh.raw_s[t] : 0;
             int pos = 0;
-            for (int j = 0; j < n; ++j) pos += static_cast<int>(fin[j] & 0xffffffffull) < idt ? 1 : 0;
-            sel_s[pos] = idt;
+            for (int j = part; j < n; j += 8) pos += sh.raw_s[j] < idt ? 1 : 0;
+            pos += __shfl_xor_sync(kFullMask, pos, 1);
+            pos += __shfl_xor_sync(kFullMask, pos, 2);
+            pos += __shfl_xor_sync(kFullMask, pos, 4);
+            if (t < n && part == 0) sel_s[pos] = idt;
         }
         __syncthreads();
     }
     for (int t = tid; t < K; t += NT) sel[t] = t < n ? sel_s[t] : -1;
-
     // --- per-head surrogate scores of the selected chunks and the fusion weights: the selected
     //     landmark rows and the G queries are staged in shared memory with one round of 16-byte
     //     loads, then every thread computes (chunk, head) dot products
@@ -397,6 +335,7 @@ __global__ void __launch_bounds__(kScoreThreads) decode_score_kernel(const DArgs
     const int pair = blockIdx.y;
     const int b = pair / s.Hkv, g = pair % s.Hkv;
     const int seq = query_seq_len(a, b);
+    STAMP_MIN(0);
     if (seq < 1 || seq > s.T) return;
     const int ncand = first_local_chunk(seq, s.W);
     const int c_begin = blockIdx.x * kScoreChunksPerCta;
@@ -471,18 +410,22 @@ __global__ void __launch_bounds__(kScoreThreads) decode_score_kernel(const DArgs
         if (t == 0 && ca < ncand) u[ca] = best[it][0];
         if (t == 1 && cb < ncand) u[cb] = best[it][1];
     }
+    STAMP_MAX(1);
     pdl_launch_dependents();
 }
 
-// One CTA per (sequence, KV head) pair: 4 warps for candidate lists of up to 4096 chunks, else 16.
-// Dynamic shared memory: one SelWarp per warp.
-__global__ void __launch_bounds__(512) decode_select_kernel(const DArgs a) {
+// One CTA per (sequence, KV head) pair: 4 warps for candidate lists of up to 1024 chunks, 8 up to 4096, else 32.
+// Dynamic shared memory: sel_dyn_bytes.
+__global__ void __launch_bounds__(kSelMaxWarps * 32) decode_select_kernel(const DArgs a) {
     __shared__ SelShared sh;
     extern __shared__ __align__(16) uint8_t sel_dyn[];
     const Shape& s = a.s;
     const int pair = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
     const int b = pair / s.Hkv, g = pair % s.Hkv;
     const int seq = query_seq_len(a, b);
+    STAMP_MIN(2);
+    pdl_wait();                                        // the previous kernels' reads and writes of the scratch are over
+    STAMP_MIN(4);
     if (seq < 1 || seq > s.T) {
         // invalid length: flag it, emit empty outputs
         if (tid == 0) { set_status(a.status, kDevBadIndex); a.pair_n[pair] = -1; a.done[pair] = 0; }
@@ -492,8 +435,8 @@ __global__ void __launch_bounds__(512) decode_select_kernel(const DArgs a) {
         if (tid < s.G) a.lse[static_cast<long long>(b) * s.Hq + g * s.G + tid] = 0.f;
         return;
     }
-    pdl_wait();                                        // group scores of decode_score are visible
     select_pair(a, pair, first_local_chunk(seq, s.W), sh, sel_dyn, nt >> 5);
+    STAMP_MAX(3);
     pdl_launch_dependents();
 }
 
@@ -535,7 +478,9 @@ decode_attend_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
         tma_prefetch_desc(&map_k);
         tma_prefetch_desc(&map_v);
     }
+    STAMP_MIN(6);
     pdl_wait();                                   // selection, weights and counters are visible
+    STAMP_MIN(8);
     for (int j = tid; j < nitems; j += kAttendThreads) {
         const long long idx = lo + j;
         const int pair = static_cast<int>(idx / slots), slot = static_cast<int>(idx % slots);
@@ -784,6 +729,7 @@ decode_attend_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
         j0 = j1;
         if (dead) break;
     }
+    STAMP_MAX(7);
 }
 
 struct Plan {
@@ -824,7 +770,7 @@ Plan make_plan(const Shape& s, int n_sm) {
 bool decode_fast_supports(const Shape& s, int dtype) {
     return dtype == HILS_BF16 && s.is_decode && s.d == kD && s.S == kS && s.W >= 1 && max_local_slots(s.W) <= 16 && (s.Hl == s.Hkv || s.Hl == s.Hq) && s.G <= 8 &&
            s.K >= 1 && s.K <= 128 && static_cast<long long>(s.B) * s.Hkv * s.T < (1ll << 31) &&
-           static_cast<long long>(s.B) * s.Hkv <= 65535;
+           static_cast<long long>(s.B) * s.Hkv <= 65535 && s.C < (1 << 24);
 }
 
 size_t decode_fast_scratch_bytes(const Shape& s) {
@@ -879,7 +825,7 @@ int launch_decode_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
         if (cudaFuncSetAttribute(decode_attend_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(attend_smem)) != cudaSuccess ||
             cudaFuncSetAttribute(decode_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 static_cast<int>(sizeof(SelWarp) * 16)) != cudaSuccess)
+                                 static_cast<int>(sel_dyn_bytes(kSelMaxWarps, kSelKeyCap))) != cudaSuccess)
             return HILS_ERR_CUDA;
         attr_once.done();
     }
@@ -899,8 +845,9 @@ int launch_decode_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
     cfg.gridDim = dim3(pairs);
     cfg.dynamicSmemBytes = 0;
     {
-        const int nw = (s.T - 1) / kS <= 4096 ? 4 : 16;
-        const size_t need = sizeof(SelWarp) * nw > kSelLmBytes ? sizeof(SelWarp) * nw : kSelLmBytes;
+        const int cmax = (s.T - 1) / kS;                       // candidates of the longest possible sequence
+        const int nw = cmax <= 1024 ? 4 : (cmax <= 4096 ? 8 : kSelMaxWarps);
+        const size_t need = sel_dyn_bytes(nw, cmax < kSelKeyCap ? cmax : 0);
         cfg.blockDim = dim3(nw * 32);
         cfg.dynamicSmemBytes = need;
         if (cudaLaunchKernelEx(&cfg, decode_select_kernel, a) != cudaSuccess) return HILS_ERR_CUDA;
