@@ -53,10 +53,10 @@ struct AtcSmem {
     // its last P V MMA, about one epilogue phase later)
     uint64_t k_ready[2];      // K tile landed (TMA bytes) and the landmark row written (one arrival)
     uint64_t v_ready[kVBufs]; // V tile landed
-    uint64_t k_empty[2];      // every S MMA that reads this K buffer has completed
-    uint64_t v_empty[kVBufs]; // every P V MMA that reads this V buffer has completed
+    uint64_t k_empty[2];      // every S MMA that reads this K buffer has completed (relayed by the softmax group)
+    uint64_t v_empty[kVBufs]; // every P V MMA that reads this V buffer has completed (relayed by the output group)
     uint64_t q_full[kQSlots]; // gathered Q rows landed (TMA bytes)
-    uint64_t q_empty[kQSlots];// the S MMA that reads this Q tile has completed
+    uint64_t q_empty[kQSlots];// the S MMA that reads this Q tile has completed (relayed by the softmax group)
     uint64_t s_full[2];       // S = Q K^T in tensor memory
     uint64_t s_empty[2];      // the slot's softmax group has read S
     uint64_t p_full[2];       // P written to tensor memory
@@ -65,7 +65,8 @@ struct AtcSmem {
     uint32_t tmem_base;
     int abort_flag;
     int tile_ent[kMetaSlots][kTok];   // entries of the tiles in flight
-    int tile_meta[kMetaSlots][4];     // pair, chunk, tokens, first entry relative to the query block
+    int tile_meta[kMetaSlots][4];     // pair, chunk, tokens | last tile of its chunk run << 8 | K buffer << 9 | V buffer << 10,
+                                      // first entry relative to the query block
     int4 recs[kBatch];
     int nchunks;                      // distinct (pair, chunk) runs in the current batch
     uint8_t cfirst[kBatch + 4];       // first tile (batch index) of each run; cfirst[nchunks] = tiles in the batch
@@ -114,7 +115,7 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
     const Shape& s = a.s;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
-        for (int i = 0; i < kQSlots; ++i) { mbar_init(&sm.q_full[i], kGatherWarps); mbar_init(&sm.q_empty[i], 1); }
+        for (int i = 0; i < kQSlots; ++i) { mbar_init(&sm.q_full[i], kGatherWarps * 32 + kGatherWarps); mbar_init(&sm.q_empty[i], 1); }
         for (int i = 0; i < kVBufs; ++i) { mbar_init(&sm.v_ready[i], 1); mbar_init(&sm.v_empty[i], 1); }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&sm.k_ready[i], 2);           // the TMA issuer's arrive.expect_tx + the landmark writer
@@ -200,9 +201,10 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
         const bool owns = lane < 8 && 2 * (e0 + lane) >= j0 && 2 * (e0 + lane) < j1;   // this lane records its entry
         const int p16 = lane & 15, hh = lane >> 4;
         const long long hstride = static_cast<long long>(s.R) * kD;
-        walk([&](int nb, uint32_t tcount, uint32_t, int t_begin, int i0) {
+        walk([&](int nb, uint32_t tcount, uint32_t ccount, int t_begin, int i0) {
             uint32_t tc = tcount;
             bool dead = false;
+            int ck = 0;                        // chunk run (ordinal within the batch) of the current tile
             // this lane's entry of the upcoming tiles, fetched two tiles ahead
             int e_next = a.entries[sm.recs[0].z + min(el, sm.recs[0].w - 1)];
             int e_next2 = nb > 1 ? a.entries[sm.recs[1].z + min(el, sm.recs[1].w - 1)] : 0;
@@ -217,7 +219,13 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                 if (*reinterpret_cast<volatile int*>(&sm.abort_flag)) { dead = true; break; }
                 if (owns) sm.tile_ent[ms][e0 + lane] = e;
                 if (gw == 0 && lane == 0) {
-                    sm.tile_meta[ms][0] = pair; sm.tile_meta[ms][1] = rec.y; sm.tile_meta[ms][2] = ntok;
+                    // A tcgen05.commit costs the issuing thread about a hundred cycles, so only the two the epilogue
+                    // groups wait on are issued; those groups pass "this Q slot / K buffer / V buffer is free" on.
+                    if (ti >= sm.cfirst[ck + 1]) ++ck;
+                    const bool last = ti + 1 >= sm.cfirst[ck + 1];
+                    const uint32_t cc = ccount + static_cast<uint32_t>(ck);
+                    sm.tile_meta[ms][0] = pair; sm.tile_meta[ms][1] = rec.y;
+                    sm.tile_meta[ms][2] = ntok | (last ? 256 : 0) | static_cast<int>((cc & 1u) << 9) | static_cast<int>((cc % kVBufs) << 10);
                     sm.tile_meta[ms][3] = rec.z - (a.whole ? 0 : t_begin * kTok);
                 }
                 {
@@ -232,22 +240,13 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                         const __nv_bfloat16* src = qb0 + (2 * j & 3) * hstride + static_cast<long long>(ej >> 8) * kD;
                         cp_async16(qaddr + swz128(row, p16 & 7), src);
                     }
-                    cp_async_commit();
                 }
-                // the previous tile's rows have landed by now: publish them
-                if (tc > tcount) {
-                    cp_async_wait<1>();
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&sm.q_full[(tc - 1) % kQSlots]);
-                }
-                ++tc;
-            }
-            cp_async_wait<0>();
-            if (tc > tcount && !dead) {
-                fence_proxy_async_smem();
+                // The tile's barrier hears from every gather thread when that thread's copies have landed (no thread
+                // waits for them), and from one lane per warp for the tile's descriptor written above.
+                asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(&sm.q_full[qs])) : "memory");
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&sm.q_full[(tc - 1) % kQSlots]);
+                if (lane == 0) mbar_arrive(&sm.q_full[qs]);
+                ++tc;
             }
             if (dead && lane == 0) { set_status(a.status, kDevTimeout); atomicExch(&sm.abort_flag, 1); }
         });
@@ -280,6 +279,13 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                 tc_fence_after_sync();
                 const uint32_t ms = tcv % kMetaSlots;
                 const int pair = sm.tile_meta[ms][0], c = sm.tile_meta[ms][1];
+                // the tile's score MMAs are done: its gathered rows, and its chunk's K tile after the chunk's last tile,
+                // may be overwritten
+                if ((warp & 3) == 0 && lane == 0) {
+                    const int flags = sm.tile_meta[ms][2];
+                    mbar_arrive(&sm.q_empty[tcv % kQSlots]);
+                    if (flags & 256) mbar_arrive(&sm.k_empty[(flags >> 9) & 1]);
+                }
                 const int orow0 = sm.tile_meta[ms][3] * kG;          // first row of the tile in the output buffers
                 const int e = sm.tile_ent[ms][tk];
                 const int il = e >> 8, slot = e & 255;
@@ -370,6 +376,11 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                 if (!ok) break;
                 tc_fence_after_sync();
                 const int orow0 = sm.tile_meta[tcv % kMetaSlots][3] * kG;
+                if (ow == 0 && lane == 0) {
+                    // the tile's P V MMAs are done: after the chunk's last tile its V tile may be overwritten
+                    const int flags = sm.tile_meta[tcv % kMetaSlots][2];
+                    if (flags & 256) mbar_arrive(&sm.v_empty[(flags >> 10) & 3]);
+                }
 #pragma unroll 1
                 for (int hb = 0; hb < 2; ++hb) {
                     uint32_t pk[32];
@@ -514,6 +525,9 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                         if (ready) {
                             if (newc) { cur_pair = rec.x; cur_c = rec.y; ++cc; }
                             const uint32_t cb = (cc - 1) & 1u;
+                            // the gathered rows were written by cp.async (generic proxy), the MMA reads them through
+                            // the async proxy
+                            fence_proxy_async_smem();
                             tc_fence_after_sync();
                             const uint32_t qa = smem_u32(qbuf + qs * kQBytes), ka = smem_u32(kbuf + cb * kKBytes);
 #pragma unroll
@@ -521,9 +535,6 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                                 umma_bf16(tmem_base + sl * 128, umma_desc_k128(qa + (ks >> 2) * 16384 + (ks & 3) * 32),
                                           umma_desc_k128(ka + (ks >> 2) * (kNS * 128) + (ks & 3) * 32), idesc_s, ks > 0 ? 1u : 0u);
                             umma_commit(&sm.s_full[sl]);
-                            umma_commit(&sm.q_empty[qs]);
-                            // last tile of its chunk in this batch: the K buffer is free once these MMAs are done
-                            if (ns + 1 >= nb || sm.recs[ns + 1].x != rec.x || sm.recs[ns + 1].y != rec.y) umma_commit(&sm.k_empty[cb]);
                             ++ns;
                             progressed = true;
                         }
@@ -545,9 +556,6 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                                 umma_bf16_ts(tmem_base + 256 + sl * 128, tmem_base + sl * 128 + kPCol + ks * 8,
                                              umma_desc_mn128(va + ks * 2048, 8192u, 1024u), idesc_o, ks > 0 ? 1u : 0u);
                             umma_commit(&sm.o_full[sl]);
-                            // last tile of its chunk in this batch: the V buffer is free once these MMAs are done
-                            const bool last = no + 1 >= nb || sm.recs[no + 1].x != reco.x || sm.recs[no + 1].y != reco.y;
-                            if (last) umma_commit(&sm.v_empty[vb]);
                             ++no;
                             progressed = true;
                         }
