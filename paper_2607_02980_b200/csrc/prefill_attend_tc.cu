@@ -35,10 +35,12 @@ constexpr int kVBytes = kS * kD * 2;            // two boxes of 64 keys x 64 dim
 constexpr int kQBytes = kRows * kD * 2;         // 32 KB
 constexpr int kPBytes = kRows * 128;            // 16 KB
 constexpr int kPCol = 96;                       // probabilities (bf16 pairs, 32 columns) behind the slot's 80 score columns
-constexpr int kBatch = 128;                     // tile records cached per batch
+constexpr int kBatch = 48;                      // tiles whose records and entries are cached in shared memory at a time
 constexpr int kQSlots = 3;                      // gathered Q tiles in flight
 constexpr int kVBufs = 3;                       // V tiles in flight (K: 2)
-constexpr int kMetaSlots = 8;                   // ring of tile descriptors (the loader is < 8 tiles ahead of the output group)
+constexpr int kMetaSlots = 16;                  // ring of tile descriptors.  The gather of tile t starts once S(t-3) is done, which
+                                                // needs softmax(t-5) under way, hence softmax(t-7) finished, hence P V(t-9) done,
+                                                // hence the output of tile t-11 finished: the output group is at most 10 tiles behind
 constexpr int kSoftThreads = 256;               // two softmax groups of 128 threads
 constexpr int kOutWarp0 = kSoftThreads / 32;    // 8
 constexpr int kGatherWarps = 4;
@@ -64,10 +66,10 @@ struct AtcSmem {
     uint64_t o_empty[2];      // the output group has read O
     uint32_t tmem_base;
     int abort_flag;
-    int tile_ent[kMetaSlots][kTok];   // entries of the tiles in flight
     int tile_meta[kMetaSlots][4];     // pair, chunk, tokens | last tile of its chunk run << 8 | K buffer << 9 | V buffer << 10,
                                       // first entry relative to the query block
     int4 recs[kBatch];
+    int ent_s[kBatch * kTok];         // entries of the batch's tiles: (token - block start) << 8 | slot
     int nchunks;                      // distinct (pair, chunk) runs in the current batch
     uint8_t cfirst[kBatch + 4];       // first tile (batch index) of each run; cfirst[nchunks] = tiles in the batch
 };
@@ -163,12 +165,16 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
             for (long long b0 = lo; b0 < hi; b0 += kBatch) {
                 const int nb = static_cast<int>(min(static_cast<long long>(kBatch), hi - b0));
                 for (int x = tid; x < nb; x += kThreads) sm.recs[x] = a.tiles[b0 + x];
+                // A list starts on a tile boundary of the global entry space, so the entries of tile t are
+                // entries[32 t .. 32 t + 31]: the batch's entries are one contiguous run, fetched now, all at once (a
+                // load per tile inside the gather loop waited several thousand cycles under the partial-output stores).
+                for (int x = tid; x < nb * kTok; x += kThreads) sm.ent_s[x] = a.entries[b0 * kTok + x];
                 __syncthreads();
                 if (sm.abort_flag) return;
                 if (warp == 0) {
                     // table of chunk runs: where each run of tiles of one (pair, chunk) starts
                     int basec = 0;
-                    for (int w = 0; w < kBatch / 32; ++w) {
+                    for (int w = 0; w < (kBatch + 31) / 32; ++w) {
                         const int x = w * 32 + lane;
                         const bool nw = x < nb && (x == 0 || sm.recs[x].x != sm.recs[x - 1].x || sm.recs[x].y != sm.recs[x - 1].y);
                         const unsigned m = __ballot_sync(kFullMask, nw);
@@ -198,26 +204,20 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
         const int j0 = gw * kPerWarp, j1 = j0 + kPerWarp;
         const int e0 = j0 >> 1;                                      // first entry this warp touches
         const int el = min(e0 + (lane & 7), kTok - 1);
-        const bool owns = lane < 8 && 2 * (e0 + lane) >= j0 && 2 * (e0 + lane) < j1;   // this lane records its entry
         const int p16 = lane & 15, hh = lane >> 4;
         const long long hstride = static_cast<long long>(s.R) * kD;
         walk([&](int nb, uint32_t tcount, uint32_t ccount, int t_begin, int i0) {
             uint32_t tc = tcount;
             bool dead = false;
             int ck = 0;                        // chunk run (ordinal within the batch) of the current tile
-            // this lane's entry of the upcoming tiles, fetched two tiles ahead
-            int e_next = a.entries[sm.recs[0].z + min(el, sm.recs[0].w - 1)];
-            int e_next2 = nb > 1 ? a.entries[sm.recs[1].z + min(el, sm.recs[1].w - 1)] : 0;
             for (int ti = 0; ti < nb; ++ti) {
                 const int4 rec = sm.recs[ti];
                 const int pair = rec.x, ntok = rec.w;
-                const int e = e_next;
-                e_next = e_next2;
-                if (ti + 2 < nb) e_next2 = a.entries[sm.recs[ti + 2].z + min(el, sm.recs[ti + 2].w - 1)];
+                // this lane's entry (rows past a ragged tile's last entry repeat that entry)
+                const int e = sm.ent_s[ti * kTok + min(el, ntok - 1)];
                 const uint32_t qs = tc % kQSlots, ms = tc % kMetaSlots;
                 if (tc >= kQSlots && !mbar_wait(&sm.q_empty[qs], ((tc / kQSlots) - 1) & 1)) { dead = true; break; }
                 if (*reinterpret_cast<volatile int*>(&sm.abort_flag)) { dead = true; break; }
-                if (owns) sm.tile_ent[ms][e0 + lane] = e;
                 if (gw == 0 && lane == 0) {
                     // A tcgen05.commit costs the issuing thread about a hundred cycles, so only the two the epilogue
                     // groups wait on are issued; those groups pass "this Q slot / K buffer / V buffer is free" on.
@@ -232,12 +232,16 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                     const uint32_t qaddr = smem_u32(qbuf + qs * kQBytes) + (p16 >> 3) * 16384;
                     const __nv_bfloat16* qb0 = a.q + (static_cast<long long>(pair / s.Hkv) * s.Hq + (pair % s.Hkv) * kG + hh) * hstride +
                                                static_cast<long long>(i0) * kD + p16 * 8;
+                    // the tokens of the warp's entries first (shuffles and copies are both ordered operations: interleaved
+                    // they would run strictly one after the other)
+                    int tokv[kPerWarp / 2];
+#pragma unroll
+                    for (int k = 0; k < kPerWarp / 2; ++k) tokv[k] = __shfl_sync(kFullMask, e, k) >> 8;
 #pragma unroll
                     for (int jj = 0; jj < kPerWarp; ++jj) {
                         const int j = j0 + jj;
-                        const int ej = __shfl_sync(kFullMask, e, (j >> 1) - e0);
                         const int row = 2 * j + hh;
-                        const __nv_bfloat16* src = qb0 + (2 * j & 3) * hstride + static_cast<long long>(ej >> 8) * kD;
+                        const __nv_bfloat16* src = qb0 + (2 * j & 3) * hstride + static_cast<long long>(tokv[jj >> 1]) * kD;
                         cp_async16(qaddr + swz128(row, p16 & 7), src);
                     }
                 }
@@ -287,7 +291,7 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                     if (flags & 256) mbar_arrive(&sm.k_empty[(flags >> 9) & 1]);
                 }
                 const int orow0 = sm.tile_meta[ms][3] * kG;          // first row of the tile in the output buffers
-                const int e = sm.tile_ent[ms][tk];
+                const int e = sm.ent_s[ti * kTok + min(tk, (sm.tile_meta[ms][2] & 255) - 1)];
                 const int il = e >> 8, slot = e & 255;
                 const bool local = slot >= s.K;                            // a chunk of the local window: mass = its exact log-sum-exp
                 const int lim = local ? s.pos0 + i0 + il - c * kS : kS - 1;   // last visible key of the chunk
@@ -381,29 +385,41 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                     const int flags = sm.tile_meta[tcv % kMetaSlots][2];
                     if (flags & 256) mbar_arrive(&sm.v_empty[(flags >> 10) & 3]);
                 }
-#pragma unroll 1
-                for (int hb = 0; hb < 2; ++hb) {
-                    uint32_t pk[32];
-                    {
-                        float v[64];
-                        tmem_ld64(t_lane + 256 + sl * 128 + hb * 64, v);
+                // The accumulator leaves tensor memory in four quarters of 32 columns; the load of the next quarter runs
+                // under the packing and staging of the current one.
+                uint32_t va[32], vb[32];
+                const uint32_t o_col = t_lane + 256 + sl * 128;
+                tmem_ld32_issue(o_col, va);
+                tmem_ld_wait32(va);
+                tmem_ld32_issue(o_col + 32, vb);
+                // the previous tile's stores (lane 0: columns 0..63, lane 1: 64..127) must have read the staging rows
+                if (lane < 2) bulk_wait_read<0>();
+                __syncwarp();
+                auto stage = [&](const uint32_t (&v)[32], int q) {
+                    // quarter q: columns 32 q .. 32 q + 31 -> four 16-byte pieces of the row's half q / 2
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) pk[j] = pack_bf16(v[2 * j], v[2 * j + 1]);
+                    for (int pc = 0; pc < 4; ++pc) {
+                        uint4 w;
+                        w.x = pack_bf16(__uint_as_float(v[8 * pc]), __uint_as_float(v[8 * pc + 1]));
+                        w.y = pack_bf16(__uint_as_float(v[8 * pc + 2]), __uint_as_float(v[8 * pc + 3]));
+                        w.z = pack_bf16(__uint_as_float(v[8 * pc + 4]), __uint_as_float(v[8 * pc + 5]));
+                        w.w = pack_bf16(__uint_as_float(v[8 * pc + 6]), __uint_as_float(v[8 * pc + 7]));
+                        *reinterpret_cast<uint4*>(obuf + (q >> 1) * kPBytes + swz128(row, (q & 1) * 4 + pc)) = w;
                     }
-                    if (hb == 0) {
-                        // the previous tile's stores (lane 0: columns 0..63, lane 1: 64..127) must have read the staging rows
-                        if (lane < 2) bulk_wait_read<0>();
-                        __syncwarp();
-                    } else {
-                        // the accumulator is free for the slot's next tile
-                        tc_fence_before_sync();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(&sm.o_empty[sl]);
-                    }
-#pragma unroll
-                    for (int pc = 0; pc < 8; ++pc)
-                        *reinterpret_cast<uint4*>(obuf + hb * kPBytes + swz128(row, pc)) = make_uint4(pk[4 * pc], pk[4 * pc + 1], pk[4 * pc + 2], pk[4 * pc + 3]);
-                }
+                };
+                stage(va, 0);
+                tmem_ld_wait32(vb);
+                tmem_ld32_issue(o_col + 64, va);
+                stage(vb, 1);
+                tmem_ld_wait32(va);
+                tmem_ld32_issue(o_col + 96, vb);
+                stage(va, 2);
+                tmem_ld_wait32(vb);
+                // the accumulator is free for the slot's next tile
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.o_empty[sl]);
+                stage(vb, 3);
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane < 2) {
