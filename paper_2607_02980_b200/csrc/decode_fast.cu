@@ -95,9 +95,20 @@ __device__ __forceinline__ int first_local_chunk(int seq, int W) { return local_
 // first -- if there are more than that, a second selection of the same kind runs on their ids.  The keys are cached
 // in shared memory after the first pass (they come from L2) when they fit.  Integer arithmetic throughout: exact and
 // independent of the thread count.
+//
+// A pass over the list costs its instructions, not its bytes (one SM works on a pair's whole list), so lists of up to
+// 16 candidates per thread take a shorter way first (select_in_registers): every thread keeps its scores in
+// registers; the span between the smallest and the largest score is cut into 2048 equal bins (equal in value: the
+// bins of a radix digit are equal in the exponent, and most scores of a list share two or three exponents, which
+// serialises their counter updates), one histogram pass and one scan find the bin the K-th best score falls into,
+// everything above it is selected and the bin's members are ranked against each other directly by (key, then lower
+// chunk id).  A bin with more than kSelTieCap members (massive ties) falls back to the passes described above.
 constexpr int kSelMaxK = 128;
 constexpr int kSelMaxWarps = 32;
 constexpr int kSelKeyCap = 40960;            // keys cached in shared memory (160 KB); longer lists re-read the scores
+constexpr int kSelTieCap = 512;              // candidates of the boundary bin that are ranked directly
+constexpr int kSelRegKeys = 16;              // keys a thread holds in registers on the short way
+constexpr int kSelBins = 2048;               // counters of the short way's histogram
 
 struct SelState {
     int hist[256];                           // summed histogram of the current pass
@@ -105,6 +116,9 @@ struct SelState {
     int remaining;                           // how many candidates matching the prefix are still wanted from the top
     int equal;                               // candidates whose key equals the finished prefix
     int nout;                                // selected so far
+    int ntie, bstar, above;                  // short way: the bin of the K-th best score
+    unsigned kmin, kmax;                     // short way: span of the scores (ordered keys)
+    int wsum[kSelMaxWarps];
 };
 
 // One selection: the `want`-th largest value of val(i) over the candidates i in [0, n) for which live(i) holds
@@ -177,9 +191,156 @@ struct SelShared {
 };
 constexpr size_t kSelLmBytes = 64 * (kD + 8) * 2;          // staged landmark rows alias the selection buffers
 // dynamic shared memory of the selection: per-warp histograms, then the cached keys
+// dynamic shared memory of the selection: histograms (nw of 256 counters, or the short way's 2048), then the cached
+// keys or the short way's boundary-bin members
+__host__ __device__ inline size_t sel_hist_ints(int nw) { return nw * 256 > kSelBins ? nw * 256 : kSelBins; }
 __host__ __device__ inline size_t sel_dyn_bytes(int nw, int ncached) {
-    const size_t need = static_cast<size_t>(nw) * 256 * sizeof(int) + static_cast<size_t>(ncached) * sizeof(unsigned);
+    const size_t keys = static_cast<size_t>(ncached) * sizeof(unsigned), ties = static_cast<size_t>(kSelTieCap) * 2 * sizeof(unsigned);
+    const size_t need = sel_hist_ints(nw) * sizeof(int) + (keys > ties ? keys : ties);
     return need > kSelLmBytes ? need : kSelLmBytes;
+}
+
+// Walks the `nbins` counters of hist from the top bin down and finds the bin in which the running count reaches
+// `need`: st.bstar = that bin, st.above = candidates in the bins above it, st.equal = candidates in it.  Called by
+// every thread; ends with a barrier.
+__device__ void scan_from_top(SelState& st, const int* hist, int nbins, int need) {
+    // (a step of a few instructions: with every warp of a large CTA taking part it would cost their issue slots, so
+    //  at most 256 threads walk the bins)
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, NT = blockDim.x < 256 ? blockDim.x : 256, nw = NT >> 5;
+    if (tid >= NT) { __syncthreads(); __syncthreads(); __syncthreads(); return; }
+    const int per = nbins > NT ? nbins / NT : 1;          // nbins and NT are powers of two
+    int mine = 0;
+    for (int x = 0; x < per; ++x) {
+        const int bk = nbins - 1 - (tid * per + x);
+        if (bk >= 0) mine += hist[bk];
+    }
+    int inc = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int nn = __shfl_up_sync(kFullMask, inc, o);
+        if (lane >= o) inc += nn;
+    }
+    if (lane == 31) st.wsum[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        const int tot = lane < nw ? st.wsum[lane] : 0;
+        int acc = tot;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int nn = __shfl_up_sync(kFullMask, acc, o);
+            if (lane >= o) acc += nn;
+        }
+        if (lane < nw) st.wsum[lane] = acc - tot;          // candidates in the bins of the warps before this one
+    }
+    __syncthreads();
+    int cum = st.wsum[warp] + inc - mine;                  // candidates in the bins above this thread's
+    if (cum < need && cum + mine >= need) {                // exactly one thread
+        for (int x = 0; x < per; ++x) {
+            const int bk = nbins - 1 - (tid * per + x);
+            const int h = bk >= 0 ? hist[bk] : 0;
+            if (cum < need && cum + h >= need) { st.bstar = bk; st.above = cum; st.equal = h; }
+            cum += h;
+        }
+    }
+    __syncthreads();
+}
+
+// Exact top-`want` of the n <= kSelRegKeys * blockDim.x scores u[0 .. n) (see above).  hist: kSelBins counters;
+// tie_k / tie_i: kSelTieCap entries each.  Returns true with the selected candidate ids in raw_s[0 .. want) (any
+// order); false, with nothing written that matters, when the bin of the K-th best score holds more than kSelTieCap
+// candidates (or the scores have no span).  Called by every thread.
+__device__ bool select_in_registers(SelState& st, int* hist, const float* u, int n, int want, int* raw_s,
+                                    unsigned* tie_k, int* tie_i) {
+    const int tid = threadIdx.x, lane = tid & 31, NT = blockDim.x;
+    float v[kSelRegKeys];
+#pragma unroll
+    for (int x = 0; x < kSelRegKeys; ++x) {
+        const int i = x * NT + tid;
+        v[x] = i < n ? __ldcg(u + i) : 0.f;
+    }
+    for (int x = tid; x < kSelBins; x += NT) hist[x] = 0;
+    if (tid == 0) { st.nout = 0; st.ntie = 0; st.kmin = 0xffffffffu; st.kmax = 0u; }
+    __syncthreads();
+    // span of the scores
+    unsigned kmin = 0xffffffffu, kmax = 0u;
+#pragma unroll
+    for (int x = 0; x < kSelRegKeys; ++x) {
+        if (x * NT + tid < n) {
+            const unsigned k = ordered_key(v[x]);
+            kmin = min(kmin, k);
+            kmax = max(kmax, k);
+        }
+    }
+    kmin = __reduce_min_sync(kFullMask, kmin);
+    kmax = __reduce_max_sync(kFullMask, kmax);
+    if (lane == 0) { atomicMin(&st.kmin, kmin); atomicMax(&st.kmax, kmax); }
+    __syncthreads();
+    const float lo = key_to_float(st.kmin), hi = key_to_float(st.kmax);
+    const float inv = static_cast<float>(kSelBins) / (hi - lo);
+    // (no span, or a span that is not a number: every candidate would land in one bin)
+    if (!(hi > lo) || !(inv > 0.f) || !(inv < INFINITY)) return false;
+    // bin of a score: the same expression wherever it is needed, non-decreasing in the score
+    auto bin_of = [&](float x) { return min(kSelBins - 1, max(0, static_cast<int>((x - lo) * inv))); };
+#pragma unroll
+    for (int x = 0; x < kSelRegKeys; ++x)
+        if (x * NT + tid < n) atomicAdd(&hist[bin_of(v[x])], 1);
+    __syncthreads();
+    scan_from_top(st, hist, kSelBins, want);
+    const int bstar = st.bstar, above = st.above, m = st.equal;
+    if (m > kSelTieCap) return false;
+#pragma unroll
+    for (int x = 0; x < kSelRegKeys; ++x) {
+        const int i = x * NT + tid;
+        if (i < n) {
+            const int bk = bin_of(v[x]);
+            if (bk > bstar) {
+                raw_s[atomicAdd(&st.nout, 1)] = i;
+            } else if (bk == bstar) {
+                const int pos = atomicAdd(&st.ntie, 1);
+                tie_k[pos] = ordered_key(v[x]);
+                tie_i[pos] = i;
+            }
+        }
+    }
+    __syncthreads();
+    // the `need` best of the bin's m members: rank = members ahead of mine (higher key, or the same key and a lower
+    // chunk id); eight lanes share a member
+    const int need = want - above;
+    for (int e0 = 0; e0 < m; e0 += NT / 8) {
+        const int e = e0 + (tid >> 3), part = tid & 7;
+        if (e0 + ((tid >> 5) << 2) >= m) continue;          // none of this warp's four members exists (warp-uniform)
+        const unsigned ke = e < m ? tie_k[e] : 0u;
+        const int ie = e < m ? tie_i[e] : 0;
+        int rank = 0;
+        for (int f = part; f < m; f += 8) {
+            const unsigned kf = tie_k[f];
+            rank += (kf > ke || (kf == ke && tie_i[f] < ie)) ? 1 : 0;
+        }
+        rank += __shfl_xor_sync(kFullMask, rank, 1);
+        rank += __shfl_xor_sync(kFullMask, rank, 2);
+        rank += __shfl_xor_sync(kFullMask, rank, 4);
+        if (e < m && part == 0 && rank < need) raw_s[above + rank] = ie;
+    }
+    __syncthreads();
+    return true;
+}
+
+// Ascending chunk ids: position = number of selected ids below mine (eight lanes share an element).  Called by every
+// thread; ends with a barrier.
+__device__ void sort_ids_ascending(const int* raw_s, int* sel_s, int n) {
+    const int tid = threadIdx.x, NT = blockDim.x;
+    for (int t0 = 0; t0 < n; t0 += NT / 8) {
+        const int t = t0 + (tid >> 3), part = tid & 7;
+        if (t0 + ((tid >> 5) << 2) >= n) continue;           // none of this warp's four elements exists (warp-uniform)
+        const int idt = t < n ? raw_s[t] : 0;
+        int pos = 0;
+        for (int j = part; j < n; j += 8) pos += raw_s[j] < idt ? 1 : 0;
+        pos += __shfl_xor_sync(kFullMask, pos, 1);
+        pos += __shfl_xor_sync(kFullMask, pos, 2);
+        pos += __shfl_xor_sync(kFullMask, pos, 4);
+        if (t < n && part == 0) sel_s[pos] = idt;
+    }
+    __syncthreads();
 }
 
 // Exact top-K of the group scores of one (sequence, KV head) pair (ties: lower chunk id), ascending ids,
@@ -196,12 +357,17 @@ __device__ void select_pair(const DArgs& a, int pair, int ncand, SelShared& sh, 
     const float* u = a.u + static_cast<long long>(pair) * a.Cpad;
     int* sel_s = sh.sel_s;
     int (*whist)[256] = reinterpret_cast<int (*)[256]>(dyn);
-    unsigned* keys = reinterpret_cast<unsigned*>(dyn + static_cast<size_t>(nw) * 256 * sizeof(int));
-    const bool cached = ncand <= kSelKeyCap;
+    unsigned* keys = reinterpret_cast<unsigned*>(dyn + sel_hist_ints(nw) * sizeof(int));
+    // room for the keys was requested at launch only if the longest possible list fits (see launch_decode_fast)
+    const bool cached = (s.T - 1) / kS < kSelKeyCap;
 
     if (ncand <= K) {
         for (int t = tid; t < K; t += NT) sel_s[t] = t < ncand ? t : -1;
         __syncthreads();
+    } else if (ncand <= kSelRegKeys * NT &&
+               select_in_registers(sh.st, reinterpret_cast<int*>(dyn), u, ncand, K, sh.raw_s, keys,
+                                   reinterpret_cast<int*>(keys + kSelTieCap))) {
+        sort_ids_ascending(sh.raw_s, sel_s, n);
     } else {
         if (cached) {
             // the scores come from L2: sixteen loads in flight per thread; the histogram of the keys' leading byte
@@ -249,18 +415,7 @@ __device__ void select_pair(const DArgs& a, int pair, int ncand, SelShared& sh, 
             }
         }
         __syncthreads();
-        // --- ascending chunk ids: position = number of selected ids below mine (eight lanes share an element)
-        for (int t0 = 0; t0 < n; t0 += NT / 8) {
-            const int t = t0 + (tid >> 3), part = tid & 7;
-            const int idt = t < n ? sh.raw_s[t] : 0;
-            int pos = 0;
-            for (int j = part; j < n; j += 8) pos += sh.raw_s[j] < idt ? 1 : 0;
-            pos += __shfl_xor_sync(kFullMask, pos, 1);
-            pos += __shfl_xor_sync(kFullMask, pos, 2);
-            pos += __shfl_xor_sync(kFullMask, pos, 4);
-            if (t < n && part == 0) sel_s[pos] = idt;
-        }
-        __syncthreads();
+        sort_ids_ascending(sh.raw_s, sel_s, n);
     }
     for (int t = tid; t < K; t += NT) sel[t] = t < n ? sel_s[t] : -1;
     // --- per-head surrogate scores of the selected chunks and the fusion weights: the selected
