@@ -157,8 +157,10 @@ def params_for(hils, cfg, decode, impl="auto", window=1):
 class Workload:
     """Device-resident inputs/outputs of one configuration and the call that runs one step."""
 
-    def __init__(self, hils, cfg, device, n_query_sets=8, window=1, with_bias=False, overlap_block=0):
+    def __init__(self, hils, cfg, device, n_query_sets=8, window=1, with_bias=False, overlap_block=0,
+                 overlap_noise=0.3, impl="auto"):
         self.hils, self.cfg, self.dev = hils, cfg, device
+        self.impl = impl                         # prefill only: "packed" = the query-major kernel (Sec. 4.2)
         self.decode = cfg.mode == "decode"
         self.window = window                     # prefill only; > 1 = the paper's operator form (Sec. 2.1)
         self.bias = wl.make_bias(cfg, device) if with_bias else None
@@ -177,7 +179,7 @@ class Workload:
             self.work, self.work_aux = lm_b + kv_b, kv_b
             self.unit, self.metric = "GB/s", "hils_decode_algorithmic_GBps"
         else:
-            self.inp = wl.make_prefill_inputs(cfg, device, overlap_block=overlap_block)
+            self.inp = wl.make_prefill_inputs(cfg, device, overlap_block=overlap_block, overlap_noise=overlap_noise)
             self.out = torch.empty_like(self.inp["q"])
             self.lse = torch.empty((cfg.B, cfg.Hq, cfg.L), dtype=torch.float32, device=device)
             self.sel = torch.empty((cfg.B, cfg.Hkv, cfg.L, cfg.K), dtype=torch.int32, device=device)
@@ -198,7 +200,8 @@ class Workload:
                                   out=self.out, lse=self.lse, sel_idx=self.sel, workspace=self.ws)
         else:
             self.hils.hils_prefill(i["q"], i["k"], i["v"], i["landmarks"], self.cfg.S, self.cfg.K, bias=self.bias,
-                                   window=self.window, out=self.out, lse=self.lse, sel_idx=self.sel, workspace=self.ws)
+                                   window=self.window, impl=self.impl, out=self.out, lse=self.lse, sel_idx=self.sel,
+                                   workspace=self.ws)
 
     def between_steps(self):
         if self.flush is not None:
@@ -428,6 +431,35 @@ def bench_backward(hils, w, peaks, steps, barrier):
                 w.inp["q"].numel() * 2 / 1e6, w.inp["q"].numel() * 4 / 1e6)}
 
 
+def bench_packed(hils, dev, barrier):
+    """The query-major packed kernel (tiles of 16 adjacent tokens over the union of their chunks, Sec. 4.2 and App.
+    "Chunk Overlap") beside the chunk-major kernels on queries that share their chunks: one base query per 16 adjacent
+    tokens plus noise.  Returns (results, launches)."""
+    res, launches = {}, 0
+    for name in ("cfg1", "cfg2"):
+        cfg = pick_cfg(name)
+        for noise in (0.3, 0.03):
+            row = {}
+            for impl in ("auto", "packed"):
+                torch.cuda.empty_cache()
+                w = Workload(hils, cfg, dev, overlap_block=16, overlap_noise=noise, impl=impl)
+                ms, _ = time_steps(w, 3, 3, barrier)
+                launches += hils.last_launch_count() * 6
+                key = "chunk_major" if impl == "auto" else "packed"
+                row[key + "_ms"] = float(np.mean(ms))
+                row[key + "_TFLOPs"] = w.rate(float(np.mean(ms)) * 1e-3)
+                if impl == "packed":
+                    st, _ = hils.hils_chunk_overlap(w.sel, 16, cfg.C)
+                    launches += 1
+                    full = st[..., 0] > 0
+                    row["mean_union_chunks"] = float(st[..., 1][full].float().mean().item())
+                    row["slots_per_block"] = 16 * cfg.K
+                del w
+            res["%s_noise_%g" % (name, noise)] = row
+    torch.cuda.empty_cache()
+    return res, launches
+
+
 def bench_chunk_overlap(hils, w, peaks, M=16, iters=10):
     """Chunk-id overlap of blocks of M adjacent queries (Sec. "Chunk Overlap", Eq. Overlap) on the selection the
     workload's last prefill wrote: the statistics, and the kernel's time against reading sel_idx once."""
@@ -594,6 +626,11 @@ def main():
     ap.add_argument("--profile-run", action="store_true",
                     help="only run warmup+steps calls of the workload (for ncu captures); no timing extras")
     ap.add_argument("--batch", type=int, default=0, help="profile runs: override the batch size (smaller footprint)")
+    ap.add_argument("--prefill-impl", choices=["auto", "packed"], default="auto",
+                    help="profile runs: the prefill kernel set (packed = query-major tiles of adjacent tokens)")
+    ap.add_argument("--overlap-block", type=int, default=0,
+                    help="profile runs: one base query per this many adjacent tokens (0 = independent queries)")
+    ap.add_argument("--overlap-noise", type=float, default=0.3, help="profile runs: noise added to the base queries")
     args = ap.parse_args()
     if args.gpus > 1 and "RANK" not in os.environ:
         sys.exit(spawn_ranks(args.gpus, sys.argv[1:]))
@@ -606,12 +643,18 @@ def main():
         cfg = pick_cfg(args.workload)
         if args.batch > 0:
             cfg = cfg.scaled(B=args.batch)
-        w = Workload(hils, cfg, torch.device("cuda", 0), n_query_sets=2)
+        w = Workload(hils, cfg, torch.device("cuda", 0), n_query_sets=2, overlap_block=args.overlap_block,
+                     overlap_noise=args.overlap_noise, impl=args.prefill_impl)
         for _ in range(args.warmup + args.steps):
             w.between_steps()
             w.step()
         torch.cuda.synchronize()
         kpc = hils.last_launch_count()
+        if args.prefill_impl != "auto":
+            print(json.dumps({"profile_run": cfg.name, "B": cfg.B, "calls": args.warmup + args.steps,
+                              "kernels_per_call": kpc, "prefill_impl": args.prefill_impl,
+                              "overlap_block": args.overlap_block, "overlap_noise": args.overlap_noise}))
+            return
         # the chunk-summary kernel over the same key tensor (two calls)
         lq = wl.make_landmark_queries(cfg, w.inp["k"].device)
         for _ in range(2):
@@ -820,6 +863,8 @@ def main():
                         "chunk_overlap": bench_chunk_overlap(hils, sw, peaks)}
                     launches += hils.last_launch_count() * (max(3, args.steps) + 6) + 13
                     del sw
+                    extras["packed_vs_chunk_major"], n_l = bench_packed(hils, dev, barrier)
+                    launches += n_l
                     # the paper's operator form (Sec. 2.1 / experiments): local window W = 512 and a non-null bias
                     torch.cuda.empty_cache()
                     pw = Workload(hils, pick_cfg(name), dev, window=512, with_bias=True)

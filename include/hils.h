@@ -70,8 +70,14 @@ typedef enum { HILS_F32 = 0, HILS_BF16 = 1 } hils_dtype;
 
 /* Which implementation to run.  AUTO picks the fastest kernel set that supports the shape;
  * GENERIC forces the shape-agnostic CUDA-core kernels (any d multiple of 32 up to 256,
- * any chunk size up to 128, any window). */
-typedef enum { HILS_IMPL_AUTO = 0, HILS_IMPL_GENERIC = 1, HILS_IMPL_FAST = 2 } hils_impl;
+ * any chunk size up to 128, any window).  PACKED (prefill only; never chosen by AUTO) is the query-major kernel of
+ * Sec. 4.2 / App. "Chunk Overlap": tiles of 16 adjacent tokens x the query heads of a KV group walk the union of the
+ * chunks the tokens selected, pairs (token, chunk) that were not selected are masked, and the retrieval-weighted mix
+ * stays in registers until `out` is written once.  Its work grows with the size of that union, so it pays only where
+ * adjacent queries select nearly the same chunks; bf16, d = 128, chunk_size = 64, Hq = 4 Hkv, Hl = Hkv, top_k <= 32,
+ * at most 4096 chunks per sequence, slice offsets that are multiples of 16; other shapes return
+ * HILS_ERR_UNSUPPORTED.  Same results as the other kernels up to the order of the fp32 sums. */
+typedef enum { HILS_IMPL_AUTO = 0, HILS_IMPL_GENERIC = 1, HILS_IMPL_FAST = 2, HILS_IMPL_PACKED = 3 } hils_impl;
 
 typedef struct hils_params {
     int32_t B, Hq, Hkv;

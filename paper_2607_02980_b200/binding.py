@@ -17,8 +17,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libhils.so")
 
 HILS_F32, HILS_BF16 = 0, 1
-IMPL_AUTO, IMPL_GENERIC, IMPL_FAST = 0, 1, 2
-_IMPL = {"auto": IMPL_AUTO, "generic": IMPL_GENERIC, "fast": IMPL_FAST}
+IMPL_AUTO, IMPL_GENERIC, IMPL_FAST, IMPL_PACKED = 0, 1, 2, 3
+_IMPL = {"auto": IMPL_AUTO, "generic": IMPL_GENERIC, "fast": IMPL_FAST, "packed": IMPL_PACKED}
 
 EXPORTS = [
     "hils_workspace_bytes", "hils_prefill", "hils_decode", "hils_host_arena_bytes",

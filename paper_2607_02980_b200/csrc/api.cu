@@ -66,7 +66,7 @@ int make_shape(const hils_params* p, int is_decode, Shape* s, long long pos0 = 0
     if (p->Hq % p->Hkv != 0) return HILS_ERR_INVALID_ARG;
     if (p->Hl != p->Hkv && p->Hl != p->Hq) return HILS_ERR_INVALID_ARG;
     if (p->dtype != HILS_F32 && p->dtype != HILS_BF16) return HILS_ERR_INVALID_ARG;
-    if (p->impl < HILS_IMPL_AUTO || p->impl > HILS_IMPL_FAST) return HILS_ERR_INVALID_ARG;
+    if (p->impl < HILS_IMPL_AUTO || p->impl > HILS_IMPL_PACKED) return HILS_ERR_INVALID_ARG;
     if (!(p->scale >= 0.f)) return HILS_ERR_INVALID_ARG;
     s->B = p->B; s->Hq = p->Hq; s->Hkv = p->Hkv; s->Hl = p->Hl; s->G = p->Hq / p->Hkv;
     s->d = p->d; s->S = p->chunk_size; s->K = p->top_k; s->W = p->window;
@@ -93,10 +93,15 @@ int make_shape(const hils_params* p, int is_decode, Shape* s, long long pos0 = 0
     return HILS_OK;
 }
 
-enum class Path { Generic, DecodeFast, PrefillFast };
+enum class Path { Generic, DecodeFast, PrefillFast, PrefillPacked };
 
 int pick_path(const Shape& s, const hils_params* p, Path* path) {
     const bool fast_ok = s.is_decode ? decode_fast_supports(s, p->dtype) : prefill_fast_supports(s, p->dtype);
+    if (p->impl == HILS_IMPL_PACKED) {
+        if (s.is_decode || !prefill_packed_supports(s, p->dtype)) return HILS_ERR_UNSUPPORTED;
+        *path = Path::PrefillPacked;
+        return HILS_OK;
+    }
     if (p->impl == HILS_IMPL_FAST) {
         if (!fast_ok) return HILS_ERR_UNSUPPORTED;
         *path = s.is_decode ? Path::DecodeFast : Path::PrefillFast;
@@ -163,6 +168,7 @@ int run(const hils_params* p, int is_decode, const void* q, const void* k, const
     switch (path) {
         case Path::DecodeFast: n = launch_decode_fast(s, t, stream); break;
         case Path::PrefillFast: n = launch_prefill_fast(s, t, stream); break;
+        case Path::PrefillPacked: n = launch_prefill_packed(s, t, stream); break;
         default: n = launch_generic(s, p->dtype, t, stream); break;
     }
     if (n < 0) return n;

@@ -132,6 +132,11 @@ bool chunk_overlap_supports(int C);
 int launch_chunk_overlap(int pairs, int R, int K, int C, int M, const int32_t* sel, int32_t* stats, float* overlap,
                          cudaStream_t stream);
 
+// Query-major packed prefill (HILS_IMPL_PACKED): selection by the tcgen05 kernel, then tiles of 16 adjacent tokens over
+// the union of their chunks; needs no scratch beyond the status block.
+bool prefill_packed_supports(const Shape& s, int dtype);
+int launch_prefill_packed(const Shape& s, const Tensors& t, cudaStream_t stream);
+
 int launch_prefill_fast(const Shape& s, const Tensors& t, cudaStream_t stream);
 bool prefill_fast_supports(const Shape& s, int dtype);
 size_t prefill_fast_scratch_bytes(const Shape& s);
