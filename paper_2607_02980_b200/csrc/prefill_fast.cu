@@ -112,7 +112,8 @@ prefill_select_kernel(const __grid_constant__ CUtensorMap map_lm, const PArgs a)
     const int ci = tiles_per_seq - 1 - static_cast<int>(blockIdx.x) / pairs;      // heavy tiles first
     const int pair = static_cast<int>(blockIdx.x) % pairs;
     const int b = pair / s.Hkv, gk = pair % s.Hkv;
-    const int ncand = ci;                       // W = 1: every earlier chunk is a candidate
+    // candidates of a token = the chunks left of its local window (Sec. 2.1); the tile's last token has the most
+    const int ncand = local_lo(s.pos0 + min(s.R, (ci + 1) * kS) - 1, s.W, kS) / kS;
     const int nst = (ncand + kS - 1) / kS;
     const int K = s.K, Kp = K + 1;
 
@@ -145,6 +146,7 @@ prefill_select_kernel(const __grid_constant__ CUtensorMap map_lm, const PArgs a)
     const unsigned qmask = 0xfu << (lane & ~3);
     const int tokA = ci * kS + warp * 16 + g, tokB = tokA + 8;
     const int ldA = min(tokA, s.R - 1), ldB = min(tokB, s.R - 1);
+    const int ncA = local_lo(s.pos0 + ldA, s.W, kS) / kS, ncB = local_lo(s.pos0 + ldB, s.W, kS) / kS;
 
     // A operands: this warp's 16 tokens, one fragment set per head of the group
     uint32_t aq[kG][8][4];
@@ -203,9 +205,10 @@ prefill_select_kernel(const __grid_constant__ CUtensorMap map_lm, const PArgs a)
 #pragma unroll
             for (int v = 0; v < 4; ++v) {
                 const int c = cb + (v & 1);
+                const int nc_tok = v < 2 ? ncA : ncB;
                 float u = um[v] * s.scale;
-                if (bias && c < ncand) u += bias[c];
-                key[v] = c < ncand ? select_key(u, c) : 0ull;
+                if (bias && c < nc_tok) u += bias[c];
+                key[v] = c < nc_tok ? select_key(u, c) : 0ull;
                 any |= key[v] > ((v < 2) ? tauA : tauB);
             }
             if (__ballot_sync(kFullMask, any) == 0u) continue;
@@ -602,9 +605,10 @@ Plan make_plan(const Shape& s, int qb_fixed = 0) {
 }  // namespace
 
 bool prefill_fast_supports(const Shape& s, int dtype) {
-    // any window whose chunks fit the fuse kernel's row table; the warp-MMA selection fallback (K > 32) knows W = 1 only
+    // any window whose chunks fit the fuse kernel's row table; the warp-MMA selection fallback (K > 32) scores one
+    // landmark row per KV head
     return dtype == HILS_BF16 && !s.is_decode && s.d == kD && s.S == kS && s.W >= 1 && max_local_slots(s.W) <= 16 &&
-           ((s.W == 1 && s.pos0 == 0 && s.Hl == s.Hkv) || (s.K <= 32 && prefill_select_tc_supports(s))) &&
+           (s.Hl == s.Hkv || (s.K <= 32 && prefill_select_tc_supports(s))) &&
            (s.Hl == s.Hkv || s.Hl == s.Hq) && s.G == kG &&
            s.K >= 1 && s.K <= 64 && static_cast<long long>(s.B) * s.Hkv * s.T < (1ll << 31) &&
            static_cast<long long>(s.B) * s.Hkv * s.C < (1ll << 24) &&

@@ -74,6 +74,12 @@ def test_argument_errors_are_returned_before_any_launch():
     assert call_prefill(good(), ws_bytes=16) == -4
     assert call_prefill(good(d=48)) == -2
     assert call_prefill(good(impl="fast", dtype=binding.HILS_F32)) == -2
+    # the packed query-major kernel: bf16, d = 128, four query heads per KV head, top_k <= 32, prefill only
+    assert call_prefill(good(impl="packed", dtype=binding.HILS_F32)) == -2
+    assert call_prefill(good(impl="packed", Hq=4)) == -2
+    assert call_prefill(good(impl="packed", top_k=33, C=64, L=4096, T_max=4096)) == -2
+    assert hils.workspace_bytes(good(impl="packed"), False) >= 256
+    assert hils.workspace_bytes(good(impl="packed"), True) == 0
     assert lib.hils_prefill(None, None, None, None, None, None, None, None, None, None, 0, None) == -1
     vp = ctypes.c_void_p
     p = good()

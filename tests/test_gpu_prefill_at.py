@@ -52,6 +52,20 @@ def test_slice_of_a_sequence_matches_the_oracle(impl, pos0, L, W):
     compare(cfg, inp, pos0, L, got, bias, W)
 
 
+@pytest.mark.parametrize("pos0,L,W", [(0, 3100, 200), (2049, 1500, 512), (1000, 900, 1)])
+def test_more_than_32_chunks_per_query_with_window_and_offset_on_the_fast_path(pos0, L, W):
+    """top_k between 33 and 64 takes the warp-MMA selection kernel: any window, any slice offset."""
+    cfg = wl.CONFIGS[1].scaled(B=1, Hq=8, Hkv=2, L=pos0 + L, K=40, seed=95)
+    inp = wl.make_prefill_inputs(cfg, "cpu")
+    bias = wl.make_bias(cfg, "cpu")
+    g = {n: t.to(DEV) for n, t in inp.items()}
+    q = g["q"][:, :, pos0:pos0 + L].contiguous()
+    got = hils.hils_prefill_at(q, g["k"], g["v"], g["landmarks"], cfg.S, cfg.K, pos0, bias=bias.to(DEV), window=W,
+                               impl="fast")
+    torch.cuda.synchronize()
+    compare(cfg, inp, pos0, L, got, bias, W)
+
+
 def test_two_slices_reproduce_the_whole_sequence_prefill_bit_for_bit():
     cfg = wl.CONFIGS[1].scaled(B=1, Hq=8, Hkv=2, L=6000, K=12, seed=92)
     inp = wl.make_prefill_inputs(cfg, "cpu")
