@@ -1,5 +1,5 @@
-// Tensor-core prefill kernels: bf16, d = 128, S = 64, G = 4, one landmark per KV head, any local window of up to
-// 16 chunks (W <= 897; K > 32 needs W = 1).
+// Tensor-core prefill kernels: bf16, d = 128, S = 64, G = 4, any local window of up to 16 chunks (W <= 897), one
+// landmark per KV head or per query head (the latter with K <= 32: the tcgen05 selection kernel).
 //
 // With independent queries the tokens that select a chunk are scattered over the sequence, so the
 // path is organised CHUNK-MAJOR: K/V of a chunk are staged once and reused by every query row that
