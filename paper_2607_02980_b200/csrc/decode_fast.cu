@@ -108,7 +108,7 @@ constexpr int kSelMaxWarps = 32;
 constexpr int kSelKeyCap = 40960;            // keys cached in shared memory (160 KB); longer lists re-read the scores
 constexpr int kSelTieCap = 512;              // candidates of the boundary bin that are ranked directly
 constexpr int kSelRegKeys = 16;              // keys a thread holds in registers on the short way
-constexpr int kSelBins = 2048;               // counters of the short way's histogram
+constexpr int kSelBins = 2048;               // counters of the short way's histogram (at most: about half a bin per candidate)
 
 struct SelState {
     int hist[256];                           // summed histogram of the current pass
@@ -258,7 +258,11 @@ __device__ bool select_in_registers(SelState& st, int* hist, const float* u, int
         const int i = x * NT + tid;
         v[x] = i < n ? __ldcg(u + i) : 0.f;
     }
-    for (int x = tid; x < kSelBins; x += NT) hist[x] = 0;
+    // about two candidates per bin: the bin of the K-th best score then holds a handful, and short lists do not pay
+    // for zeroing and walking counters they cannot fill
+    int nbins = 256;
+    while (nbins < kSelBins && 2 * nbins < n) nbins <<= 1;
+    for (int x = tid; x < nbins; x += NT) hist[x] = 0;
     if (tid == 0) { st.nout = 0; st.ntie = 0; st.kmin = 0xffffffffu; st.kmax = 0u; }
     __syncthreads();
     // span of the scores
@@ -276,16 +280,16 @@ __device__ bool select_in_registers(SelState& st, int* hist, const float* u, int
     if (lane == 0) { atomicMin(&st.kmin, kmin); atomicMax(&st.kmax, kmax); }
     __syncthreads();
     const float lo = key_to_float(st.kmin), hi = key_to_float(st.kmax);
-    const float inv = static_cast<float>(kSelBins) / (hi - lo);
+    const float inv = static_cast<float>(nbins) / (hi - lo);
     // (no span, or a span that is not a number: every candidate would land in one bin)
     if (!(hi > lo) || !(inv > 0.f) || !(inv < INFINITY)) return false;
     // bin of a score: the same expression wherever it is needed, non-decreasing in the score
-    auto bin_of = [&](float x) { return min(kSelBins - 1, max(0, static_cast<int>((x - lo) * inv))); };
+    auto bin_of = [&](float x) { return min(nbins - 1, max(0, static_cast<int>((x - lo) * inv))); };
 #pragma unroll
     for (int x = 0; x < kSelRegKeys; ++x)
         if (x * NT + tid < n) atomicAdd(&hist[bin_of(v[x])], 1);
     __syncthreads();
-    scan_from_top(st, hist, kSelBins, want);
+    scan_from_top(st, hist, nbins, want);
     const int bstar = st.bstar, above = st.above, m = st.equal;
     if (m > kSelTieCap) return false;
 #pragma unroll
@@ -564,6 +568,162 @@ __global__ void __launch_bounds__(kScoreThreads) decode_score_kernel(const DArgs
         const int ca = c0[it] + gq, cb = ca + 8;
         if (t == 0 && ca < ncand) u[ca] = best[it][0];
         if (t == 1 && cb < ncand) u[cb] = best[it][1];
+    }
+    STAMP_MAX(1);
+    pdl_launch_dependents();
+}
+
+// The same scores from a persistent kernel that streams the landmark rows through a TMA ring (one landmark row per KV
+// head: Hl = Hkv).  decode_score_kernel above runs 2048 short CTAs that each request their 64 KB, wait, compute and
+// leave: the bytes in flight drop to zero between a CTA's loads and its successor's.  Here one CTA per SM keeps
+// kScStages tiles of 64 landmark rows (16 KB each) requested at all times; the valid tiles of all (sequence, KV head)
+// pairs form one list that is cut into equal contiguous ranges, a tile is scored by the warp that owns its stage
+// (landmark rows as the B operand of the warp-level MMA, the G query heads in the A rows), the maximum over the heads
+// is taken with shuffles and the 64 group scores are written.
+constexpr int kScStages = 12;
+constexpr int kScStageBytes = kS * kD * 2;
+constexpr int kScWarps = 6;                // consumer warps: a stage is always consumed by the same warp
+constexpr int kScThreads = (kScWarps + 1) * 32;
+constexpr int kScMaxPairs = 4096;            // prefix of the pairs' tile counts in shared memory
+static_assert(kScStages % kScWarps == 0, "stage ownership must be fixed per consumer warp");
+
+struct ScoreSmem {
+    uint64_t full[kScStages];
+    uint64_t empty[kScStages];
+    int pref[kScMaxPairs + 1];               // tiles of the pairs before pair p
+    int wsum[kScThreads / 32];
+    int dead;
+};
+
+__global__ void __launch_bounds__(kScThreads, 1)
+decode_score_stream_kernel(const __grid_constant__ CUtensorMap map_lm, const DArgs a) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    ScoreSmem& sm = *reinterpret_cast<ScoreSmem*>(ring + kScStages * kScStageBytes);
+    const Shape& s = a.s;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int pairs = s.B * s.Hkv;
+    STAMP_MIN(0);
+    if (tid == 0) {
+        for (int i = 0; i < kScStages; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], 1); }
+        mbar_fence_init();
+        sm.dead = 0;
+        sm.pref[0] = 0;
+        tma_prefetch_desc(&map_lm);
+    }
+    __syncthreads();
+    // tiles of 64 candidates per pair (0 for an invalid length), inclusive scan over the pairs
+    auto pair_ncand = [&](int pr) {
+        const int seq = query_seq_len(a, pr / s.Hkv);
+        return (seq < 1 || seq > s.T) ? 0 : first_local_chunk(seq, s.W);
+    };
+    // (thread t sums the tile counts of its pairs [t ppt, (t + 1) ppt), one scan over the threads, then each thread
+    //  writes its pairs' entries: two barriers whatever the number of pairs)
+    {
+        const int ppt = (pairs + kScThreads - 1) / kScThreads;
+        const int p_begin = min(pairs, tid * ppt), p_end = min(pairs, p_begin + ppt);
+        int mine = 0;
+        for (int pr = p_begin; pr < p_end; ++pr) mine += (pair_ncand(pr) + kS - 1) / kS;
+        int inc = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int nn = __shfl_up_sync(kFullMask, inc, o);
+            if (lane >= o) inc += nn;
+        }
+        if (lane == 31) sm.wsum[warp] = inc;
+        __syncthreads();
+        int run = inc - mine;
+        for (int w = 0; w < warp; ++w) run += sm.wsum[w];
+        for (int pr = p_begin; pr < p_end; ++pr) {
+            run += (pair_ncand(pr) + kS - 1) / kS;
+            sm.pref[pr + 1] = run;
+        }
+        __syncthreads();
+    }
+    const long long total = sm.pref[pairs];
+    const int lo = static_cast<int>(total * blockIdx.x / gridDim.x), hi = static_cast<int>(total * (blockIdx.x + 1) / gridDim.x);
+    // pair of the range's first tile: last p with pref[p] <= lo
+    int p_lo = 0;
+    {
+        int l = 0, r = pairs;                     // invariant: pref[l] <= lo < pref[r] (when lo < total)
+        while (r - l > 1) {
+            const int m = (l + r) >> 1;
+            if (sm.pref[m] <= lo) l = m; else r = m;
+        }
+        p_lo = l;
+    }
+    if (hi > lo) {
+        if (warp == kScWarps) {
+            // ------------------------------------------------------------------ producer (one lane)
+            if (lane == 0) {
+                int pr = p_lo;
+                for (int x = lo; x < hi; ++x) {
+                    while (sm.pref[pr + 1] <= x) ++pr;
+                    const int k = x - lo, st = k % kScStages;
+                    if (k >= kScStages && !mbar_wait(&sm.empty[st], ((k / kScStages) - 1) & 1)) {
+                        set_status(a.status, kDevTimeout);
+                        atomicExch(&sm.dead, 1);
+                        break;
+                    }
+                    const int b = pr / s.Hkv, g = pr % s.Hkv;
+                    const int row = ((b / s.qps) * s.Hl + g) * s.C + (x - sm.pref[pr]) * kS;
+                    uint8_t* dst = ring + st * kScStageBytes;
+                    mbar_expect_tx(&sm.full[st], kScStageBytes);
+                    tma_load_2d(dst, &map_lm, &sm.full[st], 0, row);
+                    tma_load_2d(dst + 8192, &map_lm, &sm.full[st], 64, row);
+                }
+            }
+        } else {
+            // ------------------------------------------------------------------ consumers
+            const int gq = lane >> 2, t = lane & 3;
+            int pr = p_lo, cur = -1;
+            uint32_t aq[8][2];
+            for (int x = lo + warp; x < hi; x += kScWarps) {
+                while (sm.pref[pr + 1] <= x) ++pr;
+                const int b = pr / s.Hkv, g = pr % s.Hkv;
+                if (pr != cur) {
+                    cur = pr;
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) { aq[ks][0] = 0u; aq[ks][1] = 0u; }
+                    if (gq < s.G) {
+                        const __nv_bfloat16* qrow = a.q_route + (static_cast<long long>(b) * s.Hq + g * s.G + gq) * kD;
+#pragma unroll
+                        for (int ks = 0; ks < 8; ++ks) {
+                            aq[ks][0] = *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 2 * t);
+                            aq[ks][1] = *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 8 + 2 * t);
+                        }
+                    }
+                }
+                const int k = x - lo, st = k % kScStages;
+                if (!mbar_wait(&sm.full[st], (k / kScStages) & 1)) {
+                    if (lane == 0) { set_status(a.status, kDevTimeout); atomicExch(&sm.dead, 1); }
+                    break;
+                }
+                float sc[8][4];
+                qk_tile(aq, smem_u32(ring + st * kScStageBytes), lane, sc);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.empty[st]);
+                // sc[nt][0..1]: head gq, chunks c0 + 8 nt + 2 t + {0, 1}: maximum over the G heads (rows gq >= G are padding)
+                const int c0 = (x - sm.pref[pr]) * kS;
+                const int ncand = pair_ncand(pr);
+                const float* bias = a.bias ? a.bias + (static_cast<long long>(b / s.qps) * s.Hl + g) * s.C : nullptr;
+                float* u = a.u + static_cast<long long>(pr) * a.Cpad;
+#pragma unroll
+                for (int nt = 0; nt < 8; ++nt) {
+                    float m0 = gq < s.G ? sc[nt][0] : -INFINITY, m1 = gq < s.G ? sc[nt][1] : -INFINITY;
+#pragma unroll
+                    for (int o = 4; o < 32; o <<= 1) {
+                        m0 = fmaxf(m0, __shfl_xor_sync(kFullMask, m0, o));
+                        m1 = fmaxf(m1, __shfl_xor_sync(kFullMask, m1, o));
+                    }
+                    const int ca = c0 + nt * 8 + 2 * t;
+                    if (gq == 0) {
+                        if (ca < ncand) u[ca] = m0 * s.scale + (bias ? bias[ca] : 0.f);
+                        if (ca + 1 < ncand) u[ca + 1] = m1 * s.scale + (bias ? bias[ca + 1] : 0.f);
+                    }
+                }
+            }
+        }
     }
     STAMP_MAX(1);
     pdl_launch_dependents();
@@ -887,6 +1047,13 @@ decode_attend_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_con
     STAMP_MAX(7);
 }
 
+// HILS_DECODE_SCORE=segments keeps the scoring kernel with one CTA per 256-chunk segment even where the streaming one
+// applies (for tuning runs and to cross-check the two).
+const bool g_score_per_segment = [] {
+    const char* e = getenv("HILS_DECODE_SCORE");
+    return e != nullptr && e[0] == 's';
+}();
+
 struct Plan {
     int n_ctas, max_parts, Cpad;
     size_t off_u, off_wgt, off_R, off_E, off_n, off_done, off_part, off_loco, off_loclam, total;
@@ -985,8 +1152,23 @@ int launch_decode_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
         attr_once.done();
     }
 
-    const int nseg = (s.C + kScoreChunksPerCta - 1) / kScoreChunksPerCta;
-    decode_score_kernel<<<dim3(nseg > 0 ? nseg : 1, pairs), kScoreThreads, 0, stream>>>(a);
+    if (s.Hl == s.Hkv && pairs <= kScMaxPairs && !g_score_per_segment) {
+        CUtensorMap map_lm;
+        if (!make_bf16_2d_map(&map_lm, t.landmarks, static_cast<uint64_t>(s.B / s.qps) * s.Hl * s.C, kD, 64, kS))
+            return HILS_ERR_CUDA;
+        const size_t sc_smem = kScStages * kScStageBytes + sizeof(ScoreSmem) + 1024;
+        static PerDeviceOnce sc_once;
+        if (sc_once.pending()) {
+            if (cudaFuncSetAttribute(decode_score_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     static_cast<int>(sc_smem)) != cudaSuccess)
+                return HILS_ERR_CUDA;
+            sc_once.done();
+        }
+        decode_score_stream_kernel<<<sm_count(), kScThreads, sc_smem, stream>>>(map_lm, a);
+    } else {
+        const int nseg = (s.C + kScoreChunksPerCta - 1) / kScoreChunksPerCta;
+        decode_score_kernel<<<dim3(nseg > 0 ? nseg : 1, pairs), kScoreThreads, 0, stream>>>(a);
+    }
     if (cudaGetLastError() != cudaSuccess) return HILS_ERR_CUDA;
     trace_mark("decode_score", stream);
 
