@@ -126,14 +126,15 @@ int hils_decode(const hils_params* params, const void* q, const void* k_cache, c
  * free HBM to its own KV-cache pool at start-up, so that a later cudaMalloc fails; a plugin that is
  * only passed the tensors of one layer and has no allocator handle; a latency-critical loop that
  * may not call cudaMalloc because it synchronises the device.  For them this call computes exactly
- * what hils_decode computes (same kernels, same results) but keeps its scratch in a fixed 8 MiB array
+ * what hils_decode computes (same kernels, same results) but keeps its scratch in a fixed 16 MiB array
  * that is part of the library image itself; every GPU that loads libhils.so holds that array until
  * the process exits.  The caller still passes every input and output.
  *
  *  - Nothing is allocated or freed, by CUDA or otherwise, on any call.
  *  - Limit: the decode workspace of the shape, hils_workspace_bytes(params, 1) (its 256-byte status block
- *    included), must fit in 8 MiB, otherwise HILS_ERR_WORKSPACE is returned before anything is launched (both benchmark decode shapes fit: B=64 x 64K tokens with
- *    K=32 needs about 5.3 MiB, B=4 x 1M tokens with K=64 about 2.5 MiB).  Shapes outside the
+ *    included), must fit in 16 MiB, otherwise HILS_ERR_WORKSPACE is returned before anything is launched (both benchmark decode shapes fit: B=64 x 64K tokens with
+ *    K=32 needs about 13.7 MiB, B=4 x 1M tokens with K=64 about 10.9 MiB; most of it is the table of per-head
+ *    landmark scores, B x Hq x C floats).  Shapes outside the
  *    bandwidth-tuned decode kernels (bf16, d=128, chunk 64, window <= 897, one landmark per KV or per query head,
  *    at most 8 query heads per KV head) return HILS_ERR_UNSUPPORTED.
  *  - The first call on each device looks up the array's device address (with that device current);

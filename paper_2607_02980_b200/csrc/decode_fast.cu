@@ -59,6 +59,7 @@ struct DArgs {
     int* status;
     // scratch
     float* u;          // [pairs, Cpad] group scores
+    float* uh;         // [pairs, G, Cpad] per-head scores (written by the streaming scoring kernel), or NULL
     int Cpad;
     float* wgt;        // [pairs, G, K] exp(s^h_c - R_h) of the selected chunks
     float* Rh;         // [pairs, G]    max_c s^h_c over the selected chunks
@@ -425,6 +426,13 @@ __device__ void select_pair(const DArgs& a, int pair, int ncand, SelShared& sh, 
     // --- per-head surrogate scores of the selected chunks and the fusion weights: the selected
     //     landmark rows and the G queries are staged in shared memory with one round of 16-byte
     //     loads, then every thread computes (chunk, head) dot products
+    if (a.uh) {
+        // the scoring kernel left every head's scores behind: pick the selected chunks' out of that table
+        for (int x = tid; x < n * G; x += NT) {
+            const int t = x / G, h = x % G;
+            sh.lam_s[h][t] = __ldcg(a.uh + (static_cast<long long>(pair) * G + h) * a.Cpad + sel_s[t]);
+        }
+    } else {
     __nv_bfloat16 (*lm_s)[kD + 8] = reinterpret_cast<__nv_bfloat16 (*)[kD + 8]>(dyn);
     const int per = s.Hl / s.Hkv;                        // landmark rows per chunk: 1, or one per query head (G)
     const long long lrow0 = (static_cast<long long>(b / s.qps) * s.Hl + g * per) * s.C;      // landmark head 0 of this KV head
@@ -469,6 +477,7 @@ __device__ void select_pair(const DArgs& a, int pair, int ncand, SelShared& sh, 
             const float bb = a.bias ? a.bias[lrow0 + static_cast<long long>(hh) * s.C + sel_s[t0 + t]] : 0.f;
             sh.lam_s[h][t0 + t] = acc * s.scale + bb;
         }
+    }
     }
     __syncthreads();
     for (int h = warp; h < G; h += nw) {
@@ -699,27 +708,48 @@ decode_score_stream_kernel(const __grid_constant__ CUtensorMap map_lm, const DAr
                     if (lane == 0) { set_status(a.status, kDevTimeout); atomicExch(&sm.dead, 1); }
                     break;
                 }
-                float sc[8][4];
-                qk_tile(aq, smem_u32(ring + st * kScStageBytes), lane, sc);
+                // D[chunk][head] = landmark rows (A, 16 chunks per tile of the MMA, straight from the swizzled stage) x q^T
+                // (B: the G heads in the columns): every A row is a chunk, and the maximum over the heads is a maximum
+                // over a thread's own two columns and its neighbours'
+                const uint32_t lm_addr = smem_u32(ring + st * kScStageBytes);
+                float acc[4][4];
+#pragma unroll
+                for (int mt = 0; mt < 4; ++mt) {
+                    acc[mt][0] = acc[mt][1] = acc[mt][2] = acc[mt][3] = 0.f;
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const int row = mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+                        const int dim = ks * 16 + (lane >> 4) * 8;
+                        uint32_t fr[4];
+                        ldmatrix_x4(lm_addr + (dim >> 6) * 8192 + swz128(row, (dim & 63) >> 3), fr[0], fr[1], fr[2], fr[3]);
+                        mma_bf16_16816(acc[mt], fr, aq[ks][0], aq[ks][1]);
+                    }
+                }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sm.empty[st]);
-                // sc[nt][0..1]: head gq, chunks c0 + 8 nt + 2 t + {0, 1}: maximum over the G heads (rows gq >= G are padding)
+                // acc[mt][0..1]: chunk c0 + 16 mt + gq, heads 2 t, 2 t + 1; acc[mt][2..3]: chunk + 8
                 const int c0 = (x - sm.pref[pr]) * kS;
                 const int ncand = pair_ncand(pr);
                 const float* bias = a.bias ? a.bias + (static_cast<long long>(b / s.qps) * s.Hl + g) * s.C : nullptr;
                 float* u = a.u + static_cast<long long>(pr) * a.Cpad;
+                float* uh0 = a.uh + (static_cast<long long>(pr) * s.G + 2 * t) * a.Cpad;       // head 2 t (2 t + 1: + Cpad)
+                const bool h0 = 2 * t < s.G, h1 = 2 * t + 1 < s.G;
 #pragma unroll
-                for (int nt = 0; nt < 8; ++nt) {
-                    float m0 = gq < s.G ? sc[nt][0] : -INFINITY, m1 = gq < s.G ? sc[nt][1] : -INFINITY;
+                for (int mt = 0; mt < 4; ++mt) {
 #pragma unroll
-                    for (int o = 4; o < 32; o <<= 1) {
-                        m0 = fmaxf(m0, __shfl_xor_sync(kFullMask, m0, o));
-                        m1 = fmaxf(m1, __shfl_xor_sync(kFullMask, m1, o));
-                    }
-                    const int ca = c0 + nt * 8 + 2 * t;
-                    if (gq == 0) {
-                        if (ca < ncand) u[ca] = m0 * s.scale + (bias ? bias[ca] : 0.f);
-                        if (ca + 1 < ncand) u[ca + 1] = m1 * s.scale + (bias ? bias[ca + 1] : 0.f);
+                    for (int half = 0; half < 2; ++half) {
+                        const int c = c0 + mt * 16 + half * 8 + gq;
+                        const float bb = (bias && c < ncand) ? bias[c] : 0.f;
+                        const float s0 = acc[mt][2 * half] * s.scale + bb, s1 = acc[mt][2 * half + 1] * s.scale + bb;
+                        // the head's own scores: the mixing logits of whatever chunks get selected (Eq. HiLS weights)
+                        if (c < ncand) {
+                            if (h0) uh0[c] = s0;
+                            if (h1) uh0[a.Cpad + c] = s1;
+                        }
+                        float m = fmaxf(h0 ? s0 : -INFINITY, h1 ? s1 : -INFINITY);
+                        m = fmaxf(m, __shfl_xor_sync(kFullMask, m, 1));
+                        m = fmaxf(m, __shfl_xor_sync(kFullMask, m, 2));
+                        if (t == 0 && c < ncand) u[c] = m;
                     }
                 }
             }
@@ -1056,8 +1086,13 @@ const bool g_score_per_segment = [] {
 
 struct Plan {
     int n_ctas, max_parts, Cpad;
-    size_t off_u, off_wgt, off_R, off_E, off_n, off_done, off_part, off_loco, off_loclam, total;
+    size_t off_u, off_uh, off_wgt, off_R, off_E, off_n, off_done, off_part, off_loco, off_loclam, total;
 };
+
+// The streaming scoring kernel (and with it the table of per-head scores) applies to one landmark row per KV head.
+bool score_streams(const Shape& s) {
+    return s.Hl == s.Hkv && static_cast<long long>(s.B) * s.Hkv <= kScMaxPairs && !g_score_per_segment;
+}
 
 Plan make_plan(const Shape& s, int n_sm) {
     Plan p;
@@ -1075,6 +1110,7 @@ Plan make_plan(const Shape& s, int n_sm) {
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = (off + bytes + 255) / 256 * 256; return o; };
     p.off_u = take(sizeof(float) * pairs * p.Cpad);
+    p.off_uh = take(score_streams(s) ? sizeof(float) * pairs * s.G * p.Cpad : 0);
     p.off_wgt = take(sizeof(float) * pairs * s.G * s.K);
     p.off_R = take(sizeof(float) * pairs * s.G);
     p.off_E = take(sizeof(float) * pairs * s.G);
@@ -1121,6 +1157,7 @@ int launch_decode_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
     a.sel = t.sel_idx;
     a.status = t.status;
     a.u = reinterpret_cast<float*>(sc + p.off_u);
+    a.uh = score_streams(s) ? reinterpret_cast<float*>(sc + p.off_uh) : nullptr;
     a.Cpad = p.Cpad;
     a.wgt = reinterpret_cast<float*>(sc + p.off_wgt);
     a.Rh = reinterpret_cast<float*>(sc + p.off_R);
@@ -1152,7 +1189,7 @@ int launch_decode_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
         attr_once.done();
     }
 
-    if (s.Hl == s.Hkv && pairs <= kScMaxPairs && !g_score_per_segment) {
+    if (score_streams(s)) {
         CUtensorMap map_lm;
         if (!make_bf16_2d_map(&map_lm, t.landmarks, static_cast<uint64_t>(s.B / s.qps) * s.Hl * s.C, kD, 64, kS))
             return HILS_ERR_CUDA;
@@ -1201,8 +1238,8 @@ int launch_decode_fast(const Shape& s, const Tensors& t, cudaStream_t stream) {
 
 // ------------------------------------------------------------------------- allocation-free variant
 // Scratch for callers that cannot obtain device memory themselves.  The array belongs to the loaded
-// library image: every GPU that loads libhils.so carries these 8 MiB until the process exits.
-constexpr size_t kNoAllocBytes = 8u << 20;
+// library image: every GPU that loads libhils.so carries these 16 MiB until the process exits.
+constexpr size_t kNoAllocBytes = 16u << 20;
 constexpr int kMaxDevices = 64;
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
 

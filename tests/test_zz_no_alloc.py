@@ -76,7 +76,7 @@ def test_noalloc_rejects_shapes_beyond_its_fixed_scratch():
     out = torch.empty_like(g["q"])
     lse = torch.empty((1, cfg.Hq), dtype=torch.float32, device=DEV)
     sel = torch.empty((1, cfg.Hkv, cfg.K), dtype=torch.int32, device=DEV)
-    # a cache far larger than 8 MiB of scratch allows: B*Hkv*C group scores alone exceed it
+    # a cache far larger than 16 MiB of scratch allows: B*Hkv*C group scores alone exceed it
     import ctypes
     from paper_2607_02980_b200 import binding
     big = hils.make_params(B=128, Hq=32, Hkv=8, Hl=8, L=0, T_max=1 << 20, C=1 << 14, d=128, chunk_size=64,
