@@ -48,8 +48,8 @@ constexpr int kOutWarp0 = kSoftThreads / 32;    // 8
 constexpr int kGatherWarps = 4;
 constexpr int kGatherWarp0 = kOutWarp0 + 4;     // 12 .. 15
 constexpr int kLoadWarp = kGatherWarp0 + kGatherWarps;   // 16
-constexpr int kMmaWarp = kLoadWarp + 1;         // 17
-constexpr int kThreads = (kMmaWarp + 1) * 32;   // 576
+constexpr int kMmaWarp = kLoadWarp + 1;         // 17, 18: one MMA issuer per tile parity
+constexpr int kThreads = (kMmaWarp + 2) * 32;   // 608
 constexpr float kLog2e = 1.4426950408889634f;
 
 struct AtcSmem {
@@ -126,7 +126,7 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
         for (int i = 0; i < kVBufs; ++i) { mbar_init(&sm.v_ready[i], 1); mbar_init(&sm.v_empty[i], 1); }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&sm.k_ready[i], 2);           // the TMA issuer's arrive.expect_tx + the landmark writer
-            mbar_init(&sm.k_empty[i], 1);
+            mbar_init(&sm.k_empty[i], 2);
             mbar_init(&sm.s_full[i], 1);
             mbar_init(&sm.s_empty[i], 4);
             mbar_init(&sm.p_full[i], 4);
@@ -228,9 +228,13 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                     // groups wait on are issued; those groups pass "this Q slot / K buffer / V buffer is free" on.
                     if (ti >= sm.cfirst[ck + 1]) ++ck;
                     const bool last = ti + 1 >= sm.cfirst[ck + 1];
+                    // The K buffer of a chunk run is free when the score MMAs of the run's last tile of EITHER parity are
+                    // done (the two parities have an issuing thread each, and a thread's MMAs complete in order): those
+                    // two tiles arrive once each on k_empty, a run of a single tile twice.
+                    const int karr = (ti + 2 >= sm.cfirst[ck + 1] ? 1 : 0) + (sm.cfirst[ck + 1] - sm.cfirst[ck] == 1 ? 1 : 0);
                     const uint32_t cc = ccount + static_cast<uint32_t>(ck);
                     sm.tile_meta[ms][0] = pair; sm.tile_meta[ms][1] = rec.y;
-                    sm.tile_meta[ms][2] = ntok | (last ? 256 : 0) | static_cast<int>((cc & 1u) << 9) | static_cast<int>((cc % kVBufs) << 10);
+                    sm.tile_meta[ms][2] = ntok | (last ? 256 : 0) | static_cast<int>((cc & 1u) << 9) | static_cast<int>((cc % kVBufs) << 10) | (karr << 12);
                     sm.tile_meta[ms][3] = rec.z - (a.whole ? 0 : t_begin * kTok);
                 }
                 {
@@ -293,7 +297,7 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                 if ((warp & 3) == 0 && lane == 0) {
                     const int flags = sm.tile_meta[ms][2];
                     mbar_arrive(&sm.q_empty[tcv % kQSlots]);
-                    if (flags & 256) mbar_arrive(&sm.k_empty[(flags >> 9) & 1]);
+                    for (int x = (flags >> 12) & 3; x > 0; --x) mbar_arrive(&sm.k_empty[(flags >> 9) & 1]);
                 }
                 const int orow0 = sm.tile_meta[ms][3] * kG;          // first row of the tile in the output buffers
                 const int e = sm.ent_s[ti * kTok + min(tk, (sm.tile_meta[ms][2] & 255) - 1)];
@@ -515,61 +519,61 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                 }
                 if (dead && lane == 0) { set_status(a.status, kDevTimeout); atomicExch(&sm.abort_flag, 1); }
             });
-        } else if (warp == kMmaWarp) {
-            // ================================================================ MMA issuer
+        } else {
+            // ================================================================ MMA issuers (one thread per tile parity)
+            // The issuing thread is the critical path of a tile (it is blocked while the tensor pipe takes its MMAs and
+            // every barrier test is a shared-memory round trip), so the tiles are split between two of them: warp 17
+            // serves the tiles in S/P/O slot 0, warp 18 those in slot 1.  Each commits its own s_full / o_full; a
+            // thread's MMAs complete in order, which is what the K-buffer hand-back above relies on.
+            const uint32_t par = static_cast<uint32_t>(warp - kMmaWarp);
             walk([&](int nb, uint32_t tcount, uint32_t ccount, int, int) {
                 if (lane != 0) return;
                 constexpr uint32_t idesc_s = umma_idesc_bf16(kRows, kNS);
                 constexpr uint32_t idesc_o = umma_idesc_bf16(kRows, kD) | kUmmaBMnMajor;
-                uint32_t cc = ccount;
-                int cur_pair = -1, cur_c = -1;
-                // the P V queue follows the chunk runs on its own (its V buffer is the run's ordinal modulo kVBufs), so
-                // the score queue may run ahead of it as far as the S slots and the gathered Q tiles allow
-                uint32_t cco = ccount;
-                int cur_pair_o = -1, cur_c_o = -1;
+                const uint32_t sl = par;
                 bool ok = true;
-                // Two in-order queues (S MMAs, O MMAs) served by polling: an O MMA whose probabilities are
-                // ready is never held up by a Q tile that has not arrived yet, and vice versa.
-                int ns = 0, no = 0;                    // next tile (batch index) to issue S / O for
+                // Two in-order queues (S MMAs, O MMAs) over this thread's tiles, served by polling: an O MMA whose
+                // probabilities are ready is never held up by a Q tile that has not arrived yet, and vice versa.  The
+                // chunk run of a tile (its K / V buffers) is looked up in the batch's run table.
+                int ns = static_cast<int>((par ^ tcount) & 1u), no = ns;       // next tile (batch index) for S / O
+                int ck_s = 0, ck_o = 0, run_s = -1, run_o = -1;                 // run of that tile; last run waited for
                 uint32_t idle = 0;
                 while (no < nb && ok) {
                     bool progressed = false;
                     if (ns < nb) {
-                        const uint32_t tcv = tcount + ns, sl = tcv & 1u, qs = tcv % kQSlots;
-                        const int4 rec = sm.recs[ns];
-                        const bool newc = rec.x != cur_pair || rec.y != cur_c;
+                        const uint32_t tcv = tcount + ns, qs = tcv % kQSlots;
+                        while (ns >= sm.cfirst[ck_s + 1]) ++ck_s;
+                        const uint32_t cc = ccount + static_cast<uint32_t>(ck_s);
                         bool ready = mbar_test_wait(&sm.q_full[qs], (tcv / kQSlots) & 1);
-                        if (ready && newc)
-                            ready = mbar_test_wait(&sm.k_ready[cc & 1u], (cc >> 1) & 1) &&
-                                    mbar_test_wait(&sm.v_ready[cc % kVBufs], (cc / kVBufs) & 1);
+                        if (ready && run_s != ck_s) ready = mbar_test_wait(&sm.k_ready[cc & 1u], (cc >> 1) & 1);
                         if (ready && tcv >= 2) ready = mbar_test_wait(&sm.s_empty[sl], ((tcv >> 1) - 1) & 1);
                         if (ready) {
-                            if (newc) { cur_pair = rec.x; cur_c = rec.y; ++cc; }
-                            const uint32_t cb = (cc - 1) & 1u;
+                            run_s = ck_s;
                             // the gathered rows were written by cp.async (generic proxy), the MMA reads them through
                             // the async proxy
                             fence_proxy_async_smem();
                             tc_fence_after_sync();
-                            const uint32_t qa = smem_u32(qbuf + qs * kQBytes), ka = smem_u32(kbuf + cb * kKBytes);
+                            const uint32_t qa = smem_u32(qbuf + qs * kQBytes), ka = smem_u32(kbuf + (cc & 1u) * kKBytes);
 #pragma unroll
                             for (int ks = 0; ks < 8; ++ks)
                                 umma_bf16(tmem_base + sl * 128, umma_desc_k128(qa + (ks >> 2) * 16384 + (ks & 3) * 32),
                                           umma_desc_k128(ka + (ks >> 2) * (kNS * 128) + (ks & 3) * 32), idesc_s, ks > 0 ? 1u : 0u);
                             umma_commit(&sm.s_full[sl]);
-                            ++ns;
+                            ns += 2;
                             progressed = true;
                         }
                     }
                     if (no < ns) {
-                        const uint32_t tcv = tcount + no, sl = tcv & 1u;
+                        const uint32_t tcv = tcount + no;
+                        while (no >= sm.cfirst[ck_o + 1]) ++ck_o;
+                        const uint32_t cco = ccount + static_cast<uint32_t>(ck_o);
                         bool ready = mbar_test_wait(&sm.p_full[sl], (tcv >> 1) & 1);
+                        if (ready && run_o != ck_o) ready = mbar_test_wait(&sm.v_ready[cco % kVBufs], (cco / kVBufs) & 1);
                         if (ready && tcv >= 2) ready = mbar_test_wait(&sm.o_empty[sl], ((tcv >> 1) - 1) & 1);
                         if (ready) {
-                            const int4 reco = sm.recs[no];
-                            if (reco.x != cur_pair_o || reco.y != cur_c_o) { cur_pair_o = reco.x; cur_c_o = reco.y; ++cco; }
-                            const uint32_t vb = (cco - 1) % kVBufs;
+                            run_o = ck_o;
                             tc_fence_after_sync();
-                            const uint32_t va = smem_u32(vbuf + vb * kVBytes);
+                            const uint32_t va = smem_u32(vbuf + (cco % kVBufs) * kVBytes);
                             // P from tensor memory (columns kPCol.. of the slot: 8 columns = 16 keys per step), V from
                             // shared memory, 16 keys per step = two 8-row groups
 #pragma unroll
@@ -577,7 +581,7 @@ prefill_attend_tc_kernel(const __grid_constant__ CUtensorMap map_k, const __grid
                                 umma_bf16_ts(tmem_base + 256 + sl * 128, tmem_base + sl * 128 + kPCol + ks * 8,
                                              umma_desc_mn128(va + ks * 2048, 8192u, 1024u), idesc_o, ks > 0 ? 1u : 0u);
                             umma_commit(&sm.o_full[sl]);
-                            ++no;
+                            no += 2;
                             progressed = true;
                         }
                     }
