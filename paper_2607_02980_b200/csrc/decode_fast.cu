@@ -14,6 +14,9 @@
 //                  finishes a pair last mixes the partial sums with the local branch (App. C).
 #include "internal.h"
 #include "tma.cuh"
+// Timeline instrumentation, compiled only with -DX_STAMP (never in the library that is shipped): the kernels record
+// globaltimer stamps of their phases (even slots: earliest, odd slots: latest over the CTAs), hils_debug_stamps reads
+// them back.  The timelines quoted in the kernels' comments come from such builds.
 #ifdef X_STAMP
 namespace hils { __device__ unsigned long long g_dbg[16]; }
 __device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
